@@ -1,0 +1,218 @@
+/*
+ * libdeeprebirth — execution of DeepRebirth "slim layers" on NVIDIA B200 (sm_100a).
+ *
+ * A slim layer is a convolution that has absorbed the non-tensor layers around it
+ * (DeepRebirth, Section 3): BatchNorm and Scale are folded into its weights and bias by the
+ * closed form of Lemma 2 (Section 3.1, "streamline slimming"); ReLU, max-pooling and
+ * cross-channel LRN run in its epilogue instead of as layers of their own; and the parallel
+ * branches of an inception module run as one wide convolution that writes its slice of the
+ * concatenated output in place (Section 3.2, "branch slimming").  Unlike the paper, which
+ * approximates the absorbed pooling/LRN layers and re-trains, the epilogue here computes them
+ * exactly, so a slim layer returns what the original layer sequence returns.
+ *
+ * Conventions
+ *  - Plain C ABI.  Every call returns an int status: DR_OK (0) or a negative DR_ERR_* code;
+ *    dr_strerror() names it.  Arguments are validated before anything is launched; on an error
+ *    nothing has been launched unless the code is DR_ERR_CUDA or DR_ERR_DEVICE_TIMEOUT.
+ *  - All tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned, and must
+ *    stay valid until the work queued on `stream` has finished.  The library allocates no
+ *    device memory: scratch space is sized by a *_workspace_bytes call and passed in.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *    enqueue work; they do not synchronise unless stated.
+ *  - Activations are NHWC bfloat16: element (n,h,w,c) of a tensor with channel stride ldc and
+ *    channel offset coff lives at ((n*H + h)*W + w)*ldc + coff + c.  Dense tensors have
+ *    ldc = C, coff = 0.  Filters are [Cout][k][k][Cin] bfloat16; bias and BatchNorm/Scale
+ *    vectors are float32 [Cout].  Accumulation and all epilogue arithmetic are float32;
+ *    results are rounded to bfloat16 (nearest even) once, when stored.
+ *  - Device-side waits are bounded.  If one runs out, the kernel records
+ *    DR_ERR_DEVICE_TIMEOUT, releases what it holds and returns; dr_device_status() reads the
+ *    record after a synchronisation.
+ */
+#ifndef DR_H_
+#define DR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ------------------------------------------------------------------ */
+#define DR_OK                   0
+#define DR_ERR_INVALID_ARG     (-1)  /* null pointer, non-positive size, inconsistent descriptor */
+#define DR_ERR_UNSUPPORTED     (-2)  /* a valid request this build has no kernel for            */
+#define DR_ERR_ALIGNMENT       (-3)  /* pointer / ldc / coff not aligned as documented          */
+#define DR_ERR_WORKSPACE       (-4)  /* workspace missing, too small, or net not prepared       */
+#define DR_ERR_CUDA            (-5)  /* a CUDA runtime/driver call failed                       */
+#define DR_ERR_DEVICE_TIMEOUT  (-6)  /* a bounded device-side wait ran out                      */
+
+const char* dr_strerror(int status);
+
+/* ---- slim-layer descriptor --------------------------------------------------------- */
+/* Epilogue flags.  The epilogue applies, in this order: +bias, ReLU, then pooling and LRN in
+ * the order DR_LRN_BEFORE_POOL selects, then +residual, then the second ReLU.              */
+#define DR_BIAS                 0x01u
+#define DR_RELU                 0x02u
+#define DR_POOL                 0x04u  /* max-pool pool_k x pool_k / pool_stride, pad pool_pad   */
+#define DR_LRN                  0x08u  /* LRN across channels                                    */
+#define DR_RESIDUAL             0x10u  /* add a dense [B,Ho,Wo,Cout] bfloat16 tensor            */
+#define DR_LRN_BEFORE_POOL      0x20u  /* LRN then pool (GoogLeNet conv2); default pool then LRN */
+#define DR_RELU_AFTER_RESIDUAL  0x40u
+#define DR_OUT_F32              0x80u  /* store float32 instead of bfloat16 (final logits)       */
+
+typedef struct dr_conv_desc {
+    int k, stride, pad;        /* square kernel; output extent floor((H + 2*pad - k)/stride) + 1 */
+    int Cin, Cout;
+    unsigned flags;            /* DR_* epilogue flags                                            */
+    int pool_k, pool_stride, pool_pad;              /* used with DR_POOL; only 3,2,1 is built    */
+    int lrn_size;                                   /* used with DR_LRN; odd, <= 15              */
+    float lrn_alpha, lrn_beta, lrn_k;
+    int y_ldc, y_coff;         /* channel stride / offset of y; 0,0 means dense (ldc = Cout)     */
+} dr_conv_desc;
+
+/* ---- parameter generation (offline slimming) ---------------------------------------- */
+
+/* Lemma 2 / Eq. (W_B_S), Section 3.1: closed form of convolution -> BatchNorm -> Scale.
+ *   eta_j = gamma_j / sqrt(var_j/m + eps);  w_out[j,:] = eta_j * w_in[j,:];
+ *   b_out[j] = eta_j * b_in[j] + beta_j - eta_j * mean_j / m.
+ * mean/var are the stored BatchNorm blobs and m their scale factor (true statistics are
+ * mean/m and var/m); eps = 0 reproduces the paper's formula.  K = k*k*Cin values per filter.
+ * w_in, w_out: bfloat16 [Cout][K] (may alias).  b_in: float32 [Cout] or NULL (zero bias).
+ * Computed in float32, w_out rounded to bfloat16 once.  Errors: INVALID_ARG on nulls/sizes. */
+int dr_fold_bn(int Cout, int K, const void* w_in, const float* b_in, const float* mean,
+               const float* var, float m, float eps, const float* gamma, const float* beta,
+               void* w_out, float* b_out, void* stream);
+
+/* The exact form of "adjust to the same size" in Section 3.2: write a [Cout][ks][ks][Cin]
+ * filter bank, zero-embedded at the centre of kb x kb taps, into filters [joff, joff+Cout) of
+ * w_big ([*][kb][kb][Cin], bfloat16); with pad kb/2 the stride-1 convolution is unchanged.
+ * Concatenating filter banks along Cout is Eq. (W_b).  kb >= ks, both odd.                  */
+int dr_embed_filter(int Cout, int Cin, int ks, int kb, const void* w_small, int joff,
+                    void* w_big, void* stream);
+
+/* ---- slim layers -------------------------------------------------------------------- */
+
+/* One slim convolution layer (Eq. (tY_j = tW), Section 3.1, with the epilogue of the
+ * descriptor): y = epilogue(conv(x; w) ).
+ *  x: [B,H,W,Cin] dense bfloat16.   w: [Cout][k][k][Cin] bfloat16.   b: float32 [Cout] (DR_BIAS).
+ *  residual: dense [B,Ho,Wo,Cout] bfloat16 (DR_RESIDUAL) else NULL.
+ *  y: [B,Hy,Wy,*] with channel stride y_ldc, offset y_coff; (Hy,Wy) is the conv output extent,
+ *     or the pooled extent with DR_POOL.  bfloat16, or float32 with DR_OUT_F32.
+ *  argmax: NULL, or int32 [B,Hy,Wy,Cout] (DR_POOL only): flat position h*Wo+w in the conv
+ *     output plane of the first maximum in row-major window order.
+ * Restrictions: DR_POOL/DR_LRN need Cout <= 256 and exclude DR_RESIDUAL and DR_OUT_F32;
+ * y_ldc, y_coff multiples of 8.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.          */
+int dr_conv_slim(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* w,
+                 const float* b, const void* residual, void* y, int32_t* argmax, void* stream);
+
+/* Branch-slimmed inception module (Section 3.2; the merged-branch identity Eqs. (LR), (W_b)):
+ *   y[..., 0:c3)      = ReLU(conv3x3(ReLU(conv1x1(x; w[0]) + b[0]); w[1]) + b[1])
+ *   y[..., c3:c3+cm)  = ReLU(conv5x5(x; w[2]) + b[2])          (pad 2, the merged branches)
+ * written in place into y [B,H,W,c3+cm].  workspace holds the 1x1 output:
+ * dr_inception_workspace_bytes() bytes.  pool_after != 0 is not built (UNSUPPORTED): run
+ * dr_maxpool on y.                                                                          */
+typedef struct dr_inception_desc {
+    int Cin, c3r, c3, cm;
+    int pool_after;
+} dr_inception_desc;
+int dr_inception_workspace_bytes(const dr_inception_desc* desc, int B, int H, int W, size_t* bytes);
+int dr_inception_slim(const dr_inception_desc* desc, int B, int H, int W, const void* x,
+                      const void* const w[3], const float* const b[3], void* y, void* workspace,
+                      void* stream);
+
+/* ---- stand-alone non-tensor layers (the "unslimmed" baseline, Section 2 / Table 2) -------
+ * Each reads its input from and writes its output to device memory: one round trip per
+ * layer, which is the cost the slim layers remove.  All tensors dense NHWC bfloat16.       */
+int dr_relu(size_t n, const void* x, void* y, void* stream);
+/* floor-mode output extent; padding never wins; argmax as in dr_conv_slim, or NULL */
+int dr_maxpool(int B, int H, int W, int C, int k, int s, int p, const void* x, void* y,
+               int32_t* argmax, void* stream);
+/* y_c = x_c * (k + alpha/size * sum_{|c'-c| <= size/2, 0 <= c' < C} x_c'^2)^(-beta) */
+int dr_lrn(int B, int H, int W, int C, int size, float alpha, float beta, float k, const void* x,
+           void* y, void* stream);
+/* BatchNorm layer, y = (x - mean/m)/sqrt(var/m + eps); followed by the Scale layer
+ * y = gamma*y + beta when gamma is not NULL (Eq. (Y_batch_scala_conv), Section 3.1)        */
+int dr_bn(int B, int H, int W, int C, const void* x, const float* mean, const float* var, float m,
+          float eps, const float* gamma, const float* beta, void* y, void* stream);
+/* Scale layer alone: y = gamma_c * x + beta_c */
+int dr_scale(int B, int H, int W, int C, const void* x, const float* gamma, const float* beta, void* y,
+             void* stream);
+int dr_add(size_t n, const void* a, const void* b, void* y, void* stream);
+/* copy dense [npix][C] into channels [coff, coff+C) of a tensor with channel stride ldc */
+int dr_concat(size_t npix, int C, const void* x, int ldc, int coff, void* y, void* stream);
+/* mean over the H x W plane: [B,H,W,C] -> [B,1,1,C] */
+int dr_avgpool_global(int B, int H, int W, int C, const void* x, void* y, void* stream);
+
+/* ---- whole networks ----------------------------------------------------------------- */
+#define DR_ARCH_GOOGLENET  0   /* Inception-v1 topology, branch-slimmed modules (Section 4.1)    */
+#define DR_ARCH_RESNET50   1   /* bottleneck v1; every conv followed by BatchNorm+Scale (4.3)    */
+#define DR_MODE_SLIM       0   /* slim layers: folded BN, fused epilogues, merged branches       */
+#define DR_MODE_UNSLIMMED  1   /* every layer of the original sequence as its own launch         */
+
+typedef struct dr_net dr_net;
+
+typedef struct dr_param_spec {
+    char name[48];     /* e.g. "3a.b5.w", "res2a.2a.bn.gamma"                                    */
+    int dims[4];       /* filters: Cout,k,k,Cin; vectors: C,1,1,1                                */
+    int is_f32;        /* 0: bfloat16, 1: float32                                                */
+    size_t count;      /* number of elements                                                     */
+} dr_param_spec;
+
+typedef struct dr_layer_info {
+    char name[48];
+    int kind;          /* 0 tensor layer (conv / FC), 1 non-tensor layer (Section 2's definition)*/
+    int dims[4];       /* B,H,W,C of the slice this layer writes                                 */
+    int ldc, coff;     /* channel stride / offset of that slice                                  */
+    int is_f32;
+    const void* ptr;   /* device address of element (0,0,0,0) of the slice; valid after prepare  */
+    double flops;      /* 2*M*N*K for tensor layers, 0 otherwise                                 */
+    double bytes;      /* algorithmic bytes read + written                                       */
+    int conv_path;     /* which convolution kernel runs it (DR_PATH_*), -1 for non-tensor        */
+} dr_layer_info;
+
+/* Both modes take the SAME parameter list: the original, un-slimmed parameters (separate
+ * branch filters, BatchNorm/Scale vectors).  In slim mode dr_net_prepare() derives the slim
+ * parameters from them (dr_fold_bn, dr_embed_filter + concatenation) into the workspace.
+ * dr_net_create is host-only.  B,H,W: batch and input plane (3 channels).                  */
+int dr_net_create(dr_net** net, int arch, int mode, int B, int H, int W);
+int dr_net_destroy(dr_net* net);
+int dr_net_num_params(const dr_net* net);
+int dr_net_param_spec(const dr_net* net, int idx, dr_param_spec* spec);
+int dr_net_set_param(dr_net* net, int idx, const void* dev);   /* borrowed, not copied */
+int dr_net_workspace_bytes(const dr_net* net, size_t* bytes);
+/* Once per (net, workspace), after every parameter is set: derives slim parameters, lays the
+ * activation buffers out in the workspace.  Enqueues on stream.  The workspace must be
+ * 256-byte aligned and must not be used for anything else while the net is in use.        */
+int dr_net_prepare(dr_net* net, void* workspace, void* stream);
+/* x: [B,H,W,3] bfloat16; logits: float32 [B][1000].  One launch per layer on `stream`. */
+int dr_net_forward(dr_net* net, const void* x, void* workspace, float* logits, void* stream);
+int dr_net_num_layers(const dr_net* net);
+int dr_net_layer_info(const dr_net* net, int layer, dr_layer_info* info);
+/* Per-layer CUDA-event timing (the layer-wise protocol of Section 4.1): when enabled, each
+ * forward records events around every launch; dr_net_layer_time_us synchronises on them.  */
+int dr_net_set_timing(dr_net* net, int enabled);
+int dr_net_layer_time_us(dr_net* net, int layer, float* us);
+/* Bytes of the workspace that hold activations (run-time memory, Table 6's quantity). */
+int dr_net_activation_bytes(const dr_net* net, size_t* bytes);
+
+/* ---- diagnostics -------------------------------------------------------------------- */
+#define DR_PATH_AUTO         0
+#define DR_PATH_SIMT         1  /* CUDA-core implicit GEMM: any shape, slow                      */
+#define DR_PATH_UMMA_GATHER  2  /* tcgen05 MMA, operands gathered by producer warps              */
+#define DR_PATH_UMMA_TMA     3  /* tcgen05 MMA, operands loaded by TMA (im2col / tiled)          */
+/* Force a convolution kernel (tests, A/B timing); DR_PATH_AUTO picks the fastest that
+ * supports the layer.  A forced path that cannot run the layer gives DR_ERR_UNSUPPORTED.   */
+int dr_set_conv_path(int path);
+int dr_last_conv_path(void);            /* path taken by the latest dr_conv_slim call */
+/* Synchronises the device, then reads and clears the record the kernels leave when a bounded
+ * wait runs out: returns DR_OK or DR_ERR_DEVICE_TIMEOUT; info[0..3] (may be NULL) receive the
+ * code, a kernel-specific site id, the block index and the tile index.                    */
+int dr_device_status(int info[4]);
+/* Kernels of this library launched by this process so far. */
+long long dr_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DR_H_ */

@@ -1,0 +1,161 @@
+// dr_conv_slim / dr_inception_slim: validation, tiling choice and kernel dispatch.
+#include "conv_common.cuh"
+
+namespace dr {
+
+static int g_forced_path = DR_PATH_AUTO;
+static int g_last_path = -1;
+
+// Fill the derived fields of ConvParams from a descriptor.  Returns a status.
+int conv_make_params(const dr_conv_desc* d, int B, int H, int W, const void* x, const void* w, const float* b,
+                     const void* residual, void* y, int32_t* argmax, ConvParams* out) {
+    if (!d || !x || !w || !y) return DR_ERR_INVALID_ARG;
+    if (d->k <= 0 || d->stride <= 0 || d->pad < 0 || d->Cin <= 0 || d->Cout <= 0) return DR_ERR_INVALID_ARG;
+    if (B < 0 || H <= 0 || W <= 0) return DR_ERR_INVALID_ARG;
+    if (H + 2 * d->pad < d->k || W + 2 * d->pad < d->k) return DR_ERR_INVALID_ARG;
+    const unsigned f = d->flags;
+    if ((f & DR_BIAS) && !b) return DR_ERR_INVALID_ARG;
+    if ((f & DR_RESIDUAL) && !residual) return DR_ERR_INVALID_ARG;
+    if ((f & DR_RELU_AFTER_RESIDUAL) && !(f & DR_RESIDUAL)) return DR_ERR_INVALID_ARG;
+    if ((f & DR_LRN_BEFORE_POOL) && !((f & DR_LRN) && (f & DR_POOL))) return DR_ERR_INVALID_ARG;
+    if (argmax && !(f & DR_POOL)) return DR_ERR_INVALID_ARG;
+    const bool staged = f & (DR_POOL | DR_LRN);
+    if (staged && (f & (DR_RESIDUAL | DR_OUT_F32))) return DR_ERR_UNSUPPORTED;
+    if (staged && (d->Cout > 256 || (d->Cout & 1))) return DR_ERR_UNSUPPORTED;
+    if (f & DR_POOL) {
+        if (d->pool_k != 3 || d->pool_stride != 2 || d->pool_pad != 1) return DR_ERR_UNSUPPORTED;
+    }
+    if (f & DR_LRN) {
+        if (d->lrn_size < 1 || !(d->lrn_size & 1) || d->lrn_size > 15) return DR_ERR_INVALID_ARG;
+    }
+    const int ldc = d->y_ldc ? d->y_ldc : d->Cout;
+    const int coff = d->y_coff;
+    if (ldc < d->Cout || coff < 0 || coff + d->Cout > ldc) return DR_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || (residual && !aligned16(residual))) return DR_ERR_ALIGNMENT;
+    if (d->y_ldc && ((ldc & 7) || (coff & 7))) return DR_ERR_ALIGNMENT;
+
+    ConvParams p{};
+    p.x = (const __nv_bfloat16*)x; p.w = (const __nv_bfloat16*)w; p.bias = b;
+    p.residual = (const __nv_bfloat16*)residual; p.y = y; p.argmax = argmax;
+    p.status = dev_status_ptr();
+    p.B = B; p.H = H; p.W = W; p.Cin = d->Cin; p.Cout = d->Cout; p.k = d->k; p.stride = d->stride; p.pad = d->pad;
+    p.Ho = (H + 2 * d->pad - d->k) / d->stride + 1;
+    p.Wo = (W + 2 * d->pad - d->k) / d->stride + 1;
+    p.Hy = p.Ho; p.Wy = p.Wo;
+    if (f & DR_POOL) {
+        if (p.Ho + 2 < 3 || p.Wo + 2 < 3) return DR_ERR_INVALID_ARG;
+        p.Hy = (p.Ho + 2 - 3) / 2 + 1; p.Wy = (p.Wo + 2 - 3) / 2 + 1;
+    }
+    p.K = d->k * d->k * d->Cin;
+    p.flags = f;
+    p.lrn_half = (f & DR_LRN) ? d->lrn_size / 2 : 0;
+    p.lrn_alpha_n = (f & DR_LRN) ? d->lrn_alpha / d->lrn_size : 0.f;
+    p.lrn_beta = d->lrn_beta; p.lrn_k = d->lrn_k;
+    p.ldc = ldc; p.coff = coff;
+    p.M = (long long)B * p.Ho * p.Wo;
+    const int cout16 = (d->Cout + 15) / 16 * 16;
+    if (staged) {
+        p.Nt = cout16; p.n_blocks = 1;
+    } else {
+        p.n_blocks = (cout16 + 255) / 256;
+        p.Nt = ((cout16 + p.n_blocks - 1) / p.n_blocks + 15) / 16 * 16;
+    }
+    if (f & DR_POOL) {
+        static const int cand[][2] = {{3, 8}, {4, 6}, {5, 5}, {2, 12}, {8, 3}, {6, 4}};
+        long best = -1;
+        for (auto& c : cand) {
+            const long t = (long)((p.Hy + c[0] - 1) / c[0]) * ((p.Wy + c[1] - 1) / c[1]);
+            if (best < 0 || t < best) { best = t; p.PH = c[0]; p.PW = c[1]; }
+        }
+        p.patch = 1;
+        p.tiles_h = (p.Hy + p.PH - 1) / p.PH; p.tiles_w = (p.Wy + p.PW - 1) / p.PW;
+        const long long mt = (long long)B * p.tiles_h * p.tiles_w;
+        if (mt > 0x7fffffffLL) return DR_ERR_UNSUPPORTED;
+        p.m_tiles = (int)mt;
+    } else {
+        const long long mt = (p.M + TILE_M - 1) / TILE_M;
+        if (mt > 0x7fffffffLL) return DR_ERR_UNSUPPORTED;
+        p.m_tiles = (int)mt;
+    }
+    *out = p;
+    return DR_OK;
+}
+
+int conv_pick_path(const ConvParams& p, int forced) {
+    if (forced == DR_PATH_SIMT) return DR_PATH_SIMT;
+    if (forced == DR_PATH_UMMA_GATHER) return conv_umma_gather_supports(p) ? DR_PATH_UMMA_GATHER : -1;
+    if (forced == DR_PATH_UMMA_TMA) return conv_umma_tma_supports(p) ? DR_PATH_UMMA_TMA : -1;
+    if (conv_umma_tma_supports(p)) return DR_PATH_UMMA_TMA;
+    if (conv_umma_gather_supports(p)) return DR_PATH_UMMA_GATHER;
+    return DR_PATH_SIMT;
+}
+
+int conv_launch_path(const ConvParams& p, int path, cudaStream_t stream) {
+    switch (path) {
+        case DR_PATH_SIMT: return conv_simt_launch(p, stream);
+        case DR_PATH_UMMA_GATHER: return conv_umma_gather_launch(p, stream);
+        case DR_PATH_UMMA_TMA: return conv_umma_tma_launch(p, stream);
+        default: return DR_ERR_UNSUPPORTED;
+    }
+}
+
+int forced_conv_path() { return g_forced_path; }
+
+}  // namespace dr
+
+using namespace dr;
+
+extern "C" {
+
+int dr_set_conv_path(int path) {
+    if (path < DR_PATH_AUTO || path > DR_PATH_UMMA_TMA) return DR_ERR_INVALID_ARG;
+    g_forced_path = path;
+    return DR_OK;
+}
+
+int dr_last_conv_path(void) { return g_last_path; }
+
+int dr_conv_slim(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* w, const float* b,
+                 const void* residual, void* y, int32_t* argmax, void* stream) {
+    ConvParams p;
+    const int st = conv_make_params(desc, B, H, W, x, w, b, residual, y, argmax, &p);
+    if (st != DR_OK) return st;
+    if (p.M == 0) return DR_OK;
+    const int path = conv_pick_path(p, g_forced_path);
+    if (path < 0) return DR_ERR_UNSUPPORTED;
+    g_last_path = path;
+    return conv_launch_path(p, path, (cudaStream_t)stream);
+}
+
+int dr_inception_workspace_bytes(const dr_inception_desc* d, int B, int H, int W, size_t* bytes) {
+    if (!d || !bytes || B < 0 || H <= 0 || W <= 0 || d->c3r <= 0) return DR_ERR_INVALID_ARG;
+    *bytes = ((size_t)B * H * W * d->c3r * 2 + 255) / 256 * 256;
+    return DR_OK;
+}
+
+int dr_inception_slim(const dr_inception_desc* d, int B, int H, int W, const void* x, const void* const w[3],
+                      const float* const b[3], void* y, void* workspace, void* stream) {
+    if (!d || !x || !w || !b || !y) return DR_ERR_INVALID_ARG;
+    if (d->Cin <= 0 || d->c3r <= 0 || d->c3 <= 0 || d->cm <= 0) return DR_ERR_INVALID_ARG;
+    if (d->pool_after) return DR_ERR_UNSUPPORTED;
+    if (!workspace) return DR_ERR_WORKSPACE;
+    for (int i = 0; i < 3; ++i)
+        if (!w[i] || !b[i]) return DR_ERR_INVALID_ARG;
+    if ((d->c3 & 7) || (d->cm & 7)) return DR_ERR_ALIGNMENT;
+    const int ldc = d->c3 + d->cm;
+    dr_conv_desc c{};
+    c.flags = DR_BIAS | DR_RELU;
+    // 1x1 reducer of the 3x3 path -> workspace
+    c.k = 1; c.stride = 1; c.pad = 0; c.Cin = d->Cin; c.Cout = d->c3r; c.y_ldc = 0; c.y_coff = 0;
+    int st = dr_conv_slim(&c, B, H, W, x, w[0], b[0], nullptr, workspace, nullptr, stream);
+    if (st != DR_OK) return st;
+    // 3x3 -> channels [0, c3)
+    c.k = 3; c.pad = 1; c.Cin = d->c3r; c.Cout = d->c3; c.y_ldc = ldc; c.y_coff = 0;
+    st = dr_conv_slim(&c, B, H, W, workspace, w[1], b[1], nullptr, y, nullptr, stream);
+    if (st != DR_OK) return st;
+    // merged 5x5 on the module input -> channels [c3, c3+cm)
+    c.k = 5; c.pad = 2; c.Cin = d->Cin; c.Cout = d->cm; c.y_ldc = ldc; c.y_coff = d->c3;
+    return dr_conv_slim(&c, B, H, W, x, w[2], b[2], nullptr, y, nullptr, stream);
+}
+
+}  // extern "C"

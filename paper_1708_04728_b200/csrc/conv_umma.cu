@@ -1,0 +1,505 @@
+// Implicit-GEMM convolution on the 5th-generation tensor cores (tcgen05.mma, accumulators in
+// tensor memory), NHWC bf16 in, float32 accumulate.  Two kernels share the MMA issue loop, the
+// shared-memory operand layout and the epilogues of conv_common.cuh:
+//
+//   conv_umma_tma_kernel     the hot path.  Persistent, one CTA per SM.  Warp 0 streams operand
+//       tiles with TMA: the activation tile in im2col mode (128 consecutive output pixels x 64
+//       channels of one filter tap; the hardware walks rows/images and zero-fills the padding),
+//       the filter tile in tiled mode.  Warp 1 issues the MMAs.  Warps 2-5 drain the finished
+//       accumulator (bias, ReLU, residual, bf16 store) while the next tile is already being
+//       multiplied into the second TMEM buffer.
+//   conv_umma_gather_kernel  same MMA pipeline, but four producer warps build the operand tiles
+//       in shared memory with ordinary loads.  Takes what TMA cannot describe (3-channel stem)
+//       and the layers whose epilogue pools: there a tile is a 2-D patch of outputs.
+//
+// Operand tiles in shared memory: [rows][64 bf16] = 128-byte rows, 128-byte swizzle (16-byte chunk
+// index XOR row%8), 8-row groups 1024 bytes apart — the K-major layout both TMA and the MMA
+// descriptor understand.  One k-block = one filter tap x 64 input channels (zero-filled past Cin);
+// only ceil(valid/16) MMAs of K=16 are issued for a partial block.
+//
+// Every wait on an mbarrier is bounded (see ptx::mbar_wait); on a timeout the CTA records
+// DR_ERR_DEVICE_TIMEOUT, all roles leave their loops, and TMEM is released before exit.
+#include "conv_common.cuh"
+#include "umma_ptx.cuh"
+
+namespace dr {
+using namespace ptx;
+
+constexpr int A_TILE_BYTES = TILE_M * 128;   // 128 rows x 64 bf16
+constexpr int B_TILE_BYTES = 256 * 128;      // up to 256 filters x 64 bf16
+constexpr int STAGE_BYTES = A_TILE_BYTES + B_TILE_BYTES;
+
+__device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
+
+// Issue the MMAs of one k-block: A tile at a_smem, B tile at b_smem, nk16 steps of K=16.
+__device__ __forceinline__ void issue_kblock(uint32_t tmem_d, uint32_t a_smem, uint32_t b_smem, uint32_t idesc, int nk16, bool first) {
+    const uint64_t ad = make_sdesc_sw128(a_smem), bd = make_sdesc_sw128(b_smem);
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+        if (k < nk16) umma_bf16(tmem_d, ad + 2 * k, bd + 2 * k, idesc, (first && k == 0) ? 0u : 1u);
+}
+
+// Drain `ncols` accumulator columns of this thread's TMEM lane and run the direct epilogue.
+__device__ __forceinline__ void drain_direct(const ConvParams& p, uint32_t taddr, int ncols, long long m, bool row_ok, int n0) {
+    for (int c = 0; c < ncols; c += 32) {
+        uint32_t r[32];
+        if (ncols - c >= 32) {
+            tmem_ld_x32(taddr + c, r);
+            tmem_ld_wait();
+            if (row_ok) epilogue_direct<32>(p, m, n0 + c, reinterpret_cast<float*>(r));
+        } else {
+            tmem_ld_x16(taddr + c, r);
+            tmem_ld_wait();
+            if (row_ok) epilogue_direct<16>(p, m, n0 + c, reinterpret_cast<float*>(r));
+        }
+    }
+}
+
+// =====================================================================================
+//                                   gather kernel
+// =====================================================================================
+constexpr int G_STAGES = 3;
+constexpr int G_THREADS = 160;   // warps 0-3: producers, then epilogue; warp 4: MMA issue + TMEM owner
+constexpr int G_PIPE_BYTES = G_STAGES * STAGE_BYTES;
+constexpr int G_SMEM = G_PIPE_BYTES + 1024;
+
+struct GatherShared {
+    uint64_t full[G_STAGES], empty[G_STAGES], accum, drain;
+    uint32_t tmem_base;
+    int abort;
+};
+
+__global__ void __launch_bounds__(G_THREADS, 1) conv_umma_gather_kernel(const ConvParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __shared__ GatherShared sh;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tile = blockIdx.x, n0 = blockIdx.y * p.Nt;
+    const int cout16 = (p.Cout + 15) & ~15;
+    const int Nj = min(p.Nt, cout16 - n0);
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < Nj) tmem_cols <<= 1;
+
+    if (tid == 0) {
+        for (int s = 0; s < G_STAGES; ++s) { mbar_init(&sh.full[s], 128); mbar_init(&sh.empty[s], 1); }
+        mbar_init(&sh.accum, 1);
+        mbar_init(&sh.drain, 1);
+        sh.abort = 0;
+        fence_barrier_init();
+    }
+    if (warp == 4) { tmem_alloc(&sh.tmem_base, tmem_cols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+    volatile int* abort_flag = &sh.abort;
+
+    const bool scalar_k = (p.Cin & 7) != 0;          // K walked as one flat index (3-channel stem)
+    const int cpb = (p.Cin + 63) >> 6;               // 64-channel blocks per tap
+    const int nkb = scalar_k ? (p.K + 63) >> 6 : p.k * p.k * cpb;
+    const bool staged = p.flags & (DR_POOL | DR_LRN);
+
+    if (warp < 4) {
+        // ------------------------------------------------ producers: thread = tile row
+        const RowPix px = row_pixel(p, tile, tid);
+        const int h0 = px.ho * p.stride - p.pad, w0 = px.wo * p.stride - p.pad;
+        const __nv_bfloat16* ximg = p.x + (size_t)px.n * p.H * p.W * p.Cin;
+        for (int kb = 0; kb < nkb; ++kb) {
+            const int s = kb % G_STAGES, u = kb / G_STAGES;
+            if (!mbar_wait(&sh.empty[s], (u & 1) ^ 1, abort_flag)) {
+                if (!*abort_flag) report_timeout(p.status, 1, tile);
+                *abort_flag = 1;
+                break;
+            }
+            uint8_t* As = smem + s * STAGE_BYTES;
+            uint8_t* Bs = As + A_TILE_BYTES;
+            if (!scalar_k) {
+                const int tap = kb / cpb, c0 = (kb - tap * cpb) << 6;
+                const int r = tap / p.k, t = tap - r * p.k;
+                const int hi = h0 + r, wi = w0 + t;
+                const bool ok = px.valid && hi >= 0 && hi < p.H && wi >= 0 && wi < p.W;
+                const uint4* src = reinterpret_cast<const uint4*>(ximg + ((size_t)hi * p.W + wi) * p.Cin + c0);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (ok && c0 + 8 * j < p.Cin) v = __ldg(src + j);
+                    *reinterpret_cast<uint4*>(As + swz(tid, j)) = v;
+                }
+                for (int row = tid; row < Nj; row += 128) {
+                    const int jn = n0 + row;
+                    const uint4* wsrc = reinterpret_cast<const uint4*>(p.w + (size_t)jn * p.K + (size_t)tap * p.Cin + c0);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (jn < p.Cout && c0 + 8 * j < p.Cin) v = __ldg(wsrc + j);
+                        *reinterpret_cast<uint4*>(Bs + swz(row, j)) = v;
+                    }
+                }
+            } else {
+                const int k0 = kb << 6;
+                int r = k0 / (p.k * p.Cin);
+                int rem = k0 - r * p.k * p.Cin;
+                int t = rem / p.Cin;
+                int c = rem - t * p.Cin;
+                const unsigned short* xs = reinterpret_cast<const unsigned short*>(ximg);
+                for (int j = 0; j < 8; ++j) {
+                    unsigned short e[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const int kg = k0 + 8 * j + q;
+                        const int hi = h0 + r, wi = w0 + t;
+                        unsigned short v = 0;
+                        if (px.valid && kg < p.K && hi >= 0 && hi < p.H && wi >= 0 && wi < p.W)
+                            v = __ldg(xs + ((size_t)hi * p.W + wi) * p.Cin + c);
+                        e[q] = v;
+                        if (++c == p.Cin) { c = 0; if (++t == p.k) { t = 0; ++r; } }
+                    }
+                    uint4 v;
+                    v.x = e[0] | ((uint32_t)e[1] << 16); v.y = e[2] | ((uint32_t)e[3] << 16);
+                    v.z = e[4] | ((uint32_t)e[5] << 16); v.w = e[6] | ((uint32_t)e[7] << 16);
+                    *reinterpret_cast<uint4*>(As + swz(tid, j)) = v;
+                }
+                const unsigned short* wsh = reinterpret_cast<const unsigned short*>(p.w);
+                for (int row = tid; row < Nj; row += 128) {
+                    const int jn = n0 + row;
+                    for (int j = 0; j < 8; ++j) {
+                        unsigned short e[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const int kg = k0 + 8 * j + q;
+                            e[q] = (jn < p.Cout && kg < p.K) ? __ldg(wsh + (size_t)jn * p.K + kg) : (unsigned short)0;
+                        }
+                        uint4 v;
+                        v.x = e[0] | ((uint32_t)e[1] << 16); v.y = e[2] | ((uint32_t)e[3] << 16);
+                        v.z = e[4] | ((uint32_t)e[5] << 16); v.w = e[6] | ((uint32_t)e[7] << 16);
+                        *reinterpret_cast<uint4*>(Bs + swz(row, j)) = v;
+                    }
+                }
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&sh.full[s]);
+        }
+    } else {
+        // ------------------------------------------------ MMA issue: one thread
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_bf16(TILE_M, Nj);
+            bool ok = true;
+            for (int kb = 0; kb < nkb && ok; ++kb) {
+                const int s = kb % G_STAGES, u = kb / G_STAGES;
+                if (!mbar_wait(&sh.full[s], u & 1, abort_flag)) {
+                    if (!*abort_flag) report_timeout(p.status, 2, tile);
+                    *abort_flag = 1;
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                int valid;
+                if (scalar_k) valid = min(64, p.K - (kb << 6));
+                else valid = min(64, p.Cin - ((kb % cpb) << 6));
+                const uint32_t a = smem_u32(smem + s * STAGE_BYTES);
+                issue_kblock(tmem, a, a + A_TILE_BYTES, idesc, (valid + 15) >> 4, kb == 0);
+                umma_commit(&sh.empty[s]);
+            }
+            if (ok) umma_commit(&sh.accum);
+            else {   // let whatever was issued finish before TMEM is released
+                umma_commit(&sh.drain);
+                mbar_wait(&sh.drain, 0, nullptr);
+            }
+        }
+        __syncwarp();
+    }
+
+    // ---------------------------------------------------- epilogue: warps 0-3, thread = TMEM lane
+    if (warp < 4) {
+        bool ok = !*abort_flag && mbar_wait(&sh.accum, 0, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);            // warp-uniform: tcgen05.ld needs the whole warp
+        if (!ok) {
+            if (!*abort_flag) report_timeout(p.status, 3, tile);
+            *abort_flag = 1;
+        } else {
+            tc_fence_after();
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+            if (!staged) {
+                const long long m = (long long)tile * TILE_M + tid;
+                drain_direct(p, taddr, Nj, m, m < p.M, n0);
+            } else {
+                float* stage = reinterpret_cast<float*>(smem);            // the pipeline buffers are free now
+                float* stage2 = stage + (size_t)TILE_M * (p.Cout + 1);
+                const int ld = p.Cout + 1;
+                for (int c = 0; c < Nj; c += 16) {
+                    uint32_t r[16];
+                    tmem_ld_x16(taddr + c, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int ch = c + j;
+                        if (ch < p.Cout) {
+                            float v = __uint_as_float(r[j]) + ((p.flags & DR_BIAS) ? __ldg(p.bias + ch) : 0.f);
+                            if (p.flags & DR_RELU) v = fmaxf(v, 0.f);
+                            stage[tid * ld + ch] = v;
+                        }
+                    }
+                }
+                epilogue_staged<128, 1>(p, tile, stage, stage2, tid);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem, tmem_cols);
+}
+
+bool conv_umma_gather_supports(const ConvParams& p) {
+    if (p.Cout < 1 || p.Nt > 256) return false;
+    const bool staged = p.flags & (DR_POOL | DR_LRN);
+    if (staged) {
+        const bool ptl = (p.flags & DR_POOL) && (p.flags & DR_LRN) && !(p.flags & DR_LRN_BEFORE_POOL);
+        const size_t bytes = sizeof(float) * ((size_t)TILE_M * (p.Cout + 1) + (ptl ? (size_t)p.PH * p.PW * (p.Cout + 1) : 0));
+        if (bytes > (size_t)G_PIPE_BYTES) return false;
+    }
+    return true;
+}
+
+int conv_umma_gather_launch(const ConvParams& p, cudaStream_t stream) {
+    if (!conv_umma_gather_supports(p)) return DR_ERR_UNSUPPORTED;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(conv_umma_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM) != cudaSuccess) return DR_ERR_CUDA;
+        attr_set = true;
+    }
+    if (p.m_tiles <= 0) return DR_OK;
+    dim3 grid(p.m_tiles, p.n_blocks);
+    conv_umma_gather_kernel<<<grid, G_THREADS, G_SMEM, stream>>>(p);
+    count_launch();
+    return launch_status();
+}
+
+// =====================================================================================
+//                                     TMA kernel
+// =====================================================================================
+constexpr int T_STAGES = 4;
+constexpr int T_THREADS = 192;   // warp 0: TMA producer, warp 1: MMA issue + TMEM owner, warps 2-5: epilogue
+constexpr int T_SMEM = T_STAGES * STAGE_BYTES + 1024;
+constexpr int T_ACC_COLS = 256;  // columns per accumulator buffer; two buffers = all 512 TMEM columns
+
+struct TmaShared {
+    uint64_t full[T_STAGES], empty[T_STAGES], tfull[2], tempty[2];
+    uint32_t tmem_base;
+    int abort;
+};
+
+// a_mode 0: activations as a plain [M][Cin] matrix (1x1, stride 1, pad 0): 2-D tiled load.
+// a_mode 1: im2col load.
+__global__ void __launch_bounds__(T_THREADS, 1)
+conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const int a_mode) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __shared__ TmaShared sh;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < T_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 4); }
+        sh.abort = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+    }
+    if (warp == 1) { tmem_alloc(&sh.tmem_base, 2 * T_ACC_COLS); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+    volatile int* abort_flag = &sh.abort;
+
+    const int cpb = (p.Cin + 63) >> 6;
+    const int nkb = p.k * p.k * cpb;
+    const int total = p.m_tiles * p.n_blocks;
+    const int cout16 = (p.Cout + 15) & ~15;
+    const uint32_t stage_tx = A_TILE_BYTES + (uint32_t)p.Nt * 128;
+    const int hw = p.Ho * p.Wo;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // -------------------------------------------- TMA producer
+            int g = 0;
+            for (int t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
+                const int nb = t / p.m_tiles, mt = t - nb * p.m_tiles;
+                const int n0 = nb * p.Nt;
+                const long long m0 = (long long)mt * TILE_M;
+                const int img = (int)(m0 / hw);
+                const int rem = (int)(m0 - (long long)img * hw);
+                const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
+                const int hb = ho * p.stride - p.pad, wb = wo * p.stride - p.pad;
+                for (int kb = 0; kb < nkb; ++kb, ++g) {
+                    const int s = g % T_STAGES, u = g / T_STAGES;
+                    if (!mbar_wait(&sh.empty[s], (u & 1) ^ 1, abort_flag)) {
+                        if (!*abort_flag) report_timeout(p.status, 11, t);
+                        *abort_flag = 1;
+                        break;
+                    }
+                    uint8_t* As = smem + s * STAGE_BYTES;
+                    uint8_t* Bs = As + A_TILE_BYTES;
+                    const int tap = kb / cpb, c0 = (kb - tap * cpb) << 6;
+                    mbar_arrive_expect_tx(&sh.full[s], stage_tx);
+                    if (a_mode == 0) {
+                        tma_load_2d(As, &map_a, &sh.full[s], c0, (int)m0);
+                    } else {
+                        const int r = tap / p.k, tt = tap - r * p.k;
+                        tma_load_im2col_4d(As, &map_a, &sh.full[s], c0, wb, hb, img, (uint16_t)tt, (uint16_t)r);
+                    }
+                    tma_load_3d(Bs, &map_b, &sh.full[s], c0, tap, n0);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // -------------------------------------------- MMA issue
+            int g = 0, it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
+                const int nb = t / p.m_tiles;
+                const int Nj = min(p.Nt, cout16 - nb * p.Nt);
+                const uint32_t idesc = make_idesc_bf16(TILE_M, Nj);
+                const int acc = it & 1, au = it >> 1;
+                if (!mbar_wait(&sh.tempty[acc], (au & 1) ^ 1, abort_flag)) {
+                    if (!*abort_flag) report_timeout(p.status, 12, t);
+                    *abort_flag = 1;
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d = tmem + (uint32_t)(acc * T_ACC_COLS);
+                for (int kb = 0; kb < nkb; ++kb, ++g) {
+                    const int s = g % T_STAGES, u = g / T_STAGES;
+                    if (!mbar_wait(&sh.full[s], u & 1, abort_flag)) {
+                        if (!*abort_flag) report_timeout(p.status, 13, t);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const int valid = min(64, p.Cin - ((kb % cpb) << 6));
+                    const uint32_t a = smem_u32(smem + s * STAGE_BYTES);
+                    issue_kblock(d, a, a + A_TILE_BYTES, idesc, (valid + 15) >> 4, kb == 0);
+                    umma_commit(&sh.empty[s]);
+                }
+                if (ok) umma_commit(&sh.tfull[acc]);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------ epilogue warps: TMEM lane quarter = warp % 4
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        int it = 0;
+        for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
+            const int nb = t / p.m_tiles, mt = t - nb * p.m_tiles;
+            const int n0 = nb * p.Nt;
+            const int Nj = min(p.Nt, cout16 - n0);
+            const int acc = it & 1, au = it >> 1;
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[acc], au & 1, abort_flag));
+            if (!ok) {
+                if (!*abort_flag) report_timeout(p.status, 14, t);
+                *abort_flag = 1;
+                break;
+            }
+            tc_fence_after();
+            const long long m = (long long)mt * TILE_M + row;
+            drain_direct(p, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * T_ACC_COLS), Nj, m, m < p.M, n0);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.tempty[acc]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {   // give copies and MMAs still in flight time to land before shared memory and TMEM go away
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) {}
+        __syncthreads();
+    }
+    if (warp == 1) tmem_dealloc(tmem, 2 * T_ACC_COLS);
+}
+
+// ---- host: tensor maps ------------------------------------------------------------------
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*PFN_encodeIm2col)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                     const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*, CUtensorMapInterleave,
+                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static PFN_encodeTiled g_encode_tiled = nullptr;
+static PFN_encodeIm2col g_encode_im2col = nullptr;
+
+static bool load_encoders() {
+    if (g_encode_tiled && g_encode_im2col) return true;
+    cudaDriverEntryPointQueryResult q;
+    void* f = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || !f) return false;
+    g_encode_tiled = (PFN_encodeTiled)f;
+    f = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || !f) return false;
+    g_encode_im2col = (PFN_encodeIm2col)f;
+    return true;
+}
+
+bool conv_umma_tma_supports(const ConvParams& p) {
+    if (p.flags & (DR_POOL | DR_LRN)) return false;   // staged epilogues live in the gather kernel
+    if (p.patch) return false;
+    if ((p.Cin & 7) || p.Cin < 64) return false;      // TMA strides are 16-byte multiples; 128-byte rows
+    if (p.Nt > 256) return false;
+    if (p.k > 255 || p.M <= 0) return false;
+    if (p.M > 0x7fffffffLL) return false;
+    return true;
+}
+
+int conv_umma_tma_launch(const ConvParams& p, cudaStream_t stream) {
+    if (!conv_umma_tma_supports(p)) return DR_ERR_UNSUPPORTED;
+    if (!load_encoders()) return DR_ERR_CUDA;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(conv_umma_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM) != cudaSuccess) return DR_ERR_CUDA;
+        attr_set = true;
+    }
+    alignas(64) CUtensorMap map_a, map_b;
+    const int a_mode = (p.k == 1 && p.stride == 1 && p.pad == 0) ? 0 : 1;
+    if (a_mode == 0) {
+        const cuuint64_t dims[2] = {(cuuint64_t)p.Cin, (cuuint64_t)p.M};
+        const cuuint64_t strides[1] = {(cuuint64_t)p.Cin * 2};
+        const cuuint32_t box[2] = {64, TILE_M};
+        const cuuint32_t es[2] = {1, 1};
+        if (g_encode_tiled(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)p.x, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DR_ERR_CUDA;
+    } else {
+        const cuuint64_t dims[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
+        const cuuint64_t strides[3] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.W * p.Cin * 2, (cuuint64_t)p.H * p.W * p.Cin * 2};
+        // bounding box of the positions the filter's first tap visits: [-pad, extent + pad - k]
+        const int lower[2] = {-p.pad, -p.pad};
+        const int upper[2] = {p.pad - (p.k - 1), p.pad - (p.k - 1)};
+        const cuuint32_t es[4] = {1, (cuuint32_t)p.stride, (cuuint32_t)p.stride, 1};
+        if (g_encode_im2col(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void*)p.x, dims, strides, lower, upper, 64, TILE_M, es,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DR_ERR_CUDA;
+    }
+    {
+        const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
+        const cuuint64_t strides[2] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.K * 2};
+        const cuuint32_t box[3] = {64, 1, (cuuint32_t)p.Nt};
+        const cuuint32_t es[3] = {1, 1, 1};
+        if (g_encode_tiled(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)p.w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DR_ERR_CUDA;
+    }
+    const int total = p.m_tiles * p.n_blocks;
+    if (total <= 0) return DR_OK;
+    const int grid = total < num_sms() ? total : num_sms();
+    conv_umma_tma_kernel<<<grid, T_THREADS, T_SMEM, stream>>>(p, map_a, map_b, a_mode);
+    count_launch();
+    return launch_status();
+}
+
+}  // namespace dr

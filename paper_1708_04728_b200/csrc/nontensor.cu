@@ -1,0 +1,476 @@
+// Stand-alone non-tensor layers (ReLU, max-pool, LRN, BatchNorm/Scale, add, concat, global
+// average pool) and the offline parameter kernels (BN fold, filter embedding).
+//
+// These are the layers Section 2 of the paper calls "non-tensor": no weights, one pass over
+// the activations each.  On this hardware they are bound by HBM bandwidth, so every kernel
+// moves 128 bits per thread per access, coalesced along the channel axis of NHWC, with a grid
+// sized to a few waves of the SMs.
+#include "common.cuh"
+
+namespace dr {
+
+std::atomic<long long> g_launches{0};
+__device__ int g_dev_status[4] = {0, 0, 0, 0};
+
+int* dev_status_ptr() {
+    static int* ptr[64] = {nullptr};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return nullptr;
+    if (!ptr[dev] && cudaGetSymbolAddress((void**)&ptr[dev], g_dev_status) != cudaSuccess) ptr[dev] = nullptr;
+    return ptr[dev];
+}
+
+static int g_num_sms = 0;
+int num_sms() {
+    if (!g_num_sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (g_num_sms <= 0) g_num_sms = 148;
+    }
+    return g_num_sms;
+}
+
+static inline int grid_for(size_t work_items, int threads) {
+    size_t blocks = (work_items + threads - 1) / threads;
+    size_t cap = (size_t)num_sms() * 16;           // grid-stride beyond 16 blocks per SM
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+// ---------------------------------------------------------------- ReLU / add: 8 bf16 per thread
+__global__ void relu_kernel(size_t n8, size_t n, const uint4* __restrict__ x, uint4* __restrict__ y) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {
+        uint4 v = __ldg(x + i);
+        uint32_t* u = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) u[j] = pack_bf16(fmaxf(bf16_lo(u[j]), 0.f), fmaxf(bf16_hi(u[j]), 0.f));
+        y[i] = v;
+    }
+    // tail (n not a multiple of 8), handled by the first threads
+    const __nv_bfloat16* xs = reinterpret_cast<const __nv_bfloat16*>(x);
+    __nv_bfloat16* ys = reinterpret_cast<__nv_bfloat16*>(y);
+    for (size_t i = n8 * 8 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+        ys[i] = __float2bfloat16_rn(fmaxf(__bfloat162float(xs[i]), 0.f));
+}
+
+__global__ void add_kernel(size_t n8, size_t n, const uint4* __restrict__ a, const uint4* __restrict__ b,
+                           uint4* __restrict__ y) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {
+        uint4 va = __ldg(a + i), vb = __ldg(b + i), vo;
+        const uint32_t* ua = reinterpret_cast<const uint32_t*>(&va);
+        const uint32_t* ub = reinterpret_cast<const uint32_t*>(&vb);
+        uint32_t* uo = reinterpret_cast<uint32_t*>(&vo);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            uo[j] = pack_bf16(bf16_lo(ua[j]) + bf16_lo(ub[j]), bf16_hi(ua[j]) + bf16_hi(ub[j]));
+        y[i] = vo;
+    }
+    const __nv_bfloat16* as = reinterpret_cast<const __nv_bfloat16*>(a);
+    const __nv_bfloat16* bs = reinterpret_cast<const __nv_bfloat16*>(b);
+    __nv_bfloat16* ys = reinterpret_cast<__nv_bfloat16*>(y);
+    for (size_t i = n8 * 8 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+        ys[i] = __float2bfloat16_rn(__bfloat162float(as[i]) + __bfloat162float(bs[i]));
+}
+
+// ---------------------------------------------------------------- BatchNorm (+ Scale)
+// y = (x - mean/m) * g/sqrt(var/m+eps) + beta (g=1, beta=0 without Scale; mean == nullptr: Scale only).
+// One thread per 8 consecutive channels of one pixel; C must be a multiple of 8 for the
+// vector path, otherwise the scalar kernel runs.
+__global__ void bn_kernel(size_t nvec, int C8, const uint4* __restrict__ x, const float* __restrict__ mean,
+                          const float* __restrict__ var, float inv_m, float eps, const float* __restrict__ gamma,
+                          const float* __restrict__ beta, uint4* __restrict__ y) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
+        const int c0 = (int)(i % C8) * 8;
+        uint4 v = __ldg(x + i);
+        uint32_t* u = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float r[2] = {bf16_lo(u[j]), bf16_hi(u[j])};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int c = c0 + 2 * j + h;
+                const float a = (gamma ? __ldg(gamma + c) : 1.f) * (mean ? rsqrtf(__ldg(var + c) * inv_m + eps) : 1.f);
+                r[h] = (r[h] - (mean ? __ldg(mean + c) * inv_m : 0.f)) * a + (gamma ? __ldg(beta + c) : 0.f);
+            }
+            u[j] = pack_bf16(r[0], r[1]);
+        }
+        y[i] = v;
+    }
+}
+__global__ void bn_scalar_kernel(size_t n, int C, const __nv_bfloat16* __restrict__ x, const float* __restrict__ mean,
+                                 const float* __restrict__ var, float inv_m, float eps,
+                                 const float* __restrict__ gamma, const float* __restrict__ beta,
+                                 __nv_bfloat16* __restrict__ y) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        const int c = (int)(i % C);
+        const float a = (gamma ? gamma[c] : 1.f) * (mean ? rsqrtf(var[c] * inv_m + eps) : 1.f);
+        y[i] = __float2bfloat16_rn((__bfloat162float(x[i]) - (mean ? mean[c] * inv_m : 0.f)) * a + (gamma ? beta[c] : 0.f));
+    }
+}
+
+// ---------------------------------------------------------------- max-pool
+// One thread per (output pixel, 8 channels).  First maximum in row-major window order wins.
+__global__ void maxpool_kernel(int B, int H, int W, int C8, int Ho, int Wo, int k, int s, int p,
+                               const uint4* __restrict__ x, uint4* __restrict__ y, int32_t* __restrict__ argmax) {
+    const size_t total = (size_t)B * Ho * Wo * C8;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int c8 = (int)(i % C8);
+        size_t q = i / C8;
+        const int wo = (int)(q % Wo); q /= Wo;
+        const int ho = (int)(q % Ho);
+        const int n = (int)(q / Ho);
+        float best[8];
+        int where[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { best[j] = 0.f; where[j] = -1; }
+        for (int r = 0; r < k; ++r) {
+            const int hi = ho * s - p + r;
+            if (hi < 0 || hi >= H) continue;
+            for (int t = 0; t < k; ++t) {
+                const int wi = wo * s - p + t;
+                if (wi < 0 || wi >= W) continue;
+                const uint4 v = __ldg(x + (((size_t)n * H + hi) * W + wi) * C8 + c8);
+                const uint32_t* u = reinterpret_cast<const uint32_t*>(&v);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float lo = bf16_lo(u[j]), hi2 = bf16_hi(u[j]);
+                    if (where[2 * j] < 0 || lo > best[2 * j]) { best[2 * j] = lo; where[2 * j] = hi * W + wi; }
+                    if (where[2 * j + 1] < 0 || hi2 > best[2 * j + 1]) { best[2 * j + 1] = hi2; where[2 * j + 1] = hi * W + wi; }
+                }
+            }
+        }
+        uint4 o;
+        uint32_t* uo = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) uo[j] = pack_bf16(best[2 * j], best[2 * j + 1]);
+        y[i] = o;
+        if (argmax) {
+            int4* a = reinterpret_cast<int4*>(argmax + i * 8);
+            a[0] = make_int4(where[0], where[1], where[2], where[3]);
+            a[1] = make_int4(where[4], where[5], where[6], where[7]);
+        }
+    }
+}
+__global__ void maxpool_scalar_kernel(int B, int H, int W, int C, int Ho, int Wo, int k, int s, int p,
+                                      const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
+                                      int32_t* __restrict__ argmax) {
+    const size_t total = (size_t)B * Ho * Wo * C;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int c = (int)(i % C);
+        size_t q = i / C;
+        const int wo = (int)(q % Wo); q /= Wo;
+        const int ho = (int)(q % Ho);
+        const int n = (int)(q / Ho);
+        float best = 0.f; int where = -1;
+        for (int r = 0; r < k; ++r) {
+            const int hi = ho * s - p + r;
+            if (hi < 0 || hi >= H) continue;
+            for (int t = 0; t < k; ++t) {
+                const int wi = wo * s - p + t;
+                if (wi < 0 || wi >= W) continue;
+                const float v = __bfloat162float(x[(((size_t)n * H + hi) * W + wi) * C + c]);
+                if (where < 0 || v > best) { best = v; where = hi * W + wi; }
+            }
+        }
+        y[i] = __float2bfloat16_rn(best);
+        if (argmax) argmax[i] = where;
+    }
+}
+
+// ---------------------------------------------------------------- LRN across channels
+// One thread per (pixel, 8 channels).  It loads its own 16 bytes and the 16-byte groups on either
+// side (served by L1: the neighbouring threads load them as their own), so HBM sees the tensor
+// once.  Window half-width up to 8.
+__device__ __forceinline__ void unpack8(const uint4& q, float* v) {
+    const uint32_t* u = reinterpret_cast<const uint32_t*>(&q);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { v[2 * j] = bf16_lo(u[j]); v[2 * j + 1] = bf16_hi(u[j]); }
+}
+__global__ void lrn_kernel(size_t nvec, int C8, int half, float alpha_n, float beta, float kappa,
+                           const uint4* __restrict__ x, uint4* __restrict__ y) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
+        const int c8 = (int)(i % C8);
+        float v[24];
+        unpack8(__ldg(x + i), v + 8);
+        if (c8 > 0) unpack8(__ldg(x + i - 1), v);
+        else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = 0.f;
+        }
+        if (c8 + 1 < C8) unpack8(__ldg(x + i + 1), v + 16);
+        else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[16 + j] = 0.f;
+        }
+        float sq[24];
+#pragma unroll
+        for (int j = 0; j < 24; ++j) sq[j] = v[j] * v[j];
+        float r[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            float ss = sq[8 + j];
+#pragma unroll
+            for (int d = 1; d <= 8; ++d)
+                if (d <= half) ss += sq[8 + j - d] + sq[8 + j + d];
+            r[j] = v[8 + j] * lrn_pow(kappa + alpha_n * ss, beta);
+        }
+        uint4 o;
+        uint32_t* uo = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) uo[j] = pack_bf16(r[2 * j], r[2 * j + 1]);
+        y[i] = o;
+    }
+}
+__global__ void lrn_scalar_kernel(size_t n, int C, int half, float alpha_n, float beta, float kappa,
+                                  const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        const int c = (int)(i % C);
+        float ss = 0.f;
+        for (int d = -half; d <= half; ++d)
+            if (c + d >= 0 && c + d < C) { const float t = __bfloat162float(x[i + d]); ss += t * t; }
+        y[i] = __float2bfloat16_rn(__bfloat162float(x[i]) * lrn_pow(kappa + alpha_n * ss, beta));
+    }
+}
+
+// ---------------------------------------------------------------- concat: strided channel copy
+__global__ void concat_kernel(size_t nvec, int C8, int ldc8, int coff8, const uint4* __restrict__ x,
+                              uint4* __restrict__ y) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
+        const size_t pix = i / C8;
+        const int c8 = (int)(i % C8);
+        y[pix * ldc8 + coff8 + c8] = __ldg(x + i);
+    }
+}
+__global__ void concat_scalar_kernel(size_t n, int C, int ldc, int coff, const __nv_bfloat16* __restrict__ x,
+                                     __nv_bfloat16* __restrict__ y) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+        y[(i / C) * ldc + coff + (i % C)] = x[i];
+}
+
+// ---------------------------------------------------------------- global average pool
+// One block per (image, 64-channel slab): threads split the plane, partial sums meet in shared
+// memory in a fixed order (deterministic).  blockDim = (64 channels / 2, PIXSPLIT).
+constexpr int AVG_SPLIT = 8;
+__global__ void avgpool_kernel(int HW, int C, const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y) {
+    __shared__ float part[AVG_SPLIT][64];
+    const int n = blockIdx.y, c = blockIdx.x * 64 + threadIdx.x * 2;
+    float s0 = 0.f, s1 = 0.f;
+    if (c < C) {
+        for (int q = threadIdx.y; q < HW; q += AVG_SPLIT) {
+            const __nv_bfloat16* p = x + ((size_t)n * HW + q) * C + c;
+            if (c + 1 < C) {
+                const uint32_t u = *reinterpret_cast<const uint32_t*>(p);
+                s0 += bf16_lo(u); s1 += bf16_hi(u);
+            } else {
+                s0 += __bfloat162float(p[0]);
+            }
+        }
+    }
+    part[threadIdx.y][threadIdx.x * 2] = s0;
+    part[threadIdx.y][threadIdx.x * 2 + 1] = s1;
+    __syncthreads();
+    if (threadIdx.y == 0) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float s = 0.f;
+#pragma unroll
+            for (int k = 0; k < AVG_SPLIT; ++k) s += part[k][threadIdx.x * 2 + h];
+            if (c + h < C) y[(size_t)n * C + c + h] = __float2bfloat16_rn(s / (float)HW);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- Lemma 2: BN/Scale fold
+// One block per output channel j; eta_j computed once per thread, weights streamed.
+__global__ void fold_bn_kernel(int K, const __nv_bfloat16* __restrict__ w_in, const float* __restrict__ b_in,
+                               const float* __restrict__ mean, const float* __restrict__ var, float inv_m, float eps,
+                               const float* __restrict__ gamma, const float* __restrict__ beta,
+                               __nv_bfloat16* __restrict__ w_out, float* __restrict__ b_out) {
+    const int j = blockIdx.x;
+    const float eta = gamma[j] / sqrtf(var[j] * inv_m + eps);
+    for (int i = threadIdx.x; i < K; i += blockDim.x)
+        w_out[(size_t)j * K + i] = __float2bfloat16_rn(eta * __bfloat162float(w_in[(size_t)j * K + i]));
+    if (threadIdx.x == 0) b_out[j] = eta * (b_in ? b_in[j] : 0.f) + beta[j] - eta * mean[j] * inv_m;
+}
+
+// ---------------------------------------------------------------- zero-embedding of a small filter
+__global__ void embed_filter_kernel(int Cin, int ks, int kb, const __nv_bfloat16* __restrict__ w_small, int joff,
+                                    __nv_bfloat16* __restrict__ w_big) {
+    const int j = blockIdx.x, o = (kb - ks) / 2;
+    const int per = kb * kb * Cin;
+    for (int i = threadIdx.x; i < per; i += blockDim.x) {
+        const int c = i % Cin, t = i / Cin, s = t % kb - o, r = t / kb - o;
+        __nv_bfloat16 v = __float2bfloat16_rn(0.f);
+        if (r >= 0 && r < ks && s >= 0 && s < ks) v = w_small[(((size_t)j * ks + r) * ks + s) * Cin + c];
+        w_big[(size_t)(joff + j) * per + i] = v;
+    }
+}
+
+}  // namespace dr
+
+// ================================================================ C ABI
+using namespace dr;
+#define DR_REQUIRE(cond, code) do { if (!(cond)) return (code); } while (0)
+
+extern "C" {
+
+const char* dr_strerror(int status) {
+    switch (status) {
+        case DR_OK: return "ok";
+        case DR_ERR_INVALID_ARG: return "invalid argument";
+        case DR_ERR_UNSUPPORTED: return "unsupported configuration";
+        case DR_ERR_ALIGNMENT: return "pointer, channel stride or channel offset misaligned";
+        case DR_ERR_WORKSPACE: return "workspace missing or too small, or net not prepared";
+        case DR_ERR_CUDA: return "CUDA call failed";
+        case DR_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown status";
+    }
+}
+
+long long dr_launch_count(void) { return g_launches.load(); }
+
+int dr_device_status(int info[4]) {
+    int h[4] = {0, 0, 0, 0};
+    if (cudaDeviceSynchronize() != cudaSuccess) return DR_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(h, g_dev_status, sizeof(h)) != cudaSuccess) return DR_ERR_CUDA;
+    if (h[0] != 0) {
+        int z[4] = {0, 0, 0, 0};
+        if (cudaMemcpyToSymbol(g_dev_status, z, sizeof(z)) != cudaSuccess) return DR_ERR_CUDA;
+    }
+    if (info) for (int i = 0; i < 4; ++i) info[i] = h[i];
+    return h[0] == 0 ? DR_OK : DR_ERR_DEVICE_TIMEOUT;
+}
+
+int dr_relu(size_t n, const void* x, void* y, void* stream) {
+    DR_REQUIRE(x && y, DR_ERR_INVALID_ARG);
+    if (n == 0) return DR_OK;
+    DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
+    relu_kernel<<<grid_for((n + 7) / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, n, (const uint4*)x, (uint4*)y);
+    count_launch();
+    return launch_status();
+}
+
+int dr_add(size_t n, const void* a, const void* b, void* y, void* stream) {
+    DR_REQUIRE(a && b && y, DR_ERR_INVALID_ARG);
+    if (n == 0) return DR_OK;
+    DR_REQUIRE(aligned16(a) && aligned16(b) && aligned16(y), DR_ERR_ALIGNMENT);
+    add_kernel<<<grid_for((n + 7) / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, n, (const uint4*)a, (const uint4*)b, (uint4*)y);
+    count_launch();
+    return launch_status();
+}
+
+int dr_bn(int B, int H, int W, int C, const void* x, const float* mean, const float* var, float m, float eps,
+          const float* gamma, const float* beta, void* y, void* stream) {
+    DR_REQUIRE(x && y && mean && var, DR_ERR_INVALID_ARG);
+    DR_REQUIRE(B >= 0 && H >= 0 && W >= 0 && C > 0 && m != 0.f && eps >= 0.f, DR_ERR_INVALID_ARG);
+    DR_REQUIRE(gamma == nullptr || beta != nullptr, DR_ERR_INVALID_ARG);
+    const size_t n = (size_t)B * H * W * C;
+    if (n == 0) return DR_OK;
+    DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
+    if (C % 8 == 0)
+        bn_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, C / 8, (const uint4*)x, mean, var, 1.f / m, eps, gamma, beta, (uint4*)y);
+    else
+        bn_scalar_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(n, C, (const __nv_bfloat16*)x, mean, var, 1.f / m, eps, gamma, beta, (__nv_bfloat16*)y);
+    count_launch();
+    return launch_status();
+}
+
+int dr_scale(int B, int H, int W, int C, const void* x, const float* gamma, const float* beta, void* y, void* stream) {
+    DR_REQUIRE(x && y && gamma && beta, DR_ERR_INVALID_ARG);
+    DR_REQUIRE(B >= 0 && H >= 0 && W >= 0 && C > 0, DR_ERR_INVALID_ARG);
+    const size_t n = (size_t)B * H * W * C;
+    if (n == 0) return DR_OK;
+    DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
+    if (C % 8 == 0)
+        bn_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, C / 8, (const uint4*)x, nullptr, nullptr, 1.f, 0.f, gamma, beta, (uint4*)y);
+    else
+        bn_scalar_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(n, C, (const __nv_bfloat16*)x, nullptr, nullptr, 1.f, 0.f, gamma, beta, (__nv_bfloat16*)y);
+    count_launch();
+    return launch_status();
+}
+
+int dr_maxpool(int B, int H, int W, int C, int k, int s, int p, const void* x, void* y, int32_t* argmax, void* stream) {
+    DR_REQUIRE(x && y, DR_ERR_INVALID_ARG);
+    DR_REQUIRE(B >= 0 && H > 0 && W > 0 && C > 0 && k > 0 && s > 0 && p >= 0 && 2 * p < k + 1 && p < k, DR_ERR_INVALID_ARG);
+    DR_REQUIRE(H + 2 * p >= k && W + 2 * p >= k, DR_ERR_INVALID_ARG);
+    const int Ho = (H + 2 * p - k) / s + 1, Wo = (W + 2 * p - k) / s + 1;
+    const size_t n = (size_t)B * Ho * Wo * C;
+    if (n == 0) return DR_OK;
+    DR_REQUIRE(aligned16(x) && aligned16(y) && (!argmax || aligned16(argmax)), DR_ERR_ALIGNMENT);
+    if (C % 8 == 0)
+        maxpool_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C / 8, Ho, Wo, k, s, p, (const uint4*)x, (uint4*)y, argmax);
+    else
+        maxpool_scalar_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C, Ho, Wo, k, s, p, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, argmax);
+    count_launch();
+    return launch_status();
+}
+
+int dr_lrn(int B, int H, int W, int C, int size, float alpha, float beta, float k, const void* x, void* y, void* stream) {
+    DR_REQUIRE(x && y, DR_ERR_INVALID_ARG);
+    DR_REQUIRE(B >= 0 && H >= 0 && W >= 0 && C > 0 && size >= 1 && (size & 1) && size <= 15, DR_ERR_INVALID_ARG);
+    const size_t n = (size_t)B * H * W * C;
+    if (n == 0) return DR_OK;
+    DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
+    if (C % 8 == 0)
+        lrn_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, C / 8, size / 2, alpha / size, beta, k, (const uint4*)x, (uint4*)y);
+    else
+        lrn_scalar_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(n, C, size / 2, alpha / size, beta, k, (const __nv_bfloat16*)x, (__nv_bfloat16*)y);
+    count_launch();
+    return launch_status();
+}
+
+int dr_concat(size_t npix, int C, const void* x, int ldc, int coff, void* y, void* stream) {
+    DR_REQUIRE(x && y && C > 0 && ldc >= C && coff >= 0 && coff + C <= ldc, DR_ERR_INVALID_ARG);
+    if (npix == 0) return DR_OK;
+    DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
+    const size_t n = npix * C;
+    if (C % 8 == 0 && ldc % 8 == 0 && coff % 8 == 0)
+        concat_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, C / 8, ldc / 8, coff / 8, (const uint4*)x, (uint4*)y);
+    else
+        concat_scalar_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(n, C, ldc, coff, (const __nv_bfloat16*)x, (__nv_bfloat16*)y);
+    count_launch();
+    return launch_status();
+}
+
+int dr_avgpool_global(int B, int H, int W, int C, const void* x, void* y, void* stream) {
+    DR_REQUIRE(x && y && B >= 0 && H > 0 && W > 0 && C > 0, DR_ERR_INVALID_ARG);
+    if (B == 0) return DR_OK;
+    DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
+    DR_REQUIRE(C % 2 == 0, DR_ERR_UNSUPPORTED);
+    dim3 grid((C + 63) / 64, B), block(32, AVG_SPLIT);
+    avgpool_kernel<<<grid, block, 0, (cudaStream_t)stream>>>(H * W, C, (const __nv_bfloat16*)x, (__nv_bfloat16*)y);
+    count_launch();
+    return launch_status();
+}
+
+int dr_fold_bn(int Cout, int K, const void* w_in, const float* b_in, const float* mean, const float* var, float m,
+               float eps, const float* gamma, const float* beta, void* w_out, float* b_out, void* stream) {
+    DR_REQUIRE(w_in && mean && var && gamma && beta && w_out && b_out, DR_ERR_INVALID_ARG);
+    DR_REQUIRE(Cout > 0 && K > 0 && m != 0.f && eps >= 0.f, DR_ERR_INVALID_ARG);
+    fold_bn_kernel<<<Cout, 256, 0, (cudaStream_t)stream>>>(K, (const __nv_bfloat16*)w_in, b_in, mean, var, 1.f / m, eps, gamma, beta, (__nv_bfloat16*)w_out, b_out);
+    count_launch();
+    return launch_status();
+}
+
+int dr_embed_filter(int Cout, int Cin, int ks, int kb, const void* w_small, int joff, void* w_big, void* stream) {
+    DR_REQUIRE(w_small && w_big, DR_ERR_INVALID_ARG);
+    DR_REQUIRE(Cout > 0 && Cin > 0 && ks > 0 && kb >= ks && (ks & 1) && (kb & 1) && joff >= 0, DR_ERR_INVALID_ARG);
+    embed_filter_kernel<<<Cout, 256, 0, (cudaStream_t)stream>>>(Cin, ks, kb, (const __nv_bfloat16*)w_small, joff, (__nv_bfloat16*)w_big);
+    count_launch();
+    return launch_status();
+}
+
+}  // extern "C"

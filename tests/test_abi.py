@@ -1,0 +1,141 @@
+"""Host-side checks of the C-ABI library: it loads, exports every declared symbol, validates
+arguments before touching the device, and builds the two networks' layer lists (no GPU needed)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def dr():
+    from paper_1708_04728_b200 import build
+    build.build()
+    import paper_1708_04728_b200 as dr
+    return dr
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "dr.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(dr_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(dr):
+    lib = C.CDLL(dr.LIB_PATH)
+    names = declared_symbols()
+    assert len(names) >= 30
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/dr.h but not exported"
+    assert set(dr.EXPORTS) == set(names), set(dr.EXPORTS) ^ set(names)
+
+
+def test_strerror(dr):
+    assert dr.dr_strerror(0) == "ok"
+    for code in range(-6, 0):
+        assert dr.dr_strerror(code) not in ("ok", "unknown status")
+    assert dr.dr_strerror(-99) == "unknown status"
+
+
+def test_conv_validation_rejects_before_launch(dr):
+    d = dr.dr_conv_desc(k=3, stride=1, pad=1, Cin=16, Cout=16, flags=dr.DR_BIAS)
+    n0 = dr.dr_launch_count()
+    with pytest.raises(dr.DrError) as e:       # null pointers
+        dr.dr_conv_slim(d, 1, 8, 8, None, None, None, None, None, None, 0)
+    assert e.value.status == dr.DR_ERR_INVALID_ARG
+    with pytest.raises(dr.DrError) as e:       # bias flag without bias
+        dr.dr_conv_slim(d, 1, 8, 8, 256, 256, None, None, 256, None, 0)
+    assert e.value.status == dr.DR_ERR_INVALID_ARG
+    with pytest.raises(dr.DrError) as e:       # misaligned pointer
+        dr.dr_conv_slim(d, 1, 8, 8, 260, 256, 256, None, 256, None, 0)
+    assert e.value.status == dr.DR_ERR_ALIGNMENT
+    d.flags = dr.DR_POOL | dr.DR_RESIDUAL
+    d.pool_k, d.pool_stride, d.pool_pad = 3, 2, 1
+    with pytest.raises(dr.DrError) as e:       # pooling together with a residual is not built
+        dr.dr_conv_slim(d, 1, 8, 8, 256, 256, None, 256, 256, None, 0)
+    assert e.value.status == dr.DR_ERR_UNSUPPORTED
+    d.flags = dr.DR_POOL
+    d.pool_k = 2
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_conv_slim(d, 1, 8, 8, 256, 256, None, None, 256, None, 0)
+    assert e.value.status == dr.DR_ERR_UNSUPPORTED
+    d = dr.dr_conv_desc(k=3, stride=1, pad=1, Cin=16, Cout=16, flags=0, y_ldc=20, y_coff=0)
+    with pytest.raises(dr.DrError) as e:       # channel stride not a multiple of 8
+        dr.dr_conv_slim(d, 1, 8, 8, 256, 256, None, None, 256, None, 0)
+    assert e.value.status == dr.DR_ERR_ALIGNMENT
+    d = dr.dr_conv_desc(k=9, stride=1, pad=0, Cin=16, Cout=16, flags=0)
+    with pytest.raises(dr.DrError) as e:       # kernel larger than the padded plane
+        dr.dr_conv_slim(d, 1, 8, 8, 256, 256, None, None, 256, None, 0)
+    assert e.value.status == dr.DR_ERR_INVALID_ARG
+    assert dr.dr_launch_count() == n0
+
+
+def test_non_tensor_validation(dr):
+    n0 = dr.dr_launch_count()
+    for call in (lambda: dr.dr_relu(16, None, 256, 0),
+                 lambda: dr.dr_maxpool(1, 8, 8, 8, 3, 2, 1, None, 256, None, 0),
+                 lambda: dr.dr_lrn(1, 8, 8, 8, 4, 1e-4, 0.75, 1.0, 256, 256, 0),      # even window
+                 lambda: dr.dr_bn(1, 8, 8, 8, 256, 256, 256, 0.0, 0.0, None, None, 256, 0),  # m = 0
+                 lambda: dr.dr_concat(4, 8, 256, 8, 8, 256, 0),                        # slice outside ldc
+                 lambda: dr.dr_fold_bn(0, 9, 256, None, 256, 256, 1.0, 0.0, 256, 256, 256, 256, 0)):
+        with pytest.raises(dr.DrError) as e:
+            call()
+        assert e.value.status == dr.DR_ERR_INVALID_ARG
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_relu(16, 257, 256, 0)
+    assert e.value.status == dr.DR_ERR_ALIGNMENT
+    assert dr.dr_launch_count() == n0
+
+
+def test_googlenet_layer_lists(dr):
+    slim = dr.Net(dr.DR_ARCH_GOOGLENET, dr.DR_MODE_SLIM, 2)
+    uns = dr.Net(dr.DR_ARCH_GOOGLENET, dr.DR_MODE_UNSLIMMED, 2)
+    names = [slim.dr_net_layer_info(i)["name"] for i in range(slim.dr_net_num_layers())]
+    # 3 stem convs + 9 modules x 3 convs + 2 pools + avg-pool + fc
+    assert len(names) == 3 + 27 + 2 + 1 + 1
+    assert names[:3] == ["conv1", "conv2r", "conv2"] and names[-2:] == ["avgpool", "fc"]
+    assert sum(slim.dr_net_layer_info(i)["kind"] == 0 for i in range(len(names))) == 31
+    li = {slim.dr_net_layer_info(i)["name"]: slim.dr_net_layer_info(i) for i in range(len(names))}
+    assert li["conv1"]["dims"] == (2, 56, 56, 64) and li["conv2"]["dims"] == (2, 28, 28, 192)
+    assert li["3a.3x3"]["dims"] == (2, 28, 28, 128) and (li["3a.3x3"]["ldc"], li["3a.3x3"]["coff"]) == (256, 0)
+    assert li["3a.m5"]["dims"] == (2, 28, 28, 128) and (li["3a.m5"]["ldc"], li["3a.m5"]["coff"]) == (256, 128)
+    assert li["5b.m5"]["dims"] == (2, 7, 7, 640) and li["5b.m5"]["ldc"] == 1024
+    assert li["fc"]["dims"] == (2, 1, 1, 1000) and li["fc"]["is_f32"]
+    # dense merged 5x5 FLOPs: 2*M*N*K
+    assert li["3a.m5"]["flops"] == 2.0 * (2 * 28 * 28) * 128 * (25 * 192)
+    total = sum(v["flops"] for v in li.values()) / 2
+    assert abs(total / 1e9 - 16.64) < 0.02          # GFLOP per image of the branch-slimmed form
+    # both modes take the same parameter list
+    ps = [slim.dr_net_param_spec(i) for i in range(slim.dr_net_num_params())]
+    pu = [uns.dr_net_param_spec(i) for i in range(uns.dr_net_num_params())]
+    assert ps == pu and len(ps) == 2 * (3 + 9 * 5 + 1)
+    n_uns = uns.dr_net_num_layers()
+    kinds = [uns.dr_net_layer_info(i)["kind"] for i in range(n_uns)]
+    assert kinds.count(0) == 3 + 9 * 5 + 1 and n_uns > 2 * len(names)
+    assert slim.dr_net_workspace_bytes() > 0 and uns.dr_net_activation_bytes() > slim.dr_net_activation_bytes()
+    with pytest.raises(dr.DrError) as e:      # forward before prepare
+        slim.dr_net_forward(256, 256, 256, 0)
+    assert e.value.status == dr.DR_ERR_WORKSPACE
+
+
+def test_resnet50_layer_lists(dr):
+    slim = dr.Net(dr.DR_ARCH_RESNET50, dr.DR_MODE_SLIM, 1)
+    n = slim.dr_net_num_layers()
+    infos = [slim.dr_net_layer_info(i) for i in range(n)]
+    assert sum(i["kind"] == 0 for i in infos) == 54 and n == 55      # 53 convs + fc, + avg-pool
+    total = sum(i["flops"] for i in infos)
+    assert abs(total / 1e9 - 7.72) < 0.02
+    names = {i["name"]: i for i in infos}
+    assert names["res3a.2a"]["dims"] == (1, 28, 28, 128)             # stride 2 on the first 1x1
+    assert names["res5c.2c"]["dims"] == (1, 7, 7, 2048)
+    uns = dr.Net(dr.DR_ARCH_RESNET50, dr.DR_MODE_UNSLIMMED, 1)
+    ku = [uns.dr_net_layer_info(i) for i in range(uns.dr_net_num_layers())]
+    assert sum(i["kind"] == 0 for i in ku) == 54
+    # every conv is followed by BatchNorm and Scale launches of their own
+    assert sum(i["name"].endswith(".bn") for i in ku) == 53
+    with pytest.raises(dr.DrError):
+        dr.Net(7, 0, 1)
+    with pytest.raises(dr.DrError):
+        dr.Net(0, 0, 1, 16, 16)

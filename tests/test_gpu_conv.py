@@ -1,0 +1,228 @@
+"""GPU parity of dr_conv_slim / dr_inception_slim against the unfused CPU checker, per kernel path."""
+import numpy as np
+import pytest
+
+import dr_synth as S
+import dr_synth.params as P
+from util import assert_layer_close, to_dev_bf16, to_dev_f32, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dr():
+    import paper_1708_04728_b200 as dr
+    yield dr
+    dr.dr_set_conv_path(dr.DR_PATH_AUTO)
+
+
+@pytest.fixture(scope="module")
+def O():
+    import oracle
+    return oracle
+
+
+def oracle_slim_layer(O, x, w, b, k, s, p, flags, dr, residual=None, lrn=(5, 1e-4, 0.75, 1.0)):
+    """The unfused layer sequence one slim layer stands for; returns (y, argmax or None)."""
+    y = O.conv2d(x, w, b if flags & dr.DR_BIAS else None, s, p)
+    arg = None
+    if flags & dr.DR_RELU:
+        y = O.relu(y)
+    if flags & dr.DR_LRN and (flags & dr.DR_LRN_BEFORE_POOL or not flags & dr.DR_POOL):
+        y = O.lrn(y, *lrn)
+    if flags & dr.DR_POOL:
+        y, arg = O.maxpool(y, 3, 2, 1)
+        if flags & dr.DR_LRN and not flags & dr.DR_LRN_BEFORE_POOL:
+            y = O.lrn(y, *lrn)
+    if flags & dr.DR_RESIDUAL:
+        y = O.add(y, residual)
+        if flags & dr.DR_RELU_AFTER_RESIDUAL:
+            y = O.relu(y)
+    return y, arg
+
+
+def run_conv(dr, x, w, b, k, s, p, flags, residual=None, ldc=0, coff=0, lrn=(5, 1e-4, 0.75, 1.0), want_argmax=False):
+    import torch
+    B, H, W, Cin = x.shape
+    Cout = w.shape[0]
+    d = dr.dr_conv_desc(k=k, stride=s, pad=p, Cin=Cin, Cout=Cout, flags=flags, pool_k=3, pool_stride=2, pool_pad=1,
+                        lrn_size=lrn[0], lrn_alpha=lrn[1], lrn_beta=lrn[2], lrn_k=lrn[3], y_ldc=ldc, y_coff=coff)
+    Ho, Wo = (H + 2 * p - k) // s + 1, (W + 2 * p - k) // s + 1
+    if flags & dr.DR_POOL:
+        Ho, Wo = (Ho - 1) // 2 + 1, (Wo - 1) // 2 + 1
+    L = ldc or Cout
+    dt = torch.float32 if flags & dr.DR_OUT_F32 else torch.bfloat16
+    y = torch.full((B, Ho, Wo, L), 768.0, dtype=dt, device="cuda")      # canary outside the written slice
+    arg = torch.full((B, Ho, Wo, Cout), -7, dtype=torch.int32, device="cuda") if want_argmax else None
+    dr.dr_conv_slim(d, B, H, W, to_dev_bf16(x), to_dev_bf16(w), None if b is None else to_dev_f32(b),
+                    None if residual is None else to_dev_bf16(residual), y, arg)
+    st, info = dr.dr_device_status()
+    assert st == 0, f"device status {st} {info}"
+    yh = to_host(y)
+    if L != Cout:
+        mask = np.ones(L, bool); mask[coff:coff + Cout] = False
+        assert np.all(yh[..., mask] == 768.0), "wrote outside its channel slice"
+    return yh[..., coff:coff + Cout], (None if arg is None else arg.cpu().numpy())
+
+
+def paths(dr):
+    return [dr.DR_PATH_SIMT, dr.DR_PATH_UMMA_GATHER, dr.DR_PATH_UMMA_TMA]
+
+
+def force(dr, path):
+    dr.dr_set_conv_path(path)
+
+
+# (B,H,W,Cin,Cout,k,s,p): several tiles, ragged tails in M, N and K
+DIRECT_SHAPES = [
+    (2, 9, 11, 64, 64, 3, 1, 1),      # M = 198: one full tile + tail
+    (1, 28, 28, 192, 96, 1, 1, 0),    # 3a reducer
+    (1, 14, 14, 96, 128, 3, 1, 1),
+    (1, 12, 10, 48, 304, 5, 1, 2),    # two n-blocks of different width, K tail (48 of 64)
+    (3, 7, 7, 160, 320, 3, 1, 1),     # 7x7 planes, tile spans images
+    (2, 8, 8, 32, 40, 1, 2, 0),       # stride-2 1x1, Cout not a multiple of 16
+    (1, 17, 13, 16, 16, 3, 2, 1),     # stride-2 3x3
+    (2, 10, 10, 3, 64, 7, 2, 3),      # stem geometry, Cin = 3
+    (5, 1, 1, 1024, 1000, 1, 1, 0),   # FC shape
+]
+
+
+@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("shape", DIRECT_SHAPES)
+def test_conv_bias_relu(dr, O, path, shape):
+    B, H, W, Cin, Cout, k, s, p = shape
+    x = S.normal(10, "x", (B, H, W, Cin)); w = S.he_normal(10, "w", Cout, k, Cin); b = S.normal(10, "b", (Cout,), 0.1)
+    force(dr, path)
+    try:
+        got, _ = run_conv(dr, x, w, b, k, s, p, dr.DR_BIAS | dr.DR_RELU)
+    except dr.DrError as e:
+        if e.status == dr.DR_ERR_UNSUPPORTED and path != dr.DR_PATH_SIMT:
+            pytest.skip("path does not take this shape")
+        raise
+    assert dr.dr_last_conv_path() == path
+    ref, _ = oracle_slim_layer(O, x, w, b, k, s, p, dr.DR_BIAS | dr.DR_RELU, dr)
+    assert_layer_close(got, O.round_bf16(ref), f"path {path} {shape}")
+
+
+@pytest.mark.parametrize("path", [1, 2, 3])
+def test_conv_no_epilogue_f32_and_slice(dr, O, path):
+    B, H, W, Cin, Cout, k, s, p = 2, 6, 7, 32, 48, 3, 1, 1
+    x = S.normal(11, "x", (B, H, W, Cin)); w = S.he_normal(11, "w", Cout, k, Cin); b = S.normal(11, "b", (Cout,), 0.1)
+    force(dr, path)
+    try:
+        got, _ = run_conv(dr, x, w, None, k, s, p, 0, ldc=96, coff=24)             # raw conv into a channel slice
+        got32, _ = run_conv(dr, x, w, b, k, s, p, dr.DR_BIAS | dr.DR_OUT_F32)      # float32 store
+    except dr.DrError as e:
+        if e.status == dr.DR_ERR_UNSUPPORTED and path != dr.DR_PATH_SIMT:
+            pytest.skip("path does not take this shape")
+        raise
+    ref = O.conv2d(x, w, None, s, p)
+    assert_layer_close(got, O.round_bf16(ref), "slice")
+    ref32 = O.conv2d(x, w, b, s, p)
+    assert np.abs(got32 - ref32).max() <= 2e-3 * np.abs(ref32).max()   # bf16 products, fp32 accumulation, no output rounding
+
+
+@pytest.mark.parametrize("path", [1, 2, 3])
+def test_conv_residual_relu(dr, O, path):
+    B, H, W, Cin, Cout = 2, 7, 7, 64, 256
+    x = S.normal(12, "x", (B, H, W, Cin)); w = S.he_normal(12, "w", Cout, 1, Cin); b = S.normal(12, "b", (Cout,), 0.1)
+    r = S.normal(12, "r", (B, H, W, Cout))
+    flags = dr.DR_BIAS | dr.DR_RESIDUAL | dr.DR_RELU_AFTER_RESIDUAL
+    force(dr, path)
+    try:
+        got, _ = run_conv(dr, x, w, b, 1, 1, 0, flags, residual=r)
+    except dr.DrError as e:
+        if e.status == dr.DR_ERR_UNSUPPORTED and path != dr.DR_PATH_SIMT:
+            pytest.skip("path does not take this shape")
+        raise
+    ref, _ = oracle_slim_layer(O, x, w, b, 1, 1, 0, flags, dr, residual=r)
+    assert_layer_close(got, O.round_bf16(ref), "residual")
+
+
+def check_argmax(got_arg, ref_arg, pre_pool, ref_scale):
+    """Integer parity where the decision is not a near-tie in the checker's own values."""
+    B, Ho, Wo, Cc = pre_pool.shape
+    flat = pre_pool.reshape(B, Ho * Wo, Cc)
+    bad = got_arg != ref_arg
+    n_bad = int(bad.sum())
+    if n_bad == 0:
+        return 0
+    idx = np.argwhere(bad)
+    excused = 0
+    for n, ph, pw, c in idx:
+        a, b_ = got_arg[n, ph, pw, c], ref_arg[n, ph, pw, c]
+        assert 0 <= a < Ho * Wo, "argmax outside the plane"
+        # the position chosen must lie inside the window and hold a value within tolerance of the maximum
+        ah, aw = divmod(int(a), Wo)
+        assert abs(ah - 2 * ph) <= 1 and abs(aw - 2 * pw) <= 1, "argmax outside its window"
+        gap = flat[n, b_, c] - flat[n, a, c]
+        assert 0 <= gap <= 1e-3 * ref_scale, f"argmax differs on a clear decision (gap {gap})"
+        excused += 1
+    return excused
+
+
+# fused pooling / LRN epilogues (Cout <= 256): (B,H,W,Cin,Cout,k,s,p, flags-name)
+STAGED = [
+    (1, 64, 64, 3, 64, 7, 2, 3, "pool_lrn"),        # the stem configuration: ReLU -> pool -> LRN
+    (2, 20, 18, 64, 192, 3, 1, 1, "lrn_pool"),      # conv2 geometry: ReLU -> LRN -> pool
+    (2, 13, 9, 32, 48, 3, 1, 1, "pool"),
+    (1, 9, 12, 16, 32, 1, 1, 0, "lrn"),
+    (1, 5, 5, 8, 16, 3, 1, 1, "pool"),              # plane smaller than one patch
+]
+
+
+@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("case", STAGED)
+def test_conv_fused_pool_lrn(dr, O, path, case):
+    B, H, W, Cin, Cout, k, s, p, kind = case
+    flags = dr.DR_BIAS | dr.DR_RELU | {"pool_lrn": dr.DR_POOL | dr.DR_LRN, "lrn_pool": dr.DR_POOL | dr.DR_LRN | dr.DR_LRN_BEFORE_POOL,
+                                       "pool": dr.DR_POOL, "lrn": dr.DR_LRN}[kind]
+    x = S.normal(0, "x", (B, H, W, Cin)); w = S.he_normal(0, "conv1.w", Cout, k, Cin); b = S.normal(0, "conv1.b", (Cout,), 0.01)
+    lrn = (5, 1e-4, 0.75, 1.0) if kind == "pool_lrn" else (5, 0.05, 0.75, 1.0)      # second set makes LRN bite
+    force(dr, path)
+    try:
+        got, arg = run_conv(dr, x, w, b, k, s, p, flags, lrn=lrn, want_argmax=bool(flags & dr.DR_POOL))
+    except dr.DrError as e:
+        if e.status == dr.DR_ERR_UNSUPPORTED and path != dr.DR_PATH_SIMT:
+            pytest.skip("path does not take this shape")
+        raise
+    ref, ref_arg = oracle_slim_layer(O, x, w, b, k, s, p, flags, dr, lrn=lrn)
+    assert_layer_close(got, O.round_bf16(ref), f"{kind} path {path}")
+    if arg is not None:
+        pre = O.relu(O.conv2d(x, w, b, s, p))
+        if flags & dr.DR_LRN_BEFORE_POOL:
+            pre = O.lrn(pre, *lrn)
+        excused = check_argmax(arg, ref_arg, pre, np.abs(pre).max())
+        assert excused <= 0.02 * arg.size + 8, f"{excused} near-ties of {arg.size}"
+
+
+def test_inception_3a_config(dr, O):
+    """Branch-slimmed inception module at the 3a shape: batch 8, 192x28x28."""
+    import oracle.nets as N
+    import torch
+    params = P.inception_params(0, "3a")
+    cin, c1, c3r, c3, _, c5, pp = S.INCEPTION_V1["3a"]
+    cm = c1 + c5 + pp
+    B = 8
+    x = S.normal(0, "x", (B, 28, 28, cin))
+    wm = torch.empty((cm, 5, 5, cin), dtype=torch.bfloat16, device="cuda")
+    dr.dr_embed_filter(c1, cin, 1, 5, to_dev_bf16(params["3a.b1.w"]), 0, wm)
+    dr.dr_embed_filter(c5, cin, 5, 5, to_dev_bf16(params["3a.b5.w"]), c1, wm)
+    dr.dr_embed_filter(pp, cin, 3, 5, to_dev_bf16(params["3a.bp.w"]), c1 + c5, wm)
+    bm = to_dev_f32(np.concatenate([params["3a.b1.b"], params["3a.b5.b"], params["3a.bp.b"]]))
+    d = dr.dr_inception_desc(Cin=cin, c3r=c3r, c3=c3, cm=cm, pool_after=0)
+    ws = torch.empty(dr.dr_inception_workspace_bytes(d, B, 28, 28), dtype=torch.uint8, device="cuda")
+    y = torch.full((B, 28, 28, c3 + cm), 768.0, dtype=torch.bfloat16, device="cuda")
+    dr.dr_set_conv_path(dr.DR_PATH_AUTO)
+    dr.dr_inception_slim(d, B, 28, 28, to_dev_bf16(x), [to_dev_bf16(params["3a.3x3r.w"]), to_dev_bf16(params["3a.3x3.w"]), wm],
+                         [to_dev_f32(params["3a.3x3r.b"]), to_dev_f32(params["3a.3x3.b"]), bm], y, ws)
+    assert dr.dr_device_status()[0] == 0
+    got = to_host(y)
+    out = N.run(N.inception_steps(params, "3a", "x"), x)
+    assert_layer_close(got, out["3a"], "3a free-running")
+    # teacher-forced 3x3: fed the reducer output the GPU stored
+    red = to_host(ws[: B * 28 * 28 * c3r * 2].view(torch.bfloat16).reshape(B, 28, 28, c3r))
+    assert_layer_close(red, out["3a.3x3r"], "3a.3x3r")
+    forced = N.run(N.inception_steps(params, "3a", "x"), x, given={"3a.3x3r": red})
+    assert_layer_close(got[..., :c3], forced["3a.3x3"], "3a.3x3 teacher-forced")
+    assert_layer_close(got[..., c3:], forced["3a.m5"], "3a.m5")

@@ -1,0 +1,162 @@
+"""Whole-network GPU parity: slimmed GoogLeNet (batch 1 and 256) and ResNet-50 (batch 128).
+
+Per-layer checks are teacher-forced: the CPU checker's layer l is fed what the GPU stored for
+layer l-1, so each figure measures one layer.  Logits are compared free-running.  At the large
+batches the checker runs a seeded subset of the batch entries (each image is independent through
+every layer), with full per-layer outputs for entry 0.
+"""
+import numpy as np
+import pytest
+
+import dr_synth as S
+import dr_synth.params as P
+from util import LOGITS_L2, assert_layer_close, err_norms, load_params, to_dev_bf16, to_host, _wrap
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dr():
+    import paper_1708_04728_b200 as dr
+    dr.dr_set_conv_path(dr.DR_PATH_AUTO)
+    return dr
+
+
+def run_net(dr, arch, mode, B, params, x_entries_fn, hw=224):
+    """Build, prepare and run a net on the seeded batch; returns (net, workspace, logits, keepalive)."""
+    import torch
+    net = dr.Net(arch, mode, B, hw, hw)
+    keep = []
+    load_params(net, params, keep)
+    ws = torch.empty(net.dr_net_workspace_bytes() + 256, dtype=torch.uint8, device="cuda")
+    off = (-ws.data_ptr()) % 256
+    ws = ws[off:]
+    x = torch.empty((B, hw, hw, 3), dtype=torch.bfloat16, device="cuda")
+    step = 16
+    for n0 in range(0, B, step):
+        x[n0:n0 + step] = to_dev_bf16(x_entries_fn(range(n0, min(B, n0 + step))))
+    logits = torch.full((B, 1000), float("nan"), dtype=torch.float32, device="cuda")
+    net.dr_net_prepare(ws)
+    net.dr_net_forward(x, ws, logits)
+    st, info = dr.dr_device_status()
+    assert st == 0, f"device status {st} {info}"
+    keep += [ws, x]
+    return net, ws, logits, keep
+
+
+def layer_outputs(net, logits, entries):
+    """{layer name: float64 [len(entries),H,W,C]} of the slices the layers wrote, for some batch entries."""
+    import torch
+    out = {}
+    idx = torch.as_tensor(list(entries), device="cuda")
+    for i in range(net.dr_net_num_layers()):
+        li = net.dr_net_layer_info(i)
+        B, H, W, Cc = li["dims"]
+        if li["is_f32"]:
+            out[li["name"]] = to_host(logits[idx]).reshape(len(entries), 1, 1, Cc)
+            continue
+        n_el = (B * H * W - 1) * li["ldc"] + Cc
+        t = torch.as_strided(_wrap(li["ptr"], n_el), (B, H, W, Cc), (H * W * li["ldc"], W * li["ldc"], li["ldc"], 1))
+        out[li["name"]] = to_host(t[idx])
+    return out
+
+
+def check_network(dr, arch, B, entries, steps_fn, params, per_layer_tol=None):
+    import oracle.nets as N
+    images = lambda rng: np.stack([S.normal(0, f"x[{n}]", (224, 224, 3)) for n in rng])
+    net, ws, logits, keep = run_net(dr, arch, dr.DR_MODE_SLIM, B, params, images)
+    paths = {net.dr_net_layer_info(i)["name"]: net.dr_net_layer_info(i)["conv_path"] for i in range(net.dr_net_num_layers())}
+    steps = steps_fn(params)
+    # ---- per layer, teacher-forced, batch entry 0 (+ all checked entries for the logits)
+    G = layer_outputs(net, logits, entries[:1])
+    given = dict(G)
+    for st in steps:                      # concatenated module outputs are re-assembled from their slices
+        if st.virtual:
+            given[st.name] = np.concatenate([given[s] for s in st.src], axis=-1)
+    x0 = images(entries[:1])
+    forced = N.run(steps, x0, given=given)
+    report = []
+    for st in steps:
+        if st.virtual:
+            continue
+        assert st.name in G, f"GPU net has no layer {st.name}"
+        mx, l2 = assert_layer_close(G[st.name], forced[st.name], st.name)
+        report.append((st.name, paths.get(st.name), mx, l2))
+    # ---- end to end, free-running, the seeded subset
+    xs = images(entries)
+    free = N.run(steps, xs)
+    got = to_host(logits[list(entries)]).reshape(len(entries), 1, 1, 1000)
+    assert np.all(np.isfinite(got))
+    for i in range(len(entries)):
+        mx, l2 = err_norms(got[i], free["fc"][i])
+        assert l2 <= LOGITS_L2, f"logits of batch entry {entries[i]}: rel-L2 {l2:.3e} > {LOGITS_L2}"
+    # every batch entry produced something finite
+    assert bool(np.isfinite(to_host(logits)).all())
+    worst = max(report, key=lambda r: r[3])
+    print(f"\n[{['googlenet','resnet50'][arch]} B={B}] worst layer {worst[0]} path={worst[1]} max {worst[2]:.2e} l2 {worst[3]:.2e}; "
+          f"logits rel-L2 {max(err_norms(got[i], free['fc'][i])[1] for i in range(len(entries))):.2e}")
+    return net, logits, free, keep
+
+
+def subset(B, k):
+    """Entry 0 plus the first entries of a seeded permutation."""
+    rest = [int(i) for i in S.stream(0, "subset").permutation(B) if i != 0]
+    return [0] + rest[:k - 1]
+
+
+@pytest.mark.parametrize("B,k", [(1, 1), (256, 4)])
+def test_googlenet_slim(dr, B, k):
+    import oracle.nets as N
+    params = P.googlenet_params(0)
+    check_network(dr, dr.DR_ARCH_GOOGLENET, B, subset(B, k), N.googlenet_steps, params)
+
+
+@pytest.mark.parametrize("B,k", [(128, 2)])
+def test_resnet50_slim(dr, B, k):
+    import oracle.nets as N
+    params = P.resnet50_params(0)
+    check_network(dr, dr.DR_ARCH_RESNET50, B, subset(B, k), N.resnet50_steps, params)
+
+
+@pytest.mark.parametrize("arch", [0, 1])
+def test_unslimmed_path_matches(dr, arch):
+    """The layer-by-layer baseline computes the same function: logits vs the checker and vs the slim net."""
+    import oracle.nets as N
+    B = 2
+    params = P.googlenet_params(0) if arch == 0 else P.resnet50_params(0)
+    steps = (N.googlenet_steps if arch == 0 else N.resnet50_steps)(params)
+    images = lambda rng: np.stack([S.normal(0, f"x[{n}]", (224, 224, 3)) for n in rng])
+    net_u, _, logits_u, keep_u = run_net(dr, arch, dr.DR_MODE_UNSLIMMED, B, params, images)
+    net_s, _, logits_s, keep_s = run_net(dr, arch, dr.DR_MODE_SLIM, B, params, images)
+    free = N.run(steps, images(range(B)))
+    gu, gs = to_host(logits_u), to_host(logits_s)
+    for i in range(B):
+        assert err_norms(gu[i], free["fc"][i].reshape(-1))[1] <= LOGITS_L2
+        assert err_norms(gs[i], free["fc"][i].reshape(-1))[1] <= LOGITS_L2
+        assert err_norms(gu[i], gs[i])[1] <= LOGITS_L2
+    # the baseline launches every non-tensor layer separately
+    n_u = sum(net_u.dr_net_layer_info(i)["kind"] == 1 for i in range(net_u.dr_net_num_layers()))
+    n_s = sum(net_s.dr_net_layer_info(i)["kind"] == 1 for i in range(net_s.dr_net_num_layers()))
+    assert n_u > 10 * n_s
+    # group outputs of the baseline (several bf16 roundings inside one group) stay close to the checker's
+    G = layer_outputs(net_u, logits_u, [0])
+    for name in ("conv1", "conv2", "3a", "5b") if arch == 0 else ("conv1", "res2a.2c", "res5c.2c"):
+        if name in G:
+            mx, l2 = err_norms(G[name], free[name][:1])
+            assert l2 <= 2e-2, (name, l2)
+
+
+def test_net_timing_and_launch_count(dr):
+    params = P.googlenet_params(0)
+    images = lambda rng: np.stack([S.normal(0, f"x[{n}]", (224, 224, 3)) for n in rng])
+    net, ws, logits, keep = run_net(dr, dr.DR_ARCH_GOOGLENET, dr.DR_MODE_SLIM, 1, params, images)
+    x = keep[-1]
+    n0 = dr.dr_launch_count()
+    net.dr_net_set_timing(True)
+    net.dr_net_forward(x, ws, logits)
+    assert dr.dr_launch_count() - n0 == net.dr_net_num_layers()
+    total = sum(net.dr_net_layer_time_us(i) for i in range(net.dr_net_num_layers()))
+    assert total > 0
+    first = to_host(logits).copy()
+    net.dr_net_forward(x, ws, logits)                  # deterministic: no atomics anywhere
+    assert np.array_equal(first, to_host(logits))
