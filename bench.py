@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Throughput of the slimmed GoogLeNet forward pass (images/s) on B200, with its roofline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--batch 256] [--layers-out FILE]
+
+One step = one forward pass of the whole slim network (every slim layer, the two stand-alone
+pools, global average pool and FC) over one batch of synthetic images.  Prints ONE JSON line.
+With N > 1 (under torchrun) every rank runs an independent replica on its own batch (images are
+independent through every layer, so there is no collective on the data path); the time is the
+max over ranks and `value` the images all ranks processed per second.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "slim GoogLeNet forward throughput"
+UNIT = "images/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                       "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush(); self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            # samples under load: the upper half (idle samples before/after the region drag the median down)
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_images_per_s(n_images: int, steps: int = 1):
+    """The CPU checker's GoogLeNet forward, as it stands, on the host cores."""
+    import dr_synth.params as P
+    import oracle
+    import oracle.nets as N
+    oracle.build()
+    params = P.googlenet_params(0)
+    st = N.googlenet_steps(params)
+    x = P.images(0, n_images)
+    times = []
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        N.run(st, x)
+        times.append(time.perf_counter() - t0)
+    return n_images * len(times) / sum(times), oracle.num_threads(), sum(times) / len(times)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n = 4   # images per step: a bounded sample of the batch-256 workload
+    if args.warmup > 0:
+        oracle_images_per_s(1)
+    v, cores, per_step = oracle_images_per_s(n, max(args.steps, 1))
+    sample = f"{n} of {args.batch} images per step, whole network, unfused fp64 checker"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"GoogLeNet-slim forward, batch {args.batch}, 224x224x3 (configs[3])", "sample": sample},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--layers-out", default=None, help="write the per-layer table (us, roofline) as JSON")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # CPU baseline first (rank 0, N = 1 only): before the GPU is busy, ~10-20 s of host work
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        oracle_images_per_s(1)
+        n = 16
+        v, cores, _ = oracle_images_per_s(n)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"{n} of {args.batch} images, whole network, unfused fp64 checker"}
+
+    from paper_1708_04728_b200 import build as _b
+    if rank == 0:
+        _b.build()
+    if world > 1:
+        dist.barrier()
+    import dr_synth as S
+    import dr_synth.params as P
+    import paper_1708_04728_b200 as dr
+
+    B = args.batch
+    pk, pk_kind = peaks()
+    params = P.googlenet_params(0)
+
+    def make_net(mode, batch):
+        net = dr.Net(dr.DR_ARCH_GOOGLENET, mode, batch)
+        keep = []
+        for i in range(net.dr_net_num_params()):
+            name, dims, is_f32, count = net.dr_net_param_spec(i)
+            t = torch.from_numpy(np.ascontiguousarray(params[name], np.float32)).cuda()
+            t = t if is_f32 else t.to(torch.bfloat16)
+            keep.append(t); net.dr_net_set_param(i, t)
+        ws = torch.empty(net.dr_net_workspace_bytes() + 256, dtype=torch.uint8, device="cuda")
+        ws = ws[(-ws.data_ptr()) % 256:]
+        net.dr_net_prepare(ws)
+        return net, ws, keep
+
+    # synthetic N(0,1) images, bf16; per-rank seed so replicas see different data
+    g = S.stream(rank, "bench.x")
+    x_host = torch.from_numpy(S.round_bf16(g.standard_normal((B, 224, 224, 3), dtype=np.float32))).to(torch.bfloat16).pin_memory()
+    x = x_host.cuda()
+    logits = torch.empty((B, 1000), dtype=torch.float32, device="cuda")
+    logits_host = torch.empty((B, 1000), dtype=torch.float32).pin_memory()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > L2 (126 MB)
+    net, ws, keep = make_net(dr.DR_MODE_SLIM, B)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        net.dr_net_forward(x, ws, logits)
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in ev:
+            flush.zero_()                      # L2 flush between timed iterations (outside the event pair)
+            a.record(stream); fn(); b.record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in ev]
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    n0 = dr.dr_launch_count()
+    times = timed(step, args.steps, args.warmup)
+    launches = (dr.dr_launch_count() - n0) * args.steps // (args.steps + args.warmup)
+    st, info = dr.dr_device_status()
+    assert st == 0, f"device status {st} {info}"
+    assert bool(torch.isfinite(logits).all())
+    total_ms = sum(times)
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); total_ms = float(t.item())
+    value = world * B * args.steps / (total_ms * 1e-3)
+
+    # ---- end to end through the public API with host buffers: H2D of the batch, forward, D2H of the logits
+    def e2e_step():
+        x.copy_(x_host, non_blocking=True)
+        net.dr_net_forward(x, ws, logits)
+        logits_host.copy_(logits, non_blocking=True)
+    e2e_times = timed(e2e_step, max(3, args.steps // 2), 2)
+    e2e_ms = sum(e2e_times)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_ms = float(t.item())
+    e2e_value = world * B * len(e2e_times) / (e2e_ms * 1e-3)
+    clocks = sampler.stop() if sampler else None
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- per-layer times (CUDA events around every launch) for the roofline figures
+    net.dr_net_set_timing(True)
+    reps = 5
+    L = net.dr_net_num_layers()
+    infos = [net.dr_net_layer_info(i) for i in range(L)]
+    us = np.zeros((reps, L))
+    for r in range(reps):
+        flush.zero_()
+        step()
+        torch.cuda.synchronize()
+        us[r] = [net.dr_net_layer_time_us(i) for i in range(L)]
+    net.dr_net_set_timing(False)
+    us = np.median(us, axis=0)
+    tf_peak = pk["bf16_tflops_sustained"] * 1e12          # kernels are timed inside a long step
+    bw_peak = pk["hbm_gbs"] * 1e9
+    rows, t_roof_total = [], 0.0
+    for li, t_us in zip(infos, us):
+        t_roof = max(li["flops"] / (pk["bf16_tflops"] * 1e12), li["bytes"] / bw_peak) * 1e6
+        t_roof_total += t_roof
+        rows.append(dict(name=li["name"], kind=li["kind"], path=dr.PATH_NAMES[li["conv_path"]], us=float(t_us),
+                         gflop=li["flops"] / 1e9, mbytes=li["bytes"] / 1e6, roof_us=t_roof, frac=t_roof / max(float(t_us), 1e-9)))
+    tma = [r for r in rows if r["path"] == "umma_tma" and r["gflop"] * 1e9 / (pk["bf16_tflops"] * 1e12) >= r["mbytes"] * 1e6 / bw_peak]
+    tma_flops = sum(r["gflop"] for r in tma) * 1e9
+    tma_s = sum(r["us"] for r in tma) * 1e-6
+    achieved = tma_flops / tma_s / 1e12 if tma_s > 0 else 0.0
+    roofline = {"bound": "tensor", "kernel": "conv_umma_tma_kernel (tensor-bound layers: merged 5x5 and 3x3 convs)",
+                "achieved": achieved, "peak": pk["bf16_tflops_sustained"], "peak_kind": f"{pk_kind} sustained bf16 (kernel timed inside a long step)",
+                "unit": "TFLOP/s", "frac": achieved / pk["bf16_tflops_sustained"], "traffic": None,
+                "launches_per_step": len(tma), "share_of_step": sum(r["us"] for r in tma) / float(us.sum())}
+    ms_per_step = total_ms / args.steps
+    net_roofline = {"sum_layer_roofline_us": t_roof_total, "measured_us": ms_per_step * 1e3,
+                    "frac": t_roof_total / (ms_per_step * 1e3), "peaks": f"{pk_kind}: {pk['bf16_tflops']} TFLOP/s burst, {pk['hbm_gbs']} GB/s"}
+
+    # ---- context numbers: batch 1 latency regime and the unslimmed layer-by-layer path
+    extra = {}
+    try:
+        net_u, ws_u, keep_u = make_net(dr.DR_MODE_UNSLIMMED, B)
+        lu = torch.empty_like(logits)
+        tu = timed(lambda: net_u.dr_net_forward(x, ws_u, lu), 5, 2)
+        extra["unslimmed_images_per_s"] = B * len(tu) / (sum(tu) * 1e-3)
+        extra["slim_speedup_vs_unslimmed"] = value / world / extra["unslimmed_images_per_s"]
+        extra["unslimmed_activation_bytes"] = net_u.dr_net_activation_bytes()
+        extra["slim_activation_bytes"] = net.dr_net_activation_bytes()
+        net_u.dr_net_set_timing(True)
+        net_u.dr_net_forward(x, ws_u, lu); torch.cuda.synchronize()
+        tl = [(net_u.dr_net_layer_info(i)["kind"], net_u.dr_net_layer_time_us(i)) for i in range(net_u.dr_net_num_layers())]
+        extra["unslimmed_pct_latency_non_tensor"] = 100.0 * sum(t for k, t in tl if k == 1) / sum(t for _, t in tl)
+        del net_u, ws_u, keep_u
+        net1, ws1, keep1 = make_net(dr.DR_MODE_SLIM, 1)
+        l1 = torch.empty((1, 1000), dtype=torch.float32, device="cuda")
+        x1 = x[:1].contiguous()
+        t1 = timed(lambda: net1.dr_net_forward(x1, ws1, l1), 20, 5)
+        extra["bs1_images_per_s"] = len(t1) / (sum(t1) * 1e-3)
+        extra["bs1_ms"] = statistics.median(t1)
+    except Exception as e:  # context only; never hides the headline
+        extra["context_error"] = repr(e)
+
+    if args.layers_out:
+        with open(args.layers_out, "w") as f:
+            json.dump({"batch": B, "layers": rows, "net_roofline": net_roofline}, f, indent=1)
+
+    print(json.dumps({
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"GoogLeNet-slim forward, batch {B} per GPU, 224x224x3 N(0,1) bf16, He-normal weights (configs[3])",
+                   "l2": "256 MB buffer written between timed iterations (L2 flush)", "replicas": world},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": logits_host.numel() * 4},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "net_roofline": net_roofline,
+        "cpu_baseline": cpu,
+        "extra": extra,
+    }))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

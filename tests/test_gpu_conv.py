@@ -84,6 +84,13 @@ DIRECT_SHAPES = [
     (1, 17, 13, 16, 16, 3, 2, 1),     # stride-2 3x3
     (2, 10, 10, 3, 64, 7, 2, 3),      # stem geometry, Cin = 3
     (5, 1, 1, 1024, 1000, 1, 1, 0),   # FC shape
+    (2, 28, 28, 192, 128, 5, 1, 2),   # merged 5x5 of 3a
+    (3, 14, 14, 480, 304, 5, 1, 2),   # merged 5x5 of 4a: n-blocks 160 + 144, 32-channel K tail
+    (2, 7, 7, 832, 640, 5, 1, 2),     # merged 5x5 of 5b: three n-blocks, planes smaller than a tile
+    (2, 16, 16, 256, 128, 1, 2, 0),   # ResNet stride-2 1x1 (first conv of a stage)
+    (2, 15, 17, 64, 64, 3, 2, 1),     # stride-2 3x3, odd planes
+    (1, 12, 12, 64, 32, 7, 1, 3),     # 7x7
+    (2, 56, 56, 64, 256, 1, 1, 0),    # ResNet res2 expansion
 ]
 
 
