@@ -154,9 +154,9 @@ def main():
         cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"{n} of {args.batch} images, whole network, unfused fp64 checker"}
 
-    from paper_1708_04728_b200 import build as _b
     if rank == 0:
-        _b.build()
+        import __graft_entry__
+        __graft_entry__.build_cuda()
     if world > 1:
         dist.barrier()
     import dr_synth as S

@@ -1,6 +1,6 @@
 """Build libdeeprebirth.so in-tree with nvcc for sm_100a (no JIT cache, no pip install).
 
-    python -m paper_1708_04728_b200.build [--force] [--verbose]
+    python paper_1708_04728_b200/build.py [--force] [--verbose]
 
 Objects go to ``_build/`` (ignored by git); the shared library lands beside this file so that
 the Python binding, the tests and the benchmark load exactly this build.

@@ -12,6 +12,12 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200)")
 
 
+def pytest_sessionstart(session):
+    # the package refuses to import without its CUDA library: (re)build it in-tree first
+    import __graft_entry__
+    __graft_entry__.build_cuda()
+
+
 @pytest.fixture(scope="session")
 def oracle_lib():
     import oracle

@@ -11,8 +11,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 @pytest.fixture(scope="module")
 def dr():
-    from paper_1708_04728_b200 import build
-    build.build()
+    import __graft_entry__
+    __graft_entry__.build_cuda()
     import paper_1708_04728_b200 as dr
     return dr
 
