@@ -121,6 +121,31 @@ int dr_inception_slim(const dr_inception_desc* desc, int B, int H, int W, const 
                       const void* const w[3], const float* const b[3], void* y, void* workspace,
                       void* stream);
 
+/* dr_inception_slim for callers that cannot hand over scratch memory.  (The paper has no
+ * counterpart: this is a deployment convenience of the library.)
+ *
+ * Who needs it: code that runs where device allocation is off limits — a plug-in executing
+ * inside a host application's latency-critical loop, where cudaMalloc would synchronise the
+ * device and stall every stream; a process whose memory budget was fixed at start-up and whose
+ * allocator is closed afterwards; a component that may only touch the buffers it is handed for
+ * input and output.  Such callers still pass x, the parameters and y, but no workspace: the
+ * 1x1 reducer's output goes to a fixed array of DR_INCEPTION_STATIC_SCRATCH_BYTES inside the
+ * library, which every GPU that loads the library keeps reserved until the process exits.
+ *
+ * Same arithmetic, arguments and errors as dr_inception_slim, plus:
+ *  - B*H*W*c3r*2 bytes (rounded up to 256) must fit the array; a larger request returns
+ *    DR_ERR_WORKSPACE and launches nothing.  Use dr_inception_slim with your own workspace then.
+ *  - The call allocates nothing: no cudaMalloc/cudaFree, no allocating library routine.
+ *  - The first call on each device looks up the array's device address (a host-side query, no
+ *    allocation).  Make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps whatever the last call left in it.
+ *    Nothing needs clearing between calls (the reducer overwrites everything the 3x3 convolution
+ *    reads), but two calls whose kernels may overlap on the GPU — different streams without an
+ *    ordering between them — race on it.  Issue them on one stream or order them with events. */
+#define DR_INCEPTION_STATIC_SCRATCH_BYTES (4u << 20)
+int dr_inception_slim_static(const dr_inception_desc* desc, int B, int H, int W, const void* x,
+                             const void* const w[3], const float* const b[3], void* y, void* stream);
+
 /* ---- stand-alone non-tensor layers (the "unslimmed" baseline, Section 2 / Table 2) -------
  * Each reads its input from and writes its output to device memory: one round trip per
  * layer, which is the cost the slim layers remove.  All tensors dense NHWC bfloat16.       */

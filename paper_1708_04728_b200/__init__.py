@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libdeeprebirth.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
-        f"{LIB_PATH} is missing: build it with `python -m paper_1708_04728_b200.build` "
+        f"{LIB_PATH} is missing: build it with `python paper_1708_04728_b200/build.py` "
         "(there is no CPU or PyTorch fallback)")
 
 _lib = C.CDLL(LIB_PATH)
@@ -67,6 +67,7 @@ _SIGS = {
     "dr_conv_slim": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P]),
     "dr_inception_workspace_bytes": (_I, [C.POINTER(dr_inception_desc), _I, _I, _I, C.POINTER(_Z)]),
     "dr_inception_slim": (_I, [C.POINTER(dr_inception_desc), _I, _I, _I, _P, C.POINTER(_P), C.POINTER(_P), _P, _P, _P]),
+    "dr_inception_slim_static": (_I, [C.POINTER(dr_inception_desc), _I, _I, _I, _P, C.POINTER(_P), C.POINTER(_P), _P, _P]),
     "dr_relu": (_I, [_Z, _P, _P, _P]),
     "dr_maxpool": (_I, [_I, _I, _I, _I, _I, _I, _I, _P, _P, _P, _P]),
     "dr_lrn": (_I, [_I, _I, _I, _I, _I, _F, _F, _F, _P, _P, _P]),
@@ -151,6 +152,18 @@ def dr_inception_slim(desc, B, H, W, x, w, b, y, workspace, stream=None):
     ba = (_P * 3)(*[_ptr(t) for t in b])
     _check(_lib.dr_inception_slim(C.byref(desc), B, H, W, _ptr(x), wa, ba, _ptr(y), _ptr(workspace), _stream(stream)),
            "dr_inception_slim")
+
+
+DR_INCEPTION_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def dr_inception_slim_static(desc, B, H, W, x, w, b, y, stream=None):
+    """dr_inception_slim without a workspace argument: the scratch tensor lives in a fixed array
+    inside the library (see include/dr.h for the size limit and the sharing rules)."""
+    wa = (_P * 3)(*[_ptr(t) for t in w])
+    ba = (_P * 3)(*[_ptr(t) for t in b])
+    _check(_lib.dr_inception_slim_static(C.byref(desc), B, H, W, _ptr(x), wa, ba, _ptr(y), _stream(stream)),
+           "dr_inception_slim_static")
 
 
 def dr_relu(n, x, y, stream=None):

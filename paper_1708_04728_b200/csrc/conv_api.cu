@@ -158,4 +158,37 @@ int dr_inception_slim(const dr_inception_desc* d, int B, int H, int W, const voi
     return dr_conv_slim(&c, B, H, W, x, w[2], b[2], nullptr, y, nullptr, stream);
 }
 
+// ---- dr_inception_slim_static: the same module with its scratch tensor in a fixed device array ----
+// Scratch for the 1x1 reducer's output.  File-scope device storage: every GPU that loads this
+// library reserves these bytes from load until the process exits.  In host code the symbol is only
+// a handle; the address kernels can use comes from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_inception_static_scratch[DR_INCEPTION_STATIC_SCRATCH_BYTES];
+
+static void* inception_static_scratch_ptr(int* status) {
+    static void* ptr[64] = {nullptr};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *status = DR_ERR_CUDA; return nullptr; }
+    if (!ptr[dev]) {
+        void* q = nullptr;
+        if (cudaGetSymbolAddress(&q, g_inception_static_scratch) != cudaSuccess || !q) { *status = DR_ERR_CUDA; return nullptr; }
+        ptr[dev] = q;
+    }
+    *status = DR_OK;
+    return ptr[dev];
+}
+
+int dr_inception_slim_static(const dr_inception_desc* d, int B, int H, int W, const void* x, const void* const w[3],
+                             const float* const b[3], void* y, void* stream) {
+    size_t need = 0;
+    const int st = dr_inception_workspace_bytes(d, B, H, W, &need);
+    if (st != DR_OK) return st;
+    if (need > (size_t)DR_INCEPTION_STATIC_SCRATCH_BYTES) return DR_ERR_WORKSPACE;   // too large for the fixed array
+    int ps = DR_OK;
+    void* scratch = inception_static_scratch_ptr(&ps);
+    if (ps != DR_OK) return ps;
+    // Nothing in the scratch has to start at zero: the reducer writes every element of its
+    // [B,H,W,c3r] output before the 3x3 convolution reads it, so earlier contents never show.
+    return dr_inception_slim(d, B, H, W, x, w, b, y, scratch, stream);
+}
+
 }  // extern "C"
