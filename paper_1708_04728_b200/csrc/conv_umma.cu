@@ -19,6 +19,8 @@
 //
 // Every wait on an mbarrier is bounded (see ptx::mbar_wait); on a timeout the CTA records
 // DR_ERR_DEVICE_TIMEOUT, all roles leave their loops, and TMEM is released before exit.
+#include <cstdlib>
+
 #include "conv_common.cuh"
 #include "umma_ptx.cuh"
 
@@ -277,115 +279,155 @@ int conv_umma_gather_launch(const ConvParams& p, cudaStream_t stream) {
 // =====================================================================================
 //                                     TMA kernel
 // =====================================================================================
-constexpr int T_STAGES = 4;
-constexpr int T_THREADS = 192;   // warp 0: TMA producer, warp 1: MMA issue + TMEM owner, warps 2-5: epilogue
-constexpr int T_SMEM = T_STAGES * STAGE_BYTES + 1024;
-constexpr int T_ACC_COLS = 256;  // columns per accumulator buffer; two buffers = all 512 TMEM columns
+// One template, two launch shapes:
+//   PAIR = false  one CTA per tile of 128 pixels x Nt channels.
+//   PAIR = true   clusters of two CTAs act as one MMA unit (tcgen05 cta_group::2): a pair tile is
+//       256 pixels x Nt channels; each CTA loads its own 128 activation rows and HALF of the filter
+//       tile, the even CTA issues M=256 MMAs that read both shared memories, and each CTA keeps and
+//       drains its own 128 accumulator rows.  Per SM and k-block this moves 16 KB + Nt*64 B through
+//       shared memory instead of 16 KB + Nt*128 B.  TMA loads of both CTAs report to the even CTA's
+//       `full` barrier; the even CTA's commits arrive on `empty` / `tfull` of both CTAs; epilogue
+//       warps of both CTAs arrive on the even CTA's `tempty`.  No multicast loads.
+// The producer and the MMA issuer are single threads whose loop bodies sit on the critical path
+// (a lone thread issues dependent instructions several cycles apart), so both loops are kept to a
+// few dozen instructions: nested tap / channel-block loops instead of divisions, barrier and
+// stage addresses advanced incrementally, descriptors assembled from 32-bit halves.
+constexpr int T_MAX_STAGES = 8;   // stage = A tile (16 KB) + B tile; as many as fit
+constexpr int T_THREADS = 192;    // warp 0: TMA producer, warp 1: MMA issue + TMEM owner, warps 2-5: epilogue
+constexpr int T_SMEM_MAX = 227 * 1024 - 256;
+constexpr int T_ACC_COLS = 256;   // columns per accumulator buffer; two buffers = all 512 TMEM columns
 
 struct TmaShared {
-    uint64_t full[T_STAGES], empty[T_STAGES], tfull[2], tempty[2];
+    uint64_t full[T_MAX_STAGES], empty[T_MAX_STAGES], tfull[2], tempty[2];
     uint32_t tmem_base;
     int abort;
 };
 
 // a_mode 0: activations as a plain [M][Cin] matrix (1x1, stride 1, pad 0): 2-D tiled load.
 // a_mode 1: im2col load.
+template <bool PAIR>
 __global__ void __launch_bounds__(T_THREADS, 1)
-conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const int a_mode) {
+conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const int a_mode,
+                     const int stages, const int stage_bytes) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     __shared__ TmaShared sh;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;        // 0 issues the MMAs
+    const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int nunits = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (tid == 0) {
-        for (int s = 0; s < T_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 4); }
+        for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], PAIR ? 8 : 4); }
         sh.abort = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_a);
         prefetch_tensormap(&map_b);
     }
-    if (warp == 1) { tmem_alloc(&sh.tmem_base, 2 * T_ACC_COLS); tmem_relinquish(); }
+    if (warp == 1) {
+        if (PAIR) { tmem_alloc_pair(&sh.tmem_base, 2 * T_ACC_COLS); tmem_relinquish_pair(); }
+        else { tmem_alloc(&sh.tmem_base, 2 * T_ACC_COLS); tmem_relinquish(); }
+    }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();                               // both CTAs' barriers exist before any remote arrive
     tc_fence_after();
     const uint32_t tmem = sh.tmem_base;
     volatile int* abort_flag = &sh.abort;
 
     const int cpb = (p.Cin + 63) >> 6;
-    const int nkb = p.k * p.k * cpb;
-    const int total = p.m_tiles * p.n_blocks;
+    const int m_units = PAIR ? (p.m_tiles + 1) >> 1 : p.m_tiles;
+    const int total = m_units * p.n_blocks;
     const int cout16 = (p.Cout + 15) & ~15;
-    const uint32_t stage_tx = A_TILE_BYTES + (uint32_t)p.Nt * 128;
     const int hw = p.Ho * p.Wo;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t full0 = smem_u32(&sh.full[0]), empty0 = smem_u32(&sh.empty[0]);
 
     if (warp == 0) {
         if (lane == 0) {
             // -------------------------------------------- TMA producer
-            int g = 0;
-            for (int t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
-                const int nb = t / p.m_tiles, mt = t - nb * p.m_tiles;
+            const uint32_t cta_tx = A_TILE_BYTES + (uint32_t)(PAIR ? p.Nt >> 1 : p.Nt) * 128;
+            const uint32_t full_mask = PAIR ? PEER_BIT_MASK : 0xFFFFFFFFu;   // pair: bytes are reported to the even CTA
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int t = unit; t < total && ok; t += nunits) {
+                const int nb = t / m_units, mu = t - nb * m_units;
                 const int n0 = nb * p.Nt;
+                int mt = PAIR ? 2 * mu + (int)rank : mu;
+                if (mt >= p.m_tiles) mt = p.m_tiles - 1;   // odd tile count: the peer recomputes the last tile, stores nothing
                 const long long m0 = (long long)mt * TILE_M;
                 const int img = (int)(m0 / hw);
                 const int rem = (int)(m0 - (long long)img * hw);
                 const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
                 const int hb = ho * p.stride - p.pad, wb = wo * p.stride - p.pad;
-                for (int kb = 0; kb < nkb; ++kb, ++g) {
-                    const int s = g % T_STAGES, u = g / T_STAGES;
-                    if (!mbar_wait(&sh.empty[s], (u & 1) ^ 1, abort_flag)) {
-                        if (!*abort_flag) report_timeout(p.status, 11, t);
-                        *abort_flag = 1;
-                        break;
-                    }
-                    uint8_t* As = smem + s * STAGE_BYTES;
-                    uint8_t* Bs = As + A_TILE_BYTES;
-                    const int tap = kb / cpb, c0 = (kb - tap * cpb) << 6;
-                    mbar_arrive_expect_tx(&sh.full[s], stage_tx);
-                    if (a_mode == 0) {
-                        tma_load_2d(As, &map_a, &sh.full[s], c0, (int)m0);
-                    } else {
-                        const int r = tap / p.k, tt = tap - r * p.k;
-                        tma_load_im2col_4d(As, &map_a, &sh.full[s], c0, wb, hb, img, (uint16_t)tt, (uint16_t)r);
-                    }
-                    tma_load_3d(Bs, &map_b, &sh.full[s], c0, tap, n0);
-                }
+                const int brow = PAIR ? n0 + (int)rank * (min(p.Nt, cout16 - n0) >> 1) : n0;
+                int tap = 0;
+                for (int r = 0; r < p.k && ok; ++r)
+                    for (int tt = 0; tt < p.k && ok; ++tt, ++tap)
+                        for (int c0 = 0; c0 < p.Cin; c0 += 64) {
+                            if (!mbar_wait_u32(empty0 + 8 * s, ph ^ 1, abort_flag)) {
+                                if (!*abort_flag) report_timeout(p.status, 11, t);
+                                *abort_flag = 1;
+                                ok = false;
+                                break;
+                            }
+                            const uint32_t a_dst = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+                            const uint32_t fb = (full0 + 8 * s) & full_mask;
+                            if (!PAIR) mbar_expect_tx_u32(fb, cta_tx);
+                            else if (rank == 0) mbar_expect_tx_u32(fb, 2 * cta_tx);
+                            if (a_mode == 0) tma_load_2d_u32<PAIR>(a_dst, &map_a, fb, c0, (int)m0);
+                            else tma_load_im2col_4d_u32<PAIR>(a_dst, &map_a, fb, c0, wb, hb, img, (uint16_t)tt, (uint16_t)r);
+                            tma_load_3d_u32<PAIR>(a_dst + A_TILE_BYTES, &map_b, fb, c0, tap, brow);
+                            if (++s == stages) { s = 0; ph ^= 1; }
+                        }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             // -------------------------------------------- MMA issue
-            int g = 0, it = 0;
+            const uint32_t tfull0 = smem_u32(&sh.tfull[0]), tempty0 = smem_u32(&sh.tempty[0]);
+            const int ntaps = p.k * p.k;
+            const int last_nk16 = ((p.Cin - ((cpb - 1) << 6)) + 15) >> 4;
+            int s = 0, it = 0;
+            uint32_t ph = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
-                const int nb = t / p.m_tiles;
+            for (int t = unit; t < total && ok; t += nunits, ++it) {
+                const int nb = t / m_units;
                 const int Nj = min(p.Nt, cout16 - nb * p.Nt);
-                const uint32_t idesc = make_idesc_bf16(TILE_M, Nj);
+                const uint32_t idesc = make_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, Nj);
                 const int acc = it & 1, au = it >> 1;
-                if (!mbar_wait(&sh.tempty[acc], (au & 1) ^ 1, abort_flag)) {
+                if (!mbar_wait_u32(tempty0 + 8 * acc, (au & 1) ^ 1, abort_flag)) {
                     if (!*abort_flag) report_timeout(p.status, 12, t);
                     *abort_flag = 1;
-                    ok = false;
                     break;
                 }
                 tc_fence_after();
                 const uint32_t d = tmem + (uint32_t)(acc * T_ACC_COLS);
-                for (int kb = 0; kb < nkb; ++kb, ++g) {
-                    const int s = g % T_STAGES, u = g / T_STAGES;
-                    if (!mbar_wait(&sh.full[s], u & 1, abort_flag)) {
-                        if (!*abort_flag) report_timeout(p.status, 13, t);
-                        *abort_flag = 1;
-                        ok = false;
-                        break;
+                uint32_t accum = 0;
+                for (int tap = 0; tap < ntaps && ok; ++tap)
+                    for (int cc = 0; cc < cpb; ++cc) {
+                        if (!mbar_wait_u32(full0 + 8 * s, ph, abort_flag)) {
+                            if (!*abort_flag) report_timeout(p.status, 13, t);
+                            *abort_flag = 1;
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t a = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+                        const uint32_t alo = sdesc_lo(a), blo = sdesc_lo(a + A_TILE_BYTES);
+                        const int nk16 = (cc == cpb - 1) ? last_nk16 : 4;
+                        umma_bf16_lo<PAIR>(d, alo, blo, idesc, accum);
+                        accum = 1;
+                        if (nk16 > 1) umma_bf16_lo<PAIR>(d, alo + 2, blo + 2, idesc, 1u);
+                        if (nk16 > 2) umma_bf16_lo<PAIR>(d, alo + 4, blo + 4, idesc, 1u);
+                        if (nk16 > 3) umma_bf16_lo<PAIR>(d, alo + 6, blo + 6, idesc, 1u);
+                        umma_commit_u32<PAIR>(empty0 + 8 * s);
+                        if (++s == stages) { s = 0; ph ^= 1; }
                     }
-                    tc_fence_after();
-                    const int valid = min(64, p.Cin - ((kb % cpb) << 6));
-                    const uint32_t a = smem_u32(smem + s * STAGE_BYTES);
-                    issue_kblock(d, a, a + A_TILE_BYTES, idesc, (valid + 15) >> 4, kb == 0);
-                    umma_commit(&sh.empty[s]);
-                }
-                if (ok) umma_commit(&sh.tfull[acc]);
+                if (ok) umma_commit_u32<PAIR>(tfull0 + 8 * acc);
             }
         }
         __syncwarp();
@@ -394,10 +436,11 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
         const int q = warp & 3;
         const int row = q * 32 + lane;
         int it = 0;
-        for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
-            const int nb = t / p.m_tiles, mt = t - nb * p.m_tiles;
+        for (int t = unit; t < total; t += nunits, ++it) {
+            const int nb = t / m_units, mu = t - nb * m_units;
             const int n0 = nb * p.Nt;
             const int Nj = min(p.Nt, cout16 - n0);
+            const int mt = PAIR ? 2 * mu + (int)rank : mu;
             const int acc = it & 1, au = it >> 1;
             const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[acc], au & 1, abort_flag));
             if (!ok) {
@@ -407,20 +450,27 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             }
             tc_fence_after();
             const long long m = (long long)mt * TILE_M + row;
-            drain_direct(p, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * T_ACC_COLS), Nj, m, m < p.M, n0);
+            drain_direct(p, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * T_ACC_COLS), Nj, m, mt < p.m_tiles && m < p.M, n0);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.tempty[acc]);
+            if (lane == 0) {
+                if (PAIR) mbar_arrive_leader(&sh.tempty[acc]);
+                else mbar_arrive(&sh.tempty[acc]);
+            }
         }
     }
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {   // give copies and MMAs still in flight time to land before shared memory and TMEM go away
-        const uint64_t t0 = globaltimer_ns();
-        while (globaltimer_ns() - t0 < 200000ull) {}
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) {}
         __syncthreads();
     }
-    if (warp == 1) tmem_dealloc(tmem, 2 * T_ACC_COLS);
+    if (PAIR) cluster_sync_all();                               // neither CTA leaves while the other may still signal it
+    if (warp == 1) {
+        if (PAIR) tmem_dealloc_pair(tmem, 2 * T_ACC_COLS);
+        else tmem_dealloc(tmem, 2 * T_ACC_COLS);
+    }
 }
 
 // ---- host: tensor maps ------------------------------------------------------------------
@@ -445,6 +495,12 @@ static bool load_encoders() {
     return true;
 }
 
+// Integer tunable from the environment (read once per name at first use); for A/B timing.
+static int tunable(const char* name, int dflt) {
+    const char* v = getenv(name);
+    return v ? atoi(v) : dflt;
+}
+
 bool conv_umma_tma_supports(const ConvParams& p) {
     if (p.flags & (DR_POOL | DR_LRN)) return false;   // staged epilogues live in the gather kernel
     if (p.patch) return false;
@@ -455,16 +511,49 @@ bool conv_umma_tma_supports(const ConvParams& p) {
     return true;
 }
 
+static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, int a_mode, cudaStream_t stream) {
+    static bool attr_set = false;
+    static int max_clusters = 0;
+    const int stage_bytes = A_TILE_BYTES + ((p.Nt * 64 + 1023) & ~1023);
+    int stages = (T_SMEM_MAX - 1024) / stage_bytes;
+    if (stages > T_MAX_STAGES) stages = T_MAX_STAGES;
+    int smem_bytes = stages * stage_bytes + 1024;
+    if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(T_THREADS); cfg.dynamicSmemBytes = (size_t)smem_bytes; cfg.stream = stream;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(conv_umma_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+        cfg.gridDim = dim3(2 * num_sms());
+        cfg.dynamicSmemBytes = (size_t)T_SMEM_MAX;
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, conv_umma_tma_kernel<true>, &cfg) != cudaSuccess || max_clusters < 1) return DR_ERR_CUDA;
+        cfg.dynamicSmemBytes = (size_t)smem_bytes;
+        attr_set = true;
+    }
+    const int pair_tiles = ((p.m_tiles + 1) / 2) * p.n_blocks;
+    const int pairs = pair_tiles < max_clusters ? pair_tiles : max_clusters;
+    cfg.gridDim = dim3(2 * pairs);
+    if (cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true>, p, map_a, map_b, a_mode, stages, stage_bytes) != cudaSuccess) return DR_ERR_CUDA;
+    count_launch();
+    return launch_status();
+}
+
 int conv_umma_tma_launch(const ConvParams& p, cudaStream_t stream) {
     if (!conv_umma_tma_supports(p)) return DR_ERR_UNSUPPORTED;
     if (!load_encoders()) return DR_ERR_CUDA;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(conv_umma_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM) != cudaSuccess) return DR_ERR_CUDA;
+        if (cudaFuncSetAttribute(conv_umma_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
         attr_set = true;
     }
     alignas(64) CUtensorMap map_a, map_b;
     const int a_mode = (p.k == 1 && p.stride == 1 && p.pad == 0) ? 0 : 1;
+    // CTA pairs pay off where the MMAs dominate (long K, several tiles per SM pair)
+    const int pair_pref = tunable("DR_TMA_PAIR", -1);
+    const bool use_pair = pair_pref >= 0 ? pair_pref != 0 : (p.K >= 1024 && p.m_tiles >= 2);
     if (a_mode == 0) {
         const cuuint64_t dims[2] = {(cuuint64_t)p.Cin, (cuuint64_t)p.M};
         const cuuint64_t strides[1] = {(cuuint64_t)p.Cin * 2};
@@ -488,7 +577,7 @@ int conv_umma_tma_launch(const ConvParams& p, cudaStream_t stream) {
     {
         const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
         const cuuint64_t strides[2] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.K * 2};
-        const cuuint32_t box[3] = {64, 1, (cuuint32_t)p.Nt};
+        const cuuint32_t box[3] = {64, 1, (cuuint32_t)(use_pair ? p.Nt / 2 : p.Nt)};   // a pair's CTAs load half each
         const cuuint32_t es[3] = {1, 1, 1};
         if (g_encode_tiled(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)p.w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -496,8 +585,18 @@ int conv_umma_tma_launch(const ConvParams& p, cudaStream_t stream) {
     }
     const int total = p.m_tiles * p.n_blocks;
     if (total <= 0) return DR_OK;
+    if (use_pair) return launch_pair(p, map_a, map_b, a_mode, stream);
     const int grid = total < num_sms() ? total : num_sms();
-    conv_umma_tma_kernel<<<grid, T_THREADS, T_SMEM, stream>>>(p, map_a, map_b, a_mode);
+    // as many pipeline stages as shared memory holds (the B tile shrinks with Nt); always more than
+    // half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
+    const int stage_bytes = A_TILE_BYTES + ((p.Nt * 128 + 1023) & ~1023);
+    int stages = (T_SMEM_MAX - 1024) / stage_bytes;
+    if (stages > T_MAX_STAGES) stages = T_MAX_STAGES;
+    const int forced = tunable("DR_TMA_STAGES", 0);
+    if (forced >= 2 && forced < stages) stages = forced;
+    int smem_bytes = stages * stage_bytes + 1024;
+    if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
+    conv_umma_tma_kernel<false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, stage_bytes);
     count_launch();
     return launch_status();
 }
