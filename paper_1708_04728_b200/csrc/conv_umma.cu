@@ -305,14 +305,18 @@ struct TmaShared {
 
 // a_mode 0: activations as a plain [M][Cin] matrix (1x1, stride 1, pad 0): 2-D tiled load.
 // a_mode 1: im2col load.
-template <bool PAIR>
+template <bool PAIR, int KPB>
 __global__ void __launch_bounds__(T_THREADS, 1)
 conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const int a_mode,
-                     const int stages, const int stage_bytes) {
+                     const int stages, const int sub_bytes) {
+    constexpr int kpb = KPB;
+    // a pipeline stage holds `kpb` k-blocks (sub-stages of sub_bytes = A tile + B tile): one barrier
+    // round trip then covers kpb * 4 MMAs, which keeps the issuing thread ahead of the tensor pipe
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     __shared__ TmaShared sh;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int stage_bytes = kpb * sub_bytes;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;        // 0 issues the MMAs
     const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int nunits = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
@@ -337,6 +341,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
     volatile int* abort_flag = &sh.abort;
 
     const int cpb = (p.Cin + 63) >> 6;
+    const int nkb = p.k * p.k * cpb;
     const int m_units = PAIR ? (p.m_tiles + 1) >> 1 : p.m_tiles;
     const int total = m_units * p.n_blocks;
     const int cout16 = (p.Cout + 15) & ~15;
@@ -352,6 +357,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
+            uint32_t ready = mbar_test_u32(empty0, 1);
             for (int t = unit; t < total && ok; t += nunits) {
                 const int nb = t / m_units, mu = t - nb * m_units;
                 const int n0 = nb * p.Nt;
@@ -363,25 +369,42 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                 const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
                 const int hb = ho * p.stride - p.pad, wb = wo * p.stride - p.pad;
                 const int brow = PAIR ? n0 + (int)rank * (min(p.Nt, cout16 - n0) >> 1) : n0;
-                int tap = 0;
-                for (int r = 0; r < p.k && ok; ++r)
-                    for (int tt = 0; tt < p.k && ok; ++tt, ++tap)
-                        for (int c0 = 0; c0 < p.Cin; c0 += 64) {
-                            if (!mbar_wait_u32(empty0 + 8 * s, ph ^ 1, abort_flag)) {
-                                if (!*abort_flag) report_timeout(p.status, 11, t);
-                                *abort_flag = 1;
-                                ok = false;
-                                break;
-                            }
-                            const uint32_t a_dst = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
-                            const uint32_t fb = (full0 + 8 * s) & full_mask;
-                            if (!PAIR) mbar_expect_tx_u32(fb, cta_tx);
-                            else if (rank == 0) mbar_expect_tx_u32(fb, 2 * cta_tx);
-                            if (a_mode == 0) tma_load_2d_u32<PAIR>(a_dst, &map_a, fb, c0, (int)m0);
-                            else tma_load_im2col_4d_u32<PAIR>(a_dst, &map_a, fb, c0, wb, hb, img, (uint16_t)tt, (uint16_t)r);
-                            tma_load_3d_u32<PAIR>(a_dst + A_TILE_BYTES, &map_b, fb, c0, tap, brow);
-                            if (++s == stages) { s = 0; ph ^= 1; }
-                        }
+                int r = 0, tt = 0, tap = 0, c0 = 0;
+                for (int remaining = nkb; remaining > 0;) {
+                    const int nk = remaining < kpb ? remaining : kpb;
+                    if (!ready && !mbar_wait_slow_u32(empty0 + 8 * s, ph ^ 1, abort_flag)) {
+                        if (!*abort_flag) report_timeout(p.status, 11, t);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    int s2 = s + 1;
+                    uint32_t ph2 = ph;
+                    if (s2 == stages) { s2 = 0; ph2 ^= 1; }
+                    ready = mbar_test_u32(empty0 + 8 * s2, ph2 ^ 1);      // probe the next slot while this one is filled
+                    uint32_t a_dst = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+                    const uint32_t fb = (full0 + 8 * s) & full_mask;
+                    if (!PAIR) mbar_expect_tx_u32(fb, (uint32_t)nk * cta_tx);
+                    else if (rank == 0) mbar_expect_tx_u32(fb, 2u * (uint32_t)nk * cta_tx);
+#pragma unroll
+                    for (int j = 0; j < KPB; ++j, a_dst += (uint32_t)sub_bytes) {
+                        const uint32_t en = j < nk ? 1u : 0u;
+                        if (a_mode == 0) tma_load_2d_u32<PAIR>(a_dst, &map_a, fb, c0, (int)m0, en);
+                        else tma_load_im2col_4d_u32<PAIR>(a_dst, &map_a, fb, c0, wb, hb, img, (uint16_t)tt, (uint16_t)r, en);
+                        tma_load_3d_u32<PAIR>(a_dst + A_TILE_BYTES, &map_b, fb, c0, tap, brow, en);
+                        c0 += 64;
+                        const bool wrap_c = c0 >= p.Cin;
+                        c0 = wrap_c ? 0 : c0;
+                        tap += wrap_c ? 1 : 0;
+                        tt += wrap_c ? 1 : 0;
+                        const bool wrap_t = tt == p.k;
+                        tt = wrap_t ? 0 : tt;
+                        r += wrap_t ? 1 : 0;
+                    }
+                    remaining -= nk;
+                    s = s2;
+                    ph = ph2;
+                }
             }
         }
         __syncwarp();
@@ -389,11 +412,11 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
         if (lane == 0 && rank == 0) {
             // -------------------------------------------- MMA issue
             const uint32_t tfull0 = smem_u32(&sh.tfull[0]), tempty0 = smem_u32(&sh.tempty[0]);
-            const int ntaps = p.k * p.k;
             const int last_nk16 = ((p.Cin - ((cpb - 1) << 6)) + 15) >> 4;
             int s = 0, it = 0;
             uint32_t ph = 0;
             bool ok = true;
+            uint32_t ready = mbar_test_u32(full0, 0);
             for (int t = unit; t < total && ok; t += nunits, ++it) {
                 const int nb = t / m_units;
                 const int Nj = min(p.Nt, cout16 - nb * p.Nt);
@@ -407,26 +430,37 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                 tc_fence_after();
                 const uint32_t d = tmem + (uint32_t)(acc * T_ACC_COLS);
                 uint32_t accum = 0;
-                for (int tap = 0; tap < ntaps && ok; ++tap)
-                    for (int cc = 0; cc < cpb; ++cc) {
-                        if (!mbar_wait_u32(full0 + 8 * s, ph, abort_flag)) {
-                            if (!*abort_flag) report_timeout(p.status, 13, t);
-                            *abort_flag = 1;
-                            ok = false;
-                            break;
-                        }
-                        tc_fence_after();
-                        const uint32_t a = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
-                        const uint32_t alo = sdesc_lo(a), blo = sdesc_lo(a + A_TILE_BYTES);
-                        const int nk16 = (cc == cpb - 1) ? last_nk16 : 4;
-                        umma_bf16_lo<PAIR>(d, alo, blo, idesc, accum);
-                        accum = 1;
-                        if (nk16 > 1) umma_bf16_lo<PAIR>(d, alo + 2, blo + 2, idesc, 1u);
-                        if (nk16 > 2) umma_bf16_lo<PAIR>(d, alo + 4, blo + 4, idesc, 1u);
-                        if (nk16 > 3) umma_bf16_lo<PAIR>(d, alo + 6, blo + 6, idesc, 1u);
-                        umma_commit_u32<PAIR>(empty0 + 8 * s);
-                        if (++s == stages) { s = 0; ph ^= 1; }
+                int cc = 0;
+                for (int remaining = nkb; remaining > 0;) {
+                    const int nk = remaining < kpb ? remaining : kpb;
+                    if (!ready && !mbar_wait_slow_u32(full0 + 8 * s, ph, abort_flag)) {
+                        if (!*abort_flag) report_timeout(p.status, 13, t);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
                     }
+                    int s2 = s + 1;
+                    uint32_t ph2 = ph;
+                    if (s2 == stages) { s2 = 0; ph2 ^= 1; }
+                    ready = mbar_test_u32(full0 + 8 * s2, ph2);               // probe the next slot while this one is issued
+                    tc_fence_after();
+                    uint32_t a = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+#pragma unroll
+                    for (int j = 0; j < KPB; ++j, a += (uint32_t)sub_bytes) {
+                        const uint32_t alo = sdesc_lo(a), blo = sdesc_lo(a + A_TILE_BYTES);
+                        const int nk16 = j < nk ? ((cc == cpb - 1) ? last_nk16 : 4) : 0;    // 0: nothing in this sub-stage
+                        cc = (cc + 1 == cpb) ? 0 : cc + 1;
+                        umma_bf16_lo<PAIR>(d, alo, blo, idesc, accum, nk16 > 0);
+                        accum = 1;
+                        umma_bf16_lo<PAIR>(d, alo + 2, blo + 2, idesc, 1u, nk16 > 1);
+                        umma_bf16_lo<PAIR>(d, alo + 4, blo + 4, idesc, 1u, nk16 > 2);
+                        umma_bf16_lo<PAIR>(d, alo + 6, blo + 6, idesc, 1u, nk16 > 3);
+                    }
+                    umma_commit_u32<PAIR>(empty0 + 8 * s);
+                    remaining -= nk;
+                    s = s2;
+                    ph = ph2;
+                }
                 if (ok) umma_commit_u32<PAIR>(tfull0 + 8 * acc);
             }
         }
@@ -511,13 +545,30 @@ bool conv_umma_tma_supports(const ConvParams& p) {
     return true;
 }
 
+// Pipeline shape: k-blocks per stage (kpb) and number of stages.  Measured on B200: wide tiles
+// (Nt >= 208) run best with one k-block per barrier round trip, narrower ones with two (their MMAs
+// are short, so the round trip has to cover more of them); never more than the layer has.
+static void pick_pipeline(int sub_bytes, int nkb, int nt, int* kpb, int* stages) {
+    const int budget = T_SMEM_MAX - 1024;
+    int k = tunable("DR_TMA_KPB", 0);
+    if (k <= 0) k = nt >= 208 ? 1 : 2;
+    if (k >= 4) k = 4; else if (k == 3) k = 2;          // instantiated: 1, 2, 4
+    while (k > 1 && (k > nkb || budget / (k * sub_bytes) < 2)) k >>= 1;
+    int st = budget / (k * sub_bytes);
+    if (st > T_MAX_STAGES) st = T_MAX_STAGES;
+    const int forced = tunable("DR_TMA_STAGES", 0);
+    if (forced >= 2 && forced < st) st = forced;
+    *kpb = k;
+    *stages = st;
+}
+
 static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, int a_mode, cudaStream_t stream) {
     static bool attr_set = false;
     static int max_clusters = 0;
-    const int stage_bytes = A_TILE_BYTES + ((p.Nt * 64 + 1023) & ~1023);
-    int stages = (T_SMEM_MAX - 1024) / stage_bytes;
-    if (stages > T_MAX_STAGES) stages = T_MAX_STAGES;
-    int smem_bytes = stages * stage_bytes + 1024;
+    const int sub_bytes = A_TILE_BYTES + ((p.Nt * 64 + 1023) & ~1023);
+    int kpb, stages;
+    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), p.Nt, &kpb, &stages);
+    int smem_bytes = stages * kpb * sub_bytes + 1024;
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -526,17 +577,24 @@ static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUte
     cfg.blockDim = dim3(T_THREADS); cfg.dynamicSmemBytes = (size_t)smem_bytes; cfg.stream = stream;
     cfg.attrs = attr; cfg.numAttrs = 1;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(conv_umma_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+        if (cudaFuncSetAttribute(conv_umma_tma_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_umma_tma_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_umma_tma_kernel<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess)
+            return DR_ERR_CUDA;
         cfg.gridDim = dim3(2 * num_sms());
         cfg.dynamicSmemBytes = (size_t)T_SMEM_MAX;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, conv_umma_tma_kernel<true>, &cfg) != cudaSuccess || max_clusters < 1) return DR_ERR_CUDA;
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, conv_umma_tma_kernel<true, 1>, &cfg) != cudaSuccess || max_clusters < 1) return DR_ERR_CUDA;
         cfg.dynamicSmemBytes = (size_t)smem_bytes;
         attr_set = true;
     }
     const int pair_tiles = ((p.m_tiles + 1) / 2) * p.n_blocks;
     const int pairs = pair_tiles < max_clusters ? pair_tiles : max_clusters;
     cfg.gridDim = dim3(2 * pairs);
-    if (cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true>, p, map_a, map_b, a_mode, stages, stage_bytes) != cudaSuccess) return DR_ERR_CUDA;
+    cudaError_t e;
+    if (kpb == 4) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 4>, p, map_a, map_b, a_mode, stages, sub_bytes);
+    else if (kpb == 2) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 2>, p, map_a, map_b, a_mode, stages, sub_bytes);
+    else e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 1>, p, map_a, map_b, a_mode, stages, sub_bytes);
+    if (e != cudaSuccess) return DR_ERR_CUDA;
     count_launch();
     return launch_status();
 }
@@ -546,7 +604,10 @@ int conv_umma_tma_launch(const ConvParams& p, cudaStream_t stream) {
     if (!load_encoders()) return DR_ERR_CUDA;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(conv_umma_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+        if (cudaFuncSetAttribute(conv_umma_tma_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_umma_tma_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_umma_tma_kernel<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess)
+            return DR_ERR_CUDA;
         attr_set = true;
     }
     alignas(64) CUtensorMap map_a, map_b;
@@ -589,14 +650,14 @@ int conv_umma_tma_launch(const ConvParams& p, cudaStream_t stream) {
     const int grid = total < num_sms() ? total : num_sms();
     // as many pipeline stages as shared memory holds (the B tile shrinks with Nt); always more than
     // half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
-    const int stage_bytes = A_TILE_BYTES + ((p.Nt * 128 + 1023) & ~1023);
-    int stages = (T_SMEM_MAX - 1024) / stage_bytes;
-    if (stages > T_MAX_STAGES) stages = T_MAX_STAGES;
-    const int forced = tunable("DR_TMA_STAGES", 0);
-    if (forced >= 2 && forced < stages) stages = forced;
-    int smem_bytes = stages * stage_bytes + 1024;
+    const int sub_bytes = A_TILE_BYTES + ((p.Nt * 128 + 1023) & ~1023);
+    int kpb, stages;
+    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), p.Nt, &kpb, &stages);
+    int smem_bytes = stages * kpb * sub_bytes + 1024;
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
-    conv_umma_tma_kernel<false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, stage_bytes);
+    if (kpb == 4) conv_umma_tma_kernel<false, 4><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
+    else if (kpb == 2) conv_umma_tma_kernel<false, 2><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
+    else conv_umma_tma_kernel<false, 1><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
     count_launch();
     return launch_status();
 }

@@ -241,6 +241,21 @@ __device__ __forceinline__ bool mbar_try_wait_u32(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+// non-blocking probe: lets a loop ask about the NEXT barrier before it issues this step's work, so the
+// round trip to the barrier overlaps that work instead of stalling the lone issuing thread
+__device__ __forceinline__ uint32_t mbar_test_u32(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
 __device__ __noinline__ bool mbar_wait_slow_u32(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     const long long t0 = clock64();
     for (;;) {
@@ -259,73 +274,87 @@ __device__ __forceinline__ bool mbar_wait_u32(uint32_t bar, uint32_t parity, vol
 __device__ __forceinline__ void mbar_expect_tx_u32(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// The loads and MMAs below take an `enable` flag and are predicated in PTX, so a loop that
+// sometimes has nothing to issue (a partial stage, a K tail) stays free of branches.
 template <bool PAIR>
-__device__ __forceinline__ void tma_load_2d_u32(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-    if (PAIR)
-        asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-                     "l"(map), "r"(bar), "r"(c0), "r"(c1)
-                     : "memory");
-    else
-        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-                     "l"(map), "r"(bar), "r"(c0), "r"(c1)
-                     : "memory");
-}
-template <bool PAIR>
-__device__ __forceinline__ void tma_load_3d_u32(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
-    if (PAIR)
-        asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(
-                         dst),
-                     "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
-                     : "memory");
-    else
-        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
-                     "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
-                     : "memory");
-}
-template <bool PAIR>
-__device__ __forceinline__ void tma_load_im2col_4d_u32(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c, int w, int h, int n,
-                                                       uint16_t woff, uint16_t hoff) {
+__device__ __forceinline__ void tma_load_2d_u32(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, uint32_t enable) {
     if (PAIR)
         asm volatile(
-            "cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};" ::"r"(
-                dst),
-            "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(woff), "h"(hoff)
+            "{\n.reg .pred q;\nsetp.ne.b32 q, %5, 0;\n"
+            "@q cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n}\n" ::"r"(dst),
+            "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(enable)
             : "memory");
     else
         asm volatile(
-            "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};" ::"r"(
+            "{\n.reg .pred q;\nsetp.ne.b32 q, %5, 0;\n"
+            "@q cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n}\n" ::"r"(dst),
+            "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(enable)
+            : "memory");
+}
+template <bool PAIR>
+__device__ __forceinline__ void tma_load_3d_u32(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, uint32_t enable) {
+    if (PAIR)
+        asm volatile(
+            "{\n.reg .pred q;\nsetp.ne.b32 q, %6, 0;\n"
+            "@q cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n}\n" ::"r"(
                 dst),
-            "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(woff), "h"(hoff)
+            "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(enable)
+            : "memory");
+    else
+        asm volatile(
+            "{\n.reg .pred q;\nsetp.ne.b32 q, %6, 0;\n"
+            "@q cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n}\n" ::"r"(dst),
+            "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(enable)
+            : "memory");
+}
+template <bool PAIR>
+__device__ __forceinline__ void tma_load_im2col_4d_u32(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c, int w, int h, int n,
+                                                       uint16_t woff, uint16_t hoff, uint32_t enable) {
+    if (PAIR)
+        asm volatile(
+            "{\n.reg .pred q;\nsetp.ne.b32 q, %9, 0;\n"
+            "@q cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};\n}\n" ::"r"(
+                dst),
+            "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(woff), "h"(hoff), "r"(enable)
+            : "memory");
+    else
+        asm volatile(
+            "{\n.reg .pred q;\nsetp.ne.b32 q, %9, 0;\n"
+            "@q cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};\n}\n" ::"r"(
+                dst),
+            "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(woff), "h"(hoff), "r"(enable)
             : "memory");
 }
 // low word of make_sdesc_sw128 (start address + the unused leading offset); the high word is constant
 __device__ __forceinline__ uint32_t sdesc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | 0x10000u; }
 constexpr uint32_t SDESC_HI_SW128 = (1024u >> 4) | (1u << 14) | (2u << 29);
 template <bool PAIR>
-__device__ __forceinline__ void umma_bf16_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void umma_bf16_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate, uint32_t enable) {
     if (PAIR)
         asm volatile(
             "{\n"
-            ".reg .pred p;\n"
+            ".reg .pred p, q;\n"
             ".reg .b64 da, db;\n"
             "mov.b64 da, {%1, %5};\n"
             "mov.b64 db, {%2, %5};\n"
             "setp.ne.b32 p, %4, 0;\n"
-            "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n"
+            "setp.ne.b32 q, %6, 0;\n"
+            "@q tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n"
             "}\n" ::"r"(d_tmem),
-            "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(SDESC_HI_SW128)
+            "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(SDESC_HI_SW128), "r"(enable)
             : "memory");
     else
         asm volatile(
             "{\n"
-            ".reg .pred p;\n"
+            ".reg .pred p, q;\n"
             ".reg .b64 da, db;\n"
             "mov.b64 da, {%1, %5};\n"
             "mov.b64 db, {%2, %5};\n"
             "setp.ne.b32 p, %4, 0;\n"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n"
+            "setp.ne.b32 q, %6, 0;\n"
+            "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n"
             "}\n" ::"r"(d_tmem),
-            "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(SDESC_HI_SW128)
+            "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(SDESC_HI_SW128), "r"(enable)
             : "memory");
 }
 template <bool PAIR>
