@@ -226,6 +226,8 @@ int dr_net_activation_bytes(const dr_net* net, size_t* bytes);
 #define DR_PATH_SIMT         1  /* CUDA-core implicit GEMM: any shape, slow                      */
 #define DR_PATH_UMMA_GATHER  2  /* tcgen05 MMA, operands gathered by producer warps              */
 #define DR_PATH_UMMA_TMA     3  /* tcgen05 MMA, operands loaded by TMA (im2col / tiled)          */
+#define DR_PATH_UMMA_PATCH   4  /* pooling layers: 2-D output patches, TMA box loads, fused pool/LRN */
+#define DR_PATH_UMMA_STEM    5  /* the 7x7/2 3-channel stem with fused pool/LRN                  */
 /* Force a convolution kernel (tests, A/B timing); DR_PATH_AUTO picks the fastest that
  * supports the layer.  A forced path that cannot run the layer gives DR_ERR_UNSUPPORTED.   */
 int dr_set_conv_path(int path);

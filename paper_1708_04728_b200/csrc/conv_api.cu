@@ -85,6 +85,10 @@ int conv_pick_path(const ConvParams& p, int forced) {
     if (forced == DR_PATH_SIMT) return DR_PATH_SIMT;
     if (forced == DR_PATH_UMMA_GATHER) return conv_umma_gather_supports(p) ? DR_PATH_UMMA_GATHER : -1;
     if (forced == DR_PATH_UMMA_TMA) return conv_umma_tma_supports(p) ? DR_PATH_UMMA_TMA : -1;
+    if (forced == DR_PATH_UMMA_PATCH) return conv_patch_tma_supports(p) ? DR_PATH_UMMA_PATCH : -1;
+    if (forced == DR_PATH_UMMA_STEM) return conv_stem_supports(p) ? DR_PATH_UMMA_STEM : -1;
+    if (conv_stem_supports(p)) return DR_PATH_UMMA_STEM;
+    if (conv_patch_tma_supports(p)) return DR_PATH_UMMA_PATCH;
     if (conv_umma_tma_supports(p)) return DR_PATH_UMMA_TMA;
     if (conv_umma_gather_supports(p)) return DR_PATH_UMMA_GATHER;
     return DR_PATH_SIMT;
@@ -95,6 +99,8 @@ int conv_launch_path(const ConvParams& p, int path, cudaStream_t stream) {
         case DR_PATH_SIMT: return conv_simt_launch(p, stream);
         case DR_PATH_UMMA_GATHER: return conv_umma_gather_launch(p, stream);
         case DR_PATH_UMMA_TMA: return conv_umma_tma_launch(p, stream);
+        case DR_PATH_UMMA_PATCH: return conv_patch_tma_launch(p, stream);
+        case DR_PATH_UMMA_STEM: return conv_stem_launch(p, stream);
         default: return DR_ERR_UNSUPPORTED;
     }
 }
@@ -108,7 +114,7 @@ using namespace dr;
 extern "C" {
 
 int dr_set_conv_path(int path) {
-    if (path < DR_PATH_AUTO || path > DR_PATH_UMMA_TMA) return DR_ERR_INVALID_ARG;
+    if (path < DR_PATH_AUTO || path > DR_PATH_UMMA_STEM) return DR_ERR_INVALID_ARG;
     g_forced_path = path;
     return DR_OK;
 }

@@ -1,0 +1,455 @@
+// Patch-tiled convolution kernels for the slim layers whose epilogue max-pools (and optionally
+// LRN-normalises): a tile is the (2*PH+1) x (2*PW+1) patch of convolution outputs that PH x PW pooled
+// outputs need (the first row / column is a halo the neighbouring tile recomputes), so the pooled
+// tensor is the only thing written to HBM.  Both kernels are persistent (one CTA per SM), use
+// tcgen05 MMAs with two TMEM accumulator buffers, and share conv_fused_epilogue.cuh.
+//
+//   conv_patch_tma_kernel   stride-1 layers with Cin a multiple of 8 (GoogLeNet conv2/3x3): the
+//       activation patch of one filter tap is ONE tiled 4-D TMA box (64 channels x patch width x patch
+//       height), zero-filled outside the image; filters stream through TMA as in the main kernel.
+//   conv_stem_kernel        the 7x7 / stride-2 / 3-channel stem (GoogLeNet and ResNet conv1).  TMA
+//       cannot address 6-byte pixels, so four producer warps bring the input patch into shared memory
+//       with 4-byte cp.async (next tile's patch in flight while this one is used) and build the im2col
+//       tile from there.  K is laid out as 7 tap-rows x 24 slots (21 = 7 taps x 3 channels used, 3 slots
+//       and the tail up to 192 carry zero weights), which makes every tap-row a 48-byte run that starts
+//       4-byte aligned in the patch and 16-byte aligned in the operand tile.  The 64 x 192 filter tile is
+//       built once per CTA and stays resident.
+#include <cstdlib>
+
+#include "conv_common.cuh"
+#include "conv_fused_epilogue.cuh"
+#include "umma_ptx.cuh"
+
+namespace dr {
+using namespace ptx;
+
+constexpr int P_A_BYTES = TILE_M * 128;
+constexpr int P_THREADS = 192;          // warp 0 TMA, warp 1 MMA, warps 2-5 epilogue
+constexpr int P_MAX_STAGES = 6;
+constexpr int P_SMEM_MAX = 227 * 1024 - 256;
+
+__device__ __forceinline__ uint32_t swz128(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
+
+struct PatchShared {
+    uint64_t full[P_MAX_STAGES], empty[P_MAX_STAGES], tfull[2], tempty[2];
+    uint32_t tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ void tma_load_4d_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
+                 "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+
+__global__ void __launch_bounds__(P_THREADS, 1)
+conv_patch_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const int stages,
+                      const int stage_bytes) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __shared__ PatchShared sh;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    uint8_t* fe_stage = smem + stages * stage_bytes;
+
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 4); }
+        sh.abort = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+    }
+    if (warp == 1) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+    volatile int* abort_flag = &sh.abort;
+
+    const int cpb = (p.Cin + 63) >> 6;
+    const int total = p.m_tiles;
+    const int per = p.tiles_h * p.tiles_w;
+    const int pwc = 2 * p.PW + 1, phc = 2 * p.PH + 1;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t full0 = smem_u32(&sh.full[0]), empty0 = smem_u32(&sh.empty[0]);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint32_t tx = (uint32_t)(pwc * phc) * 128u + (uint32_t)p.Nt * 128u;
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+                const int n = t / per, tt_ = t - n * per;
+                const int th = tt_ / p.tiles_w, tw = tt_ - th * p.tiles_w;
+                const int h0 = 2 * th * p.PH - 1 - p.pad, w0 = 2 * tw * p.PW - 1 - p.pad;   // stride 1
+                int tap = 0;
+                for (int r = 0; r < p.k && ok; ++r)
+                    for (int q = 0; q < p.k && ok; ++q, ++tap)
+                        for (int c0 = 0; c0 < p.Cin; c0 += 64) {
+                            if (!mbar_wait_u32(empty0 + 8 * s, ph ^ 1, abort_flag)) {
+                                if (!*abort_flag) report_timeout(p.status, 31, t);
+                                *abort_flag = 1;
+                                ok = false;
+                                break;
+                            }
+                            const uint32_t a_dst = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+                            const uint32_t fb = full0 + 8 * s;
+                            mbar_expect_tx_u32(fb, tx);
+                            tma_load_4d_tile(a_dst, &map_a, fb, c0, w0 + q, h0 + r, n);
+                            tma_load_3d_u32<false>(a_dst + P_A_BYTES, &map_b, fb, c0, tap, 0, 1u);
+                            if (++s == stages) { s = 0; ph ^= 1; }
+                        }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t tfull0 = smem_u32(&sh.tfull[0]), tempty0 = smem_u32(&sh.tempty[0]);
+            const int ntaps = p.k * p.k;
+            const int last_nk16 = ((p.Cin - ((cpb - 1) << 6)) + 15) >> 4;
+            const uint32_t idesc = make_idesc_bf16(TILE_M, p.Nt);
+            int s = 0, it = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
+                const int acc = it & 1, au = it >> 1;
+                if (!mbar_wait_u32(tempty0 + 8 * acc, (au & 1) ^ 1, abort_flag)) {
+                    if (!*abort_flag) report_timeout(p.status, 32, t);
+                    *abort_flag = 1;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d = tmem + (uint32_t)(acc * 256);
+                uint32_t accum = 0;
+                for (int tap = 0; tap < ntaps && ok; ++tap)
+                    for (int cc = 0; cc < cpb; ++cc) {
+                        if (!mbar_wait_u32(full0 + 8 * s, ph, abort_flag)) {
+                            if (!*abort_flag) report_timeout(p.status, 33, t);
+                            *abort_flag = 1;
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t a = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+                        const uint32_t alo = sdesc_lo(a), blo = sdesc_lo(a + P_A_BYTES);
+                        const int nk16 = (cc == cpb - 1) ? last_nk16 : 4;
+                        umma_bf16_lo<false>(d, alo, blo, idesc, accum, 1u);
+                        accum = 1;
+                        umma_bf16_lo<false>(d, alo + 2, blo + 2, idesc, 1u, nk16 > 1);
+                        umma_bf16_lo<false>(d, alo + 4, blo + 4, idesc, 1u, nk16 > 2);
+                        umma_bf16_lo<false>(d, alo + 6, blo + 6, idesc, 1u, nk16 > 3);
+                        umma_commit_u32<false>(empty0 + 8 * s);
+                        if (++s == stages) { s = 0; ph ^= 1; }
+                    }
+                if (ok) umma_commit_u32<false>(tfull0 + 8 * acc);
+            }
+        }
+        __syncwarp();
+    } else {
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        int it = 0;
+        for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
+            const int acc = it & 1, au = it >> 1;
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[acc], au & 1, abort_flag));
+            if (!ok) {
+                if (!*abort_flag) report_timeout(p.status, 34, t);
+                *abort_flag = 1;
+                break;
+            }
+            tc_fence_after();
+            uint64_t* te = &sh.tempty[acc];
+            fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * 256), fe_stage, row, 1, [&]() {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(te);
+            });
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) {}
+        __syncthreads();
+    }
+    if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+// =====================================================================================
+//                                     stem kernel
+// =====================================================================================
+constexpr int S_THREADS = 288;          // warps 0-3 producers, warp 4 MMA, warps 5-8 epilogue
+constexpr int S_KSLOTS = 24;            // K slots per tap-row (k * Cin = 21 used)
+constexpr int S_SUBTILES = 3;           // K' = 192 = 3 x 64
+constexpr int S_A_BYTES = S_SUBTILES * P_A_BYTES;          // one im2col tile: 48 KB
+constexpr int S_B_BYTES = S_SUBTILES * 64 * 128;            // resident filters: 24 KB (64 filters)
+
+struct StemShared {
+    uint64_t afull[2], aempty[2], tfull[2], tempty[2];
+    uint32_t tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ void cp_async4_zfill(uint32_t dst, const void* src, bool valid) {
+    const int sz = valid ? 4 : 0;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+
+// Layer fixed to k = 7, stride 2, pad 3, Cin = 3, Cout = 64 (host checks).
+__global__ void __launch_bounds__(S_THREADS, 1) conv_stem_kernel(const ConvParams p, const int in_rows, const int in_words) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __shared__ StemShared sh;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    uint8_t* Bs = smem;                                   // [3][64 rows][128 B]
+    uint8_t* As = Bs + S_B_BYTES;                         // 2 x [3][128 rows][128 B]
+    uint8_t* fe_stage = As + 2 * S_A_BYTES;
+    uint32_t* inp = reinterpret_cast<uint32_t*>(fe_stage + fe_smem_bytes(p));   // 2 x [in_rows][in_words] input patches
+    const int patch_words = in_rows * in_words;
+
+    if (tid == 0) {
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&sh.afull[a], 128); mbar_init(&sh.aempty[a], 1);
+            mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 4);
+        }
+        sh.abort = 0;
+        fence_barrier_init();
+    }
+    if (warp == 4) { tmem_alloc(&sh.tmem_base, 128); tmem_relinquish(); }
+    // resident filter tile in K' order, zero elsewhere; operand tiles start zeroed (their unused
+    // K' slots must stay finite: they meet zero weights)
+    for (int i = tid; i < (S_B_BYTES + 2 * S_A_BYTES) / 16; i += S_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    for (int i = tid; i < 64 * 147; i += S_THREADS) {
+        const int j = i / 147, e = i - j * 147;           // filter j, element (r, s, c) flattened
+        const int r = e / 21, sc = e - r * 21;
+        const int kp = r * S_KSLOTS + sc;                 // K' index
+        const int sub = kp >> 6, within = kp & 63;
+        const uint32_t off = (uint32_t)sub * (64 * 128) + swz128(j, within >> 3) + (within & 7) * 2;
+        *reinterpret_cast<unsigned short*>(Bs + off) = (j < p.Cout) ? reinterpret_cast<const unsigned short*>(p.w)[(size_t)j * 147 + e] : (unsigned short)0;
+    }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+    volatile int* abort_flag = &sh.abort;
+
+    const int total = p.m_tiles;
+    const int per = p.tiles_h * p.tiles_w;
+    const int pwc = 2 * p.PW + 1, phc = 2 * p.PH + 1;
+
+    if (warp < 4) {
+        // ------------------------------------------------ producers: thread = patch row (conv pixel)
+        const int pi = tid / pwc, pj = tid - pi * pwc;
+        const bool row_used = pi < phc;
+        // issue the cp.async loads of tile t's input patch into buffer b
+        auto load_patch = [&](int t, int b) {
+            const int n = t / per, tt_ = t - n * per;
+            const int th = tt_ / p.tiles_w, tw = tt_ - th * p.tiles_w;
+            const int hi0 = 2 * (2 * th * p.PH - 1) - 3;              // first input row of the patch
+            const int wi0 = 2 * (2 * tw * p.PW - 1) - 3 - 1;          // first input column, one early: even element index
+            const unsigned short* ximg = reinterpret_cast<const unsigned short*>(p.x) + (size_t)n * p.H * p.W * 3;
+            const uint32_t dst0 = smem_u32(inp + b * patch_words);
+            for (int i = tid; i < patch_words; i += 128) {
+                const int rr = i / in_words, ww = i - rr * in_words;
+                const int hi = hi0 + rr;
+                const int e = 3 * wi0 + 2 * ww;                        // element index inside the image row (even)
+                const bool ok = hi >= 0 && hi < p.H && e >= 0 && e + 1 < 3 * p.W;
+                const unsigned short* src = ximg + ((size_t)(ok ? hi : 0) * p.W) * 3 + (ok ? e : 0);
+                cp_async4_zfill(dst0 + 4u * i, src, ok);
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        int it = 0;
+        if ((int)blockIdx.x < total) load_patch(blockIdx.x, 0);
+        for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
+            const int b = it & 1, u = it >> 1;
+            const int tn = t + gridDim.x;
+            if (tn < total) load_patch(tn, b ^ 1);
+            else asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 1;" ::: "memory");       // this tile's patch has landed (for this thread)
+            asm volatile("bar.sync 2, 128;" ::: "memory");             // ... and for the other producers
+            bool ok = mbar_wait(&sh.aempty[b], (u & 1) ^ 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) {
+                if (!*abort_flag) report_timeout(p.status, 41, t);
+                *abort_flag = 1;
+                break;
+            }
+            if (row_used) {
+                uint8_t* At = As + b * S_A_BYTES;
+                const uint32_t* src = inp + b * patch_words;
+#pragma unroll
+                for (int r = 0; r < 7; ++r) {
+                    // tap-row r of this pixel: 24 elements (12 words) starting at patch row 2*pi + r, element 6*pj + 3
+                    // (+3: the patch starts one pixel early)
+                    const uint32_t* s32 = src + (2 * pi + r) * in_words;
+                    const int e0 = 6 * pj + 3;                         // odd element index -> words straddle: realign below
+                    uint32_t wv[13];
+#pragma unroll
+                    for (int k = 0; k < 13; ++k) wv[k] = s32[(e0 >> 1) + k];
+                    uint32_t ov[12];
+#pragma unroll
+                    for (int k = 0; k < 12; ++k) ov[k] = __funnelshift_r(wv[k], wv[k + 1], 16);   // drop the leading half word
+#pragma unroll
+                    for (int m = 0; m < 3; ++m) {
+                        const int q = 3 * r + m;                       // 16-byte chunk index along K'
+                        const uint32_t off = (uint32_t)(q >> 3) * P_A_BYTES + swz128(tid, q & 7);
+                        *reinterpret_cast<uint4*>(At + off) = make_uint4(ov[4 * m], ov[4 * m + 1], ov[4 * m + 2], ov[4 * m + 3]);
+                    }
+                }
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&sh.afull[b]);
+            asm volatile("bar.sync 2, 128;" ::: "memory");             // everyone is done reading this patch buffer
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    } else if (warp == 4) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_bf16(TILE_M, 64);
+            const uint32_t b_lo = sdesc_lo(smem_u32(Bs));
+            int it = 0;
+            for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
+                const int b = it & 1, u = it >> 1;
+                if (!mbar_wait(&sh.tempty[b], (u & 1) ^ 1, abort_flag) || !mbar_wait(&sh.afull[b], u & 1, abort_flag)) {
+                    if (!*abort_flag) report_timeout(p.status, 42, t);
+                    *abort_flag = 1;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d = tmem + (uint32_t)(b * 64);
+                const uint32_t a_lo = sdesc_lo(smem_u32(As + b * S_A_BYTES));
+#pragma unroll
+                for (int kk = 0; kk < 11; ++kk) {                      // K' = 176 of 192: the rest is zero weights
+                    const uint32_t sub = kk >> 2, k4 = kk & 3;
+                    umma_bf16_lo<false>(d, a_lo + sub * (P_A_BYTES >> 4) + 2 * k4, b_lo + sub * ((64 * 128) >> 4) + 2 * k4, idesc, kk > 0, 1u);
+                }
+                umma_commit(&sh.aempty[b]);
+                umma_commit(&sh.tfull[b]);
+            }
+        }
+        __syncwarp();
+    } else {
+        const int q = warp & 3;                                        // warps 5-8 -> TMEM lane quarters 1,2,3,0
+        const int row = q * 32 + lane;
+        int it = 0;
+        for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
+            const int b = it & 1, u = it >> 1;
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[b], u & 1, abort_flag));
+            if (!ok) {
+                if (!*abort_flag) report_timeout(p.status, 44, t);
+                *abort_flag = 1;
+                break;
+            }
+            tc_fence_after();
+            uint64_t* te = &sh.tempty[b];
+            fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * 64), fe_stage, row, 1, [&]() {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(te);
+            });
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) {}
+        __syncthreads();
+    }
+    if (warp == 4) tmem_dealloc(tmem, 128);
+}
+
+// ---- host --------------------------------------------------------------------------------
+typedef CUresult (*PFN_encodeTiledP)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                     const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                     CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static PFN_encodeTiledP g_enc = nullptr;
+static bool load_enc() {
+    if (g_enc) return true;
+    cudaDriverEntryPointQueryResult q;
+    void* f = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || !f) return false;
+    g_enc = (PFN_encodeTiledP)f;
+    return true;
+}
+
+bool conv_patch_tma_supports(const ConvParams& p) {
+    if (!p.patch || !fe_supports(p)) return false;
+    if (p.stride != 1 || (p.Cin & 7) || p.Cin < 64 || p.k > 15) return false;
+    const int stage_bytes = P_A_BYTES + ((p.Nt * 128 + 1023) & ~1023);
+    return 2 * stage_bytes + fe_smem_bytes(p) + 2048 <= P_SMEM_MAX;
+}
+
+int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
+    if (!conv_patch_tma_supports(p)) return DR_ERR_UNSUPPORTED;
+    if (!load_enc()) return DR_ERR_CUDA;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(conv_patch_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+        attr_set = true;
+    }
+    alignas(64) CUtensorMap map_a, map_b;
+    {
+        const cuuint64_t dims[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
+        const cuuint64_t strides[3] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.W * p.Cin * 2, (cuuint64_t)p.H * p.W * p.Cin * 2};
+        const cuuint32_t box[4] = {64, (cuuint32_t)(2 * p.PW + 1), (cuuint32_t)(2 * p.PH + 1), 1};
+        const cuuint32_t es[4] = {1, 1, 1, 1};
+        if (g_enc(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void*)p.x, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DR_ERR_CUDA;
+    }
+    {
+        const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
+        const cuuint64_t strides[2] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.K * 2};
+        const cuuint32_t box[3] = {64, 1, (cuuint32_t)p.Nt};
+        const cuuint32_t es[3] = {1, 1, 1};
+        if (g_enc(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)p.w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DR_ERR_CUDA;
+    }
+    if (p.m_tiles <= 0) return DR_OK;
+    const int stage_bytes = P_A_BYTES + ((p.Nt * 128 + 1023) & ~1023);
+    int stages = (P_SMEM_MAX - 2048 - fe_smem_bytes(p)) / stage_bytes;
+    if (stages > P_MAX_STAGES) stages = P_MAX_STAGES;
+    int smem_bytes = stages * stage_bytes + fe_smem_bytes(p) + 1024;
+    if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;     // one CTA per SM: each CTA takes all of TMEM
+    const int grid = p.m_tiles < num_sms() ? p.m_tiles : num_sms();
+    conv_patch_tma_kernel<<<grid, P_THREADS, smem_bytes, stream>>>(p, map_a, map_b, stages, stage_bytes);
+    count_launch();
+    return launch_status();
+}
+
+static void stem_patch_dims(const ConvParams& p, int* rows, int* words) {
+    *rows = 2 * (2 * p.PH + 1) + 5;                                   // input rows under the conv patch
+    const int pixels = 2 * (2 * p.PW + 1) + 5 + 1 + 1;                // + one early pixel (alignment) + one late (13th word)
+    *words = (3 * pixels + 1) / 2 + 1;
+}
+
+bool conv_stem_supports(const ConvParams& p) {
+    if (!p.patch || !fe_supports(p)) return false;
+    if (p.k != 7 || p.stride != 2 || p.pad != 3 || p.Cin != 3 || p.Cout != 64 || (p.W & 1)) return false;
+    int rows, words;
+    stem_patch_dims(p, &rows, &words);
+    return S_B_BYTES + 2 * S_A_BYTES + fe_smem_bytes(p) + 2 * rows * words * 4 + 2048 <= P_SMEM_MAX;
+}
+
+int conv_stem_launch(const ConvParams& p, cudaStream_t stream) {
+    if (!conv_stem_supports(p)) return DR_ERR_UNSUPPORTED;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(conv_stem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+        attr_set = true;
+    }
+    if (p.m_tiles <= 0) return DR_OK;
+    int rows, words;
+    stem_patch_dims(p, &rows, &words);
+    const int smem_bytes = S_B_BYTES + 2 * S_A_BYTES + fe_smem_bytes(p) + 2 * rows * words * 4 + 1024;
+    const int grid = p.m_tiles < num_sms() ? p.m_tiles : num_sms();
+    conv_stem_kernel<<<grid, S_THREADS, smem_bytes, stream>>>(p, rows, words);
+    count_launch();
+    return launch_status();
+}
+
+}  // namespace dr

@@ -256,7 +256,7 @@ __device__ __forceinline__ uint32_t mbar_test_u32(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
-__device__ __noinline__ bool mbar_wait_slow_u32(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+static __device__ __noinline__ bool mbar_wait_slow_u32(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1

@@ -175,10 +175,16 @@ STAGED = [
     (2, 13, 9, 32, 48, 3, 1, 1, "pool"),
     (1, 9, 12, 16, 32, 1, 1, 0, "lrn"),
     (1, 5, 5, 8, 16, 3, 1, 1, "pool"),              # plane smaller than one patch
+    (3, 56, 56, 64, 192, 3, 1, 1, "lrn_pool"),      # GoogLeNet conv2 at its real plane size
+    (2, 30, 26, 128, 64, 3, 1, 1, "pool"),          # two channel blocks per tap
+    (2, 21, 19, 64, 96, 5, 1, 2, "pool_lrn"),       # 5x5, pool then LRN, float32 staging with 96 channels
+    (2, 224, 224, 3, 64, 7, 2, 3, "pool_lrn"),      # GoogLeNet conv1 at full size
+    (2, 70, 50, 3, 64, 7, 2, 3, "pool"),            # ResNet conv1 form (no LRN), ragged tiles
+    (1, 38, 42, 3, 64, 7, 2, 3, "lrn_pool"),        # stem with LRN first
 ]
 
 
-@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("path", [1, 2, 3, 4, 5])
 @pytest.mark.parametrize("case", STAGED)
 def test_conv_fused_pool_lrn(dr, O, path, case):
     B, H, W, Cin, Cout, k, s, p, kind = case
@@ -188,7 +194,7 @@ def test_conv_fused_pool_lrn(dr, O, path, case):
     lrn = (5, 1e-4, 0.75, 1.0) if kind == "pool_lrn" else (5, 0.05, 0.75, 1.0)      # second set makes LRN bite
     force(dr, path)
     try:
-        got, arg = run_conv(dr, x, w, b, k, s, p, flags, lrn=lrn, want_argmax=bool(flags & dr.DR_POOL))
+        got, arg = run_conv(dr, x, w, b, k, s, p, flags, lrn=lrn, want_argmax=bool(flags & dr.DR_POOL) and path <= 3)
     except dr.DrError as e:
         if e.status == dr.DR_ERR_UNSUPPORTED and path != dr.DR_PATH_SIMT:
             pytest.skip("path does not take this shape")
