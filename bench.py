@@ -122,6 +122,51 @@ def run_reference(args):
     }))
 
 
+def run_layer(args):
+    """One slim layer of GoogLeNet through dr_conv_slim, timed with CUDA events (L2 flushed between launches)."""
+    import numpy as np
+    import torch
+    import __graft_entry__
+    __graft_entry__.build_cuda()
+    import dr_synth as S
+    import paper_1708_04728_b200 as dr
+    B = args.batch
+    table = {"conv1": (224, 3, 64, 7, 2, 3, dr.DR_POOL | dr.DR_LRN), "conv2r": (56, 64, 64, 1, 1, 0, 0),
+             "conv2": (56, 64, 192, 3, 1, 1, dr.DR_POOL | dr.DR_LRN | dr.DR_LRN_BEFORE_POOL)}
+    H = 28
+    for m, (cin, c1, c3r, c3, _c5r, c5, pp) in S.INCEPTION_V1.items():
+        H = 14 if m == "4a" else 7 if m == "5a" else H
+        table[m + ".3x3r"] = (H, cin, c3r, 1, 1, 0, 0)
+        table[m + ".3x3"] = (H, c3r, c3, 3, 1, 1, 0)
+        table[m + ".m5"] = (H, cin, c1 + c5 + pp, 5, 1, 2, 0)
+    H, cin, cout, k, s_, p_, fl = table[args.layer]
+    g = S.stream(0, "layer." + args.layer)
+    x = torch.from_numpy(g.standard_normal((B, H, H, cin), dtype=np.float32)).cuda().to(torch.bfloat16)
+    w = torch.from_numpy(g.standard_normal((cout, k, k, cin), dtype=np.float32) * np.float32((2.0 / (k * k * cin)) ** 0.5)).cuda().to(torch.bfloat16)
+    b = torch.zeros(cout, device="cuda")
+    Ho = (H + 2 * p_ - k) // s_ + 1
+    Hy = (Ho - 1) // 2 + 1 if fl & dr.DR_POOL else Ho
+    y = torch.empty((B, Hy, Hy, cout), dtype=torch.bfloat16, device="cuda")
+    d = dr.dr_conv_desc(k=k, stride=s_, pad=p_, Cin=cin, Cout=cout, flags=dr.DR_BIAS | dr.DR_RELU | fl, pool_k=3, pool_stride=2,
+                        pool_pad=1, lrn_size=5, lrn_alpha=1e-4, lrn_beta=0.75, lrn_k=1.0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    ts = []
+    for i in range(args.warmup + args.steps):
+        flush.zero_()
+        a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); dr.dr_conv_slim(d, B, H, H, x, w, b, None, y); e.record()
+        torch.cuda.synchronize()
+        if i >= args.warmup:
+            ts.append(a.elapsed_time(e) * 1e3)
+    st, info = dr.dr_device_status()
+    assert st == 0, info
+    us = statistics.median(ts)
+    flops = 2.0 * B * Ho * Ho * cout * k * k * cin
+    nbytes = 2.0 * (B * H * H * cin + cout * k * k * cin + B * Hy * Hy * cout)
+    print(json.dumps({"layer": args.layer, "batch": B, "us": us, "tflops": flops / us * 1e-6, "gbs": nbytes / us * 1e-3,
+                      "gflop": flops * 1e-9, "mbytes": nbytes * 1e-6, "path": dr.PATH_NAMES[dr.dr_last_conv_path()]}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -131,9 +176,14 @@ def main():
     ap.add_argument("--batch", type=int, default=256)
     ap.add_argument("--layers-out", default=None, help="write the per-layer table (us, roofline) as JSON")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layer", default=None,
+                    help="time ONE slim layer of the network (e.g. conv1, conv2, 3b.m5, 4e.3x3) instead of the whole step; "
+                         "this is the small case the ncu captures under profiles/ run")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.layer:
+        return run_layer(args)
 
     import numpy as np
     import torch
