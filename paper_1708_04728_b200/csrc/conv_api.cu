@@ -1,4 +1,6 @@
 // dr_conv_slim / dr_inception_slim: validation, tiling choice and kernel dispatch.
+#include <cmath>
+
 #include "conv_common.cuh"
 
 namespace dr {
@@ -51,6 +53,15 @@ int conv_make_params(const dr_conv_desc* d, int B, int H, int W, const void* x, 
     p.lrn_half = (f & DR_LRN) ? d->lrn_size / 2 : 0;
     p.lrn_alpha_n = (f & DR_LRN) ? d->lrn_alpha / d->lrn_size : 0.f;
     p.lrn_beta = d->lrn_beta; p.lrn_k = d->lrn_k;
+    if (f & DR_LRN) {
+        const double be = d->lrn_beta, kk = d->lrn_k;
+        p.lrn_inv_k = kk > 0 ? (float)(1.0 / kk) : 0.f;
+        p.lrn_kpow = kk > 0 ? (float)pow(kk, -be) : 0.f;
+        p.lrn_c1 = (float)(-be);
+        p.lrn_c2 = (float)(be * (be + 1) / 2);
+        p.lrn_c3 = (float)(-be * (be + 1) * (be + 2) / 6);
+        p.lrn_c4 = (float)(be * (be + 1) * (be + 2) * (be + 3) / 24);
+    }
     p.ldc = ldc; p.coff = coff;
     p.M = (long long)B * p.Ho * p.Wo;
     const int cout16 = (d->Cout + 15) / 16 * 16;

@@ -36,6 +36,8 @@ struct ConvParams {
     unsigned flags;
     int lrn_half;
     float lrn_alpha_n, lrn_beta, lrn_k;
+    float lrn_inv_k, lrn_kpow;   // 1/k and k^(-beta)
+    float lrn_c1, lrn_c2, lrn_c3, lrn_c4;   // binomial series of (1+u)^(-beta)
     int ldc, coff;
     long long M;           // B*Ho*Wo
     int Nt;                // output channels per n-block (multiple of 16, <= 256)

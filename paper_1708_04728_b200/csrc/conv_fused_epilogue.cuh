@@ -6,10 +6,17 @@
 //       register sliding window over 32-column TMEM chunks; the result goes to shared memory as
 //       bf16 (max-pooling commutes with the monotone bf16 rounding, so rounding before the max gives
 //       the same stored value as rounding after it), then 3x3/2 max over rows.
-//   pool first (ReLU -> pool [-> LRN]): ReLU'd float32 values are staged, the 3x3/2 max is taken in
-//       float32, and LRN (if any) runs on the pooled float32 values before the single bf16 rounding.
+//   pool first (ReLU -> pool [-> LRN]): the raw float32 accumulators are staged and the 3x3/2 max is
+//       taken on them; bias and ReLU are applied to the pooled values only (adding a per-channel
+//       constant and clamping are monotone, so they commute with the max: 4-5x fewer evaluations),
+//       then LRN (if any) on the pooled float32 values, then the single bf16 rounding.
 // Rows of the patch that fall outside the convolution plane are staged as -inf, so the max needs no
 // masks ("padding never wins"; every window holds at least one real pixel).
+//
+// LRN scale s^(-beta), s = k + (alpha/n) * sum x^2: when the normalised excess u = (s-k)/k is below
+// 1/32 for a whole 32-channel chunk of the warp, (1+u)^(-beta) is evaluated by its binomial series
+// to the u^4 term (truncation error < 2e-8 relative, below float32 resolution); otherwise the chunk
+// takes the exp2/log2 route.  The special-function unit would otherwise bound the layer.
 #pragma once
 #include "conv_common.cuh"
 #include "umma_ptx.cuh"
@@ -20,30 +27,44 @@ constexpr int FE_THREADS = 128;          // epilogue threads (4 warps)
 
 __device__ __forceinline__ void fe_bar(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(FE_THREADS) : "memory"); }
 
-// bytes of shared memory the epilogue needs for a layer
-__host__ __device__ inline int fe_stage_pitch(const ConvParams& p) {
-    const bool lrn_first = (p.flags & DR_LRN) && (p.flags & DR_LRN_BEFORE_POOL);
-    const bool f32 = (p.flags & DR_LRN) && !lrn_first;          // pool first and LRN after: keep float32
-    return f32 ? (p.Cout * 4 + 16) : (p.Cout * 2 + 16);          // +16 B: conflict-free 16-byte row-wise stores
-}
+__host__ __device__ inline bool fe_lrn_first(const ConvParams& p) { return (p.flags & DR_LRN) && (p.flags & DR_LRN_BEFORE_POOL); }
+// bytes of one staged row: bf16 after LRN-first, float32 raw accumulators otherwise (+16 B: 16-byte
+// row-wise stores of a warp then fall on distinct banks)
+__host__ __device__ inline int fe_stage_pitch(const ConvParams& p) { return fe_lrn_first(p) ? (p.Cout * 2 + 16) : (p.Cout * 4 + 16); }
 __host__ __device__ inline int fe_smem_bytes(const ConvParams& p) {
-    const bool lrn_first = (p.flags & DR_LRN) && (p.flags & DR_LRN_BEFORE_POOL);
-    const bool f32 = (p.flags & DR_LRN) && !lrn_first;
-    int b = TILE_M * fe_stage_pitch(p);
-    if (f32) b += p.PH * p.PW * (p.Cout + 8) * 4;               // pooled float32 values, 4 floats of halo each side
+    int b = TILE_M * fe_stage_pitch(p) + 256 * 4;                       // stage + bias copy
+    if ((p.flags & DR_LRN) && !fe_lrn_first(p)) b += p.PH * p.PW * (p.Cout + 8) * 4;   // pooled float32 values, 4 floats of halo each side
     return (b + 1023) & ~1023;
 }
 inline bool fe_supports(const ConvParams& p) {
     if (!(p.flags & DR_POOL) || p.argmax) return false;          // argmax and LRN-only layers: gather kernel
     if (p.Cout % 32 || p.Cout > 256) return false;
-    if ((p.flags & DR_LRN) && p.lrn_half != 2) return false;
+    if ((p.flags & DR_LRN) && (p.lrn_half != 2 || p.lrn_k <= 0.f || p.lrn_alpha_n < 0.f)) return false;
     if (p.flags & (DR_RESIDUAL | DR_OUT_F32)) return false;
     if ((p.ldc & 7) || (p.coff & 7)) return false;
     return true;
 }
+// the kernels call this once (all threads) before the first tile
+__device__ __forceinline__ void fe_init(const ConvParams& p, uint8_t* stage, int tid, int nthreads) {
+    float* bias_s = reinterpret_cast<float*>(stage + TILE_M * fe_stage_pitch(p));
+    for (int i = tid; i < 256; i += nthreads) bias_s[i] = ((p.flags & DR_BIAS) && i < p.Cout) ? p.bias[i] : 0.f;
+}
 
-__device__ __forceinline__ float fe_lrn5(float a, float b, float c, float d, float e, float alpha_n, float beta, float kappa) {
-    return c * lrn_pow(kappa + alpha_n * (a * a + b * b + c * c + d * d + e * e), beta);
+// LRN scale factors for N window sums at once; the series/exact choice is uniform over the warp.
+template <int N>
+__device__ __forceinline__ void fe_lrn_scale(const ConvParams& p, const float* ss, float* scale) {
+    float umax = 0.f;
+    float u[N];
+#pragma unroll
+    for (int j = 0; j < N; ++j) { u[j] = p.lrn_alpha_n * p.lrn_inv_k * ss[j]; umax = fmaxf(umax, u[j]); }
+    if (__all_sync(0xffffffffu, umax < 0.03125f)) {
+#pragma unroll
+        for (int j = 0; j < N; ++j)
+            scale[j] = p.lrn_kpow * fmaf(u[j], fmaf(u[j], fmaf(u[j], fmaf(u[j], p.lrn_c4, p.lrn_c3), p.lrn_c2), p.lrn_c1), 1.f);
+    } else {
+#pragma unroll
+        for (int j = 0; j < N; ++j) scale[j] = __powf(fmaf(p.lrn_alpha_n, ss[j], p.lrn_k), -p.lrn_beta);
+    }
 }
 
 // taddr: TMEM address of this thread's lane, column 0 of the accumulator.  row = 0..127.
@@ -53,9 +74,10 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
                                                Release release) {
     const int C = p.Cout;
     const bool lrn = p.flags & DR_LRN;
-    const bool lrn_first = lrn && (p.flags & DR_LRN_BEFORE_POOL);
-    const bool f32 = lrn && !lrn_first;
+    const bool lrn_first = fe_lrn_first(p);
+    const bool relu = p.flags & DR_RELU;
     const int pitch = fe_stage_pitch(p);
+    const float* bias_s = reinterpret_cast<const float*>(stage + TILE_M * pitch);
     const int pwc = 2 * p.PW + 1, phc = 2 * p.PH + 1;
     const int per = p.tiles_h * p.tiles_w;
     const int n = tile / per, t = tile - n * per;
@@ -65,7 +87,7 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
     const bool valid = pi < phc && ho >= 0 && ho < p.Ho && wo >= 0 && wo < p.Wo;
     uint8_t* srow = stage + (size_t)row * pitch;
 
-    // ---- drain TMEM, bias, ReLU, (LRN), stage
+    // ---- drain TMEM (+ bias, ReLU, LRN when LRN comes first), stage
     if (lrn_first) {
         float cur[32], nxt[32];
         float pm2 = 0.f, pm1 = 0.f;                      // x[c-2], x[c-1] of the chunk before
@@ -74,9 +96,14 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
             ptx::tmem_ld_x32(taddr, r);
             ptx::tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                float v = __uint_as_float(r[j]) + ((p.flags & DR_BIAS) ? __ldg(p.bias + j) : 0.f);
-                cur[j] = (p.flags & DR_RELU) ? fmaxf(v, 0.f) : v;
+            for (int q = 0; q < 8; ++q) {
+                const float4 b4 = *reinterpret_cast<const float4*>(bias_s + 4 * q);
+                const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float v = __uint_as_float(r[4 * q + k]) + bb[k];
+                    cur[4 * q + k] = relu ? fmaxf(v, 0.f) : v;
+                }
             }
         }
         for (int c0 = 0; c0 < C; c0 += 32) {
@@ -85,29 +112,36 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
                 ptx::tmem_ld_x32(taddr + c0 + 32, r);
                 ptx::tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    float v = __uint_as_float(r[j]) + ((p.flags & DR_BIAS) ? __ldg(p.bias + c0 + 32 + j) : 0.f);
-                    nxt[j] = (p.flags & DR_RELU) ? fmaxf(v, 0.f) : v;
+                for (int q = 0; q < 8; ++q) {
+                    const float4 b4 = *reinterpret_cast<const float4*>(bias_s + c0 + 32 + 4 * q);
+                    const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float v = __uint_as_float(r[4 * q + k]) + bb[k];
+                        nxt[4 * q + k] = relu ? fmaxf(v, 0.f) : v;
+                    }
                 }
             } else {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) nxt[j] = 0.f;
             }
-            float o[32];
+            float sq[36];                                  // squares of x[c0-2 .. c0+33]
+            sq[0] = pm2 * pm2; sq[1] = pm1 * pm1;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float a = j >= 2 ? cur[j - 2] : (j == 0 ? pm2 : pm1);
-                const float b = j >= 1 ? cur[j - 1] : pm1;
-                const float d = j + 1 < 32 ? cur[j + 1] : nxt[0];
-                const float e = j + 2 < 32 ? cur[j + 2] : nxt[j + 2 - 32];
-                o[j] = fe_lrn5(a, b, cur[j], d, e, p.lrn_alpha_n, p.lrn_beta, p.lrn_k);
-            }
+            for (int j = 0; j < 32; ++j) sq[2 + j] = cur[j] * cur[j];
+            sq[34] = nxt[0] * nxt[0]; sq[35] = nxt[1] * nxt[1];
+            float ss[32], sc[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ss[j] = (sq[j] + sq[j + 1]) + (sq[j + 2] + sq[j + 3]) + sq[j + 4];
+            fe_lrn_scale<32>(p, ss, sc);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 uint4 v;
                 if (valid) {
-                    v.x = pack_bf16(o[8 * q + 0], o[8 * q + 1]); v.y = pack_bf16(o[8 * q + 2], o[8 * q + 3]);
-                    v.z = pack_bf16(o[8 * q + 4], o[8 * q + 5]); v.w = pack_bf16(o[8 * q + 6], o[8 * q + 7]);
+                    v.x = pack_bf16(cur[8 * q + 0] * sc[8 * q + 0], cur[8 * q + 1] * sc[8 * q + 1]);
+                    v.y = pack_bf16(cur[8 * q + 2] * sc[8 * q + 2], cur[8 * q + 3] * sc[8 * q + 3]);
+                    v.z = pack_bf16(cur[8 * q + 4] * sc[8 * q + 4], cur[8 * q + 5] * sc[8 * q + 5]);
+                    v.w = pack_bf16(cur[8 * q + 6] * sc[8 * q + 6], cur[8 * q + 7] * sc[8 * q + 7]);
                 } else {
                     v.x = v.y = v.z = v.w = 0xFF80FF80u;     // -inf, -inf
                 }
@@ -123,25 +157,11 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
             uint32_t r[32];
             ptx::tmem_ld_x32(taddr + c0, r);
             ptx::tmem_ld_wait();
-            float v[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                float x = __uint_as_float(r[j]) + ((p.flags & DR_BIAS) ? __ldg(p.bias + c0 + j) : 0.f);
-                x = (p.flags & DR_RELU) ? fmaxf(x, 0.f) : x;
-                v[j] = valid ? x : __int_as_float(0xff800000);
-            }
-            if (f32) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    *reinterpret_cast<float4*>(srow + (c0 + 4 * q) * 4) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-            } else {
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint4 u;
-                    u.x = pack_bf16(v[8 * q + 0], v[8 * q + 1]); u.y = pack_bf16(v[8 * q + 2], v[8 * q + 3]);
-                    u.z = pack_bf16(v[8 * q + 4], v[8 * q + 5]); u.w = pack_bf16(v[8 * q + 6], v[8 * q + 7]);
-                    *reinterpret_cast<uint4*>(srow + (c0 + 8 * q) * 2) = u;
-                }
+            for (int q = 0; q < 8; ++q) {
+                uint4 v = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+                if (!valid) v.x = v.y = v.z = v.w = 0xff800000u;   // -inf
+                *reinterpret_cast<uint4*>(srow + (c0 + 4 * q) * 4) = v;
             }
         }
     }
@@ -151,33 +171,41 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
 
     // ---- 3x3 / 2 max over the staged patch
     __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.y);
-    if (!f32) {
+    const int npp = p.PH * p.PW;
+    if (lrn_first) {
         const int C8 = C >> 3;
-        for (int it = row; it < p.PH * p.PW * C8; it += FE_THREADS) {
-            const int pp = it / C8, c = (it - pp * C8) << 3;
+        const int dpp = FE_THREADS / C8, dc8 = FE_THREADS - dpp * C8;      // step of the (pp, c8) item index per pass
+        int pp = row / C8, c8 = row - pp * C8;
+        while (pp < npp) {
             const int ppi = pp / p.PW, ppj = pp - ppi * p.PW;
             const int ph = th * p.PH + ppi, pw = tw * p.PW + ppj;
-            if (ph >= p.Hy || pw >= p.Wy) continue;
-            const uint8_t* base = stage + (size_t)((2 * ppi) * pwc + 2 * ppj) * pitch + c * 2;
-            uint4 m = *reinterpret_cast<const uint4*>(base);
-            __nv_bfloat162* mm = reinterpret_cast<__nv_bfloat162*>(&m);
+            if (ph < p.Hy && pw < p.Wy) {
+                const uint8_t* base = stage + (size_t)((2 * ppi) * pwc + 2 * ppj) * pitch + c8 * 16;
+                uint4 m = *reinterpret_cast<const uint4*>(base);
+                __nv_bfloat162* mm = reinterpret_cast<__nv_bfloat162*>(&m);
 #pragma unroll
-            for (int d = 1; d < 9; ++d) {
-                const uint4 u = *reinterpret_cast<const uint4*>(base + (size_t)((d / 3) * pwc + (d % 3)) * pitch);
-                const __nv_bfloat162* uu = reinterpret_cast<const __nv_bfloat162*>(&u);
+                for (int d = 1; d < 9; ++d) {
+                    const uint4 u = *reinterpret_cast<const uint4*>(base + (size_t)((d / 3) * pwc + (d % 3)) * pitch);
+                    const __nv_bfloat162* uu = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) mm[k] = __hmax2(mm[k], uu[k]);
+                    for (int k = 0; k < 4; ++k) mm[k] = __hmax2(mm[k], uu[k]);
+                }
+                const long long q = ((long long)n * p.Hy + ph) * p.Wy + pw;
+                *reinterpret_cast<uint4*>(y + q * p.ldc + p.coff + c8 * 8) = m;
             }
-            const long long q = ((long long)n * p.Hy + ph) * p.Wy + pw;
-            *reinterpret_cast<uint4*>(y + q * p.ldc + p.coff + c) = m;
+            pp += dpp; c8 += dc8;
+            if (c8 >= C8) { c8 -= C8; ++pp; }
         }
     } else {
-        float* pooled = reinterpret_cast<float*>(stage + (size_t)TILE_M * pitch);   // [pp][4 halo | C | 4 halo]
+        float* pooled = reinterpret_cast<float*>(stage + (size_t)TILE_M * pitch + 256 * 4);   // [pp][4 halo | C | 4 halo]
         const int ldp = C + 8;
         const int C4 = C >> 2;
-        for (int it = row; it < p.PH * p.PW * C4; it += FE_THREADS) {
-            const int pp = it / C4, c = (it - pp * C4) << 2;
+        const int dpp = FE_THREADS / C4, dc4 = FE_THREADS - dpp * C4;
+        int pp = row / C4, c4 = row - pp * C4;
+        while (pp < npp) {
             const int ppi = pp / p.PW, ppj = pp - ppi * p.PW;
+            const int ph = th * p.PH + ppi, pw = tw * p.PW + ppj;
+            const int c = c4 << 2;
             const uint8_t* base = stage + (size_t)((2 * ppi) * pwc + 2 * ppj) * pitch + c * 4;
             float4 m = *reinterpret_cast<const float4*>(base);
 #pragma unroll
@@ -185,28 +213,50 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
                 const float4 u = *reinterpret_cast<const float4*>(base + (size_t)((d / 3) * pwc + (d % 3)) * pitch);
                 m.x = fmaxf(m.x, u.x); m.y = fmaxf(m.y, u.y); m.z = fmaxf(m.z, u.z); m.w = fmaxf(m.w, u.w);
             }
-            *reinterpret_cast<float4*>(pooled + pp * ldp + 4 + c) = m;
-            if (c == 0) { pooled[pp * ldp + 2] = 0.f; pooled[pp * ldp + 3] = 0.f; pooled[pp * ldp + C + 4] = 0.f; pooled[pp * ldp + C + 5] = 0.f; }
+            const float4 b4 = *reinterpret_cast<const float4*>(bias_s + c);
+            m.x += b4.x; m.y += b4.y; m.z += b4.z; m.w += b4.w;
+            if (relu) { m.x = fmaxf(m.x, 0.f); m.y = fmaxf(m.y, 0.f); m.z = fmaxf(m.z, 0.f); m.w = fmaxf(m.w, 0.f); }
+            if (lrn) {
+                *reinterpret_cast<float4*>(pooled + pp * ldp + 4 + c) = m;
+                if (c == 0) { pooled[pp * ldp + 2] = 0.f; pooled[pp * ldp + 3] = 0.f; pooled[pp * ldp + C + 4] = 0.f; pooled[pp * ldp + C + 5] = 0.f; }
+            } else if (ph < p.Hy && pw < p.Wy) {
+                const long long q = ((long long)n * p.Hy + ph) * p.Wy + pw;
+                uint2 o;
+                o.x = pack_bf16(m.x, m.y); o.y = pack_bf16(m.z, m.w);
+                *reinterpret_cast<uint2*>(y + q * p.ldc + p.coff + c) = o;
+            }
+            pp += dpp; c4 += dc4;
+            if (c4 >= C4) { c4 -= C4; ++pp; }
         }
-        fe_bar(bar_id);
-        // LRN on the pooled float32 values, 8 channels per thread
-        const int C8 = C >> 3;
-        for (int it = row; it < p.PH * p.PW * C8; it += FE_THREADS) {
-            const int pp = it / C8, c = (it - pp * C8) << 3;
-            const int ppi = pp / p.PW, ppj = pp - ppi * p.PW;
-            const int ph = th * p.PH + ppi, pw = tw * p.PW + ppj;
-            if (ph >= p.Hy || pw >= p.Wy) continue;
-            const float* s = pooled + pp * ldp + 2 + c;       // s[0] = x[c-2]
-            float v[12];
+        if (lrn) {
+            fe_bar(bar_id);
+            // LRN on the pooled float32 values, 8 channels per thread
+            const int C8 = C >> 3;
+            const int dpp8 = FE_THREADS / C8, dc8 = FE_THREADS - dpp8 * C8;
+            int pq = row / C8, c8 = row - pq * C8;
+            const int iters = (npp * C8 + FE_THREADS - 1) / FE_THREADS;   // same trip count for every lane: the
+            for (int itn = 0; itn < iters; ++itn) {                         // series/exact vote below is warp-wide
+                const bool active = pq < npp;
+                const int pr = active ? pq : npp - 1;
+                const int ppi = pr / p.PW, ppj = pr - ppi * p.PW;
+                const int ph = th * p.PH + ppi, pw = tw * p.PW + ppj;
+                const float* s = pooled + pr * ldp + 2 + (c8 << 3);      // s[0] = x[c-2]
+                float v[12], sq[12], ss[8], sc[8];
 #pragma unroll
-            for (int j = 0; j < 12; ++j) v[j] = s[j];
-            float o[8];
+                for (int j = 0; j < 12; ++j) { v[j] = s[j]; sq[j] = v[j] * v[j]; }
 #pragma unroll
-            for (int j = 0; j < 8; ++j) o[j] = fe_lrn5(v[j], v[j + 1], v[j + 2], v[j + 3], v[j + 4], p.lrn_alpha_n, p.lrn_beta, p.lrn_k);
-            uint4 u;
-            u.x = pack_bf16(o[0], o[1]); u.y = pack_bf16(o[2], o[3]); u.z = pack_bf16(o[4], o[5]); u.w = pack_bf16(o[6], o[7]);
-            const long long q = ((long long)n * p.Hy + ph) * p.Wy + pw;
-            *reinterpret_cast<uint4*>(y + q * p.ldc + p.coff + c) = u;
+                for (int j = 0; j < 8; ++j) ss[j] = (sq[j] + sq[j + 1]) + (sq[j + 2] + sq[j + 3]) + sq[j + 4];
+                fe_lrn_scale<8>(p, ss, sc);
+                if (active && ph < p.Hy && pw < p.Wy) {
+                    uint4 u;
+                    u.x = pack_bf16(v[2] * sc[0], v[3] * sc[1]); u.y = pack_bf16(v[4] * sc[2], v[5] * sc[3]);
+                    u.z = pack_bf16(v[6] * sc[4], v[7] * sc[5]); u.w = pack_bf16(v[8] * sc[6], v[9] * sc[7]);
+                    const long long q = ((long long)n * p.Hy + ph) * p.Wy + pw;
+                    *reinterpret_cast<uint4*>(y + q * p.ldc + p.coff + (c8 << 3)) = u;
+                }
+                pq += dpp8; c8 += dc8;
+                if (c8 >= C8) { c8 -= C8; ++pq; }
+            }
         }
     }
     fe_bar(bar_id);                                       // the stage may be overwritten by the next tile

@@ -60,6 +60,7 @@ conv_patch_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap ma
         prefetch_tensormap(&map_b);
     }
     if (warp == 1) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
+    fe_init(p, fe_stage, tid, P_THREADS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -229,6 +230,7 @@ __global__ void __launch_bounds__(S_THREADS, 1) conv_stem_kernel(const ConvParam
         const uint32_t off = (uint32_t)sub * (64 * 128) + swz128(j, within >> 3) + (within & 7) * 2;
         *reinterpret_cast<unsigned short*>(Bs + off) = (j < p.Cout) ? reinterpret_cast<const unsigned short*>(p.w)[(size_t)j * 147 + e] : (unsigned short)0;
     }
+    fe_init(p, fe_stage, tid, S_THREADS);
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -245,20 +247,32 @@ __global__ void __launch_bounds__(S_THREADS, 1) conv_stem_kernel(const ConvParam
         const int pi = tid / pwc, pj = tid - pi * pwc;
         const bool row_used = pi < phc;
         // issue the cp.async loads of tile t's input patch into buffer b
+        // each thread copies the same word slots of every patch: (row, 2*word) of slot k, fixed for the kernel
+        constexpr int MAX_SLOTS = 12;
+        int slot_rr[MAX_SLOTS], slot_e[MAX_SLOTS];
+#pragma unroll
+        for (int k = 0; k < MAX_SLOTS; ++k) {
+            const int i = tid + 128 * k;
+            slot_rr[k] = i < patch_words ? i / in_words : -1;
+            slot_e[k] = i < patch_words ? 2 * (i - (i / in_words) * in_words) : 0;
+        }
+        const int row_elems = 3 * p.W;
         auto load_patch = [&](int t, int b) {
             const int n = t / per, tt_ = t - n * per;
             const int th = tt_ / p.tiles_w, tw = tt_ - th * p.tiles_w;
             const int hi0 = 2 * (2 * th * p.PH - 1) - 3;              // first input row of the patch
-            const int wi0 = 2 * (2 * tw * p.PW - 1) - 3 - 1;          // first input column, one early: even element index
+            const int e0 = 3 * (2 * (2 * tw * p.PW - 1) - 3 - 1);     // first element of a patch row: one pixel early, so even
             const unsigned short* ximg = reinterpret_cast<const unsigned short*>(p.x) + (size_t)n * p.H * p.W * 3;
-            const uint32_t dst0 = smem_u32(inp + b * patch_words);
-            for (int i = tid; i < patch_words; i += 128) {
-                const int rr = i / in_words, ww = i - rr * in_words;
-                const int hi = hi0 + rr;
-                const int e = 3 * wi0 + 2 * ww;                        // element index inside the image row (even)
-                const bool ok = hi >= 0 && hi < p.H && e >= 0 && e + 1 < 3 * p.W;
-                const unsigned short* src = ximg + ((size_t)(ok ? hi : 0) * p.W) * 3 + (ok ? e : 0);
-                cp_async4_zfill(dst0 + 4u * i, src, ok);
+            const uint32_t dst0 = smem_u32(inp + b * patch_words) + 4u * tid;
+#pragma unroll
+            for (int k = 0; k < MAX_SLOTS; ++k) {
+                if (slot_rr[k] >= 0) {
+                    const int hi = hi0 + slot_rr[k];
+                    const int e = e0 + slot_e[k];                      // element index inside the image row (even)
+                    const bool ok = hi >= 0 && hi < p.H && e >= 0 && e + 1 < row_elems;
+                    const unsigned short* src = ximg + (ok ? hi * row_elems + e : 0);
+                    cp_async4_zfill(dst0 + 512u * k, src, ok);
+                }
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
         };
@@ -432,6 +446,7 @@ bool conv_stem_supports(const ConvParams& p) {
     if (p.k != 7 || p.stride != 2 || p.pad != 3 || p.Cin != 3 || p.Cout != 64 || (p.W & 1)) return false;
     int rows, words;
     stem_patch_dims(p, &rows, &words);
+    if (rows * words > 12 * 128) return false;                         // word slots per producer thread
     return S_B_BYTES + 2 * S_A_BYTES + fe_smem_bytes(p) + 2 * rows * words * 4 + 2048 <= P_SMEM_MAX;
 }
 
