@@ -68,7 +68,9 @@ __device__ __forceinline__ void fe_lrn_scale(const ConvParams& p, const float* s
 }
 
 // taddr: TMEM address of this thread's lane, column 0 of the accumulator.  row = 0..127.
-// Called by the 4 epilogue warps together; `release` is invoked by each warp once its TMEM reads are done.
+// Called by the 4 warps of one epilogue group together (a kernel may run two groups on alternate tiles,
+// each with its own stage buffer and named barrier); `release` is invoked by each warp once its TMEM
+// reads are done.
 template <class Release>
 __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, uint32_t taddr, uint8_t* stage, int row, int bar_id,
                                                Release release) {
@@ -240,10 +242,16 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
                 const int pr = active ? pq : npp - 1;
                 const int ppi = pr / p.PW, ppj = pr - ppi * p.PW;
                 const int ph = th * p.PH + ppi, pw = tw * p.PW + ppj;
-                const float* s = pooled + pr * ldp + 2 + (c8 << 3);      // s[0] = x[c-2]
+                const float4* s4 = reinterpret_cast<const float4*>(pooled + pr * ldp + (c8 << 3));   // x[c-4 .. c+11]
+                float w16[16];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float4 f = s4[j];
+                    w16[4 * j] = f.x; w16[4 * j + 1] = f.y; w16[4 * j + 2] = f.z; w16[4 * j + 3] = f.w;
+                }
                 float v[12], sq[12], ss[8], sc[8];
 #pragma unroll
-                for (int j = 0; j < 12; ++j) { v[j] = s[j]; sq[j] = v[j] * v[j]; }
+                for (int j = 0; j < 12; ++j) { v[j] = w16[j + 2]; sq[j] = v[j] * v[j]; }          // v[0] = x[c-2]
 #pragma unroll
                 for (int j = 0; j < 8; ++j) ss[j] = (sq[j] + sq[j + 1]) + (sq[j + 2] + sq[j + 3]) + sq[j + 4];
                 fe_lrn_scale<8>(p, ss, sc);

@@ -24,7 +24,7 @@ namespace dr {
 using namespace ptx;
 
 constexpr int P_A_BYTES = TILE_M * 128;
-constexpr int P_THREADS = 192;          // warp 0 TMA, warp 1 MMA, warps 2-5 epilogue
+constexpr int P_THREADS = 320;          // warp 0 TMA, warp 1 MMA, warps 2-5 and 6-9: two epilogue groups (alternate tiles)
 constexpr int P_MAX_STAGES = 6;
 constexpr int P_SMEM_MAX = 227 * 1024 - 256;
 
@@ -60,7 +60,9 @@ conv_patch_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap ma
         prefetch_tensormap(&map_b);
     }
     if (warp == 1) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
+    const int fe_bytes = fe_smem_bytes(p);
     fe_init(p, fe_stage, tid, P_THREADS);
+    fe_init(p, fe_stage + fe_bytes, tid, P_THREADS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -77,42 +79,56 @@ conv_patch_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap ma
     if (warp == 0) {
         if (lane == 0) {
             const uint32_t tx = (uint32_t)(pwc * phc) * 128u + (uint32_t)p.Nt * 128u;
+            const int nkb = p.k * p.k * cpb;
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
+            uint32_t ready = mbar_test_u32(empty0, 1);
             for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
                 const int n = t / per, tt_ = t - n * per;
                 const int th = tt_ / p.tiles_w, tw = tt_ - th * p.tiles_w;
                 const int h0 = 2 * th * p.PH - 1 - p.pad, w0 = 2 * tw * p.PW - 1 - p.pad;   // stride 1
-                int tap = 0;
-                for (int r = 0; r < p.k && ok; ++r)
-                    for (int q = 0; q < p.k && ok; ++q, ++tap)
-                        for (int c0 = 0; c0 < p.Cin; c0 += 64) {
-                            if (!mbar_wait_u32(empty0 + 8 * s, ph ^ 1, abort_flag)) {
-                                if (!*abort_flag) report_timeout(p.status, 31, t);
-                                *abort_flag = 1;
-                                ok = false;
-                                break;
-                            }
-                            const uint32_t a_dst = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
-                            const uint32_t fb = full0 + 8 * s;
-                            mbar_expect_tx_u32(fb, tx);
-                            tma_load_4d_tile(a_dst, &map_a, fb, c0, w0 + q, h0 + r, n);
-                            tma_load_3d_u32<false>(a_dst + P_A_BYTES, &map_b, fb, c0, tap, 0, 1u);
-                            if (++s == stages) { s = 0; ph ^= 1; }
-                        }
+                int r = 0, q = 0, tap = 0, c0 = 0;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!ready && !mbar_wait_slow_u32(empty0 + 8 * s, ph ^ 1, abort_flag)) {
+                        if (!*abort_flag) report_timeout(p.status, 31, t);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    int s2 = s + 1;
+                    uint32_t ph2 = ph;
+                    if (s2 == stages) { s2 = 0; ph2 ^= 1; }
+                    ready = mbar_test_u32(empty0 + 8 * s2, ph2 ^ 1);
+                    const uint32_t a_dst = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+                    const uint32_t fb = full0 + 8 * s;
+                    mbar_expect_tx_u32(fb, tx);
+                    tma_load_4d_tile(a_dst, &map_a, fb, c0, w0 + q, h0 + r, n);
+                    tma_load_3d_u32<false>(a_dst + P_A_BYTES, &map_b, fb, c0, tap, 0, 1u);
+                    c0 += 64;
+                    const bool wrap_c = c0 >= p.Cin;
+                    c0 = wrap_c ? 0 : c0;
+                    tap += wrap_c ? 1 : 0;
+                    q += wrap_c ? 1 : 0;
+                    const bool wrap_q = q == p.k;
+                    q = wrap_q ? 0 : q;
+                    r += wrap_q ? 1 : 0;
+                    s = s2;
+                    ph = ph2;
+                }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t tfull0 = smem_u32(&sh.tfull[0]), tempty0 = smem_u32(&sh.tempty[0]);
-            const int ntaps = p.k * p.k;
+            const int nkb = p.k * p.k * cpb;
             const int last_nk16 = ((p.Cin - ((cpb - 1) << 6)) + 15) >> 4;
             const uint32_t idesc = make_idesc_bf16(TILE_M, p.Nt);
             int s = 0, it = 0;
             uint32_t ph = 0;
             bool ok = true;
+            uint32_t ready = mbar_test_u32(full0, 0);
             for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
                 const int acc = it & 1, au = it >> 1;
                 if (!mbar_wait_u32(tempty0 + 8 * acc, (au & 1) ^ 1, abort_flag)) {
@@ -123,45 +139,51 @@ conv_patch_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap ma
                 tc_fence_after();
                 const uint32_t d = tmem + (uint32_t)(acc * 256);
                 uint32_t accum = 0;
-                for (int tap = 0; tap < ntaps && ok; ++tap)
-                    for (int cc = 0; cc < cpb; ++cc) {
-                        if (!mbar_wait_u32(full0 + 8 * s, ph, abort_flag)) {
-                            if (!*abort_flag) report_timeout(p.status, 33, t);
-                            *abort_flag = 1;
-                            ok = false;
-                            break;
-                        }
-                        tc_fence_after();
-                        const uint32_t a = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
-                        const uint32_t alo = sdesc_lo(a), blo = sdesc_lo(a + P_A_BYTES);
-                        const int nk16 = (cc == cpb - 1) ? last_nk16 : 4;
-                        umma_bf16_lo<false>(d, alo, blo, idesc, accum, 1u);
-                        accum = 1;
-                        umma_bf16_lo<false>(d, alo + 2, blo + 2, idesc, 1u, nk16 > 1);
-                        umma_bf16_lo<false>(d, alo + 4, blo + 4, idesc, 1u, nk16 > 2);
-                        umma_bf16_lo<false>(d, alo + 6, blo + 6, idesc, 1u, nk16 > 3);
-                        umma_commit_u32<false>(empty0 + 8 * s);
-                        if (++s == stages) { s = 0; ph ^= 1; }
+                int cc = 0;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!ready && !mbar_wait_slow_u32(full0 + 8 * s, ph, abort_flag)) {
+                        if (!*abort_flag) report_timeout(p.status, 33, t);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
                     }
+                    int s2 = s + 1;
+                    uint32_t ph2 = ph;
+                    if (s2 == stages) { s2 = 0; ph2 ^= 1; }
+                    ready = mbar_test_u32(full0 + 8 * s2, ph2);
+                    tc_fence_after();
+                    const uint32_t a = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+                    const uint32_t alo = sdesc_lo(a), blo = sdesc_lo(a + P_A_BYTES);
+                    const int nk16 = (cc == cpb - 1) ? last_nk16 : 4;
+                    cc = (cc + 1 == cpb) ? 0 : cc + 1;
+                    umma_bf16_lo<false>(d, alo, blo, idesc, accum, 1u);
+                    accum = 1;
+                    umma_bf16_lo<false>(d, alo + 2, blo + 2, idesc, 1u, nk16 > 1);
+                    umma_bf16_lo<false>(d, alo + 4, blo + 4, idesc, 1u, nk16 > 2);
+                    umma_bf16_lo<false>(d, alo + 6, blo + 6, idesc, 1u, nk16 > 3);
+                    umma_commit_u32<false>(empty0 + 8 * s);
+                    s = s2;
+                    ph = ph2;
+                }
                 if (ok) umma_commit_u32<false>(tfull0 + 8 * acc);
             }
         }
         __syncwarp();
     } else {
+        // two epilogue groups: group g takes the tiles whose accumulator buffer is g
+        const int g = (warp - 2) >> 2;
         const int q = warp & 3;
         const int row = q * 32 + lane;
-        int it = 0;
-        for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
-            const int acc = it & 1, au = it >> 1;
-            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[acc], au & 1, abort_flag));
+        for (int t = blockIdx.x + g * gridDim.x, au = 0; t < total; t += 2 * gridDim.x, ++au) {
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[g], au & 1, abort_flag));
             if (!ok) {
                 if (!*abort_flag) report_timeout(p.status, 34, t);
                 *abort_flag = 1;
                 break;
             }
             tc_fence_after();
-            uint64_t* te = &sh.tempty[acc];
-            fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * 256), fe_stage, row, 1, [&]() {
+            uint64_t* te = &sh.tempty[g];
+            fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 256), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(te);
             });
@@ -180,7 +202,7 @@ conv_patch_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap ma
 // =====================================================================================
 //                                     stem kernel
 // =====================================================================================
-constexpr int S_THREADS = 288;          // warps 0-3 producers, warp 4 MMA, warps 5-8 epilogue
+constexpr int S_THREADS = 416;          // warps 0-3 producers, warp 4 MMA, warps 5-8 and 9-12: two epilogue groups
 constexpr int S_KSLOTS = 24;            // K slots per tap-row (k * Cin = 21 used)
 constexpr int S_SUBTILES = 3;           // K' = 192 = 3 x 64
 constexpr int S_A_BYTES = S_SUBTILES * P_A_BYTES;          // one im2col tile: 48 KB
@@ -206,7 +228,8 @@ __global__ void __launch_bounds__(S_THREADS, 1) conv_stem_kernel(const ConvParam
     uint8_t* Bs = smem;                                   // [3][64 rows][128 B]
     uint8_t* As = Bs + S_B_BYTES;                         // 2 x [3][128 rows][128 B]
     uint8_t* fe_stage = As + 2 * S_A_BYTES;
-    uint32_t* inp = reinterpret_cast<uint32_t*>(fe_stage + fe_smem_bytes(p));   // 2 x [in_rows][in_words] input patches
+    const int fe_bytes = fe_smem_bytes(p);
+    uint32_t* inp = reinterpret_cast<uint32_t*>(fe_stage + 2 * fe_bytes);       // 2 x [in_rows][in_words] input patches
     const int patch_words = in_rows * in_words;
 
     if (tid == 0) {
@@ -231,6 +254,7 @@ __global__ void __launch_bounds__(S_THREADS, 1) conv_stem_kernel(const ConvParam
         *reinterpret_cast<unsigned short*>(Bs + off) = (j < p.Cout) ? reinterpret_cast<const unsigned short*>(p.w)[(size_t)j * 147 + e] : (unsigned short)0;
     }
     fe_init(p, fe_stage, tid, S_THREADS);
+    fe_init(p, fe_stage + fe_bytes, tid, S_THREADS);
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -346,20 +370,21 @@ __global__ void __launch_bounds__(S_THREADS, 1) conv_stem_kernel(const ConvParam
         }
         __syncwarp();
     } else {
-        const int q = warp & 3;                                        // warps 5-8 -> TMEM lane quarters 1,2,3,0
+        // two epilogue groups (warps 5-8 and 9-12; each covers the four TMEM lane quarters): group g takes
+        // the tiles whose accumulator buffer is g
+        const int g = (warp - 5) >> 2;
+        const int q = warp & 3;
         const int row = q * 32 + lane;
-        int it = 0;
-        for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
-            const int b = it & 1, u = it >> 1;
-            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[b], u & 1, abort_flag));
+        for (int t = blockIdx.x + g * gridDim.x, u = 0; t < total; t += 2 * gridDim.x, ++u) {
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[g], u & 1, abort_flag));
             if (!ok) {
                 if (!*abort_flag) report_timeout(p.status, 44, t);
                 *abort_flag = 1;
                 break;
             }
             tc_fence_after();
-            uint64_t* te = &sh.tempty[b];
-            fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * 64), fe_stage, row, 1, [&]() {
+            uint64_t* te = &sh.tempty[g];
+            fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 64), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(te);
             });
@@ -393,7 +418,7 @@ bool conv_patch_tma_supports(const ConvParams& p) {
     if (!p.patch || !fe_supports(p)) return false;
     if (p.stride != 1 || (p.Cin & 7) || p.Cin < 64 || p.k > 15) return false;
     const int stage_bytes = P_A_BYTES + ((p.Nt * 128 + 1023) & ~1023);
-    return 2 * stage_bytes + fe_smem_bytes(p) + 2048 <= P_SMEM_MAX;
+    return 2 * stage_bytes + 2 * fe_smem_bytes(p) + 2048 <= P_SMEM_MAX;
 }
 
 int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
@@ -425,9 +450,9 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
     }
     if (p.m_tiles <= 0) return DR_OK;
     const int stage_bytes = P_A_BYTES + ((p.Nt * 128 + 1023) & ~1023);
-    int stages = (P_SMEM_MAX - 2048 - fe_smem_bytes(p)) / stage_bytes;
+    int stages = (P_SMEM_MAX - 2048 - 2 * fe_smem_bytes(p)) / stage_bytes;
     if (stages > P_MAX_STAGES) stages = P_MAX_STAGES;
-    int smem_bytes = stages * stage_bytes + fe_smem_bytes(p) + 1024;
+    int smem_bytes = stages * stage_bytes + 2 * fe_smem_bytes(p) + 1024;
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;     // one CTA per SM: each CTA takes all of TMEM
     const int grid = p.m_tiles < num_sms() ? p.m_tiles : num_sms();
     conv_patch_tma_kernel<<<grid, P_THREADS, smem_bytes, stream>>>(p, map_a, map_b, stages, stage_bytes);
@@ -447,7 +472,7 @@ bool conv_stem_supports(const ConvParams& p) {
     int rows, words;
     stem_patch_dims(p, &rows, &words);
     if (rows * words > 12 * 128) return false;                         // word slots per producer thread
-    return S_B_BYTES + 2 * S_A_BYTES + fe_smem_bytes(p) + 2 * rows * words * 4 + 2048 <= P_SMEM_MAX;
+    return S_B_BYTES + 2 * S_A_BYTES + 2 * fe_smem_bytes(p) + 2 * rows * words * 4 + 2048 <= P_SMEM_MAX;
 }
 
 int conv_stem_launch(const ConvParams& p, cudaStream_t stream) {
@@ -460,7 +485,7 @@ int conv_stem_launch(const ConvParams& p, cudaStream_t stream) {
     if (p.m_tiles <= 0) return DR_OK;
     int rows, words;
     stem_patch_dims(p, &rows, &words);
-    const int smem_bytes = S_B_BYTES + 2 * S_A_BYTES + fe_smem_bytes(p) + 2 * rows * words * 4 + 1024;
+    const int smem_bytes = S_B_BYTES + 2 * S_A_BYTES + 2 * fe_smem_bytes(p) + 2 * rows * words * 4 + 1024;
     const int grid = p.m_tiles < num_sms() ? p.m_tiles : num_sms();
     conv_stem_kernel<<<grid, S_THREADS, smem_bytes, stream>>>(p, rows, words);
     count_launch();
