@@ -57,6 +57,55 @@ __device__ __forceinline__ void drain_direct(const ConvParams& p, uint32_t taddr
     }
 }
 
+// Lean epilogue of the common case (bias and/or ReLU only, bf16 out, Cout a multiple of 16, aligned
+// slice): bias comes from a shared-memory copy as float4, the ReLU choice is a template argument, and
+// a thread stores its 64 bytes per 32-column chunk with four 16-byte stores.
+template <bool RELU>
+__device__ __forceinline__ void drain_fast(const ConvParams& p, uint32_t taddr, int ncols, long long m, bool row_ok, int n0,
+                                           const float* bias_s) {
+    uint4* y = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.y) + m * p.ldc + p.coff + n0);
+    const float4* b4 = reinterpret_cast<const float4*>(bias_s + n0);
+    int c = 0;
+    for (; c + 32 <= ncols; c += 32) {
+        uint32_t r[32];
+        tmem_ld_x32(taddr + c, r);
+        tmem_ld_wait();
+        uint32_t o[16];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float4 b = b4[(c >> 2) + q];
+            float v0 = __uint_as_float(r[4 * q]) + b.x, v1 = __uint_as_float(r[4 * q + 1]) + b.y;
+            float v2 = __uint_as_float(r[4 * q + 2]) + b.z, v3 = __uint_as_float(r[4 * q + 3]) + b.w;
+            if (RELU) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); v2 = fmaxf(v2, 0.f); v3 = fmaxf(v3, 0.f); }
+            o[2 * q] = pack_bf16(v0, v1);
+            o[2 * q + 1] = pack_bf16(v2, v3);
+        }
+        if (row_ok) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) y[(c >> 3) + q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+        }
+    }
+    if (c < ncols) {   // 16-column tail
+        uint32_t r[16];
+        tmem_ld_x16(taddr + c, r);
+        tmem_ld_wait();
+        uint32_t o[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float4 b = b4[(c >> 2) + q];
+            float v0 = __uint_as_float(r[4 * q]) + b.x, v1 = __uint_as_float(r[4 * q + 1]) + b.y;
+            float v2 = __uint_as_float(r[4 * q + 2]) + b.z, v3 = __uint_as_float(r[4 * q + 3]) + b.w;
+            if (RELU) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); v2 = fmaxf(v2, 0.f); v3 = fmaxf(v3, 0.f); }
+            o[2 * q] = pack_bf16(v0, v1);
+            o[2 * q + 1] = pack_bf16(v2, v3);
+        }
+        if (row_ok) {
+            y[(c >> 3)] = make_uint4(o[0], o[1], o[2], o[3]);
+            y[(c >> 3) + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+        }
+    }
+}
+
 // =====================================================================================
 //                                   gather kernel
 // =====================================================================================
@@ -293,8 +342,9 @@ int conv_umma_gather_launch(const ConvParams& p, cudaStream_t stream) {
 // few dozen instructions: nested tap / channel-block loops instead of divisions, barrier and
 // stage addresses advanced incrementally, descriptors assembled from 32-bit halves.
 constexpr int T_MAX_STAGES = 8;   // stage = A tile (16 KB) + B tile; as many as fit
-constexpr int T_THREADS = 192;    // warp 0: TMA producer, warp 1: MMA issue + TMEM owner, warps 2-5: epilogue
-constexpr int T_SMEM_MAX = 227 * 1024 - 256;
+constexpr int T_THREADS = 320;    // warp 0: TMA producer, warp 1: MMA issue + TMEM owner, warps 2-5 / 6-9: two epilogue groups
+constexpr int T_BIAS_MAX = 1024;  // channels of the shared-memory bias copy (lean epilogue)
+constexpr int T_SMEM_MAX = 227 * 1024 - 5120;   // dynamic part; the static part holds barriers and the bias copy
 constexpr int T_ACC_COLS = 256;   // columns per accumulator buffer; two buffers = all 512 TMEM columns
 
 struct TmaShared {
@@ -315,8 +365,13 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     __shared__ TmaShared sh;
+    __shared__ __align__(16) float bias_s[T_BIAS_MAX];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int stage_bytes = kpb * sub_bytes;
+    // lean epilogue: bias/ReLU only, bf16 out, every 16-column chunk inside Cout, aligned slice
+    const bool lean = !(p.flags & (DR_RESIDUAL | DR_OUT_F32)) && (p.Cout & 15) == 0 && p.Cout <= T_BIAS_MAX && (p.ldc & 7) == 0 && (p.coff & 7) == 0;
+    if (lean)
+        for (int i = tid; i < p.Cout; i += T_THREADS) bias_s[i] = (p.flags & DR_BIAS) ? p.bias[i] : 0.f;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;        // 0 issues the MMAs
     const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int nunits = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
@@ -466,17 +521,17 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------ epilogue warps: TMEM lane quarter = warp % 4
+        // ------------------------------------------------ epilogue: two groups of four warps; group g drains
+        // accumulator buffer g, i.e. every other tile of this CTA.  TMEM lane quarter = warp % 4.
+        const int g = (warp - 2) >> 2;
         const int q = warp & 3;
         const int row = q * 32 + lane;
-        int it = 0;
-        for (int t = unit; t < total; t += nunits, ++it) {
+        for (int t = unit + g * nunits, au = 0; t < total; t += 2 * nunits, ++au) {
             const int nb = t / m_units, mu = t - nb * m_units;
             const int n0 = nb * p.Nt;
             const int Nj = min(p.Nt, cout16 - n0);
             const int mt = PAIR ? 2 * mu + (int)rank : mu;
-            const int acc = it & 1, au = it >> 1;
-            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[acc], au & 1, abort_flag));
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[g], au & 1, abort_flag));
             if (!ok) {
                 if (!*abort_flag) report_timeout(p.status, 14, t);
                 *abort_flag = 1;
@@ -484,12 +539,19 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             }
             tc_fence_after();
             const long long m = (long long)mt * TILE_M + row;
-            drain_direct(p, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * T_ACC_COLS), Nj, m, mt < p.m_tiles && m < p.M, n0);
+            const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * T_ACC_COLS);
+            const bool row_ok = mt < p.m_tiles && m < p.M;
+            if (lean) {
+                if (p.flags & DR_RELU) drain_fast<true>(p, taddr, Nj, m, row_ok, n0, bias_s);
+                else drain_fast<false>(p, taddr, Nj, m, row_ok, n0, bias_s);
+            } else {
+                drain_direct(p, taddr, Nj, m, row_ok, n0);
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
-                if (PAIR) mbar_arrive_leader(&sh.tempty[acc]);
-                else mbar_arrive(&sh.tempty[acc]);
+                if (PAIR) mbar_arrive_leader(&sh.tempty[g]);
+                else mbar_arrive(&sh.tempty[g]);
             }
         }
     }
