@@ -68,8 +68,22 @@ int conv_make_params(const dr_conv_desc* d, int B, int H, int W, const void* x, 
     if (staged) {
         p.Nt = cout16; p.n_blocks = 1;
     } else {
-        p.n_blocks = (cout16 + 255) / 256;
-        p.Nt = ((cout16 + p.n_blocks - 1) / p.n_blocks + 15) / 16 * 16;
+        // Split N into near-equal blocks of at most 256 columns.  Among the smallest block counts pick the one
+        // with the lowest estimated time: rounds of the persistent grid (CTA pairs for long-K layers) times the
+        // measured cost of a k-block, about 0.2 us of fixed hand-shake plus 1 ns per output column.
+        const long long m_tiles = (p.M + TILE_M - 1) / TILE_M;
+        const bool pairs = p.K >= 1024 && m_tiles >= 2;
+        const long long capacity = pairs ? num_sms() / 2 : num_sms();
+        const long long m_units = pairs ? (m_tiles + 1) / 2 : m_tiles;
+        const int nb_min = (cout16 + 255) / 256;
+        double best = -1.0;
+        for (int nb = nb_min; nb <= nb_min + 2 && nb * 16 <= cout16; ++nb) {
+            const int nt = ((cout16 + nb - 1) / nb + 15) / 16 * 16;
+            if ((long long)nt * (nb - 1) >= cout16) continue;          // last block would be empty
+            const long long rounds = (m_units * nb + capacity - 1) / capacity;
+            const double cost = (double)rounds * (0.20 + 0.00094 * nt);
+            if (best < 0 || cost < best * 0.97) { best = cost; p.n_blocks = nb; p.Nt = nt; }
+        }
     }
     if (f & DR_POOL) {
         static const int cand[][2] = {{3, 8}, {4, 6}, {5, 5}, {2, 12}, {8, 3}, {6, 4}};
