@@ -159,6 +159,34 @@ __global__ void maxpool_kernel(int B, int H, int W, int C8, int Ho, int Wo, int 
         }
     }
 }
+// Without argmax the maximum is taken on packed bf16 pairs (4 instructions per tap and 8 channels).
+__global__ void maxpool_noarg_kernel(int B, int H, int W, int C8, int Ho, int Wo, int k, int s, int p,
+                                     const uint4* __restrict__ x, uint4* __restrict__ y) {
+    const size_t total = (size_t)B * Ho * Wo * C8;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int c8 = (int)(i % C8);
+        size_t q = i / C8;
+        const int wo = (int)(q % Wo); q /= Wo;
+        const int ho = (int)(q % Ho);
+        const int n = (int)(q / Ho);
+        uint4 m = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // -inf: padding never wins
+        __nv_bfloat162* mm = reinterpret_cast<__nv_bfloat162*>(&m);
+        for (int r = 0; r < k; ++r) {
+            const int hi = ho * s - p + r;
+            if (hi < 0 || hi >= H) continue;
+            for (int t = 0; t < k; ++t) {
+                const int wi = wo * s - p + t;
+                if (wi < 0 || wi >= W) continue;
+                const uint4 v = __ldg(x + (((size_t)n * H + hi) * W + wi) * C8 + c8);
+                const __nv_bfloat162* vv = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) mm[j] = __hmax2(mm[j], vv[j]);
+            }
+        }
+        y[i] = m;
+    }
+}
 __global__ void maxpool_scalar_kernel(int B, int H, int W, int C, int Ho, int Wo, int k, int s, int p,
                                       const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
                                       int32_t* __restrict__ argmax) {
@@ -410,7 +438,9 @@ int dr_maxpool(int B, int H, int W, int C, int k, int s, int p, const void* x, v
     const size_t n = (size_t)B * Ho * Wo * C;
     if (n == 0) return DR_OK;
     DR_REQUIRE(aligned16(x) && aligned16(y) && (!argmax || aligned16(argmax)), DR_ERR_ALIGNMENT);
-    if (C % 8 == 0)
+    if (C % 8 == 0 && !argmax)
+        maxpool_noarg_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C / 8, Ho, Wo, k, s, p, (const uint4*)x, (uint4*)y);
+    else if (C % 8 == 0)
         maxpool_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C / 8, Ho, Wo, k, s, p, (const uint4*)x, (uint4*)y, argmax);
     else
         maxpool_scalar_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C, Ho, Wo, k, s, p, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, argmax);

@@ -61,6 +61,9 @@ def test_maxpool_bit_exact_with_argmax(dr, O, shape):
     dr.dr_maxpool(B, H, W, Cc, 3, 2, 1, to_dev_bf16(x), y, arg)
     assert np.array_equal(to_host(y), ref)
     assert np.array_equal(arg.cpu().numpy(), ref_arg)
+    y2 = _empty_like_bf16(ref.shape)
+    dr.dr_maxpool(B, H, W, Cc, 3, 2, 1, to_dev_bf16(x), y2, None)     # the path without argmax (packed maxima)
+    assert np.array_equal(to_host(y2), ref)
 
 
 def test_maxpool_other_geometry(dr, O):
