@@ -44,7 +44,7 @@ __device__ __forceinline__ void tma_load_4d_tile(uint32_t dst, const CUtensorMap
 
 __global__ void __launch_bounds__(P_THREADS, 1)
 conv_patch_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const int stages,
-                      const int stage_bytes) {
+                      const int stage_bytes, const int groups) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     __shared__ PatchShared sh;
@@ -62,7 +62,7 @@ conv_patch_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap ma
     if (warp == 1) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
     const int fe_bytes = fe_smem_bytes(p);
     fe_init(p, fe_stage, tid, P_THREADS);
-    fe_init(p, fe_stage + fe_bytes, tid, P_THREADS);
+    if (groups > 1) fe_init(p, fe_stage + fe_bytes, tid, P_THREADS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -170,23 +170,29 @@ conv_patch_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap ma
         }
         __syncwarp();
     } else {
-        // two epilogue groups: group g takes the tiles whose accumulator buffer is g
+        // epilogue groups of four warps: with two groups, group g takes the tiles whose accumulator buffer is g;
+        // with one group (more shared memory left for pipeline stages) it takes every tile
         const int g = (warp - 2) >> 2;
         const int q = warp & 3;
         const int row = q * 32 + lane;
-        for (int t = blockIdx.x + g * gridDim.x, au = 0; t < total; t += 2 * gridDim.x, ++au) {
-            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[g], au & 1, abort_flag));
-            if (!ok) {
-                if (!*abort_flag) report_timeout(p.status, 34, t);
-                *abort_flag = 1;
-                break;
+        if (g < groups) {
+            for (int it = g;; it += groups) {
+                const int t = blockIdx.x + it * gridDim.x;
+                if (t >= total) break;
+                const int acc = it & 1, au = it >> 1;
+                const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[acc], au & 1, abort_flag));
+                if (!ok) {
+                    if (!*abort_flag) report_timeout(p.status, 34, t);
+                    *abort_flag = 1;
+                    break;
+                }
+                tc_fence_after();
+                uint64_t* te = &sh.tempty[acc];
+                fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * 256), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(te);
+                });
             }
-            tc_fence_after();
-            uint64_t* te = &sh.tempty[g];
-            fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 256), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(te);
-            });
         }
     }
     tc_fence_before();
@@ -418,7 +424,7 @@ bool conv_patch_tma_supports(const ConvParams& p) {
     if (!p.patch || !fe_supports(p)) return false;
     if (p.stride != 1 || (p.Cin & 7) || p.Cin < 64 || p.k > 15) return false;
     const int stage_bytes = P_A_BYTES + ((p.Nt * 128 + 1023) & ~1023);
-    return 2 * stage_bytes + 2 * fe_smem_bytes(p) + 2048 <= P_SMEM_MAX;
+    return 2 * stage_bytes + fe_smem_bytes(p) + 2048 <= P_SMEM_MAX;
 }
 
 int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
@@ -450,12 +456,17 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
     }
     if (p.m_tiles <= 0) return DR_OK;
     const int stage_bytes = P_A_BYTES + ((p.Nt * 128 + 1023) & ~1023);
-    int stages = (P_SMEM_MAX - 2048 - 2 * fe_smem_bytes(p)) / stage_bytes;
+    // two epilogue groups when that still leaves three pipeline stages, else one group and the extra stages
+    // (conv2 of GoogLeNet: 350 us with 2 groups / 3 stages, 361 us with 1 group / 4 stages)
+    int groups = (P_SMEM_MAX - 2048 - 2 * fe_smem_bytes(p)) / stage_bytes >= 3 ? 2 : 1;
+    if (getenv("DR_PATCH_GROUPS")) groups = atoi(getenv("DR_PATCH_GROUPS")) == 2 ? 2 : 1;
+    if (groups == 2 && (P_SMEM_MAX - 2048 - 2 * fe_smem_bytes(p)) / stage_bytes < 2) groups = 1;
+    int stages = (P_SMEM_MAX - 2048 - groups * fe_smem_bytes(p)) / stage_bytes;
     if (stages > P_MAX_STAGES) stages = P_MAX_STAGES;
-    int smem_bytes = stages * stage_bytes + 2 * fe_smem_bytes(p) + 1024;
+    int smem_bytes = stages * stage_bytes + groups * fe_smem_bytes(p) + 1024;
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;     // one CTA per SM: each CTA takes all of TMEM
     const int grid = p.m_tiles < num_sms() ? p.m_tiles : num_sms();
-    conv_patch_tma_kernel<<<grid, P_THREADS, smem_bytes, stream>>>(p, map_a, map_b, stages, stage_bytes);
+    conv_patch_tma_kernel<<<grid, P_THREADS, smem_bytes, stream>>>(p, map_a, map_b, stages, stage_bytes, groups);
     count_launch();
     return launch_status();
 }
