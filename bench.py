@@ -175,13 +175,17 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--batch", type=int, default=None, help="default 256 (GoogLeNet), 128 (ResNet-50)")
+    ap.add_argument("--arch", default="googlenet", choices=["googlenet", "resnet50"],
+                    help="googlenet = the headline workload; resnet50 = the BN-folded bottleneck network (context)")
     ap.add_argument("--layers-out", default=None, help="write the per-layer table (us, roofline) as JSON")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layer", default=None,
                     help="time ONE slim layer of the network (e.g. conv1, conv2, 3b.m5, 4e.3x3) instead of the whole step; "
                          "this is the small case the ncu captures under profiles/ run")
     args = ap.parse_args()
+    if args.batch is None:
+        args.batch = 256 if args.arch == "googlenet" else 128
     if args.impl == "reference":
         return run_reference(args)
     if args.layer:
@@ -217,10 +221,13 @@ def main():
 
     B = args.batch
     pk, pk_kind = peaks()
-    params = P.googlenet_params(0)
+    resnet = args.arch == "resnet50"
+    params = P.resnet50_params(0) if resnet else P.googlenet_params(0)
+    arch_id = dr.DR_ARCH_RESNET50 if resnet else dr.DR_ARCH_GOOGLENET
+    arch_name = "ResNet-50 (BN folded)" if resnet else "GoogLeNet-slim"
 
     def make_net(mode, batch):
-        net = dr.Net(dr.DR_ARCH_GOOGLENET, mode, batch)
+        net = dr.Net(arch_id, mode, batch)
         keep = []
         for i in range(net.dr_net_num_params()):
             name, dims, is_f32, count = net.dr_net_param_spec(i)
@@ -350,7 +357,7 @@ def main():
     achieved = top["gflop"] / top["us"] * 1e3 if top else 0.0   # GFLOP/us = PFLOP/s
     # DRAM bytes of that launch from the ncu capture in profiles/conv_umma_tma_kernel_3b_merged5x5_bs256.md
     # (dram__bytes_read.sum + dram__bytes_write.sum); valid for batch 256 only
-    traffic = NCU_TRAFFIC_3B_M5 if (top and top["name"] == "3b.m5" and B == 256) else None
+    traffic = NCU_TRAFFIC_3B_M5 if (top and not resnet and top["name"] == "3b.m5" and B == 256) else None
     roofline = {"bound": "tensor", "kernel": f"conv_umma_tma_kernel, launch {top['name'] if top else '-'} (largest of {len(tma)} tensor-bound launches per step)",
                 "achieved": achieved, "peak": pk["bf16_tflops_sustained"], "peak_kind": f"{pk_kind} sustained bf16 (kernel timed inside a long step)",
                 "unit": "TFLOP/s", "frac": achieved / pk["bf16_tflops_sustained"], "traffic": traffic,
@@ -403,10 +410,10 @@ def main():
             json.dump({"batch": B, "layers": rows, "net_roofline": net_roofline}, f, indent=1)
 
     print(json.dumps({
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": METRIC if not resnet else "slim ResNet-50 forward throughput", "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"GoogLeNet-slim forward, batch {B} per GPU, 224x224x3 N(0,1) bf16, He-normal weights (configs[3])",
+        "config": {"workload": f"{arch_name} forward, batch {B} per GPU, 224x224x3 N(0,1) bf16, He-normal weights (configs[{4 if resnet else 3}])",
                    "l2": "256 MB buffer written between timed iterations (L2 flush)", "replicas": world},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": logits_host.numel() * 4},
         "gpu_launches": int(launches),

@@ -60,10 +60,13 @@ __device__ __forceinline__ void drain_direct(const ConvParams& p, uint32_t taddr
 // Lean epilogue of the common case (bias and/or ReLU only, bf16 out, Cout a multiple of 16, aligned
 // slice): bias comes from a shared-memory copy as float4, the ReLU choice is a template argument, and
 // a thread stores its 64 bytes per 32-column chunk with four 16-byte stores.
-template <bool RELU>
+// MODE 0: +bias;  1: +bias, ReLU;  2: +bias, +residual;  3: +bias, +residual, ReLU.
+template <int MODE>
 __device__ __forceinline__ void drain_fast(const ConvParams& p, uint32_t taddr, int ncols, long long m, bool row_ok, int n0,
                                            const float* bias_s) {
+    constexpr bool RELU = (MODE & 1) != 0, RES = (MODE & 2) != 0;
     uint4* y = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.y) + m * p.ldc + p.coff + n0);
+    const uint4* res = reinterpret_cast<const uint4*>(p.residual + (RES && row_ok ? m * p.Cout + n0 : 0));
     const float4* b4 = reinterpret_cast<const float4*>(bias_s + n0);
     int c = 0;
     for (; c + 32 <= ncols; c += 32) {
@@ -71,11 +74,20 @@ __device__ __forceinline__ void drain_fast(const ConvParams& p, uint32_t taddr, 
         tmem_ld_x32(taddr + c, r);
         tmem_ld_wait();
         uint32_t o[16];
+        uint32_t rr[16];
+        if (RES && row_ok) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint4 u = __ldg(res + (c >> 3) + q);
+                rr[4 * q] = u.x; rr[4 * q + 1] = u.y; rr[4 * q + 2] = u.z; rr[4 * q + 3] = u.w;
+            }
+        }
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
             const float4 b = b4[(c >> 2) + q];
             float v0 = __uint_as_float(r[4 * q]) + b.x, v1 = __uint_as_float(r[4 * q + 1]) + b.y;
             float v2 = __uint_as_float(r[4 * q + 2]) + b.z, v3 = __uint_as_float(r[4 * q + 3]) + b.w;
+            if (RES && row_ok) { v0 += bf16_lo(rr[2 * q]); v1 += bf16_hi(rr[2 * q]); v2 += bf16_lo(rr[2 * q + 1]); v3 += bf16_hi(rr[2 * q + 1]); }
             if (RELU) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); v2 = fmaxf(v2, 0.f); v3 = fmaxf(v3, 0.f); }
             o[2 * q] = pack_bf16(v0, v1);
             o[2 * q + 1] = pack_bf16(v2, v3);
@@ -90,11 +102,20 @@ __device__ __forceinline__ void drain_fast(const ConvParams& p, uint32_t taddr, 
         tmem_ld_x16(taddr + c, r);
         tmem_ld_wait();
         uint32_t o[8];
+        uint32_t rr[8];
+        if (RES && row_ok) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const uint4 u = __ldg(res + (c >> 3) + q);
+                rr[4 * q] = u.x; rr[4 * q + 1] = u.y; rr[4 * q + 2] = u.z; rr[4 * q + 3] = u.w;
+            }
+        }
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const float4 b = b4[(c >> 2) + q];
             float v0 = __uint_as_float(r[4 * q]) + b.x, v1 = __uint_as_float(r[4 * q + 1]) + b.y;
             float v2 = __uint_as_float(r[4 * q + 2]) + b.z, v3 = __uint_as_float(r[4 * q + 3]) + b.w;
+            if (RES && row_ok) { v0 += bf16_lo(rr[2 * q]); v1 += bf16_hi(rr[2 * q]); v2 += bf16_lo(rr[2 * q + 1]); v3 += bf16_hi(rr[2 * q + 1]); }
             if (RELU) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); v2 = fmaxf(v2, 0.f); v3 = fmaxf(v3, 0.f); }
             o[2 * q] = pack_bf16(v0, v1);
             o[2 * q + 1] = pack_bf16(v2, v3);
@@ -343,8 +364,8 @@ int conv_umma_gather_launch(const ConvParams& p, cudaStream_t stream) {
 // stage addresses advanced incrementally, descriptors assembled from 32-bit halves.
 constexpr int T_MAX_STAGES = 8;   // stage = A tile (16 KB) + B tile; as many as fit
 constexpr int T_THREADS = 320;    // warp 0: TMA producer, warp 1: MMA issue + TMEM owner, warps 2-5 / 6-9: two epilogue groups
-constexpr int T_BIAS_MAX = 1024;  // channels of the shared-memory bias copy (lean epilogue)
-constexpr int T_SMEM_MAX = 227 * 1024 - 5120;   // dynamic part; the static part holds barriers and the bias copy
+constexpr int T_BIAS_MAX = 2048;  // channels of the shared-memory bias copy (lean epilogue)
+constexpr int T_SMEM_MAX = 227 * 1024 - 9216;   // dynamic part; the static part holds barriers and the bias copy
 constexpr int T_ACC_COLS = 256;   // columns per accumulator buffer; two buffers = all 512 TMEM columns
 
 struct TmaShared {
@@ -368,8 +389,11 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
     __shared__ __align__(16) float bias_s[T_BIAS_MAX];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int stage_bytes = kpb * sub_bytes;
-    // lean epilogue: bias/ReLU only, bf16 out, every 16-column chunk inside Cout, aligned slice
-    const bool lean = !(p.flags & (DR_RESIDUAL | DR_OUT_F32)) && (p.Cout & 15) == 0 && p.Cout <= T_BIAS_MAX && (p.ldc & 7) == 0 && (p.coff & 7) == 0;
+    // lean epilogue: bias, ReLU, residual (+ReLU); bf16 out, every 16-column chunk inside Cout, aligned slice.
+    // (ReLU before a residual add is the one order it does not take.)
+    const bool lean = !(p.flags & DR_OUT_F32) && !((p.flags & DR_RESIDUAL) && (p.flags & DR_RELU)) && (p.Cout & 15) == 0 &&
+                      p.Cout <= T_BIAS_MAX && (p.ldc & 7) == 0 && (p.coff & 7) == 0;
+    const int lean_mode = (p.flags & DR_RESIDUAL) ? ((p.flags & DR_RELU_AFTER_RESIDUAL) ? 3 : 2) : ((p.flags & DR_RELU) ? 1 : 0);
     if (lean)
         for (int i = tid; i < p.Cout; i += T_THREADS) bias_s[i] = (p.flags & DR_BIAS) ? p.bias[i] : 0.f;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;        // 0 issues the MMAs
@@ -542,8 +566,10 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * T_ACC_COLS);
             const bool row_ok = mt < p.m_tiles && m < p.M;
             if (lean) {
-                if (p.flags & DR_RELU) drain_fast<true>(p, taddr, Nj, m, row_ok, n0, bias_s);
-                else drain_fast<false>(p, taddr, Nj, m, row_ok, n0, bias_s);
+                if (lean_mode == 1) drain_fast<1>(p, taddr, Nj, m, row_ok, n0, bias_s);
+                else if (lean_mode == 3) drain_fast<3>(p, taddr, Nj, m, row_ok, n0, bias_s);
+                else if (lean_mode == 0) drain_fast<0>(p, taddr, Nj, m, row_ok, n0, bias_s);
+                else drain_fast<2>(p, taddr, Nj, m, row_ok, n0, bias_s);
             } else {
                 drain_direct(p, taddr, Nj, m, row_ok, n0);
             }
