@@ -176,7 +176,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=None, help="default 256 (GoogLeNet), 128 (ResNet-50)")
-    ap.add_argument("--arch", default="googlenet", choices=["googlenet", "resnet50"],
+    ap.add_argument("--arch", default="googlenet", choices=["googlenet", "resnet50", "googlenet_paper"],
                     help="googlenet = the headline workload; resnet50 = the BN-folded bottleneck network (context)")
     ap.add_argument("--layers-out", default=None, help="write the per-layer table (us, roofline) as JSON")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -221,10 +221,11 @@ def main():
 
     B = args.batch
     pk, pk_kind = peaks()
-    resnet = args.arch == "resnet50"
-    params = P.resnet50_params(0) if resnet else P.googlenet_params(0)
-    arch_id = dr.DR_ARCH_RESNET50 if resnet else dr.DR_ARCH_GOOGLENET
-    arch_name = "ResNet-50 (BN folded)" if resnet else "GoogLeNet-slim"
+    resnet = args.arch != "googlenet"          # any context arm: no headline metric, no stored ncu traffic
+    params = {"googlenet": P.googlenet_params, "resnet50": P.resnet50_params, "googlenet_paper": P.googlenet_paper_params}[args.arch](0)
+    arch_id = {"googlenet": dr.DR_ARCH_GOOGLENET, "resnet50": dr.DR_ARCH_RESNET50, "googlenet_paper": dr.DR_ARCH_GOOGLENET_PAPER}[args.arch]
+    cfg_name = {"googlenet": "configs[3]", "resnet50": "configs[4]", "googlenet_paper": "Section 3.2 form, context"}[args.arch]
+    arch_name = {"googlenet": "GoogLeNet-slim", "resnet50": "ResNet-50 (BN folded)", "googlenet_paper": "GoogLeNet, paper-form branch slimming"}[args.arch]
 
     def make_net(mode, batch):
         net = dr.Net(arch_id, mode, batch)
@@ -410,10 +411,10 @@ def main():
             json.dump({"batch": B, "layers": rows, "net_roofline": net_roofline}, f, indent=1)
 
     print(json.dumps({
-        "metric": METRIC if not resnet else "slim ResNet-50 forward throughput", "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": METRIC if not resnet else f"{arch_name} forward throughput", "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{arch_name} forward, batch {B} per GPU, 224x224x3 N(0,1) bf16, He-normal weights (configs[{4 if resnet else 3}])",
+        "config": {"workload": f"{arch_name} forward, batch {B} per GPU, 224x224x3 N(0,1) bf16, He-normal weights ({cfg_name})",
                    "l2": "256 MB buffer written between timed iterations (L2 flush)", "replicas": world},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": logits_host.numel() * 4},
         "gpu_launches": int(launches),

@@ -59,6 +59,22 @@ def googlenet_params(seed=0):
     return p
 
 
+def googlenet_paper_params(seed=0):
+    """GoogLeNet slimmed the paper's way: per module 1x1 (Cin -> c3r/2), 3x3 (-> c3+c1), 1x1 (Cin -> c5r),
+    5x5 (-> c5+pp); stem and classifier as in googlenet_params."""
+    p = {}
+    p.update(conv_params(seed, "conv1", 64, 7, 3))
+    p.update(conv_params(seed, "conv2r", 64, 1, 64))
+    p.update(conv_params(seed, "conv2", 192, 3, 64))
+    for m, (cin, c1, c3r, c3, c5r, c5, pp) in INCEPTION_V1.items():
+        p.update(conv_params(seed, f"{m}.p3r", c3r // 2, 1, cin))
+        p.update(conv_params(seed, f"{m}.p3", c3 + c1, 3, c3r // 2))
+        p.update(conv_params(seed, f"{m}.p5r", c5r, 1, cin))
+        p.update(conv_params(seed, f"{m}.p5", c5 + pp, 5, c5r))
+    p.update(conv_params(seed, "fc", 1000, 1, 1024))
+    return p
+
+
 def resnet50_conv_names():
     """(name, Cout, k, Cin) of every convolution, in execution order."""
     out = [("conv1", 64, 7, 3)]

@@ -111,6 +111,38 @@ def googlenet_steps(params):
     return steps
 
 
+def googlenet_paper_steps(params):
+    """GoogLeNet with the paper's own branch slimming (Section 3.2, Method / Branch Reducing / Tensor-Branch
+    Slimming): per module a 1x1 reducer with half the original width feeding a 3x3 convolution of c3 + c1
+    outputs, and the original 5x5 reducer feeding a 5x5 convolution of c5 + pp outputs; the two branch
+    outputs are concatenated.  Each convolution is followed by its own ReLU pass."""
+    def conv2r(x):
+        return O.relu(_conv(params, "conv2r", x, 1, 0))
+
+    def conv2(x):
+        y = O.lrn(O.relu(_conv(params, "conv2", x, 1, 1)), **_LRN)
+        return O.maxpool(y, 3, 2, 1)[0]
+
+    steps = stem_steps(params) + [Step("conv2r", ["conv1"], conv2r), Step("conv2", ["conv2r"], conv2)]
+    src = "conv2"
+    for m in _INCEPTION:
+        steps += [
+            Step(f"{m}.p3r", [src], lambda x, m=m: O.relu(_conv(params, f"{m}.p3r", x, 1, 0))),
+            Step(f"{m}.p3", [f"{m}.p3r"], lambda x, m=m: O.relu(_conv(params, f"{m}.p3", x, 1, 1))),
+            Step(f"{m}.p5r", [src], lambda x, m=m: O.relu(_conv(params, f"{m}.p5r", x, 1, 0))),
+            Step(f"{m}.p5", [f"{m}.p5r"], lambda x, m=m: O.relu(_conv(params, f"{m}.p5", x, 1, 2))),
+            Step(m, [f"{m}.p3", f"{m}.p5"], lambda a, b: O.concat([a, b]), virtual=True),
+        ]
+        src = m
+        if m in ("3b", "4e"):
+            name = "pool3" if m == "3b" else "pool4"
+            steps.append(Step(name, [src], lambda x: O.maxpool(x, 3, 2, 1)[0]))
+            src = name
+    steps.append(Step("avgpool", [src], O.avgpool_global))
+    steps.append(Step("fc", ["avgpool"], lambda x: _conv(params, "fc", x, 1, 0), stored_bf16=False))
+    return steps
+
+
 def resnet50_steps(params, eps=1e-5):
     def conv1(x):
         y = O.relu(_conv_bn_scale(params, "conv1", x, 2, 3, eps))

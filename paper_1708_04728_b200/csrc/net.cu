@@ -257,6 +257,68 @@ static void build_googlenet(dr_net* n) {
     n->t_logits = add_conv(n, "fc", t, 1, 1, 0, 1000, DR_BIAS | DR_OUT_F32, w, b);
 }
 
+// GoogLeNet with the paper's own branch slimming (Section 3.2): per module the 3x3 reducer is halved
+// ("branch reducing"), the 1x1 branch is absorbed into the 3x3 convolution, whose output widens from c3 to
+// c3 + c1 ("tensor-branch slimming"), and the pooling branch is absorbed into the 5x5 convolution, which keeps
+// its reducer and widens from c5 to c5 + pp.  Two branches instead of four, same output width.  The paper
+// re-trains these layers; here they carry random weights and the unslimmed mode runs the same two-branch
+// topology with every ReLU / concat as its own launch.
+static void build_googlenet_paper(dr_net* n) {
+    const bool slim = n->mode == DR_MODE_SLIM;
+    const int x = n->tensor(n->B, n->H, n->W, 3, 0, true);
+    n->t_input = x;
+    auto conv_p = [&](const std::string& name, int cout, int k, int cin, PRef* w, PRef* b) {
+        *w = rawref(n->filt(name, cout, k, cin));
+        *b = rawref(n->vec(name + ".b", cout));
+    };
+    auto cr = [&](const std::string& name, int in, int k, int pad, int cout, int out = -2, int coff = 0) {
+        PRef w, b;
+        conv_p(name, cout, k, n->T(in).C, &w, &b);
+        if (slim) return add_conv(n, name, in, k, 1, pad, cout, BR, w, b, out, coff);
+        const int t = add_conv(n, name + ".conv", in, k, 1, pad, cout, DR_BIAS, w, b);
+        const int r = add_simple(n, OP_RELU, name, t);
+        if (out != -2) { add_concat(n, name + ".cat", r, out, coff); return out; }
+        return r;
+    };
+    PRef w, b;
+    int t;
+    conv_p("conv1", 64, 7, 3, &w, &b);
+    if (slim) {
+        t = add_conv(n, "conv1", x, 7, 2, 3, 64, BR | DR_POOL | DR_LRN, w, b);
+    } else {
+        t = add_conv(n, "conv1.conv", x, 7, 2, 3, 64, DR_BIAS, w, b);
+        t = add_simple(n, OP_RELU, "conv1.relu", t);
+        t = add_simple(n, OP_MAXPOOL, "conv1.pool", t);
+        t = add_simple(n, OP_LRN, "conv1", t);
+    }
+    t = cr("conv2r", t, 1, 0, 64);
+    conv_p("conv2", 192, 3, 64, &w, &b);
+    if (slim) {
+        t = add_conv(n, "conv2", t, 3, 1, 1, 192, BR | DR_POOL | DR_LRN | DR_LRN_BEFORE_POOL, w, b);
+    } else {
+        t = add_conv(n, "conv2.conv", t, 3, 1, 1, 192, DR_BIAS, w, b);
+        t = add_simple(n, OP_RELU, "conv2.relu", t);
+        t = add_simple(n, OP_LRN, "conv2.lrn", t);
+        t = add_simple(n, OP_MAXPOOL, "conv2", t);
+    }
+    for (const Inc& m : kInception) {
+        const std::string mn = m.name;
+        const Tensor ti = n->T(t);
+        const int a3 = m.c3 + m.c1, a5 = m.c5 + m.pp;
+        const int out = n->tensor(ti.B, ti.H, ti.W, a3 + a5);
+        const int r3 = cr(mn + ".p3r", t, 1, 0, m.c3r / 2);
+        cr(mn + ".p3", r3, 3, 1, a3, out, 0);
+        const int r5 = cr(mn + ".p5r", t, 1, 0, m.c5r);
+        cr(mn + ".p5", r5, 5, 2, a5, out, a3);
+        t = out;
+        if (mn == "3b") t = add_simple(n, OP_MAXPOOL, "pool3", t);
+        if (mn == "4e") t = add_simple(n, OP_MAXPOOL, "pool4", t);
+    }
+    t = add_simple(n, OP_AVGPOOL, "avgpool", t);
+    conv_p("fc", 1000, 1, 1024, &w, &b);
+    n->t_logits = add_conv(n, "fc", t, 1, 1, 0, 1000, DR_BIAS | DR_OUT_F32, w, b);
+}
+
 static void build_resnet50(dr_net* n) {
     const bool slim = n->mode == DR_MODE_SLIM;
     const int x = n->tensor(n->B, n->H, n->W, 3, 0, true);
@@ -315,13 +377,15 @@ extern "C" {
 
 int dr_net_create(dr_net** net, int arch, int mode, int B, int H, int W) {
     if (!net || B <= 0 || H <= 0 || W <= 0) return DR_ERR_INVALID_ARG;
-    if (arch != DR_ARCH_GOOGLENET && arch != DR_ARCH_RESNET50) return DR_ERR_INVALID_ARG;
+    if (arch != DR_ARCH_GOOGLENET && arch != DR_ARCH_RESNET50 && arch != DR_ARCH_GOOGLENET_PAPER) return DR_ERR_INVALID_ARG;
     if (mode != DR_MODE_SLIM && mode != DR_MODE_UNSLIMMED) return DR_ERR_INVALID_ARG;
     // five halvings (stem conv, four pools / strided stages) must leave at least one pixel
     if (H < 32 || W < 32) return DR_ERR_INVALID_ARG;
     dr_net* n = new dr_net();
     n->arch = arch; n->mode = mode; n->B = B; n->H = H; n->W = W;
-    if (arch == DR_ARCH_GOOGLENET) build_googlenet(n); else build_resnet50(n);
+    if (arch == DR_ARCH_GOOGLENET) build_googlenet(n);
+    else if (arch == DR_ARCH_GOOGLENET_PAPER) build_googlenet_paper(n);
+    else build_resnet50(n);
     *net = n;
     return DR_OK;
 }

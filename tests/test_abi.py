@@ -120,6 +120,19 @@ def test_googlenet_layer_lists(dr):
     assert e.value.status == dr.DR_ERR_WORKSPACE
 
 
+def test_googlenet_paper_form_layer_list(dr):
+    net = dr.Net(dr.DR_ARCH_GOOGLENET_PAPER, dr.DR_MODE_SLIM, 1)
+    infos = {net.dr_net_layer_info(i)["name"]: net.dr_net_layer_info(i) for i in range(net.dr_net_num_layers())}
+    assert net.dr_net_num_layers() == 3 + 9 * 4 + 2 + 1 + 1
+    # the numbers Section 3.2 gives for inception_3a: reducer 96 -> 48, 3x3 128 -> 192, 5x5 32 -> 64
+    assert infos["3a.p3r"]["dims"] == (1, 28, 28, 48)
+    assert infos["3a.p3"]["dims"] == (1, 28, 28, 192) and (infos["3a.p3"]["ldc"], infos["3a.p3"]["coff"]) == (256, 0)
+    assert infos["3a.p5"]["dims"] == (1, 28, 28, 64) and (infos["3a.p5"]["ldc"], infos["3a.p5"]["coff"]) == (256, 192)
+    assert infos["5b.p5"]["ldc"] == 1024
+    gflop = sum(v["flops"] for v in infos.values()) / 1e9
+    assert 1.5 < gflop < 3.5          # far fewer FLOPs than the merged-5x5 form (16.6)
+
+
 def test_resnet50_layer_lists(dr):
     slim = dr.Net(dr.DR_ARCH_RESNET50, dr.DR_MODE_SLIM, 1)
     n = slim.dr_net_num_layers()

@@ -339,6 +339,28 @@ def test_googlenet_composition_vs_torch_one_image():
     assert np.abs(out["fc"] - ref).max() <= 1e-10 * np.abs(ref).max()
 
 
+def test_googlenet_paper_form_composition_vs_torch():
+    p = P.googlenet_paper_params(0)
+    x = P.images(0, 1, 96, 96)
+    out = N.run(N.googlenet_paper_steps(p), x, rounding=False)
+    lrn = lambda t: F.local_response_norm(t, 5, alpha=1e-4, beta=0.75, k=1.0)
+    pool = lambda t: F.max_pool2d(t, 3, 2, 1)
+    t = nhwc_to_torch(x.astype(np.float64))
+    t = lrn(pool(F.relu(_t_conv(p, "conv1", t, 2, 3))))
+    t = F.relu(_t_conv(p, "conv2r", t, 1, 0))
+    t = pool(lrn(F.relu(_t_conv(p, "conv2", t, 1, 1))))
+    for m in S.INCEPTION_V1:
+        a = F.relu(_t_conv(p, f"{m}.p3", F.relu(_t_conv(p, f"{m}.p3r", t, 1, 0)), 1, 1))
+        b = F.relu(_t_conv(p, f"{m}.p5", F.relu(_t_conv(p, f"{m}.p5r", t, 1, 0)), 1, 2))
+        t = torch.cat([a, b], dim=1)
+        if m in ("3b", "4e"):
+            t = pool(t)
+    ref = torch_to_nhwc(_t_conv(p, "fc", t.mean(dim=(2, 3), keepdim=True), 1, 0))
+    assert np.abs(out["fc"] - ref).max() <= 1e-10 * np.abs(ref).max()
+    # Section 3.2's numbers for 3a: 3x3 reducer 96 -> 48, 3x3 conv 128 -> 192 (printed "196"), 5x5 conv 32 -> 64
+    assert p["3a.p3r.w"].shape[0] == 48 and p["3a.p3.w"].shape[0] == 192 and p["3a.p5.w"].shape[0] == 64
+
+
 def test_resnet50_composition_vs_torch_small_image():
     p = P.resnet50_params(0)
     x = P.images(0, 1, 64, 64)
