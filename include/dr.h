@@ -239,6 +239,10 @@ int dr_last_conv_path(void);            /* path taken by the latest dr_conv_slim
  * wait runs out: returns DR_OK or DR_ERR_DEVICE_TIMEOUT; info[0..3] (may be NULL) receive the
  * code, a kernel-specific site id, the block index and the tile index.                    */
 int dr_device_status(int info[4]);
+/* Self-test of the bounded-wait path: launches one small kernel that waits, for at most limit_cycles SM cycles
+ * (1 .. 2e9), on a barrier nothing arrives on, and then leaves the same record a convolution kernel would.
+ * dr_device_status() afterwards returns DR_ERR_DEVICE_TIMEOUT with info[1] = 99; the context stays usable. */
+int dr_selftest_wait_timeout(long long limit_cycles, void* stream);
 /* Kernels of this library launched by this process so far. */
 long long dr_launch_count(void);
 

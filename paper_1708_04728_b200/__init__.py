@@ -92,6 +92,7 @@ _SIGS = {
     "dr_set_conv_path": (_I, [_I]),
     "dr_last_conv_path": (_I, []),
     "dr_device_status": (_I, [C.POINTER(_I)]),
+    "dr_selftest_wait_timeout": (_I, [C.c_longlong, _P]),
     "dr_launch_count": (C.c_longlong, []),
 }
 for _name, (_res, _args) in _SIGS.items():
@@ -211,6 +212,10 @@ def dr_device_status():
     info = (_I * 4)()
     st = _lib.dr_device_status(info)
     return st, list(info)
+
+
+def dr_selftest_wait_timeout(limit_cycles: int, stream=None):
+    _check(_lib.dr_selftest_wait_timeout(limit_cycles, _stream(stream)), "dr_selftest_wait_timeout")
 
 
 def dr_launch_count() -> int:

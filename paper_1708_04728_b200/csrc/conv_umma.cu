@@ -750,4 +750,29 @@ int conv_umma_tma_launch(const ConvParams& p, cudaStream_t stream) {
     return launch_status();
 }
 
+
+// ---- self-test of the bounded wait -------------------------------------------------------
+// One CTA waits on an mbarrier that nothing ever arrives on, with a short cycle limit, and takes the
+// same way out as the convolution kernels: record DR_ERR_DEVICE_TIMEOUT and return.
+__global__ void wait_timeout_selftest_kernel(int* status, long long limit_cycles) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_barrier_init();
+        const long long t0 = clock64();
+        bool done = false;
+        while (!done && clock64() - t0 < limit_cycles) done = mbar_try_wait(&bar, 0);
+        if (!done) report_timeout(status, 99, -1);
+    }
+}
+
 }  // namespace dr
+
+extern "C" int dr_selftest_wait_timeout(long long limit_cycles, void* stream) {
+    if (limit_cycles <= 0 || limit_cycles > 2000000000ll) return DR_ERR_INVALID_ARG;
+    int* status = dr::dev_status_ptr();
+    if (!status) return DR_ERR_CUDA;
+    dr::wait_timeout_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(status, limit_cycles);
+    dr::count_launch();
+    return dr::launch_status();
+}

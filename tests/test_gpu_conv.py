@@ -240,3 +240,20 @@ def test_inception_3a_config(dr, O):
     forced = N.run(N.inception_steps(params, "3a", "x"), x, given={"3a.3x3r": red})
     assert_layer_close(got[..., :c3], forced["3a.3x3"], "3a.3x3 teacher-forced")
     assert_layer_close(got[..., c3:], forced["3a.m5"], "3a.m5")
+
+
+def test_bounded_wait_reports_timeout_and_context_survives(dr, O):
+    """A wait that can never be satisfied runs out after its limit, leaves DR_ERR_DEVICE_TIMEOUT in the status
+    record, and the next layer on the same context still computes correctly."""
+    assert dr.dr_device_status()[0] == 0
+    dr.dr_selftest_wait_timeout(200000)                 # ~0.1 ms
+    st, info = dr.dr_device_status()
+    assert st == dr.DR_ERR_DEVICE_TIMEOUT and info[0] == dr.DR_ERR_DEVICE_TIMEOUT and info[1] == 99
+    assert dr.dr_device_status()[0] == 0                # reading clears the record
+    x = S.normal(20, "x", (1, 8, 8, 64)); w = S.he_normal(20, "w", 64, 3, 64); b = S.normal(20, "b", (64,), 0.1)
+    dr.dr_set_conv_path(dr.DR_PATH_AUTO)
+    got, _ = run_conv(dr, x, w, b, 3, 1, 1, dr.DR_BIAS | dr.DR_RELU)
+    ref, _ = oracle_slim_layer(O, x, w, b, 3, 1, 1, dr.DR_BIAS | dr.DR_RELU, dr)
+    assert_layer_close(got, O.round_bf16(ref), "after timeout")
+    with pytest.raises(dr.DrError):
+        dr.dr_selftest_wait_timeout(0)
