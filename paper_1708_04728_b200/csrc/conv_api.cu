@@ -72,7 +72,7 @@ int conv_make_params(const dr_conv_desc* d, int B, int H, int W, const void* x, 
         // with the lowest estimated time: rounds of the persistent grid (CTA pairs for long-K layers) times the
         // measured cost of a k-block, about 0.2 us of fixed hand-shake plus 1 ns per output column.
         const long long m_tiles = (p.M + TILE_M - 1) / TILE_M;
-        const bool pairs = p.K >= 1024 && m_tiles >= 2;
+        const bool pairs = (p.K >= 1024 || (p.k > 1 && p.K >= 512)) && m_tiles >= 2;
         const long long capacity = pairs ? num_sms() / 2 : num_sms();
         const long long m_units = pairs ? (m_tiles + 1) / 2 : m_tiles;
         const int nb_min = (cout16 + 255) / 256;

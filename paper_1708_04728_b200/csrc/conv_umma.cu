@@ -700,9 +700,10 @@ int conv_umma_tma_launch(const ConvParams& p, cudaStream_t stream) {
     }
     alignas(64) CUtensorMap map_a, map_b;
     const int a_mode = (p.k == 1 && p.stride == 1 && p.pad == 0) ? 0 : 1;
-    // CTA pairs pay off where the MMAs dominate (long K, several tiles per SM pair)
+    // CTA pairs pay off where the MMAs dominate: long K, or a spatial filter with K >= 512 (measured: +12 % on the
+    // 3x3 layers, -20 % on the 1x1 reducers)
     const int pair_pref = tunable("DR_TMA_PAIR", -1);
-    const bool use_pair = pair_pref >= 0 ? pair_pref != 0 : (p.K >= 1024 && p.m_tiles >= 2);
+    const bool use_pair = pair_pref >= 0 ? pair_pref != 0 : ((p.K >= 1024 || (p.k > 1 && p.K >= 512)) && p.m_tiles >= 2);
     if (a_mode == 0) {
         const cuuint64_t dims[2] = {(cuuint64_t)p.Cin, (cuuint64_t)p.M};
         const cuuint64_t strides[1] = {(cuuint64_t)p.Cin * 2};
