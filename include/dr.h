@@ -231,6 +231,7 @@ int dr_net_activation_bytes(const dr_net* net, size_t* bytes);
 #define DR_PATH_UMMA_PATCH   4  /* pooling layers: 2-D output patches, TMA box loads, fused pool/LRN */
 #define DR_PATH_UMMA_STEM    5  /* the 7x7/2 3-channel stem with fused pool/LRN                  */
 #define DR_PATH_UMMA_STEM_T  6  /* the same stem computed transposed: pooling in registers       */
+#define DR_PATH_UMMA_STEM_D  7  /* the stem with the MMA reading the input rows in place (no im2col) */
 /* Force a convolution kernel (tests, A/B timing); DR_PATH_AUTO picks the fastest that
  * supports the layer.  A forced path that cannot run the layer gives DR_ERR_UNSUPPORTED.   */
 int dr_set_conv_path(int path);

@@ -275,6 +275,8 @@ int conv_stem_launch(const ConvParams& p, cudaStream_t stream);
 bool conv_stem_supports(const ConvParams& p);
 int conv_stem_t_launch(const ConvParams& p, cudaStream_t stream);
 bool conv_stem_t_supports(const ConvParams& p);
+int conv_stem_d_launch(const ConvParams& p, cudaStream_t stream);
+bool conv_stem_d_supports(const ConvParams& p);
 bool conv_umma_gather_supports(const ConvParams& p);
 
 }  // namespace dr

@@ -182,10 +182,11 @@ STAGED = [
     (2, 70, 50, 3, 64, 7, 2, 3, "pool"),            # ResNet conv1 form (no LRN), ragged tiles
     (1, 38, 42, 3, 64, 7, 2, 3, "lrn_pool"),        # stem with LRN first
     (3, 100, 60, 3, 64, 7, 2, 3, "pool_lrn"),       # stem, ragged tiles in both directions, several images
+    (120, 64, 64, 3, 64, 7, 2, 3, "pool_lrn"),      # stem, many images: long per-stream ranges that cross image boundaries
 ]
 
 
-@pytest.mark.parametrize("path", [1, 2, 3, 4, 5, 6])
+@pytest.mark.parametrize("path", [1, 2, 3, 4, 5, 6, 7])
 @pytest.mark.parametrize("case", STAGED)
 def test_conv_fused_pool_lrn(dr, O, path, case):
     B, H, W, Cin, Cout, k, s, p, kind = case
