@@ -22,9 +22,12 @@
 // add bias, clamp, and transpose through shared memory for the cross-channel LRN and the NHWC store.
 //
 // Work split: all row pairs of the batch, in (image, pair) order, are cut into one contiguous range
-// per stream; two independent streams per CTA (each: one loader warp, one MMA warp, four epilogue
-// warps, a 24-row ring of input rows, two accumulators).  A range that starts inside an image first
-// computes the pair above it for the carry only.
+// per stream; two independent streams per CTA.  A stream is a pipeline of one loader warp (a 24-row
+// ring of input rows filled by cp.async three tiles ahead), one MMA warp (two accumulators), four
+// pooling warps (tensor memory -> pooled, biased, clamped values in the transpose buffer) and four
+// LRN/store warps that drain the transpose buffer half a row at a time.  A range that starts inside
+// an image first computes the pair above it for the carry only.  Registers are re-split at kernel
+// start: the pooling warps hold a row of maxima each and take 144, the others give theirs up.
 #include <cstdlib>
 
 #include "conv_common.cuh"
@@ -34,16 +37,18 @@
 namespace dr {
 using namespace ptx;
 
-constexpr int SD_THREADS = 384;          // warps 0-3 / 4-7: epilogue of stream 0 / 1; warps 8, 9: MMA; warps 10, 11: loaders
+constexpr int SD_THREADS = 640;          // warps 0-3 / 4-7: pooling of stream 0 / 1; 8-11 / 12-15: LRN + store; 16, 17: MMA; 18, 19: loaders
+constexpr int SD_REGS_POOL = 144, SD_REGS_LRN = 64, SD_REGS_AUX = 64;     // per thread after the re-split
+static_assert(256 * SD_REGS_POOL + 256 * SD_REGS_LRN + 128 * SD_REGS_AUX <= SD_THREADS * 96, "register split exceeds the launch allocation");
 constexpr int SD_NQ = 6;                 // ring depth in quads (4 input rows = what one tile adds)
 constexpr int SD_NR = 4 * SD_NQ;         // ring rows
-constexpr int SD_LA = 3;                 // quads a loader keeps in flight; SD_LA + 3 <= SD_NQ or loader and MMA wait on each other
 constexpr int SD_WT_BYTES = 36 * 2048;   // filters: 36 K chunks x 128 rows x 16 B
 constexpr int SD_LB_PITCH = 76;          // floats per pooled pixel in the transpose buffer: 4 halo + 64 + 4 halo + 4 (bank spread)
 constexpr int SD_SMEM_MAX = 227 * 1024 - 512;     // dynamic part; the static part holds the barriers
 
 struct SdShared {
     uint64_t qfull[2][SD_NQ], qempty[2][SD_NQ], tfull[2][2], tempty[2][2];
+    uint64_t lfull[2][2], lempty[2][2];      // halves of the transpose buffer: pooling warps -> LRN warps and back
     uint32_t tmem_base;
     int abort;
 };
@@ -89,6 +94,12 @@ __device__ __forceinline__ bool sd_bar_and(int id, bool ok) {     // AND over th
         : "r"((uint32_t)ok), "r"(id)
         : "memory");
     return out != 0;
+}
+
+__device__ __forceinline__ float sd_max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
 }
 
 // The stream's range of row pairs, one image segment at a time.
@@ -137,7 +148,7 @@ __device__ __forceinline__ void sd_hpool(uint32_t taddr, int Wo, Emit emit) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
                 const float a = j == 0 ? prev : v[2 * j - 1];
-                emit(16 * k + j, fmaxf(fmaxf(a, v[2 * j]), v[2 * j + 1]));
+                emit(16 * k + j, sd_max3(a, v[2 * j], v[2 * j + 1]));
             }
             prev = v[31];
         }
@@ -145,6 +156,8 @@ __device__ __forceinline__ void sd_hpool(uint32_t taddr, int Wo, Emit emit) {
 }
 
 // Layer fixed to k = 7, stride 2, pad 3, Cin = 3, Cout = 64, pool 3x3/2 pad 1 after the ReLU (host checks).
+// WO: the output width when it is known at compile time (the width guards fold away), 0 for any width.
+template <int WO>
 __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvParams p, const SdGeom gm) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -152,7 +165,7 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int ring_bytes = SD_NR * gm.pitch + 256;                        // + the run-over of junk columns past the last row
     const int sa_bytes = 64 * gm.sa_pitch * 4;
-    const int lb_bytes = 4 * p.Wy * SD_LB_PITCH;
+    const int lb_bytes = 4 * (WO ? (WO + 1) / 2 : p.Wy) * SD_LB_PITCH;
     uint8_t* Wt = smem;
     uint8_t* ring0 = Wt + SD_WT_BYTES;
     uint8_t* sa0 = ring0 + 2 * ring_bytes;
@@ -162,12 +175,15 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
     if (tid == 0) {
         for (int g = 0; g < 2; ++g) {
             for (int q = 0; q < SD_NQ; ++q) { mbar_init(&sh.qfull[g][q], 32); mbar_init(&sh.qempty[g][q], 1); }
-            for (int b = 0; b < 2; ++b) { mbar_init(&sh.tfull[g][b], 1); mbar_init(&sh.tempty[g][b], 4); }
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(&sh.tfull[g][b], 1); mbar_init(&sh.tempty[g][b], 4);
+                mbar_init(&sh.lfull[g][b], 64); mbar_init(&sh.lempty[g][b], 4);
+            }
         }
         sh.abort = 0;
         fence_barrier_init();
     }
-    if (warp == 8) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
+    if (warp == 16) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
     // everything starts at zero: padding slots, the two spare elements of every slot, unused filter slots, LRN halos
     for (int i = tid; i < total_bytes / 16; i += SD_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
@@ -191,9 +207,10 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
     volatile int* abort_flag = &sh.abort;
     const int streams = 2 * gridDim.x;
 
-    if (warp >= 10) {
+    if (warp >= 18) {
         // ------------------------------------------------------------- loader of stream g
-        const int g = warp - 10;
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(SD_REGS_AUX));
+        const int g = warp - 18;
         SdSegments seg(gm.total, streams, 2 * blockIdx.x + g, gm.NP);
         const uint32_t ring = smem_u32(ring0 + g * ring_bytes);
         const int pairs = p.W >> 1;
@@ -229,22 +246,15 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
                         sd_cp_async4(dst + 8, src + 4, yin);
                     }
                 }
-                asm volatile("cp.async.commit_group;" ::: "memory");
-                if (Ql >= SD_LA) {
-                    asm volatile("cp.async.wait_group %0;" ::"n"(SD_LA) : "memory");
-                    fence_proxy_async_smem();
-                    mbar_arrive(&sh.qfull[g][(int)((Ql - SD_LA) % SD_NQ)]);
-                }
+                // this lane's arrival on the quad's barrier fires when its copies above have landed
+                asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sh.qfull[g][slot])) : "memory");
             }
         }
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        fence_proxy_async_smem();
-        if (!dead) {
-            for (long long qq = Ql > SD_LA ? Ql - SD_LA : 0; qq < Ql; ++qq) mbar_arrive(&sh.qfull[g][(int)(qq % SD_NQ)]);
-        }
-    } else if (warp >= 8) {
+        asm volatile("cp.async.wait_all;" ::: "memory");
+    } else if (warp >= 16) {
         // ------------------------------------------------------------- MMA issue of stream g
-        const int g = warp - 8;
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(SD_REGS_AUX));
+        const int g = warp - 16;
         if (lane == 0) {
             SdSegments seg(gm.total, streams, 2 * blockIdx.x + g, gm.NP);
             const uint32_t ring = smem_u32(ring0 + g * ring_bytes);
@@ -271,6 +281,7 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
                         break;
                     }
                     tc_fence_after();
+                    fence_proxy_async_smem();                              // the loader's copies, seen through the barrier, before the MMA reads them
                     const uint32_t d = tmem + (uint32_t)(g * 256) + buf * 128u;
                     const int row0 = (int)((4 * (Qb + t)) % SD_NR);
 #pragma unroll
@@ -295,22 +306,83 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
             }
         }
         __syncwarp();
+    } else if (warp >= 8) {
+        // ------------------------------------------------------------- LRN + store of stream g
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(SD_REGS_LRN));
+        const int g = (warp - 8) >> 2;
+        const int L = ((warp - 8) & 3) * 32 + lane;
+        const int Wy = WO ? (WO + 1) / 2 : p.Wy;
+        const int hs = ((Wy + 1) / 2 + 3) & ~3;                            // columns in the first half of the transpose buffer
+        const float* lb = reinterpret_cast<const float*>(lb0 + g * lb_bytes);
+        const bool lrn = p.flags & DR_LRN;
+        __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.y);
+        SdSegments seg(gm.total, streams, 2 * blockIdx.x + g, gm.NP);
+        uint32_t lc = 0;                                                   // output tiles so far
+        bool dead = false;
+        int n, j0, T;
+        bool halo;
+        while (!dead && seg.next(n, j0, T, halo)) {
+            for (int t = halo ? 1 : 0; t < T && !dead; ++t, ++lc) {
+                const long long qrow = ((long long)n * p.Hy + (j0 + t)) * Wy;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.lfull[g][h], lc & 1, abort_flag));
+                    if (!ok) {
+                        if (!*abort_flag) report_timeout(p.status, 64, (int)lc);
+                        *abort_flag = 1;
+                        dead = true;
+                        break;
+                    }
+                    const int pw0 = h ? hs : 0;
+                    const int items = ((h ? Wy : hs) - pw0) * 8;           // item = (pooled column, group of 8 channels)
+                    for (int it = L; (it & ~31) < items; it += 128) {      // whole warps leave together (warp votes inside)
+                        const bool active = it < items;
+                        const int pw = pw0 + (active ? it >> 3 : 0), c8 = it & 7;
+                        const float4* s4 = reinterpret_cast<const float4*>(lb + pw * SD_LB_PITCH + (c8 << 3));   // x[c-4 .. c+11]
+                        float w16[16];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float4 f = s4[j];
+                            w16[4 * j] = f.x; w16[4 * j + 1] = f.y; w16[4 * j + 2] = f.z; w16[4 * j + 3] = f.w;
+                        }
+                        uint4 u;
+                        if (lrn) {
+                            float v[12], sq[12], ss[8], sc[8];
+#pragma unroll
+                            for (int j = 0; j < 12; ++j) { v[j] = w16[j + 2]; sq[j] = v[j] * v[j]; }          // v[0] = x[c-2]
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) ss[j] = (sq[j] + sq[j + 1]) + (sq[j + 2] + sq[j + 3]) + sq[j + 4];
+                            fe_lrn_scale<8>(p, ss, sc);
+                            u.x = pack_bf16(v[2] * sc[0], v[3] * sc[1]); u.y = pack_bf16(v[4] * sc[2], v[5] * sc[3]);
+                            u.z = pack_bf16(v[6] * sc[4], v[7] * sc[5]); u.w = pack_bf16(v[8] * sc[6], v[9] * sc[7]);
+                        } else {
+                            u.x = pack_bf16(w16[4], w16[5]); u.y = pack_bf16(w16[6], w16[7]);
+                            u.z = pack_bf16(w16[8], w16[9]); u.w = pack_bf16(w16[10], w16[11]);
+                        }
+                        if (active) *reinterpret_cast<uint4*>(y + (qrow + pw) * p.ldc + p.coff + (c8 << 3)) = u;
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh.lempty[g][h]);
+                }
+            }
+        }
     } else {
-        // ------------------------------------------------------------- epilogue of stream g
+        // ------------------------------------------------------------- pooling of stream g
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(SD_REGS_POOL));
         const int g = warp >> 2, q = warp & 3;
         const int L = q * 32 + lane, c = L & 63;
         const bool phb = L >= 64;                                         // this thread's lane is a channel of row 2i+1
-        const int Wo = p.Wo, Wy = p.Wy, sp = gm.sa_pitch;
+        const int Wo = WO ? WO : p.Wo, Wy = WO ? (WO + 1) / 2 : p.Wy, sp = gm.sa_pitch;
+        const int hs = ((Wy + 1) / 2 + 3) & ~3;
         float* sa = reinterpret_cast<float*>(sa0 + g * sa_bytes) + c * sp;   // this channel's partial maxima
         float* lb = reinterpret_cast<float*>(lb0 + g * lb_bytes);           // [pw][4 | 64 | 4 (+4)]
         const float bias = (p.flags & DR_BIAS) ? p.bias[c] : 0.f;
-        const bool relu = p.flags & DR_RELU, lrn = p.flags & DR_LRN;
+        const bool relu = p.flags & DR_RELU;
         const float NEG = __uint_as_float(0xff800000u);
         const int bar0 = 1 + 3 * g;
-        __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.y);
         SdSegments seg(gm.total, streams, 2 * blockIdx.x + g, gm.NP);
-        uint32_t tcount = 0;
-        bool dead = false;
+        uint32_t tcount = 0, lc = 0;
+        bool dead = false, fail = false;
         int n, j0, T;
         bool halo;
         float keep[64];                       // row 2i threads: this tile's horizontal maxima; row 2i+1 threads: the carry
@@ -319,7 +391,7 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
             for (int j = 0; j < 64; ++j) keep[j] = NEG;
             for (int t = 0; t < T; ++t, ++tcount) {
                 const uint32_t buf = tcount & 1;
-                bool ok = mbar_wait(&sh.tfull[g][buf], (tcount >> 1) & 1, abort_flag);
+                bool ok = mbar_wait(&sh.tfull[g][buf], (tcount >> 1) & 1, abort_flag) && !fail;
                 ok = sd_bar_and(bar0, ok);
                 if (!ok) {
                     if (!*abort_flag) report_timeout(p.status, 63, (int)tcount);
@@ -360,50 +432,31 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
                     for (int f = 0; f < 16; ++f) {
                         if (4 * f < Wy) {
                             const float4 m4 = *reinterpret_cast<const float4*>(sa + 4 * f);
-                            const float mm[4] = {m4.x, m4.y, m4.z, m4.w};
+                            keep[4 * f] = fmaxf(keep[4 * f], m4.x); keep[4 * f + 1] = fmaxf(keep[4 * f + 1], m4.y);
+                            keep[4 * f + 2] = fmaxf(keep[4 * f + 2], m4.z); keep[4 * f + 3] = fmaxf(keep[4 * f + 3], m4.w);
+                        }
+                    }
+                }
+                asm volatile("bar.sync %0, 128;" ::"r"(bar0 + 2) : "memory");   // the partial maxima may be overwritten
+                if (!phb) {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                float v = fmaxf(keep[4 * f + e], mm[e]) + bias;
-                                if (relu) v = fmaxf(v, 0.f);
-                                if (4 * f + e < Wy) lb[(4 * f + e) * SD_LB_PITCH + 4 + c] = v;
+                    for (int h = 0; h < 2; ++h) {
+                        if (!mbar_wait(&sh.lempty[g][h], (lc & 1) ^ 1, abort_flag)) fail = true;   // reported at the next tile's vote
+#pragma unroll
+                        for (int f = 0; f < 16; ++f) {
+                            if (4 * f < Wy && (4 * f >= hs) == (h == 1)) {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    float v = keep[4 * f + e] + bias;
+                                    if (relu) v = fmaxf(v, 0.f);
+                                    if (4 * f + e < Wy) lb[(4 * f + e) * SD_LB_PITCH + 4 + c] = v;
+                                }
                             }
                         }
+                        mbar_arrive(&sh.lfull[g][h]);
                     }
                 }
-                asm volatile("bar.sync %0, 128;" ::"r"(bar0 + 2) : "memory");
-                // cross-channel LRN and store: item = (pooled column, group of 8 channels)
-                {
-                    const int items = Wy * 8;
-                    const int iters = (items + 127) >> 7;                  // same trip count for every lane (warp votes inside)
-                    const long long qrow = ((long long)n * p.Hy + i) * p.Wy;
-                    for (int itn = 0; itn < iters; ++itn) {
-                        const int it = L + (itn << 7);
-                        const bool active = it < items;
-                        const int pw = active ? it >> 3 : Wy - 1, c8 = it & 7;
-                        const float4* s4 = reinterpret_cast<const float4*>(lb + pw * SD_LB_PITCH + (c8 << 3));   // x[c-4 .. c+11]
-                        float w16[16];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float4 f = s4[j];
-                            w16[4 * j] = f.x; w16[4 * j + 1] = f.y; w16[4 * j + 2] = f.z; w16[4 * j + 3] = f.w;
-                        }
-                        uint4 u;
-                        if (lrn) {
-                            float v[12], sq[12], ss[8], sc[8];
-#pragma unroll
-                            for (int j = 0; j < 12; ++j) { v[j] = w16[j + 2]; sq[j] = v[j] * v[j]; }          // v[0] = x[c-2]
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) ss[j] = (sq[j] + sq[j + 1]) + (sq[j + 2] + sq[j + 3]) + sq[j + 4];
-                            fe_lrn_scale<8>(p, ss, sc);
-                            u.x = pack_bf16(v[2] * sc[0], v[3] * sc[1]); u.y = pack_bf16(v[4] * sc[2], v[5] * sc[3]);
-                            u.z = pack_bf16(v[6] * sc[4], v[7] * sc[5]); u.w = pack_bf16(v[8] * sc[6], v[9] * sc[7]);
-                        } else {
-                            u.x = pack_bf16(w16[4], w16[5]); u.y = pack_bf16(w16[6], w16[7]);
-                            u.z = pack_bf16(w16[8], w16[9]); u.w = pack_bf16(w16[10], w16[11]);
-                        }
-                        if (active) *reinterpret_cast<uint4*>(y + (qrow + pw) * p.ldc + p.coff + (c8 << 3)) = u;
-                    }
-                }
+                ++lc;
             }
         }
     }
@@ -414,7 +467,7 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
         while (clock64() - t0 < 400000ll) {}
         __syncthreads();
     }
-    if (warp == 8) tmem_dealloc(tmem, 512);
+    if (warp == 16) tmem_dealloc(tmem, 512);
 }
 
 // ---- host --------------------------------------------------------------------------------
@@ -443,7 +496,8 @@ int conv_stem_d_launch(const ConvParams& p, cudaStream_t stream) {
     if (!conv_stem_d_supports(p)) return DR_ERR_UNSUPPORTED;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(conv_stem_d_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SD_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+        if (cudaFuncSetAttribute(conv_stem_d_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SD_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+        if (cudaFuncSetAttribute(conv_stem_d_kernel<112>, cudaFuncAttributeMaxDynamicSharedMemorySize, SD_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
         attr_set = true;
     }
     const SdGeom g = sd_geom(p);
@@ -452,7 +506,8 @@ int conv_stem_d_launch(const ConvParams& p, cudaStream_t stream) {
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;              // one CTA per SM: each CTA takes all of tensor memory
     const long long want = (g.total + 1) / 2;
     const int grid = want < num_sms() ? (int)want : num_sms();
-    conv_stem_d_kernel<<<grid, SD_THREADS, smem_bytes, stream>>>(p, g);
+    if (p.Wo == 112) conv_stem_d_kernel<112><<<grid, SD_THREADS, smem_bytes, stream>>>(p, g);
+    else conv_stem_d_kernel<0><<<grid, SD_THREADS, smem_bytes, stream>>>(p, g);
     count_launch();
     return launch_status();
 }
