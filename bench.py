@@ -176,7 +176,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=None, help="default 256 (GoogLeNet), 128 (ResNet-50)")
-    ap.add_argument("--arch", default="googlenet", choices=["googlenet", "resnet50", "googlenet_paper"],
+    ap.add_argument("--arch", default="googlenet", choices=["googlenet", "resnet50", "googlenet_paper", "googlenet_streamline"],
                     help="googlenet = the headline workload; resnet50 = the BN-folded bottleneck network (context)")
     ap.add_argument("--layers-out", default=None, help="write the per-layer table (us, roofline) as JSON")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -185,7 +185,7 @@ def main():
                          "this is the small case the ncu captures under profiles/ run")
     args = ap.parse_args()
     if args.batch is None:
-        args.batch = 256 if args.arch == "googlenet" else 128
+        args.batch = 256 if args.arch in ("googlenet", "googlenet_streamline") else 128
     if args.impl == "reference":
         return run_reference(args)
     if args.layer:
@@ -222,10 +222,14 @@ def main():
     B = args.batch
     pk, pk_kind = peaks()
     resnet = args.arch != "googlenet"          # any context arm: no headline metric, no stored ncu traffic
-    params = {"googlenet": P.googlenet_params, "resnet50": P.resnet50_params, "googlenet_paper": P.googlenet_paper_params}[args.arch](0)
-    arch_id = {"googlenet": dr.DR_ARCH_GOOGLENET, "resnet50": dr.DR_ARCH_RESNET50, "googlenet_paper": dr.DR_ARCH_GOOGLENET_PAPER}[args.arch]
-    cfg_name = {"googlenet": "configs[3]", "resnet50": "configs[4]", "googlenet_paper": "Section 3.2 form, context"}[args.arch]
-    arch_name = {"googlenet": "GoogLeNet-slim", "resnet50": "ResNet-50 (BN folded)", "googlenet_paper": "GoogLeNet, paper-form branch slimming"}[args.arch]
+    params = {"googlenet": P.googlenet_params, "resnet50": P.resnet50_params, "googlenet_paper": P.googlenet_paper_params,
+              "googlenet_streamline": P.googlenet_params}[args.arch](0)
+    arch_id = {"googlenet": dr.DR_ARCH_GOOGLENET, "resnet50": dr.DR_ARCH_RESNET50, "googlenet_paper": dr.DR_ARCH_GOOGLENET_PAPER,
+               "googlenet_streamline": dr.DR_ARCH_GOOGLENET_STREAMLINE}[args.arch]
+    cfg_name = {"googlenet": "configs[3]", "resnet50": "configs[4]", "googlenet_paper": "Section 3.2 form, context",
+                "googlenet_streamline": "Section 3.1 approximate stem, context"}[args.arch]
+    arch_name = {"googlenet": "GoogLeNet-slim", "resnet50": "ResNet-50 (BN folded)", "googlenet_paper": "GoogLeNet, paper-form branch slimming",
+                 "googlenet_streamline": "GoogLeNet-slim, stride-product stem without LRN"}[args.arch]
 
     def make_net(mode, batch):
         net = dr.Net(arch_id, mode, batch)

@@ -174,6 +174,11 @@ int dr_avgpool_global(int B, int H, int W, int C, const void* x, void* y, void* 
 #define DR_ARCH_RESNET50   1   /* bottleneck v1; every conv followed by BatchNorm+Scale (4.3)    */
 #define DR_ARCH_GOOGLENET_PAPER 2 /* GoogLeNet slimmed the paper's way (Section 3.2): per module two branches,
                                      1x1 -> 3x3 (reducer halved, output c3+c1) and 1x1 -> 5x5 (output c5+pp)   */
+#define DR_ARCH_GOOGLENET_STREAMLINE 3 /* DR_ARCH_GOOGLENET with the stem in the paper's approximate streamline form
+                                          (Section 3.1): the pools after conv1 and conv2 are dropped and their stride
+                                          multiplied into the convolution (7x7/4, 3x3/2), both LRN layers pruned.  Not
+                                          function-preserving: the paper re-trains; here it is a timing workload with
+                                          parity against its own definition.                                          */
 #define DR_MODE_SLIM       0   /* slim layers: folded BN, fused epilogues, merged branches       */
 #define DR_MODE_UNSLIMMED  1   /* every layer of the original sequence as its own launch         */
 

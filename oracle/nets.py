@@ -89,7 +89,10 @@ def inception_steps(params, m, src, table=None):
     ]
 
 
-def googlenet_steps(params):
+def googlenet_steps(params, streamline=False):
+    """streamline: the stem in the approximate form of Section 3.1 (Method): each pooling layer is removed and its
+    stride multiplied into the convolution below it (conv1 7x7/4, conv2 3x3/2), each LRN layer is pruned; the ReLU
+    stays.  The inception stages are unchanged."""
     def conv2r(x):
         return O.relu(_conv(params, "conv2r", x, 1, 0))
 
@@ -97,7 +100,11 @@ def googlenet_steps(params):
         y = O.lrn(O.relu(_conv(params, "conv2", x, 1, 1)), **_LRN)
         return O.maxpool(y, 3, 2, 1)[0]
 
-    steps = stem_steps(params) + [Step("conv2r", ["conv1"], conv2r), Step("conv2", ["conv2r"], conv2)]
+    if streamline:
+        steps = [Step("conv1", ["x"], lambda x: O.relu(_conv(params, "conv1", x, 4, 3))), Step("conv2r", ["conv1"], conv2r),
+                 Step("conv2", ["conv2r"], lambda x: O.relu(_conv(params, "conv2", x, 2, 1)))]
+    else:
+        steps = stem_steps(params) + [Step("conv2r", ["conv1"], conv2r), Step("conv2", ["conv2r"], conv2)]
     src = "conv2"
     for m in _INCEPTION:
         steps += inception_steps(params, m, src)
@@ -109,6 +116,10 @@ def googlenet_steps(params):
     steps.append(Step("avgpool", [src], O.avgpool_global))
     steps.append(Step("fc", ["avgpool"], lambda x: _conv(params, "fc", x, 1, 0), stored_bf16=False))
     return steps
+
+
+def googlenet_streamline_steps(params):
+    return googlenet_steps(params, streamline=True)
 
 
 def googlenet_paper_steps(params):

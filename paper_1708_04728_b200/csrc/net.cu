@@ -176,8 +176,11 @@ static const Inc kInception[9] = {
     {"4e", 528, 256, 160, 320, 32, 128, 128}, {"5a", 832, 256, 160, 320, 32, 128, 128},
     {"5b", 832, 384, 192, 384, 48, 128, 128}};
 
+// arch DR_ARCH_GOOGLENET_STREAMLINE: the stem in the approximate form of Section 3.1 (Method): a pooling layer is
+// dropped and its stride multiplied into the convolution below it (conv1 7x7/4, conv2 3x3/2), an LRN layer is pruned.
 static void build_googlenet(dr_net* n) {
     const bool slim = n->mode == DR_MODE_SLIM;
+    const bool streamline = n->arch == DR_ARCH_GOOGLENET_STREAMLINE;
     const int x = n->tensor(n->B, n->H, n->W, 3, 0, true);
     n->t_input = x;
     auto conv_p = [&](const std::string& name, int cout, int k, int cin, PRef* w, PRef* b) {
@@ -188,7 +191,10 @@ static void build_googlenet(dr_net* n) {
     int t;
     // conv1: 7x7/2 -> ReLU -> pool -> LRN
     conv_p("conv1", 64, 7, 3, &w, &b);
-    if (slim) {
+    if (streamline) {
+        if (slim) t = add_conv(n, "conv1", x, 7, 4, 3, 64, BR, w, b);
+        else { t = add_conv(n, "conv1.conv", x, 7, 4, 3, 64, DR_BIAS, w, b); t = add_simple(n, OP_RELU, "conv1", t); }
+    } else if (slim) {
         t = add_conv(n, "conv1", x, 7, 2, 3, 64, BR | DR_POOL | DR_LRN, w, b);
     } else {
         t = add_conv(n, "conv1.conv", x, 7, 2, 3, 64, DR_BIAS, w, b);
@@ -201,7 +207,10 @@ static void build_googlenet(dr_net* n) {
     if (slim) t = add_conv(n, "conv2r", t, 1, 1, 0, 64, BR, w, b);
     else { t = add_conv(n, "conv2r.conv", t, 1, 1, 0, 64, DR_BIAS, w, b); t = add_simple(n, OP_RELU, "conv2r", t); }
     conv_p("conv2", 192, 3, 64, &w, &b);
-    if (slim) {
+    if (streamline) {
+        if (slim) t = add_conv(n, "conv2", t, 3, 2, 1, 192, BR, w, b);
+        else { t = add_conv(n, "conv2.conv", t, 3, 2, 1, 192, DR_BIAS, w, b); t = add_simple(n, OP_RELU, "conv2", t); }
+    } else if (slim) {
         t = add_conv(n, "conv2", t, 3, 1, 1, 192, BR | DR_POOL | DR_LRN | DR_LRN_BEFORE_POOL, w, b);
     } else {
         t = add_conv(n, "conv2.conv", t, 3, 1, 1, 192, DR_BIAS, w, b);
@@ -377,13 +386,13 @@ extern "C" {
 
 int dr_net_create(dr_net** net, int arch, int mode, int B, int H, int W) {
     if (!net || B <= 0 || H <= 0 || W <= 0) return DR_ERR_INVALID_ARG;
-    if (arch != DR_ARCH_GOOGLENET && arch != DR_ARCH_RESNET50 && arch != DR_ARCH_GOOGLENET_PAPER) return DR_ERR_INVALID_ARG;
+    if (arch < DR_ARCH_GOOGLENET || arch > DR_ARCH_GOOGLENET_STREAMLINE) return DR_ERR_INVALID_ARG;
     if (mode != DR_MODE_SLIM && mode != DR_MODE_UNSLIMMED) return DR_ERR_INVALID_ARG;
     // five halvings (stem conv, four pools / strided stages) must leave at least one pixel
     if (H < 32 || W < 32) return DR_ERR_INVALID_ARG;
     dr_net* n = new dr_net();
     n->arch = arch; n->mode = mode; n->B = B; n->H = H; n->W = W;
-    if (arch == DR_ARCH_GOOGLENET) build_googlenet(n);
+    if (arch == DR_ARCH_GOOGLENET || arch == DR_ARCH_GOOGLENET_STREAMLINE) build_googlenet(n);
     else if (arch == DR_ARCH_GOOGLENET_PAPER) build_googlenet_paper(n);
     else build_resnet50(n);
     *net = n;

@@ -133,6 +133,23 @@ def test_googlenet_paper_form_layer_list(dr):
     assert 1.5 < gflop < 3.5          # far fewer FLOPs than the merged-5x5 form (16.6)
 
 
+def test_googlenet_streamline_layer_list(dr):
+    """Section 3.1's approximate stem: pool strides multiplied into conv1 / conv2, LRN pruned; the rest as DR_ARCH_GOOGLENET."""
+    net = dr.Net(dr.DR_ARCH_GOOGLENET_STREAMLINE, dr.DR_MODE_SLIM, 1)
+    ref = dr.Net(dr.DR_ARCH_GOOGLENET, dr.DR_MODE_SLIM, 1)
+    assert net.dr_net_num_layers() == ref.dr_net_num_layers()
+    infos = {net.dr_net_layer_info(i)["name"]: net.dr_net_layer_info(i) for i in range(net.dr_net_num_layers())}
+    rinfos = {ref.dr_net_layer_info(i)["name"]: ref.dr_net_layer_info(i) for i in range(ref.dr_net_num_layers())}
+    assert infos["conv1"]["dims"] == (1, 56, 56, 64) and infos["conv2"]["dims"] == (1, 28, 28, 192)
+    # stride 4 instead of 2: a quarter of conv1's multiply-adds; stride 2 instead of 1: a quarter of conv2's
+    assert abs(infos["conv1"]["flops"] * 4 - rinfos["conv1"]["flops"]) <= 1e-6 * rinfos["conv1"]["flops"]
+    assert abs(infos["conv2"]["flops"] * 4 - rinfos["conv2"]["flops"]) <= 1e-6 * rinfos["conv2"]["flops"]
+    assert infos["3a.m5"]["dims"] == rinfos["3a.m5"]["dims"] and infos["fc"]["dims"] == rinfos["fc"]["dims"]
+    uns = dr.Net(dr.DR_ARCH_GOOGLENET_STREAMLINE, dr.DR_MODE_UNSLIMMED, 1)
+    names = [uns.dr_net_layer_info(i)["name"] for i in range(uns.dr_net_num_layers())]
+    assert "conv1.pool" not in names and "conv2.lrn" not in names and "conv1.conv" in names
+
+
 def test_resnet50_layer_lists(dr):
     slim = dr.Net(dr.DR_ARCH_RESNET50, dr.DR_MODE_SLIM, 1)
     n = slim.dr_net_num_layers()

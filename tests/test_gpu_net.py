@@ -93,7 +93,7 @@ def check_network(dr, arch, B, entries, steps_fn, params, per_layer_tol=None):
     # every batch entry produced something finite
     assert bool(np.isfinite(to_host(logits)).all())
     worst = max(report, key=lambda r: r[3])
-    print(f"\n[{['googlenet','resnet50','googlenet-paper'][arch]} B={B}] worst layer {worst[0]} path={worst[1]} max {worst[2]:.2e} l2 {worst[3]:.2e}; "
+    print(f"\n[{['googlenet','resnet50','googlenet-paper','googlenet-streamline'][arch]} B={B}] worst layer {worst[0]} path={worst[1]} max {worst[2]:.2e} l2 {worst[3]:.2e}; "
           f"logits rel-L2 {max(err_norms(got[i], free['fc'][i])[1] for i in range(len(entries))):.2e}")
     return net, logits, free, keep
 
@@ -117,6 +117,14 @@ def test_googlenet_paper_form(dr, B, k):
     import oracle.nets as N
     params = P.googlenet_paper_params(0)
     check_network(dr, dr.DR_ARCH_GOOGLENET_PAPER, B, subset(B, k), N.googlenet_paper_steps, params)
+
+
+@pytest.mark.parametrize("B,k", [(1, 1), (64, 2)])
+def test_googlenet_streamline_form(dr, B, k):
+    """GoogLeNet with the stem in Section 3.1's approximate form (7x7/4, 3x3/2, no pool, no LRN): parity with its own definition."""
+    import oracle.nets as N
+    params = P.googlenet_params(0)
+    check_network(dr, dr.DR_ARCH_GOOGLENET_STREAMLINE, B, subset(B, k), N.googlenet_streamline_steps, params)
 
 
 @pytest.mark.parametrize("B,k", [(128, 2)])

@@ -361,6 +361,30 @@ def test_googlenet_paper_form_composition_vs_torch():
     assert p["3a.p3r.w"].shape[0] == 48 and p["3a.p3.w"].shape[0] == 192 and p["3a.p5.w"].shape[0] == 64
 
 
+def test_googlenet_streamline_composition_vs_torch():
+    """Stem of Section 3.1 (Method): conv stride = conv stride x pool stride, no pool, no LRN, ReLU kept."""
+    p = P.googlenet_params(0)
+    x = P.images(0, 1, 96, 96)
+    out = N.run(N.googlenet_streamline_steps(p), x, rounding=False)
+    pool = lambda t: F.max_pool2d(t, 3, 2, 1)
+    t = nhwc_to_torch(x.astype(np.float64))
+    t = F.relu(_t_conv(p, "conv1", t, 4, 3))
+    assert tuple(out["conv1"].shape) == (1, 24, 24, 64) and np.abs(out["conv1"] - torch_to_nhwc(t)).max() <= 1e-10 * float(t.abs().max())
+    t = F.relu(_t_conv(p, "conv2", F.relu(_t_conv(p, "conv2r", t, 1, 0)), 2, 1))
+    assert tuple(out["conv2"].shape) == (1, 12, 12, 192)
+    for m in S.INCEPTION_V1:
+        three = F.relu(_t_conv(p, f"{m}.3x3", F.relu(_t_conv(p, f"{m}.3x3r", t, 1, 0)), 1, 1))
+        t = torch.cat([three, F.relu(_t_conv(p, f"{m}.b1", t, 1, 0)), F.relu(_t_conv(p, f"{m}.b5", t, 1, 2)),
+                       F.relu(_t_conv(p, f"{m}.bp", t, 1, 1))], dim=1)
+        if m in ("3b", "4e"):
+            t = pool(t)
+    ref = torch_to_nhwc(_t_conv(p, "fc", t.mean(dim=(2, 3), keepdim=True), 1, 0))
+    assert np.abs(out["fc"] - ref).max() <= 1e-10 * np.abs(ref).max()
+    # the exact stem and the approximate one give different functions (the paper re-trains): same shapes only
+    exact = N.run(N.googlenet_steps(p), x, rounding=False)
+    assert exact["conv2"].shape == out["conv2"].shape and np.abs(exact["conv2"] - out["conv2"]).max() > 1e-3
+
+
 def test_resnet50_composition_vs_torch_small_image():
     p = P.resnet50_params(0)
     x = P.images(0, 1, 64, 64)
