@@ -106,6 +106,23 @@ int dr_embed_filter(int Cout, int Cin, int ks, int kb, const void* w_small, int 
 int dr_conv_slim(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* w,
                  const float* b, const void* residual, void* y, int32_t* argmax, void* stream);
 
+/* dr_conv_slim with scratch memory at hand.  A layer with few output pixels and a long
+ * reduction (single-image inference, the regime of the paper's timings in Section 4.1: the 14x14
+ * and 7x7 stages have 196 and 49 pixels against K = k*k*Cin up to 20800) is then computed split
+ * along K: every SM multiplies a slice of K for one output tile, the float32 partial tiles meet
+ * in the workspace and are summed in slice order, so the result does not depend on timing.
+ * Same arithmetic (float32 accumulation, one rounding at the store), arguments and errors as
+ * dr_conv_slim.  dr_conv_workspace_bytes() gives the size the layer can use (0: it would run as
+ * in dr_conv_slim).  workspace: NULL, or device memory aligned to 256 bytes whose first
+ * DR_CONV_WS_COUNTER_BYTES are zero before the first call; every call leaves them zero again, so
+ * calls on one stream can share a workspace.  Calls that may overlap on the GPU need their own.
+ * A workspace smaller than the layer wants is not an error: the layer runs as in dr_conv_slim. */
+#define DR_CONV_WS_COUNTER_BYTES 1024
+int dr_conv_workspace_bytes(const dr_conv_desc* desc, int B, int H, int W, size_t* bytes);
+int dr_conv_slim_ws(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* w,
+                    const float* b, const void* residual, void* y, int32_t* argmax, void* workspace,
+                    size_t workspace_bytes, void* stream);
+
 /* Branch-slimmed inception module (Section 3.2; the merged-branch identity Eqs. (LR), (W_b)):
  *   y[..., 0:c3)      = ReLU(conv3x3(ReLU(conv1x1(x; w[0]) + b[0]); w[1]) + b[1])
  *   y[..., c3:c3+cm)  = ReLU(conv5x5(x; w[2]) + b[2])          (pad 2, the merged branches)
@@ -237,6 +254,7 @@ int dr_net_activation_bytes(const dr_net* net, size_t* bytes);
 #define DR_PATH_UMMA_STEM    5  /* the 7x7/2 3-channel stem with fused pool/LRN                  */
 #define DR_PATH_UMMA_STEM_T  6  /* the same stem computed transposed: pooling in registers       */
 #define DR_PATH_UMMA_STEM_D  7  /* the stem with the MMA reading the input rows in place (no im2col) */
+#define DR_PATH_UMMA_SPLITK  8  /* few output tiles: K split across the SMs, partial tiles summed in scratch (needs a workspace) */
 /* Force a convolution kernel (tests, A/B timing); DR_PATH_AUTO picks the fastest that
  * supports the layer.  A forced path that cannot run the layer gives DR_ERR_UNSUPPORTED.   */
 int dr_set_conv_path(int path);

@@ -29,7 +29,10 @@ DR_LRN_BEFORE_POOL, DR_RELU_AFTER_RESIDUAL, DR_OUT_F32 = 0x20, 0x40, 0x80
 DR_ARCH_GOOGLENET, DR_ARCH_RESNET50, DR_ARCH_GOOGLENET_PAPER, DR_ARCH_GOOGLENET_STREAMLINE = 0, 1, 2, 3
 DR_MODE_SLIM, DR_MODE_UNSLIMMED = 0, 1
 DR_PATH_AUTO, DR_PATH_SIMT, DR_PATH_UMMA_GATHER, DR_PATH_UMMA_TMA, DR_PATH_UMMA_PATCH, DR_PATH_UMMA_STEM, DR_PATH_UMMA_STEM_T, DR_PATH_UMMA_STEM_D = 0, 1, 2, 3, 4, 5, 6, 7
-PATH_NAMES = {0: "auto", 1: "simt", 2: "umma_gather", 3: "umma_tma", 4: "umma_patch", 5: "umma_stem", 6: "umma_stem_t", 7: "umma_stem_d", -1: "-"}
+DR_PATH_UMMA_SPLITK = 8
+DR_CONV_WS_COUNTER_BYTES = 1024
+PATH_NAMES = {0: "auto", 1: "simt", 2: "umma_gather", 3: "umma_tma", 4: "umma_patch", 5: "umma_stem", 6: "umma_stem_t", 7: "umma_stem_d",
+              8: "umma_splitk", -1: "-"}
 
 
 class dr_conv_desc(C.Structure):
@@ -65,6 +68,8 @@ _SIGS = {
     "dr_fold_bn": (_I, [_I, _I, _P, _P, _P, _P, _F, _F, _P, _P, _P, _P, _P]),
     "dr_embed_filter": (_I, [_I, _I, _I, _I, _P, _I, _P, _P]),
     "dr_conv_slim": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P]),
+    "dr_conv_workspace_bytes": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, C.POINTER(_Z)]),
+    "dr_conv_slim_ws": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _Z, _P]),
     "dr_inception_workspace_bytes": (_I, [C.POINTER(dr_inception_desc), _I, _I, _I, C.POINTER(_Z)]),
     "dr_inception_slim": (_I, [C.POINTER(dr_inception_desc), _I, _I, _I, _P, C.POINTER(_P), C.POINTER(_P), _P, _P, _P]),
     "dr_inception_slim_static": (_I, [C.POINTER(dr_inception_desc), _I, _I, _I, _P, C.POINTER(_P), C.POINTER(_P), _P, _P]),
@@ -140,6 +145,17 @@ def dr_embed_filter(Cout, Cin, ks, kb, w_small, joff, w_big, stream=None):
 def dr_conv_slim(desc, B, H, W, x, w, b, residual, y, argmax=None, stream=None):
     _check(_lib.dr_conv_slim(C.byref(desc), B, H, W, _ptr(x), _ptr(w), _ptr(b), _ptr(residual), _ptr(y), _ptr(argmax),
                              _stream(stream)), "dr_conv_slim")
+
+
+def dr_conv_workspace_bytes(desc, B, H, W) -> int:
+    n = _Z(0)
+    _check(_lib.dr_conv_workspace_bytes(C.byref(desc), B, H, W, C.byref(n)), "dr_conv_workspace_bytes")
+    return n.value
+
+
+def dr_conv_slim_ws(desc, B, H, W, x, w, b, residual, y, argmax, workspace, workspace_bytes, stream=None):
+    _check(_lib.dr_conv_slim_ws(C.byref(desc), B, H, W, _ptr(x), _ptr(w), _ptr(b), _ptr(residual), _ptr(y), _ptr(argmax),
+                                _ptr(workspace), workspace_bytes, _stream(stream)), "dr_conv_slim_ws")
 
 
 def dr_inception_workspace_bytes(desc, B, H, W) -> int:

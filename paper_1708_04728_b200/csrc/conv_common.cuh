@@ -15,6 +15,8 @@
 // and/or LRN): the tile's ReLU'd float32 values are staged in shared memory as [row][C+1], then
 // LRN (window along the row) and the 3x3 max (window across rows) read it from there.
 #pragma once
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace dr {
@@ -46,6 +48,9 @@ struct ConvParams {
     int patch;             // 0 linear, 1 patch
     int PH, PW;            // pooled tile extent in patch mode
     int tiles_h, tiles_w;  // pooled tiles per image
+    int* sk_counters;      // split-K kernel only (nullptr: not available): DR_CONV_WS_COUNTER_BYTES of zeroed tile counters
+    float* sk_scratch;     // and scratch for the partial tiles
+    size_t sk_scratch_bytes;
 };
 
 struct RowPix {
@@ -278,5 +283,15 @@ bool conv_stem_t_supports(const ConvParams& p);
 int conv_stem_d_launch(const ConvParams& p, cudaStream_t stream);
 bool conv_stem_d_supports(const ConvParams& p);
 bool conv_umma_gather_supports(const ConvParams& p);
+int conv_splitk_launch(const ConvParams& p, cudaStream_t stream);
+bool conv_splitk_supports(const ConvParams& p);
+size_t conv_splitk_scratch_bytes(const ConvParams& p);   // partial-tile scratch the split-K kernel wants; 0: it would not take the layer
+// two layers that read the same input in one split-K launch (a: long K; b: short, e.g. a 1x1 reducer); scratch and
+// counters are taken from a
+int conv_splitk_pair_launch(const ConvParams& a, const ConvParams& b, cudaStream_t stream);
+bool conv_splitk_pair_supports(const ConvParams& a, const ConvParams& b);
+size_t conv_splitk_pair_scratch_bytes(const ConvParams& a, const ConvParams& b);
+int encode_conv_maps(const ConvParams& p, int b_box_rows, CUtensorMap* map_a, CUtensorMap* map_b, int* a_mode);
+int tunable(const char* name, int dflt);
 
 }  // namespace dr

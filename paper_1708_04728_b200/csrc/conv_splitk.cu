@@ -1,0 +1,495 @@
+// Split-K implicit-GEMM convolution for layers with few output tiles (single-image inference, the
+// regime the paper times: one forward pass of one image, Section 4.1).
+//
+// At batch 1 the 14x14 and 7x7 stages of GoogLeNet have 196 and 49 output pixels: one or two
+// 128-row tiles.  The persistent kernel of conv_umma.cu would run such a layer on a handful of SMs,
+// each walking the whole K = k*k*Cin (up to 20800) alone while the layer's weights (up to 27 MB)
+// trickle in through one SM's load path.  Here the K range of every output tile is cut into
+// `splits` slices, one CTA per (tile, n-block, slice), so that the whole GPU streams the weights:
+//
+//   1. each CTA multiplies its K slice (TMA im2col / tiled loads -> shared memory -> tcgen05.mma,
+//      accumulator in tensor memory) exactly like the persistent kernel does;
+//   2. it writes its float32 partial tile to scratch memory and arrives on the tile's counter;
+//   3. it waits until all slices of the tile have arrived (the grid is launched cooperatively, i.e.
+//      every CTA is resident, so the wait ends; it is bounded all the same);
+//   4. it sums 1/splits of the tile over all partials, each element in slice order 0..splits-1 — a fixed order, so
+//      the result does not depend on timing — applies bias / ReLU / residual and stores bf16 or f32.
+//
+// Scratch memory: `counters` (one int per output tile, zero on entry, back at zero when the kernel has finished) and `scratch`
+// (tiles x splits x 128 x Nt floats, contents irrelevant on entry).
+#include "conv_common.cuh"
+#include "umma_ptx.cuh"
+
+namespace dr {
+using namespace ptx;
+
+constexpr int SK_A_BYTES = TILE_M * 128;        // 128 pixels x 64 bf16
+constexpr int SK_MAX_STAGES = 12;
+constexpr int SK_THREADS = 192;                 // warp 0: TMA producer, warp 1: MMA issue + TMEM owner, warps 2-5: drain; all: reduction
+constexpr int SK_SMEM_MAX = 227 * 1024 - 2048;  // dynamic part
+constexpr int SK_MAX_TILES = DR_CONV_WS_COUNTER_BYTES / 4;
+
+struct SkShared {
+    uint64_t full[SK_MAX_STAGES], empty[SK_MAX_STAGES], accum;
+    uint32_t tmem_base;
+    int abort;
+};
+
+struct SkPlan {
+    int nt, n_blocks, splits, kps, nkb, stages, sub_bytes;
+    uint32_t tmem_cols;
+    size_t scratch_bytes;
+};
+
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// One job = one convolution layer cut into (tile, n-block, slice) work items.  A launch carries one job, or two
+// independent jobs that read the same input (an inception module's 1x1 reducer beside its merged 5x5 branch):
+// CTAs [0, second_begin) work on the first, the rest on the second.
+struct alignas(64) SkJob {
+    CUtensorMap map_a, map_b;
+    ConvParams p;
+    int a_mode, stages, sub_bytes, splits, kps;
+    uint32_t tmem_cols;
+    float* scratch;
+    int* counters;
+};
+struct SkJobs { SkJob j[2]; };
+
+__global__ void __launch_bounds__(SK_THREADS, 1)
+conv_splitk_kernel(const __grid_constant__ SkJobs jobs, const int second_begin) {
+    const bool second = (int)blockIdx.x >= second_begin;
+    const SkJob* const J = second ? &jobs.j[1] : &jobs.j[0];
+    const int bid = second ? (int)blockIdx.x - second_begin : (int)blockIdx.x;
+    const ConvParams& p = J->p;
+    const CUtensorMap& map_a = J->map_a;
+    const CUtensorMap& map_b = J->map_b;
+    const int a_mode = J->a_mode, stages = J->stages, sub_bytes = J->sub_bytes, splits = J->splits, kps = J->kps;
+    const uint32_t tmem_cols = J->tmem_cols;
+    float* __restrict__ scratch = J->scratch;
+    int* __restrict__ counters = J->counters;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __shared__ SkShared sh;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // work item of this CTA: K slice `split` of output tile (mt, nb)
+    const int split = bid % splits, tile = bid / splits;
+    const int nb = tile / p.m_tiles, mt = tile - nb * p.m_tiles;
+    const int n0 = nb * p.Nt;
+    const int cout16 = (p.Cout + 15) & ~15;
+    const int Nj = min(p.Nt, cout16 - n0);
+    const int cpb = (p.Cin + 63) >> 6;
+    const int nkb = p.k * p.k * cpb;
+    const int kb0 = split * kps, kb1 = min(nkb, kb0 + kps);
+
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        mbar_init(&sh.accum, 1);
+        sh.abort = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+    }
+    if (warp == 1) { tmem_alloc(&sh.tmem_base, tmem_cols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+    volatile int* abort_flag = &sh.abort;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t full0 = smem_u32(&sh.full[0]), empty0 = smem_u32(&sh.empty[0]);
+    // The next kernel in the stream may be scheduled from here on (it waits for this one to finish before it
+    // touches anything this one writes); every thread but the producer waits for the previous kernel right away.
+    grid_launch_dependents();
+    if (tid != 0) grid_dependency_wait();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // -------------------------------------------- TMA producer
+            const uint32_t tx = SK_A_BYTES + (uint32_t)p.Nt * 128;
+            const long long m0 = (long long)mt * TILE_M;
+            const int hw = p.Ho * p.Wo;
+            const int img = (int)(m0 / hw);
+            const int rem = (int)(m0 - (long long)img * hw);
+            const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
+            const int hb = ho * p.stride - p.pad, wb = wo * p.stride - p.pad;
+            int tap = kb0 / cpb;
+            int c0 = (kb0 - tap * cpb) << 6;
+            int r = tap / p.k, tt = tap - r * p.k;
+            // The filters do not depend on the layer before this one: their loads for the first round of pipeline
+            // stages go out before the wait for that layer, so the weights stream in while it finishes.
+            const int npre = min(stages, kb1 - kb0);
+            {
+                int tap_b = tap, c0_b = c0;
+                for (int i = 0; i < npre; ++i) {
+                    const uint32_t fb = full0 + 8 * i;
+                    mbar_expect_tx_u32(fb, tx);
+                    tma_load_3d_u32<false>(smem_base + (uint32_t)i * (uint32_t)sub_bytes + SK_A_BYTES, &map_b, fb, c0_b, tap_b, n0, 1u);
+                    c0_b += 64;
+                    if (c0_b >= p.Cin) { c0_b = 0; ++tap_b; }
+                }
+            }
+            grid_dependency_wait();
+            int s = 0;
+            uint32_t ph = 0;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                const int i = kb - kb0;
+                if (i >= stages && !mbar_wait_u32(empty0 + 8 * s, ph ^ 1, abort_flag)) {
+                    if (!*abort_flag) report_timeout(p.status, 21, tile);
+                    *abort_flag = 1;
+                    break;
+                }
+                const uint32_t dst = smem_base + (uint32_t)s * (uint32_t)sub_bytes;
+                const uint32_t fb = full0 + 8 * s;
+                if (i >= npre) mbar_expect_tx_u32(fb, tx);
+                if (a_mode == 0) tma_load_2d_u32<false>(dst, &map_a, fb, c0, (int)m0, 1u);
+                else tma_load_im2col_4d_u32<false>(dst, &map_a, fb, c0, wb, hb, img, (uint16_t)tt, (uint16_t)r, 1u);
+                if (i >= npre) tma_load_3d_u32<false>(dst + SK_A_BYTES, &map_b, fb, c0, tap, n0, 1u);
+                c0 += 64;
+                if (c0 >= p.Cin) {
+                    c0 = 0; ++tap; ++tt;
+                    if (tt == p.k) { tt = 0; ++r; }
+                }
+                if (++s == stages) { s = 0; ph ^= 1; }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // -------------------------------------------- MMA issue
+            const uint32_t idesc = make_idesc_bf16(TILE_M, Nj);
+            const int last_nk16 = ((p.Cin - ((cpb - 1) << 6)) + 15) >> 4;
+            int cc = kb0 % cpb;
+            int s = 0;
+            uint32_t ph = 0, accum = 0;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait_u32(full0 + 8 * s, ph, abort_flag)) {
+                    if (!*abort_flag) report_timeout(p.status, 22, tile);
+                    *abort_flag = 1;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t a = smem_base + (uint32_t)s * (uint32_t)sub_bytes;
+                const uint32_t alo = sdesc_lo(a), blo = sdesc_lo(a + SK_A_BYTES);
+                const int nk16 = (cc == cpb - 1) ? last_nk16 : 4;
+                cc = (cc + 1 == cpb) ? 0 : cc + 1;
+                umma_bf16_lo<false>(tmem, alo, blo, idesc, accum, 1u);
+                accum = 1;
+                umma_bf16_lo<false>(tmem, alo + 2, blo + 2, idesc, 1u, nk16 > 1);
+                umma_bf16_lo<false>(tmem, alo + 4, blo + 4, idesc, 1u, nk16 > 2);
+                umma_bf16_lo<false>(tmem, alo + 6, blo + 6, idesc, 1u, nk16 > 3);
+                umma_commit_u32<false>(empty0 + 8 * s);
+                if (++s == stages) { s = 0; ph ^= 1; }
+            }
+            umma_commit_u32<false>(smem_u32(&sh.accum));   // also on a timeout: fires once whatever was issued has finished
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------ drain: float32 partial tile -> scratch.  TMEM lane quarter = warp % 4.
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.accum, 0, abort_flag));
+        if (!ok) {
+            if (!*abort_flag) report_timeout(p.status, 23, tile);
+            *abort_flag = 1;
+        } else if (!*abort_flag) {
+            tc_fence_after();
+            const long long m = (long long)mt * TILE_M + row;
+            const bool row_ok = m < p.M;
+            const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16);
+            float4* dst = reinterpret_cast<float4*>(scratch + (((size_t)tile * splits + split) * TILE_M + row) * p.Nt);
+            int c = 0;
+            for (; c + 32 <= Nj; c += 32) {
+                uint32_t v[32];
+                tmem_ld_x32(taddr + c, v);
+                tmem_ld_wait();
+                if (row_ok) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        dst[(c >> 2) + j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                                                        __uint_as_float(v[4 * j + 3]));
+                }
+            }
+            if (c < Nj) {   // 16-column tail
+                uint32_t v[16];
+                tmem_ld_x16(taddr + c, v);
+                tmem_ld_wait();
+                if (row_ok) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        dst[(c >> 2) + j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                                                        __uint_as_float(v[4 * j + 3]));
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------- all slices of the tile meet here
+    // This CTA's share of the tile: float4 elements [f0, f1) of valid_rows x Nj/4, one element per thread and pass;
+    // a thread sums the slices of its element in order 0..splits-1 with up to 16 loads in flight.
+    const long long mrem = p.M - (long long)mt * TILE_M;
+    const int valid_rows = mrem < TILE_M ? (int)mrem : TILE_M;
+    const int nq = Nj >> 2;
+    const int total = valid_rows * nq;
+    const int per = (total + splits - 1) / splits;
+    const int f0 = split * per, f1 = min(total, f0 + per);
+    // bias of the first element this thread finishes, fetched before the wait (it does not depend on the partials)
+    float4 bias0 = make_float4(0.f, 0.f, 0.f, 0.f);
+    if ((p.flags & DR_BIAS) && f0 + tid < f1) {
+        const int col = n0 + 4 * ((f0 + tid) % nq);
+        if (col < p.Cout) bias0 = make_float4(__ldg(p.bias + col), __ldg(p.bias + col + 1), __ldg(p.bias + col + 2), __ldg(p.bias + col + 3));
+    }
+    tc_fence_before();
+    __syncthreads();                     // the whole partial tile has been written (by this CTA's threads, in CTA order)
+    if (tid == 0) {
+        __threadfence();                 // ... and is visible device-wide before the arrival is (cumulative over the barrier)
+        // the counter runs 0 .. 2*splits-1 and wraps to zero: first arrivals take it to `splits`, second ones back to 0
+        const unsigned old = atomicInc(reinterpret_cast<unsigned*>(&counters[tile]), 2u * (unsigned)splits - 1u);
+        if ((int)old + 1 < splits) {     // arrives even after a timeout above, so that the other slices do not wait for nothing
+            const long long t0 = clock64();
+            while (ld_acquire_gpu(&counters[tile]) < splits) {
+                if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                    if (!*abort_flag) report_timeout(p.status, 24, tile);
+                    *abort_flag = 1;
+                    break;
+                }
+            }
+        }
+        __threadfence();
+    }
+    __syncthreads();
+
+    if (!*abort_flag) {
+        const size_t slice4 = (size_t)TILE_M * (p.Nt >> 2);      // float4 per partial tile
+        const float4* part = reinterpret_cast<const float4*>(scratch) + (size_t)tile * splits * slice4;
+        const bool f32 = p.flags & DR_OUT_F32;
+        for (int e = f0 + tid; e < f1; e += SK_THREADS) {
+            const int row = e / nq;
+            const int cq = e - row * nq;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4* src = part + (size_t)row * (p.Nt >> 2) + cq;
+#pragma unroll 16
+            for (int sp = 0; sp < splits; ++sp, src += slice4) {
+                const float4 v = __ldcg(src);
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            }
+            const int col = n0 + 4 * cq;
+            if (col < p.Cout) {
+                const long long m = (long long)mt * TILE_M + row;
+                if (p.flags & DR_BIAS) {
+                    float4 b = bias0;
+                    if (e != f0 + tid) b = make_float4(__ldg(p.bias + col), __ldg(p.bias + col + 1), __ldg(p.bias + col + 2), __ldg(p.bias + col + 3));
+                    acc.x += b.x; acc.y += b.y; acc.z += b.z; acc.w += b.w;
+                }
+                if (p.flags & DR_RELU) { acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f); acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f); }
+                if (p.flags & DR_RESIDUAL) {
+                    const uint2 u = __ldg(reinterpret_cast<const uint2*>(p.residual + m * p.Cout + col));
+                    acc.x += bf16_lo(u.x); acc.y += bf16_hi(u.x); acc.z += bf16_lo(u.y); acc.w += bf16_hi(u.y);
+                    if (p.flags & DR_RELU_AFTER_RESIDUAL) { acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f); acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f); }
+                }
+                if (f32) {
+                    *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.y) + m * p.ldc + p.coff + col) = acc;
+                } else {
+                    uint2 o;
+                    o.x = pack_bf16(acc.x, acc.y);
+                    o.y = pack_bf16(acc.z, acc.w);
+                    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.y) + m * p.ldc + p.coff + col) = o;
+                }
+            }
+        }
+    }
+
+    __syncthreads();                     // every thread of this CTA has finished reading the partials
+    if (tid == 0)                        // second arrival, not waited for: the last of them wraps the counter back to zero
+        asm volatile("red.relaxed.gpu.global.inc.u32 [%0], %1;" ::"l"(&counters[tile]), "r"(2u * (unsigned)splits - 1u) : "memory");
+    if (*abort_flag) {   // give copies and MMAs still in flight time to land before shared memory and TMEM go away
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) {}
+        __syncthreads();
+    }
+    if (warp == 1) tmem_dealloc(tmem, tmem_cols);
+}
+
+// ---- host ---------------------------------------------------------------------------------
+static bool splitk_shape_ok(const ConvParams& p) {
+    if (p.flags & (DR_POOL | DR_LRN)) return false;
+    if (p.patch) return false;
+    if ((p.Cin & 7) || p.Cin < 64) return false;
+    if ((p.Cout & 3) || (p.ldc & 3) || (p.coff & 3)) return false;
+    if (p.k > 255 || p.M <= 0 || p.M > 0x7fffffffLL) return false;
+    return true;
+}
+
+// Choice of n-block width and slice count for a layer that may use `budget` CTAs.  Measured on B200 (batch 1,
+// GoogLeNet's inception layers): n-blocks of about 80 columns and at most 32 slices are within a microsecond of
+// the best plan of every layer; a slice has at least two k-blocks unless `single` allows plans without splitting.
+static bool splitk_plan_budget(const ConvParams& p, int budget, bool single, SkPlan* out) {
+    if (!splitk_shape_ok(p)) return false;
+    const int cpb = (p.Cin + 63) >> 6;
+    const int nkb = p.k * p.k * cpb;
+    const int cout16 = (p.Cout + 15) & ~15;
+    const int nb_min = (cout16 + 255) / 256;
+    int nb = tunable("DR_SPLITK_NB", 0);
+    if (nb <= 0) nb = (cout16 + 40) / 80;
+    if (nb < nb_min) nb = nb_min;
+    while (nb > nb_min && (long long)p.m_tiles * nb * (single ? 1 : 2) > budget) --nb;
+    int nt = ((cout16 + nb - 1) / nb + 15) / 16 * 16;
+    while ((long long)nt * (nb - 1) >= cout16 && nb > 1) { --nb; nt = ((cout16 + nb - 1) / nb + 15) / 16 * 16; }   // no empty block
+    const long long tiles = (long long)p.m_tiles * nb;
+    if (tiles > SK_MAX_TILES || tiles > budget) return false;
+    int S = (int)(budget / tiles);
+    if (S > nkb / 2) S = nkb / 2;
+    int s_max = tunable("DR_SPLITK_S", 0);
+    if (s_max <= 0) s_max = 32;
+    if (S > s_max) S = s_max;
+    if (S < 1) S = 1;
+    if (S < 2 && !single) return false;
+    SkPlan b{};
+    b.kps = (nkb + S - 1) / S;
+    b.splits = (nkb + b.kps - 1) / b.kps;                               // no empty slice
+    b.nt = nt; b.n_blocks = nb; b.nkb = nkb;
+    b.sub_bytes = SK_A_BYTES + ((b.nt * 128 + 1023) & ~1023);
+    int st = (tunable("DR_SPLITK_SMEM_KB", 200) * 1024 - 1024) / b.sub_bytes;
+    if (st > SK_MAX_STAGES) st = SK_MAX_STAGES;
+    if (st > b.kps) st = b.kps;
+    b.stages = st;
+    b.tmem_cols = 32;
+    while ((int)b.tmem_cols < b.nt) b.tmem_cols <<= 1;
+    b.scratch_bytes = ((size_t)p.m_tiles * b.n_blocks * b.splits * TILE_M * b.nt * sizeof(float) + 255) / 256 * 256;
+    *out = b;
+    return true;
+}
+
+// A layer on its own: worth splitting when the persistent kernel would leave most of the GPU idle AND walk a long K
+// per CTA.  Measured: from about 24 k-blocks on (16 when the layer has only one or two output tiles); below that
+// the hand-over between the slices costs more than the shorter loop saves (the 1x1 reducers stay where they were).
+static bool splitk_plan(const ConvParams& p, SkPlan* out) {
+    if (!splitk_shape_ok(p)) return false;
+    const int sms = num_sms();
+    const int force = tunable("DR_SPLITK", -1);            // 0: never, 1: whenever the shape allows
+    if (force == 0) return false;
+    const int nkb = p.k * p.k * ((p.Cin + 63) >> 6);
+    if (force != 1) {
+        if ((long long)p.m_tiles * p.n_blocks * 2 > sms) return false;
+        if (nkb < 16 || (nkb < 24 && p.m_tiles > 2)) return false;
+    }
+    if (nkb < 4) return false;
+    return splitk_plan_budget(p, sms, false, out);
+}
+
+size_t conv_splitk_scratch_bytes(const ConvParams& p) {
+    SkPlan pl;
+    if (!splitk_plan(p, &pl)) return 0;
+    return pl.scratch_bytes;
+}
+
+bool conv_splitk_supports(const ConvParams& p) {
+    if (!p.sk_counters || !p.sk_scratch || ((uintptr_t)p.sk_scratch & 15)) return false;
+    SkPlan pl;
+    if (!splitk_plan(p, &pl)) return false;
+    return p.sk_scratch_bytes >= pl.scratch_bytes;
+}
+
+// Two layers in one launch: `a` (the long one) and `b` (a short one reading the same input, e.g. a 1x1 reducer).
+// b takes up to 24 CTAs, a the rest.  b's scratch follows a's; b's counters follow a's tiles.
+static const int SK_PAIR_SMALL_CTAS = 24;
+static bool splitk_pair_plan(const ConvParams& a, const ConvParams& b, SkPlan* pa, SkPlan* pb) {
+    if (tunable("DR_SPLITK_PAIR", 1) == 0) return false;
+    if (a.x != b.x || a.B != b.B || a.H != b.H || a.W != b.W || a.Cin != b.Cin) return false;
+    if (!splitk_plan_budget(b, SK_PAIR_SMALL_CTAS, true, pb)) return false;
+    const int used = b.m_tiles * pb->n_blocks * pb->splits;
+    SkPlan alone;
+    if (!splitk_plan(a, &alone)) return false;                         // a must be a split-K layer in its own right
+    if (!splitk_plan_budget(a, num_sms() - used, false, pa)) return false;
+    if ((long long)a.m_tiles * pa->n_blocks + (long long)b.m_tiles * pb->n_blocks > SK_MAX_TILES) return false;
+    return true;
+}
+
+size_t conv_splitk_pair_scratch_bytes(const ConvParams& a, const ConvParams& b) {
+    SkPlan pa, pb;
+    if (!splitk_pair_plan(a, b, &pa, &pb)) return 0;
+    return pa.scratch_bytes + pb.scratch_bytes;
+}
+
+bool conv_splitk_pair_supports(const ConvParams& a, const ConvParams& b) {
+    if (!a.sk_counters || !a.sk_scratch || ((uintptr_t)a.sk_scratch & 255)) return false;
+    SkPlan pa, pb;
+    if (!splitk_pair_plan(a, b, &pa, &pb)) return false;
+    return a.sk_scratch_bytes >= pa.scratch_bytes + pb.scratch_bytes;
+}
+
+static int fill_job(const ConvParams& p0, const SkPlan& pl, float* scratch, int* counters, SkJob* j) {
+    j->p = p0;
+    j->p.Nt = pl.nt;
+    j->p.n_blocks = pl.n_blocks;
+    const int est = encode_conv_maps(j->p, pl.nt, &j->map_a, &j->map_b, &j->a_mode);
+    if (est != DR_OK) return est;
+    j->stages = pl.stages; j->sub_bytes = pl.sub_bytes; j->splits = pl.splits; j->kps = pl.kps; j->tmem_cols = pl.tmem_cols;
+    j->scratch = scratch; j->counters = counters;
+    return DR_OK;
+}
+
+static int launch_jobs(const SkJobs& jobs, int ctas0, int ctas1, int smem_bytes, cudaStream_t stream) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(conv_splitk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+        attr_set = true;
+    }
+    // Launch mode.  Programmatic (default): the kernel may start while the previous kernel of the stream drains, and
+    // prefetches its filters meanwhile; the grid never exceeds the SM count, and the kernel before it never waits on
+    // this one, so every slice becomes resident.  DR_SPLITK_PDL=0: a cooperative launch (residency checked by the
+    // runtime), no overlap.
+    const bool pdl = tunable("DR_SPLITK_PDL", 1) != 0;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    if (pdl) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+    } else {
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+    }
+    cfg.gridDim = dim3((unsigned)(ctas0 + ctas1));
+    cfg.blockDim = dim3(SK_THREADS);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, conv_splitk_kernel, jobs, ctas0) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DR_ERR_CUDA;
+    }
+    count_launch();
+    return launch_status();
+}
+
+int conv_splitk_launch(const ConvParams& p, cudaStream_t stream) {
+    SkPlan pl;
+    if (!conv_splitk_supports(p) || !splitk_plan(p, &pl)) return DR_ERR_UNSUPPORTED;
+    SkJobs jobs{};
+    const int st = fill_job(p, pl, p.sk_scratch, p.sk_counters, &jobs.j[0]);
+    if (st != DR_OK) return st;
+    // as many stages as the slice has k-blocks, up to 200 KB: short slices leave room for a CTA of the next layer
+    // beside one of this layer on the same SM (at most 256 TMEM columns each)
+    return launch_jobs(jobs, p.m_tiles * pl.n_blocks * pl.splits, 0, pl.stages * pl.sub_bytes + 1024, stream);
+}
+
+int conv_splitk_pair_launch(const ConvParams& a, const ConvParams& b, cudaStream_t stream) {
+    SkPlan pa, pb;
+    if (!conv_splitk_pair_supports(a, b) || !splitk_pair_plan(a, b, &pa, &pb)) return DR_ERR_UNSUPPORTED;
+    SkJobs jobs{};
+    int st = fill_job(a, pa, a.sk_scratch, a.sk_counters, &jobs.j[0]);
+    if (st != DR_OK) return st;
+    float* scratch_b = reinterpret_cast<float*>(reinterpret_cast<char*>(a.sk_scratch) + pa.scratch_bytes);
+    st = fill_job(b, pb, scratch_b, a.sk_counters + a.m_tiles * pa.n_blocks, &jobs.j[1]);
+    if (st != DR_OK) return st;
+    const int sa = pa.stages * pa.sub_bytes, sb = pb.stages * pb.sub_bytes;
+    return launch_jobs(jobs, a.m_tiles * pa.n_blocks * pa.splits, b.m_tiles * pb.n_blocks * pb.splits, (sa > sb ? sa : sb) + 1024, stream);
+}
+
+}  // namespace dr

@@ -617,8 +617,45 @@ static bool load_encoders() {
     return true;
 }
 
-// Integer tunable from the environment (read once per name at first use); for A/B timing.
-static int tunable(const char* name, int dflt) {
+// Tensor maps of one convolution for the TMA kernels.  A: the activations, as a plain [M][Cin] matrix for
+// 1x1 / stride 1 / pad 0 layers (*a_mode = 0, 2-D tiled boxes of 128 rows x 64 channels) and in im2col mode
+// otherwise (*a_mode = 1: 128 output pixels x 64 channels of one filter tap per load).  B: the filters as
+// (Cin, taps, Cout) with boxes of 64 channels x 1 tap x b_box_rows filters.
+int encode_conv_maps(const ConvParams& p, int b_box_rows, CUtensorMap* map_a, CUtensorMap* map_b, int* a_mode) {
+    if (!load_encoders()) return DR_ERR_CUDA;
+    *a_mode = (p.k == 1 && p.stride == 1 && p.pad == 0) ? 0 : 1;
+    if (*a_mode == 0) {
+        const cuuint64_t dims[2] = {(cuuint64_t)p.Cin, (cuuint64_t)p.M};
+        const cuuint64_t strides[1] = {(cuuint64_t)p.Cin * 2};
+        const cuuint32_t box[2] = {64, TILE_M};
+        const cuuint32_t es[2] = {1, 1};
+        if (g_encode_tiled(map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)p.x, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DR_ERR_CUDA;
+    } else {
+        const cuuint64_t dims[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
+        const cuuint64_t strides[3] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.W * p.Cin * 2, (cuuint64_t)p.H * p.W * p.Cin * 2};
+        // bounding box of the positions the filter's first tap visits: [-pad, extent + pad - k]
+        const int lower[2] = {-p.pad, -p.pad};
+        const int upper[2] = {p.pad - (p.k - 1), p.pad - (p.k - 1)};
+        const cuuint32_t es[4] = {1, (cuuint32_t)p.stride, (cuuint32_t)p.stride, 1};
+        if (g_encode_im2col(map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void*)p.x, dims, strides, lower, upper, 64, TILE_M, es,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DR_ERR_CUDA;
+    }
+    const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
+    const cuuint64_t strides[2] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.K * 2};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)b_box_rows};
+    const cuuint32_t es[3] = {1, 1, 1};
+    if (g_encode_tiled(map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)p.w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return DR_ERR_CUDA;
+    return DR_OK;
+}
+
+// Integer tunable from the environment; for A/B timing.
+int tunable(const char* name, int dflt) {
     const char* v = getenv(name);
     return v ? atoi(v) : dflt;
 }
@@ -689,7 +726,6 @@ static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUte
 
 int conv_umma_tma_launch(const ConvParams& p, cudaStream_t stream) {
     if (!conv_umma_tma_supports(p)) return DR_ERR_UNSUPPORTED;
-    if (!load_encoders()) return DR_ERR_CUDA;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(conv_umma_tma_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
@@ -698,41 +734,14 @@ int conv_umma_tma_launch(const ConvParams& p, cudaStream_t stream) {
             return DR_ERR_CUDA;
         attr_set = true;
     }
-    alignas(64) CUtensorMap map_a, map_b;
-    const int a_mode = (p.k == 1 && p.stride == 1 && p.pad == 0) ? 0 : 1;
     // CTA pairs pay off where the MMAs dominate: long K, or a spatial filter with K >= 512 (measured: +12 % on the
     // 3x3 layers, -20 % on the 1x1 reducers)
     const int pair_pref = tunable("DR_TMA_PAIR", -1);
     const bool use_pair = pair_pref >= 0 ? pair_pref != 0 : ((p.K >= 1024 || (p.k > 1 && p.K >= 512)) && p.m_tiles >= 2);
-    if (a_mode == 0) {
-        const cuuint64_t dims[2] = {(cuuint64_t)p.Cin, (cuuint64_t)p.M};
-        const cuuint64_t strides[1] = {(cuuint64_t)p.Cin * 2};
-        const cuuint32_t box[2] = {64, TILE_M};
-        const cuuint32_t es[2] = {1, 1};
-        if (g_encode_tiled(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)p.x, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return DR_ERR_CUDA;
-    } else {
-        const cuuint64_t dims[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
-        const cuuint64_t strides[3] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.W * p.Cin * 2, (cuuint64_t)p.H * p.W * p.Cin * 2};
-        // bounding box of the positions the filter's first tap visits: [-pad, extent + pad - k]
-        const int lower[2] = {-p.pad, -p.pad};
-        const int upper[2] = {p.pad - (p.k - 1), p.pad - (p.k - 1)};
-        const cuuint32_t es[4] = {1, (cuuint32_t)p.stride, (cuuint32_t)p.stride, 1};
-        if (g_encode_im2col(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void*)p.x, dims, strides, lower, upper, 64, TILE_M, es,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return DR_ERR_CUDA;
-    }
-    {
-        const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
-        const cuuint64_t strides[2] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.K * 2};
-        const cuuint32_t box[3] = {64, 1, (cuuint32_t)(use_pair ? p.Nt / 2 : p.Nt)};   // a pair's CTAs load half each
-        const cuuint32_t es[3] = {1, 1, 1};
-        if (g_encode_tiled(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)p.w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return DR_ERR_CUDA;
-    }
+    alignas(64) CUtensorMap map_a, map_b;
+    int a_mode = 0;
+    const int est = encode_conv_maps(p, use_pair ? p.Nt / 2 : p.Nt, &map_a, &map_b, &a_mode);   // a pair's CTAs load half of B each
+    if (est != DR_OK) return est;
     const int total = p.m_tiles * p.n_blocks;
     if (total <= 0) return DR_OK;
     if (use_pair) return launch_pair(p, map_a, map_b, a_mode, stream);

@@ -52,6 +52,9 @@ struct Op {
     float eps = 0.f;
     double flops = 0, bytes = 0;
     int path = -1;
+    int conv_index = -1;     // OP_CONV: ordinal among the convolutions (its block of split-K counters)
+    int pair = -1;           // OP_CONV: a later convolution reading the same input that may share this one's launch
+    bool pair_ok = false;    // decided by dr_net_prepare
 };
 
 // Derivations done once by dr_net_prepare
@@ -73,9 +76,12 @@ struct dr_net {
     std::vector<EmbedJob> embeds;
     std::vector<CopyJob> copies;
     size_t param_bytes = 0, act_bytes = 0;
+    size_t sk_scratch_bytes = 0;   // split-K scratch shared by all layers (they run one after another), after the arena
+    int n_conv = 0;                // each convolution has its own block of tile counters after that
     int t_input = -1, t_logits = -1;
     void* prepared_ws = nullptr;
     bool timing = false;
+    std::vector<char> done;        // per forward pass: layers that shared an earlier layer's launch
     std::vector<cudaEvent_t> ev;   // 2 per op
     float eps = 1e-5f;
 
@@ -129,6 +135,7 @@ static int add_conv(dr_net* n, const std::string& name, int in, int k, int s, in
     op.out = out; op.coff = coff;
     op.cd.y_ldc = n->T(out).C; op.cd.y_coff = coff;
     op.w = w; op.b = b;
+    op.conv_index = n->n_conv++;
     op.bytes = xin + (double)cout * k * k * ti.C * 2 + (double)ti.B * Ho * Wo * cout * ((flags & DR_OUT_F32) ? 4 : 2) +
                ((flags & DR_RESIDUAL) ? (double)ti.B * Ho * Wo * cout * 2 : 0.0) + ((flags & DR_BIAS) ? cout * 4.0 : 0.0);
     n->ops.push_back(op);
@@ -239,8 +246,12 @@ static void build_googlenet(dr_net* n) {
             n->copies.push_back({b5.raw, bm + (size_t)m.c1 * 4, (size_t)m.c5 * 4});
             n->copies.push_back({bp.raw, bm + (size_t)(m.c1 + m.c5) * 4, (size_t)m.pp * 4});
             const int r = add_conv(n, mn + ".3x3r", t, 1, 1, 0, m.c3r, BR, w3r, b3r);
+            const size_t i_reducer = n->ops.size() - 1;
             add_conv(n, mn + ".3x3", r, 3, 1, 1, m.c3, BR, w3, b3, out, 0);
             add_conv(n, mn + ".m5", t, 5, 1, 2, cm, BR, wsref(wm), wsref(bm), out, m.c3);
+            // the reducer and the merged branch read the same tensor and write different ones: at small batch they
+            // may go out as one launch
+            n->ops[i_reducer].pair = (int)n->ops.size() - 1;
         } else {
             int r = add_conv(n, mn + ".3x3r.conv", t, 1, 1, 0, m.c3r, DR_BIAS, w3r, b3r);
             r = add_simple(n, OP_RELU, mn + ".3x3r", r);
@@ -374,6 +385,18 @@ static void build_resnet50(dr_net* n) {
     n->t_logits = add_conv(n, "fc", t, 1, 1, 0, 1000, DR_BIAS | DR_OUT_F32, rawref(wi), rawref(bi));
 }
 
+// Split-K scratch of the workspace: [parameters][activation arena][scratch][counters, one block per convolution]
+static size_t sk_region_bytes(const dr_net* n) {
+    return n->sk_scratch_bytes ? (n->sk_scratch_bytes + 255) / 256 * 256 + (size_t)n->n_conv * DR_CONV_WS_COUNTER_BYTES : 0;
+}
+static void set_splitk_scratch(const dr_net* n, const Op& op, char* ws, ConvParams* p) {
+    if (!n->sk_scratch_bytes || n->mode != DR_MODE_SLIM) return;
+    char* base = ws + n->param_bytes + n->act_bytes;
+    p->sk_scratch = reinterpret_cast<float*>(base);
+    p->sk_scratch_bytes = n->sk_scratch_bytes;
+    p->sk_counters = reinterpret_cast<int*>(base + (n->sk_scratch_bytes + 255) / 256 * 256 + (size_t)op.conv_index * DR_CONV_WS_COUNTER_BYTES);
+}
+
 static const char* tensor_ptr(const dr_net* n, int id, const void* x, const char* arena, const float* logits) {
     if (id == n->t_input) return (const char*)x;
     if (id == n->t_logits) return (const char*)logits;
@@ -395,6 +418,26 @@ int dr_net_create(dr_net** net, int arch, int mode, int B, int H, int W) {
     if (arch == DR_ARCH_GOOGLENET || arch == DR_ARCH_GOOGLENET_STREAMLINE) build_googlenet(n);
     else if (arch == DR_ARCH_GOOGLENET_PAPER) build_googlenet_paper(n);
     else build_resnet50(n);
+    // scratch the split-K kernel wants for the layers with few output tiles (slim mode only: the unslimmed
+    // baseline keeps one plain launch per layer)
+    if (mode == DR_MODE_SLIM)
+        for (const Op& op : n->ops) {
+            if (op.kind != OP_CONV) continue;
+            const Tensor& ti = n->T(op.in0);
+            ConvParams p;
+            const void* dummy = reinterpret_cast<const void*>(uintptr_t(256));
+            if (conv_make_params(&op.cd, ti.B, ti.H, ti.W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &p) != DR_OK) continue;
+            size_t need = conv_splitk_scratch_bytes(p);
+            if (op.pair >= 0) {
+                const Op& oa = n->ops[op.pair];
+                ConvParams pa;
+                if (conv_make_params(&oa.cd, ti.B, ti.H, ti.W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &pa) == DR_OK) {
+                    const size_t both = conv_splitk_pair_scratch_bytes(pa, p);
+                    if (both > need) need = both;
+                }
+            }
+            if (need > n->sk_scratch_bytes) n->sk_scratch_bytes = need;
+        }
     *net = n;
     return DR_OK;
 }
@@ -424,7 +467,7 @@ int dr_net_set_param(dr_net* n, int idx, const void* dev) {
 
 int dr_net_workspace_bytes(const dr_net* n, size_t* bytes) {
     if (!n || !bytes) return DR_ERR_INVALID_ARG;
-    *bytes = n->param_bytes + n->act_bytes + 256;
+    *bytes = n->param_bytes + n->act_bytes + sk_region_bytes(n) + 256;
     return DR_OK;
 }
 
@@ -453,6 +496,10 @@ int dr_net_prepare(dr_net* n, void* workspace, void* stream) {
     }
     for (const CopyJob& c : n->copies)
         if (cudaMemcpyAsync(ws + c.dst_off, n->raw[c.src], c.bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return DR_ERR_CUDA;
+    if (n->sk_scratch_bytes && n->mode == DR_MODE_SLIM) {   // tile counters start at zero; the kernels leave them at zero
+        char* counters = ws + n->param_bytes + n->act_bytes + (n->sk_scratch_bytes + 255) / 256 * 256;
+        if (cudaMemsetAsync(counters, 0, (size_t)n->n_conv * DR_CONV_WS_COUNTER_BYTES, s) != cudaSuccess) return DR_ERR_CUDA;
+    }
     // decide the kernel of every convolution once
     const char* arena = ws + n->param_bytes;
     for (Op& op : n->ops) {
@@ -462,8 +509,21 @@ int dr_net_prepare(dr_net* n, void* workspace, void* stream) {
         const char* dummy = arena;   // addresses only need to be aligned for validation here
         const int st = conv_make_params(&op.cd, ti.B, ti.H, ti.W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &p);
         if (st != DR_OK) return st;
+        set_splitk_scratch(n, op, ws, &p);
         op.path = conv_pick_path(p, forced_conv_path());
         if (op.path < 0) return DR_ERR_UNSUPPORTED;
+    }
+    for (Op& op : n->ops) {
+        op.pair_ok = false;
+        if (op.kind != OP_CONV || op.pair < 0 || forced_conv_path() != DR_PATH_AUTO) continue;
+        const Op& oa = n->ops[op.pair];
+        const Tensor& ti = n->T(op.in0);
+        ConvParams pa, pb;
+        const char* dummy = arena;
+        if (conv_make_params(&oa.cd, ti.B, ti.H, ti.W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &pa) != DR_OK) continue;
+        if (conv_make_params(&op.cd, ti.B, ti.H, ti.W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &pb) != DR_OK) continue;
+        set_splitk_scratch(n, oa, ws, &pa);
+        op.pair_ok = oa.path == DR_PATH_UMMA_SPLITK && conv_splitk_pair_supports(pa, pb);
     }
     n->prepared_ws = workspace;
     return DR_OK;
@@ -482,7 +542,9 @@ int dr_net_forward(dr_net* n, const void* x, void* workspace, float* logits, voi
         for (auto& e : n->ev)
             if (cudaEventCreate(&e) != cudaSuccess) return DR_ERR_CUDA;
     }
+    n->done.assign(n->ops.size(), 0);
     for (size_t i = 0; i < n->ops.size(); ++i) {
+        if (n->done[i]) continue;              // went out together with an earlier layer
         const Op& op = n->ops[i];
         const Tensor& ti = n->T(op.in0);
         const Tensor& to = n->T(op.out);
@@ -496,7 +558,23 @@ int dr_net_forward(dr_net* n, const void* x, void* workspace, float* logits, voi
                 ConvParams p;
                 st = conv_make_params(&op.cd, ti.B, ti.H, ti.W, in0, op.w.resolve(n->raw, ws), (const float*)op.b.resolve(n->raw, ws),
                                       (op.cd.flags & DR_RESIDUAL) ? in1 : nullptr, out, nullptr, &p);
-                if (st == DR_OK) st = conv_launch_path(p, op.path, s);
+                if (st == DR_OK && op.pair_ok && !n->timing) {
+                    // this layer and a later one that reads the same input, as one launch (per-layer timing keeps them apart)
+                    const Op& oa = n->ops[op.pair];
+                    ConvParams pa;
+                    st = conv_make_params(&oa.cd, ti.B, ti.H, ti.W, in0, oa.w.resolve(n->raw, ws), (const float*)oa.b.resolve(n->raw, ws),
+                                          nullptr, (char*)tensor_ptr(n, oa.out, x, arena, logits), nullptr, &pa);
+                    if (st == DR_OK) {
+                        set_splitk_scratch(n, oa, (char*)workspace, &pa);
+                        st = conv_splitk_pair_launch(pa, p, s);
+                        n->done[op.pair] = 1;
+                    }
+                    break;
+                }
+                if (st == DR_OK) {
+                    set_splitk_scratch(n, op, (char*)workspace, &p);
+                    st = conv_launch_path(p, op.path, s);
+                }
                 break;
             }
             case OP_RELU: st = dr_relu((size_t)ti.B * ti.H * ti.W * ti.C, in0, out, stream); break;

@@ -72,6 +72,24 @@ def test_conv_validation_rejects_before_launch(dr):
     assert dr.dr_launch_count() == n0
 
 
+def test_conv_workspace_query_and_validation(dr):
+    """Host-only: which layers want split-K scratch, and argument checks of dr_conv_slim_ws."""
+    d = dr.dr_conv_desc(k=5, stride=1, pad=2, Cin=832, Cout=640, flags=dr.DR_BIAS | dr.DR_RELU)
+    small, large = dr.dr_conv_workspace_bytes(d, 1, 7, 7), dr.dr_conv_workspace_bytes(d, 256, 7, 7)
+    assert small > dr.DR_CONV_WS_COUNTER_BYTES and large == 0
+    assert small < 64 << 20
+    d3 = dr.dr_conv_desc(k=7, stride=2, pad=3, Cin=3, Cout=64, flags=dr.DR_BIAS)      # stem: never split
+    assert dr.dr_conv_workspace_bytes(d3, 1, 224, 224) == 0
+    n0 = dr.dr_launch_count()
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_conv_slim_ws(d, 1, 7, 7, 256, 256, 256, None, 256, None, 260, 1 << 20, 0)   # workspace not 256-byte aligned
+    assert e.value.status == dr.DR_ERR_ALIGNMENT
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_conv_slim_ws(d, 1, 7, 7, None, 256, 256, None, 256, None, 256, 1 << 20, 0)
+    assert e.value.status == dr.DR_ERR_INVALID_ARG
+    assert dr.dr_launch_count() == n0
+
+
 def test_non_tensor_validation(dr):
     n0 = dr.dr_launch_count()
     for call in (lambda: dr.dr_relu(16, None, 256, 0),
