@@ -286,11 +286,11 @@ bool conv_umma_gather_supports(const ConvParams& p);
 int conv_splitk_launch(const ConvParams& p, cudaStream_t stream);
 bool conv_splitk_supports(const ConvParams& p);
 size_t conv_splitk_scratch_bytes(const ConvParams& p);   // partial-tile scratch the split-K kernel wants; 0: it would not take the layer
-// two layers that read the same input in one split-K launch (a: long K; b: short, e.g. a 1x1 reducer); scratch and
-// counters are taken from a
-int conv_splitk_pair_launch(const ConvParams& a, const ConvParams& b, cudaStream_t stream);
-bool conv_splitk_pair_supports(const ConvParams& a, const ConvParams& b);
-size_t conv_splitk_pair_scratch_bytes(const ConvParams& a, const ConvParams& b);
+// layers of one inception module in one split-K launch: a (long K) and b (short, e.g. the 1x1 reducer) read the same
+// input; c (optional) reads b's output.  Scratch and counters are taken from a.
+int conv_splitk_group_launch(const ConvParams& a, const ConvParams& b, const ConvParams* c, cudaStream_t stream);
+bool conv_splitk_group_supports(const ConvParams& a, const ConvParams& b, const ConvParams* c);
+size_t conv_splitk_group_scratch_bytes(const ConvParams& a, const ConvParams& b, const ConvParams* c);
 int encode_conv_maps(const ConvParams& p, int b_box_rows, CUtensorMap* map_a, CUtensorMap* map_b, int* a_mode);
 int tunable(const char* name, int dflt);
 

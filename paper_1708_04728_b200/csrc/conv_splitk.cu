@@ -16,7 +16,7 @@
 //      the result does not depend on timing — applies bias / ReLU / residual and stores bf16 or f32.
 //
 // Scratch memory: `counters` (one int per output tile, zero on entry, back at zero when the kernel has finished) and `scratch`
-// (tiles x splits x 128 x Nt floats, contents irrelevant on entry).
+// (tiles x splits x Nt/4 x 128 float4, contents irrelevant on entry).
 #include "conv_common.cuh"
 #include "umma_ptx.cuh"
 
@@ -47,34 +47,42 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
     return v;
 }
 
-// One job = one convolution layer cut into (tile, n-block, slice) work items.  A launch carries one job, or two
-// independent jobs that read the same input (an inception module's 1x1 reducer beside its merged 5x5 branch):
-// CTAs [0, second_begin) work on the first, the rest on the second.
+// One job = one convolution layer cut into (tile, n-block, slice) work items.  A launch carries up to three jobs
+// of one inception module: CTAs [0, small_begin) work on job 0 (the merged 5x5 branch); the remaining "small group"
+// works on job 1 (the 1x1 reducer, which reads the same input as job 0) and then, once every CTA of job 1 has
+// stored its output, on job 2 (the 3x3 convolution that reads the reducer's output).
 struct alignas(64) SkJob {
     CUtensorMap map_a, map_b;
     ConvParams p;
     int a_mode, stages, sub_bytes, splits, kps;
+    int ctas;                 // work items of this job = tiles x slices
     uint32_t tmem_cols;
     float* scratch;
     int* counters;
 };
-struct SkJobs { SkJob j[2]; };
+struct SkJobs {
+    SkJob j[3];
+    int n;                    // 1, 2 or 3 jobs
+    int small_begin;          // first CTA of the small group (n >= 2)
+    int* dep;                 // n == 3: counter on which job 2 waits for job 1
+};
 
-__global__ void __launch_bounds__(SK_THREADS, 1)
-conv_splitk_kernel(const __grid_constant__ SkJobs jobs, const int second_begin) {
-    const bool second = (int)blockIdx.x >= second_begin;
-    const SkJob* const J = second ? &jobs.j[1] : &jobs.j[0];
-    const int bid = second ? (int)blockIdx.x - second_begin : (int)blockIdx.x;
+__device__ __forceinline__ void red_inc_gpu(int* p, unsigned wrap) {
+    asm volatile("red.relaxed.gpu.global.inc.u32 [%0], %1;" ::"l"(p), "r"(wrap) : "memory");
+}
+
+// The whole CTA runs work item `bid` of job J.  `first`: this is the CTA's first job (wait for the previous kernel
+// of the stream after the filter prefetch).  `dep_wait` >= 0: before reading its input, wait until *dep has
+// reached dep_wait (the producing job's CTA count).  `dep_wrap` > 0: announce on *dep when this CTA is done with
+// the job (producers: after their stores; consumers: after the wait), the counter wrapping to 0 at dep_wrap.
+__device__ __forceinline__ void sk_run_job(const SkJob* const J, const int bid, SkShared& sh, uint8_t* smem, const uint32_t tmem,
+                                           const bool first, int* dep, const int dep_wait, const bool dep_signal, const unsigned dep_wrap) {
     const ConvParams& p = J->p;
     const CUtensorMap& map_a = J->map_a;
     const CUtensorMap& map_b = J->map_b;
     const int a_mode = J->a_mode, stages = J->stages, sub_bytes = J->sub_bytes, splits = J->splits, kps = J->kps;
-    const uint32_t tmem_cols = J->tmem_cols;
     float* __restrict__ scratch = J->scratch;
     int* __restrict__ counters = J->counters;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    __shared__ SkShared sh;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // work item of this CTA: K slice `split` of output tile (mt, nb)
@@ -87,30 +95,15 @@ conv_splitk_kernel(const __grid_constant__ SkJobs jobs, const int second_begin) 
     const int nkb = p.k * p.k * cpb;
     const int kb0 = split * kps, kb1 = min(nkb, kb0 + kps);
 
-    if (tid == 0) {
-        for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-        mbar_init(&sh.accum, 1);
-        sh.abort = 0;
-        fence_barrier_init();
-        prefetch_tensormap(&map_a);
-        prefetch_tensormap(&map_b);
-    }
-    if (warp == 1) { tmem_alloc(&sh.tmem_base, tmem_cols); tmem_relinquish(); }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = sh.tmem_base;
     volatile int* abort_flag = &sh.abort;
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t full0 = smem_u32(&sh.full[0]), empty0 = smem_u32(&sh.empty[0]);
-    // The next kernel in the stream may be scheduled from here on (it waits for this one to finish before it
-    // touches anything this one writes); every thread but the producer waits for the previous kernel right away.
-    grid_launch_dependents();
-    if (tid != 0) grid_dependency_wait();
 
     if (warp == 0) {
         if (lane == 0) {
             // -------------------------------------------- TMA producer
+            prefetch_tensormap(&map_a);
+            prefetch_tensormap(&map_b);
             const uint32_t tx = SK_A_BYTES + (uint32_t)p.Nt * 128;
             const long long m0 = (long long)mt * TILE_M;
             const int hw = p.Ho * p.Wo;
@@ -134,7 +127,20 @@ conv_splitk_kernel(const __grid_constant__ SkJobs jobs, const int second_begin) 
                     if (c0_b >= p.Cin) { c0_b = 0; ++tap_b; }
                 }
             }
-            grid_dependency_wait();
+            if (first) grid_dependency_wait();
+            if (dep_wait >= 0) {
+                // the input of this job is written by another job of this launch
+                const long long t0 = clock64();
+                while (ld_acquire_gpu(dep) < dep_wait) {
+                    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                        if (!*abort_flag) report_timeout(p.status, 25, tile);
+                        *abort_flag = 1;
+                        break;
+                    }
+                }
+                fence_proxy_async_all();      // those writes went through the generic proxy; the loads below are TMA's
+                red_inc_gpu(dep, dep_wrap);   // consumers count too, so that the last of them wraps the counter to zero
+            }
             int s = 0;
             uint32_t ph = 0;
             for (int kb = kb0; kb < kb1; ++kb) {
@@ -159,6 +165,7 @@ conv_splitk_kernel(const __grid_constant__ SkJobs jobs, const int second_begin) 
             }
         }
         __syncwarp();
+        if (first && lane != 0) grid_dependency_wait();
     } else if (warp == 1) {
         if (lane == 0) {
             // -------------------------------------------- MMA issue
@@ -202,7 +209,8 @@ conv_splitk_kernel(const __grid_constant__ SkJobs jobs, const int second_begin) 
             const long long m = (long long)mt * TILE_M + row;
             const bool row_ok = m < p.M;
             const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16);
-            float4* dst = reinterpret_cast<float4*>(scratch + (((size_t)tile * splits + split) * TILE_M + row) * p.Nt);
+            // partial tile layout [column quad][row]: the 32 rows of a warp are 512 contiguous bytes per store
+            float4* dst = reinterpret_cast<float4*>(scratch + ((size_t)tile * splits + split) * TILE_M * p.Nt) + row;
             int c = 0;
             for (; c + 32 <= Nj; c += 32) {
                 uint32_t v[32];
@@ -211,7 +219,7 @@ conv_splitk_kernel(const __grid_constant__ SkJobs jobs, const int second_begin) 
                 if (row_ok) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        dst[(c >> 2) + j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                        dst[((c >> 2) + j) * TILE_M] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
                                                         __uint_as_float(v[4 * j + 3]));
                 }
             }
@@ -222,7 +230,7 @@ conv_splitk_kernel(const __grid_constant__ SkJobs jobs, const int second_begin) 
                 if (row_ok) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
-                        dst[(c >> 2) + j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                        dst[((c >> 2) + j) * TILE_M] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
                                                         __uint_as_float(v[4 * j + 3]));
                 }
             }
@@ -230,20 +238,15 @@ conv_splitk_kernel(const __grid_constant__ SkJobs jobs, const int second_begin) 
     }
 
     // ---------------------------------------------------- all slices of the tile meet here
-    // This CTA's share of the tile: float4 elements [f0, f1) of valid_rows x Nj/4, one element per thread and pass;
-    // a thread sums the slices of its element in order 0..splits-1 with up to 16 loads in flight.
+    // This CTA's share of the tile: elements [f0, f1) of the Nj/4 x valid_rows float4 values (column quad major, so
+    // that consecutive threads read consecutive rows of the partial tiles).  A thread owns up to four elements
+    // (e, e + 192, ...) and sums their slices in order 0..splits-1, sixteen loads in flight.
     const long long mrem = p.M - (long long)mt * TILE_M;
     const int valid_rows = mrem < TILE_M ? (int)mrem : TILE_M;
     const int nq = Nj >> 2;
     const int total = valid_rows * nq;
     const int per = (total + splits - 1) / splits;
     const int f0 = split * per, f1 = min(total, f0 + per);
-    // bias of the first element this thread finishes, fetched before the wait (it does not depend on the partials)
-    float4 bias0 = make_float4(0.f, 0.f, 0.f, 0.f);
-    if ((p.flags & DR_BIAS) && f0 + tid < f1) {
-        const int col = n0 + 4 * ((f0 + tid) % nq);
-        if (col < p.Cout) bias0 = make_float4(__ldg(p.bias + col), __ldg(p.bias + col + 1), __ldg(p.bias + col + 2), __ldg(p.bias + col + 3));
-    }
     tc_fence_before();
     __syncthreads();                     // the whole partial tile has been written (by this CTA's threads, in CTA order)
     if (tid == 0) {
@@ -268,46 +271,125 @@ conv_splitk_kernel(const __grid_constant__ SkJobs jobs, const int second_begin) 
         const size_t slice4 = (size_t)TILE_M * (p.Nt >> 2);      // float4 per partial tile
         const float4* part = reinterpret_cast<const float4*>(scratch) + (size_t)tile * splits * slice4;
         const bool f32 = p.flags & DR_OUT_F32;
-        for (int e = f0 + tid; e < f1; e += SK_THREADS) {
-            const int row = e / nq;
-            const int cq = e - row * nq;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            const float4* src = part + (size_t)row * (p.Nt >> 2) + cq;
-#pragma unroll 16
-            for (int sp = 0; sp < splits; ++sp, src += slice4) {
-                const float4 v = __ldcg(src);
-                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        for (int base = f0 + tid; base < f1; base += 4 * SK_THREADS) {
+            int row[4], col[4];
+            const float4* src[4];
+            float4 acc[4], bias[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int e = min(base + q * SK_THREADS, f1 - 1);          // clamped: the extra sums are not stored
+                const int cq = e / valid_rows;
+                row[q] = e - cq * valid_rows;
+                col[q] = n0 + 4 * cq;
+                src[q] = part + (size_t)cq * TILE_M + row[q];
+                acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                bias[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if ((p.flags & DR_BIAS) && col[q] < p.Cout)
+                    bias[q] = make_float4(__ldg(p.bias + col[q]), __ldg(p.bias + col[q] + 1), __ldg(p.bias + col[q] + 2), __ldg(p.bias + col[q] + 3));
             }
-            const int col = n0 + 4 * cq;
-            if (col < p.Cout) {
-                const long long m = (long long)mt * TILE_M + row;
-                if (p.flags & DR_BIAS) {
-                    float4 b = bias0;
-                    if (e != f0 + tid) b = make_float4(__ldg(p.bias + col), __ldg(p.bias + col + 1), __ldg(p.bias + col + 2), __ldg(p.bias + col + 3));
-                    acc.x += b.x; acc.y += b.y; acc.z += b.z; acc.w += b.w;
+#pragma unroll 4
+            for (int sp = 0; sp < splits; ++sp) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float4 v = __ldcg(src[q] + (size_t)sp * slice4);
+                    acc[q].x += v.x; acc[q].y += v.y; acc[q].z += v.z; acc[q].w += v.w;
                 }
-                if (p.flags & DR_RELU) { acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f); acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f); }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (base + q * SK_THREADS >= f1 || col[q] >= p.Cout) continue;
+                float4 a = acc[q];
+                const long long m = (long long)mt * TILE_M + row[q];
+                a.x += bias[q].x; a.y += bias[q].y; a.z += bias[q].z; a.w += bias[q].w;
+                if (p.flags & DR_RELU) { a.x = fmaxf(a.x, 0.f); a.y = fmaxf(a.y, 0.f); a.z = fmaxf(a.z, 0.f); a.w = fmaxf(a.w, 0.f); }
                 if (p.flags & DR_RESIDUAL) {
-                    const uint2 u = __ldg(reinterpret_cast<const uint2*>(p.residual + m * p.Cout + col));
-                    acc.x += bf16_lo(u.x); acc.y += bf16_hi(u.x); acc.z += bf16_lo(u.y); acc.w += bf16_hi(u.y);
-                    if (p.flags & DR_RELU_AFTER_RESIDUAL) { acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f); acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f); }
+                    const uint2 u = __ldg(reinterpret_cast<const uint2*>(p.residual + m * p.Cout + col[q]));
+                    a.x += bf16_lo(u.x); a.y += bf16_hi(u.x); a.z += bf16_lo(u.y); a.w += bf16_hi(u.y);
+                    if (p.flags & DR_RELU_AFTER_RESIDUAL) { a.x = fmaxf(a.x, 0.f); a.y = fmaxf(a.y, 0.f); a.z = fmaxf(a.z, 0.f); a.w = fmaxf(a.w, 0.f); }
                 }
                 if (f32) {
-                    *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.y) + m * p.ldc + p.coff + col) = acc;
+                    *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.y) + m * p.ldc + p.coff + col[q]) = a;
                 } else {
                     uint2 o;
-                    o.x = pack_bf16(acc.x, acc.y);
-                    o.y = pack_bf16(acc.z, acc.w);
-                    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.y) + m * p.ldc + p.coff + col) = o;
+                    o.x = pack_bf16(a.x, a.y);
+                    o.y = pack_bf16(a.z, a.w);
+                    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.y) + m * p.ldc + p.coff + col[q]) = o;
                 }
             }
         }
     }
 
-    __syncthreads();                     // every thread of this CTA has finished reading the partials
-    if (tid == 0)                        // second arrival, not waited for: the last of them wraps the counter back to zero
-        asm volatile("red.relaxed.gpu.global.inc.u32 [%0], %1;" ::"l"(&counters[tile]), "r"(2u * (unsigned)splits - 1u) : "memory");
-    if (*abort_flag) {   // give copies and MMAs still in flight time to land before shared memory and TMEM go away
+    __syncthreads();                     // every thread of this CTA has finished reading the partials and has stored its outputs
+    if (tid == 0) {
+        // second arrival, not waited for: the last of them wraps the counter back to zero
+        red_inc_gpu(&counters[tile], 2u * (unsigned)splits - 1u);
+        if (dep_signal) {                // this CTA's share of the job's output is in memory: tell the job that reads it
+            __threadfence();
+            red_inc_gpu(dep, dep_wrap);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(SK_THREADS, 1) conv_splitk_kernel(const __grid_constant__ SkJobs jobs) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __shared__ SkShared sh;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const bool small = jobs.n >= 2 && (int)blockIdx.x >= jobs.small_begin;
+    const int bid = small ? (int)blockIdx.x - jobs.small_begin : (int)blockIdx.x;
+    const int j0 = small ? 1 : 0;                               // first job of this CTA
+    const int j1 = small && jobs.n == 3 ? 2 : j0;               // last job of this CTA
+    uint32_t tmem_cols = 32;
+    for (int j = j0; j <= j1; ++j) tmem_cols = max(tmem_cols, jobs.j[j].tmem_cols);
+
+    if (tid == 0) {
+        for (int s = 0; s < SK_MAX_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        mbar_init(&sh.accum, 1);
+        sh.abort = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) { tmem_alloc(&sh.tmem_base, tmem_cols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+    // The next kernel in the stream may be scheduled from here on (it waits for this one to finish before it
+    // touches anything this one writes).  Every warp but the producer's waits for the previous kernel right away; the
+    // producer's warp as a whole waits after the filter prefetch (lanes parked in the wait would hold lane 0 back).
+    grid_launch_dependents();
+    if (warp != 0) grid_dependency_wait();
+
+    const unsigned dep_wrap = jobs.n == 3 ? (unsigned)(jobs.j[1].ctas + jobs.j[2].ctas - 1) : 0u;
+    for (int j = j0; j <= j1; ++j) {
+        if (j != j0) {
+            // same CTA, next job: barriers start over (their phases depend on how many k-blocks the last job had)
+            __syncthreads();
+            if (tid == 0) {
+                for (int s = 0; s < SK_MAX_STAGES; ++s) {
+                    mbar_inval(&sh.full[s]); mbar_inval(&sh.empty[s]);
+                    mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1);
+                }
+                mbar_inval(&sh.accum);
+                mbar_init(&sh.accum, 1);
+                fence_barrier_init();
+            }
+            tc_fence_before();
+            __syncthreads();
+            tc_fence_after();
+        }
+        const bool has_work = bid < jobs.j[j].ctas;
+        // one call site per job: inside each, the job's fields are kernel parameters at fixed offsets (constant-bank
+        // operands); a job picked by a run-time index would be read through generic loads again and again
+        if (has_work) {
+            if (j == 0) sk_run_job(&jobs.j[0], bid, sh, smem, tmem, true, nullptr, -1, false, 0u);
+            else if (j == 1) sk_run_job(&jobs.j[1], bid, sh, smem, tmem, true, jobs.dep, -1, jobs.n == 3, dep_wrap);
+            else sk_run_job(&jobs.j[2], bid, sh, smem, tmem, false, jobs.dep, jobs.j[1].ctas, false, dep_wrap);
+        } else if (j == j0 && warp == 0) {
+            grid_dependency_wait();
+        }
+    }
+    __syncthreads();
+    if (sh.abort) {   // give copies and MMAs still in flight time to land before shared memory and TMEM go away
         const long long t0 = clock64();
         while (clock64() - t0 < 400000ll) {}
         __syncthreads();
@@ -395,32 +477,42 @@ bool conv_splitk_supports(const ConvParams& p) {
     return p.sk_scratch_bytes >= pl.scratch_bytes;
 }
 
-// Two layers in one launch: `a` (the long one) and `b` (a short one reading the same input, e.g. a 1x1 reducer).
-// b takes up to 24 CTAs, a the rest.  b's scratch follows a's; b's counters follow a's tiles.
-static const int SK_PAIR_SMALL_CTAS = 24;
-static bool splitk_pair_plan(const ConvParams& a, const ConvParams& b, SkPlan* pa, SkPlan* pb) {
+// Layers of one inception module in one launch: `a` (the long one, job 0), `b` (a short one reading the same input:
+// the 1x1 reducer, job 1) and optionally `c` (the convolution that reads b's output, job 2).  b and c share a small
+// group of CTAs, a takes the rest.  Scratch: a's, then b's, then c's; counters: a's tiles, b's, c's, then the
+// counter on which c waits for b.
+static bool splitk_group_plan(const ConvParams& a, const ConvParams& b, const ConvParams* c, SkPlan* pa, SkPlan* pb, SkPlan* pc) {
     if (tunable("DR_SPLITK_PAIR", 1) == 0) return false;
     if (a.x != b.x || a.B != b.B || a.H != b.H || a.W != b.W || a.Cin != b.Cin) return false;
-    if (!splitk_plan_budget(b, SK_PAIR_SMALL_CTAS, true, pb)) return false;
-    const int used = b.m_tiles * pb->n_blocks * pb->splits;
+    const int small = tunable("DR_SPLITK_SMALL_CTAS", 48);
+    if (!splitk_plan_budget(b, small, true, pb)) return false;
+    int used = b.m_tiles * pb->n_blocks * pb->splits;
+    long long tiles = (long long)b.m_tiles * pb->n_blocks;
+    if (c) {
+        if (c->x != b.y || c->Cin != b.Cout || b.ldc != b.Cout || b.coff != 0 || (b.flags & DR_OUT_F32)) return false;   // c reads b's dense output
+        if (!splitk_plan_budget(*c, small, true, pc)) return false;
+        const int used_c = c->m_tiles * pc->n_blocks * pc->splits;
+        if (used_c > used) used = used_c;
+        tiles += (long long)c->m_tiles * pc->n_blocks + 1;
+    }
     SkPlan alone;
     if (!splitk_plan(a, &alone)) return false;                         // a must be a split-K layer in its own right
     if (!splitk_plan_budget(a, num_sms() - used, false, pa)) return false;
-    if ((long long)a.m_tiles * pa->n_blocks + (long long)b.m_tiles * pb->n_blocks > SK_MAX_TILES) return false;
+    if ((long long)a.m_tiles * pa->n_blocks + tiles > SK_MAX_TILES) return false;
     return true;
 }
 
-size_t conv_splitk_pair_scratch_bytes(const ConvParams& a, const ConvParams& b) {
-    SkPlan pa, pb;
-    if (!splitk_pair_plan(a, b, &pa, &pb)) return 0;
-    return pa.scratch_bytes + pb.scratch_bytes;
+size_t conv_splitk_group_scratch_bytes(const ConvParams& a, const ConvParams& b, const ConvParams* c) {
+    SkPlan pa, pb, pc{};
+    if (!splitk_group_plan(a, b, c, &pa, &pb, &pc)) return 0;
+    return pa.scratch_bytes + pb.scratch_bytes + (c ? pc.scratch_bytes : 0);
 }
 
-bool conv_splitk_pair_supports(const ConvParams& a, const ConvParams& b) {
+bool conv_splitk_group_supports(const ConvParams& a, const ConvParams& b, const ConvParams* c) {
     if (!a.sk_counters || !a.sk_scratch || ((uintptr_t)a.sk_scratch & 255)) return false;
-    SkPlan pa, pb;
-    if (!splitk_pair_plan(a, b, &pa, &pb)) return false;
-    return a.sk_scratch_bytes >= pa.scratch_bytes + pb.scratch_bytes;
+    SkPlan pa, pb, pc{};
+    if (!splitk_group_plan(a, b, c, &pa, &pb, &pc)) return false;
+    return a.sk_scratch_bytes >= pa.scratch_bytes + pb.scratch_bytes + (c ? pc.scratch_bytes : 0);
 }
 
 static int fill_job(const ConvParams& p0, const SkPlan& pl, float* scratch, int* counters, SkJob* j) {
@@ -431,10 +523,11 @@ static int fill_job(const ConvParams& p0, const SkPlan& pl, float* scratch, int*
     if (est != DR_OK) return est;
     j->stages = pl.stages; j->sub_bytes = pl.sub_bytes; j->splits = pl.splits; j->kps = pl.kps; j->tmem_cols = pl.tmem_cols;
     j->scratch = scratch; j->counters = counters;
+    j->ctas = p0.m_tiles * pl.n_blocks * pl.splits;
     return DR_OK;
 }
 
-static int launch_jobs(const SkJobs& jobs, int ctas0, int ctas1, int smem_bytes, cudaStream_t stream) {
+static int launch_jobs(const SkJobs& jobs, int ctas, int smem_bytes, cudaStream_t stream) {
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(conv_splitk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
@@ -454,13 +547,13 @@ static int launch_jobs(const SkJobs& jobs, int ctas0, int ctas1, int smem_bytes,
         attr[0].id = cudaLaunchAttributeCooperative;
         attr[0].val.cooperative = 1;
     }
-    cfg.gridDim = dim3((unsigned)(ctas0 + ctas1));
+    cfg.gridDim = dim3((unsigned)ctas);
     cfg.blockDim = dim3(SK_THREADS);
     cfg.dynamicSmemBytes = (size_t)smem_bytes;
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, conv_splitk_kernel, jobs, ctas0) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, conv_splitk_kernel, jobs) != cudaSuccess) {
         (void)cudaGetLastError();
         return DR_ERR_CUDA;
     }
@@ -474,22 +567,38 @@ int conv_splitk_launch(const ConvParams& p, cudaStream_t stream) {
     SkJobs jobs{};
     const int st = fill_job(p, pl, p.sk_scratch, p.sk_counters, &jobs.j[0]);
     if (st != DR_OK) return st;
+    jobs.n = 1;
     // as many stages as the slice has k-blocks, up to 200 KB: short slices leave room for a CTA of the next layer
     // beside one of this layer on the same SM (at most 256 TMEM columns each)
-    return launch_jobs(jobs, p.m_tiles * pl.n_blocks * pl.splits, 0, pl.stages * pl.sub_bytes + 1024, stream);
+    return launch_jobs(jobs, jobs.j[0].ctas, pl.stages * pl.sub_bytes + 1024, stream);
 }
 
-int conv_splitk_pair_launch(const ConvParams& a, const ConvParams& b, cudaStream_t stream) {
-    SkPlan pa, pb;
-    if (!conv_splitk_pair_supports(a, b) || !splitk_pair_plan(a, b, &pa, &pb)) return DR_ERR_UNSUPPORTED;
+int conv_splitk_group_launch(const ConvParams& a, const ConvParams& b, const ConvParams* c, cudaStream_t stream) {
+    SkPlan pa, pb, pc{};
+    if (!conv_splitk_group_supports(a, b, c) || !splitk_group_plan(a, b, c, &pa, &pb, &pc)) return DR_ERR_UNSUPPORTED;
     SkJobs jobs{};
     int st = fill_job(a, pa, a.sk_scratch, a.sk_counters, &jobs.j[0]);
     if (st != DR_OK) return st;
-    float* scratch_b = reinterpret_cast<float*>(reinterpret_cast<char*>(a.sk_scratch) + pa.scratch_bytes);
-    st = fill_job(b, pb, scratch_b, a.sk_counters + a.m_tiles * pa.n_blocks, &jobs.j[1]);
+    char* scratch = reinterpret_cast<char*>(a.sk_scratch) + pa.scratch_bytes;
+    int* counters = a.sk_counters + a.m_tiles * pa.n_blocks;
+    st = fill_job(b, pb, reinterpret_cast<float*>(scratch), counters, &jobs.j[1]);
     if (st != DR_OK) return st;
-    const int sa = pa.stages * pa.sub_bytes, sb = pb.stages * pb.sub_bytes;
-    return launch_jobs(jobs, a.m_tiles * pa.n_blocks * pa.splits, b.m_tiles * pb.n_blocks * pb.splits, (sa > sb ? sa : sb) + 1024, stream);
+    int smem = pa.stages * pa.sub_bytes;
+    if (pb.stages * pb.sub_bytes > smem) smem = pb.stages * pb.sub_bytes;
+    int small = jobs.j[1].ctas;
+    jobs.n = 2;
+    if (c) {
+        scratch += pb.scratch_bytes;
+        counters += b.m_tiles * pb.n_blocks;
+        st = fill_job(*c, pc, reinterpret_cast<float*>(scratch), counters, &jobs.j[2]);
+        if (st != DR_OK) return st;
+        jobs.dep = counters + c->m_tiles * pc.n_blocks;
+        if (pc.stages * pc.sub_bytes > smem) smem = pc.stages * pc.sub_bytes;
+        if (jobs.j[2].ctas > small) small = jobs.j[2].ctas;
+        jobs.n = 3;
+    }
+    jobs.small_begin = jobs.j[0].ctas;
+    return launch_jobs(jobs, jobs.j[0].ctas + small, smem + 1024, stream);
 }
 
 }  // namespace dr

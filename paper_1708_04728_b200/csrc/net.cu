@@ -53,8 +53,9 @@ struct Op {
     double flops = 0, bytes = 0;
     int path = -1;
     int conv_index = -1;     // OP_CONV: ordinal among the convolutions (its block of split-K counters)
-    int pair = -1;           // OP_CONV: a later convolution reading the same input that may share this one's launch
-    bool pair_ok = false;    // decided by dr_net_prepare
+    int pair = -1;           // OP_CONV: a later convolution reading the same input that may share this one's launch,
+    int chain = -1;          //          and the convolution that reads this one's output (it may join them)
+    int group = 0;           // decided by dr_net_prepare: 0 own launch, 2 with `pair`, 3 with `pair` and `chain`
 };
 
 // Derivations done once by dr_net_prepare
@@ -252,6 +253,7 @@ static void build_googlenet(dr_net* n) {
             // the reducer and the merged branch read the same tensor and write different ones: at small batch they
             // may go out as one launch
             n->ops[i_reducer].pair = (int)n->ops.size() - 1;
+            n->ops[i_reducer].chain = (int)i_reducer + 1;
         } else {
             int r = add_conv(n, mn + ".3x3r.conv", t, 1, 1, 0, m.c3r, DR_BIAS, w3r, b3r);
             r = add_simple(n, OP_RELU, mn + ".3x3r", r);
@@ -430,10 +432,13 @@ int dr_net_create(dr_net** net, int arch, int mode, int B, int H, int W) {
             size_t need = conv_splitk_scratch_bytes(p);
             if (op.pair >= 0) {
                 const Op& oa = n->ops[op.pair];
-                ConvParams pa;
-                if (conv_make_params(&oa.cd, ti.B, ti.H, ti.W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &pa) == DR_OK) {
-                    const size_t both = conv_splitk_pair_scratch_bytes(pa, p);
-                    if (both > need) need = both;
+                const Op& oc = n->ops[op.chain];
+                ConvParams pa, pc;
+                if (conv_make_params(&oa.cd, ti.B, ti.H, ti.W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &pa) == DR_OK &&
+                    conv_make_params(&oc.cd, ti.B, ti.H, ti.W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &pc) == DR_OK) {
+                    const size_t two = conv_splitk_group_scratch_bytes(pa, p, nullptr), three = conv_splitk_group_scratch_bytes(pa, p, &pc);
+                    if (two > need) need = two;
+                    if (three > need) need = three;
                 }
             }
             if (need > n->sk_scratch_bytes) n->sk_scratch_bytes = need;
@@ -514,16 +519,20 @@ int dr_net_prepare(dr_net* n, void* workspace, void* stream) {
         if (op.path < 0) return DR_ERR_UNSUPPORTED;
     }
     for (Op& op : n->ops) {
-        op.pair_ok = false;
+        op.group = 0;
         if (op.kind != OP_CONV || op.pair < 0 || forced_conv_path() != DR_PATH_AUTO) continue;
         const Op& oa = n->ops[op.pair];
+        const Op& oc = n->ops[op.chain];
         const Tensor& ti = n->T(op.in0);
-        ConvParams pa, pb;
+        ConvParams pa, pb, pc;
         const char* dummy = arena;
         if (conv_make_params(&oa.cd, ti.B, ti.H, ti.W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &pa) != DR_OK) continue;
         if (conv_make_params(&op.cd, ti.B, ti.H, ti.W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &pb) != DR_OK) continue;
+        if (conv_make_params(&oc.cd, ti.B, ti.H, ti.W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &pc) != DR_OK) continue;
         set_splitk_scratch(n, oa, ws, &pa);
-        op.pair_ok = oa.path == DR_PATH_UMMA_SPLITK && conv_splitk_pair_supports(pa, pb);
+        if (oa.path != DR_PATH_UMMA_SPLITK) continue;
+        if (conv_splitk_group_supports(pa, pb, &pc)) op.group = 3;
+        else if (conv_splitk_group_supports(pa, pb, nullptr)) op.group = 2;
     }
     n->prepared_ws = workspace;
     return DR_OK;
@@ -558,16 +567,24 @@ int dr_net_forward(dr_net* n, const void* x, void* workspace, float* logits, voi
                 ConvParams p;
                 st = conv_make_params(&op.cd, ti.B, ti.H, ti.W, in0, op.w.resolve(n->raw, ws), (const float*)op.b.resolve(n->raw, ws),
                                       (op.cd.flags & DR_RESIDUAL) ? in1 : nullptr, out, nullptr, &p);
-                if (st == DR_OK && op.pair_ok && !n->timing) {
-                    // this layer and a later one that reads the same input, as one launch (per-layer timing keeps them apart)
+                if (st == DR_OK && op.group && !n->timing) {
+                    // this layer, the later one that reads the same input and (group 3) the one that reads this layer's
+                    // output, as one launch (per-layer timing keeps them apart)
                     const Op& oa = n->ops[op.pair];
-                    ConvParams pa;
+                    const Op& oc = n->ops[op.chain];
+                    ConvParams pa, pc;
                     st = conv_make_params(&oa.cd, ti.B, ti.H, ti.W, in0, oa.w.resolve(n->raw, ws), (const float*)oa.b.resolve(n->raw, ws),
                                           nullptr, (char*)tensor_ptr(n, oa.out, x, arena, logits), nullptr, &pa);
+                    if (st == DR_OK && op.group == 3) {
+                        const Tensor& tc = n->T(oc.in0);
+                        st = conv_make_params(&oc.cd, tc.B, tc.H, tc.W, out, oc.w.resolve(n->raw, ws), (const float*)oc.b.resolve(n->raw, ws),
+                                              nullptr, (char*)tensor_ptr(n, oc.out, x, arena, logits), nullptr, &pc);
+                    }
                     if (st == DR_OK) {
                         set_splitk_scratch(n, oa, (char*)workspace, &pa);
-                        st = conv_splitk_pair_launch(pa, p, s);
+                        st = conv_splitk_group_launch(pa, p, op.group == 3 ? &pc : nullptr, s);
                         n->done[op.pair] = 1;
+                        if (op.group == 3) n->done[op.chain] = 1;
                     }
                     break;
                 }
