@@ -102,8 +102,6 @@ __device__ __forceinline__ void sk_run_job(const SkJob* const J, const int bid, 
     if (warp == 0) {
         if (lane == 0) {
             // -------------------------------------------- TMA producer
-            prefetch_tensormap(&map_a);
-            prefetch_tensormap(&map_b);
             const uint32_t tx = SK_A_BYTES + (uint32_t)p.Nt * 128;
             const long long m0 = (long long)mt * TILE_M;
             const int hw = p.Ho * p.Wo;
@@ -347,6 +345,8 @@ __global__ void __launch_bounds__(SK_THREADS, 1) conv_splitk_kernel(const __grid
         mbar_init(&sh.accum, 1);
         sh.abort = 0;
         fence_barrier_init();
+        // the descriptors of every job this CTA will run, ahead of their first use
+        for (int j = j0; j <= j1; ++j) { prefetch_tensormap(&jobs.j[j].map_a); prefetch_tensormap(&jobs.j[j].map_b); }
     }
     if (warp == 1) { tmem_alloc(&sh.tmem_base, tmem_cols); tmem_relinquish(); }
     tc_fence_before();
