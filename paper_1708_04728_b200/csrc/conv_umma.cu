@@ -376,7 +376,11 @@ struct TmaShared {
 
 // a_mode 0: activations as a plain [M][Cin] matrix (1x1, stride 1, pad 0): 2-D tiled load.
 // a_mode 1: im2col load.
-template <bool PAIR, int KPB>
+// WIDE: a tile carries TWO n-blocks of Nt columns (accumulators at TMEM columns 0 and 256): the activation tile
+// is loaded once and multiplied against both filter sub-tiles, which halves the activation traffic of layers
+// with more than 256 output channels.  All 512 TMEM columns then belong to one tile: the MMAs of the next tile
+// start when both epilogue groups (group g drains sub-block g) have emptied it.
+template <bool PAIR, int KPB, bool WIDE>
 __global__ void __launch_bounds__(T_THREADS, 1)
 conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const int a_mode,
                      const int stages, const int sub_bytes) {
@@ -402,7 +406,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
 
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], PAIR ? 8 : 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], (PAIR ? 8 : 4) * (WIDE ? 2 : 1)); }
         sh.abort = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_a);
@@ -425,13 +429,15 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
     const int total = m_units * p.n_blocks;
     const int cout16 = (p.Cout + 15) & ~15;
     const int hw = p.Ho * p.Wo;
+    const int tile_n = WIDE ? 2 * p.Nt : p.Nt;                 // output channels per tile
+    const uint32_t b_sub_bytes = WIDE ? (uint32_t)(sub_bytes - A_TILE_BYTES) >> 1 : 0u;   // one filter sub-tile
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t full0 = smem_u32(&sh.full[0]), empty0 = smem_u32(&sh.empty[0]);
 
     if (warp == 0) {
         if (lane == 0) {
             // -------------------------------------------- TMA producer
-            const uint32_t cta_tx = A_TILE_BYTES + (uint32_t)(PAIR ? p.Nt >> 1 : p.Nt) * 128;
+            const uint32_t cta_tx = A_TILE_BYTES + (uint32_t)(PAIR ? p.Nt >> 1 : p.Nt) * 128 * (WIDE ? 2 : 1);
             const uint32_t full_mask = PAIR ? PEER_BIT_MASK : 0xFFFFFFFFu;   // pair: bytes are reported to the even CTA
             int s = 0;
             uint32_t ph = 0;
@@ -439,7 +445,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             uint32_t ready = mbar_test_u32(empty0, 1);
             for (int t = unit; t < total && ok; t += nunits) {
                 const int nb = t / m_units, mu = t - nb * m_units;
-                const int n0 = nb * p.Nt;
+                const int n0 = nb * tile_n;
                 int mt = PAIR ? 2 * mu + (int)rank : mu;
                 if (mt >= p.m_tiles) mt = p.m_tiles - 1;   // odd tile count: the peer recomputes the last tile, stores nothing
                 const long long m0 = (long long)mt * TILE_M;
@@ -448,6 +454,8 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                 const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
                 const int hb = ho * p.stride - p.pad, wb = wo * p.stride - p.pad;
                 const int brow = PAIR ? n0 + (int)rank * (min(p.Nt, cout16 - n0) >> 1) : n0;
+                // second sub-block (WIDE); may be narrower than the first, or empty (its rows are then past the tensor: zero fill)
+                const int brow1 = PAIR ? n0 + p.Nt + (int)rank * (max(0, min(p.Nt, cout16 - n0 - p.Nt)) >> 1) : n0 + p.Nt;
                 int r = 0, tt = 0, tap = 0, c0 = 0;
                 for (int remaining = nkb; remaining > 0;) {
                     const int nk = remaining < kpb ? remaining : kpb;
@@ -471,6 +479,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                         if (a_mode == 0) tma_load_2d_u32<PAIR>(a_dst, &map_a, fb, c0, (int)m0, en);
                         else tma_load_im2col_4d_u32<PAIR>(a_dst, &map_a, fb, c0, wb, hb, img, (uint16_t)tt, (uint16_t)r, en);
                         tma_load_3d_u32<PAIR>(a_dst + A_TILE_BYTES, &map_b, fb, c0, tap, brow, en);
+                        if (WIDE) tma_load_3d_u32<PAIR>(a_dst + A_TILE_BYTES + b_sub_bytes, &map_b, fb, c0, tap, brow1, en);
                         c0 += 64;
                         const bool wrap_c = c0 >= p.Cin;
                         c0 = wrap_c ? 0 : c0;
@@ -488,32 +497,37 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0 && rank == 0) {
-            // -------------------------------------------- MMA issue
+        if (rank == 0) {
+            // -------------------------------------------- MMA issue.  The whole warp walks the loop (so that the
+            // addresses and descriptors are warp-uniform values); lane 0 alone issues the MMAs and commits.
+            const uint32_t el = lane == 0 ? 1u : 0u;
             const uint32_t tfull0 = smem_u32(&sh.tfull[0]), tempty0 = smem_u32(&sh.tempty[0]);
             const int last_nk16 = ((p.Cin - ((cpb - 1) << 6)) + 15) >> 4;
             int s = 0, it = 0;
             uint32_t ph = 0;
             bool ok = true;
-            uint32_t ready = mbar_test_u32(full0, 0);
+            bool ready = __all_sync(0xffffffffu, mbar_test_u32(full0, 0) != 0);
             for (int t = unit; t < total && ok; t += nunits, ++it) {
                 const int nb = t / m_units;
-                const int Nj = min(p.Nt, cout16 - nb * p.Nt);
+                const int Nj = min(p.Nt, cout16 - nb * tile_n);
                 const uint32_t idesc = make_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, Nj);
-                const int acc = it & 1, au = it >> 1;
-                if (!mbar_wait_u32(tempty0 + 8 * acc, (au & 1) ^ 1, abort_flag)) {
-                    if (!*abort_flag) report_timeout(p.status, 12, t);
+                const int Nj1 = WIDE ? min(p.Nt, cout16 - nb * tile_n - p.Nt) : 0;          // second sub-block; <= 0: none
+                const uint32_t idesc1 = make_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, Nj1 > 0 ? Nj1 : 16);
+                const uint32_t el1 = (WIDE && Nj1 > 0) ? el : 0u;
+                const int acc = WIDE ? 0 : (it & 1), au = WIDE ? it : (it >> 1);
+                if (!__all_sync(0xffffffffu, mbar_wait_u32(tempty0 + 8 * acc, (au & 1) ^ 1, abort_flag))) {
+                    if (el && !*abort_flag) report_timeout(p.status, 12, t);
                     *abort_flag = 1;
                     break;
                 }
                 tc_fence_after();
                 const uint32_t d = tmem + (uint32_t)(acc * T_ACC_COLS);
-                uint32_t accum = 0;
+                uint32_t accum = 0, accum1 = 0;
                 int cc = 0;
                 for (int remaining = nkb; remaining > 0;) {
                     const int nk = remaining < kpb ? remaining : kpb;
-                    if (!ready && !mbar_wait_slow_u32(full0 + 8 * s, ph, abort_flag)) {
-                        if (!*abort_flag) report_timeout(p.status, 13, t);
+                    if (!ready && !__all_sync(0xffffffffu, mbar_wait_slow_u32(full0 + 8 * s, ph, abort_flag))) {
+                        if (el && !*abort_flag) report_timeout(p.status, 13, t);
                         *abort_flag = 1;
                         ok = false;
                         break;
@@ -521,7 +535,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                     int s2 = s + 1;
                     uint32_t ph2 = ph;
                     if (s2 == stages) { s2 = 0; ph2 ^= 1; }
-                    ready = mbar_test_u32(full0 + 8 * s2, ph2);               // probe the next slot while this one is issued
+                    ready = __all_sync(0xffffffffu, mbar_test_u32(full0 + 8 * s2, ph2) != 0);   // probe the next slot while this one is issued
                     tc_fence_after();
                     uint32_t a = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
 #pragma unroll
@@ -529,18 +543,27 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                         const uint32_t alo = sdesc_lo(a), blo = sdesc_lo(a + A_TILE_BYTES);
                         const int nk16 = j < nk ? ((cc == cpb - 1) ? last_nk16 : 4) : 0;    // 0: nothing in this sub-stage
                         cc = (cc + 1 == cpb) ? 0 : cc + 1;
-                        umma_bf16_lo<PAIR>(d, alo, blo, idesc, accum, nk16 > 0);
+                        umma_bf16_lo<PAIR>(d, alo, blo, idesc, accum, (nk16 > 0) & el);
                         accum = 1;
-                        umma_bf16_lo<PAIR>(d, alo + 2, blo + 2, idesc, 1u, nk16 > 1);
-                        umma_bf16_lo<PAIR>(d, alo + 4, blo + 4, idesc, 1u, nk16 > 2);
-                        umma_bf16_lo<PAIR>(d, alo + 6, blo + 6, idesc, 1u, nk16 > 3);
+                        umma_bf16_lo<PAIR>(d, alo + 2, blo + 2, idesc, 1u, (nk16 > 1) & el);
+                        umma_bf16_lo<PAIR>(d, alo + 4, blo + 4, idesc, 1u, (nk16 > 2) & el);
+                        umma_bf16_lo<PAIR>(d, alo + 6, blo + 6, idesc, 1u, (nk16 > 3) & el);
+                        if (WIDE) {
+                            const uint32_t blo1 = sdesc_lo(a + A_TILE_BYTES + b_sub_bytes);
+                            const uint32_t d1 = d + (uint32_t)T_ACC_COLS;
+                            umma_bf16_lo<PAIR>(d1, alo, blo1, idesc1, accum1, (nk16 > 0) & el1);
+                            accum1 = 1;
+                            umma_bf16_lo<PAIR>(d1, alo + 2, blo1 + 2, idesc1, 1u, (nk16 > 1) & el1);
+                            umma_bf16_lo<PAIR>(d1, alo + 4, blo1 + 4, idesc1, 1u, (nk16 > 2) & el1);
+                            umma_bf16_lo<PAIR>(d1, alo + 6, blo1 + 6, idesc1, 1u, (nk16 > 3) & el1);
+                        }
                     }
-                    umma_commit_u32<PAIR>(empty0 + 8 * s);
+                    if (el) umma_commit_u32<PAIR>(empty0 + 8 * s);
                     remaining -= nk;
                     s = s2;
                     ph = ph2;
                 }
-                if (ok) umma_commit_u32<PAIR>(tfull0 + 8 * acc);
+                if (ok && el) umma_commit_u32<PAIR>(tfull0 + 8 * acc);
             }
         }
         __syncwarp();
@@ -550,12 +573,12 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
         const int g = (warp - 2) >> 2;
         const int q = warp & 3;
         const int row = q * 32 + lane;
-        for (int t = unit + g * nunits, au = 0; t < total; t += 2 * nunits, ++au) {
+        for (int t = WIDE ? unit : unit + g * nunits, au = 0; t < total; t += WIDE ? nunits : 2 * nunits, ++au) {
             const int nb = t / m_units, mu = t - nb * m_units;
-            const int n0 = nb * p.Nt;
-            const int Nj = min(p.Nt, cout16 - n0);
+            const int n0 = WIDE ? nb * tile_n + g * p.Nt : nb * p.Nt;      // WIDE: group g drains sub-block g of every tile
+            const int Nj = min(p.Nt, cout16 - n0);                         // WIDE: may be <= 0 (no second sub-block)
             const int mt = PAIR ? 2 * mu + (int)rank : mu;
-            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[g], au & 1, abort_flag));
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[WIDE ? 0 : g], au & 1, abort_flag));
             if (!ok) {
                 if (!*abort_flag) report_timeout(p.status, 14, t);
                 *abort_flag = 1;
@@ -565,7 +588,9 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             const long long m = (long long)mt * TILE_M + row;
             const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * T_ACC_COLS);
             const bool row_ok = mt < p.m_tiles && m < p.M;
-            if (lean) {
+            if (WIDE && Nj <= 0) {
+                // nothing to drain
+            } else if (lean) {
                 if (lean_mode == 1) drain_fast<1>(p, taddr, Nj, m, row_ok, n0, bias_s);
                 else if (lean_mode == 3) drain_fast<3>(p, taddr, Nj, m, row_ok, n0, bias_s);
                 else if (lean_mode == 0) drain_fast<0>(p, taddr, Nj, m, row_ok, n0, bias_s);
@@ -576,8 +601,8 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
-                if (PAIR) mbar_arrive_leader(&sh.tempty[g]);
-                else mbar_arrive(&sh.tempty[g]);
+                if (PAIR) mbar_arrive_leader(&sh.tempty[WIDE ? 0 : g]);
+                else mbar_arrive(&sh.tempty[WIDE ? 0 : g]);
             }
         }
     }
@@ -687,12 +712,12 @@ static void pick_pipeline(int sub_bytes, int nkb, int nt, int* kpb, int* stages)
     *stages = st;
 }
 
-static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, int a_mode, cudaStream_t stream) {
+static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, int a_mode, bool wide, cudaStream_t stream) {
     static bool attr_set = false;
     static int max_clusters = 0;
-    const int sub_bytes = A_TILE_BYTES + ((p.Nt * 64 + 1023) & ~1023);
+    const int sub_bytes = A_TILE_BYTES + (wide ? 2 : 1) * ((p.Nt * 64 + 1023) & ~1023);
     int kpb, stages;
-    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), p.Nt, &kpb, &stages);
+    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, &kpb, &stages);
     int smem_bytes = stages * kpb * sub_bytes + 1024;
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
     cudaLaunchConfig_t cfg = {};
@@ -702,13 +727,14 @@ static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUte
     cfg.blockDim = dim3(T_THREADS); cfg.dynamicSmemBytes = (size_t)smem_bytes; cfg.stream = stream;
     cfg.attrs = attr; cfg.numAttrs = 1;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(conv_umma_tma_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
-            cudaFuncSetAttribute(conv_umma_tma_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
-            cudaFuncSetAttribute(conv_umma_tma_kernel<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess)
+        if (cudaFuncSetAttribute(conv_umma_tma_kernel<true, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_umma_tma_kernel<true, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_umma_tma_kernel<true, 4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_umma_tma_kernel<true, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess)
             return DR_ERR_CUDA;
         cfg.gridDim = dim3(2 * num_sms());
         cfg.dynamicSmemBytes = (size_t)T_SMEM_MAX;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, conv_umma_tma_kernel<true, 1>, &cfg) != cudaSuccess || max_clusters < 1) return DR_ERR_CUDA;
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, conv_umma_tma_kernel<true, 1, false>, &cfg) != cudaSuccess || max_clusters < 1) return DR_ERR_CUDA;
         cfg.dynamicSmemBytes = (size_t)smem_bytes;
         attr_set = true;
     }
@@ -716,46 +742,72 @@ static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUte
     const int pairs = pair_tiles < max_clusters ? pair_tiles : max_clusters;
     cfg.gridDim = dim3(2 * pairs);
     cudaError_t e;
-    if (kpb == 4) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 4>, p, map_a, map_b, a_mode, stages, sub_bytes);
-    else if (kpb == 2) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 2>, p, map_a, map_b, a_mode, stages, sub_bytes);
-    else e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 1>, p, map_a, map_b, a_mode, stages, sub_bytes);
+    if (wide) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 1, true>, p, map_a, map_b, a_mode, stages, sub_bytes);
+    else if (kpb == 4) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 4, false>, p, map_a, map_b, a_mode, stages, sub_bytes);
+    else if (kpb == 2) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 2, false>, p, map_a, map_b, a_mode, stages, sub_bytes);
+    else e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 1, false>, p, map_a, map_b, a_mode, stages, sub_bytes);
     if (e != cudaSuccess) return DR_ERR_CUDA;
     count_launch();
     return launch_status();
 }
 
-int conv_umma_tma_launch(const ConvParams& p, cudaStream_t stream) {
-    if (!conv_umma_tma_supports(p)) return DR_ERR_UNSUPPORTED;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(conv_umma_tma_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
-            cudaFuncSetAttribute(conv_umma_tma_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
-            cudaFuncSetAttribute(conv_umma_tma_kernel<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess)
-            return DR_ERR_CUDA;
-        attr_set = true;
-    }
+int conv_umma_tma_launch(const ConvParams& p_in, cudaStream_t stream) {
+    if (!conv_umma_tma_supports(p_in)) return DR_ERR_UNSUPPORTED;
+    ConvParams p = p_in;
     // CTA pairs pay off where the MMAs dominate: long K, or a spatial filter with K >= 512 (measured: +12 % on the
     // 3x3 layers, -20 % on the 1x1 reducers)
     const int pair_pref = tunable("DR_TMA_PAIR", -1);
     const bool use_pair = pair_pref >= 0 ? pair_pref != 0 : ((p.K >= 1024 || (p.k > 1 && p.K >= 512)) && p.m_tiles >= 2);
+    // More than 256 output channels and a long K: wide tiles (two n-blocks per tile sharing the activation tile) of
+    // near-equal sub-blocks, e.g. 288 -> one tile of 144 + 144, unless the coarser tiles cost more in rounds of the
+    // persistent grid than the shared activation tile saves (measured: 5 to 9 % on the merged 5x5 layers of stage 4;
+    // short-K layers lose more to the epilogue, which wide tiles do not overlap with the next tile's MMAs).
+    const int cout16_ = (p.Cout + 15) / 16 * 16;
+    const int wide_pref = tunable("DR_TMA_WIDE", -1);
+    bool wide = false;
+    int nt_w = 0, n_wide = 0;
+    if (cout16_ > 32) {
+        n_wide = (cout16_ + 511) / 512;
+        nt_w = ((cout16_ + 2 * n_wide - 1) / (2 * n_wide) + 15) / 16 * 16;
+        const long long capacity = use_pair ? num_sms() / 2 : num_sms();
+        const long long m_units = use_pair ? (p.m_tiles + 1) / 2 : p.m_tiles;
+        const long long cost_n = (m_units * p.n_blocks + capacity - 1) / capacity * p.Nt;
+        const long long cost_w = (m_units * n_wide + capacity - 1) / capacity * 2 * nt_w;
+        const int nkb_ = p.k * p.k * ((p.Cin + 63) / 64);
+        wide = wide_pref >= 0 ? wide_pref != 0 : (cout16_ > 256 && nkb_ >= 48 && cost_w * 95 <= cost_n * 100);
+    }
+    if (wide) {
+        p.Nt = nt_w;
+        p.n_blocks = n_wide;
+    }
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(conv_umma_tma_kernel<false, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_umma_tma_kernel<false, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_umma_tma_kernel<false, 4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_umma_tma_kernel<false, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess)
+            return DR_ERR_CUDA;
+        attr_set = true;
+    }
     alignas(64) CUtensorMap map_a, map_b;
     int a_mode = 0;
     const int est = encode_conv_maps(p, use_pair ? p.Nt / 2 : p.Nt, &map_a, &map_b, &a_mode);   // a pair's CTAs load half of B each
     if (est != DR_OK) return est;
     const int total = p.m_tiles * p.n_blocks;
     if (total <= 0) return DR_OK;
-    if (use_pair) return launch_pair(p, map_a, map_b, a_mode, stream);
+    if (use_pair) return launch_pair(p, map_a, map_b, a_mode, wide, stream);
     const int grid = total < num_sms() ? total : num_sms();
     // as many pipeline stages as shared memory holds (the B tile shrinks with Nt); always more than
     // half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
-    const int sub_bytes = A_TILE_BYTES + ((p.Nt * 128 + 1023) & ~1023);
+    const int sub_bytes = A_TILE_BYTES + (wide ? 2 : 1) * ((p.Nt * 128 + 1023) & ~1023);
     int kpb, stages;
-    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), p.Nt, &kpb, &stages);
+    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, &kpb, &stages);
     int smem_bytes = stages * kpb * sub_bytes + 1024;
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
-    if (kpb == 4) conv_umma_tma_kernel<false, 4><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
-    else if (kpb == 2) conv_umma_tma_kernel<false, 2><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
-    else conv_umma_tma_kernel<false, 1><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
+    if (wide) conv_umma_tma_kernel<false, 1, true><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
+    else if (kpb == 4) conv_umma_tma_kernel<false, 4, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
+    else if (kpb == 2) conv_umma_tma_kernel<false, 2, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
+    else conv_umma_tma_kernel<false, 1, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
     count_launch();
     return launch_status();
 }
