@@ -206,6 +206,223 @@ conv_patch_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap ma
 }
 
 // =====================================================================================
+//                         patch kernel on CTA pairs, filters resident
+// =====================================================================================
+// conv_patch_tma_kernel streams the filter tile of every tap again for every patch: 24 KB of filters next to
+// 15 KB of activations per k-block (GoogLeNet conv2: 1.9 GB of filter loads against 1.2 GB of activation loads
+// per batch of 256).  Here two CTAs
+// of a cluster form one MMA unit (tcgen05 cta_group::2, M = 256 = one patch per CTA); each keeps HALF of the
+// filter bank in shared memory for the whole kernel (`resident`), or streams only its half (`!resident`), and the
+// even CTA issues MMAs that read both shared memories.  Barrier protocol as in conv_umma_tma_kernel<PAIR>:
+// loads of both CTAs report to the even CTA's barriers, its commits arrive in both CTAs, epilogue warps of both
+// CTAs arrive on the even CTA's `tempty`.  No multicast loads.
+struct PatchPairShared {
+    uint64_t full[P_MAX_STAGES], empty[P_MAX_STAGES], tfull[2], tempty[2], wfull;
+    uint32_t tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ void tma_load_4d_tile_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(
+                     dst),
+                 "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+
+__global__ void __launch_bounds__(P_THREADS, 1)
+conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const int stages,
+                       const int stage_bytes, const int groups, const int resident, const int bsub_bytes) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __shared__ PatchPairShared sh;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cpb = (p.Cin + 63) >> 6;
+    const int nkb = p.k * p.k * cpb;
+    uint8_t* b_res = smem + stages * stage_bytes;                            // resident half filter bank: nkb sub-tiles
+    uint8_t* fe_stage = b_res + (resident ? nkb * bsub_bytes : 0);
+    const uint32_t rank = cluster_ctarank();                                 // 0 issues the MMAs
+    const int unit = (int)(blockIdx.x >> 1), nunits = (int)(gridDim.x >> 1);
+
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 8); }
+        mbar_init(&sh.wfull, 1);
+        sh.abort = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+    }
+    if (warp == 1) { tmem_alloc_pair(&sh.tmem_base, 512); tmem_relinquish_pair(); }
+    const int fe_bytes = fe_smem_bytes(p);
+    fe_init(p, fe_stage, tid, P_THREADS);
+    if (groups > 1) fe_init(p, fe_stage + fe_bytes, tid, P_THREADS);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                                      // both CTAs' barriers exist before any remote arrive
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+    volatile int* abort_flag = &sh.abort;
+
+    const int total = p.m_tiles;
+    const int units = (total + 1) >> 1;                                      // pair tiles: patches 2u and 2u+1
+    const int per = p.tiles_h * p.tiles_w;
+    const int pwc = 2 * p.PW + 1, phc = 2 * p.PH + 1;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t full0 = smem_u32(&sh.full[0]), empty0 = smem_u32(&sh.empty[0]);
+    const uint32_t b_res0 = smem_u32(b_res);
+    const uint32_t half_rows = (uint32_t)p.Nt >> 1;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint32_t a_tx = (uint32_t)(pwc * phc) * 128u;
+            const uint32_t b_tx = half_rows * 128u;
+            const int brow = (int)rank * (int)half_rows;
+            if (resident) {
+                const uint32_t wb = smem_u32(&sh.wfull) & PEER_BIT_MASK;
+                if (rank == 0) mbar_expect_tx_u32(wb, 2u * (uint32_t)nkb * b_tx);
+                int tap = 0, c0 = 0;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    tma_load_3d_u32<true>(b_res0 + (uint32_t)kb * (uint32_t)bsub_bytes, &map_b, wb, c0, tap, brow, 1u);
+                    c0 += 64;
+                    if (c0 >= p.Cin) { c0 = 0; ++tap; }
+                }
+            }
+            const uint32_t tx = a_tx + (resident ? 0u : b_tx);
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            uint32_t ready = mbar_test_u32(empty0, 1);
+            for (int u = unit; u < units && ok; u += nunits) {
+                int t = 2 * u + (int)rank;
+                if (t >= total) t = total - 1;                               // odd patch count: the peer repeats the last patch (same values stored twice)
+                const int n = t / per, tt_ = t - n * per;
+                const int th = tt_ / p.tiles_w, tw = tt_ - th * p.tiles_w;
+                const int h0 = 2 * th * p.PH - 1 - p.pad, w0 = 2 * tw * p.PW - 1 - p.pad;   // stride 1
+                int r = 0, q = 0, tap = 0, c0 = 0;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!ready && !mbar_wait_slow_u32(empty0 + 8 * s, ph ^ 1, abort_flag)) {
+                        if (!*abort_flag) report_timeout(p.status, 41, t);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    int s2 = s + 1;
+                    uint32_t ph2 = ph;
+                    if (s2 == stages) { s2 = 0; ph2 ^= 1; }
+                    ready = mbar_test_u32(empty0 + 8 * s2, ph2 ^ 1);
+                    const uint32_t a_dst = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+                    const uint32_t fb = (full0 + 8 * s) & PEER_BIT_MASK;
+                    if (rank == 0) mbar_expect_tx_u32(fb, 2u * tx);
+                    tma_load_4d_tile_pair(a_dst, &map_a, fb, c0, w0 + q, h0 + r, n);
+                    if (!resident) tma_load_3d_u32<true>(a_dst + P_A_BYTES, &map_b, fb, c0, tap, brow, 1u);
+                    c0 += 64;
+                    const bool wrap_c = c0 >= p.Cin;
+                    c0 = wrap_c ? 0 : c0;
+                    tap += wrap_c ? 1 : 0;
+                    q += wrap_c ? 1 : 0;
+                    const bool wrap_q = q == p.k;
+                    q = wrap_q ? 0 : q;
+                    r += wrap_q ? 1 : 0;
+                    s = s2;
+                    ph = ph2;
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            const uint32_t tfull0 = smem_u32(&sh.tfull[0]), tempty0 = smem_u32(&sh.tempty[0]);
+            const int last_nk16 = ((p.Cin - ((cpb - 1) << 6)) + 15) >> 4;
+            const uint32_t idesc = make_idesc_bf16(2 * TILE_M, p.Nt);
+            int s = 0, it = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            if (resident && !mbar_wait(&sh.wfull, 0, abort_flag)) {
+                if (!*abort_flag) report_timeout(p.status, 45, 0);
+                *abort_flag = 1;
+                ok = false;
+            }
+            uint32_t ready = mbar_test_u32(full0, 0);
+            for (int u = unit; u < units && ok; u += nunits, ++it) {
+                const int acc = it & 1, au = it >> 1;
+                if (!mbar_wait_u32(tempty0 + 8 * acc, (au & 1) ^ 1, abort_flag)) {
+                    if (!*abort_flag) report_timeout(p.status, 42, u);
+                    *abort_flag = 1;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d = tmem + (uint32_t)(acc * 256);
+                uint32_t accum = 0;
+                int cc = 0;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!ready && !mbar_wait_slow_u32(full0 + 8 * s, ph, abort_flag)) {
+                        if (!*abort_flag) report_timeout(p.status, 43, u);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    int s2 = s + 1;
+                    uint32_t ph2 = ph;
+                    if (s2 == stages) { s2 = 0; ph2 ^= 1; }
+                    ready = mbar_test_u32(full0 + 8 * s2, ph2);
+                    tc_fence_after();
+                    const uint32_t a = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+                    const uint32_t alo = sdesc_lo(a);
+                    const uint32_t blo = sdesc_lo(resident ? b_res0 + (uint32_t)kb * (uint32_t)bsub_bytes : a + P_A_BYTES);
+                    const int nk16 = (cc == cpb - 1) ? last_nk16 : 4;
+                    cc = (cc + 1 == cpb) ? 0 : cc + 1;
+                    umma_bf16_lo<true>(d, alo, blo, idesc, accum, 1u);
+                    accum = 1;
+                    umma_bf16_lo<true>(d, alo + 2, blo + 2, idesc, 1u, nk16 > 1);
+                    umma_bf16_lo<true>(d, alo + 4, blo + 4, idesc, 1u, nk16 > 2);
+                    umma_bf16_lo<true>(d, alo + 6, blo + 6, idesc, 1u, nk16 > 3);
+                    umma_commit_u32<true>(empty0 + 8 * s);
+                    s = s2;
+                    ph = ph2;
+                }
+                if (ok) umma_commit_u32<true>(tfull0 + 8 * acc);
+            }
+        }
+        __syncwarp();
+    } else {
+        // epilogue groups of four warps, as in conv_patch_tma_kernel; each CTA drains its own patch
+        const int g = (warp - 2) >> 2;
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        if (g < groups) {
+            for (int it = g;; it += groups) {
+                const int u = unit + it * nunits;
+                if (u >= units) break;
+                int t = 2 * u + (int)rank;
+                if (t >= total) t = total - 1;
+                const int acc = it & 1, au = it >> 1;
+                const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[acc], au & 1, abort_flag));
+                if (!ok) {
+                    if (!*abort_flag) report_timeout(p.status, 44, t);
+                    *abort_flag = 1;
+                    break;
+                }
+                tc_fence_after();
+                uint64_t* te = &sh.tempty[acc];
+                fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * 256), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_leader(te);
+                });
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) {}
+        __syncthreads();
+    }
+    cluster_sync_all();                                                      // neither CTA leaves while the other may still signal it
+    if (warp == 1) tmem_dealloc_pair(tmem, 512);
+}
+
+// =====================================================================================
 //                                     stem kernel
 // =====================================================================================
 constexpr int S_THREADS = 416;          // warps 0-3 producers, warp 4 MMA, warps 5-8 and 9-12: two epilogue groups
@@ -455,6 +672,59 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
             return DR_ERR_CUDA;
     }
     if (p.m_tiles <= 0) return DR_OK;
+    // CTA pairs with each CTA's half of the filter bank resident in shared memory (or, if that does not fit, streamed):
+    // the filters are what this layer moves most of otherwise.  Measured on GoogLeNet conv2 at batch 256.
+    if (tunable("DR_PATCH_PAIR", 1) != 0 && p.m_tiles >= 2 && (p.Nt & 31) == 0) {
+        static bool pair_attr = false;
+        static int max_clusters = 0;
+        const int nkb = p.k * p.k * ((p.Cin + 63) / 64);
+        const int bsub = ((p.Nt / 2) * 128 + 1023) & ~1023;
+        const int budget = P_SMEM_MAX - 2048;
+        const int fe = fe_smem_bytes(p);
+        int groups = 0, stages = 0, resident = 0, stage_bytes = 0;
+        const int res_pref = tunable("DR_PATCH_RESIDENT", -1);
+        // two epilogue groups first (the fused LRN / pooling epilogue is what bounds these layers: conv2 takes 336 us with
+        // two groups and streamed half-filters, 433 us with one group and resident filters), then resident filters
+        for (int g = 2; g >= 1 && !groups; --g)
+            for (int res = 1; res >= 0 && !groups; --res) {
+                if (res_pref >= 0 && res != res_pref) continue;
+                const int sb = P_A_BYTES + (res ? 0 : bsub);
+                const int left = budget - g * fe - (res ? nkb * bsub : 0);
+                if (left / sb >= 3) { groups = g; resident = res; stage_bytes = sb; stages = left / sb; }
+            }
+        if (groups) {
+            if (stages > P_MAX_STAGES) stages = P_MAX_STAGES;
+            cudaLaunchConfig_t cfg = {};
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.blockDim = dim3(P_THREADS); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
+            if (!pair_attr) {
+                if (cudaFuncSetAttribute(conv_patch_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+                cfg.gridDim = dim3(2 * num_sms());
+                cfg.dynamicSmemBytes = (size_t)P_SMEM_MAX;
+                if (cudaOccupancyMaxActiveClusters(&max_clusters, conv_patch_pair_kernel, &cfg) != cudaSuccess || max_clusters < 1) return DR_ERR_CUDA;
+                pair_attr = true;
+            }
+            alignas(64) CUtensorMap map_bh;
+            const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
+            const cuuint64_t strides[2] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.K * 2};
+            const cuuint32_t box[3] = {64, 1, (cuuint32_t)(p.Nt / 2)};      // each CTA of a pair holds half of the filters
+            const cuuint32_t es[3] = {1, 1, 1};
+            if (g_enc(&map_bh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)p.w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return DR_ERR_CUDA;
+            int smem_bytes = stages * stage_bytes + (resident ? nkb * bsub : 0) + groups * fe + 1024;
+            if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
+            const int units = (p.m_tiles + 1) / 2;
+            const int pairs = units < max_clusters ? units : max_clusters;
+            cfg.gridDim = dim3(2 * pairs);
+            cfg.dynamicSmemBytes = (size_t)smem_bytes;
+            if (cudaLaunchKernelEx(&cfg, conv_patch_pair_kernel, p, map_a, map_bh, stages, stage_bytes, groups, resident, bsub) != cudaSuccess) return DR_ERR_CUDA;
+            count_launch();
+            return launch_status();
+        }
+    }
     const int stage_bytes = P_A_BYTES + ((p.Nt * 128 + 1023) & ~1023);
     // two epilogue groups when that still leaves three pipeline stages, else one group and the extra stages
     // (conv2 of GoogLeNet: 350 us with 2 groups / 3 stages, 361 us with 1 group / 4 stages)
