@@ -28,7 +28,7 @@ if ROOT not in sys.path:
 METRIC = "slim GoogLeNet forward throughput"
 UNIT = "images/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of conv_umma_tma_kernel on layer 3b.m5 at batch 256 (ncu --set full)
-NCU_TRAFFIC_3B_M5 = 207.338e6 + 87.581e6
+NCU_TRAFFIC_3B_M5 = 106.539e6 + 69.194e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -49,7 +49,7 @@ class ClockSampler:
     def __init__(self, index: int):
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
-            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
                                        "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
@@ -64,25 +64,27 @@ class ClockSampler:
         except Exception:
             self.p.kill()
         self.f.flush(); self.f.seek(0)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         for line in self.f.read().splitlines():
             c = [x.strip() for x in line.split(",")]
             if len(c) < 9:
                 continue
             try:
-                sm.append(float(c[1])); mx.append(float(c[2]))
+                sm.append(float(c[1])); mx.append(float(c[2])); pw.append(float(c[3]))
             except ValueError:
                 continue
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
+        if len(sm) >= 4:      # samples under load: the half with the higher power draw (idle samples before/after the region drag the median)
+            order = sorted(range(len(sm)), key=lambda i: pw[i])[len(sm) // 2:]
+            sm = [sm[i] for i in order]
         self.f.close()
         try:
             os.unlink(self.f.name)
         except OSError:
             pass
         if sm:
-            # samples under load: the upper half (idle samples before/after the region drag the median down)
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
         return out
 
@@ -176,7 +178,7 @@ def run_layer(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=None, help="default 256 (GoogLeNet), 128 (ResNet-50)")
