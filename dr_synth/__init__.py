@@ -83,3 +83,12 @@ INCEPTION_V1 = {
 
 # ResNet-50 stages: (bottleneck width, number of blocks); output channels are 4x the width.
 RESNET50_STAGES = ((64, 3), (128, 4), (256, 6), (512, 3))
+
+
+# AlexNet (the grouped two-tower form): (name, Cout, k, stride, pad, groups, Cin of the whole layer).
+# fc6 is written as a 6x6 convolution over the 6x6x256 plane that pool5 leaves for a 227x227 image.
+ALEXNET_CONVS = (
+    ("conv1", 96, 11, 4, 0, 1, 3), ("conv2", 256, 5, 1, 2, 2, 96), ("conv3", 384, 3, 1, 1, 1, 256),
+    ("conv4", 384, 3, 1, 1, 2, 384), ("conv5", 256, 3, 1, 1, 2, 384),
+    ("fc6", 4096, 6, 1, 0, 1, 256), ("fc7", 4096, 1, 1, 0, 1, 4096), ("fc8", 1000, 1, 1, 0, 1, 4096),
+)

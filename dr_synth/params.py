@@ -18,7 +18,7 @@ from __future__ import annotations
 
 import numpy as np
 
-from . import INCEPTION_V1, RESNET50_STAGES, he_normal, normal, uniform
+from . import ALEXNET_CONVS, INCEPTION_V1, RESNET50_STAGES, he_normal, normal, uniform
 
 
 def conv_params(seed, name, cout, k, cin, bias=True):
@@ -97,6 +97,14 @@ def resnet50_params(seed=0):
         p.update(conv_params(seed, name, cout, k, cin, bias=False))
         p.update(bn_params(seed, f"{name}.bn", cout))
     p.update(conv_params(seed, "fc", 1000, 1, 2048))
+    return p
+
+
+def alexnet_params(seed=0):
+    """AlexNet: grouped filters are stored per group, [Cout][k][k][Cin / groups]; He-normal on that fan-in."""
+    p = {}
+    for name, cout, k, _s, _p, groups, cin in ALEXNET_CONVS:
+        p.update(conv_params(seed, name, cout, k, cin // groups))
     return p
 
 

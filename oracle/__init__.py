@@ -70,6 +70,18 @@ def conv2d(x, w, bias=None, stride=1, pad=0):
     return y
 
 
+def conv2d_grouped(x, w, bias=None, stride=1, pad=0, groups=1):
+    """Grouped convolution by its definition: group g convolves input channels [g*Cin_g, (g+1)*Cin_g) with filters
+    [g*Cout_g, (g+1)*Cout_g) and the group outputs are concatenated along channels.  w: [Cout][k][k][Cin_g]."""
+    Cout, Cin_g = w.shape[0], w.shape[3]
+    assert x.shape[3] == Cin_g * groups and Cout % groups == 0
+    cg = Cout // groups
+    parts = [conv2d(np.ascontiguousarray(x[..., g * Cin_g:(g + 1) * Cin_g]), np.ascontiguousarray(w[g * cg:(g + 1) * cg]),
+                    None if bias is None else np.ascontiguousarray(np.asarray(bias)[g * cg:(g + 1) * cg]), stride, pad)
+             for g in range(groups)]
+    return concat(parts)
+
+
 def batchnorm(x, mu, sigma2, m=1.0, eps=0.0):
     C = x.shape[-1]
     x, px = _d(x); mu, pm = _d(mu); sigma2, pv = _d(sigma2)

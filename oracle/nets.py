@@ -182,6 +182,38 @@ def resnet50_steps(params, eps=1e-5):
     return steps
 
 
+# AlexNet, two-tower (grouped) form: (name, stride, pad, groups); LRN after conv1 and conv2, 3x3/2 pooling without
+# padding after norm1, norm2 and conv5; fc6 is a 6x6 convolution over the 6x6 plane; dropout is the identity at
+# inference; no softmax (logits).
+_ALEXNET = (("conv1", 4, 0, 1), ("conv2", 1, 2, 2), ("conv3", 1, 1, 1), ("conv4", 1, 1, 2), ("conv5", 1, 1, 2),
+            ("fc6", 1, 0, 1), ("fc7", 1, 0, 1), ("fc8", 1, 0, 1))
+
+
+def alexnet_steps(params):
+    """AlexNet as the unfused layer sequence conv -> ReLU -> LRN -> pool (Section 4.3 slims "the first two
+    convolution layers followed by LRN layers": the slim layers are conv1 = conv + ReLU + LRN and conv2 = grouped
+    conv + ReLU + LRN).  Pooling: 3x3, stride 2, no padding (227 -> 55 -> 27 -> 13 -> 6)."""
+    def gconv(name, stride, pad, groups):
+        return lambda x: O.conv2d_grouped(x, _p(params, name + ".w"), _p(params, name + ".b"), stride, pad, groups)
+
+    cfg = {n: (s, p, g) for n, s, p, g in _ALEXNET}
+    pool = lambda x: O.maxpool(x, 3, 2, 0)[0]
+    steps = [
+        Step("conv1", ["x"], lambda x: O.lrn(O.relu(gconv("conv1", *cfg["conv1"])(x)), **_LRN)),
+        Step("pool1", ["conv1"], pool),
+        Step("conv2", ["pool1"], lambda x: O.lrn(O.relu(gconv("conv2", *cfg["conv2"])(x)), **_LRN)),
+        Step("pool2", ["conv2"], pool),
+        Step("conv3", ["pool2"], lambda x: O.relu(gconv("conv3", *cfg["conv3"])(x))),
+        Step("conv4", ["conv3"], lambda x: O.relu(gconv("conv4", *cfg["conv4"])(x))),
+        Step("conv5", ["conv4"], lambda x: O.relu(gconv("conv5", *cfg["conv5"])(x))),
+        Step("pool5", ["conv5"], pool),
+        Step("fc6", ["pool5"], lambda x: O.relu(gconv("fc6", *cfg["fc6"])(x))),
+        Step("fc7", ["fc6"], lambda x: O.relu(gconv("fc7", *cfg["fc7"])(x))),
+        Step("fc8", ["fc7"], gconv("fc8", *cfg["fc8"]), stored_bf16=False),
+    ]
+    return steps
+
+
 def run(steps, x, given=None, rounding=True):
     """Run a step list.
 

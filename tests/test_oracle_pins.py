@@ -413,3 +413,53 @@ def test_teacher_forcing_uses_given_tensors():
     forced = N.run(N.stem_steps(p), x * 0, given={"x": x})
     assert np.array_equal(free["conv1"], forced["conv1"])
     assert np.array_equal(free["conv1"], O.round_bf16(free["conv1"]))
+
+
+# ---- grouped convolution and AlexNet (Section 4.3: conv1 + norm1, conv2 + norm2 slimmed) ------------------
+def test_grouped_conv_vs_torch_and_block_diagonal_dense():
+    """Grouped convolution against the library routine, and against the dense convolution whose filters are the
+    grouped ones placed block-diagonally (zeros across groups): the identity the GPU path relies on."""
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((2, 9, 7, 12))
+    w = rng.standard_normal((10, 3, 3, 6))           # groups = 2: Cin_g = 6, Cout_g = 5
+    b = rng.standard_normal(10)
+    y = O.conv2d_grouped(x, w, b, 1, 1, 2)
+    ref = F.conv2d(nhwc_to_torch(x), w_to_torch(w), torch.from_numpy(b), stride=1, padding=1, groups=2)
+    assert np.abs(y - torch_to_nhwc(ref)).max() <= 1e-12 * float(ref.abs().max())
+    dense = np.zeros((10, 3, 3, 12))
+    dense[:5, :, :, :6] = w[:5]
+    dense[5:, :, :, 6:] = w[5:]
+    assert np.array_equal(O.conv2d(x, dense, b, 1, 1), y) or np.abs(O.conv2d(x, dense, b, 1, 1) - y).max() <= 1e-13 * np.abs(y).max()
+    # a wrong group assignment is caught: swapping the input halves changes the result
+    assert np.abs(O.conv2d_grouped(x[..., ::-1].copy(), w, b, 1, 1, 2) - y).max() > 1e-3
+    # groups = 1 is the plain convolution
+    w1 = rng.standard_normal((4, 3, 3, 12))
+    assert np.array_equal(O.conv2d_grouped(x, w1, None, 2, 0, 1), O.conv2d(x, w1, None, 2, 0))
+
+
+def test_alexnet_composition_vs_torch():
+    """Whole AlexNet (227x227, two-tower groups, LRN after conv1/conv2, unpadded 3x3/2 pools) vs PyTorch float64."""
+    p = P.alexnet_params(0)
+    assert p["conv2.w"].shape == (256, 5, 5, 48) and p["conv4.w"].shape == (384, 3, 3, 192) and p["fc6.w"].shape == (4096, 6, 6, 256)
+    x = P.images(0, 1, 227, 227)
+    steps = N.alexnet_steps(p)
+    out = N.run(steps, x, rounding=False)
+    assert [out[n].shape[1] for n in ("conv1", "pool1", "conv2", "pool2", "conv5", "pool5", "fc6")] == [55, 27, 27, 13, 13, 6, 1]
+
+    def tc(name, t, s, pad, groups=1):
+        return F.conv2d(t, w_to_torch(p[name + ".w"].astype(np.float64)), torch.from_numpy(p[name + ".b"].astype(np.float64)),
+                        stride=s, padding=pad, groups=groups)
+    lrn = lambda t: F.local_response_norm(t, 5, alpha=1e-4, beta=0.75, k=1.0)
+    pool = lambda t: F.max_pool2d(t, 3, 2, 0)
+    t = nhwc_to_torch(x.astype(np.float64))
+    t = pool(lrn(F.relu(tc("conv1", t, 4, 0))))
+    assert np.abs(out["pool1"] - torch_to_nhwc(t)).max() <= 1e-10 * float(t.abs().max())
+    t = pool(lrn(F.relu(tc("conv2", t, 1, 2, 2))))
+    assert np.abs(out["pool2"] - torch_to_nhwc(t)).max() <= 1e-10 * float(t.abs().max())
+    t = F.relu(tc("conv3", t, 1, 1))
+    t = F.relu(tc("conv4", t, 1, 1, 2))
+    t = pool(F.relu(tc("conv5", t, 1, 1, 2)))
+    t = F.relu(tc("fc6", t, 1, 0))
+    t = F.relu(tc("fc7", t, 1, 0))
+    ref = torch_to_nhwc(tc("fc8", t, 1, 0))
+    assert out["fc8"].shape == (1, 1, 1, 1000) and np.abs(out["fc8"] - ref).max() <= 1e-10 * np.abs(ref).max()
