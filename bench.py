@@ -182,7 +182,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=None, help="default 256 (GoogLeNet), 128 (ResNet-50)")
-    ap.add_argument("--arch", default="googlenet", choices=["googlenet", "resnet50", "googlenet_paper", "googlenet_streamline"],
+    ap.add_argument("--arch", default="googlenet", choices=["googlenet", "resnet50", "googlenet_paper", "googlenet_streamline", "alexnet"],
                     help="googlenet = the headline workload; resnet50 = the BN-folded bottleneck network (context)")
     ap.add_argument("--layers-out", default=None, help="write the per-layer table (us, roofline) as JSON")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -191,7 +191,7 @@ def main():
                          "this is the small case the ncu captures under profiles/ run")
     args = ap.parse_args()
     if args.batch is None:
-        args.batch = 256 if args.arch in ("googlenet", "googlenet_streamline") else 128
+        args.batch = 256 if args.arch in ("googlenet", "googlenet_streamline", "alexnet") else 128
     if args.impl == "reference":
         return run_reference(args)
     if args.layer:
@@ -229,16 +229,17 @@ def main():
     pk, pk_kind = peaks()
     resnet = args.arch != "googlenet"          # any context arm: no headline metric, no stored ncu traffic
     params = {"googlenet": P.googlenet_params, "resnet50": P.resnet50_params, "googlenet_paper": P.googlenet_paper_params,
-              "googlenet_streamline": P.googlenet_params}[args.arch](0)
+              "googlenet_streamline": P.googlenet_params, "alexnet": P.alexnet_params}[args.arch](0)
     arch_id = {"googlenet": dr.DR_ARCH_GOOGLENET, "resnet50": dr.DR_ARCH_RESNET50, "googlenet_paper": dr.DR_ARCH_GOOGLENET_PAPER,
-               "googlenet_streamline": dr.DR_ARCH_GOOGLENET_STREAMLINE}[args.arch]
+               "googlenet_streamline": dr.DR_ARCH_GOOGLENET_STREAMLINE, "alexnet": dr.DR_ARCH_ALEXNET}[args.arch]
+    hw = 227 if args.arch == "alexnet" else 224
     cfg_name = {"googlenet": "configs[3]", "resnet50": "configs[4]", "googlenet_paper": "Section 3.2 form, context",
-                "googlenet_streamline": "Section 3.1 approximate stem, context"}[args.arch]
+                "googlenet_streamline": "Section 3.1 approximate stem, context", "alexnet": "Section 4.3, conv1+norm1 and conv2+norm2 slimmed, context"}[args.arch]
     arch_name = {"googlenet": "GoogLeNet-slim", "resnet50": "ResNet-50 (BN folded)", "googlenet_paper": "GoogLeNet, paper-form branch slimming",
-                 "googlenet_streamline": "GoogLeNet-slim, stride-product stem without LRN"}[args.arch]
+                 "googlenet_streamline": "GoogLeNet-slim, stride-product stem without LRN", "alexnet": "AlexNet, LRN layers absorbed"}[args.arch]
 
     def make_net(mode, batch):
-        net = dr.Net(arch_id, mode, batch)
+        net = dr.Net(arch_id, mode, batch, hw, hw)
         keep = []
         for i in range(net.dr_net_num_params()):
             name, dims, is_f32, count = net.dr_net_param_spec(i)
@@ -252,7 +253,7 @@ def main():
 
     # synthetic N(0,1) images, bf16; per-rank seed so replicas see different data
     g = S.stream(rank, "bench.x")
-    x_host = torch.from_numpy(S.round_bf16(g.standard_normal((B, 224, 224, 3), dtype=np.float32))).to(torch.bfloat16).pin_memory()
+    x_host = torch.from_numpy(S.round_bf16(g.standard_normal((B, hw, hw, 3), dtype=np.float32))).to(torch.bfloat16).pin_memory()
     x = x_host.cuda()
     logits = torch.empty((B, 1000), dtype=torch.float32, device="cuda")
     logits_host = torch.empty((B, 1000), dtype=torch.float32).pin_memory()
@@ -431,7 +432,7 @@ def main():
         "metric": METRIC if not resnet else f"{arch_name} forward throughput", "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{arch_name} forward, batch {B} per GPU, 224x224x3 N(0,1) bf16, He-normal weights ({cfg_name})",
+        "config": {"workload": f"{arch_name} forward, batch {B} per GPU, {hw}x{hw}x3 N(0,1) bf16, He-normal weights ({cfg_name})",
                    "l2": "256 MB buffer written between timed iterations (L2 flush)", "replicas": world},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": logits_host.numel() * 4},
         "gpu_launches": int(launches),

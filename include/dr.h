@@ -91,6 +91,14 @@ int dr_fold_bn(int Cout, int K, const void* w_in, const float* b_in, const float
 int dr_embed_filter(int Cout, int Cin, int ks, int kb, const void* w_small, int joff,
                     void* w_big, void* stream);
 
+/* A grouped convolution (AlexNet's two-tower layers, Section 4.3) as the dense convolution it is a special case
+ * of: w_grouped [Cout][k][k][Cin_g] (filter j belongs to group j / (Cout/groups) and sees input channels
+ * [g*Cin_g, (g+1)*Cin_g)) is written into w_dense [Cout][k][k][Cin_g*groups] with zeros across groups.  The
+ * slim layer the paper generates for such a layer is an ordinary convolution layer; the convolution kernels
+ * never look at the zeros.  Errors: INVALID_ARG (Cout not a multiple of groups, nulls, sizes).               */
+int dr_embed_groups(int Cout, int Cin_g, int k, int groups, const void* w_grouped, void* w_dense,
+                    void* stream);
+
 /* ---- slim layers -------------------------------------------------------------------- */
 
 /* One slim convolution layer (Eq. (tY_j = tW), Section 3.1, with the epilogue of the
@@ -196,6 +204,9 @@ int dr_avgpool_global(int B, int H, int W, int C, const void* x, void* y, void* 
                                           multiplied into the convolution (7x7/4, 3x3/2), both LRN layers pruned.  Not
                                           function-preserving: the paper re-trains; here it is a timing workload with
                                           parity against its own definition.                                          */
+#define DR_ARCH_ALEXNET 4 /* AlexNet (two-tower groups, 227x227 input; Section 4.3): slim layers conv1 = conv + ReLU + LRN and
+                             conv2 = grouped conv + ReLU + LRN; the unpadded 3x3/2 pools stay layers of their own, as in
+                             the paper's Table "AlexNet Result" (conv1+norm1 -> conv1, conv2+norm2 -> conv2)            */
 #define DR_MODE_SLIM       0   /* slim layers: folded BN, fused epilogues, merged branches       */
 #define DR_MODE_UNSLIMMED  1   /* every layer of the original sequence as its own launch         */
 

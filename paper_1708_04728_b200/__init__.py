@@ -26,7 +26,7 @@ DR_OK, DR_ERR_INVALID_ARG, DR_ERR_UNSUPPORTED, DR_ERR_ALIGNMENT = 0, -1, -2, -3
 DR_ERR_WORKSPACE, DR_ERR_CUDA, DR_ERR_DEVICE_TIMEOUT = -4, -5, -6
 DR_BIAS, DR_RELU, DR_POOL, DR_LRN, DR_RESIDUAL = 0x01, 0x02, 0x04, 0x08, 0x10
 DR_LRN_BEFORE_POOL, DR_RELU_AFTER_RESIDUAL, DR_OUT_F32 = 0x20, 0x40, 0x80
-DR_ARCH_GOOGLENET, DR_ARCH_RESNET50, DR_ARCH_GOOGLENET_PAPER, DR_ARCH_GOOGLENET_STREAMLINE = 0, 1, 2, 3
+DR_ARCH_GOOGLENET, DR_ARCH_RESNET50, DR_ARCH_GOOGLENET_PAPER, DR_ARCH_GOOGLENET_STREAMLINE, DR_ARCH_ALEXNET = 0, 1, 2, 3, 4
 DR_MODE_SLIM, DR_MODE_UNSLIMMED = 0, 1
 DR_PATH_AUTO, DR_PATH_SIMT, DR_PATH_UMMA_GATHER, DR_PATH_UMMA_TMA, DR_PATH_UMMA_PATCH, DR_PATH_UMMA_STEM, DR_PATH_UMMA_STEM_T, DR_PATH_UMMA_STEM_D = 0, 1, 2, 3, 4, 5, 6, 7
 DR_PATH_UMMA_SPLITK = 8
@@ -67,6 +67,7 @@ _SIGS = {
     "dr_strerror": (C.c_char_p, [_I]),
     "dr_fold_bn": (_I, [_I, _I, _P, _P, _P, _P, _F, _F, _P, _P, _P, _P, _P]),
     "dr_embed_filter": (_I, [_I, _I, _I, _I, _P, _I, _P, _P]),
+    "dr_embed_groups": (_I, [_I, _I, _I, _I, _P, _P, _P]),
     "dr_conv_slim": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P]),
     "dr_conv_workspace_bytes": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, C.POINTER(_Z)]),
     "dr_conv_slim_ws": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _Z, _P]),
@@ -140,6 +141,10 @@ def dr_fold_bn(Cout, K, w_in, b_in, mean, var, m, eps, gamma, beta, w_out, b_out
 
 def dr_embed_filter(Cout, Cin, ks, kb, w_small, joff, w_big, stream=None):
     _check(_lib.dr_embed_filter(Cout, Cin, ks, kb, _ptr(w_small), joff, _ptr(w_big), _stream(stream)), "dr_embed_filter")
+
+
+def dr_embed_groups(Cout, Cin_g, k, groups, w_grouped, w_dense, stream=None):
+    _check(_lib.dr_embed_groups(Cout, Cin_g, k, groups, _ptr(w_grouped), _ptr(w_dense), _stream(stream)), "dr_embed_groups")
 
 
 def dr_conv_slim(desc, B, H, W, x, w, b, residual, y, argmax=None, stream=None):

@@ -127,6 +127,62 @@ __device__ __forceinline__ void drain_fast(const ConvParams& p, uint32_t taddr, 
     }
 }
 
+// Epilogue of a layer that ends in LRN across channels without pooling (bias, ReLU, LRN, bf16 store): the thread owns
+// every channel of its output pixel (one tile spans all of Cout <= 256), so the LRN window is a sliding sum over the
+// accumulator row, read from TMEM in chunks of W columns with two columns of look-back (kept in registers) and two
+// of look-ahead (a two-column TMEM load).  Windows of 1, 3 or 5 channels (half <= 2); beyond the row: zeros.
+template <int W>
+__device__ __forceinline__ void lrn_chunk(const ConvParams& p, uint32_t taddr, int c, int ncols, bool row_ok, const float* bias_s,
+                                          float& pm2, float& pm1, __nv_bfloat16* yrow) {
+    uint32_t r[W], nx[2] = {0u, 0u};
+    if (W == 32) tmem_ld_x32(taddr + c, r); else tmem_ld_x16(taddr + c, r);
+    const bool more = c + W < ncols;
+    if (more) tmem_ld_x2(taddr + c + W, nx);
+    tmem_ld_wait();
+    const bool relu = p.flags & DR_RELU;
+    float x[W + 4];
+    x[0] = pm2; x[1] = pm1;
+#pragma unroll
+    for (int j = 0; j < W; ++j) {
+        float v = __uint_as_float(r[j]) + bias_s[c + j];
+        x[2 + j] = relu ? fmaxf(v, 0.f) : v;
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        float v = more ? __uint_as_float(nx[j]) + bias_s[c + W + j] : 0.f;
+        x[2 + W + j] = (relu && more) ? fmaxf(v, 0.f) : v;
+    }
+    pm2 = x[W]; pm1 = x[W + 1];
+    const bool h1 = p.lrn_half >= 1, h2 = p.lrn_half >= 2;
+    uint32_t o[W / 2];
+#pragma unroll
+    for (int j = 0; j < W; j += 2) {
+        float y2[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int i = 2 + j + e;
+            float ss = x[i] * x[i];
+            if (h1) ss += x[i - 1] * x[i - 1] + x[i + 1] * x[i + 1];
+            if (h2) ss += x[i - 2] * x[i - 2] + x[i + 2] * x[i + 2];
+            y2[e] = x[i] * lrn_pow(p.lrn_k + p.lrn_alpha_n * ss, p.lrn_beta);
+        }
+        o[j >> 1] = pack_bf16(y2[0], y2[1]);
+    }
+    if (row_ok) {
+        uint4* y = reinterpret_cast<uint4*>(yrow + c);
+#pragma unroll
+        for (int q = 0; q < W / 8; ++q) y[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+    }
+}
+
+__device__ __forceinline__ void drain_lrn(const ConvParams& p, uint32_t taddr, int ncols, long long m, bool row_ok, const float* bias_s) {
+    __nv_bfloat16* yrow = reinterpret_cast<__nv_bfloat16*>(p.y) + m * p.ldc + p.coff;
+    float pm2 = 0.f, pm1 = 0.f;
+    int c = 0;
+    for (; c + 32 <= ncols; c += 32) lrn_chunk<32>(p, taddr, c, ncols, row_ok, bias_s, pm2, pm1, yrow);
+    if (c < ncols) lrn_chunk<16>(p, taddr, c, ncols, row_ok, bias_s, pm2, pm1, yrow);
+}
+
 // =====================================================================================
 //                                   gather kernel
 // =====================================================================================
@@ -397,6 +453,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
     // (ReLU before a residual add is the one order it does not take.)
     const bool lean = !(p.flags & DR_OUT_F32) && !((p.flags & DR_RESIDUAL) && (p.flags & DR_RELU)) && (p.Cout & 15) == 0 &&
                       p.Cout <= T_BIAS_MAX && (p.ldc & 7) == 0 && (p.coff & 7) == 0;
+    const bool lrn_ep = (p.flags & DR_LRN) != 0;                // host side guarantees: no pooling, one n-block, lean preconditions
     const int lean_mode = (p.flags & DR_RESIDUAL) ? ((p.flags & DR_RELU_AFTER_RESIDUAL) ? 3 : 2) : ((p.flags & DR_RELU) ? 1 : 0);
     if (lean)
         for (int i = tid; i < p.Cout; i += T_THREADS) bias_s[i] = (p.flags & DR_BIAS) ? p.bias[i] : 0.f;
@@ -590,6 +647,8 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             const bool row_ok = mt < p.m_tiles && m < p.M;
             if (WIDE && Nj <= 0) {
                 // nothing to drain
+            } else if (lrn_ep) {
+                drain_lrn(p, taddr, Nj, m, row_ok, bias_s);
             } else if (lean) {
                 if (lean_mode == 1) drain_fast<1>(p, taddr, Nj, m, row_ok, n0, bias_s);
                 else if (lean_mode == 3) drain_fast<3>(p, taddr, Nj, m, row_ok, n0, bias_s);
@@ -686,7 +745,12 @@ int tunable(const char* name, int dflt) {
 }
 
 bool conv_umma_tma_supports(const ConvParams& p) {
-    if (p.flags & (DR_POOL | DR_LRN)) return false;   // staged epilogues live in the gather kernel
+    if (p.flags & DR_POOL) return false;              // pooling epilogues live in the patch / stem / gather kernels
+    if (p.flags & DR_LRN) {
+        // LRN without pooling: the in-register sliding window of drain_lrn, one tile across all output channels
+        if (p.flags & (DR_RESIDUAL | DR_OUT_F32)) return false;
+        if (p.n_blocks != 1 || (p.Cout & 15) || p.Cout > 256 || p.lrn_half > 2 || (p.ldc & 7) || (p.coff & 7) || p.argmax) return false;
+    }
     if (p.patch) return false;
     if ((p.Cin & 7) || p.Cin < 64) return false;      // TMA strides are 16-byte multiples; 128-byte rows
     if (p.Nt > 256) return false;
@@ -775,6 +839,7 @@ int conv_umma_tma_launch(const ConvParams& p_in, cudaStream_t stream) {
         const long long cost_w = (m_units * n_wide + capacity - 1) / capacity * 2 * nt_w;
         const int nkb_ = p.k * p.k * ((p.Cin + 63) / 64);
         wide = wide_pref >= 0 ? wide_pref != 0 : (cout16_ > 256 && nkb_ >= 48 && cost_w * 95 <= cost_n * 100);
+        if (p.flags & DR_LRN) wide = false;                      // the LRN window runs along one accumulator row
     }
     if (wide) {
         p.Nt = nt_w;

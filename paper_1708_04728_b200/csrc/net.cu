@@ -55,6 +55,7 @@ struct Op {
     int conv_index = -1;     // OP_CONV: ordinal among the convolutions (its block of split-K counters)
     int pair = -1;           // OP_CONV: a later convolution reading the same input that may share this one's launch,
     int chain = -1;          //          and the convolution that reads this one's output (it may join them)
+    int pool_pad = 1;        // OP_MAXPOOL: 3x3 / 2 with this padding
     int group = 0;           // decided by dr_net_prepare: 0 own launch, 2 with `pair`, 3 with `pair` and `chain`
 };
 
@@ -62,6 +63,7 @@ struct Op {
 struct FoldJob { int w, mean, var, gamma, beta; size_t w_off, b_off; int Cout, K; };
 struct EmbedJob { int w_small; int Cout, Cin, ks, kb, joff; size_t w_off; };
 struct CopyJob { int src; size_t dst_off; size_t bytes; };
+struct GroupJob { int w_grouped; int Cout, Cin_g, k, groups; size_t w_off; };
 
 }  // namespace dr
 
@@ -76,6 +78,7 @@ struct dr_net {
     std::vector<FoldJob> folds;
     std::vector<EmbedJob> embeds;
     std::vector<CopyJob> copies;
+    std::vector<GroupJob> group_jobs;
     size_t param_bytes = 0, act_bytes = 0;
     size_t sk_scratch_bytes = 0;   // split-K scratch shared by all layers (they run one after another), after the arena
     int n_conv = 0;                // each convolution has its own block of tile counters after that
@@ -143,12 +146,12 @@ static int add_conv(dr_net* n, const std::string& name, int in, int k, int s, in
     return out;
 }
 
-static int add_simple(dr_net* n, OpKind kind, const std::string& name, int in0, int in1 = -2) {
+static int add_simple(dr_net* n, OpKind kind, const std::string& name, int in0, int in1 = -2, int pool_pad = 1) {
     const Tensor ti = n->T(in0);
     Op op;
-    op.kind = kind; op.name = name; op.in0 = in0; op.in1 = in1;
+    op.kind = kind; op.name = name; op.in0 = in0; op.in1 = in1; op.pool_pad = pool_pad;
     int H = ti.H, W = ti.W;
-    if (kind == OP_MAXPOOL) { H = out_size(H, 3, 2, 1); W = out_size(W, 3, 2, 1); }
+    if (kind == OP_MAXPOOL) { H = out_size(H, 3, 2, pool_pad); W = out_size(W, 3, 2, pool_pad); }
     if (kind == OP_AVGPOOL) { H = 1; W = 1; }
     op.out = n->tensor(ti.B, H, W, ti.C);
     op.bytes = (double)ti.bytes * (kind == OP_ADD ? 2 : 1) + (double)n->T(op.out).bytes;
@@ -399,6 +402,50 @@ static void set_splitk_scratch(const dr_net* n, const Op& op, char* ws, ConvPara
     p->sk_counters = reinterpret_cast<int*>(base + (n->sk_scratch_bytes + 255) / 256 * 256 + (size_t)op.conv_index * DR_CONV_WS_COUNTER_BYTES);
 }
 
+// AlexNet (two-tower form, 227x227 input).  Slim layers (Section 4.3): conv1 = conv + ReLU + LRN, conv2 = grouped
+// conv + ReLU + LRN; the unpadded 3x3/2 pools stay separate, as in the paper's table.  Grouped layers run as dense
+// convolutions over block-diagonal filters (dr_embed_groups) in both modes; fc6 is a 6x6 convolution over the 6x6
+// plane pool5 leaves.  Dropout is the identity at inference.
+static void build_alexnet(dr_net* n) {
+    const bool slim = n->mode == DR_MODE_SLIM;
+    const int x = n->tensor(n->B, n->H, n->W, 3, 0, true);
+    n->t_input = x;
+    struct L { const char* name; int cout, k, s, p, groups; bool lrn, pool, relu; };
+    static const L layers[8] = {{"conv1", 96, 11, 4, 0, 1, true, true, true},   {"conv2", 256, 5, 1, 2, 2, true, true, true},
+                                {"conv3", 384, 3, 1, 1, 1, false, false, true}, {"conv4", 384, 3, 1, 1, 2, false, false, true},
+                                {"conv5", 256, 3, 1, 1, 2, false, true, true},  {"fc6", 4096, 6, 1, 0, 1, false, false, true},
+                                {"fc7", 4096, 1, 1, 0, 1, false, false, true},  {"fc8", 1000, 1, 1, 0, 1, false, false, false}};
+    int t = x;
+    for (int i = 0; i < 8; ++i) {
+        const L& l = layers[i];
+        const std::string name = l.name;
+        const int cin = n->T(t).C;
+        const int wi = n->param(name + ".w", l.cout, l.k, l.k, cin / l.groups, 0);
+        const int bi = n->vec(name + ".b", l.cout);
+        PRef w = rawref(wi);
+        if (l.groups > 1) {
+            const size_t wo = n->ws_alloc((size_t)l.cout * l.k * l.k * cin * 2);
+            n->group_jobs.push_back({wi, l.cout, cin / l.groups, l.k, l.groups, wo});
+            w = wsref(wo);
+        }
+        const bool last = i == 7;
+        const char* pool_name = i == 0 ? "pool1" : i == 1 ? "pool2" : "pool5";
+        if (slim) {
+            unsigned f = DR_BIAS | (l.relu ? DR_RELU : 0) | (l.lrn ? DR_LRN : 0) | (last ? DR_OUT_F32 : 0);
+            t = add_conv(n, name, t, l.k, l.s, l.p, l.cout, f, w, rawref(bi));
+            n->ops.back().flops /= l.groups;        // algorithmic work of the grouped layer, not of its dense stand-in
+        } else {
+            const bool plain = !l.relu && !l.lrn;
+            t = add_conv(n, plain ? name : name + ".conv", t, l.k, l.s, l.p, l.cout, DR_BIAS | (last ? DR_OUT_F32 : 0), w, rawref(bi));
+            n->ops.back().flops /= l.groups;
+            if (l.relu) t = add_simple(n, OP_RELU, l.lrn ? name + ".relu" : name, t);
+            if (l.lrn) t = add_simple(n, OP_LRN, name, t);
+        }
+        if (l.pool) t = add_simple(n, OP_MAXPOOL, pool_name, t, -2, 0);
+        if (last) n->t_logits = t;
+    }
+}
+
 static const char* tensor_ptr(const dr_net* n, int id, const void* x, const char* arena, const float* logits) {
     if (id == n->t_input) return (const char*)x;
     if (id == n->t_logits) return (const char*)logits;
@@ -411,7 +458,8 @@ extern "C" {
 
 int dr_net_create(dr_net** net, int arch, int mode, int B, int H, int W) {
     if (!net || B <= 0 || H <= 0 || W <= 0) return DR_ERR_INVALID_ARG;
-    if (arch < DR_ARCH_GOOGLENET || arch > DR_ARCH_GOOGLENET_STREAMLINE) return DR_ERR_INVALID_ARG;
+    if (arch < DR_ARCH_GOOGLENET || arch > DR_ARCH_ALEXNET) return DR_ERR_INVALID_ARG;
+    if (arch == DR_ARCH_ALEXNET && (H != 227 || W != 227)) return DR_ERR_INVALID_ARG;   // fc6 is a 6x6 convolution over pool5's 6x6 plane
     if (mode != DR_MODE_SLIM && mode != DR_MODE_UNSLIMMED) return DR_ERR_INVALID_ARG;
     // five halvings (stem conv, four pools / strided stages) must leave at least one pixel
     if (H < 32 || W < 32) return DR_ERR_INVALID_ARG;
@@ -419,6 +467,7 @@ int dr_net_create(dr_net** net, int arch, int mode, int B, int H, int W) {
     n->arch = arch; n->mode = mode; n->B = B; n->H = H; n->W = W;
     if (arch == DR_ARCH_GOOGLENET || arch == DR_ARCH_GOOGLENET_STREAMLINE) build_googlenet(n);
     else if (arch == DR_ARCH_GOOGLENET_PAPER) build_googlenet_paper(n);
+    else if (arch == DR_ARCH_ALEXNET) build_alexnet(n);
     else build_resnet50(n);
     // scratch the split-K kernel wants for the layers with few output tiles (slim mode only: the unslimmed
     // baseline keeps one plain launch per layer)
@@ -497,6 +546,10 @@ int dr_net_prepare(dr_net* n, void* workspace, void* stream) {
     }
     for (const EmbedJob& e : n->embeds) {
         const int st = dr_embed_filter(e.Cout, e.Cin, e.ks, e.kb, n->raw[e.w_small], e.joff, ws + e.w_off, stream);
+        if (st != DR_OK) return st;
+    }
+    for (const GroupJob& g : n->group_jobs) {
+        const int st = dr_embed_groups(g.Cout, g.Cin_g, g.k, g.groups, n->raw[g.w_grouped], ws + g.w_off, stream);
         if (st != DR_OK) return st;
     }
     for (const CopyJob& c : n->copies)
@@ -595,7 +648,7 @@ int dr_net_forward(dr_net* n, const void* x, void* workspace, float* logits, voi
                 break;
             }
             case OP_RELU: st = dr_relu((size_t)ti.B * ti.H * ti.W * ti.C, in0, out, stream); break;
-            case OP_MAXPOOL: st = dr_maxpool(ti.B, ti.H, ti.W, ti.C, 3, 2, 1, in0, out, nullptr, stream); break;
+            case OP_MAXPOOL: st = dr_maxpool(ti.B, ti.H, ti.W, ti.C, 3, 2, op.pool_pad, in0, out, nullptr, stream); break;
             case OP_LRN: st = dr_lrn(ti.B, ti.H, ti.W, ti.C, 5, 1e-4f, 0.75f, 1.f, in0, out, stream); break;
             case OP_BN:
                 st = dr_bn(ti.B, ti.H, ti.W, ti.C, in0, (const float*)op.v0.resolve(n->raw, ws), (const float*)op.v1.resolve(n->raw, ws),

@@ -347,6 +347,21 @@ __global__ void embed_filter_kernel(int Cin, int ks, int kb, const __nv_bfloat16
     }
 }
 
+// ---------------------------------------------------------------- grouped filters as block-diagonal dense filters
+// w_grouped [Cout][k][k][Cin_g] -> w_dense [Cout][k][k][Cin_g * groups]: filter j keeps its values at the input
+// channels of its own group (j / (Cout / groups)) and is zero elsewhere.
+__global__ void embed_groups_kernel(int Cout, int Cin_g, int kk, int groups, const __nv_bfloat16* __restrict__ w_grouped,
+                                    __nv_bfloat16* __restrict__ w_dense) {
+    const int j = blockIdx.x, g = j / (Cout / groups);
+    const int Cin = Cin_g * groups, per = kk * Cin;
+    for (int i = threadIdx.x; i < per; i += blockDim.x) {
+        const int c = i % Cin, t = i / Cin, cg = c - g * Cin_g;
+        __nv_bfloat16 v = __float2bfloat16_rn(0.f);
+        if (cg >= 0 && cg < Cin_g) v = w_grouped[((size_t)j * kk + t) * Cin_g + cg];
+        w_dense[(size_t)j * per + i] = v;
+    }
+}
+
 }  // namespace dr
 
 // ================================================================ C ABI
@@ -499,6 +514,14 @@ int dr_embed_filter(int Cout, int Cin, int ks, int kb, const void* w_small, int 
     DR_REQUIRE(w_small && w_big, DR_ERR_INVALID_ARG);
     DR_REQUIRE(Cout > 0 && Cin > 0 && ks > 0 && kb >= ks && (ks & 1) && (kb & 1) && joff >= 0, DR_ERR_INVALID_ARG);
     embed_filter_kernel<<<Cout, 256, 0, (cudaStream_t)stream>>>(Cin, ks, kb, (const __nv_bfloat16*)w_small, joff, (__nv_bfloat16*)w_big);
+    count_launch();
+    return launch_status();
+}
+
+int dr_embed_groups(int Cout, int Cin_g, int k, int groups, const void* w_grouped, void* w_dense, void* stream) {
+    DR_REQUIRE(w_grouped && w_dense, DR_ERR_INVALID_ARG);
+    DR_REQUIRE(Cout > 0 && Cin_g > 0 && k > 0 && groups > 0 && Cout % groups == 0, DR_ERR_INVALID_ARG);
+    embed_groups_kernel<<<Cout, 256, 0, (cudaStream_t)stream>>>(Cout, Cin_g, k * k, groups, (const __nv_bfloat16*)w_grouped, (__nv_bfloat16*)w_dense);
     count_launch();
     return launch_status();
 }

@@ -174,6 +174,9 @@ STAGED = [
     (2, 20, 18, 64, 192, 3, 1, 1, "lrn_pool"),      # conv2 geometry: ReLU -> LRN -> pool
     (2, 13, 9, 32, 48, 3, 1, 1, "pool"),
     (1, 9, 12, 16, 32, 1, 1, 0, "lrn"),
+    (2, 13, 11, 64, 96, 3, 1, 1, "lrn"),            # LRN without pooling on the TMA kernel: 3 chunks of 32 channels
+    (1, 27, 27, 96, 256, 5, 1, 2, "lrn"),           # AlexNet conv2 as a dense layer: 256 channels, 32-channel K tail
+    (3, 6, 5, 128, 48, 1, 1, 0, "lrn"),             # 16-channel tail chunk
     (1, 5, 5, 8, 16, 3, 1, 1, "pool"),              # plane smaller than one patch
     (3, 56, 56, 64, 192, 3, 1, 1, "lrn_pool"),      # GoogLeNet conv2 at its real plane size
     (2, 30, 26, 128, 64, 3, 1, 1, "pool"),          # two channel blocks per tap

@@ -61,10 +61,10 @@ def layer_outputs(net, logits, entries):
     return out
 
 
-def check_network(dr, arch, B, entries, steps_fn, params, per_layer_tol=None):
+def check_network(dr, arch, B, entries, steps_fn, params, per_layer_tol=None, hw=224, out="fc"):
     import oracle.nets as N
-    images = lambda rng: np.stack([S.normal(0, f"x[{n}]", (224, 224, 3)) for n in rng])
-    net, ws, logits, keep = run_net(dr, arch, dr.DR_MODE_SLIM, B, params, images)
+    images = lambda rng: np.stack([S.normal(0, f"x[{n}]", (hw, hw, 3)) for n in rng])
+    net, ws, logits, keep = run_net(dr, arch, dr.DR_MODE_SLIM, B, params, images, hw=hw)
     paths = {net.dr_net_layer_info(i)["name"]: net.dr_net_layer_info(i)["conv_path"] for i in range(net.dr_net_num_layers())}
     steps = steps_fn(params)
     # ---- per layer, teacher-forced, batch entry 0 (+ all checked entries for the logits)
@@ -88,13 +88,13 @@ def check_network(dr, arch, B, entries, steps_fn, params, per_layer_tol=None):
     got = to_host(logits[list(entries)]).reshape(len(entries), 1, 1, 1000)
     assert np.all(np.isfinite(got))
     for i in range(len(entries)):
-        mx, l2 = err_norms(got[i], free["fc"][i])
+        mx, l2 = err_norms(got[i], free[out][i])
         assert l2 <= LOGITS_L2, f"logits of batch entry {entries[i]}: rel-L2 {l2:.3e} > {LOGITS_L2}"
     # every batch entry produced something finite
     assert bool(np.isfinite(to_host(logits)).all())
     worst = max(report, key=lambda r: r[3])
-    print(f"\n[{['googlenet','resnet50','googlenet-paper','googlenet-streamline'][arch]} B={B}] worst layer {worst[0]} path={worst[1]} max {worst[2]:.2e} l2 {worst[3]:.2e}; "
-          f"logits rel-L2 {max(err_norms(got[i], free['fc'][i])[1] for i in range(len(entries))):.2e}")
+    print(f"\n[{['googlenet','resnet50','googlenet-paper','googlenet-streamline','alexnet'][arch]} B={B}] worst layer {worst[0]} path={worst[1]} max {worst[2]:.2e} l2 {worst[3]:.2e}; "
+          f"logits rel-L2 {max(err_norms(got[i], free[out][i])[1] for i in range(len(entries))):.2e}")
     return net, logits, free, keep
 
 
@@ -125,6 +125,20 @@ def test_googlenet_streamline_form(dr, B, k):
     import oracle.nets as N
     params = P.googlenet_params(0)
     check_network(dr, dr.DR_ARCH_GOOGLENET_STREAMLINE, B, subset(B, k), N.googlenet_streamline_steps, params)
+
+
+@pytest.mark.parametrize("B,k", [(1, 1), (32, 2)])
+def test_alexnet_slim(dr, B, k):
+    """AlexNet with conv1 + norm1 and conv2 + norm2 as slim layers (Section 4.3), grouped layers as block-diagonal
+    dense convolutions: per-layer and logits parity with the grouped, unfused checker."""
+    import oracle.nets as N
+    params = P.alexnet_params(0)
+    net, logits, free, keep = check_network(dr, dr.DR_ARCH_ALEXNET, B, subset(B, k), N.alexnet_steps, params, hw=227, out="fc8")
+    names = [net.dr_net_layer_info(i)["name"] for i in range(net.dr_net_num_layers())]
+    assert names == ["conv1", "pool1", "conv2", "pool2", "conv3", "conv4", "conv5", "pool5", "fc6", "fc7", "fc8"]
+    # the baseline runs ReLU and LRN as layers of their own
+    uns = dr.Net(dr.DR_ARCH_ALEXNET, dr.DR_MODE_UNSLIMMED, B, 227, 227)
+    assert uns.dr_net_num_layers() == 11 + 7 + 2
 
 
 @pytest.mark.parametrize("B,k", [(128, 2)])
