@@ -99,6 +99,19 @@ int dr_embed_filter(int Cout, int Cin, int ks, int kb, const void* w_small, int 
 int dr_embed_groups(int Cout, int Cin_g, int k, int groups, const void* w_grouped, void* w_dense,
                     void* stream);
 
+/* A strided convolution over few input channels (AlexNet's 11x11/4 and the stride-product 7x7/4 stem of Section 3.1
+ * on 3-channel images) as a stride-1 convolution over a space-to-depth copy of the input: with kp = ceil(k/s),
+ *   y[n][R][S][(ah*s + aw)*C + c] = x[n][R*s + ah - pad][S*s + aw - pad][c]        (zero outside the image),
+ *   w_out[j][R][S][(ah*s + aw)*C + c] = w[j][R*s + ah][S*s + aw][c]                 (zero for taps >= k),
+ * the kp x kp / stride 1 / pad 0 convolution of y with w_out equals the k x k / stride s / pad `pad` convolution
+ * of x with w, exactly.  y has Ho + kp - 1 rows and Wo + kp - 1 columns (Ho, Wo the convolution's output extent)
+ * and Cp >= s*s*C channels (a multiple of 8; the extra ones are zero), so the tensor-core kernels can load it.
+ * dr_space_to_depth runs per forward pass (one read of x, one write of y); dr_s2d_filter once per filter bank.
+ * Errors: INVALID_ARG, ALIGNMENT.                                                                            */
+int dr_space_to_depth(int B, int H, int W, int C, int k, int s, int pad, int Cp, const void* x, void* y,
+                      void* stream);
+int dr_s2d_filter(int Cout, int k, int C, int s, int Cp, const void* w, void* w_out, void* stream);
+
 /* ---- slim layers -------------------------------------------------------------------- */
 
 /* One slim convolution layer (Eq. (tY_j = tW), Section 3.1, with the epilogue of the

@@ -68,6 +68,8 @@ _SIGS = {
     "dr_fold_bn": (_I, [_I, _I, _P, _P, _P, _P, _F, _F, _P, _P, _P, _P, _P]),
     "dr_embed_filter": (_I, [_I, _I, _I, _I, _P, _I, _P, _P]),
     "dr_embed_groups": (_I, [_I, _I, _I, _I, _P, _P, _P]),
+    "dr_space_to_depth": (_I, [_I, _I, _I, _I, _I, _I, _I, _I, _P, _P, _P]),
+    "dr_s2d_filter": (_I, [_I, _I, _I, _I, _I, _P, _P, _P]),
     "dr_conv_slim": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P]),
     "dr_conv_workspace_bytes": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, C.POINTER(_Z)]),
     "dr_conv_slim_ws": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _Z, _P]),
@@ -145,6 +147,14 @@ def dr_embed_filter(Cout, Cin, ks, kb, w_small, joff, w_big, stream=None):
 
 def dr_embed_groups(Cout, Cin_g, k, groups, w_grouped, w_dense, stream=None):
     _check(_lib.dr_embed_groups(Cout, Cin_g, k, groups, _ptr(w_grouped), _ptr(w_dense), _stream(stream)), "dr_embed_groups")
+
+
+def dr_space_to_depth(B, H, W, Cc, k, s, pad, Cp, x, y, stream=None):
+    _check(_lib.dr_space_to_depth(B, H, W, Cc, k, s, pad, Cp, _ptr(x), _ptr(y), _stream(stream)), "dr_space_to_depth")
+
+
+def dr_s2d_filter(Cout, k, Cc, s, Cp, w, w_out, stream=None):
+    _check(_lib.dr_s2d_filter(Cout, k, Cc, s, Cp, _ptr(w), _ptr(w_out), _stream(stream)), "dr_s2d_filter")
 
 
 def dr_conv_slim(desc, B, H, W, x, w, b, residual, y, argmax=None, stream=None):

@@ -154,17 +154,34 @@ __device__ __forceinline__ void lrn_chunk(const ConvParams& p, uint32_t taddr, i
     }
     pm2 = x[W]; pm1 = x[W + 1];
     const bool h1 = p.lrn_half >= 1, h2 = p.lrn_half >= 2;
+    // scale^(-beta), scale = k (1 + u), u = (alpha/n) ss / k.  While u < 1/32 for the whole chunk of the warp (always so
+    // for the usual alpha = 1e-4) the binomial series of (1 + u)^(-beta) to u^4 is exact to float32 resolution and
+    // needs no special-function unit; otherwise exp2/log2.
+    float sq[W + 4], u[W];
+#pragma unroll
+    for (int j = 0; j < W + 4; ++j) sq[j] = x[j] * x[j];
+    const float au = p.lrn_alpha_n * p.lrn_inv_k;
+    float umax = 0.f;
+#pragma unroll
+    for (int j = 0; j < W; ++j) {
+        float ss = sq[2 + j];
+        if (h1) ss += sq[1 + j] + sq[3 + j];
+        if (h2) ss += sq[j] + sq[4 + j];
+        u[j] = au * ss;
+        umax = fmaxf(umax, u[j]);
+    }
+    const bool series = !__any_sync(0xffffffffu, !(umax < 0.03125f));
     uint32_t o[W / 2];
 #pragma unroll
     for (int j = 0; j < W; j += 2) {
         float y2[2];
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-            const int i = 2 + j + e;
-            float ss = x[i] * x[i];
-            if (h1) ss += x[i - 1] * x[i - 1] + x[i + 1] * x[i + 1];
-            if (h2) ss += x[i - 2] * x[i - 2] + x[i + 2] * x[i + 2];
-            y2[e] = x[i] * lrn_pow(p.lrn_k + p.lrn_alpha_n * ss, p.lrn_beta);
+            const float uu = u[j + e];
+            float f;
+            if (series) f = p.lrn_kpow * fmaf(uu, fmaf(uu, fmaf(uu, fmaf(uu, p.lrn_c4, p.lrn_c3), p.lrn_c2), p.lrn_c1), 1.f);
+            else f = p.lrn_kpow * exp2f(-p.lrn_beta * log2f(1.f + uu));
+            y2[e] = x[2 + j + e] * f;
         }
         o[j >> 1] = pack_bf16(y2[0], y2[1]);
     }
@@ -749,7 +766,7 @@ bool conv_umma_tma_supports(const ConvParams& p) {
     if (p.flags & DR_LRN) {
         // LRN without pooling: the in-register sliding window of drain_lrn, one tile across all output channels
         if (p.flags & (DR_RESIDUAL | DR_OUT_F32)) return false;
-        if (p.n_blocks != 1 || (p.Cout & 15) || p.Cout > 256 || p.lrn_half > 2 || (p.ldc & 7) || (p.coff & 7) || p.argmax) return false;
+        if (p.n_blocks != 1 || (p.Cout & 15) || p.Cout > 256 || p.lrn_half > 2 || !(p.lrn_k > 0.f) || p.lrn_alpha_n < 0.f || (p.ldc & 7) || (p.coff & 7) || p.argmax) return false;
     }
     if (p.patch) return false;
     if ((p.Cin & 7) || p.Cin < 64) return false;      // TMA strides are 16-byte multiples; 128-byte rows

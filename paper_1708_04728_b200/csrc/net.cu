@@ -20,7 +20,7 @@ int conv_pick_path(const ConvParams& p, int forced);
 int conv_launch_path(const ConvParams& p, int path, cudaStream_t stream);
 int forced_conv_path();
 
-enum OpKind { OP_CONV, OP_RELU, OP_MAXPOOL, OP_LRN, OP_BN, OP_SCALE, OP_ADD, OP_CONCAT, OP_AVGPOOL };
+enum OpKind { OP_CONV, OP_RELU, OP_MAXPOOL, OP_LRN, OP_BN, OP_SCALE, OP_ADD, OP_CONCAT, OP_AVGPOOL, OP_S2D };
 
 struct Tensor {
     int B, H, W, C;
@@ -56,6 +56,7 @@ struct Op {
     int pair = -1;           // OP_CONV: a later convolution reading the same input that may share this one's launch,
     int chain = -1;          //          and the convolution that reads this one's output (it may join them)
     int pool_pad = 1;        // OP_MAXPOOL: 3x3 / 2 with this padding
+    int s2d_k = 0, s2d_s = 0, s2d_pad = 0;   // OP_S2D: the convolution whose input this op re-lays
     int group = 0;           // decided by dr_net_prepare: 0 own launch, 2 with `pair`, 3 with `pair` and `chain`
 };
 
@@ -63,6 +64,7 @@ struct Op {
 struct FoldJob { int w, mean, var, gamma, beta; size_t w_off, b_off; int Cout, K; };
 struct EmbedJob { int w_small; int Cout, Cin, ks, kb, joff; size_t w_off; };
 struct CopyJob { int src; size_t dst_off; size_t bytes; };
+struct S2dJob { int w; int Cout, k, C, s, Cp; size_t w_off; };
 struct GroupJob { int w_grouped; int Cout, Cin_g, k, groups; size_t w_off; };
 
 }  // namespace dr
@@ -79,6 +81,7 @@ struct dr_net {
     std::vector<EmbedJob> embeds;
     std::vector<CopyJob> copies;
     std::vector<GroupJob> group_jobs;
+    std::vector<S2dJob> s2d_jobs;
     size_t param_bytes = 0, act_bytes = 0;
     size_t sk_scratch_bytes = 0;   // split-K scratch shared by all layers (they run one after another), after the arena
     int n_conv = 0;                // each convolution has its own block of tile counters after that
@@ -165,6 +168,31 @@ static int add_norm(dr_net* n, OpKind kind, const std::string& name, int in, int
     return out;
 }
 
+static PRef rawref(int idx) { PRef r; r.raw = idx; return r; }
+static PRef wsref(size_t off) { PRef r; r.ws_off = off; return r; }
+
+// A k x k / stride s convolution over a few-channel image (s >= 2, s*s*C <= 64) as a space-to-depth copy of the
+// image (a non-tensor layer of its own: one more pass over the input) followed by a ceil(k/s)^2 / stride 1
+// convolution over 64 channels with re-laid filters: the form the TMA tensor-core kernel takes.
+static int add_conv_s2d(dr_net* n, const std::string& name, int in, int k, int s, int p, int cout, unsigned flags, int wi, PRef b) {
+    const Tensor ti = n->T(in);
+    const int kp = (k + s - 1) / s, Cp = 64;
+    const int Ho = out_size(ti.H, k, s, p), Wo = out_size(ti.W, k, s, p);
+    Op op;
+    op.kind = OP_S2D; op.name = name + ".s2d"; op.in0 = in;
+    op.s2d_k = k; op.s2d_s = s; op.s2d_pad = p;
+    op.out = n->tensor(ti.B, Ho + kp - 1, Wo + kp - 1, Cp);
+    op.bytes = (double)ti.bytes + (double)n->T(op.out).bytes;
+    n->ops.push_back(op);
+    const size_t wo = n->ws_alloc((size_t)cout * kp * kp * Cp * 2);
+    n->s2d_jobs.push_back({wi, cout, k, ti.C, s, Cp, wo});
+    const int out = add_conv(n, name, op.out, kp, 1, 0, cout, flags, wsref(wo), b);
+    Op& c = n->ops.back();                      // algorithmic work and bytes of the original convolution
+    c.flops = 2.0 * (double)ti.B * Ho * Wo * cout * k * k * ti.C;
+    c.bytes += (double)cout * k * k * ti.C * 2 - (double)cout * kp * kp * Cp * 2;
+    return out;
+}
+
 static void add_concat(dr_net* n, const std::string& name, int in, int out, int coff) {
     Op op;
     op.kind = OP_CONCAT; op.name = name; op.in0 = in; op.out = out; op.coff = coff;
@@ -172,8 +200,6 @@ static void add_concat(dr_net* n, const std::string& name, int in, int out, int 
     n->ops.push_back(op);
 }
 
-static PRef rawref(int idx) { PRef r; r.raw = idx; return r; }
-static PRef wsref(size_t off) { PRef r; r.ws_off = off; return r; }
 
 static const unsigned BR = DR_BIAS | DR_RELU;
 
@@ -203,8 +229,8 @@ static void build_googlenet(dr_net* n) {
     // conv1: 7x7/2 -> ReLU -> pool -> LRN
     conv_p("conv1", 64, 7, 3, &w, &b);
     if (streamline) {
-        if (slim) t = add_conv(n, "conv1", x, 7, 4, 3, 64, BR, w, b);
-        else { t = add_conv(n, "conv1.conv", x, 7, 4, 3, 64, DR_BIAS, w, b); t = add_simple(n, OP_RELU, "conv1", t); }
+        if (slim) t = add_conv_s2d(n, "conv1", x, 7, 4, 3, 64, BR, w.raw, b);
+        else { t = add_conv_s2d(n, "conv1.conv", x, 7, 4, 3, 64, DR_BIAS, w.raw, b); t = add_simple(n, OP_RELU, "conv1", t); }
     } else if (slim) {
         t = add_conv(n, "conv1", x, 7, 2, 3, 64, BR | DR_POOL | DR_LRN, w, b);
     } else {
@@ -430,13 +456,17 @@ static void build_alexnet(dr_net* n) {
         }
         const bool last = i == 7;
         const char* pool_name = i == 0 ? "pool1" : i == 1 ? "pool2" : "pool5";
+        const bool s2d = l.s >= 2 && l.s * l.s * cin <= 64;      // conv1: 11x11/4 over 3 channels
         if (slim) {
             unsigned f = DR_BIAS | (l.relu ? DR_RELU : 0) | (l.lrn ? DR_LRN : 0) | (last ? DR_OUT_F32 : 0);
-            t = add_conv(n, name, t, l.k, l.s, l.p, l.cout, f, w, rawref(bi));
+            if (s2d) t = add_conv_s2d(n, name, t, l.k, l.s, l.p, l.cout, f, wi, rawref(bi));
+            else t = add_conv(n, name, t, l.k, l.s, l.p, l.cout, f, w, rawref(bi));
             n->ops.back().flops /= l.groups;        // algorithmic work of the grouped layer, not of its dense stand-in
         } else {
             const bool plain = !l.relu && !l.lrn;
-            t = add_conv(n, plain ? name : name + ".conv", t, l.k, l.s, l.p, l.cout, DR_BIAS | (last ? DR_OUT_F32 : 0), w, rawref(bi));
+            const unsigned f = DR_BIAS | (last ? DR_OUT_F32 : 0);
+            if (s2d) t = add_conv_s2d(n, plain ? name : name + ".conv", t, l.k, l.s, l.p, l.cout, f, wi, rawref(bi));
+            else t = add_conv(n, plain ? name : name + ".conv", t, l.k, l.s, l.p, l.cout, f, w, rawref(bi));
             n->ops.back().flops /= l.groups;
             if (l.relu) t = add_simple(n, OP_RELU, l.lrn ? name + ".relu" : name, t);
             if (l.lrn) t = add_simple(n, OP_LRN, name, t);
@@ -546,6 +576,10 @@ int dr_net_prepare(dr_net* n, void* workspace, void* stream) {
     }
     for (const EmbedJob& e : n->embeds) {
         const int st = dr_embed_filter(e.Cout, e.Cin, e.ks, e.kb, n->raw[e.w_small], e.joff, ws + e.w_off, stream);
+        if (st != DR_OK) return st;
+    }
+    for (const S2dJob& j : n->s2d_jobs) {
+        const int st = dr_s2d_filter(j.Cout, j.k, j.C, j.s, j.Cp, n->raw[j.w], ws + j.w_off, stream);
         if (st != DR_OK) return st;
     }
     for (const GroupJob& g : n->group_jobs) {
@@ -660,6 +694,7 @@ int dr_net_forward(dr_net* n, const void* x, void* workspace, float* logits, voi
             case OP_ADD: st = dr_add((size_t)ti.B * ti.H * ti.W * ti.C, in0, in1, out, stream); break;
             case OP_CONCAT: st = dr_concat((size_t)ti.B * ti.H * ti.W, ti.C, in0, to.C, op.coff, out, stream); break;
             case OP_AVGPOOL: st = dr_avgpool_global(ti.B, ti.H, ti.W, ti.C, in0, out, stream); break;
+            case OP_S2D: st = dr_space_to_depth(ti.B, ti.H, ti.W, ti.C, op.s2d_k, op.s2d_s, op.s2d_pad, to.C, in0, out, stream); break;
         }
         if (st != DR_OK) return st;
         if (n->timing && cudaEventRecord(n->ev[2 * i + 1], s) != cudaSuccess) return DR_ERR_CUDA;

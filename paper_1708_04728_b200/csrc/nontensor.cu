@@ -362,6 +362,87 @@ __global__ void embed_groups_kernel(int Cout, int Cin_g, int kk, int groups, con
     }
 }
 
+// ---------------------------------------------------------------- space-to-depth form of a strided few-channel convolution
+// y[n][R][S][(ah*s + aw)*C + c] = x[n][R*s + ah - pad][S*s + aw - pad][c] (zero outside the image and for channels
+// >= s*s*C); one thread per 8 output channels.
+__global__ void s2d_kernel(size_t total8, int H, int W, int C, int s, int pad, int Hs, int Ws, int Cp, const unsigned short* __restrict__ x,
+                           uint4* __restrict__ y) {
+    const int c8n = Cp >> 3;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total8; i += (size_t)gridDim.x * blockDim.x) {
+        const int c8 = (int)(i % c8n);
+        size_t pix = i / c8n;
+        const int S = (int)(pix % Ws); pix /= Ws;
+        const int R = (int)(pix % Hs);
+        const size_t n = pix / Hs;
+        unsigned short e[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int ch = c8 * 8 + j;
+            unsigned short v = 0;
+            if (ch < s * s * C) {
+                const int a = ch / C, c = ch - a * C;
+                const int ah = a / s, aw = a - ah * s;
+                const int h = R * s + ah - pad, w = S * s + aw - pad;
+                if (h >= 0 && h < H && w >= 0 && w < W) v = __ldg(x + ((n * H + h) * W + w) * C + c);
+            }
+            e[j] = v;
+        }
+        uint4 o;
+        o.x = e[0] | ((uint32_t)e[1] << 16); o.y = e[2] | ((uint32_t)e[3] << 16);
+        o.z = e[4] | ((uint32_t)e[5] << 16); o.w = e[6] | ((uint32_t)e[7] << 16);
+        y[i] = o;
+    }
+}
+
+// The same copy for s*C a multiple of 4 (e.g. stride 4 over 3 channels): one thread per (output pixel, ah) moves the
+// s*C contiguous input elements of image row R*s + ah - pad, columns S*s - pad .. S*s - pad + s - 1, to output
+// channels [ah*s*C, (ah+1)*s*C) with 8-byte stores; the thread with ah = 0 also clears channels [s*s*C, Cp).
+__global__ void s2d_rows_kernel(size_t total, int H, int W, int C, int s, int pad, int Hs, int Ws, int Cp, const unsigned short* __restrict__ x,
+                                unsigned short* __restrict__ y) {
+    const int run = s * C;                                   // elements per (pixel, ah); multiple of 4
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int ah = (int)(i % s);
+        size_t pix = i / s;
+        const int S = (int)(pix % Ws);
+        const size_t nr = pix / Ws;                          // n * Hs + R
+        const int R = (int)(nr % Hs);
+        const size_t n = nr / Hs;
+        const int h = R * s + ah - pad, w0 = S * s - pad;
+        const bool row_ok = h >= 0 && h < H;
+        const unsigned short* src = x + ((n * H + (row_ok ? h : 0)) * W) * C;
+        uint2* dst = reinterpret_cast<uint2*>(y + pix * Cp + (size_t)ah * run);
+        for (int e = 0; e < run; e += 4) {
+            unsigned short v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int idx = e + j, w = w0 + idx / C;     // element idx of the run = (aw, c)
+                v[j] = (row_ok && w >= 0 && w < W) ? __ldg(src + ((long long)w0 * C + idx)) : (unsigned short)0;
+            }
+            dst[e >> 2] = make_uint2(v[0] | ((uint32_t)v[1] << 16), v[2] | ((uint32_t)v[3] << 16));
+        }
+        if (ah == 0) {
+            uint2* z = reinterpret_cast<uint2*>(y + pix * Cp + (size_t)s * run);
+            for (int e = 0; e < Cp - s * run; e += 4) z[e >> 2] = make_uint2(0u, 0u);
+        }
+    }
+}
+
+// w [Cout][k][k][C] -> w_out [Cout][kp][kp][Cp], kp = ceil(k/s): tap (R*s + ah, S*s + aw) of the original filter
+// becomes channel (ah*s + aw)*C + c of tap (R, S); taps past k and channels past s*s*C are zero.
+__global__ void s2d_filter_kernel(int k, int C, int s, int kp, int Cp, const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ w_out) {
+    const int j = blockIdx.x, per = kp * kp * Cp;
+    for (int i = threadIdx.x; i < per; i += blockDim.x) {
+        const int ch = i % Cp, t = i / Cp, S = t % kp, R = t / kp;
+        __nv_bfloat16 v = __float2bfloat16_rn(0.f);
+        if (ch < s * s * C) {
+            const int a = ch / C, c = ch - a * C;
+            const int r = R * s + a / s, q = S * s + a % s;
+            if (r < k && q < k) v = w[(((size_t)j * k + r) * k + q) * C + c];
+        }
+        w_out[(size_t)j * per + i] = v;
+    }
+}
+
 }  // namespace dr
 
 // ================================================================ C ABI
@@ -514,6 +595,33 @@ int dr_embed_filter(int Cout, int Cin, int ks, int kb, const void* w_small, int 
     DR_REQUIRE(w_small && w_big, DR_ERR_INVALID_ARG);
     DR_REQUIRE(Cout > 0 && Cin > 0 && ks > 0 && kb >= ks && (ks & 1) && (kb & 1) && joff >= 0, DR_ERR_INVALID_ARG);
     embed_filter_kernel<<<Cout, 256, 0, (cudaStream_t)stream>>>(Cin, ks, kb, (const __nv_bfloat16*)w_small, joff, (__nv_bfloat16*)w_big);
+    count_launch();
+    return launch_status();
+}
+
+int dr_space_to_depth(int B, int H, int W, int C, int k, int s, int pad, int Cp, const void* x, void* y, void* stream) {
+    DR_REQUIRE(x && y && B >= 0 && H > 0 && W > 0 && C > 0 && k > 0 && s > 0 && pad >= 0, DR_ERR_INVALID_ARG);
+    DR_REQUIRE(H + 2 * pad >= k && W + 2 * pad >= k && Cp >= s * s * C && (Cp & 7) == 0, DR_ERR_INVALID_ARG);
+    DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
+    const int kp = (k + s - 1) / s;
+    const int Hs = (H + 2 * pad - k) / s + kp, Ws = (W + 2 * pad - k) / s + kp;     // Ho + kp - 1
+    const size_t total8 = (size_t)B * Hs * Ws * (Cp / 8);
+    if (total8 == 0) return DR_OK;
+    if ((s * C) % 4 == 0 && (Cp - s * s * C) % 4 == 0) {
+        const size_t total = (size_t)B * Hs * Ws * s;
+        s2d_rows_kernel<<<grid_for(total, 256), 256, 0, (cudaStream_t)stream>>>(total, H, W, C, s, pad, Hs, Ws, Cp, (const unsigned short*)x,
+                                                                                 (unsigned short*)y);
+    } else {
+        s2d_kernel<<<grid_for(total8, 256), 256, 0, (cudaStream_t)stream>>>(total8, H, W, C, s, pad, Hs, Ws, Cp, (const unsigned short*)x, (uint4*)y);
+    }
+    count_launch();
+    return launch_status();
+}
+
+int dr_s2d_filter(int Cout, int k, int C, int s, int Cp, const void* w, void* w_out, void* stream) {
+    DR_REQUIRE(w && w_out && Cout > 0 && k > 0 && C > 0 && s > 0 && Cp >= s * s * C, DR_ERR_INVALID_ARG);
+    const int kp = (k + s - 1) / s;
+    s2d_filter_kernel<<<Cout, 256, 0, (cudaStream_t)stream>>>(k, C, s, kp, Cp, (const __nv_bfloat16*)w, (__nv_bfloat16*)w_out);
     count_launch();
     return launch_status();
 }

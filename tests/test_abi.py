@@ -155,7 +155,7 @@ def test_googlenet_streamline_layer_list(dr):
     """Section 3.1's approximate stem: pool strides multiplied into conv1 / conv2, LRN pruned; the rest as DR_ARCH_GOOGLENET."""
     net = dr.Net(dr.DR_ARCH_GOOGLENET_STREAMLINE, dr.DR_MODE_SLIM, 1)
     ref = dr.Net(dr.DR_ARCH_GOOGLENET, dr.DR_MODE_SLIM, 1)
-    assert net.dr_net_num_layers() == ref.dr_net_num_layers()
+    assert net.dr_net_num_layers() == ref.dr_net_num_layers() + 1       # + the space-to-depth copy in front of conv1
     infos = {net.dr_net_layer_info(i)["name"]: net.dr_net_layer_info(i) for i in range(net.dr_net_num_layers())}
     rinfos = {ref.dr_net_layer_info(i)["name"]: ref.dr_net_layer_info(i) for i in range(ref.dr_net_num_layers())}
     assert infos["conv1"]["dims"] == (1, 56, 56, 64) and infos["conv2"]["dims"] == (1, 28, 28, 192)
@@ -166,6 +166,24 @@ def test_googlenet_streamline_layer_list(dr):
     uns = dr.Net(dr.DR_ARCH_GOOGLENET_STREAMLINE, dr.DR_MODE_UNSLIMMED, 1)
     names = [uns.dr_net_layer_info(i)["name"] for i in range(uns.dr_net_num_layers())]
     assert "conv1.pool" not in names and "conv2.lrn" not in names and "conv1.conv" in names
+    assert infos["conv1.s2d"]["kind"] == 1 and infos["conv1.s2d"]["dims"] == (1, 57, 57, 64)   # 7x7/4 -> 2x2/1 over 64 channels
+
+
+def test_alexnet_layer_list(dr):
+    """AlexNet (Section 4.3): conv1 + norm1 and conv2 + norm2 as slim layers; 227x227 input only."""
+    net = dr.Net(dr.DR_ARCH_ALEXNET, dr.DR_MODE_SLIM, 2, 227, 227)
+    infos = [net.dr_net_layer_info(i) for i in range(net.dr_net_num_layers())]
+    assert [i["name"] for i in infos] == ["conv1.s2d", "conv1", "pool1", "conv2", "pool2", "conv3", "conv4", "conv5", "pool5", "fc6", "fc7", "fc8"]
+    li = {i["name"]: i for i in infos}
+    assert li["conv1.s2d"]["dims"] == (2, 57, 57, 64) and li["conv1"]["dims"] == (2, 55, 55, 96) and li["pool1"]["dims"] == (2, 27, 27, 96)
+    assert li["conv2"]["dims"] == (2, 27, 27, 256) and li["pool5"]["dims"] == (2, 6, 6, 256) and li["fc8"]["dims"] == (2, 1, 1, 1000)
+    assert li["conv1"]["flops"] == 2.0 * 2 * 55 * 55 * 96 * 11 * 11 * 3           # of the 11x11/4 layer, not of its re-laid form
+    assert li["conv2"]["flops"] == 2.0 * 2 * 27 * 27 * 256 * 25 * 48              # grouped: half of the dense stand-in
+    names = [net.dr_net_param_spec(i)[0] for i in range(net.dr_net_num_params())]
+    assert net.dr_net_param_spec(names.index("conv2.w"))[1] == (256, 5, 5, 48)
+    with pytest.raises(dr.DrError) as e:
+        dr.Net(dr.DR_ARCH_ALEXNET, dr.DR_MODE_SLIM, 1, 224, 224)
+    assert e.value.status == dr.DR_ERR_INVALID_ARG
 
 
 def test_resnet50_layer_lists(dr):

@@ -135,10 +135,10 @@ def test_alexnet_slim(dr, B, k):
     params = P.alexnet_params(0)
     net, logits, free, keep = check_network(dr, dr.DR_ARCH_ALEXNET, B, subset(B, k), N.alexnet_steps, params, hw=227, out="fc8")
     names = [net.dr_net_layer_info(i)["name"] for i in range(net.dr_net_num_layers())]
-    assert names == ["conv1", "pool1", "conv2", "pool2", "conv3", "conv4", "conv5", "pool5", "fc6", "fc7", "fc8"]
+    assert names == ["conv1.s2d", "conv1", "pool1", "conv2", "pool2", "conv3", "conv4", "conv5", "pool5", "fc6", "fc7", "fc8"]
     # the baseline runs ReLU and LRN as layers of their own
     uns = dr.Net(dr.DR_ARCH_ALEXNET, dr.DR_MODE_UNSLIMMED, B, 227, 227)
-    assert uns.dr_net_num_layers() == 11 + 7 + 2
+    assert uns.dr_net_num_layers() == 12 + 7 + 2
 
 
 @pytest.mark.parametrize("B,k", [(128, 2)])

@@ -145,3 +145,26 @@ def test_embed_filter_exact(dr, O):
     ref = np.zeros((24, 5, 5, Cin))
     O.embed_filter(w1, 5, ref, 0); O.embed_filter(w5, 5, ref, 8); O.embed_filter(w3, 5, ref, 12)
     assert np.array_equal(to_host(big), ref)
+
+
+@pytest.mark.parametrize("B,H,W,k,s,pad,Cout", [(2, 227, 227, 11, 4, 0, 96), (1, 224, 224, 7, 4, 3, 64), (3, 37, 29, 5, 2, 2, 32)])
+def test_space_to_depth_conv(dr, O, B, H, W, k, s, pad, Cout):
+    """dr_space_to_depth / dr_s2d_filter: the re-laid tensors are bit-exact copies (against a restatement of the index
+    map), and the stride-1 convolution over them matches the checker's strided convolution of the original."""
+    import torch
+    from test_oracle_pins import _np_s2d_filter, _np_space_to_depth
+    x = S.normal(40, "x", (B, H, W, 3)); w = S.he_normal(40, "w", Cout, k, 3); b = S.normal(40, "b", (Cout,), 0.1)
+    kp = -(-k // s)
+    Ho, Wo = (H + 2 * pad - k) // s + 1, (W + 2 * pad - k) // s + 1
+    y = torch.full((B, Ho + kp - 1, Wo + kp - 1, 64), 7.0, dtype=torch.bfloat16, device="cuda")
+    wr = torch.full((Cout, kp, kp, 64), 7.0, dtype=torch.bfloat16, device="cuda")
+    dr.dr_space_to_depth(B, H, W, 3, k, s, pad, 64, to_dev_bf16(x), y)
+    dr.dr_s2d_filter(Cout, k, 3, s, 64, to_dev_bf16(w), wr)
+    assert np.array_equal(to_host(y), _np_space_to_depth(x.astype(np.float64), k, s, pad, 64))
+    assert np.array_equal(to_host(wr), _np_s2d_filter(w.astype(np.float64), s, 64))
+    d = dr.dr_conv_desc(k=kp, stride=1, pad=0, Cin=64, Cout=Cout, flags=dr.DR_BIAS | dr.DR_RELU)
+    out = torch.empty((B, Ho, Wo, Cout), dtype=torch.bfloat16, device="cuda")
+    dr.dr_set_conv_path(dr.DR_PATH_AUTO)
+    dr.dr_conv_slim(d, B, Ho + kp - 1, Wo + kp - 1, y, wr, to_dev_f32(b), None, out)
+    assert dr.dr_device_status()[0] == 0 and dr.dr_last_conv_path() == dr.DR_PATH_UMMA_TMA
+    assert_layer_close(to_host(out), O.round_bf16(O.relu(O.conv2d(x, w, b, s, pad))), "space-to-depth conv")

@@ -463,3 +463,40 @@ def test_alexnet_composition_vs_torch():
     t = F.relu(tc("fc7", t, 1, 0))
     ref = torch_to_nhwc(tc("fc8", t, 1, 0))
     assert out["fc8"].shape == (1, 1, 1, 1000) and np.abs(out["fc8"] - ref).max() <= 1e-10 * np.abs(ref).max()
+
+
+def _np_space_to_depth(x, k, s, pad, Cp):
+    """y[n][R][S][(ah*s + aw)*C + c] = x[n][R*s + ah - pad][S*s + aw - pad][c], zero elsewhere (written out for the pin)."""
+    B, H, W, C = x.shape
+    kp = -(-k // s)
+    Hs, Ws = (H + 2 * pad - k) // s + kp, (W + 2 * pad - k) // s + kp
+    y = np.zeros((B, Hs, Ws, Cp), x.dtype)
+    for R in range(Hs):
+        for S_ in range(Ws):
+            for ah in range(s):
+                for aw in range(s):
+                    h, w = R * s + ah - pad, S_ * s + aw - pad
+                    if 0 <= h < H and 0 <= w < W:
+                        y[:, R, S_, (ah * s + aw) * C:(ah * s + aw + 1) * C] = x[:, h, w, :]
+    return y
+
+
+def _np_s2d_filter(w, s, Cp):
+    Cout, k, _, C = w.shape
+    kp = -(-k // s)
+    o = np.zeros((Cout, kp, kp, Cp), w.dtype)
+    for r in range(k):
+        for q in range(k):
+            o[:, r // s, q // s, ((r % s) * s + q % s) * C:((r % s) * s + q % s + 1) * C] = w[:, r, q, :]
+    return o
+
+
+@pytest.mark.parametrize("H,W,k,s,pad", [(35, 31, 11, 4, 0), (32, 40, 7, 4, 3), (17, 18, 5, 2, 2), (20, 20, 3, 3, 1)])
+def test_space_to_depth_identity(H, W, k, s, pad):
+    """A strided convolution over a few channels equals the stride-1 convolution of the space-to-depth image with
+    the re-laid filters (the form the tensor-core kernels run AlexNet's conv1 and the stride-product stem in)."""
+    rng = np.random.default_rng(7)
+    x = rng.standard_normal((2, H, W, 3)); w = rng.standard_normal((5, k, k, 3)); b = rng.standard_normal(5)
+    ref = O.conv2d(x, w, b, s, pad)
+    got = O.conv2d(_np_space_to_depth(x, k, s, pad, 64), _np_s2d_filter(w, s, 64), b, 1, 0)
+    assert got.shape == ref.shape and np.abs(got - ref).max() <= 1e-12 * np.abs(ref).max()
