@@ -261,3 +261,23 @@ def test_bounded_wait_reports_timeout_and_context_survives(dr, O):
     assert_layer_close(got, O.round_bf16(ref), "after timeout")
     with pytest.raises(dr.DrError):
         dr.dr_selftest_wait_timeout(0)
+
+
+def test_conv_degenerate_shapes(dr, O):
+    """Empty batch (nothing launched, canary untouched), a single output pixel, and a plane smaller than the filter's
+    reach on every side (all taps but the centre ones fall on padding)."""
+    import torch
+    dr.dr_set_conv_path(dr.DR_PATH_AUTO)
+    d = dr.dr_conv_desc(k=3, stride=1, pad=1, Cin=64, Cout=64, flags=dr.DR_BIAS | dr.DR_RELU)
+    y = torch.full((4, 4, 64), 768.0, dtype=torch.bfloat16, device="cuda")
+    w = to_dev_bf16(S.he_normal(50, "w", 64, 3, 64)); b = to_dev_f32(S.normal(50, "b", (64,), 0.1))
+    n0 = dr.dr_launch_count()
+    dr.dr_conv_slim(d, 0, 4, 4, y, w, b, None, y)
+    need = dr.dr_conv_workspace_bytes(d, 0, 4, 4)
+    assert need == 0 and dr.dr_launch_count() == n0 and bool((y == 768.0).all())
+    for shape in [(1, 1, 1, 64, 64, 3, 1, 1), (2, 2, 1, 128, 32, 5, 1, 2), (1, 1, 1, 64, 48, 7, 1, 3)]:
+        B, H, W, Cin, Cout, k, s, p = shape
+        x = S.normal(51, "x", (B, H, W, Cin)); wf = S.he_normal(51, "w", Cout, k, Cin); bf = S.normal(51, "b", (Cout,), 0.1)
+        got, _ = run_conv(dr, x, wf, bf, k, s, p, dr.DR_BIAS | dr.DR_RELU)
+        ref, _ = oracle_slim_layer(O, x, wf, bf, k, s, p, dr.DR_BIAS | dr.DR_RELU, dr)
+        assert_layer_close(got, O.round_bf16(ref), f"degenerate {shape}")
