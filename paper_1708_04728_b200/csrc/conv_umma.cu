@@ -127,6 +127,115 @@ __device__ __forceinline__ void drain_fast(const ConvParams& p, uint32_t taddr, 
     }
 }
 
+// Lean epilogue with TMA stores (bias and/or ReLU, bf16 out): row-per-thread 16-byte global stores cost 32 memory
+// wavefronts per warp instruction (32 rows, 32 different lines), which bounds the layers whose output is large
+// against their K (1x1 convolutions at 56x56: 4.2 us per 128 x 256 tile).  Here the four warps of an epilogue group
+// write 64-column chunks of their rows into a shared-memory buffer in the 128-byte-swizzled layout (16-byte
+// shared-memory stores: 4 wavefronts per instruction) and one thread hands the 128 x 64 box to the TMA unit, which
+// writes full lines; two buffers per group, so the store of chunk c overlaps the drain of chunk c+1.  Rows past M
+// are clipped by the tensor map.  Columns beyond the last full 64 go out through drain_fast.
+template <bool RELU>
+__device__ __forceinline__ void drain_tma_store(const ConvParams& p, const CUtensorMap* map_y, uint32_t taddr, int ncols, long long m, bool row_ok,
+                                                bool tile_ok, long long m0, int n0, const float* bias_s, uint8_t* stage, int row, bool elected, int bar,
+                                                int& it) {
+    const uint32_t stage_u32 = smem_u32(stage);
+    const int sw = row & 7;
+    int c = 0;
+    // `it` counts this group's chunks across tiles: buffer it & 1 was last read by store it - 2, whose reading the elected
+    // thread waited for before the barrier of chunk it - 1
+    for (; c + 64 <= ncols; c += 64, ++it) {
+        uint8_t* srow = stage + (it & 1) * 16384 + row * 128;
+#pragma unroll
+        for (int h = 0; h < 64; h += 32) {
+            uint32_t r[32];
+            tmem_ld_x32(taddr + c + h, r);
+            tmem_ld_wait();
+            const float4* b4 = reinterpret_cast<const float4*>(bias_s + n0 + c + h);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {                            // 8 columns = one 16-byte chunk of bfloat16
+                const float4 ba = b4[2 * q], bb = b4[2 * q + 1];
+                float v[8] = {__uint_as_float(r[8 * q]) + ba.x,     __uint_as_float(r[8 * q + 1]) + ba.y, __uint_as_float(r[8 * q + 2]) + ba.z,
+                              __uint_as_float(r[8 * q + 3]) + ba.w, __uint_as_float(r[8 * q + 4]) + bb.x, __uint_as_float(r[8 * q + 5]) + bb.y,
+                              __uint_as_float(r[8 * q + 6]) + bb.z, __uint_as_float(r[8 * q + 7]) + bb.w};
+                if (RELU) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) v[e] = fmaxf(v[e], 0.f);
+                }
+                *reinterpret_cast<uint4*>(srow + ((((h >> 3) + q) ^ sw) << 4)) =
+                    make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+            }
+        }
+        fence_proxy_async_smem();                                     // these writes are read by the TMA unit
+        if (elected) tma_store_wait_read();                           // the store before this one has let go of the other buffer
+        asm volatile("bar.sync %0, 128;" ::"r"(bar) : "memory");
+        if (elected && tile_ok) {
+            tma_store_2d(map_y, stage_u32 + (uint32_t)(it & 1) * 16384u, p.coff + n0 + c, (int)m0);
+            tma_store_commit();
+        }
+    }
+    if (c < ncols) {
+        if (RELU) drain_fast<1>(p, taddr + c, ncols - c, m, row_ok, n0 + c, bias_s);
+        else drain_fast<0>(p, taddr + c, ncols - c, m, row_ok, n0 + c, bias_s);
+    }
+}
+
+// The same with a residual (bias, + residual, optional ReLU): the residual's 128 x 64 box is brought into the buffer
+// by a TMA load (ring of three buffers per group: the box of chunk j+2 is requested when chunk j has been stored; the
+// first two of a tile before the group waits for the tile's MMAs), each thread adds its accumulator row to its row
+// of the buffer in place, and the box goes back out by a TMA store.  ncols is a multiple of 64 (host side).
+__device__ __forceinline__ void residual_box_load(const CUtensorMap* map_r, uint8_t* stage, uint64_t* rfull, int it, int col, int m0) {
+    const int b = it % 3;
+    mbar_arrive_expect_tx(&rfull[b], 16384u);
+    tma_load_2d(stage + b * 16384, map_r, &rfull[b], col, m0);
+}
+
+template <bool RELU>
+__device__ __forceinline__ bool drain_tma_residual(const ConvParams& p, const CUtensorMap* map_y, const CUtensorMap* map_r, uint32_t taddr, int ncols,
+                                                   long long m0, int n0, const float* bias_s, uint8_t* stage, uint64_t* rfull, int row, bool elected,
+                                                   int bar, int& it, volatile int* abort_flag) {
+    const uint32_t stage_u32 = smem_u32(stage);
+    const int sw = row & 7;
+    const int nch = ncols >> 6;
+    for (int j = 0; j < nch; ++j, ++it) {
+        const int b = it % 3, c = j << 6;
+        if (!__all_sync(0xffffffffu, mbar_wait(&rfull[b], (uint32_t)(it / 3) & 1u, abort_flag))) return false;
+        uint8_t* srow = stage + b * 16384 + row * 128;
+#pragma unroll
+        for (int h = 0; h < 64; h += 32) {
+            uint32_t r[32];
+            tmem_ld_x32(taddr + c + h, r);
+            tmem_ld_wait();
+            const float4* b4 = reinterpret_cast<const float4*>(bias_s + n0 + c + h);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {                            // 8 columns = one 16-byte chunk of bfloat16
+                uint4* cell = reinterpret_cast<uint4*>(srow + ((((h >> 3) + q) ^ sw) << 4));
+                const uint4 u = *cell;
+                const float4 ba = b4[2 * q], bb = b4[2 * q + 1];
+                float v[8] = {__uint_as_float(r[8 * q]) + ba.x + bf16_lo(u.x),     __uint_as_float(r[8 * q + 1]) + ba.y + bf16_hi(u.x),
+                              __uint_as_float(r[8 * q + 2]) + ba.z + bf16_lo(u.y), __uint_as_float(r[8 * q + 3]) + ba.w + bf16_hi(u.y),
+                              __uint_as_float(r[8 * q + 4]) + bb.x + bf16_lo(u.z), __uint_as_float(r[8 * q + 5]) + bb.y + bf16_hi(u.z),
+                              __uint_as_float(r[8 * q + 6]) + bb.z + bf16_lo(u.w), __uint_as_float(r[8 * q + 7]) + bb.w + bf16_hi(u.w)};
+                if (RELU) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) v[e] = fmaxf(v[e], 0.f);
+                }
+                *cell = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+            }
+        }
+        fence_proxy_async_smem();
+        asm volatile("bar.sync %0, 128;" ::"r"(bar) : "memory");
+        if (elected) {
+            tma_store_2d(map_y, stage_u32 + (uint32_t)b * 16384u, p.coff + n0 + c, (int)m0);
+            tma_store_commit();
+            if (j + 2 < nch) {
+                asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store of chunk it-1 has let go of buffer (it+2) % 3
+                residual_box_load(map_r, stage, rfull, it + 2, n0 + c + 128, (int)m0);
+            }
+        }
+    }
+    return true;
+}
+
 // Epilogue of a layer that ends in LRN across channels without pooling (bias, ReLU, LRN, bf16 store): the thread owns
 // every channel of its output pixel (one tile spans all of Cout <= 256), so the LRN window is a sliding sum over the
 // accumulator row, read from TMEM in chunks of W columns with two columns of look-back (kept in registers) and two
@@ -443,6 +552,7 @@ constexpr int T_ACC_COLS = 256;   // columns per accumulator buffer; two buffers
 
 struct TmaShared {
     uint64_t full[T_MAX_STAGES], empty[T_MAX_STAGES], tfull[2], tempty[2];
+    uint64_t rfull[2][3];      // residual boxes of the TMA epilogue: per epilogue group, ring of three
     uint32_t tmem_base;
     int abort;
 };
@@ -455,8 +565,9 @@ struct TmaShared {
 // start when both epilogue groups (group g drains sub-block g) have emptied it.
 template <bool PAIR, int KPB, bool WIDE>
 __global__ void __launch_bounds__(T_THREADS, 1)
-conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const int a_mode,
-                     const int stages, const int sub_bytes) {
+conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                     const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_r, const int a_mode, const int stages,
+                     const int sub_bytes, const int ep_stage_off) {
     constexpr int kpb = KPB;
     // a pipeline stage holds `kpb` k-blocks (sub-stages of sub_bytes = A tile + B tile): one barrier
     // round trip then covers kpb * 4 MMAs, which keeps the issuing thread ahead of the tensor pipe
@@ -481,6 +592,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], (PAIR ? 8 : 4) * (WIDE ? 2 : 1)); }
+        for (int a = 0; a < 6; ++a) mbar_init(&sh.rfull[a / 3][a % 3], 1);
         sh.abort = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_a);
@@ -647,11 +759,19 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
         const int g = (warp - 2) >> 2;
         const int q = warp & 3;
         const int row = q * 32 + lane;
+        int ep_it = 0;                                           // chunks this group has handed to the TMA unit so far
         for (int t = WIDE ? unit : unit + g * nunits, au = 0; t < total; t += WIDE ? nunits : 2 * nunits, ++au) {
             const int nb = t / m_units, mu = t - nb * m_units;
             const int n0 = WIDE ? nb * tile_n + g * p.Nt : nb * p.Nt;      // WIDE: group g drains sub-block g of every tile
             const int Nj = min(p.Nt, cout16 - n0);                         // WIDE: may be <= 0 (no second sub-block)
             const int mt = PAIR ? 2 * mu + (int)rank : mu;
+            const bool res_tma = lean && ep_stage_off > 0 && lean_mode >= 2 && mt < p.m_tiles;
+            if (res_tma && ((warp - 2) & 3) == 0 && lane == 0) {
+                // this tile's first two residual boxes, requested before the wait for its MMAs
+                uint8_t* st = smem + ep_stage_off + g * 49152;
+                residual_box_load(&map_r, st, sh.rfull[g], ep_it, n0, (int)((long long)mt * TILE_M));
+                if (Nj > 64) residual_box_load(&map_r, st, sh.rfull[g], ep_it + 1, n0 + 64, (int)((long long)mt * TILE_M));
+            }
             const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[WIDE ? 0 : g], au & 1, abort_flag));
             if (!ok) {
                 if (!*abort_flag) report_timeout(p.status, 14, t);
@@ -666,6 +786,26 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                 // nothing to drain
             } else if (lrn_ep) {
                 drain_lrn(p, taddr, Nj, m, row_ok, bias_s);
+            } else if (lean && ep_stage_off > 0 && lean_mode >= 2) {
+                if (res_tma) {
+                    uint8_t* st = smem + ep_stage_off + g * 49152;
+                    const bool elected = ((warp - 2) & 3) == 0 && lane == 0;
+                    const long long m0 = (long long)mt * TILE_M;
+                    const bool done = lean_mode == 3
+                        ? drain_tma_residual<true>(p, &map_y, &map_r, taddr, Nj, m0, n0, bias_s, st, sh.rfull[g], row, elected, 1 + g, ep_it, abort_flag)
+                        : drain_tma_residual<false>(p, &map_y, &map_r, taddr, Nj, m0, n0, bias_s, st, sh.rfull[g], row, elected, 1 + g, ep_it, abort_flag);
+                    if (!done) {
+                        if (!*abort_flag) report_timeout(p.status, 15, t);
+                        *abort_flag = 1;
+                        break;
+                    }
+                }
+            } else if (lean && ep_stage_off > 0 && lean_mode < 2) {
+                uint8_t* st = smem + ep_stage_off + g * 32768;
+                const bool elected = ((warp - 2) & 3) == 0 && lane == 0;
+                const long long m0 = (long long)mt * TILE_M;
+                if (lean_mode == 1) drain_tma_store<true>(p, &map_y, taddr, Nj, m, row_ok, mt < p.m_tiles, m0, n0, bias_s, st, row, elected, 1 + g, ep_it);
+                else drain_tma_store<false>(p, &map_y, taddr, Nj, m, row_ok, mt < p.m_tiles, m0, n0, bias_s, st, row, elected, 1 + g, ep_it);
             } else if (lean) {
                 if (lean_mode == 1) drain_fast<1>(p, taddr, Nj, m, row_ok, n0, bias_s);
                 else if (lean_mode == 3) drain_fast<3>(p, taddr, Nj, m, row_ok, n0, bias_s);
@@ -682,6 +822,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             }
         }
     }
+    if (ep_stage_off > 0 && warp >= 2 && ((warp - 2) & 3) == 0 && lane == 0) tma_store_wait_all();   // TMA stores of this thread have landed
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {   // give copies and MMAs still in flight time to land before shared memory and TMEM go away
@@ -779,8 +920,8 @@ bool conv_umma_tma_supports(const ConvParams& p) {
 // Pipeline shape: k-blocks per stage (kpb) and number of stages.  Measured on B200: wide tiles
 // (Nt >= 208) run best with one k-block per barrier round trip, narrower ones with two (their MMAs
 // are short, so the round trip has to cover more of them); never more than the layer has.
-static void pick_pipeline(int sub_bytes, int nkb, int nt, int* kpb, int* stages) {
-    const int budget = T_SMEM_MAX - 1024;
+static void pick_pipeline(int sub_bytes, int nkb, int nt, int ep_bytes, int* kpb, int* stages) {
+    const int budget = T_SMEM_MAX - 1024 - ep_bytes;
     int k = tunable("DR_TMA_KPB", 0);
     if (k <= 0) k = nt >= 208 ? 1 : 2;
     if (k >= 4) k = 4; else if (k == 3) k = 2;          // instantiated: 1, 2, 4
@@ -793,13 +934,55 @@ static void pick_pipeline(int sub_bytes, int nkb, int nt, int* kpb, int* stages)
     *stages = st;
 }
 
+// The TMA epilogue pays where the output is large against K (few k-blocks per tile: the pipeline then needs little
+// shared memory, and the row-per-thread stores would bound the layer): bias / ReLU and residual epilogues of layers
+// with at most 4 k-blocks (residual: n-blocks that are multiples of 64 columns).  Returns the shared memory it needs
+// (0: not used).  map_y: y as a [M][coff + Cout] matrix with row pitch ldc; map_r: the residual as [M][Cout]; boxes of
+// 128 rows x 64 columns, 128-byte swizzle.
+static int tma_epilogue_bytes(const ConvParams& p, bool pair_or_wide, CUtensorMap* map_y, CUtensorMap* map_r) {
+    if (tunable("DR_TMA_STORE_EP", 1) == 0 || pair_or_wide) return 0;
+    if (p.flags & (DR_OUT_F32 | DR_LRN)) return 0;
+    if ((p.flags & DR_RESIDUAL) && (p.flags & DR_RELU)) return 0;
+    if ((p.Cout & 15) || p.Cout > T_BIAS_MAX || (p.ldc & 7) || (p.coff & 7) || p.Nt < 64) return 0;
+    const int nkb = p.k * p.k * ((p.Cin + 63) / 64);
+    const bool res = (p.flags & DR_RESIDUAL) != 0;
+    // measured (ResNet-50 at batch 128, GoogLeNet at 256): a gain up to 4 k-blocks with a residual or with at least 256
+    // output channels, up to 2 k-blocks otherwise; beyond that the lost pipeline stages cost more than the stores
+    if (res ? (nkb > 4 || (p.Nt & 63) || (p.Cout & 63)) : (nkb > 4 || (nkb > 2 && p.Cout < 256))) return 0;
+    if (!load_encoders()) return 0;
+    const cuuint32_t box[2] = {64, TILE_M};
+    const cuuint32_t es[2] = {1, 1};
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)(p.coff + p.Cout), (cuuint64_t)p.M};
+        const cuuint64_t strides[1] = {(cuuint64_t)p.ldc * 2};
+        if (g_encode_tiled(map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.y, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return 0;
+    }
+    if (res) {
+        const cuuint64_t dims[2] = {(cuuint64_t)p.Cout, (cuuint64_t)p.M};
+        const cuuint64_t strides[1] = {(cuuint64_t)p.Cout * 2};
+        if (g_encode_tiled(map_r, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)p.residual, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return 0;
+    }
+    return res ? 2 * 3 * 16384 : 2 * 2 * 16384;                  // per epilogue group: three / two 16 KB buffers
+}
+
 static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, int a_mode, bool wide, cudaStream_t stream) {
     static bool attr_set = false;
     static int max_clusters = 0;
     const int sub_bytes = A_TILE_BYTES + (wide ? 2 : 1) * ((p.Nt * 64 + 1023) & ~1023);
     int kpb, stages;
-    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, &kpb, &stages);
-    int smem_bytes = stages * kpb * sub_bytes + 1024;
+    alignas(64) CUtensorMap map_y = map_a, map_r = map_a;        // placeholders when the TMA epilogue is off
+    int ep_bytes = tma_epilogue_bytes(p, true, &map_y, &map_r);
+    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, ep_bytes, &kpb, &stages);
+    if (ep_bytes && stages < 2) {                                // not enough room left for the operand pipeline: do without
+        ep_bytes = 0;
+        pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, 0, &kpb, &stages);
+    }
+    const int ep_off = ep_bytes ? stages * kpb * sub_bytes : 0;
+    int smem_bytes = stages * kpb * sub_bytes + ep_bytes + 1024;
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -823,10 +1006,10 @@ static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUte
     const int pairs = pair_tiles < max_clusters ? pair_tiles : max_clusters;
     cfg.gridDim = dim3(2 * pairs);
     cudaError_t e;
-    if (wide) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 1, true>, p, map_a, map_b, a_mode, stages, sub_bytes);
-    else if (kpb == 4) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 4, false>, p, map_a, map_b, a_mode, stages, sub_bytes);
-    else if (kpb == 2) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 2, false>, p, map_a, map_b, a_mode, stages, sub_bytes);
-    else e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 1, false>, p, map_a, map_b, a_mode, stages, sub_bytes);
+    if (wide) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 1, true>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
+    else if (kpb == 4) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 4, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
+    else if (kpb == 2) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 2, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
+    else e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 1, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
     if (e != cudaSuccess) return DR_ERR_CUDA;
     count_launch();
     return launch_status();
@@ -883,13 +1066,20 @@ int conv_umma_tma_launch(const ConvParams& p_in, cudaStream_t stream) {
     // half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
     const int sub_bytes = A_TILE_BYTES + (wide ? 2 : 1) * ((p.Nt * 128 + 1023) & ~1023);
     int kpb, stages;
-    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, &kpb, &stages);
-    int smem_bytes = stages * kpb * sub_bytes + 1024;
+    alignas(64) CUtensorMap map_y = map_a, map_r = map_a;        // placeholders when the TMA epilogue is off
+    int ep_bytes = tma_epilogue_bytes(p, wide, &map_y, &map_r);
+    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, ep_bytes, &kpb, &stages);
+    if (ep_bytes && stages < 2) {                                // not enough room left for the operand pipeline: do without
+        ep_bytes = 0;
+        pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, 0, &kpb, &stages);
+    }
+    const int ep_off = ep_bytes ? stages * kpb * sub_bytes : 0;
+    int smem_bytes = stages * kpb * sub_bytes + ep_bytes + 1024;
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
-    if (wide) conv_umma_tma_kernel<false, 1, true><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
-    else if (kpb == 4) conv_umma_tma_kernel<false, 4, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
-    else if (kpb == 2) conv_umma_tma_kernel<false, 2, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
-    else conv_umma_tma_kernel<false, 1, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, a_mode, stages, sub_bytes);
+    if (wide) conv_umma_tma_kernel<false, 1, true><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
+    else if (kpb == 4) conv_umma_tma_kernel<false, 4, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
+    else if (kpb == 2) conv_umma_tma_kernel<false, 2, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
+    else conv_umma_tma_kernel<false, 1, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
     count_launch();
     return launch_status();
 }
