@@ -89,6 +89,22 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(ms: float, world: int, device: str = "cuda") -> float:
+    """Time of the slowest replica (the replicas run side by side; the job ends with the last of them)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_images_per_s(ms_max: float, images_per_rank_step: int, steps: int, world: int) -> float:
+    """Images all replicas processed per second: every rank runs `steps` steps of its own batch (weak scaling)."""
+    return world * images_per_rank_step * steps / (ms_max * 1e-3)
+
+
 def oracle_images_per_s(n_images: int, steps: int = 1):
     """The CPU checker's GoogLeNet forward, as it stands, on the host cores."""
     import dr_synth.params as P
@@ -289,9 +305,8 @@ def main():
     assert st == 0, f"device status {st} {info}"
     assert bool(torch.isfinite(logits).all())
     total_ms = sum(times)
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); total_ms = float(t.item())
-    value = world * B * args.steps / (total_ms * 1e-3)
+    total_ms = max_over_ranks(total_ms, world)
+    value = whole_job_images_per_s(total_ms, B, args.steps, world)
 
     # ---- end to end through the public API with host buffers: every step copies its batch from pinned host
     # memory, runs the forward pass and copies the logits back.  The copy of step i+1 runs on a second
@@ -329,9 +344,8 @@ def main():
     if world > 1:
         dist.barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_ms = float(t.item())
-    e2e_value = world * B * e2e_steps / (e2e_ms * 1e-3)
+    e2e_ms = max_over_ranks(e2e_ms, world)
+    e2e_value = whole_job_images_per_s(e2e_ms, B, e2e_steps, world)
     assert bool(torch.isfinite(logits_host).all())
     clocks = sampler.stop() if sampler else None
 
