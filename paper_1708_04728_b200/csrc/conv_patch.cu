@@ -260,6 +260,7 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
     __syncthreads();
     cluster_sync_all();                                                      // both CTAs' barriers exist before any remote arrive
     tc_fence_after();
+    grid_launch_dependents();                                                // a split-K layer behind this one may start its prologue
     const uint32_t tmem = sh.tmem_base;
     volatile int* abort_flag = &sh.abort;
 

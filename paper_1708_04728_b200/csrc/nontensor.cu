@@ -119,6 +119,9 @@ __global__ void bn_scalar_kernel(size_t n, int C, const __nv_bfloat16* __restric
 // One thread per (output pixel, 8 channels).  First maximum in row-major window order wins.
 __global__ void maxpool_kernel(int B, int H, int W, int C8, int Ho, int Wo, int k, int s, int p,
                                const uint4* __restrict__ x, uint4* __restrict__ y, int32_t* __restrict__ argmax) {
+    // a kernel launched behind this one with programmatic serialization (the split-K convolution) may start its
+    // prologue and filter prefetch now; it waits for this kernel's completion before it reads y
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const size_t total = (size_t)B * Ho * Wo * C8;
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
@@ -294,6 +297,7 @@ __global__ void concat_scalar_kernel(size_t n, int C, int ldc, int coff, const _
 constexpr int AVG_SPLIT = 8;
 __global__ void avgpool_kernel(int HW, int C, const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y) {
     __shared__ float part[AVG_SPLIT][64];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see maxpool_noarg_kernel
     const int n = blockIdx.y, c = blockIdx.x * 64 + threadIdx.x * 2;
     float s0 = 0.f, s1 = 0.f;
     if (c < C) {
