@@ -61,6 +61,12 @@ int conv_make_params(const dr_conv_desc* d, int B, int H, int W, const void* x, 
         p.lrn_c2 = (float)(be * (be + 1) / 2);
         p.lrn_c3 = (float)(-be * (be + 1) * (be + 2) / 6);
         p.lrn_c4 = (float)(be * (be + 1) * (be + 2) * (be + 3) / 24);
+        const double au = kk > 0 ? (double)p.lrn_alpha_n / kk : 0.0, kp = kk > 0 ? pow(kk, -be) : 0.0;
+        p.lrn_s1 = (float)(kp * p.lrn_c1 * au);
+        p.lrn_s2 = (float)(kp * p.lrn_c2 * au * au);
+        p.lrn_s3 = (float)(kp * p.lrn_c3 * au * au * au);
+        p.lrn_s4 = (float)(kp * p.lrn_c4 * au * au * au * au);
+        p.lrn_ss_max = au > 0 ? (float)(0.03125 / au) : 3.0e38f;
     }
     p.ldc = ldc; p.coff = coff;
     p.M = (long long)B * p.Ho * p.Wo;

@@ -40,6 +40,9 @@ struct ConvParams {
     float lrn_alpha_n, lrn_beta, lrn_k;
     float lrn_inv_k, lrn_kpow;   // 1/k and k^(-beta)
     float lrn_c1, lrn_c2, lrn_c3, lrn_c4;   // binomial series of (1+u)^(-beta)
+    // the same series in the window sum ss itself, k^(-beta) folded in: scale = s0 + ss (s1 + ss (s2 + ss (s3 + ss s4))),
+    // valid while ss < lrn_ss_max (u = (alpha/n) ss / k below 1/32)
+    float lrn_s1, lrn_s2, lrn_s3, lrn_s4, lrn_ss_max;
     int ldc, coff;
     long long M;           // B*Ho*Wo
     int Nt;                // output channels per n-block (multiple of 16, <= 256)

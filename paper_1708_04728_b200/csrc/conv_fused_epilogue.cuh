@@ -67,6 +67,71 @@ __device__ __forceinline__ void fe_lrn_scale(const ConvParams& p, const float* s
     }
 }
 
+// 32 accumulator columns starting at column c (+ bias, ReLU) into x; zeros when the chunk lies past the last channel.
+__device__ __forceinline__ void fe_load_chunk(uint32_t taddr, const float* bias_s, int c, bool present, bool relu, float* x) {
+    if (present) {
+        uint32_t r[32];
+        ptx::tmem_ld_x32(taddr + c, r);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float4 b4 = *reinterpret_cast<const float4*>(bias_s + c + 4 * q);
+            const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float v = __uint_as_float(r[4 * q + k]) + bb[k];
+                x[4 * q + k] = relu ? fmaxf(v, 0.f) : v;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) x[j] = 0.f;
+    }
+}
+
+// LRN (window of five) of the 32 channels in cur, given the two channels before (pm2, pm1) and the chunk after;
+// the result goes to dst as bfloat16 (-inf for rows outside the convolution plane).  The window sum slides:
+// ss[j] = ss[j-1] + x[j+2]^2 - x[j-3]^2, restarted from its five terms every 8 channels.  The scale is the series in
+// ss with k^(-beta) folded in while every ss of the warp's chunk is below lrn_ss_max; exp2/log2 otherwise.
+__device__ __forceinline__ void fe_lrn_chunk(const ConvParams& p, const float* cur, const float* nxt, float& pm2, float& pm1, uint8_t* dst,
+                                             bool valid) {
+    float sq[36];                                  // squares of x[c0-2 .. c0+33]
+    sq[0] = pm2 * pm2; sq[1] = pm1 * pm1;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) sq[2 + j] = cur[j] * cur[j];
+    sq[34] = nxt[0] * nxt[0]; sq[35] = nxt[1] * nxt[1];
+    float ss[32], sc[32];
+    float smax = 0.f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        if ((j & 7) == 0) ss[j] = (sq[j] + sq[j + 1]) + (sq[j + 2] + sq[j + 3]) + sq[j + 4];
+        else ss[j] = fmaxf((ss[j - 1] - sq[j - 1]) + sq[j + 4], 0.f);
+        smax = fmaxf(smax, ss[j]);
+    }
+    if (__all_sync(0xffffffffu, smax < p.lrn_ss_max)) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sc[j] = fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], p.lrn_s4, p.lrn_s3), p.lrn_s2), p.lrn_s1), p.lrn_kpow);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sc[j] = __powf(fmaf(p.lrn_alpha_n, ss[j], p.lrn_k), -p.lrn_beta);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint4 v;
+        if (valid) {
+            v.x = pack_bf16(cur[8 * q + 0] * sc[8 * q + 0], cur[8 * q + 1] * sc[8 * q + 1]);
+            v.y = pack_bf16(cur[8 * q + 2] * sc[8 * q + 2], cur[8 * q + 3] * sc[8 * q + 3]);
+            v.z = pack_bf16(cur[8 * q + 4] * sc[8 * q + 4], cur[8 * q + 5] * sc[8 * q + 5]);
+            v.w = pack_bf16(cur[8 * q + 6] * sc[8 * q + 6], cur[8 * q + 7] * sc[8 * q + 7]);
+        } else {
+            v.x = v.y = v.z = v.w = 0xFF80FF80u;     // -inf, -inf
+        }
+        *reinterpret_cast<uint4*>(dst + 16 * q) = v;
+    }
+    pm2 = cur[30];
+    pm1 = cur[31];
+}
+
 // taddr: TMEM address of this thread's lane, column 0 of the accumulator.  row = 0..127.
 // Called by the 4 warps of one epilogue group together (a kernel may run two groups on alternate tiles,
 // each with its own stage buffer and named barrier); `release` is invoked by each warp once its TMEM
@@ -91,68 +156,17 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
 
     // ---- drain TMEM (+ bias, ReLU, LRN when LRN comes first), stage
     if (lrn_first) {
-        float cur[32], nxt[32];
+        // two register chunks used alternately as "current" and "next" (no copy between them)
+        float xa[32], xb[32];
         float pm2 = 0.f, pm1 = 0.f;                      // x[c-2], x[c-1] of the chunk before
-        {
-            uint32_t r[32];
-            ptx::tmem_ld_x32(taddr, r);
-            ptx::tmem_ld_wait();
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                const float4 b4 = *reinterpret_cast<const float4*>(bias_s + 4 * q);
-                const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float v = __uint_as_float(r[4 * q + k]) + bb[k];
-                    cur[4 * q + k] = relu ? fmaxf(v, 0.f) : v;
-                }
-            }
-        }
-        for (int c0 = 0; c0 < C; c0 += 32) {
+        fe_load_chunk(taddr, bias_s, 0, true, relu, xa);
+        for (int c0 = 0; c0 < C; c0 += 64) {
+            fe_load_chunk(taddr, bias_s, c0 + 32, c0 + 32 < C, relu, xb);
+            fe_lrn_chunk(p, xa, xb, pm2, pm1, srow + c0 * 2, valid);
             if (c0 + 32 < C) {
-                uint32_t r[32];
-                ptx::tmem_ld_x32(taddr + c0 + 32, r);
-                ptx::tmem_ld_wait();
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float4 b4 = *reinterpret_cast<const float4*>(bias_s + c0 + 32 + 4 * q);
-                    const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float v = __uint_as_float(r[4 * q + k]) + bb[k];
-                        nxt[4 * q + k] = relu ? fmaxf(v, 0.f) : v;
-                    }
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) nxt[j] = 0.f;
+                fe_load_chunk(taddr, bias_s, c0 + 64, c0 + 64 < C, relu, xa);
+                fe_lrn_chunk(p, xb, xa, pm2, pm1, srow + (c0 + 32) * 2, valid);
             }
-            float sq[36];                                  // squares of x[c0-2 .. c0+33]
-            sq[0] = pm2 * pm2; sq[1] = pm1 * pm1;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) sq[2 + j] = cur[j] * cur[j];
-            sq[34] = nxt[0] * nxt[0]; sq[35] = nxt[1] * nxt[1];
-            float ss[32], sc[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) ss[j] = (sq[j] + sq[j + 1]) + (sq[j + 2] + sq[j + 3]) + sq[j + 4];
-            fe_lrn_scale<32>(p, ss, sc);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint4 v;
-                if (valid) {
-                    v.x = pack_bf16(cur[8 * q + 0] * sc[8 * q + 0], cur[8 * q + 1] * sc[8 * q + 1]);
-                    v.y = pack_bf16(cur[8 * q + 2] * sc[8 * q + 2], cur[8 * q + 3] * sc[8 * q + 3]);
-                    v.z = pack_bf16(cur[8 * q + 4] * sc[8 * q + 4], cur[8 * q + 5] * sc[8 * q + 5]);
-                    v.w = pack_bf16(cur[8 * q + 6] * sc[8 * q + 6], cur[8 * q + 7] * sc[8 * q + 7]);
-                } else {
-                    v.x = v.y = v.z = v.w = 0xFF80FF80u;     // -inf, -inf
-                }
-                *reinterpret_cast<uint4*>(srow + (c0 + 8 * q) * 2) = v;
-            }
-            pm2 = cur[30];
-            pm1 = cur[31];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) cur[j] = nxt[j];
         }
     } else {
         for (int c0 = 0; c0 < C; c0 += 32) {
