@@ -53,14 +53,12 @@ __device__ __forceinline__ void fe_init(const ConvParams& p, uint8_t* stage, int
 // LRN scale factors for N window sums at once; the series/exact choice is uniform over the warp.
 template <int N>
 __device__ __forceinline__ void fe_lrn_scale(const ConvParams& p, const float* ss, float* scale) {
-    float umax = 0.f;
-    float u[N];
+    float smax = 0.f;
 #pragma unroll
-    for (int j = 0; j < N; ++j) { u[j] = p.lrn_alpha_n * p.lrn_inv_k * ss[j]; umax = fmaxf(umax, u[j]); }
-    if (__all_sync(0xffffffffu, umax < 0.03125f)) {
+    for (int j = 0; j < N; ++j) smax = fmaxf(smax, ss[j]);
+    if (__all_sync(0xffffffffu, smax < p.lrn_ss_max)) {      // series in ss, k^(-beta) folded into the coefficients
 #pragma unroll
-        for (int j = 0; j < N; ++j)
-            scale[j] = p.lrn_kpow * fmaf(u[j], fmaf(u[j], fmaf(u[j], fmaf(u[j], p.lrn_c4, p.lrn_c3), p.lrn_c2), p.lrn_c1), 1.f);
+        for (int j = 0; j < N; ++j) scale[j] = fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], p.lrn_s4, p.lrn_s3), p.lrn_s2), p.lrn_s1), p.lrn_kpow);
     } else {
 #pragma unroll
         for (int j = 0; j < N; ++j) scale[j] = __powf(fmaf(p.lrn_alpha_n, ss[j], p.lrn_k), -p.lrn_beta);
@@ -91,8 +89,9 @@ __device__ __forceinline__ void fe_load_chunk(uint32_t taddr, const float* bias_
 
 // LRN (window of five) of the 32 channels in cur, given the two channels before (pm2, pm1) and the chunk after;
 // the result goes to dst as bfloat16 (-inf for rows outside the convolution plane).  The window sum slides:
-// ss[j] = ss[j-1] + x[j+2]^2 - x[j-3]^2, restarted from its five terms every 8 channels.  The scale is the series in
-// ss with k^(-beta) folded in while every ss of the warp's chunk is below lrn_ss_max; exp2/log2 otherwise.
+// ss[j] = ss[j-1] + x[j+2]^2 - x[j-3]^2, restarted from its five terms every 8 channels (a sum that cancels to a few
+// ulps below zero is harmless: the scale is k + (alpha/n) ss with k > 0).  The scale is the series in ss with k^(-beta)
+// folded in while the sum of all squares of the warp's chunk is below lrn_ss_max; exp2/log2 otherwise.
 __device__ __forceinline__ void fe_lrn_chunk(const ConvParams& p, const float* cur, const float* nxt, float& pm2, float& pm1, uint8_t* dst,
                                              bool valid) {
     float sq[36];                                  // squares of x[c0-2 .. c0+33]
@@ -101,14 +100,14 @@ __device__ __forceinline__ void fe_lrn_chunk(const ConvParams& p, const float* c
     for (int j = 0; j < 32; ++j) sq[2 + j] = cur[j] * cur[j];
     sq[34] = nxt[0] * nxt[0]; sq[35] = nxt[1] * nxt[1];
     float ss[32], sc[32];
-    float smax = 0.f;
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
         if ((j & 7) == 0) ss[j] = (sq[j] + sq[j + 1]) + (sq[j + 2] + sq[j + 3]) + sq[j + 4];
-        else ss[j] = fmaxf((ss[j - 1] - sq[j - 1]) + sq[j + 4], 0.f);
-        smax = fmaxf(smax, ss[j]);
+        else ss[j] = (ss[j - 1] - sq[j - 1]) + sq[j + 4];
     }
-    if (__all_sync(0xffffffffu, smax < p.lrn_ss_max)) {
+    // every window sum is at most the sum of all squares = seven disjoint windows + the last square
+    const float total = ((ss[0] + ss[5]) + (ss[10] + ss[15])) + ((ss[20] + ss[25]) + (ss[30] + sq[35]));
+    if (__all_sync(0xffffffffu, total < p.lrn_ss_max)) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) sc[j] = fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], p.lrn_s4, p.lrn_s3), p.lrn_s2), p.lrn_s1), p.lrn_kpow);
     } else {

@@ -265,31 +265,31 @@ __device__ __forceinline__ void lrn_chunk(const ConvParams& p, uint32_t taddr, i
     const bool h1 = p.lrn_half >= 1, h2 = p.lrn_half >= 2;
     // scale^(-beta), scale = k (1 + u), u = (alpha/n) ss / k.  While u < 1/32 for the whole chunk of the warp (always so
     // for the usual alpha = 1e-4) the binomial series of (1 + u)^(-beta) to u^4 is exact to float32 resolution and
-    // needs no special-function unit; otherwise exp2/log2.
-    float sq[W + 4], u[W];
+    // needs no special-function unit (evaluated in ss itself, k^(-beta) folded into its coefficients); otherwise exp2/log2.
+    float sq[W + 4], ss[W];
 #pragma unroll
     for (int j = 0; j < W + 4; ++j) sq[j] = x[j] * x[j];
-    const float au = p.lrn_alpha_n * p.lrn_inv_k;
-    float umax = 0.f;
+    float total = 0.f;                                        // sum of all squares: an upper bound of every window sum
 #pragma unroll
     for (int j = 0; j < W; ++j) {
-        float ss = sq[2 + j];
-        if (h1) ss += sq[1 + j] + sq[3 + j];
-        if (h2) ss += sq[j] + sq[4 + j];
-        u[j] = au * ss;
-        umax = fmaxf(umax, u[j]);
+        float v = sq[2 + j];
+        if (h1) v += sq[1 + j] + sq[3 + j];
+        if (h2) v += sq[j] + sq[4 + j];
+        ss[j] = v;
     }
-    const bool series = !__any_sync(0xffffffffu, !(umax < 0.03125f));
+#pragma unroll
+    for (int j = 0; j < W + 4; j += 4) total += (sq[j] + sq[j + 1]) + (sq[j + 2] + sq[j + 3]);
+    const bool series = !__any_sync(0xffffffffu, !(total < p.lrn_ss_max));
     uint32_t o[W / 2];
 #pragma unroll
     for (int j = 0; j < W; j += 2) {
         float y2[2];
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-            const float uu = u[j + e];
+            const float s1 = ss[j + e];
             float f;
-            if (series) f = p.lrn_kpow * fmaf(uu, fmaf(uu, fmaf(uu, fmaf(uu, p.lrn_c4, p.lrn_c3), p.lrn_c2), p.lrn_c1), 1.f);
-            else f = p.lrn_kpow * exp2f(-p.lrn_beta * log2f(1.f + uu));
+            if (series) f = fmaf(s1, fmaf(s1, fmaf(s1, fmaf(s1, p.lrn_s4, p.lrn_s3), p.lrn_s2), p.lrn_s1), p.lrn_kpow);
+            else f = exp2f(-p.lrn_beta * log2f(fmaf(p.lrn_alpha_n, s1, p.lrn_k)));
             y2[e] = x[2 + j + e] * f;
         }
         o[j >> 1] = pack_bf16(y2[0], y2[1]);
