@@ -940,7 +940,9 @@ static void pick_pipeline(int sub_bytes, int nkb, int nt, int ep_bytes, int* kpb
 // (0: not used).  map_y: y as a [M][coff + Cout] matrix with row pitch ldc; map_r: the residual as [M][Cout]; boxes of
 // 128 rows x 64 columns, 128-byte swizzle.
 static int tma_epilogue_bytes(const ConvParams& p, bool pair_or_wide, CUtensorMap* map_y, CUtensorMap* map_r) {
-    if (tunable("DR_TMA_STORE_EP", 1) == 0 || pair_or_wide) return 0;
+    const int ep_pref = tunable("DR_TMA_STORE_EP", 1);          // 0: never, 1: where it pays, 2: wherever the shape allows
+    if (ep_pref == 0 || pair_or_wide) return 0;
+    if (ep_pref == 1 && p.m_tiles < num_sms()) return 0;        // less than one tile per SM: latency matters, not store bandwidth
     if (p.flags & (DR_OUT_F32 | DR_LRN)) return 0;
     if ((p.flags & DR_RESIDUAL) && (p.flags & DR_RELU)) return 0;
     if ((p.Cout & 15) || p.Cout > T_BIAS_MAX || (p.ldc & 7) || (p.coff & 7) || p.Nt < 64) return 0;
@@ -948,7 +950,8 @@ static int tma_epilogue_bytes(const ConvParams& p, bool pair_or_wide, CUtensorMa
     const bool res = (p.flags & DR_RESIDUAL) != 0;
     // measured (ResNet-50 at batch 128, GoogLeNet at 256): a gain up to 4 k-blocks with a residual or with at least 256
     // output channels, up to 2 k-blocks otherwise; beyond that the lost pipeline stages cost more than the stores
-    if (res ? (nkb > 4 || (p.Nt & 63) || (p.Cout & 63)) : (nkb > 4 || (nkb > 2 && p.Cout < 256))) return 0;
+    if (res ? ((p.Nt & 63) || (p.Cout & 63)) : false) return 0;
+    if (ep_pref == 1 && (res ? nkb > 4 : (nkb > 4 || (nkb > 2 && p.Cout < 256)))) return 0;
     if (!load_encoders()) return 0;
     const cuuint32_t box[2] = {64, TILE_M};
     const cuuint32_t es[2] = {1, 1};

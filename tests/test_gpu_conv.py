@@ -281,3 +281,31 @@ def test_conv_degenerate_shapes(dr, O):
         got, _ = run_conv(dr, x, wf, bf, k, s, p, dr.DR_BIAS | dr.DR_RELU)
         ref, _ = oracle_slim_layer(O, x, wf, bf, k, s, p, dr.DR_BIAS | dr.DR_RELU, dr)
         assert_layer_close(got, O.round_bf16(ref), f"degenerate {shape}")
+
+
+@pytest.mark.parametrize("residual", [False, True])
+def test_tma_epilogue_tail_rows_and_channel_slice(dr, O, residual, monkeypatch):
+    """The shared-memory / TMA-store epilogue forced onto a small layer: a last tile with 41 of 128 rows (the tensor map
+    clips the rest), a 64 + 32 column split (the 32 go out through the direct stores), a channel slice of a wider
+    tensor (nothing outside it may be written), and the residual variant (boxes loaded by TMA, added in place)."""
+    monkeypatch.setenv("DR_TMA_STORE_EP", "2")
+    dr.dr_set_conv_path(dr.DR_PATH_UMMA_TMA)
+    B, H, W, Cin = 3, 9, 11, 64
+    Cout = 128 if residual else 96
+    x = S.normal(60, "x", (B, H, W, Cin)); w = S.he_normal(60, "w", Cout, 1, Cin); b = S.normal(60, "b", (Cout,), 0.1)
+    if residual:
+        r = S.normal(60, "r", (B, H, W, Cout))
+        flags = dr.DR_BIAS | dr.DR_RESIDUAL | dr.DR_RELU_AFTER_RESIDUAL
+        got, _ = run_conv(dr, x, w, b, 1, 1, 0, flags, residual=r, ldc=256, coff=64)
+        ref = O.relu(O.add(O.conv2d(x, w, b, 1, 0), r))
+    else:
+        got, _ = run_conv(dr, x, w, b, 1, 1, 0, dr.DR_BIAS | dr.DR_RELU, ldc=256, coff=64)
+        ref = O.relu(O.conv2d(x, w, b, 1, 0))
+    assert_layer_close(got, O.round_bf16(ref), "TMA epilogue")
+    monkeypatch.setenv("DR_TMA_STORE_EP", "0")
+    if residual:
+        got0, _ = run_conv(dr, x, w, b, 1, 1, 0, flags, residual=r, ldc=256, coff=64)
+    else:
+        got0, _ = run_conv(dr, x, w, b, 1, 1, 0, dr.DR_BIAS | dr.DR_RELU, ldc=256, coff=64)
+    assert np.array_equal(got, got0)                 # same arithmetic, one rounding: bit-identical to the direct stores
+    dr.dr_set_conv_path(dr.DR_PATH_AUTO)
