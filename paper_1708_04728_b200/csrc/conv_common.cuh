@@ -51,6 +51,9 @@ struct ConvParams {
     int patch;             // 0 linear, 1 patch
     int PH, PW;            // pooled tile extent in patch mode
     int tiles_h, tiles_w;  // pooled tiles per image
+    int overlap_prev;      // TMA kernel: 1 = the layer does not read what the kernel before it in the stream writes; it is
+                           // launched with programmatic serialization (its CTAs fill SMs that kernel has left) and waits
+                           // for that kernel only before it exits, so that whatever follows sees both complete
     int* sk_counters;      // split-K kernel only (nullptr: not available): DR_CONV_WS_COUNTER_BYTES of zeroed tile counters
     float* sk_scratch;     // and scratch for the partial tiles
     size_t sk_scratch_bytes;

@@ -606,6 +606,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
     __syncthreads();
     if (PAIR) cluster_sync_all();                               // both CTAs' barriers exist before any remote arrive
     tc_fence_after();
+    grid_launch_dependents();                                   // a kernel launched behind this one with programmatic serialization may be scheduled
     const uint32_t tmem = sh.tmem_base;
     volatile int* abort_flag = &sh.abort;
 
@@ -831,6 +832,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
         __syncthreads();
     }
     if (PAIR) cluster_sync_all();                               // neither CTA leaves while the other may still signal it
+    if (p.overlap_prev) grid_dependency_wait();                 // launched ahead of the previous kernel's end: do not finish before it has
     if (warp == 1) {
         if (PAIR) tmem_dealloc_pair(tmem, 2 * T_ACC_COLS);
         else tmem_dealloc(tmem, 2 * T_ACC_COLS);
@@ -988,9 +990,11 @@ static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUte
     int smem_bytes = stages * kpb * sub_bytes + ep_bytes + 1024;
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(T_THREADS); cfg.dynamicSmemBytes = (size_t)smem_bytes; cfg.stream = stream;
     cfg.attrs = attr; cfg.numAttrs = 1;
     if (!attr_set) {
@@ -1008,6 +1012,7 @@ static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUte
     const int pair_tiles = ((p.m_tiles + 1) / 2) * p.n_blocks;
     const int pairs = pair_tiles < max_clusters ? pair_tiles : max_clusters;
     cfg.gridDim = dim3(2 * pairs);
+    cfg.numAttrs = p.overlap_prev ? 2 : 1;
     cudaError_t e;
     if (wide) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 1, true>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
     else if (kpb == 4) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 4, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
@@ -1079,10 +1084,18 @@ int conv_umma_tma_launch(const ConvParams& p_in, cudaStream_t stream) {
     const int ep_off = ep_bytes ? stages * kpb * sub_bytes : 0;
     int smem_bytes = stages * kpb * sub_bytes + ep_bytes + 1024;
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
-    if (wide) conv_umma_tma_kernel<false, 1, true><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
-    else if (kpb == 4) conv_umma_tma_kernel<false, 4, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
-    else if (kpb == 2) conv_umma_tma_kernel<false, 2, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
-    else conv_umma_tma_kernel<false, 1, false><<<grid, T_THREADS, smem_bytes, stream>>>(p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(T_THREADS); cfg.dynamicSmemBytes = (size_t)smem_bytes; cfg.stream = stream;
+    cfg.attrs = attr; cfg.numAttrs = p.overlap_prev ? 1 : 0;
+    cudaError_t e;
+    if (wide) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<false, 1, true>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
+    else if (kpb == 4) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<false, 4, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
+    else if (kpb == 2) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<false, 2, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
+    else e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<false, 1, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return DR_ERR_CUDA; }
     count_launch();
     return launch_status();
 }

@@ -675,6 +675,41 @@ int dr_net_forward(dr_net* n, const void* x, void* workspace, float* logits, voi
                     }
                     break;
                 }
+                if (st == DR_OK && op.pair >= 0 && !op.group && !n->timing && op.path == DR_PATH_UMMA_TMA &&
+                    n->ops[op.pair].path == DR_PATH_UMMA_TMA && tunable("DR_NET_OVERLAP", 2) != 0) {
+                    // Large batch.  DR_NET_OVERLAP = 2 (default): this layer, then the merged 5x5 (which reads the same input),
+                    // then the 3x3 that reads this layer's output, launched so that its CTAs fill the SMs the merged 5x5's
+                    // last round of tiles leaves idle.  DR_NET_OVERLAP = 1: the merged 5x5 first and this short layer
+                    // behind it in that way (measured: 3.99 ms per step without, 3.91 with 1, 3.89 with 2).  The overlapped layer reads nothing the merged 5x5
+                    // writes and does not finish before it has.
+                    const Op& oa = n->ops[op.pair];
+                    const Op& oc = n->ops[op.chain];
+                    const int mode = tunable("DR_NET_OVERLAP", 2);
+                    ConvParams pa, pc;
+                    st = conv_make_params(&oa.cd, ti.B, ti.H, ti.W, in0, oa.w.resolve(n->raw, ws), (const float*)oa.b.resolve(n->raw, ws),
+                                          nullptr, (char*)tensor_ptr(n, oa.out, x, arena, logits), nullptr, &pa);
+                    if (st == DR_OK && mode == 2 && oc.path == DR_PATH_UMMA_TMA) {
+                        const Tensor& tc = n->T(oc.in0);
+                        st = conv_make_params(&oc.cd, tc.B, tc.H, tc.W, out, oc.w.resolve(n->raw, ws), (const float*)oc.b.resolve(n->raw, ws),
+                                              nullptr, (char*)tensor_ptr(n, oc.out, x, arena, logits), nullptr, &pc);
+                        if (st == DR_OK) st = conv_launch_path(p, op.path, s);
+                        if (st == DR_OK) st = conv_launch_path(pa, oa.path, s);
+                        if (st == DR_OK) {
+                            pc.overlap_prev = 1;
+                            st = conv_launch_path(pc, oc.path, s);
+                            n->done[op.pair] = 1;
+                            n->done[op.chain] = 1;
+                        }
+                        break;
+                    }
+                    if (st == DR_OK) st = conv_launch_path(pa, oa.path, s);
+                    if (st == DR_OK) {
+                        p.overlap_prev = 1;
+                        st = conv_launch_path(p, op.path, s);
+                        n->done[op.pair] = 1;
+                    }
+                    break;
+                }
                 if (st == DR_OK) {
                     set_splitk_scratch(n, op, (char*)workspace, &p);
                     st = conv_launch_path(p, op.path, s);
