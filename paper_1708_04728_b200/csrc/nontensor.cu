@@ -190,6 +190,43 @@ __global__ void maxpool_noarg_kernel(int B, int H, int W, int C8, int Ho, int Wo
         y[i] = m;
     }
 }
+// The 3x3 window unrolled: the nine loads go out together (taps outside the plane load a clamped, valid address and
+// are replaced by -inf afterwards), then the maxima.
+__global__ void maxpool3_noarg_kernel(int B, int H, int W, int C8, int Ho, int Wo, int s, int p, const uint4* __restrict__ x,
+                                      uint4* __restrict__ y) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see maxpool_noarg_kernel
+    const size_t total = (size_t)B * Ho * Wo * C8;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int c8 = (int)(i % C8);
+        size_t q = i / C8;
+        const int wo = (int)(q % Wo); q /= Wo;
+        const int ho = (int)(q % Ho);
+        const size_t n = q / Ho;
+        const int h0 = ho * s - p, w0 = wo * s - p;
+        uint4 v[9];
+        bool ok[9];
+#pragma unroll
+        for (int r = 0; r < 3; ++r)
+#pragma unroll
+            for (int t = 0; t < 3; ++t) {
+                const int hi = h0 + r, wi = w0 + t;
+                ok[3 * r + t] = hi >= 0 && hi < H && wi >= 0 && wi < W;
+                const int hc = min(max(hi, 0), H - 1), wc = min(max(wi, 0), W - 1);     // clamped: always a valid address
+                v[3 * r + t] = __ldg(x + ((n * H + hc) * W + wc) * C8 + c8);
+            }
+        uint4 m = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);       // -inf: padding never wins
+        __nv_bfloat162* mm = reinterpret_cast<__nv_bfloat162*>(&m);
+#pragma unroll
+        for (int d = 0; d < 9; ++d) {
+            const uint4 u = ok[d] ? v[d] : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+            const __nv_bfloat162* uu = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) mm[j] = __hmax2(mm[j], uu[j]);
+        }
+        y[i] = m;
+    }
+}
 __global__ void maxpool_scalar_kernel(int B, int H, int W, int C, int Ho, int Wo, int k, int s, int p,
                                       const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
                                       int32_t* __restrict__ argmax) {
@@ -294,6 +331,36 @@ __global__ void concat_scalar_kernel(size_t n, int C, int ldc, int coff, const _
 // ---------------------------------------------------------------- global average pool
 // One block per (image, 64-channel slab): threads split the plane, partial sums meet in shared
 // memory in a fixed order (deterministic).  blockDim = (64 channels / 2, PIXSPLIT).
+// For C a multiple of 8: one block per (image, slab of 32 x 8 channels), blockDim = (32, 8): a thread sums every 8th
+// position of its 8 channels with 16-byte loads; the eight partial sums meet in shared memory in a fixed order.
+__global__ void avgpool8_kernel(int HW, int C8, const uint4* __restrict__ x, uint4* __restrict__ y) {
+    __shared__ float part[8][32][9];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see maxpool_noarg_kernel
+    const int n = blockIdx.y, c8 = blockIdx.x * 32 + threadIdx.x;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (c8 < C8) {
+        for (int q = threadIdx.y; q < HW; q += 8) {
+            const uint4 v = __ldg(x + ((size_t)n * HW + q) * C8 + c8);
+            acc[0] += bf16_lo(v.x); acc[1] += bf16_hi(v.x); acc[2] += bf16_lo(v.y); acc[3] += bf16_hi(v.y);
+            acc[4] += bf16_lo(v.z); acc[5] += bf16_hi(v.z); acc[6] += bf16_lo(v.w); acc[7] += bf16_hi(v.w);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) part[threadIdx.y][threadIdx.x][j] = acc[j];
+    __syncthreads();
+    if (threadIdx.y == 0 && c8 < C8) {
+        float t[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            t[j] = 0.f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) t[j] += part[k][threadIdx.x][j];
+            t[j] = t[j] / (float)HW;
+        }
+        y[(size_t)n * C8 + c8] = make_uint4(pack_bf16(t[0], t[1]), pack_bf16(t[2], t[3]), pack_bf16(t[4], t[5]), pack_bf16(t[6], t[7]));
+    }
+}
+
 constexpr int AVG_SPLIT = 8;
 __global__ void avgpool_kernel(int HW, int C, const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y) {
     __shared__ float part[AVG_SPLIT][64];
@@ -538,7 +605,9 @@ int dr_maxpool(int B, int H, int W, int C, int k, int s, int p, const void* x, v
     const size_t n = (size_t)B * Ho * Wo * C;
     if (n == 0) return DR_OK;
     DR_REQUIRE(aligned16(x) && aligned16(y) && (!argmax || aligned16(argmax)), DR_ERR_ALIGNMENT);
-    if (C % 8 == 0 && !argmax)
+    if (C % 8 == 0 && !argmax && k == 3)
+        maxpool3_noarg_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C / 8, Ho, Wo, s, p, (const uint4*)x, (uint4*)y);
+    else if (C % 8 == 0 && !argmax)
         maxpool_noarg_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C / 8, Ho, Wo, k, s, p, (const uint4*)x, (uint4*)y);
     else if (C % 8 == 0)
         maxpool_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C / 8, Ho, Wo, k, s, p, (const uint4*)x, (uint4*)y, argmax);
@@ -580,6 +649,12 @@ int dr_avgpool_global(int B, int H, int W, int C, const void* x, void* y, void* 
     if (B == 0) return DR_OK;
     DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
     DR_REQUIRE(C % 2 == 0, DR_ERR_UNSUPPORTED);
+    if (C % 8 == 0) {
+        dim3 grid((C / 8 + 31) / 32, B), block(32, 8);
+        avgpool8_kernel<<<grid, block, 0, (cudaStream_t)stream>>>(H * W, C / 8, (const uint4*)x, (uint4*)y);
+        count_launch();
+        return launch_status();
+    }
     dim3 grid((C + 63) / 64, B), block(32, AVG_SPLIT);
     avgpool_kernel<<<grid, block, 0, (cudaStream_t)stream>>>(H * W, C, (const __nv_bfloat16*)x, (__nv_bfloat16*)y);
     count_launch();
