@@ -191,6 +191,49 @@ def run_layer(args):
                       "gflop": flops * 1e-9, "mbytes": nbytes * 1e-6, "path": dr.PATH_NAMES[dr.dr_last_conv_path()]}))
 
 
+def run_nontensor(args):
+    """Achieved HBM bandwidth of the stand-alone non-tensor kernels (the layers of the unslimmed baseline) on the tensors
+    they meet in GoogLeNet / ResNet-50 at the bench batch: algorithmic bytes (read + write of the tensor; pooling
+    1 + 1/4) over the CUDA-event time, against the measured copy bandwidth.  L2 flushed before every launch."""
+    import torch
+    import __graft_entry__
+    __graft_entry__.build_cuda()
+    import paper_1708_04728_b200 as dr
+    B = args.batch
+    pk, pk_kind = peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    mk = lambda *shape: torch.randn(*shape, device="cuda").to(torch.bfloat16)
+    vec = lambda c: torch.rand(c, device="cuda") + 0.5
+    cases = []
+    x1 = mk(B, 112, 112, 64); y1 = torch.empty_like(x1)                      # conv1 output of GoogLeNet / ResNet-50
+    cases.append(("relu 112x112x64", 2 * x1.numel() * 2, lambda: dr.dr_relu(x1.numel(), x1, y1)))
+    bn = [vec(64) for _ in range(4)]
+    cases.append(("bn+scale 112x112x64", 2 * x1.numel() * 2,
+                  lambda: dr.dr_bn(B, 112, 112, 64, x1, bn[0], bn[1], 1.0, 1e-5, bn[2], bn[3], y1)))
+    yp = torch.empty((B, 56, 56, 64), dtype=torch.bfloat16, device="cuda")
+    cases.append(("maxpool 3x3/2 112x112x64", (x1.numel() + yp.numel()) * 2, lambda: dr.dr_maxpool(B, 112, 112, 64, 3, 2, 1, x1, yp)))
+    x2 = mk(B, 56, 56, 192); y2 = torch.empty_like(x2)                       # conv2 output of GoogLeNet
+    cases.append(("lrn 56x56x192", 2 * x2.numel() * 2, lambda: dr.dr_lrn(B, 56, 56, 192, 5, 1e-4, 0.75, 1.0, x2, y2)))
+    x3 = mk(B, 56, 56, 256); r3 = mk(B, 56, 56, 256); y3 = torch.empty_like(x3)   # res2 block output of ResNet-50
+    cases.append(("add 56x56x256", 3 * x3.numel() * 2, lambda: dr.dr_add(x3.numel(), x3, r3, y3)))
+    x4 = mk(B, 28, 28, 480); y4 = torch.empty((B, 14, 14, 480), dtype=torch.bfloat16, device="cuda")
+    cases.append(("maxpool 3x3/2 28x28x480", (x4.numel() + y4.numel()) * 2, lambda: dr.dr_maxpool(B, 28, 28, 480, 3, 2, 1, x4, y4)))
+    x5 = mk(B, 7, 7, 1024); y5 = torch.empty((B, 1, 1, 1024), dtype=torch.bfloat16, device="cuda")
+    cases.append(("avgpool 7x7x1024", (x5.numel() + y5.numel()) * 2, lambda: dr.dr_avgpool_global(B, 7, 7, 1024, x5, y5)))
+    rows = []
+    for name, nbytes, fn in cases:
+        ts = []
+        for i in range(args.warmup + min(args.steps, 20)):
+            flush.zero_()
+            a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); e.record(); torch.cuda.synchronize()
+            if i >= args.warmup:
+                ts.append(a.elapsed_time(e) * 1e3)
+        us = statistics.median(ts)
+        rows.append({"kernel": name, "us": us, "mbytes": nbytes / 1e6, "gbs": nbytes / us * 1e-3, "frac": nbytes / us * 1e-3 / pk["hbm_gbs"]})
+    print(json.dumps({"batch": B, "peak_gbs": pk["hbm_gbs"], "peak_kind": pk_kind, "kernels": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -205,6 +248,7 @@ def main():
     ap.add_argument("--layer", default=None,
                     help="time ONE slim layer of the network (e.g. conv1, conv2, 3b.m5, 4e.3x3) instead of the whole step; "
                          "this is the small case the ncu captures under profiles/ run")
+    ap.add_argument("--nontensor", action="store_true", help="achieved HBM GB/s of the stand-alone non-tensor kernels")
     args = ap.parse_args()
     if args.batch is None:
         args.batch = 256 if args.arch in ("googlenet", "googlenet_streamline", "alexnet") else 128
@@ -212,6 +256,8 @@ def main():
         return run_reference(args)
     if args.layer:
         return run_layer(args)
+    if args.nontensor:
+        return run_nontensor(args)
 
     import numpy as np
     import torch

@@ -43,8 +43,8 @@ __device__ __forceinline__ float bf16_to_float(const __nv_bfloat16 v) { return _
 // scale^(-beta) for LRN; beta = 0.75 (the usual value) avoids the general pow.
 __device__ __forceinline__ float lrn_pow(float s, float beta) {
     if (beta == 0.75f) {
-        const float r = rsqrtf(s);
-        return r * sqrtf(r);
+        const float r = rsqrtf(s);              // s^(-1/2)
+        return r * (r * rsqrtf(r));             // s^(-1/2) * sqrt(s^(-1/2)), sqrt(r) = r * rsqrt(r): no correctly-rounded sqrt sequence
     }
     return exp2f(-beta * log2f(s));
 }
