@@ -66,6 +66,8 @@ struct EmbedJob { int w_small; int Cout, Cin, ks, kb, joff; size_t w_off; };
 struct CopyJob { int src; size_t dst_off; size_t bytes; };
 struct S2dJob { int w; int Cout, k, C, s, Cp; size_t w_off; };
 struct GroupJob { int w_grouped; int Cout, Cin_g, k, groups; size_t w_off; };
+// Zero-padded copy of a parameter: `rows` rows of `row_bytes` placed `pitch` bytes apart in a zeroed block of `total`.
+struct PadJob { int src; size_t dst_off, total, rows, row_bytes, pitch; };
 
 }  // namespace dr
 
@@ -82,6 +84,7 @@ struct dr_net {
     std::vector<CopyJob> copies;
     std::vector<GroupJob> group_jobs;
     std::vector<S2dJob> s2d_jobs;
+    std::vector<PadJob> pad_jobs;
     size_t param_bytes = 0, act_bytes = 0;
     size_t sk_scratch_bytes = 0;   // split-K scratch shared by all layers (they run one after another), after the arena
     int n_conv = 0;                // each convolution has its own block of tile counters after that
@@ -322,15 +325,38 @@ static void build_googlenet_paper(dr_net* n) {
         *w = rawref(n->filt(name, cout, k, cin));
         *b = rawref(n->vec(name + ".b", cout));
     };
-    auto cr = [&](const std::string& name, int in, int k, int pad, int cout, int out = -2, int coff = 0) {
+    // `cin` is the layer's own input width; the tensor `in` may carry more channels (zeros, see `reducer`), in which
+    // case the filters get zero taps for them.  `cpad` > cout adds output channels with zero filters and zero bias,
+    // which stay zero through the ReLU.  Work and bytes are counted for the layer as the paper defines it.
+    auto cr = [&](const std::string& name, int in, int cin, int k, int pad, int cout, int cpad, int out = -2, int coff = 0) {
         PRef w, b;
-        conv_p(name, cout, k, n->T(in).C, &w, &b);
-        if (slim) return add_conv(n, name, in, k, 1, pad, cout, BR, w, b, out, coff);
-        const int t = add_conv(n, name + ".conv", in, k, 1, pad, cout, DR_BIAS, w, b);
-        const int r = add_simple(n, OP_RELU, name, t);
-        if (out != -2) { add_concat(n, name + ".cat", r, out, coff); return out; }
+        conv_p(name, cout, k, cin, &w, &b);
+        const int cin_t = n->T(in).C;
+        if (cin_t != cin || cpad != cout) {
+            const size_t wo = n->ws_alloc((size_t)cpad * k * k * cin_t * 2), bo = n->ws_alloc((size_t)cpad * 4);
+            n->pad_jobs.push_back({w.raw, wo, (size_t)cpad * k * k * cin_t * 2, (size_t)cout * k * k, (size_t)cin * 2, (size_t)cin_t * 2});
+            n->pad_jobs.push_back({b.raw, bo, (size_t)cpad * 4, 1, (size_t)cout * 4, (size_t)cpad * 4});
+            w = wsref(wo); b = wsref(bo);
+        }
+        const size_t first = n->ops.size();
+        int r;
+        if (slim) {
+            r = add_conv(n, name, in, k, 1, pad, cpad, BR, w, b, out, coff);
+        } else {
+            const int t = add_conv(n, name + ".conv", in, k, 1, pad, cpad, DR_BIAS, w, b);
+            r = add_simple(n, OP_RELU, name, t);
+            if (out != -2) { add_concat(n, name + ".cat", r, out, coff); r = out; }
+        }
+        Op& c = n->ops[first];
+        const Tensor& ti = n->T(in);
+        const double M = (double)ti.B * ti.H * ti.W;
+        c.flops = 2.0 * M * cout * k * k * cin;
+        c.bytes = M * cin * 2 + (double)cout * k * k * cin * 2 + M * cout * 2 + cout * 4.0;
         return r;
     };
+    // Reducers feed a spatial convolution whose tensor-core kernel takes input channels in blocks of 64: their
+    // output tensor is rounded up to that, the extra channels zero.
+    auto pad64 = [](int c) { return (c + 63) / 64 * 64; };
     PRef w, b;
     int t;
     conv_p("conv1", 64, 7, 3, &w, &b);
@@ -342,7 +368,7 @@ static void build_googlenet_paper(dr_net* n) {
         t = add_simple(n, OP_MAXPOOL, "conv1.pool", t);
         t = add_simple(n, OP_LRN, "conv1", t);
     }
-    t = cr("conv2r", t, 1, 0, 64);
+    t = cr("conv2r", t, 64, 1, 0, 64, 64);
     conv_p("conv2", 192, 3, 64, &w, &b);
     if (slim) {
         t = add_conv(n, "conv2", t, 3, 1, 1, 192, BR | DR_POOL | DR_LRN | DR_LRN_BEFORE_POOL, w, b);
@@ -357,10 +383,10 @@ static void build_googlenet_paper(dr_net* n) {
         const Tensor ti = n->T(t);
         const int a3 = m.c3 + m.c1, a5 = m.c5 + m.pp;
         const int out = n->tensor(ti.B, ti.H, ti.W, a3 + a5);
-        const int r3 = cr(mn + ".p3r", t, 1, 0, m.c3r / 2);
-        cr(mn + ".p3", r3, 3, 1, a3, out, 0);
-        const int r5 = cr(mn + ".p5r", t, 1, 0, m.c5r);
-        cr(mn + ".p5", r5, 5, 2, a5, out, a3);
+        const int r3 = cr(mn + ".p3r", t, ti.C, 1, 0, m.c3r / 2, pad64(m.c3r / 2));
+        cr(mn + ".p3", r3, m.c3r / 2, 3, 1, a3, a3, out, 0);
+        const int r5 = cr(mn + ".p5r", t, ti.C, 1, 0, m.c5r, pad64(m.c5r));
+        cr(mn + ".p5", r5, m.c5r, 5, 2, a5, a5, out, a3);
         t = out;
         if (mn == "3b") t = add_simple(n, OP_MAXPOOL, "pool3", t);
         if (mn == "4e") t = add_simple(n, OP_MAXPOOL, "pool4", t);
@@ -585,6 +611,12 @@ int dr_net_prepare(dr_net* n, void* workspace, void* stream) {
     for (const GroupJob& g : n->group_jobs) {
         const int st = dr_embed_groups(g.Cout, g.Cin_g, g.k, g.groups, n->raw[g.w_grouped], ws + g.w_off, stream);
         if (st != DR_OK) return st;
+    }
+    for (const PadJob& j : n->pad_jobs) {
+        if (cudaMemsetAsync(ws + j.dst_off, 0, j.total, s) != cudaSuccess) return DR_ERR_CUDA;
+        if (cudaMemcpy2DAsync(ws + j.dst_off, j.pitch, n->raw[j.src], j.row_bytes, j.row_bytes, j.rows, cudaMemcpyDeviceToDevice, s) !=
+            cudaSuccess)
+            return DR_ERR_CUDA;
     }
     for (const CopyJob& c : n->copies)
         if (cudaMemcpyAsync(ws + c.dst_off, n->raw[c.src], c.bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return DR_ERR_CUDA;

@@ -143,7 +143,11 @@ def test_googlenet_paper_form_layer_list(dr):
     infos = {net.dr_net_layer_info(i)["name"]: net.dr_net_layer_info(i) for i in range(net.dr_net_num_layers())}
     assert net.dr_net_num_layers() == 3 + 9 * 4 + 2 + 1 + 1
     # the numbers Section 3.2 gives for inception_3a: reducer 96 -> 48, 3x3 128 -> 192, 5x5 32 -> 64
-    assert infos["3a.p3r"]["dims"] == (1, 28, 28, 48)
+    # the 48-channel reducer is stored in a 64-channel tensor (the rest zeros: the 3x3 kernel reads channels in 64s);
+    # its work is counted for 48 channels, and so is the 3x3's
+    assert infos["3a.p3r"]["dims"] == (1, 28, 28, 64)
+    assert infos["3a.p3r"]["flops"] == 2.0 * 784 * 48 * 192 and infos["3a.p3"]["flops"] == 2.0 * 784 * 192 * 9 * 48
+    assert infos["3a.p5r"]["dims"] == (1, 28, 28, 64) and infos["3a.p5"]["flops"] == 2.0 * 784 * 64 * 25 * 16
     assert infos["3a.p3"]["dims"] == (1, 28, 28, 192) and (infos["3a.p3"]["ldc"], infos["3a.p3"]["coff"]) == (256, 0)
     assert infos["3a.p5"]["dims"] == (1, 28, 28, 64) and (infos["3a.p5"]["ldc"], infos["3a.p5"]["coff"]) == (256, 192)
     assert infos["5b.p5"]["ldc"] == 1024

@@ -69,11 +69,18 @@ def check_network(dr, arch, B, entries, steps_fn, params, per_layer_tol=None, hw
     steps = steps_fn(params)
     # ---- per layer, teacher-forced, batch entry 0 (+ all checked entries for the logits)
     G = layer_outputs(net, logits, entries[:1])
+    x0 = images(entries[:1])
+    if arch == dr.DR_ARCH_GOOGLENET_PAPER:
+        # reducers are stored in tensors rounded up to 64 channels: the extra channels must be exactly zero
+        widths = {k: v.shape[-1] for k, v in N.run(steps, x0).items()}
+        for name, c in widths.items():
+            if name in G and G[name].shape[-1] > c:
+                assert not np.any(G[name][..., c:]), f"{name}: padded channels are not zero"
+                G[name] = G[name][..., :c]
     given = dict(G)
     for st in steps:                      # concatenated module outputs are re-assembled from their slices
         if st.virtual:
             given[st.name] = np.concatenate([given[s] for s in st.src], axis=-1)
-    x0 = images(entries[:1])
     forced = N.run(steps, x0, given=given)
     report = []
     for st in steps:
