@@ -142,8 +142,8 @@ def test_steps_recover_a_realisable_teacher():
     w, b = np.zeros_like(wt), np.zeros(2)
     vw, vb = np.zeros_like(w), np.zeros(2)
     losses = []
-    for _ in range(300):
-        w, b, vw, vb, loss, _, _ = F.regression_step(x, yt, w, b, vw, vb, lr=0.02, momentum=0.5, relu=False)
+    for _ in range(600):
+        w, b, vw, vb, loss, _, _ = F.regression_step(x, yt, w, b, vw, vb, lr=0.05, momentum=0.0, relu=False)
         losses.append(loss)
     assert losses[-1] < 1e-10 * losses[0] and all(b_ <= a_ for a_, b_ in zip(losses[5:], losses[6:]) if a_ > 1e-20 * losses[0])
     np.testing.assert_allclose(w, wt, atol=1e-5); np.testing.assert_allclose(b, bt, atol=1e-5)
