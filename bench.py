@@ -234,6 +234,63 @@ def run_nontensor(args):
     print(json.dumps({"batch": B, "peak_gbs": pk["hbm_gbs"], "peak_kind": pk_kind, "kernels": rows}))
 
 
+def run_finetune(args):
+    """One SGD step of the layer-wise regression of a slim layer (Section 3.1, Eq. (w_b)) on layers the method re-learns in
+    GoogLeNet, at the bench batch: forward, gradient of the Euclidean loss, filter gradient on the tensor cores, update.
+    Reports the step time, and the filter-gradient kernel alone against the measured bf16 peak (2 M N K FLOPs)."""
+    import torch
+    import __graft_entry__
+    __graft_entry__.build_cuda()
+    import paper_1708_04728_b200 as dr
+    B = args.batch
+    pk, pk_kind = peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    layers = [("streamline conv2 3x3/2 64->192 @56", 56, 64, 192, 3, 2, 1),
+              ("paper-form 3a.p3 3x3 64->192 @28", 28, 64, 192, 3, 1, 1),
+              ("merged 3a.m5 5x5 192->128 @28", 28, 192, 128, 5, 1, 2),
+              ("merged 4e.m5 5x5 528->512 @14", 14, 528, 512, 5, 1, 2)]
+    rows = []
+    for name, hw, cin, cout, k, s, p in layers:
+        d = dr.dr_conv_desc(k=k, stride=s, pad=p, Cin=cin, Cout=cout, flags=dr.DR_BIAS | dr.DR_RELU, pool_k=3, pool_stride=2, pool_pad=1,
+                            lrn_size=5, lrn_alpha=1e-4, lrn_beta=0.75, lrn_k=1.0, y_ldc=0, y_coff=0)
+        ho = (hw + 2 * p - k) // s + 1
+        x = torch.randn(B, hw, hw, cin, device="cuda").to(torch.bfloat16)
+        yt = torch.randn(B, ho, ho, cout, device="cuda").abs().to(torch.bfloat16)
+        w = torch.randn(cout, k, k, cin, device="cuda") * (2.0 / (k * k * cin)) ** 0.5
+        shadow = w.to(torch.bfloat16)
+        b = torch.zeros(cout, device="cuda")
+        vw, vb = torch.zeros_like(w), torch.zeros_like(b)
+        y = torch.empty_like(yt); dz = torch.empty_like(yt)
+        dw = torch.empty_like(w); db = torch.empty_like(b)
+        loss = torch.zeros(1, device="cuda")
+        need = dr.dr_regress_step_workspace_bytes(d, B, hw, hw)
+        ws = torch.zeros(need + 256, dtype=torch.uint8, device="cuda")
+        ws = ws[(-ws.data_ptr()) % 256:]
+        wg_need = dr.dr_conv_wgrad_workspace_bytes(d, B, hw, hw)
+        step = lambda: dr.dr_regress_step(d, B, hw, hw, x, yt, w, b, vw, vb, shadow, 1e-6, 0.9, 1e-4, y, dz, dw, db, loss, ws, ws.numel())
+        wgrad = lambda: dr.dr_conv_wgrad(d, B, hw, hw, x, dz, dw, ws, wg_need)
+        fwd = lambda: dr.dr_conv_slim_ws(d, B, hw, hw, x, shadow, b, None, y, None, None, 0)
+        t = {}
+        for what, fn in (("step", step), ("wgrad", wgrad), ("forward", fwd)):
+            ts = []
+            for i in range(args.warmup + min(args.steps, 20)):
+                flush.zero_()
+                a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); e.record(); torch.cuda.synchronize()
+                if i >= args.warmup:
+                    ts.append(a.elapsed_time(e) * 1e3)
+            t[what] = statistics.median(ts)
+        st, info = dr.dr_device_status()
+        assert st == 0, (st, info)
+        flops = 2.0 * B * ho * ho * cout * k * k * cin
+        rows.append({"layer": name, "step_us": t["step"], "forward_us": t["forward"], "wgrad_us": t["wgrad"],
+                     "images_per_s": B / t["step"] * 1e6, "wgrad_tflops": flops / t["wgrad"] * 1e-6,
+                     "wgrad_frac": flops / t["wgrad"] * 1e-6 / pk["bf16_tflops"], "forward_tflops": flops / t["forward"] * 1e-6,
+                     "loss": float(loss)})
+    print(json.dumps({"metric": "layer-wise regression step of a slim layer", "batch": B, "peak_tflops": pk["bf16_tflops"], "peak_kind": pk_kind,
+                      "l2": "flushed before every timed call", "layers": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -249,6 +306,7 @@ def main():
                     help="time ONE slim layer of the network (e.g. conv1, conv2, 3b.m5, 4e.3x3) instead of the whole step; "
                          "this is the small case the ncu captures under profiles/ run")
     ap.add_argument("--nontensor", action="store_true", help="achieved HBM GB/s of the stand-alone non-tensor kernels")
+    ap.add_argument("--finetune", action="store_true", help="time one SGD step of the layer-wise regression of a slim layer (Eq. (w_b))")
     args = ap.parse_args()
     if args.batch is None:
         args.batch = 256 if args.arch in ("googlenet", "googlenet_streamline", "alexnet") else 128
@@ -258,6 +316,8 @@ def main():
         return run_layer(args)
     if args.nontensor:
         return run_nontensor(args)
+    if args.finetune:
+        return run_finetune(args)
 
     import numpy as np
     import torch

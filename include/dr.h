@@ -291,6 +291,51 @@ int dr_device_status(int info[4]);
  * (1 .. 2e9), on a barrier nothing arrives on, and then leaves the same record a convolution kernel would.
  * dr_device_status() afterwards returns DR_ERR_DEVICE_TIMEOUT with info[1] = 99; the context stays usable. */
 int dr_selftest_wait_timeout(long long limit_cycles, void* stream);
+/* ---- layer-wise regression of a slim layer (Section 3.1, Eq. (w_b) and Lemma 1) -------------------------
+ * The slim layer f~(W, b; X) = ReLU(conv(X; W) + b) is re-learned from pairs (X, Y_CNN) of the input and the
+ * output feature map of the layer group it replaces, by SGD on L = 1/(2B) * sum_i ||Y_CNN^i - f~(W, b; X^i)||_F^2
+ * over mini-batches of B images.  The paper fixes neither the constant in front of the sum nor the form of the
+ * update; the constant is the Euclidean loss's 1/(2B), the update is
+ *     v <- momentum * v + lr * (g + decay * w);   w <- w - v.
+ * One step = dr_conv_slim (forward, Y) -> dr_regress_grad -> dr_conv_wgrad -> dr_sgd_update (filters, bias);
+ * dr_regress_step runs exactly that sequence.  All device buffers are the caller's; nothing is allocated.      */
+
+/* dZ = dL/dZ for Y = ReLU(Z): (Y - Y_CNN) / B where Y > 0 (everywhere when relu == 0), rounded to bfloat16;
+ * db[c] = sum over pixels of that (rounded) dZ; *loss = 1/(2B) * sum (Y - Y_CNN)^2 (loss may be NULL).
+ *  y, yt, dz: dense [B,H,W,C] bfloat16 (dz may not alias y or yt), C a multiple of 8 and <= 2048; db: float32 [C].
+ *  workspace: dr_regress_workspace_bytes(C) bytes, 256-byte aligned.  Sums are taken in a fixed order.
+ * Errors: INVALID_ARG, UNSUPPORTED (C), ALIGNMENT, WORKSPACE.                                                   */
+int dr_regress_workspace_bytes(int C, size_t* bytes);
+int dr_regress_grad(int B, int H, int W, int C, const void* y, const void* yt, int relu, void* dz, float* db,
+                    float* loss, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Filter gradient of the convolution of `desc` (k, stride, pad, Cin, Cout; flags and y_ldc are not looked at):
+ *   dw[j][r][s][c] = sum over (n, ho, wo) of dz[n][ho][wo][j] * x[n][ho*stride - pad + r][wo*stride - pad + s][c]
+ * with x zero outside the image.  x: [B,H,W,Cin] dense bfloat16; dz: [B,Ho,Wo,Cout] dense bfloat16;
+ * dw: float32 [Cout][k][k][Cin], overwritten.  Products are exact, sums float32 on the tensor cores; the pixel
+ * range is cut into pieces whose partial sums (in `workspace`) are added in a fixed order.
+ * Restrictions: Cin >= 64, Cin and Cout multiples of 8 (else DR_ERR_UNSUPPORTED).
+ * workspace: dr_conv_wgrad_workspace_bytes bytes, 256-byte aligned.  Errors: INVALID_ARG, ALIGNMENT, WORKSPACE. */
+int dr_conv_wgrad_workspace_bytes(const dr_conv_desc* desc, int B, int H, int W, size_t* bytes);
+int dr_conv_wgrad(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* dz, float* dw,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* v <- momentum * v + lr * (g + decay * w);  w <- w - v  over n float32 elements, in place; w_bf16 (NULL or n
+ * bfloat16) receives the updated w rounded to nearest even, the copy the next forward pass reads.             */
+int dr_sgd_update(size_t n, float* w, float* v, const float* g, float lr, float momentum, float decay,
+                  void* w_bf16, void* stream);
+
+/* One whole step on a mini-batch.  desc: the slim layer (DR_BIAS required; DR_RELU optional; no pooling, LRN,
+ * residual, float32 output or channel slice).  x: [B,H,W,Cin]; yt: Y_CNN, [B,Ho,Wo,Cout]; w, b: float32 master
+ * parameters, vw, vb: their momentum buffers, w_bf16: the bfloat16 filters the forward pass reads (all updated);
+ * y, dz: [B,Ho,Wo,Cout] bfloat16 scratch (y holds the forward output of the parameters before the update);
+ * dw: float32 [Cout][k][k][Cin] and db: float32 [Cout] receive the gradients; *loss the loss before the update.
+ * The bias takes no weight decay.  workspace: dr_regress_step_workspace_bytes bytes, 256-byte aligned.         */
+int dr_regress_step_workspace_bytes(const dr_conv_desc* desc, int B, int H, int W, size_t* bytes);
+int dr_regress_step(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* yt, float* w, float* b,
+                    float* vw, float* vb, void* w_bf16, float lr, float momentum, float decay, void* y, void* dz,
+                    float* dw, float* db, float* loss, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Kernels of this library launched by this process so far. */
 long long dr_launch_count(void);
 

@@ -71,6 +71,13 @@ _SIGS = {
     "dr_space_to_depth": (_I, [_I, _I, _I, _I, _I, _I, _I, _I, _P, _P, _P]),
     "dr_s2d_filter": (_I, [_I, _I, _I, _I, _I, _P, _P, _P]),
     "dr_conv_slim": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P]),
+    "dr_regress_workspace_bytes": (_I, [_I, C.POINTER(_Z)]),
+    "dr_regress_grad": (_I, [_I, _I, _I, _I, _P, _P, _I, _P, _P, _P, _P, _Z, _P]),
+    "dr_conv_wgrad_workspace_bytes": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, C.POINTER(_Z)]),
+    "dr_conv_wgrad": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _Z, _P]),
+    "dr_sgd_update": (_I, [_Z, _P, _P, _P, _F, _F, _F, _P, _P]),
+    "dr_regress_step_workspace_bytes": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, C.POINTER(_Z)]),
+    "dr_regress_step": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _F, _F, _F, _P, _P, _P, _P, _P, _P, _Z, _P]),
     "dr_conv_workspace_bytes": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, C.POINTER(_Z)]),
     "dr_conv_slim_ws": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _Z, _P]),
     "dr_inception_workspace_bytes": (_I, [C.POINTER(dr_inception_desc), _I, _I, _I, C.POINTER(_Z)]),
@@ -160,6 +167,45 @@ def dr_s2d_filter(Cout, k, Cc, s, Cp, w, w_out, stream=None):
 def dr_conv_slim(desc, B, H, W, x, w, b, residual, y, argmax=None, stream=None):
     _check(_lib.dr_conv_slim(C.byref(desc), B, H, W, _ptr(x), _ptr(w), _ptr(b), _ptr(residual), _ptr(y), _ptr(argmax),
                              _stream(stream)), "dr_conv_slim")
+
+
+def dr_regress_workspace_bytes(Cc) -> int:
+    n = _Z(0)
+    _check(_lib.dr_regress_workspace_bytes(Cc, C.byref(n)), "dr_regress_workspace_bytes")
+    return n.value
+
+
+def dr_regress_grad(B, H, W, Cc, y, yt, relu, dz, db, loss, workspace, workspace_bytes, stream=None):
+    _check(_lib.dr_regress_grad(B, H, W, Cc, _ptr(y), _ptr(yt), int(relu), _ptr(dz), _ptr(db), _ptr(loss), _ptr(workspace),
+                                workspace_bytes, _stream(stream)), "dr_regress_grad")
+
+
+def dr_conv_wgrad_workspace_bytes(desc, B, H, W) -> int:
+    n = _Z(0)
+    _check(_lib.dr_conv_wgrad_workspace_bytes(C.byref(desc), B, H, W, C.byref(n)), "dr_conv_wgrad_workspace_bytes")
+    return n.value
+
+
+def dr_conv_wgrad(desc, B, H, W, x, dz, dw, workspace, workspace_bytes, stream=None):
+    _check(_lib.dr_conv_wgrad(C.byref(desc), B, H, W, _ptr(x), _ptr(dz), _ptr(dw), _ptr(workspace), workspace_bytes,
+                              _stream(stream)), "dr_conv_wgrad")
+
+
+def dr_sgd_update(n, w, v, g, lr, momentum, decay, w_bf16=None, stream=None):
+    _check(_lib.dr_sgd_update(n, _ptr(w), _ptr(v), _ptr(g), lr, momentum, decay, _ptr(w_bf16), _stream(stream)), "dr_sgd_update")
+
+
+def dr_regress_step_workspace_bytes(desc, B, H, W) -> int:
+    n = _Z(0)
+    _check(_lib.dr_regress_step_workspace_bytes(C.byref(desc), B, H, W, C.byref(n)), "dr_regress_step_workspace_bytes")
+    return n.value
+
+
+def dr_regress_step(desc, B, H, W, x, yt, w, b, vw, vb, w_bf16, lr, momentum, decay, y, dz, dw, db, loss, workspace,
+                    workspace_bytes, stream=None):
+    _check(_lib.dr_regress_step(C.byref(desc), B, H, W, _ptr(x), _ptr(yt), _ptr(w), _ptr(b), _ptr(vw), _ptr(vb), _ptr(w_bf16),
+                                lr, momentum, decay, _ptr(y), _ptr(dz), _ptr(dw), _ptr(db), _ptr(loss), _ptr(workspace),
+                                workspace_bytes, _stream(stream)), "dr_regress_step")
 
 
 def dr_conv_workspace_bytes(desc, B, H, W) -> int:

@@ -866,6 +866,32 @@ static bool load_encoders() {
 // otherwise (*a_mode = 1: 128 output pixels x 64 channels of one filter tap per load).  B: the filters as
 // (Cin, taps, Cout) with boxes of 64 channels x 1 tap x b_box_rows filters.
 int encode_conv_maps(const ConvParams& p, int b_box_rows, CUtensorMap* map_a, CUtensorMap* map_b, int* a_mode) {
+    const int st = encode_input_map(p, map_a, a_mode);
+    if (st != DR_OK) return st;
+    const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
+    const cuuint64_t strides[2] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.K * 2};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)b_box_rows};
+    const cuuint32_t es[3] = {1, 1, 1};
+    if (g_encode_tiled(map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)p.w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return DR_ERR_CUDA;
+    return DR_OK;
+}
+
+// A [rows][cols] bf16 matrix with row pitch ld (elements) in boxes of 128 rows x 64 columns, 128-byte swizzle.
+int encode_rows_map(const void* ptr, long long rows, int cols, int ld, CUtensorMap* map) {
+    if (!load_encoders()) return DR_ERR_CUDA;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {64, TILE_M};
+    const cuuint32_t es[2] = {1, 1};
+    return g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)ptr, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS
+               ? DR_OK : DR_ERR_CUDA;
+}
+
+// The input-side map alone (see encode_conv_maps).
+int encode_input_map(const ConvParams& p, CUtensorMap* map_a, int* a_mode) {
     if (!load_encoders()) return DR_ERR_CUDA;
     *a_mode = (p.k == 1 && p.stride == 1 && p.pad == 0) ? 0 : 1;
     if (*a_mode == 0) {
@@ -888,13 +914,6 @@ int encode_conv_maps(const ConvParams& p, int b_box_rows, CUtensorMap* map_a, CU
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return DR_ERR_CUDA;
     }
-    const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
-    const cuuint64_t strides[2] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.K * 2};
-    const cuuint32_t box[3] = {64, 1, (cuuint32_t)b_box_rows};
-    const cuuint32_t es[3] = {1, 1, 1};
-    if (g_encode_tiled(map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)p.w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return DR_ERR_CUDA;
     return DR_OK;
 }
 

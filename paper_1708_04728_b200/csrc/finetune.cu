@@ -1,0 +1,441 @@
+// One SGD step of the layer-wise regression that re-learns a slim layer (Section 3.1, Eq. (w_b), Lemma 1):
+//   f~(W, b; X) = ReLU(conv(X; W) + b) is fitted to the feature map Y_CNN of the layer group it replaces.
+// The forward pass is the slim-layer convolution itself.  This file holds what the step adds:
+//   regress_grad_kernel   dZ = (Y - Y_CNN) / B where Y > 0, as bf16; per-block partial sums of the loss and of dL/db
+//   conv_wgrad_kernel     dL/dW[j, r, s, c] = sum over output pixels of dZ[m, j] * x[m @ tap (r, s), c] on the tensor
+//                         cores: both operands are read with the pixel index as the contraction dimension
+//   wgrad_reduce_kernel   sums the pixel-range partials in a fixed order
+//   sgd_update_kernel     v <- momentum v + lr (g + decay w);  w <- w - v;  bf16 copy of w for the next forward pass
+#include "conv_common.cuh"
+#include "umma_ptx.cuh"
+
+namespace dr {
+using namespace ptx;
+
+constexpr int WG_THREADS = 192;          // warp 0: TMA producer, warp 1: MMA issue, warps 2-5: drain
+constexpr int WG_BOX = TILE_M * 128;     // one TMA box: 128 pixels x 64 channels of bf16
+constexpr int WG_MAX_UNITS = 4;          // filter-column units (one tap x 64 input channels) per CTA: 256 accumulator columns
+constexpr int WG_STAGES = 2;
+constexpr int WG_STAGE_BYTES = (2 + WG_MAX_UNITS) * WG_BOX;
+constexpr int WG_SMEM_BYTES = WG_STAGES * WG_STAGE_BYTES + 1024;
+constexpr int RG_BLOCKS = 512;           // blocks (and partial rows) of regress_grad_kernel
+constexpr int RG_THREADS = 256;
+
+struct WgParams {
+    int Cin, Cout, k, stride, pad, Ho, Wo;
+    long long M;        // output pixels B*Ho*Wo: the contraction length
+    int K;              // k*k*Cin
+    int cpb;            // 64-channel blocks per tap
+    int units;          // k*k*cpb
+    int groups;         // ceil(units / WG_MAX_UNITS)
+    int n_ct;           // tiles of 128 output channels
+    int splits;         // pixel ranges; each writes its own partial
+    int pblocks;        // ceil(M / 128)
+    int a_mode;         // 0: x read as a [M][Cin] matrix (1x1 / stride 1 / pad 0), 1: im2col
+    float* partial;     // [splits][Cout][K]
+    int* status;
+};
+
+struct WgShared {
+    uint64_t full[WG_STAGES], empty[WG_STAGES], accum;
+    uint32_t tmem_base;
+    int abort;
+};
+
+// Shared-memory operand descriptor for an operand whose contraction index is the row of a 128-byte-swizzled tile
+// (rows of 64 non-contracted elements, 128 bytes): groups of 8 contraction rows are 1024 bytes apart (stride offset);
+// the next 64 non-contracted elements are a whole box further (leading offset).
+__device__ __forceinline__ uint64_t make_sdesc_mn_sw128(uint32_t smem_addr, uint32_t chunk_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((chunk_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+__global__ void __launch_bounds__(WG_THREADS, 1)
+conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_dz, const WgParams p) {
+    extern __shared__ uint8_t wg_smem_raw[];
+    __shared__ WgShared sh;
+    const uint32_t smem_base = (smem_u32(wg_smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bid = blockIdx.x;
+    const int g = bid % p.groups;
+    const int ct = (bid / p.groups) % p.n_ct;
+    const int split = bid / (p.groups * p.n_ct);
+    const int u0 = g * WG_MAX_UNITS;
+    const int nu = min(WG_MAX_UNITS, p.units - u0);
+    const int N = nu * 64;
+    const int pb0 = (int)((long long)split * p.pblocks / p.splits);
+    const int pb1 = (int)((long long)(split + 1) * p.pblocks / p.splits);
+    const bool second_half = ct * TILE_M + 64 < p.Cout;      // output channels 64..127 of this tile exist
+    volatile int* abort_flag = &sh.abort;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < WG_STAGES; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], 1); }
+        mbar_init(&sh.accum, 1);
+        sh.abort = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_dz);
+    }
+    if (warp == 1) { tmem_alloc(&sh.tmem_base, 256); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint32_t tx = (uint32_t)((second_half ? 2 : 1) + nu) * WG_BOX;
+            const int hw = p.Ho * p.Wo;
+            int s = 0;
+            uint32_t ph = 0;
+            for (int pb = pb0; pb < pb1; ++pb) {
+                if (pb - pb0 >= WG_STAGES && !mbar_wait(&sh.empty[s], ph ^ 1, abort_flag)) {
+                    if (!*abort_flag) report_timeout(p.status, 61, bid);
+                    *abort_flag = 1;
+                    break;
+                }
+                uint8_t* dst = wg_smem_raw + (smem_base - smem_u32(wg_smem_raw)) + (size_t)s * WG_STAGE_BYTES;
+                const long long m0 = (long long)pb * TILE_M;
+                mbar_arrive_expect_tx(&sh.full[s], tx);
+                tma_load_2d(dst, &map_dz, &sh.full[s], ct * TILE_M, (int)m0);
+                if (second_half) tma_load_2d(dst + WG_BOX, &map_dz, &sh.full[s], ct * TILE_M + 64, (int)m0);
+                const int img = (int)(m0 / hw);
+                const int rem = (int)(m0 - (long long)img * hw);
+                const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
+                const int hb = ho * p.stride - p.pad, wb = wo * p.stride - p.pad;
+                for (int u = 0; u < nu; ++u) {
+                    const int unit = u0 + u;
+                    const int tap = unit / p.cpb, c0 = (unit - tap * p.cpb) << 6;
+                    const int r = tap / p.k, t = tap - r * p.k;
+                    uint8_t* xd = dst + (size_t)(2 + u) * WG_BOX;
+                    if (p.a_mode == 0) tma_load_2d(xd, &map_x, &sh.full[s], c0, (int)m0);
+                    else tma_load_im2col_4d(xd, &map_x, &sh.full[s], c0, wb, hb, img, (uint16_t)t, (uint16_t)r);
+                }
+                if (++s == WG_STAGES) { s = 0; ph ^= 1; }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_bf16(TILE_M, N) | (1u << 15) | (1u << 16);   // both operands contraction-row ("MN-major")
+            int s = 0;
+            uint32_t ph = 0, accum = 0;
+            for (int pb = pb0; pb < pb1; ++pb) {
+                if (!mbar_wait(&sh.full[s], ph, abort_flag)) {
+                    if (!*abort_flag) report_timeout(p.status, 62, bid);
+                    *abort_flag = 1;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t a = smem_base + (uint32_t)s * WG_STAGE_BYTES;
+                const uint32_t b = a + 2 * WG_BOX;
+#pragma unroll
+                for (int ks = 0; ks < TILE_M / 16; ++ks) {       // 16 pixels per MMA: two 8-row groups
+                    umma_bf16(tmem, make_sdesc_mn_sw128(a + ks * 2048, WG_BOX), make_sdesc_mn_sw128(b + ks * 2048, WG_BOX), idesc, accum);
+                    accum = 1;
+                }
+                umma_commit(&sh.empty[s]);
+                if (++s == WG_STAGES) { s = 0; ph ^= 1; }
+            }
+            umma_commit(&sh.accum);      // also after a timeout: fires once whatever was issued has finished
+        }
+        __syncwarp();
+    } else {
+        // drain: TMEM lane = output channel of the tile, column = (unit, channel within the unit)
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const int j = ct * TILE_M + row;
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.accum, 0, abort_flag));
+        if (!ok) {
+            if (!*abort_flag) report_timeout(p.status, 63, bid);
+            *abort_flag = 1;
+        } else if (!*abort_flag && pb1 > pb0) {
+            tc_fence_after();
+            const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16);
+            float* out = p.partial + ((size_t)split * p.Cout + (j < p.Cout ? j : 0)) * p.K;
+            for (int c = 0; c < N; c += 32) {
+                uint32_t v[32];
+                tmem_ld_x32(taddr + c, v);
+                tmem_ld_wait();
+                const int unit = u0 + (c >> 6);
+                const int tap = unit / p.cpb;
+                const int ch0 = ((unit - tap * p.cpb) << 6) + (c & 63);
+                if (j < p.Cout) {
+                    float4* dst = reinterpret_cast<float4*>(out + (size_t)tap * p.Cin + ch0);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (ch0 + 4 * i < p.Cin)
+                            dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
+                                                 __uint_as_float(v[4 * i + 3]));
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, 256);
+}
+
+// dw[i] = sum over the pixel-range partials, in range order (the same result on every run).
+__global__ void wgrad_reduce_kernel(const float4* __restrict__ partial, int splits, size_t n4, float4* __restrict__ dw) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        float4 a = partial[i];
+        for (int s = 1; s < splits; ++s) {
+            const float4 b = partial[(size_t)s * n4 + i];
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
+        dw[i] = a;
+    }
+}
+
+// dZ, loss and bias-gradient partials.  y, yt, dz: dense [M][C] bf16, C a multiple of 8, C / 8 <= RG_THREADS.
+// Thread t works on the 8-channel vector t % (C/8) of rows t / (C/8), + rows_per_pass, ...: a thread stays on its
+// channels, so its eight bias sums live in registers; the rows of a block are contiguous, so loads are coalesced.
+// partials: [RG_BLOCKS][C + 1] floats, column C = the block's sum of (y - yt)^2.
+__global__ void __launch_bounds__(RG_THREADS)
+regress_grad_kernel(const uint4* __restrict__ y, const uint4* __restrict__ yt, long long M, int C, float scale, int relu,
+                    uint4* __restrict__ dz, float* __restrict__ partials) {
+    __shared__ float red[RG_THREADS * 9];
+    const int nv = C >> 3;
+    const int rows_per_pass = RG_THREADS / nv;
+    const int t = threadIdx.x;
+    const int vc = t % nv, ro = t / nv;
+    const long long rows_per_block = (M + gridDim.x - 1) / gridDim.x;
+    const long long r0 = (long long)blockIdx.x * rows_per_block;
+    const long long r1 = r0 + rows_per_block < M ? r0 + rows_per_block : M;
+    float sb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    float sl = 0.f;
+    if (ro < rows_per_pass) {
+        for (long long r = r0 + ro; r < r1; r += rows_per_pass) {
+            const size_t i = (size_t)r * nv + vc;
+            const uint4 a = y[i], b = yt[i];
+            const uint32_t au[4] = {a.x, a.y, a.z, a.w}, bu[4] = {b.x, b.y, b.z, b.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float y0 = bf16_lo(au[k]), y1 = bf16_hi(au[k]);
+                const float e0 = y0 - bf16_lo(bu[k]), e1 = y1 - bf16_hi(bu[k]);
+                sl = fmaf(e0, e0, sl);
+                sl = fmaf(e1, e1, sl);
+                const float g0 = (relu && !(y0 > 0.f)) ? 0.f : e0 * scale;
+                const float g1 = (relu && !(y1 > 0.f)) ? 0.f : e1 * scale;
+                o[k] = pack_bf16(g0, g1);
+                sb[2 * k] += bf16_lo(o[k]);          // the bias gradient sums what the filter gradient sees: the rounded dZ
+                sb[2 * k + 1] += bf16_hi(o[k]);
+            }
+            dz[i] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) red[t * 9 + k] = sb[k];
+    red[t * 9 + 8] = sl;
+    __syncthreads();
+    float* out = partials + (size_t)blockIdx.x * (C + 1);
+    if (t < nv) {                                   // fixed order over the rows-in-flight of this block
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int rr = 0; rr < rows_per_pass; ++rr)
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc[k] += red[(rr * nv + t) * 9 + k];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) out[t * 8 + k] = acc[k];
+    }
+    if (t == RG_THREADS - 1) {
+        float acc = 0.f;
+        for (int i = 0; i < RG_THREADS; ++i) acc += red[i * 9 + 8];
+        out[C] = acc;
+    }
+}
+
+// db[c] = sum over blocks of the partials, loss = loss_scale * sum of the squared-error partials; fixed order.
+__global__ void regress_finalize_kernel(const float* __restrict__ partials, int blocks, int C, float loss_scale, float* __restrict__ db,
+                                        float* __restrict__ loss) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c > C) return;
+    float acc = 0.f;
+    for (int b = 0; b < blocks; ++b) acc += partials[(size_t)b * (C + 1) + c];
+    if (c < C) db[c] = acc;
+    else if (loss) *loss = acc * loss_scale;
+}
+
+__global__ void sgd_update_kernel(size_t n, float* __restrict__ w, float* __restrict__ v, const float* __restrict__ g, float lr, float momentum,
+                                  float decay, __nv_bfloat16* __restrict__ w_bf16) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const float wi = w[i];
+        const float vi = momentum * v[i] + lr * (g[i] + decay * wi);
+        const float wn = wi - vi;
+        v[i] = vi;
+        w[i] = wn;
+        if (w_bf16) w_bf16[i] = __float2bfloat16_rn(wn);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+struct WgPlan { WgParams p; size_t partial_bytes; int ctas; };
+
+static int wgrad_plan(const dr_conv_desc* d, int B, int H, int W, WgPlan* out) {
+    if (!d || d->k <= 0 || d->stride <= 0 || d->pad < 0 || d->Cin <= 0 || d->Cout <= 0 || B < 0 || H <= 0 || W <= 0) return DR_ERR_INVALID_ARG;
+    if (H + 2 * d->pad < d->k || W + 2 * d->pad < d->k) return DR_ERR_INVALID_ARG;
+    if ((d->Cin & 7) || d->Cin < 64 || (d->Cout & 7) || d->k > 255) return DR_ERR_UNSUPPORTED;   // TMA rows of 128 bytes; 16-byte pitches
+    WgParams& p = out->p;
+    p.Cin = d->Cin; p.Cout = d->Cout; p.k = d->k; p.stride = d->stride; p.pad = d->pad;
+    p.Ho = (H + 2 * d->pad - d->k) / d->stride + 1;
+    p.Wo = (W + 2 * d->pad - d->k) / d->stride + 1;
+    p.M = (long long)B * p.Ho * p.Wo;
+    if (p.M > 0x7fffffffLL - TILE_M) return DR_ERR_UNSUPPORTED;
+    p.K = d->k * d->k * d->Cin;
+    p.cpb = (d->Cin + 63) / 64;
+    p.units = d->k * d->k * p.cpb;
+    p.groups = (p.units + WG_MAX_UNITS - 1) / WG_MAX_UNITS;
+    p.n_ct = (d->Cout + TILE_M - 1) / TILE_M;
+    p.pblocks = (int)((p.M + TILE_M - 1) / TILE_M);
+    p.a_mode = (d->k == 1 && d->stride == 1 && d->pad == 0) ? 0 : 1;
+    // pixel ranges: about two CTAs per SM in all, at least four pixel blocks each
+    const int tiles = p.n_ct * p.groups;
+    int s = tunable("DR_WGRAD_SPLITS", 0);
+    if (s <= 0) s = (2 * num_sms() + tiles - 1) / tiles;
+    if (s > p.pblocks / 4) s = p.pblocks / 4;
+    if (s < 1) s = 1;
+    p.splits = s;
+    out->ctas = tiles * s;
+    out->partial_bytes = p.M ? (size_t)s * d->Cout * p.K * sizeof(float) : 0;      // an empty batch needs no scratch
+    return DR_OK;
+}
+
+}  // namespace dr
+
+using namespace dr;
+
+extern "C" int dr_conv_wgrad_workspace_bytes(const dr_conv_desc* desc, int B, int H, int W, size_t* bytes) {
+    if (!bytes) return DR_ERR_INVALID_ARG;
+    WgPlan pl;
+    const int st = wgrad_plan(desc, B, H, W, &pl);
+    if (st != DR_OK) return st;
+    *bytes = (pl.partial_bytes + 255) / 256 * 256;
+    return DR_OK;
+}
+
+extern "C" int dr_conv_wgrad(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* dz, float* dw, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    WgPlan pl;
+    const int st = wgrad_plan(desc, B, H, W, &pl);
+    if (st != DR_OK) return st;
+    if (!x || !dz || !dw || !workspace) return DR_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(dz) || !aligned16(dw) || ((uintptr_t)workspace & 255)) return DR_ERR_ALIGNMENT;
+    if (workspace_bytes < pl.partial_bytes) return DR_ERR_WORKSPACE;
+    cudaStream_t s = (cudaStream_t)stream;
+    WgParams& p = pl.p;
+    const size_t n = (size_t)p.Cout * p.K;
+    if (p.M == 0) return cuda_status(cudaMemsetAsync(dw, 0, n * sizeof(float), s));
+    p.partial = reinterpret_cast<float*>(workspace);
+    p.status = dev_status_ptr();
+    ConvParams cp = {};
+    cp.x = reinterpret_cast<const __nv_bfloat16*>(x);
+    cp.B = B; cp.H = H; cp.W = W; cp.Cin = p.Cin; cp.Cout = p.Cout; cp.k = p.k; cp.stride = p.stride; cp.pad = p.pad;
+    cp.Ho = p.Ho; cp.Wo = p.Wo; cp.M = p.M; cp.K = p.K;
+    alignas(64) CUtensorMap map_x, map_dz;
+    int a_mode = 0;
+    int est = encode_input_map(cp, &map_x, &a_mode);
+    if (est == DR_OK) est = encode_rows_map(dz, p.M, p.Cout, p.Cout, &map_dz);
+    if (est != DR_OK) return est;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_BYTES) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return DR_ERR_CUDA;
+        }
+        attr_set = true;
+    }
+    conv_wgrad_kernel<<<pl.ctas, WG_THREADS, WG_SMEM_BYTES, s>>>(map_x, map_dz, p);
+    count_launch();
+    int lst = launch_status();
+    if (lst != DR_OK) return lst;
+    const size_t n4 = n / 4;                       // K is a multiple of 8
+    size_t blocks = (n4 + 255) / 256;
+    if (blocks > (size_t)num_sms() * 8) blocks = (size_t)num_sms() * 8;
+    wgrad_reduce_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(p.partial), p.splits, n4, reinterpret_cast<float4*>(dw));
+    count_launch();
+    return launch_status();
+}
+
+extern "C" int dr_regress_workspace_bytes(int C, size_t* bytes) {
+    if (!bytes || C <= 0) return DR_ERR_INVALID_ARG;
+    *bytes = ((size_t)RG_BLOCKS * (C + 1) * sizeof(float) + 255) / 256 * 256;
+    return DR_OK;
+}
+
+extern "C" int dr_regress_grad(int B, int H, int W, int C, const void* y, const void* yt, int relu, void* dz, float* db, float* loss,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+    if (B <= 0 || H <= 0 || W <= 0 || C <= 0 || !y || !yt || !dz || !db || !workspace) return DR_ERR_INVALID_ARG;
+    if ((C & 7) || (C >> 3) > RG_THREADS) return DR_ERR_UNSUPPORTED;
+    if (!aligned16(y) || !aligned16(yt) || !aligned16(dz) || ((uintptr_t)workspace & 255)) return DR_ERR_ALIGNMENT;
+    size_t need = 0;
+    dr_regress_workspace_bytes(C, &need);
+    if (workspace_bytes < need) return DR_ERR_WORKSPACE;
+    cudaStream_t s = (cudaStream_t)stream;
+    const long long M = (long long)B * H * W;
+    float* partials = reinterpret_cast<float*>(workspace);
+    regress_grad_kernel<<<RG_BLOCKS, RG_THREADS, 0, s>>>(reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(yt), M, C, 1.f / (float)B,
+                                                       relu ? 1 : 0, reinterpret_cast<uint4*>(dz), partials);
+    count_launch();
+    int st = launch_status();
+    if (st != DR_OK) return st;
+    regress_finalize_kernel<<<(C + 1 + 255) / 256, 256, 0, s>>>(partials, RG_BLOCKS, C, 0.5f / (float)B, db, loss);
+    count_launch();
+    return launch_status();
+}
+
+extern "C" int dr_sgd_update(size_t n, float* w, float* v, const float* g, float lr, float momentum, float decay, void* w_bf16, void* stream) {
+    if (!w || !v || !g) return DR_ERR_INVALID_ARG;
+    if (n == 0) return DR_OK;
+    size_t blocks = (n + 255) / 256;
+    if (blocks > (size_t)num_sms() * 8) blocks = (size_t)num_sms() * 8;
+    sgd_update_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(n, w, v, g, lr, momentum, decay, reinterpret_cast<__nv_bfloat16*>(w_bf16));
+    count_launch();
+    return launch_status();
+}
+
+static size_t round256(size_t b) { return (b + 255) / 256 * 256; }
+
+extern "C" int dr_regress_step_workspace_bytes(const dr_conv_desc* desc, int B, int H, int W, size_t* bytes) {
+    if (!bytes || !desc) return DR_ERR_INVALID_ARG;
+    size_t a = 0, b = 0, c = 0;
+    int st = dr_conv_wgrad_workspace_bytes(desc, B, H, W, &a);
+    if (st == DR_OK) st = dr_regress_workspace_bytes(desc->Cout, &b);
+    if (st == DR_OK) st = dr_conv_workspace_bytes(desc, B, H, W, &c);
+    if (st != DR_OK) return st;
+    *bytes = round256(a) + round256(b) + round256(c);
+    return DR_OK;
+}
+
+extern "C" int dr_regress_step(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* yt, float* w, float* b, float* vw,
+                               float* vb, void* w_bf16, float lr, float momentum, float decay, void* y, void* dz, float* dw, float* db,
+                               float* loss, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!desc || !x || !yt || !w || !b || !vw || !vb || !w_bf16 || !y || !dz || !dw || !db || !workspace) return DR_ERR_INVALID_ARG;
+    if (!(desc->flags & DR_BIAS) || (desc->flags & ~(unsigned)(DR_BIAS | DR_RELU))) return DR_ERR_UNSUPPORTED;
+    if ((desc->y_ldc && desc->y_ldc != desc->Cout) || desc->y_coff) return DR_ERR_UNSUPPORTED;
+    if ((uintptr_t)workspace & 255) return DR_ERR_ALIGNMENT;
+    size_t wa = 0, wb = 0, wc = 0, need = 0;
+    int st = dr_regress_step_workspace_bytes(desc, B, H, W, &need);
+    if (st != DR_OK) return st;
+    if (workspace_bytes < need) return DR_ERR_WORKSPACE;
+    dr_conv_wgrad_workspace_bytes(desc, B, H, W, &wa);
+    dr_regress_workspace_bytes(desc->Cout, &wb);
+    dr_conv_workspace_bytes(desc, B, H, W, &wc);
+    char* ws = reinterpret_cast<char*>(workspace);
+    const int Ho = (H + 2 * desc->pad - desc->k) / desc->stride + 1, Wo = (W + 2 * desc->pad - desc->k) / desc->stride + 1;
+    st = dr_conv_slim_ws(desc, B, H, W, x, w_bf16, b, nullptr, y, nullptr, wc ? ws + round256(wa) + round256(wb) : nullptr, wc, stream);
+    if (st != DR_OK) return st;
+    st = dr_regress_grad(B, Ho, Wo, desc->Cout, y, yt, (desc->flags & DR_RELU) ? 1 : 0, dz, db, loss, ws + round256(wa), wb, stream);
+    if (st != DR_OK) return st;
+    st = dr_conv_wgrad(desc, B, H, W, x, dz, dw, ws, wa, stream);
+    if (st != DR_OK) return st;
+    const size_t n = (size_t)desc->Cout * desc->k * desc->k * desc->Cin;
+    st = dr_sgd_update(n, w, vw, dw, lr, momentum, decay, w_bf16, stream);
+    if (st != DR_OK) return st;
+    return dr_sgd_update((size_t)desc->Cout, b, vb, db, lr, momentum, 0.f, nullptr, stream);
+}

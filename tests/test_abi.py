@@ -90,6 +90,37 @@ def test_conv_workspace_query_and_validation(dr):
     assert dr.dr_launch_count() == n0
 
 
+def test_regression_entry_points_validate_before_launch(dr):
+    """Host-only: workspace queries and argument checks of the layer-wise regression calls (Eq. (w_b))."""
+    d = dr.dr_conv_desc(k=3, stride=1, pad=1, Cin=64, Cout=192, flags=dr.DR_BIAS | dr.DR_RELU)
+    wg = dr.dr_conv_wgrad_workspace_bytes(d, 256, 28, 28)
+    assert wg % 256 == 0 and wg >= 192 * 576 * 4 and wg % (192 * 576 * 4) == 0      # whole partial copies of the gradient
+    assert dr.dr_conv_wgrad_workspace_bytes(d, 0, 28, 28) == 0
+    assert dr.dr_regress_workspace_bytes(192) >= 193 * 4
+    assert dr.dr_regress_step_workspace_bytes(d, 256, 28, 28) >= wg + dr.dr_regress_workspace_bytes(192)
+    n0 = dr.dr_launch_count()
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_conv_wgrad(d, 4, 8, 8, 256, 256, 256, 260, 1 << 30, 0)                  # workspace not 256-byte aligned
+    assert e.value.status == dr.DR_ERR_ALIGNMENT
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_conv_wgrad(d, 4, 8, 8, None, 256, 256, 256, 1 << 30, 0)
+    assert e.value.status == dr.DR_ERR_INVALID_ARG
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_regress_grad(4, 8, 8, 20, 256, 256, 1, 256, 256, None, 256, 1 << 20, 0)   # channels not a multiple of 8
+    assert e.value.status == dr.DR_ERR_UNSUPPORTED
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_regress_grad(4, 8, 8, 64, 256, 256, 1, 256, 256, None, 256, 16, 0)
+    assert e.value.status == dr.DR_ERR_WORKSPACE
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_sgd_update(16, None, 256, 256, 0.1, 0.9, 0.0, None, 0)
+    assert e.value.status == dr.DR_ERR_INVALID_ARG
+    dp = dr.dr_conv_desc(k=3, stride=1, pad=1, Cin=64, Cout=192, flags=dr.DR_BIAS | dr.DR_RELU | dr.DR_POOL, pool_k=3, pool_stride=2, pool_pad=1)
+    with pytest.raises(dr.DrError) as e:                                               # only bias / ReLU layers are re-learned
+        dr.dr_regress_step(dp, 4, 8, 8, 256, 256, 256, 256, 256, 256, 256, 0.1, 0.9, 0.0, 256, 256, 256, 256, None, 256, 1 << 30, 0)
+    assert e.value.status == dr.DR_ERR_UNSUPPORTED
+    assert dr.dr_launch_count() == n0
+
+
 def test_non_tensor_validation(dr):
     n0 = dr.dr_launch_count()
     for call in (lambda: dr.dr_relu(16, None, 256, 0),

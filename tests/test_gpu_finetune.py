@@ -1,0 +1,196 @@
+"""GPU parity of the layer-wise regression step (Section 3.1, Eq. (w_b), Lemma 1) against the CPU checker:
+the pre-activation gradient with loss and bias gradient, the tensor-core filter gradient, the SGD update, and
+whole steps on a slim layer fitted to the feature map of conv -> BatchNorm -> Scale -> ReLU."""
+import numpy as np
+import pytest
+
+import dr_synth as S
+from util import LAYER_L2, LAYER_MAX, err_norms, to_dev_bf16, to_dev_f32, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dr():
+    import paper_1708_04728_b200 as dr
+    dr.dr_set_conv_path(dr.DR_PATH_AUTO)
+    return dr
+
+
+@pytest.fixture(scope="module")
+def F():
+    import oracle.finetune as F
+    return F
+
+
+def workspace(nbytes, poison=True):
+    import torch
+    ws = torch.empty(max(nbytes, 4096) + 256, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    if poison:
+        ws.fill_(0xFF)                       # NaN bit patterns: stale scratch must never reach a result
+    return ws
+
+
+def status_ok(dr):
+    st, info = dr.dr_device_status()
+    assert st == 0, f"device status {st} {info}"
+
+
+def desc_of(dr, k, s, p, Cin, Cout, flags=0):
+    return dr.dr_conv_desc(k=k, stride=s, pad=p, Cin=Cin, Cout=Cout, flags=flags, pool_k=3, pool_stride=2, pool_pad=1,
+                           lrn_size=5, lrn_alpha=1e-4, lrn_beta=0.75, lrn_k=1.0, y_ldc=0, y_coff=0)
+
+
+WGRAD_CASES = [
+    # B, H, W, Cin, Cout, k, s, p
+    (2, 14, 14, 64, 64, 3, 1, 1),       # 392 pixels: three full pixel blocks and a tail of 8
+    (3, 17, 13, 96, 200, 3, 2, 1),      # channel tails on both sides (96 = 64 + 32, 200 = 128 + 72), stride 2
+    (4, 8, 8, 128, 128, 1, 1, 0),       # 1x1: x read as a matrix
+    (2, 9, 9, 64, 48, 5, 1, 2),         # 25 taps: seven column groups, the last with one unit; fewer than 64 filters
+    (8, 28, 28, 64, 192, 3, 1, 1),      # 6272 pixels: several pixel ranges per output tile
+    (1, 7, 7, 64, 8, 3, 1, 1),          # fewer pixels than one block
+]
+
+
+@pytest.mark.parametrize("B,H,W,Cin,Cout,k,s,p", WGRAD_CASES)
+def test_wgrad_parity(dr, F, B, H, W, Cin, Cout, k, s, p):
+    import torch
+    Ho, Wo = (H + 2 * p - k) // s + 1, (W + 2 * p - k) // s + 1
+    x = S.round_bf16(S.normal(0, f"ft.x{B}.{H}.{Cin}", (B, H, W, Cin)))
+    dz = S.round_bf16(S.normal(0, f"ft.dz{B}.{H}.{Cout}", (B, Ho, Wo, Cout)))
+    d = desc_of(dr, k, s, p, Cin, Cout)
+    need = dr.dr_conv_wgrad_workspace_bytes(d, B, H, W)
+    ws = workspace(need)
+    xd, dzd = to_dev_bf16(x), to_dev_bf16(dz)
+    dw = torch.full((Cout, k, k, Cin), float("nan"), dtype=torch.float32, device="cuda")
+    dr.dr_conv_wgrad(d, B, H, W, xd, dzd, dw, ws, ws.numel())
+    status_ok(dr)
+    ref = F.conv2d_wgrad(x, dz, k, s, p)
+    got = to_host(dw)
+    assert np.all(np.isfinite(got))
+    mx, l2 = err_norms(got, ref)
+    # exact products, float32 sums over at most a few thousand pixels
+    assert mx <= 2e-5 and l2 <= 1e-5, f"max-rel {mx:.3e}, rel-L2 {l2:.3e}"
+    dw2 = torch.zeros_like(dw)
+    dr.dr_conv_wgrad(d, B, H, W, xd, dzd, dw2, ws, ws.numel())
+    status_ok(dr)
+    assert torch.equal(dw, dw2), "the filter gradient is not the same on a second run"
+
+
+def test_wgrad_degenerate(dr):
+    import torch
+    d = desc_of(dr, 3, 1, 1, 64, 64)
+    dw = torch.full((64, 3, 3, 64), 5.0, dtype=torch.float32, device="cuda")
+    ws = workspace(4096)
+    x = torch.zeros(16, dtype=torch.bfloat16, device="cuda")
+    dr.dr_conv_wgrad(d, 0, 8, 8, x, x, dw, ws, ws.numel())           # empty batch: the gradient is zero
+    assert float(dw.abs().sum()) == 0.0
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_conv_wgrad(d, 4, 8, 8, x, x, dw, ws, 16)                # workspace too small
+    assert e.value.status == dr.DR_ERR_WORKSPACE
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_conv_wgrad(desc_of(dr, 3, 1, 1, 24, 64), 4, 8, 8, x, x, dw, ws, ws.numel())
+    assert e.value.status == dr.DR_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("B,H,W,C,relu", [(4, 9, 7, 64, 1), (4, 5, 5, 200, 0), (3, 14, 14, 192, 1), (2, 3, 3, 2048, 1), (1, 1, 1, 8, 1)])
+def test_regress_grad_parity(dr, F, B, H, W, C, relu):
+    import torch
+    y = S.round_bf16(np.maximum(S.normal(0, f"rg.y{B}.{C}", (B, H, W, C)), 0.0) if relu else S.normal(0, f"rg.y{B}.{C}", (B, H, W, C)))
+    yt = S.round_bf16(np.abs(S.normal(0, f"rg.t{B}.{C}", (B, H, W, C))))
+    ws = workspace(dr.dr_regress_workspace_bytes(C))
+    dz = torch.full((B, H, W, C), float("nan"), dtype=torch.bfloat16, device="cuda")
+    db = torch.full((C,), float("nan"), dtype=torch.float32, device="cuda")
+    loss = torch.full((1,), float("nan"), dtype=torch.float32, device="cuda")
+    dr.dr_regress_grad(B, H, W, C, to_dev_bf16(y), to_dev_bf16(yt), relu, dz, db, loss, ws, ws.numel())
+    ref = F.grad_preactivation(y, yt, bool(relu))
+    got = to_host(dz)
+    if B & (B - 1) == 0:
+        # 1/B is a power of two: the difference of two bf16 values and its scaling are exact in float32, so the
+        # rounding to bf16 is the only rounding on both sides
+        assert np.array_equal(got, S.round_bf16(ref))
+    else:
+        assert np.abs(got - ref).max() <= 2.0 ** -8 * np.abs(ref).max()
+    assert np.array_equal(got == 0.0, ref == 0.0) or not relu
+    assert abs(float(loss) - F.regression_loss(y, yt)) <= 1e-5 * F.regression_loss(y, yt)
+    ref_db = F.bias_grad(got)                                            # the sums of the stored (rounded) dZ
+    assert np.abs(to_host(db) - ref_db).max() <= 1e-5 * max(np.abs(ref_db).max(), 1e-30)
+
+
+def test_sgd_update_parity(dr, F):
+    import torch
+    n = 100003
+    w = S.normal(0, "sgd.w", (n,)).astype(np.float32)
+    v = (0.1 * S.normal(0, "sgd.v", (n,))).astype(np.float32)
+    g = S.normal(0, "sgd.g", (n,)).astype(np.float32)
+    wd, vd, gd = to_dev_f32(w), to_dev_f32(v), to_dev_f32(g)
+    shadow = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    dr.dr_sgd_update(n, wd, vd, gd, 0.01, 0.9, 5e-4, shadow)
+    w_ref, v_ref = F.sgd_update(w, v, g, np.float32(0.01), np.float32(0.9), np.float32(5e-4))
+    assert np.abs(to_host(vd) - v_ref).max() <= 1e-6 * np.abs(v_ref).max()
+    assert np.abs(to_host(wd) - w_ref).max() <= 1e-6 * np.abs(w_ref).max()
+    assert np.array_equal(to_host(shadow), S.round_bf16(to_host(wd)))   # the copy is the stored float32 value, rounded once
+
+
+def test_regression_steps_on_a_folded_layer(dr, F):
+    """A 3x3 slim layer is fitted to the output of conv -> BatchNorm -> Scale -> ReLU (Eq. (conv_bn_sl)): the
+    gradients of one step against the checker fed the same stored forward output, then the loss trajectory of
+    free-running steps on both sides."""
+    import oracle as O
+    import torch
+    B, H, W, Cin, Cout, k, s, p = 4, 14, 14, 64, 96, 3, 1, 1
+    x = S.round_bf16(S.normal(0, "ft.step.x", (B, H, W, Cin)))
+    wt = S.he_normal(0, "ft.step.wt", Cout, k, Cin)
+    mu, var = S.normal(0, "ft.mu", (Cout,), 0.1), S.uniform(0, "ft.var", (Cout,), 0.5, 1.5)
+    gamma, beta = S.uniform(0, "ft.gamma", (Cout,), 0.5, 1.5), S.normal(0, "ft.beta", (Cout,), 0.1)
+    yt = S.round_bf16(O.relu(O.scale(O.batchnorm(O.conv2d(x, wt, None, s, p), mu, var, 1.0, 1e-5), gamma, beta)))
+    w0 = S.round_bf16(S.he_normal(0, "ft.step.w0", Cout, k, Cin))       # master and bf16 copy start equal
+    b0 = np.zeros(Cout)
+    lr, mom, decay = 0.001, 0.9, 1e-4
+    d = desc_of(dr, k, s, p, Cin, Cout, dr.DR_BIAS | dr.DR_RELU)
+    ws = workspace(dr.dr_regress_step_workspace_bytes(d, B, H, W), poison=False)
+    ws.zero_()                                                           # the forward pass may keep tile counters there
+    wd, bd = to_dev_f32(w0), to_dev_f32(b0)
+    vw, vb = torch.zeros_like(wd), torch.zeros_like(bd)
+    shadow = to_dev_bf16(w0)
+    xd, ytd = to_dev_bf16(x), to_dev_bf16(yt)
+    y = torch.zeros((B, H, W, Cout), dtype=torch.bfloat16, device="cuda")
+    dz = torch.zeros_like(y)
+    dw = torch.zeros((Cout, k, k, Cin), dtype=torch.float32, device="cuda")
+    db = torch.zeros(Cout, dtype=torch.float32, device="cuda")
+    loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+    n0 = dr.dr_launch_count()
+
+    def step():
+        dr.dr_regress_step(d, B, H, W, xd, ytd, wd, bd, vw, vb, shadow, lr, mom, decay, y, dz, dw, db, loss, ws, ws.numel())
+        return float(loss)
+
+    l0 = step()
+    status_ok(dr)
+    assert dr.dr_launch_count() - n0 >= 7          # forward, gradient + its reduction, filter gradient + its reduction, two updates
+    # one step, teacher-forced on the stored forward output
+    y_gpu = to_host(y)
+    y_ref = F.slim_forward(x, w0, b0, s, p)
+    assert err_norms(y_gpu, y_ref)[1] <= LAYER_L2
+    dz_ref = F.grad_preactivation(y_gpu, yt)
+    mx, l2 = err_norms(to_host(dw), F.conv2d_wgrad(x, dz_ref, k, s, p))
+    assert mx <= LAYER_MAX and l2 <= LAYER_L2, f"filter gradient: max-rel {mx:.3e}, rel-L2 {l2:.3e}"
+    mx, l2 = err_norms(to_host(db), F.bias_grad(dz_ref))
+    assert mx <= LAYER_MAX and l2 <= LAYER_L2, f"bias gradient: max-rel {mx:.3e}, rel-L2 {l2:.3e}"
+    assert abs(l0 - F.regression_loss(y_gpu, yt)) <= 1e-4 * l0
+    w1_ref, _ = F.sgd_update(w0, np.zeros_like(w0), to_host(dw), lr, mom, decay)
+    assert err_norms(to_host(wd), w1_ref)[0] <= 1e-6
+    assert np.array_equal(to_host(shadow), S.round_bf16(to_host(wd)))
+    # free-running: the checker takes its own steps in float64 from the same start
+    w, b, rvw, rvb = w0.copy(), b0.copy(), np.zeros_like(w0), np.zeros(Cout)
+    ref_losses, gpu_losses = [], [l0]
+    for i in range(12):
+        w, b, rvw, rvb, l, _, _ = F.regression_step(x, yt, w, b, rvw, rvb, lr, mom, decay, s, p)
+        ref_losses.append(l)
+        if i < 11:
+            gpu_losses.append(step())
+    status_ok(dr)
+    for i, (a, r) in enumerate(zip(gpu_losses, ref_losses)):
+        assert abs(a - r) <= 2e-2 * r, f"step {i}: loss {a} vs {r}"
+    assert gpu_losses[-1] < 0.7 * gpu_losses[0], gpu_losses
