@@ -298,8 +298,8 @@ int conv_splitk_group_launch(const ConvParams& a, const ConvParams& b, const Con
 bool conv_splitk_group_supports(const ConvParams& a, const ConvParams& b, const ConvParams* c);
 size_t conv_splitk_group_scratch_bytes(const ConvParams& a, const ConvParams& b, const ConvParams* c);
 int encode_conv_maps(const ConvParams& p, int b_box_rows, CUtensorMap* map_a, CUtensorMap* map_b, int* a_mode);
-int encode_input_map(const ConvParams& p, CUtensorMap* map_a, int* a_mode);
-int encode_rows_map(const void* ptr, long long rows, int cols, int ld, CUtensorMap* map);
+int encode_input_map(const ConvParams& p, CUtensorMap* map_a, int* a_mode, int box_rows = TILE_M);
+int encode_rows_map(const void* ptr, long long rows, int cols, int ld, CUtensorMap* map, int box_rows = TILE_M);
 int tunable(const char* name, int dflt);
 
 }  // namespace dr

@@ -878,12 +878,12 @@ int encode_conv_maps(const ConvParams& p, int b_box_rows, CUtensorMap* map_a, CU
     return DR_OK;
 }
 
-// A [rows][cols] bf16 matrix with row pitch ld (elements) in boxes of 128 rows x 64 columns, 128-byte swizzle.
-int encode_rows_map(const void* ptr, long long rows, int cols, int ld, CUtensorMap* map) {
+// A [rows][cols] bf16 matrix with row pitch ld (elements) in boxes of box_rows rows x 64 columns, 128-byte swizzle.
+int encode_rows_map(const void* ptr, long long rows, int cols, int ld, CUtensorMap* map, int box_rows) {
     if (!load_encoders()) return DR_ERR_CUDA;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-    const cuuint32_t box[2] = {64, TILE_M};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     const cuuint32_t es[2] = {1, 1};
     return g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)ptr, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS
@@ -891,13 +891,13 @@ int encode_rows_map(const void* ptr, long long rows, int cols, int ld, CUtensorM
 }
 
 // The input-side map alone (see encode_conv_maps).
-int encode_input_map(const ConvParams& p, CUtensorMap* map_a, int* a_mode) {
+int encode_input_map(const ConvParams& p, CUtensorMap* map_a, int* a_mode, int box_rows) {
     if (!load_encoders()) return DR_ERR_CUDA;
     *a_mode = (p.k == 1 && p.stride == 1 && p.pad == 0) ? 0 : 1;
     if (*a_mode == 0) {
         const cuuint64_t dims[2] = {(cuuint64_t)p.Cin, (cuuint64_t)p.M};
         const cuuint64_t strides[1] = {(cuuint64_t)p.Cin * 2};
-        const cuuint32_t box[2] = {64, TILE_M};
+        const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
         const cuuint32_t es[2] = {1, 1};
         if (g_encode_tiled(map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)p.x, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -909,7 +909,7 @@ int encode_input_map(const ConvParams& p, CUtensorMap* map_a, int* a_mode) {
         const int lower[2] = {-p.pad, -p.pad};
         const int upper[2] = {p.pad - (p.k - 1), p.pad - (p.k - 1)};
         const cuuint32_t es[4] = {1, (cuuint32_t)p.stride, (cuuint32_t)p.stride, 1};
-        if (g_encode_im2col(map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void*)p.x, dims, strides, lower, upper, 64, TILE_M, es,
+        if (g_encode_im2col(map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void*)p.x, dims, strides, lower, upper, 64, (cuuint32_t)box_rows, es,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return DR_ERR_CUDA;

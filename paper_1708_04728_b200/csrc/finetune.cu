@@ -13,31 +13,38 @@ namespace dr {
 using namespace ptx;
 
 constexpr int WG_THREADS = 192;          // warp 0: TMA producer, warp 1: MMA issue, warps 2-5: drain
-constexpr int WG_BOX = TILE_M * 128;     // one TMA box: 128 pixels x 64 channels of bf16
-constexpr int WG_MAX_UNITS = 4;          // filter-column units (one tap x 64 input channels) per CTA: 256 accumulator columns
-constexpr int WG_STAGES = 2;
-constexpr int WG_STAGE_BYTES = (2 + WG_MAX_UNITS) * WG_BOX;
-constexpr int WG_SMEM_BYTES = WG_STAGES * WG_STAGE_BYTES + 1024;
+constexpr int WG_PIX = 128;              // pixels (contraction rows) per pipeline stage
+constexpr int WG_BOX = WG_PIX * 128;     // one TMA box: WG_PIX pixels x 64 channels of bf16
+constexpr int WG_MAX_STAGES = 4;
+constexpr int WG_SMEM_MAX = 200 * 1024;
 constexpr int RG_BLOCKS = 512;           // blocks (and partial rows) of regress_grad_kernel
 constexpr int RG_THREADS = 256;
 
+// The gradient as a matrix: rows = filter columns (tap, input channel) in units of one tap x 64 channels, columns =
+// output channels.  A CTA owns a tile of two units (128 accumulator lanes) x cpt output channels (at most 256
+// accumulator columns) and a range of pixel blocks.  In pair mode two CTAs of a cluster share a tile of four units x
+// cpt channels: each loads its own two units of x and its half of the dZ columns, the even CTA issues MMAs of 256 rows
+// that read both halves, and each drains its own 128 accumulator lanes: half the shared-memory fill per FLOP.
 struct WgParams {
     int Cin, Cout, k, stride, pad, Ho, Wo;
     long long M;        // output pixels B*Ho*Wo: the contraction length
     int K;              // k*k*Cin
     int cpb;            // 64-channel blocks per tap
     int units;          // k*k*cpb
-    int groups;         // ceil(units / WG_MAX_UNITS)
-    int n_ct;           // tiles of 128 output channels
+    int pair;           // 1: CTA pairs
+    int n_rt;           // row tiles: ceil(units / 2), pairs: ceil(units / 4)
+    int n_ct;           // column tiles
+    int cpt;            // output channels per column tile (a multiple of 64, <= 256; pairs: 128 or 256)
     int splits;         // pixel ranges; each writes its own partial
-    int pblocks;        // ceil(M / 128)
+    int pblocks;        // ceil(M / WG_PIX)
+    int stages, stage_bytes;
     int a_mode;         // 0: x read as a [M][Cin] matrix (1x1 / stride 1 / pad 0), 1: im2col
     float* partial;     // [splits][Cout][K]
     int* status;
 };
 
 struct WgShared {
-    uint64_t full[WG_STAGES], empty[WG_STAGES], accum;
+    uint64_t full[WG_MAX_STAGES], empty[WG_MAX_STAGES], accum;
     uint32_t tmem_base;
     int abort;
 };
@@ -55,74 +62,94 @@ __device__ __forceinline__ uint64_t make_sdesc_mn_sw128(uint32_t smem_addr, uint
     return d;
 }
 
+template <bool PAIR>
 __global__ void __launch_bounds__(WG_THREADS, 1)
 conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_dz, const WgParams p) {
     extern __shared__ uint8_t wg_smem_raw[];
     __shared__ WgShared sh;
     const uint32_t smem_base = (smem_u32(wg_smem_raw) + 1023u) & ~1023u;
+    uint8_t* const smem_al = wg_smem_raw + (smem_base - smem_u32(wg_smem_raw));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bid = blockIdx.x;
-    const int g = bid % p.groups;
-    const int ct = (bid / p.groups) % p.n_ct;
-    const int split = bid / (p.groups * p.n_ct);
-    const int u0 = g * WG_MAX_UNITS;
-    const int nu = min(WG_MAX_UNITS, p.units - u0);
-    const int N = nu * 64;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;       // pairs: 0 issues the MMAs
+    const int bid = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int rt = bid % p.n_rt;
+    const int ct = (bid / p.n_rt) % p.n_ct;
+    const int split = bid / (p.n_rt * p.n_ct);
+    const int u0 = PAIR ? 4 * rt + 2 * (int)rank : 2 * rt;
+    const int n_units = max(0, min(2, p.units - u0));           // units in this CTA's accumulator lanes (0: pairs only)
+    const int tile_units = PAIR ? min(4, p.units - 4 * rt) : n_units;
+    const int j0 = ct * p.cpt;                                  // first output channel of the tile
+    // 64-channel boxes of dZ: all of the tile's, or in a pair this CTA's half of N = 128 or 256 columns
+    const int N = PAIR ? (p.Cout - j0 > 128 ? 256 : 128) : ((min(p.cpt, p.Cout - j0) + 63) >> 6) * 64;
+    const int nb = PAIR ? N >> 7 : N >> 6;
+    const int jb = PAIR ? j0 + (int)rank * (N >> 1) : j0;       // first channel this CTA loads
     const int pb0 = (int)((long long)split * p.pblocks / p.splits);
     const int pb1 = (int)((long long)(split + 1) * p.pblocks / p.splits);
-    const bool second_half = ct * TILE_M + 64 < p.Cout;      // output channels 64..127 of this tile exist
+    const int stages = p.stages;
     volatile int* abort_flag = &sh.abort;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < WG_STAGES; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], 1); }
+        for (int i = 0; i < WG_MAX_STAGES; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], 1); }
         mbar_init(&sh.accum, 1);
         sh.abort = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_x);
         prefetch_tensormap(&map_dz);
     }
-    if (warp == 1) { tmem_alloc(&sh.tmem_base, 256); tmem_relinquish(); }
+    if (warp == 1) {
+        if (PAIR) { tmem_alloc_pair(&sh.tmem_base, 256); tmem_relinquish_pair(); }
+        else { tmem_alloc(&sh.tmem_base, 256); tmem_relinquish(); }
+    }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();                               // both CTAs' barriers exist before any remote arrive
     tc_fence_after();
     const uint32_t tmem = sh.tmem_base;
 
     if (warp == 0) {
         if (lane == 0) {
-            const uint32_t tx = (uint32_t)((second_half ? 2 : 1) + nu) * WG_BOX;
+            // bytes that land per stage: in a pair both CTAs' loads report to the even CTA's barrier
+            const uint32_t tx = (uint32_t)(tile_units + (PAIR ? 2 : 1) * nb) * WG_BOX;
             const int hw = p.Ho * p.Wo;
             int s = 0;
             uint32_t ph = 0;
             for (int pb = pb0; pb < pb1; ++pb) {
-                if (pb - pb0 >= WG_STAGES && !mbar_wait(&sh.empty[s], ph ^ 1, abort_flag)) {
+                if (pb - pb0 >= stages && !mbar_wait(&sh.empty[s], ph ^ 1, abort_flag)) {
                     if (!*abort_flag) report_timeout(p.status, 61, bid);
                     *abort_flag = 1;
                     break;
                 }
-                uint8_t* dst = wg_smem_raw + (smem_base - smem_u32(wg_smem_raw)) + (size_t)s * WG_STAGE_BYTES;
-                const long long m0 = (long long)pb * TILE_M;
-                mbar_arrive_expect_tx(&sh.full[s], tx);
-                tma_load_2d(dst, &map_dz, &sh.full[s], ct * TILE_M, (int)m0);
-                if (second_half) tma_load_2d(dst + WG_BOX, &map_dz, &sh.full[s], ct * TILE_M + 64, (int)m0);
+                uint8_t* dst = smem_al + (size_t)s * p.stage_bytes;
+                const long long m0 = (long long)pb * WG_PIX;
+                if (rank == 0) mbar_arrive_expect_tx(&sh.full[s], tx);
                 const int img = (int)(m0 / hw);
                 const int rem = (int)(m0 - (long long)img * hw);
                 const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
                 const int hb = ho * p.stride - p.pad, wb = wo * p.stride - p.pad;
-                for (int u = 0; u < nu; ++u) {
+                for (int u = 0; u < n_units; ++u) {
                     const int unit = u0 + u;
                     const int tap = unit / p.cpb, c0 = (unit - tap * p.cpb) << 6;
                     const int r = tap / p.k, t = tap - r * p.k;
-                    uint8_t* xd = dst + (size_t)(2 + u) * WG_BOX;
-                    if (p.a_mode == 0) tma_load_2d(xd, &map_x, &sh.full[s], c0, (int)m0);
-                    else tma_load_im2col_4d(xd, &map_x, &sh.full[s], c0, wb, hb, img, (uint16_t)t, (uint16_t)r);
+                    uint8_t* xd = dst + (size_t)u * WG_BOX;
+                    if (PAIR) {
+                        if (p.a_mode == 0) tma_load_2d_pair(xd, &map_x, &sh.full[s], c0, (int)m0);
+                        else tma_load_im2col_4d_pair(xd, &map_x, &sh.full[s], c0, wb, hb, img, (uint16_t)t, (uint16_t)r);
+                    } else {
+                        if (p.a_mode == 0) tma_load_2d(xd, &map_x, &sh.full[s], c0, (int)m0);
+                        else tma_load_im2col_4d(xd, &map_x, &sh.full[s], c0, wb, hb, img, (uint16_t)t, (uint16_t)r);
+                    }
                 }
-                if (++s == WG_STAGES) { s = 0; ph ^= 1; }
+                for (int i = 0; i < nb; ++i) {
+                    if (PAIR) tma_load_2d_pair(dst + (size_t)(2 + i) * WG_BOX, &map_dz, &sh.full[s], jb + 64 * i, (int)m0);
+                    else tma_load_2d(dst + (size_t)(2 + i) * WG_BOX, &map_dz, &sh.full[s], jb + 64 * i, (int)m0);
+                }
+                if (++s == stages) { s = 0; ph ^= 1; }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_bf16(TILE_M, N) | (1u << 15) | (1u << 16);   // both operands contraction-row ("MN-major")
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, N) | (1u << 15) | (1u << 16);   // both operands contraction-row ("MN-major")
             int s = 0;
             uint32_t ph = 0, accum = 0;
             for (int pb = pb0; pb < pb1; ++pb) {
@@ -132,24 +159,32 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     break;
                 }
                 tc_fence_after();
-                const uint32_t a = smem_base + (uint32_t)s * WG_STAGE_BYTES;
-                const uint32_t b = a + 2 * WG_BOX;
+                const uint32_t a = smem_base + (uint32_t)s * (uint32_t)p.stage_bytes;       // x: the accumulator's lanes
+                const uint32_t b = a + 2 * WG_BOX;                                          // dZ: its columns
 #pragma unroll
-                for (int ks = 0; ks < TILE_M / 16; ++ks) {       // 16 pixels per MMA: two 8-row groups
-                    umma_bf16(tmem, make_sdesc_mn_sw128(a + ks * 2048, WG_BOX), make_sdesc_mn_sw128(b + ks * 2048, WG_BOX), idesc, accum);
+                for (int ks = 0; ks < WG_PIX / 16; ++ks) {       // 16 pixels per MMA: two 8-row groups
+                    const uint64_t da = make_sdesc_mn_sw128(a + ks * 2048, WG_BOX), db = make_sdesc_mn_sw128(b + ks * 2048, WG_BOX);
+                    if (PAIR) umma_bf16_pair(tmem, da, db, idesc, accum);
+                    else umma_bf16(tmem, da, db, idesc, accum);
                     accum = 1;
                 }
-                umma_commit(&sh.empty[s]);
-                if (++s == WG_STAGES) { s = 0; ph ^= 1; }
+                if (PAIR) umma_commit_pair(&sh.empty[s], 3);
+                else umma_commit(&sh.empty[s]);
+                if (++s == stages) { s = 0; ph ^= 1; }
             }
-            umma_commit(&sh.accum);      // also after a timeout: fires once whatever was issued has finished
+            if (PAIR) umma_commit_pair(&sh.accum, 3);   // also after a timeout: fires once whatever was issued has finished
+            else umma_commit(&sh.accum);
         }
         __syncwarp();
     } else {
-        // drain: TMEM lane = output channel of the tile, column = (unit, channel within the unit)
+        // drain: TMEM lane = (unit, input channel within the unit), column = output channel of the tile.  The 32
+        // lanes of a warp are 32 consecutive input channels of one tap: each store instruction writes 128 contiguous bytes.
         const int q = warp & 3;
         const int row = q * 32 + lane;
-        const int j = ct * TILE_M + row;
+        const int unit = u0 + (row >> 6);
+        const int tap = unit / p.cpb;
+        const int ch = ((unit - tap * p.cpb) << 6) + (row & 63);
+        const bool row_ok = (row >> 6) < n_units && ch < p.Cin;
         const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.accum, 0, abort_flag));
         if (!ok) {
             if (!*abort_flag) report_timeout(p.status, 63, bid);
@@ -157,28 +192,26 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         } else if (!*abort_flag && pb1 > pb0) {
             tc_fence_after();
             const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16);
-            float* out = p.partial + ((size_t)split * p.Cout + (j < p.Cout ? j : 0)) * p.K;
+            float* out = p.partial + ((size_t)split * p.Cout + j0) * p.K + (size_t)tap * p.Cin + ch;
             for (int c = 0; c < N; c += 32) {
                 uint32_t v[32];
                 tmem_ld_x32(taddr + c, v);
                 tmem_ld_wait();
-                const int unit = u0 + (c >> 6);
-                const int tap = unit / p.cpb;
-                const int ch0 = ((unit - tap * p.cpb) << 6) + (c & 63);
-                if (j < p.Cout) {
-                    float4* dst = reinterpret_cast<float4*>(out + (size_t)tap * p.Cin + ch0);
+                if (row_ok) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        if (ch0 + 4 * i < p.Cin)
-                            dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
-                                                 __uint_as_float(v[4 * i + 3]));
+                    for (int i = 0; i < 32; ++i)
+                        if (j0 + c + i < p.Cout) out[(size_t)(c + i) * p.K] = __uint_as_float(v[i]);
                 }
             }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 256);
+    if (PAIR) cluster_sync_all();                               // neither CTA leaves while the other may still signal it
+    if (warp == 1) {
+        if (PAIR) tmem_dealloc_pair(tmem, 256);
+        else tmem_dealloc(tmem, 256);
+    }
 }
 
 // dw[i] = sum over the pixel-range partials, in range order (the same result on every run).
@@ -286,22 +319,49 @@ static int wgrad_plan(const dr_conv_desc* d, int B, int H, int W, WgPlan* out) {
     p.Ho = (H + 2 * d->pad - d->k) / d->stride + 1;
     p.Wo = (W + 2 * d->pad - d->k) / d->stride + 1;
     p.M = (long long)B * p.Ho * p.Wo;
-    if (p.M > 0x7fffffffLL - TILE_M) return DR_ERR_UNSUPPORTED;
+    if (p.M > 0x7fffffffLL - WG_PIX) return DR_ERR_UNSUPPORTED;
     p.K = d->k * d->k * d->Cin;
     p.cpb = (d->Cin + 63) / 64;
     p.units = d->k * d->k * p.cpb;
-    p.groups = (p.units + WG_MAX_UNITS - 1) / WG_MAX_UNITS;
-    p.n_ct = (d->Cout + TILE_M - 1) / TILE_M;
-    p.pblocks = (int)((p.M + TILE_M - 1) / TILE_M);
+    p.n_rt = (p.units + 1) / 2;
+    p.n_ct = (d->Cout + 255) / 256;
+    p.cpt = ((d->Cout + p.n_ct - 1) / p.n_ct + 63) / 64 * 64;    // even column tiles: 288 filters run as 192 + 96, not 256 + 32
+    p.n_ct = (d->Cout + p.cpt - 1) / p.cpt;
+    // CTA pairs where their coarser tiles (4 units x 128 or 256 channels) waste little: share of the MMA work that is real
+    {
+        const int n_rt2 = (p.units + 3) / 4, n_ct2 = (d->Cout + 255) / 256;
+        const int cols2 = (n_ct2 - 1) * 256 + (d->Cout - (n_ct2 - 1) * 256 > 128 ? 256 : 128);
+        const double eff1 = (double)p.units / (2 * p.n_rt) * d->Cout / ((double)(p.n_ct - 1) * p.cpt + ((d->Cout - (p.n_ct - 1) * p.cpt + 63) / 64 * 64));
+        const double eff2 = (double)p.units / (4 * n_rt2) * d->Cout / cols2;
+        const int pref = tunable("DR_WGRAD_PAIR", -1);
+        p.pair = pref >= 0 ? (pref != 0) : (eff2 >= 0.85 * eff1);
+        if (p.pair) { p.n_rt = n_rt2; p.n_ct = n_ct2; p.cpt = 256; }
+    }
+    p.stage_bytes = p.pair ? 4 * WG_BOX : (2 + p.cpt / 64) * WG_BOX;
+    p.stages = WG_SMEM_MAX / p.stage_bytes;
+    if (p.stages > WG_MAX_STAGES) p.stages = WG_MAX_STAGES;
+    p.pblocks = (int)((p.M + WG_PIX - 1) / WG_PIX);
     p.a_mode = (d->k == 1 && d->stride == 1 && d->pad == 0) ? 0 : 1;
-    // pixel ranges: about two CTAs per SM in all, at least four pixel blocks each
-    const int tiles = p.n_ct * p.groups;
+    // Pixel ranges.  One CTA per SM at a time (shared memory), so the launch runs in rounds of num_sms CTAs: take the
+    // number of ranges with the least rounds x pixel blocks per range, counting what a range adds (its partial tile is
+    // written and read again: about three pixel blocks' worth), with at least four pixel blocks per range.
+    const int tiles = p.n_rt * p.n_ct;
     int s = tunable("DR_WGRAD_SPLITS", 0);
-    if (s <= 0) s = (2 * num_sms() + tiles - 1) / tiles;
-    if (s > p.pblocks / 4) s = p.pblocks / 4;
+    if (s <= 0) {
+        const int sms = num_sms();
+        long long best = -1;
+        const int smax = p.pblocks / 4 < 64 ? p.pblocks / 4 : 64;
+        s = 1;
+        for (int c = 1; c <= smax; ++c) {
+            const long long rounds = ((long long)tiles * c * (p.pair ? 2 : 1) + sms - 1) / sms;
+            const long long cost = rounds * ((p.pblocks + c - 1) / c + 3);
+            if (best < 0 || cost < best) { best = cost; s = c; }
+        }
+    }
+    if (s > p.pblocks) s = p.pblocks;
     if (s < 1) s = 1;
     p.splits = s;
-    out->ctas = tiles * s;
+    out->ctas = tiles * s * (p.pair ? 2 : 1);
     out->partial_bytes = p.M ? (size_t)s * d->Cout * p.K * sizeof(float) : 0;      // an empty batch needs no scratch
     return DR_OK;
 }
@@ -339,18 +399,30 @@ extern "C" int dr_conv_wgrad(const dr_conv_desc* desc, int B, int H, int W, cons
     cp.Ho = p.Ho; cp.Wo = p.Wo; cp.M = p.M; cp.K = p.K;
     alignas(64) CUtensorMap map_x, map_dz;
     int a_mode = 0;
-    int est = encode_input_map(cp, &map_x, &a_mode);
-    if (est == DR_OK) est = encode_rows_map(dz, p.M, p.Cout, p.Cout, &map_dz);
+    int est = encode_input_map(cp, &map_x, &a_mode, WG_PIX);
+    if (est == DR_OK) est = encode_rows_map(dz, p.M, p.Cout, p.Cout, &map_dz, WG_PIX);
     if (est != DR_OK) return est;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_BYTES) != cudaSuccess) {
+        if (cudaFuncSetAttribute(conv_wgrad_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_MAX + 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_wgrad_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_MAX + 1024) != cudaSuccess) {
             (void)cudaGetLastError();
             return DR_ERR_CUDA;
         }
         attr_set = true;
     }
-    conv_wgrad_kernel<<<pl.ctas, WG_THREADS, WG_SMEM_BYTES, s>>>(map_x, map_dz, p);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.gridDim = dim3((unsigned)pl.ctas); cfg.blockDim = dim3(WG_THREADS);
+        cfg.dynamicSmemBytes = (size_t)p.stages * p.stage_bytes + 1024; cfg.stream = s;
+        cfg.attrs = attr; cfg.numAttrs = p.pair ? 1 : 0;
+        const cudaError_t e = p.pair ? cudaLaunchKernelEx(&cfg, conv_wgrad_kernel<true>, map_x, map_dz, p)
+                                     : cudaLaunchKernelEx(&cfg, conv_wgrad_kernel<false>, map_x, map_dz, p);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return DR_ERR_CUDA; }
+    }
     count_launch();
     int lst = launch_status();
     if (lst != DR_OK) return lst;

@@ -50,12 +50,17 @@ WGRAD_CASES = [
     (2, 9, 9, 64, 48, 5, 1, 2),         # 25 taps: seven column groups, the last with one unit; fewer than 64 filters
     (8, 28, 28, 64, 192, 3, 1, 1),      # 6272 pixels: several pixel ranges per output tile
     (1, 7, 7, 64, 8, 3, 1, 1),          # fewer pixels than one block
+    (2, 14, 14, 528, 320, 3, 1, 1),     # 9 channel blocks per tap, the last of 16 channels; two column tiles (256 + 64)
 ]
 
 
+@pytest.mark.parametrize("pair", [0, 1])
 @pytest.mark.parametrize("B,H,W,Cin,Cout,k,s,p", WGRAD_CASES)
-def test_wgrad_parity(dr, F, B, H, W, Cin, Cout, k, s, p):
+def test_wgrad_parity(dr, F, monkeypatch, B, H, W, Cin, Cout, k, s, p, pair):
+    """Both tilings of the kernel on every case: one CTA per tile, and CTA pairs sharing a tile of twice the rows
+    (forced here; the library picks by how much of the coarser tile a layer fills)."""
     import torch
+    monkeypatch.setenv("DR_WGRAD_PAIR", str(pair))
     Ho, Wo = (H + 2 * p - k) // s + 1, (W + 2 * p - k) // s + 1
     x = S.round_bf16(S.normal(0, f"ft.x{B}.{H}.{Cin}", (B, H, W, Cin)))
     dz = S.round_bf16(S.normal(0, f"ft.dz{B}.{H}.{Cout}", (B, Ho, Wo, Cout)))
