@@ -249,6 +249,8 @@ def run_finetune(args):
               ("paper-form 3a.p3 3x3 64->192 @28", 28, 64, 192, 3, 1, 1),
               ("merged 3a.m5 5x5 192->128 @28", 28, 192, 128, 5, 1, 2),
               ("merged 4e.m5 5x5 528->512 @14", 14, 528, 512, 5, 1, 2)]
+    if args.ft_layer is not None:
+        layers = [layers[args.ft_layer]]
     rows = []
     for name, hw, cin, cout, k, s, p in layers:
         d = dr.dr_conv_desc(k=k, stride=s, pad=p, Cin=cin, Cout=cout, flags=dr.DR_BIAS | dr.DR_RELU, pool_k=3, pool_stride=2, pool_pad=1,
@@ -307,6 +309,7 @@ def main():
                          "this is the small case the ncu captures under profiles/ run")
     ap.add_argument("--nontensor", action="store_true", help="achieved HBM GB/s of the stand-alone non-tensor kernels")
     ap.add_argument("--finetune", action="store_true", help="time one SGD step of the layer-wise regression of a slim layer (Eq. (w_b))")
+    ap.add_argument("--ft-layer", type=int, default=None, help="with --finetune: only layer 0..3 of its list (the small case of the ncu captures)")
     args = ap.parse_args()
     if args.batch is None:
         args.batch = 256 if args.arch in ("googlenet", "googlenet_streamline", "alexnet") else 128

@@ -13,9 +13,7 @@ namespace dr {
 using namespace ptx;
 
 constexpr int WG_THREADS = 192;          // warp 0: TMA producer, warp 1: MMA issue, warps 2-5: drain
-constexpr int WG_PIX = 128;              // pixels (contraction rows) per pipeline stage
-constexpr int WG_BOX = WG_PIX * 128;     // one TMA box: WG_PIX pixels x 64 channels of bf16
-constexpr int WG_MAX_STAGES = 4;
+constexpr int WG_MAX_STAGES = 8;
 constexpr int WG_SMEM_MAX = 200 * 1024;
 constexpr int RG_BLOCKS = 512;           // blocks (and partial rows) of regress_grad_kernel
 constexpr int RG_THREADS = 256;
@@ -36,7 +34,8 @@ struct WgParams {
     int n_ct;           // column tiles
     int cpt;            // output channels per column tile (a multiple of 64, <= 256; pairs: 128 or 256)
     int splits;         // pixel ranges; each writes its own partial
-    int pblocks;        // ceil(M / WG_PIX)
+    int pix;            // pixels (contraction rows) per pipeline stage: 64 or 128
+    int pblocks;        // ceil(M / pix)
     int stages, stage_bytes;
     int a_mode;         // 0: x read as a [M][Cin] matrix (1x1 / stride 1 / pad 0), 1: im2col
     float* partial;     // [splits][Cout][K]
@@ -51,20 +50,16 @@ struct WgShared {
 
 // Shared-memory operand descriptor for an operand whose contraction index is the row of a 128-byte-swizzled tile
 // (rows of 64 non-contracted elements, 128 bytes): groups of 8 contraction rows are 1024 bytes apart (stride offset);
-// the next 64 non-contracted elements are a whole box further (leading offset).
-__device__ __forceinline__ uint64_t make_sdesc_mn_sw128(uint32_t smem_addr, uint32_t chunk_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)((chunk_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
+// the next 64 non-contracted elements are a whole box further (leading offset).  This is its low word (start
+// address, leading offset); the high word (stride offset, version, swizzle) is that of the K-major form, SDESC_HI_SW128.
+__device__ __forceinline__ uint32_t sdesc_mn_lo(uint32_t smem_addr, uint32_t chunk_bytes) {
+    return ((smem_addr & 0x3FFFFu) >> 4) | (((chunk_bytes >> 4) & 0x3FFFu) << 16);
 }
 
-template <bool PAIR>
+template <bool PAIR, int PIX>
 __global__ void __launch_bounds__(WG_THREADS, 1)
 conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_dz, const WgParams p) {
+    constexpr int BOX = PIX * 128;                               // one TMA box: PIX pixels x 64 channels of bf16
     extern __shared__ uint8_t wg_smem_raw[];
     __shared__ WgShared sh;
     const uint32_t smem_base = (smem_u32(wg_smem_raw) + 1023u) & ~1023u;
@@ -109,39 +104,48 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     if (warp == 0) {
         if (lane == 0) {
             // bytes that land per stage: in a pair both CTAs' loads report to the even CTA's barrier
-            const uint32_t tx = (uint32_t)(tile_units + (PAIR ? 2 : 1) * nb) * WG_BOX;
-            const int hw = p.Ho * p.Wo;
+            const uint32_t tx = (uint32_t)(tile_units + (PAIR ? 2 : 1) * nb) * BOX;
+            // the single issuing thread is on the critical path: everything that does not change per stage is computed
+            // here, and the pixel coordinates advance with one division per stage
+            const uint32_t hw = (uint32_t)(p.Ho * p.Wo), Wo = (uint32_t)p.Wo;
+            int uc0[2], ur[2], ut[2];
+            for (int u = 0; u < 2; ++u) {
+                const int unit = min(u0 + u, p.units - 1);
+                const int tap = unit / p.cpb;
+                uc0[u] = (unit - tap * p.cpb) << 6;
+                ur[u] = tap / p.k;
+                ut[u] = tap - ur[u] * p.k;
+            }
+            long long m0 = (long long)pb0 * PIX;
+            uint32_t img = (uint32_t)(m0 / hw);
+            uint32_t rem = (uint32_t)(m0 - (long long)img * hw);
             int s = 0;
             uint32_t ph = 0;
-            for (int pb = pb0; pb < pb1; ++pb) {
+            for (int pb = pb0; pb < pb1; ++pb, m0 += PIX, rem += PIX) {
                 if (pb - pb0 >= stages && !mbar_wait(&sh.empty[s], ph ^ 1, abort_flag)) {
                     if (!*abort_flag) report_timeout(p.status, 61, bid);
                     *abort_flag = 1;
                     break;
                 }
                 uint8_t* dst = smem_al + (size_t)s * p.stage_bytes;
-                const long long m0 = (long long)pb * WG_PIX;
                 if (rank == 0) mbar_arrive_expect_tx(&sh.full[s], tx);
-                const int img = (int)(m0 / hw);
-                const int rem = (int)(m0 - (long long)img * hw);
-                const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
-                const int hb = ho * p.stride - p.pad, wb = wo * p.stride - p.pad;
+                while (rem >= hw) { rem -= hw; ++img; }
+                const uint32_t ho = rem / Wo, wo = rem - ho * Wo;
+                const int hb = (int)ho * p.stride - p.pad, wb = (int)wo * p.stride - p.pad;
                 for (int u = 0; u < n_units; ++u) {
-                    const int unit = u0 + u;
-                    const int tap = unit / p.cpb, c0 = (unit - tap * p.cpb) << 6;
-                    const int r = tap / p.k, t = tap - r * p.k;
-                    uint8_t* xd = dst + (size_t)u * WG_BOX;
+                    const int c0 = uc0[u], r = ur[u], t = ut[u];
+                    uint8_t* xd = dst + (size_t)u * BOX;
                     if (PAIR) {
                         if (p.a_mode == 0) tma_load_2d_pair(xd, &map_x, &sh.full[s], c0, (int)m0);
-                        else tma_load_im2col_4d_pair(xd, &map_x, &sh.full[s], c0, wb, hb, img, (uint16_t)t, (uint16_t)r);
+                        else tma_load_im2col_4d_pair(xd, &map_x, &sh.full[s], c0, wb, hb, (int)img, (uint16_t)t, (uint16_t)r);
                     } else {
                         if (p.a_mode == 0) tma_load_2d(xd, &map_x, &sh.full[s], c0, (int)m0);
-                        else tma_load_im2col_4d(xd, &map_x, &sh.full[s], c0, wb, hb, img, (uint16_t)t, (uint16_t)r);
+                        else tma_load_im2col_4d(xd, &map_x, &sh.full[s], c0, wb, hb, (int)img, (uint16_t)t, (uint16_t)r);
                     }
                 }
                 for (int i = 0; i < nb; ++i) {
-                    if (PAIR) tma_load_2d_pair(dst + (size_t)(2 + i) * WG_BOX, &map_dz, &sh.full[s], jb + 64 * i, (int)m0);
-                    else tma_load_2d(dst + (size_t)(2 + i) * WG_BOX, &map_dz, &sh.full[s], jb + 64 * i, (int)m0);
+                    if (PAIR) tma_load_2d_pair(dst + (size_t)(2 + i) * BOX, &map_dz, &sh.full[s], jb + 64 * i, (int)m0);
+                    else tma_load_2d(dst + (size_t)(2 + i) * BOX, &map_dz, &sh.full[s], jb + 64 * i, (int)m0);
                 }
                 if (++s == stages) { s = 0; ph ^= 1; }
             }
@@ -160,12 +164,12 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 }
                 tc_fence_after();
                 const uint32_t a = smem_base + (uint32_t)s * (uint32_t)p.stage_bytes;       // x: the accumulator's lanes
-                const uint32_t b = a + 2 * WG_BOX;                                          // dZ: its columns
+                const uint32_t b = a + 2 * BOX;                                          // dZ: its columns
 #pragma unroll
-                for (int ks = 0; ks < WG_PIX / 16; ++ks) {       // 16 pixels per MMA: two 8-row groups
-                    const uint64_t da = make_sdesc_mn_sw128(a + ks * 2048, WG_BOX), db = make_sdesc_mn_sw128(b + ks * 2048, WG_BOX);
-                    if (PAIR) umma_bf16_pair(tmem, da, db, idesc, accum);
-                    else umma_bf16(tmem, da, db, idesc, accum);
+                for (int ks = 0; ks < PIX / 16; ++ks) {       // 16 pixels per MMA: two 8-row groups
+                    // descriptors as 32-bit low words (start address, leading offset); the high word is the constant
+                    // of the 128-byte swizzle: one MMA costs the issuing thread a few instructions, not a few dozen
+                    umma_bf16_lo<PAIR>(tmem, sdesc_mn_lo(a, BOX) + ks * 128, sdesc_mn_lo(b, BOX) + ks * 128, idesc, accum, 1u);
                     accum = 1;
                 }
                 if (PAIR) umma_commit_pair(&sh.empty[s], 3);
@@ -319,7 +323,7 @@ static int wgrad_plan(const dr_conv_desc* d, int B, int H, int W, WgPlan* out) {
     p.Ho = (H + 2 * d->pad - d->k) / d->stride + 1;
     p.Wo = (W + 2 * d->pad - d->k) / d->stride + 1;
     p.M = (long long)B * p.Ho * p.Wo;
-    if (p.M > 0x7fffffffLL - WG_PIX) return DR_ERR_UNSUPPORTED;
+    if (p.M > 0x7fffffffLL - 128) return DR_ERR_UNSUPPORTED;
     p.K = d->k * d->k * d->Cin;
     p.cpb = (d->Cin + 63) / 64;
     p.units = d->k * d->k * p.cpb;
@@ -337,10 +341,15 @@ static int wgrad_plan(const dr_conv_desc* d, int B, int H, int W, WgPlan* out) {
         p.pair = pref >= 0 ? (pref != 0) : (eff2 >= 0.85 * eff1);
         if (p.pair) { p.n_rt = n_rt2; p.n_ct = n_ct2; p.cpt = 256; }
     }
-    p.stage_bytes = p.pair ? 4 * WG_BOX : (2 + p.cpt / 64) * WG_BOX;
+    p.pix = tunable("DR_WGRAD_PIX", 128) == 64 ? 64 : 128;
+    p.stage_bytes = (p.pair ? 4 : 2 + p.cpt / 64) * p.pix * 128;
     p.stages = WG_SMEM_MAX / p.stage_bytes;
     if (p.stages > WG_MAX_STAGES) p.stages = WG_MAX_STAGES;
-    p.pblocks = (int)((p.M + WG_PIX - 1) / WG_PIX);
+    {
+        const int st = tunable("DR_WGRAD_STAGES", 0);
+        if (st >= 1 && st < p.stages) p.stages = st;
+    }
+    p.pblocks = (int)((p.M + p.pix - 1) / p.pix);
     p.a_mode = (d->k == 1 && d->stride == 1 && d->pad == 0) ? 0 : 1;
     // Pixel ranges.  One CTA per SM at a time (shared memory), so the launch runs in rounds of num_sms CTAs: take the
     // number of ranges with the least rounds x pixel blocks per range, counting what a range adds (its partial tile is
@@ -350,11 +359,12 @@ static int wgrad_plan(const dr_conv_desc* d, int B, int H, int W, WgPlan* out) {
     if (s <= 0) {
         const int sms = num_sms();
         long long best = -1;
-        const int smax = p.pblocks / 4 < 64 ? p.pblocks / 4 : 64;
+        const int per128 = 128 / p.pix;                          // pixel blocks per 128 pixels
+        const int smax = p.pblocks / (4 * per128) < 64 ? p.pblocks / (4 * per128) : 64;
         s = 1;
         for (int c = 1; c <= smax; ++c) {
             const long long rounds = ((long long)tiles * c * (p.pair ? 2 : 1) + sms - 1) / sms;
-            const long long cost = rounds * ((p.pblocks + c - 1) / c + 3);
+            const long long cost = rounds * ((p.pblocks + c - 1) / c + 3 * per128);
             if (best < 0 || cost < best) { best = cost; s = c; }
         }
     }
@@ -399,13 +409,15 @@ extern "C" int dr_conv_wgrad(const dr_conv_desc* desc, int B, int H, int W, cons
     cp.Ho = p.Ho; cp.Wo = p.Wo; cp.M = p.M; cp.K = p.K;
     alignas(64) CUtensorMap map_x, map_dz;
     int a_mode = 0;
-    int est = encode_input_map(cp, &map_x, &a_mode, WG_PIX);
-    if (est == DR_OK) est = encode_rows_map(dz, p.M, p.Cout, p.Cout, &map_dz, WG_PIX);
+    int est = encode_input_map(cp, &map_x, &a_mode, p.pix);
+    if (est == DR_OK) est = encode_rows_map(dz, p.M, p.Cout, p.Cout, &map_dz, p.pix);
     if (est != DR_OK) return est;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(conv_wgrad_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_MAX + 1024) != cudaSuccess ||
-            cudaFuncSetAttribute(conv_wgrad_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_MAX + 1024) != cudaSuccess) {
+        if (cudaFuncSetAttribute(conv_wgrad_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_MAX + 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_wgrad_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_MAX + 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_wgrad_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_MAX + 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(conv_wgrad_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_MAX + 1024) != cudaSuccess) {
             (void)cudaGetLastError();
             return DR_ERR_CUDA;
         }
@@ -419,8 +431,11 @@ extern "C" int dr_conv_wgrad(const dr_conv_desc* desc, int B, int H, int W, cons
         cfg.gridDim = dim3((unsigned)pl.ctas); cfg.blockDim = dim3(WG_THREADS);
         cfg.dynamicSmemBytes = (size_t)p.stages * p.stage_bytes + 1024; cfg.stream = s;
         cfg.attrs = attr; cfg.numAttrs = p.pair ? 1 : 0;
-        const cudaError_t e = p.pair ? cudaLaunchKernelEx(&cfg, conv_wgrad_kernel<true>, map_x, map_dz, p)
-                                     : cudaLaunchKernelEx(&cfg, conv_wgrad_kernel<false>, map_x, map_dz, p);
+        cudaError_t e;
+        if (p.pix == 64) e = p.pair ? cudaLaunchKernelEx(&cfg, conv_wgrad_kernel<true, 64>, map_x, map_dz, p)
+                                    : cudaLaunchKernelEx(&cfg, conv_wgrad_kernel<false, 64>, map_x, map_dz, p);
+        else e = p.pair ? cudaLaunchKernelEx(&cfg, conv_wgrad_kernel<true, 128>, map_x, map_dz, p)
+                        : cudaLaunchKernelEx(&cfg, conv_wgrad_kernel<false, 128>, map_x, map_dz, p);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return DR_ERR_CUDA; }
     }
     count_launch();
