@@ -12,7 +12,7 @@
 namespace dr {
 using namespace ptx;
 
-constexpr int WG_THREADS = 192;          // warp 0: TMA producer, warp 1: MMA issue, warps 2-5: drain
+constexpr int WG_THREADS = 224;          // warp 0: TMA producer of x, warp 1: MMA issue, warps 2-5: drain, warp 6: TMA producer of dZ
 constexpr int WG_MAX_STAGES = 8;
 constexpr int WG_SMEM_MAX = 200 * 1024;
 constexpr int RG_BLOCKS = 512;           // blocks (and partial rows) of regress_grad_kernel
@@ -143,9 +143,27 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                         else tma_load_im2col_4d(xd, &map_x, &sh.full[s], c0, wb, hb, (int)img, (uint16_t)t, (uint16_t)r);
                     }
                 }
+                if (++s == stages) { s = 0; ph ^= 1; }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 6) {
+        if (lane == 0) {
+            // the dZ boxes of every stage, issued by a thread of their own so that the two operands' loads go out side by
+            // side; the bytes are expected on the barrier by the x producer of the even CTA (they may land first)
+            int s = 0;
+            uint32_t ph = 0;
+            int m0 = pb0 * PIX;
+            for (int pb = pb0; pb < pb1; ++pb, m0 += PIX) {
+                if (pb - pb0 >= stages && !mbar_wait(&sh.empty[s], ph ^ 1, abort_flag)) {
+                    if (!*abort_flag) report_timeout(p.status, 64, bid);
+                    *abort_flag = 1;
+                    break;
+                }
+                uint8_t* dst = smem_al + (size_t)s * p.stage_bytes + 2 * BOX;
                 for (int i = 0; i < nb; ++i) {
-                    if (PAIR) tma_load_2d_pair(dst + (size_t)(2 + i) * BOX, &map_dz, &sh.full[s], jb + 64 * i, (int)m0);
-                    else tma_load_2d(dst + (size_t)(2 + i) * BOX, &map_dz, &sh.full[s], jb + 64 * i, (int)m0);
+                    if (PAIR) tma_load_2d_pair(dst + (size_t)i * BOX, &map_dz, &sh.full[s], jb + 64 * i, m0);
+                    else tma_load_2d(dst + (size_t)i * BOX, &map_dz, &sh.full[s], jb + 64 * i, m0);
                 }
                 if (++s == stages) { s = 0; ph ^= 1; }
             }
@@ -341,10 +359,18 @@ static int wgrad_plan(const dr_conv_desc* d, int B, int H, int W, WgPlan* out) {
         p.pair = pref >= 0 ? (pref != 0) : (eff2 >= 0.85 * eff1);
         if (p.pair) { p.n_rt = n_rt2; p.n_ct = n_ct2; p.cpt = 256; }
     }
-    p.pix = tunable("DR_WGRAD_PIX", 128) == 64 ? 64 : 128;
-    p.stage_bytes = (p.pair ? 4 : 2 + p.cpt / 64) * p.pix * 128;
+    // Pipeline shape, measured at batch 256 on B200.  Pairs with 256 columns: stages of 128 pixels, three of them.  Pairs
+    // with 128 columns: stages of 64 pixels, three of them, so that two CTAs share an SM (one drains or starts while
+    // the other computes; each holds 256 of the 512 TMEM columns).  Single CTAs: stages of 64 pixels, as many as fit.
+    const bool narrow_pair = p.pair && d->Cout <= 128;
+    {
+        const int px = tunable("DR_WGRAD_PIX", 0);
+        p.pix = px == 64 || px == 128 ? px : ((p.pair && !narrow_pair) ? 128 : 64);
+    }
+    p.stage_bytes = (p.pair ? (narrow_pair ? 3 : 4) : 2 + p.cpt / 64) * p.pix * 128;
     p.stages = WG_SMEM_MAX / p.stage_bytes;
     if (p.stages > WG_MAX_STAGES) p.stages = WG_MAX_STAGES;
+    if (narrow_pair && p.pix == 64 && p.stages > 4) p.stages = 4;   // 4 x 24 KB: two CTAs per SM
     {
         const int st = tunable("DR_WGRAD_STAGES", 0);
         if (st >= 1 && st < p.stages) p.stages = st;
