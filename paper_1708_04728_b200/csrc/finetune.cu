@@ -306,15 +306,26 @@ regress_grad_kernel(const uint4* __restrict__ y, const uint4* __restrict__ yt, l
     }
 }
 
-// db[c] = sum over blocks of the partials, loss = loss_scale * sum of the squared-error partials; fixed order.
-__global__ void regress_finalize_kernel(const float* __restrict__ partials, int blocks, int C, float loss_scale, float* __restrict__ db,
-                                        float* __restrict__ loss) {
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
-    if (c > C) return;
+// db[c] = sum over blocks of the partials, loss = loss_scale * sum of the squared-error partials.  32 columns per
+// block, 16 threads per column: each sums every 16th partial row in order, then the 16 sums are added in order.
+__global__ void __launch_bounds__(512)
+regress_finalize_kernel(const float* __restrict__ partials, int blocks, int C, float loss_scale, float* __restrict__ db,
+                        float* __restrict__ loss) {
+    __shared__ float red[16][33];
+    const int cx = threadIdx.x & 31, part = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + cx;
     float acc = 0.f;
-    for (int b = 0; b < blocks; ++b) acc += partials[(size_t)b * (C + 1) + c];
-    if (c < C) db[c] = acc;
-    else if (loss) *loss = acc * loss_scale;
+    if (c <= C)
+        for (int b = part; b < blocks; b += 16) acc += partials[(size_t)b * (C + 1) + c];
+    red[part][cx] = acc;
+    __syncthreads();
+    if (part == 0 && c <= C) {
+        float t = 0.f;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) t += red[k][cx];
+        if (c < C) db[c] = t;
+        else if (loss) *loss = t * loss_scale;
+    }
 }
 
 __global__ void sgd_update_kernel(size_t n, float* __restrict__ w, float* __restrict__ v, const float* __restrict__ g, float lr, float momentum,
@@ -497,7 +508,7 @@ extern "C" int dr_regress_grad(int B, int H, int W, int C, const void* y, const 
     count_launch();
     int st = launch_status();
     if (st != DR_OK) return st;
-    regress_finalize_kernel<<<(C + 1 + 255) / 256, 256, 0, s>>>(partials, RG_BLOCKS, C, 0.5f / (float)B, db, loss);
+    regress_finalize_kernel<<<(C + 1 + 31) / 32, 512, 0, s>>>(partials, RG_BLOCKS, C, 0.5f / (float)B, db, loss);
     count_launch();
     return launch_status();
 }
