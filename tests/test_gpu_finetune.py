@@ -83,6 +83,32 @@ def test_wgrad_parity(dr, F, monkeypatch, B, H, W, Cin, Cout, k, s, p, pair):
     assert torch.equal(dw, dw2), "the filter gradient is not the same on a second run"
 
 
+@pytest.mark.parametrize("H,Cin,Cout,k,s,p", [(14, 528, 512, 5, 1, 2),      # 4e merged 5x5: CTA pairs, 128-pixel stages
+                                              (56, 64, 192, 3, 2, 1)])       # streamline conv2: single CTAs, 64-pixel stages
+def test_wgrad_bench_size_sampled_filters(dr, F, H, Cin, Cout, k, s, p):
+    """The layers and batch `bench.py --finetune` times, in the launch shape the library picks for them; the checker
+    computes the gradient of a seeded sample of filters (its cost is proportional to the number of filters)."""
+    import torch
+    B = 256
+    Ho = (H + 2 * p - k) // s + 1
+    x = S.round_bf16(S.normal(0, f"ftb.x{H}", (B, H, H, Cin)).astype(np.float32))
+    dz = S.round_bf16(S.normal(0, f"ftb.dz{H}", (B, Ho, Ho, Cout)).astype(np.float32))
+    d = desc_of(dr, k, s, p, Cin, Cout)
+    ws = workspace(dr.dr_conv_wgrad_workspace_bytes(d, B, H, H))
+    dw = torch.full((Cout, k, k, Cin), float("nan"), dtype=torch.float32, device="cuda")
+    dr.dr_conv_wgrad(d, B, H, H, to_dev_bf16(x), to_dev_bf16(dz), dw, ws, ws.numel())
+    status_ok(dr)
+    got = to_host(dw)
+    assert np.all(np.isfinite(got))
+    js = sorted(int(j) for j in S.stream(0, f"ftb.sample{H}").choice(Cout, size=4, replace=False)) + [0, Cout - 1]
+    ref = F.conv2d_wgrad(x, dz[..., js], k, s, p)
+    mx, l2 = err_norms(got[js], ref)
+    assert mx <= 5e-5 and l2 <= 2e-5, f"max-rel {mx:.3e}, rel-L2 {l2:.3e}"      # float32 sums over 50 k - 200 k pixels
+    # the rest: every filter's gradient has the size the sampled ones have (a dropped or doubled pixel range would not)
+    norms = np.sqrt((got.reshape(Cout, -1) ** 2).sum(axis=1))
+    assert norms.min() > 0.8 * np.median(norms) and norms.max() < 1.25 * np.median(norms)
+
+
 def test_wgrad_degenerate(dr):
     import torch
     d = desc_of(dr, 3, 1, 1, 64, 64)
