@@ -289,8 +289,27 @@ def run_finetune(args):
                      "images_per_s": B / t["step"] * 1e6, "wgrad_tflops": flops / t["wgrad"] * 1e-6,
                      "wgrad_frac": flops / t["wgrad"] * 1e-6 / pk["bf16_tflops"], "forward_tflops": flops / t["forward"] * 1e-6,
                      "loss": float(loss)})
+    cpu = None
+    if not args.no_cpu_baseline:
+        # the checker's own step on a bounded sample: 4 images of the first layer, float64, on the host cores
+        import time
+        import numpy as np
+        import oracle as O
+        import oracle.finetune as F
+        name, hw, cin, cout, k, s, p = layers[0]
+        ho = (hw + 2 * p - k) // s + 1
+        rng = np.random.default_rng(0)
+        n = 4
+        x = rng.normal(size=(n, hw, hw, cin)); yt = np.abs(rng.normal(size=(n, ho, ho, cout)))
+        w = rng.normal(size=(cout, k, k, cin)) * (2.0 / (k * k * cin)) ** 0.5
+        b = np.zeros(cout)
+        F.regression_step(x[:1], yt[:1], w, b, np.zeros_like(w), np.zeros(cout), 1e-6, 0.9, 1e-4, s, p)     # warm-up
+        t0 = time.perf_counter()
+        F.regression_step(x, yt, w, b, np.zeros_like(w), np.zeros(cout), 1e-6, 0.9, 1e-4, s, p)
+        dt = time.perf_counter() - t0
+        cpu = {"value": n / dt, "unit": "images/s", "cores": O.num_threads(), "kind": "oracle", "sample": f"one step on {n} images of '{name}'"}
     print(json.dumps({"metric": "layer-wise regression step of a slim layer", "batch": B, "peak_tflops": pk["bf16_tflops"], "peak_kind": pk_kind,
-                      "l2": "flushed before every timed call", "layers": rows}))
+                      "l2": "flushed before every timed call", "layers": rows, "cpu_baseline": cpu}))
 
 
 def main():
