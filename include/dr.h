@@ -330,7 +330,11 @@ int dr_sgd_update(size_t n, float* w, float* v, const float* g, float lr, float 
  * parameters, vw, vb: their momentum buffers, w_bf16: the bfloat16 filters the forward pass reads (all updated);
  * y, dz: [B,Ho,Wo,Cout] bfloat16 scratch (y holds the forward output of the parameters before the update);
  * dw: float32 [Cout][k][k][Cin] and db: float32 [Cout] receive the gradients; *loss the loss before the update.
- * The bias takes no weight decay.  workspace: dr_regress_step_workspace_bytes bytes, 256-byte aligned.         */
+ * The bias takes no weight decay.  workspace: dr_regress_step_workspace_bytes bytes, 256-byte aligned, zero-filled
+ * before the first call (the forward pass of a layer with few output tiles keeps its tile counters there and
+ * leaves them at zero; the gradient scratch in front of them is overwritten every call).
+ * Errors: INVALID_ARG, UNSUPPORTED (flags, channel slice, Cin < 64 or channels not multiples of 8), ALIGNMENT,
+ * WORKSPACE, and whatever the forward pass returns.                                                           */
 int dr_regress_step_workspace_bytes(const dr_conv_desc* desc, int B, int H, int W, size_t* bytes);
 int dr_regress_step(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* yt, float* w, float* b,
                     float* vw, float* vb, void* w_bf16, float lr, float momentum, float decay, void* y, void* dz,
