@@ -111,6 +111,11 @@ int dr_embed_groups(int Cout, int Cin_g, int k, int groups, const void* w_groupe
 int dr_space_to_depth(int B, int H, int W, int C, int k, int s, int pad, int Cp, const void* x, void* y,
                       void* stream);
 int dr_s2d_filter(int Cout, int k, int C, int s, int Cp, const void* w, void* w_out, void* stream);
+/* The same re-layout read backwards, for the layer-wise regression (Eq. (w_b)) of such a layer: the filter gradient
+ * of the stride-1 stand-in, dw_s2d float32 [Cout][kp][kp][Cp] (from dr_conv_wgrad on the space-to-depth image), gives
+ * the gradient of the original filter, dw float32 [Cout][k][k][C]: dw[j][r][q][c] = dw_s2d[j][r/s][q/s][((r%s)*s + q%s)*C + c].
+ * The update is applied to the original filter, which dr_s2d_filter then lays out again.                       */
+int dr_s2d_filter_grad(int Cout, int k, int C, int s, int Cp, const float* dw_s2d, float* dw, void* stream);
 
 /* ---- slim layers -------------------------------------------------------------------- */
 

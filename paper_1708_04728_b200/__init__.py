@@ -70,6 +70,7 @@ _SIGS = {
     "dr_embed_groups": (_I, [_I, _I, _I, _I, _P, _P, _P]),
     "dr_space_to_depth": (_I, [_I, _I, _I, _I, _I, _I, _I, _I, _P, _P, _P]),
     "dr_s2d_filter": (_I, [_I, _I, _I, _I, _I, _P, _P, _P]),
+    "dr_s2d_filter_grad": (_I, [_I, _I, _I, _I, _I, _P, _P, _P]),
     "dr_conv_slim": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P]),
     "dr_regress_workspace_bytes": (_I, [_I, C.POINTER(_Z)]),
     "dr_regress_grad": (_I, [_I, _I, _I, _I, _P, _P, _I, _P, _P, _P, _P, _Z, _P]),
@@ -162,6 +163,10 @@ def dr_space_to_depth(B, H, W, Cc, k, s, pad, Cp, x, y, stream=None):
 
 def dr_s2d_filter(Cout, k, Cc, s, Cp, w, w_out, stream=None):
     _check(_lib.dr_s2d_filter(Cout, k, Cc, s, Cp, _ptr(w), _ptr(w_out), _stream(stream)), "dr_s2d_filter")
+
+
+def dr_s2d_filter_grad(Cout, k, Cc, s, Cp, dw_s2d, dw, stream=None):
+    _check(_lib.dr_s2d_filter_grad(Cout, k, Cc, s, Cp, _ptr(dw_s2d), _ptr(dw), _stream(stream)), "dr_s2d_filter_grad")
 
 
 def dr_conv_slim(desc, B, H, W, x, w, b, residual, y, argmax=None, stream=None):

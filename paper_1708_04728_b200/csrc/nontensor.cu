@@ -548,6 +548,17 @@ __global__ void s2d_filter_kernel(int k, int C, int s, int kp, int Cp, const __n
     }
 }
 
+// The inverse gather, for gradients: dw [Cout][k][k][C] (float32) takes each element from the one place of
+// dw_s2d [Cout][kp][kp][Cp] that s2d_filter_kernel copies it to; the places that hold structural zeros are not read.
+__global__ void s2d_filter_grad_kernel(int k, int C, int s, int kp, int Cp, const float* __restrict__ dw_s2d, float* __restrict__ dw) {
+    const int j = blockIdx.x, per = k * k * C;
+    for (int i = threadIdx.x; i < per; i += blockDim.x) {
+        const int c = i % C, t = i / C, q = t % k, r = t / k;
+        const int R = r / s, S = q / s, a = (r - R * s) * s + (q - S * s);
+        dw[(size_t)j * per + i] = dw_s2d[(((size_t)j * kp + R) * kp + S) * Cp + a * C + c];
+    }
+}
+
 }  // namespace dr
 
 // ================================================================ C ABI
@@ -742,6 +753,14 @@ int dr_s2d_filter(int Cout, int k, int C, int s, int Cp, const void* w, void* w_
     DR_REQUIRE(w && w_out && Cout > 0 && k > 0 && C > 0 && s > 0 && Cp >= s * s * C, DR_ERR_INVALID_ARG);
     const int kp = (k + s - 1) / s;
     s2d_filter_kernel<<<Cout, 256, 0, (cudaStream_t)stream>>>(k, C, s, kp, Cp, (const __nv_bfloat16*)w, (__nv_bfloat16*)w_out);
+    count_launch();
+    return launch_status();
+}
+
+int dr_s2d_filter_grad(int Cout, int k, int C, int s, int Cp, const float* dw_s2d, float* dw, void* stream) {
+    DR_REQUIRE(dw_s2d && dw && Cout > 0 && k > 0 && C > 0 && s > 0 && Cp >= s * s * C, DR_ERR_INVALID_ARG);
+    const int kp = (k + s - 1) / s;
+    s2d_filter_grad_kernel<<<Cout, 256, 0, (cudaStream_t)stream>>>(k, C, s, kp, Cp, dw_s2d, dw);
     count_launch();
     return launch_status();
 }

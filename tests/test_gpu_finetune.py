@@ -44,7 +44,7 @@ def desc_of(dr, k, s, p, Cin, Cout, flags=0):
 
 WGRAD_CASES = [
     # B, H, W, Cin, Cout, k, s, p
-    (2, 14, 14, 64, 64, 3, 1, 1),       # 392 pixels: three full pixel blocks and a tail of 8
+    (2, 14, 14, 64, 64, 3, 1, 1),       # 392 pixels: full pixel blocks (of 64 or 128) and a tail of 8
     (3, 17, 13, 96, 200, 3, 2, 1),      # channel tails on both sides (96 = 64 + 32, 200 = 128 + 72), stride 2
     (4, 8, 8, 128, 128, 1, 1, 0),       # 1x1: x read as a matrix
     (2, 9, 9, 64, 48, 5, 1, 2),         # 25 taps: seven column groups, the last with one unit; fewer than 64 filters
@@ -107,6 +107,30 @@ def test_wgrad_bench_size_sampled_filters(dr, F, H, Cin, Cout, k, s, p):
     # the rest: every filter's gradient has the size the sampled ones have (a dropped or doubled pixel range would not)
     norms = np.sqrt((got.reshape(Cout, -1) ** 2).sum(axis=1))
     assert norms.min() > 0.8 * np.median(norms) and norms.max() < 1.25 * np.median(norms)
+
+
+@pytest.mark.parametrize("H,k,s,p", [(64, 7, 4, 3), (51, 11, 4, 0)])
+def test_wgrad_of_a_strided_three_channel_stem(dr, F, H, k, s, p):
+    """The stride-product stem of Section 3.1 (7x7/4 on RGB) and AlexNet's 11x11/4: the filter gradient is taken on the
+    space-to-depth form (a stride-1 convolution over 64 channels) and gathered back to the original filter layout."""
+    import torch
+    B, C, Cout, Cp = 4, 3, 64, 64
+    kp = (k + s - 1) // s
+    Ho = (H + 2 * p - k) // s + 1
+    x = S.round_bf16(S.normal(0, f"fts.x{k}", (B, H, H, C)))
+    dz = S.round_bf16(S.normal(0, f"fts.dz{k}", (B, Ho, Ho, Cout)))
+    xs = torch.zeros((B, Ho + kp - 1, Ho + kp - 1, Cp), dtype=torch.bfloat16, device="cuda")
+    dr.dr_space_to_depth(B, H, H, C, k, s, p, Cp, to_dev_bf16(x), xs)
+    d = desc_of(dr, kp, 1, 0, Cp, Cout)
+    Hs = Ho + kp - 1
+    ws = workspace(dr.dr_conv_wgrad_workspace_bytes(d, B, Hs, Hs))
+    dws = torch.full((Cout, kp, kp, Cp), float("nan"), dtype=torch.float32, device="cuda")
+    dr.dr_conv_wgrad(d, B, Hs, Hs, xs, to_dev_bf16(dz), dws, ws, ws.numel())
+    dw = torch.full((Cout, k, k, C), float("nan"), dtype=torch.float32, device="cuda")
+    dr.dr_s2d_filter_grad(Cout, k, C, s, Cp, dws, dw)
+    status_ok(dr)
+    mx, l2 = err_norms(to_host(dw), F.conv2d_wgrad(x, dz, k, s, p))
+    assert mx <= 2e-5 and l2 <= 1e-5, f"max-rel {mx:.3e}, rel-L2 {l2:.3e}"
 
 
 def test_wgrad_degenerate(dr):
