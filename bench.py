@@ -269,11 +269,20 @@ def run_finetune(args):
         ws = torch.zeros(need + 256, dtype=torch.uint8, device="cuda")
         ws = ws[(-ws.data_ptr()) % 256:]
         wg_need = dr.dr_conv_wgrad_workspace_bytes(d, B, hw, hw)
-        step = lambda: dr.dr_regress_step(d, B, hw, hw, x, yt, w, b, vw, vb, shadow, 1e-6, 0.9, 1e-4, y, dz, dw, db, loss, ws, ws.numel())
+        step = lambda st=None: dr.dr_regress_step(d, B, hw, hw, x, yt, w, b, vw, vb, shadow, 1e-6, 0.9, 1e-4, y, dz, dw, db, loss, ws, ws.numel(), st)
+        # the same step captured once into a CUDA graph (the calls allocate nothing and are stream-ordered): seven launches
+        gstream = torch.cuda.Stream()
+        gstream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(gstream):
+            step(gstream)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=gstream):
+                step(gstream)
+        torch.cuda.current_stream().wait_stream(gstream)
         wgrad = lambda: dr.dr_conv_wgrad(d, B, hw, hw, x, dz, dw, ws, wg_need)
         fwd = lambda: dr.dr_conv_slim_ws(d, B, hw, hw, x, shadow, b, None, y, None, None, 0)
         t = {}
-        for what, fn in (("step", step), ("wgrad", wgrad), ("forward", fwd)):
+        for what, fn in (("step", step), ("step_graph", graph.replay), ("wgrad", wgrad), ("forward", fwd)):
             ts = []
             for i in range(args.warmup + min(args.steps, 20)):
                 flush.zero_()
@@ -285,7 +294,7 @@ def run_finetune(args):
         st, info = dr.dr_device_status()
         assert st == 0, (st, info)
         flops = 2.0 * B * ho * ho * cout * k * k * cin
-        rows.append({"layer": name, "step_us": t["step"], "forward_us": t["forward"], "wgrad_us": t["wgrad"],
+        rows.append({"layer": name, "step_us": t["step"], "step_graph_us": t["step_graph"], "forward_us": t["forward"], "wgrad_us": t["wgrad"],
                      "images_per_s": B / t["step"] * 1e6, "wgrad_tflops": flops / t["wgrad"] * 1e-6,
                      "wgrad_frac": flops / t["wgrad"] * 1e-6 / pk["bf16_tflops"], "forward_tflops": flops / t["forward"] * 1e-6,
                      "loss": float(loss)})
