@@ -155,13 +155,13 @@ def test_resnet50_slim(dr, B, k):
     check_network(dr, dr.DR_ARCH_RESNET50, B, subset(B, k), N.resnet50_steps, params)
 
 
-@pytest.mark.parametrize("arch", [0, 1])
+@pytest.mark.parametrize("arch", [0, 1, 2])
 def test_unslimmed_path_matches(dr, arch):
     """The layer-by-layer baseline computes the same function: logits vs the checker and vs the slim net."""
     import oracle.nets as N
     B = 2
-    params = P.googlenet_params(0) if arch == 0 else P.resnet50_params(0)
-    steps = (N.googlenet_steps if arch == 0 else N.resnet50_steps)(params)
+    params = [P.googlenet_params, P.resnet50_params, P.googlenet_paper_params][arch](0)
+    steps = [N.googlenet_steps, N.resnet50_steps, N.googlenet_paper_steps][arch](params)
     images = lambda rng: np.stack([S.normal(0, f"x[{n}]", (224, 224, 3)) for n in rng])
     net_u, _, logits_u, keep_u = run_net(dr, arch, dr.DR_MODE_UNSLIMMED, B, params, images)
     net_s, _, logits_s, keep_s = run_net(dr, arch, dr.DR_MODE_SLIM, B, params, images)
@@ -177,7 +177,7 @@ def test_unslimmed_path_matches(dr, arch):
     assert n_u > 10 * n_s
     # group outputs of the baseline (several bf16 roundings inside one group) stay close to the checker's
     G = layer_outputs(net_u, logits_u, [0])
-    for name in ("conv1", "conv2", "3a", "5b") if arch == 0 else ("conv1", "res2a.2c", "res5c.2c"):
+    for name in ("conv1", "conv2", "3a", "5b") if arch != 1 else ("conv1", "res2a.2c", "res5c.2c"):
         if name in G:
             mx, l2 = err_norms(G[name], free[name][:1])
             assert l2 <= 2e-2, (name, l2)
