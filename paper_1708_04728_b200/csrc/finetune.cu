@@ -388,20 +388,22 @@ static int wgrad_plan(const dr_conv_desc* d, int B, int H, int W, WgPlan* out) {
     }
     p.pblocks = (int)((p.M + p.pix - 1) / p.pix);
     p.a_mode = (d->k == 1 && d->stride == 1 && d->pad == 0) ? 0 : 1;
-    // Pixel ranges.  One CTA per SM at a time (shared memory), so the launch runs in rounds of num_sms CTAs: take the
-    // number of ranges with the least rounds x pixel blocks per range, counting what a range adds (its partial tile is
-    // written and read again: about three pixel blocks' worth), with at least four pixel blocks per range.
+    // Pixel ranges.  The launch runs in rounds of as many CTAs as the SMs hold: take the number of ranges with the least
+    // rounds x (pixel blocks per range + what a range adds).  Fitted on the 4e merged 5x5 layer at batch 256
+    // (3 .. 14 ranges: 472 .. 601 us): a CTA's start, drain and the trip of its partial tile through the reduction cost
+    // as much as 14 blocks of 128 pixels.  At least four blocks of 128 pixels per range.
     const int tiles = p.n_rt * p.n_ct;
     int s = tunable("DR_WGRAD_SPLITS", 0);
     if (s <= 0) {
-        const int sms = num_sms();
+        // CTAs that run at a time: one per SM, two where the pipeline leaves room in shared memory
+        const int slots = num_sms() * ((p.stages * p.stage_bytes + 1024) * 2 <= 226 * 1024 ? 2 : 1);
         long long best = -1;
         const int per128 = 128 / p.pix;                          // pixel blocks per 128 pixels
         const int smax = p.pblocks / (4 * per128) < 64 ? p.pblocks / (4 * per128) : 64;
         s = 1;
         for (int c = 1; c <= smax; ++c) {
-            const long long rounds = ((long long)tiles * c * (p.pair ? 2 : 1) + sms - 1) / sms;
-            const long long cost = rounds * ((p.pblocks + c - 1) / c + 3 * per128);
+            const long long rounds = ((long long)tiles * c * (p.pair ? 2 : 1) + slots - 1) / slots;
+            const long long cost = rounds * ((p.pblocks + c - 1) / c + 14 * per128);
             if (best < 0 || cost < best) { best = cost; s = c; }
         }
     }
