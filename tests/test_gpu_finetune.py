@@ -133,6 +133,40 @@ def test_wgrad_of_a_strided_three_channel_stem(dr, F, H, k, s, p):
     assert mx <= 2e-5 and l2 <= 1e-5, f"max-rel {mx:.3e}, rel-L2 {l2:.3e}"
 
 
+def test_wgrad_seeded_random_shapes(dr, F, monkeypatch):
+    """Thirty seeded shapes around the tile edges: channel counts that are not multiples of 64, more than two column
+    tiles, every kernel size and stride the networks use, pixel counts around the stage sizes; the tiling alternates
+    between the library's choice, single CTAs and CTA pairs."""
+    import torch
+    r = S.stream(0, "ft.fuzz")
+    for case in range(30):
+        k = int(r.choice([1, 2, 3, 5, 7]))
+        s_ = int(r.choice([1, 2]))
+        p_ = int(r.integers(0, k // 2 + 1))
+        Cin = int(r.choice([64, 72, 96, 128, 136, 200, 256]))
+        Cout = int(r.choice([8, 40, 64, 120, 128, 136, 192, 256, 264, 320, 520, 600]))
+        B = int(r.integers(1, 4))
+        H = int(r.integers(max(k, 5), 19)); W = int(r.integers(max(k, 5), 19))
+        Ho, Wo = (H + 2 * p_ - k) // s_ + 1, (W + 2 * p_ - k) // s_ + 1
+        mode = ["", "0", "1"][case % 3]
+        if mode:
+            monkeypatch.setenv("DR_WGRAD_PAIR", mode)
+        else:
+            monkeypatch.delenv("DR_WGRAD_PAIR", raising=False)
+        x = S.round_bf16(S.normal(0, f"fz.x{case}", (B, H, W, Cin)))
+        dz = S.round_bf16(S.normal(0, f"fz.dz{case}", (B, Ho, Wo, Cout)))
+        d = desc_of(dr, k, s_, p_, Cin, Cout)
+        ws = workspace(dr.dr_conv_wgrad_workspace_bytes(d, B, H, W))
+        dw = torch.full((Cout, k, k, Cin), float("nan"), dtype=torch.float32, device="cuda")
+        dr.dr_conv_wgrad(d, B, H, W, to_dev_bf16(x), to_dev_bf16(dz), dw, ws, ws.numel())
+        status_ok(dr)
+        got = to_host(dw)
+        what = f"case {case}: B{B} {H}x{W} Cin{Cin} Cout{Cout} k{k} s{s_} p{p_} pair='{mode}'"
+        assert np.all(np.isfinite(got)), what
+        mx, l2 = err_norms(got, F.conv2d_wgrad(x, dz, k, s_, p_))
+        assert mx <= 2e-5 and l2 <= 1e-5, f"{what}: max-rel {mx:.3e}, rel-L2 {l2:.3e}"
+
+
 def test_wgrad_degenerate(dr):
     import torch
     d = desc_of(dr, 3, 1, 1, 64, 64)
