@@ -319,8 +319,9 @@ int dr_regress_grad(int B, int H, int W, int C, const void* y, const void* yt, i
  * with x zero outside the image.  x: [B,H,W,Cin] dense bfloat16; dz: [B,Ho,Wo,Cout] dense bfloat16;
  * dw: float32 [Cout][k][k][Cin], overwritten.  Products are exact, sums float32 on the tensor cores; the pixel
  * range is cut into pieces whose partial sums (in `workspace`) are added in a fixed order.
- * Restrictions: Cin >= 64, Cin and Cout multiples of 8 (else DR_ERR_UNSUPPORTED).
- * workspace: dr_conv_wgrad_workspace_bytes bytes, 256-byte aligned.  Errors: INVALID_ARG, ALIGNMENT, WORKSPACE. */
+ * Layers with Cin < 64, or with Cin or Cout not a multiple of 8, run on a plain CUDA-core kernel instead (one thread
+ * per filter element, pixels summed in order; there for completeness, needs no workspace).
+ * workspace: dr_conv_wgrad_workspace_bytes bytes (may be 0), 256-byte aligned.  Errors: INVALID_ARG, ALIGNMENT, WORKSPACE. */
 int dr_conv_wgrad_workspace_bytes(const dr_conv_desc* desc, int B, int H, int W, size_t* bytes);
 int dr_conv_wgrad(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* dz, float* dw,
                   void* workspace, size_t workspace_bytes, void* stream);

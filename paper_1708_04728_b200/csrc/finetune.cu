@@ -236,6 +236,30 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     }
 }
 
+// Layers the tensor-core kernel does not take (fewer than 64 input channels, channel counts that are not multiples of
+// 8): one thread per filter element walks all output pixels in order.  For completeness, not speed.
+__global__ void conv_wgrad_simt_kernel(int B, int H, int W, int Cin, int Cout, int k, int stride, int pad, int Ho, int Wo,
+                                       const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ dz, float* __restrict__ dw) {
+    const int jt = blockIdx.x;                      // (filter j, tap)
+    const int j = jt / (k * k), tap = jt - j * (k * k);
+    const int r = tap / k, t = tap - r * k;
+    for (int c = threadIdx.x; c < Cin; c += blockDim.x) {
+        float acc = 0.f;
+        for (int n = 0; n < B; ++n)
+            for (int ho = 0; ho < Ho; ++ho) {
+                const int hi = ho * stride - pad + r;
+                if (hi < 0 || hi >= H) continue;
+                for (int wo = 0; wo < Wo; ++wo) {
+                    const int wi = wo * stride - pad + t;
+                    if (wi < 0 || wi >= W) continue;
+                    acc = fmaf(__bfloat162float(dz[(((size_t)n * Ho + ho) * Wo + wo) * Cout + j]),
+                               __bfloat162float(x[(((size_t)n * H + hi) * W + wi) * Cin + c]), acc);
+                }
+            }
+        dw[(size_t)jt * Cin + c] = acc;
+    }
+}
+
 // dw[i] = sum over the pixel-range partials, in range order (the same result on every run).
 __global__ void wgrad_reduce_kernel(const float4* __restrict__ partial, int splits, size_t n4, float4* __restrict__ dw) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
@@ -341,13 +365,14 @@ __global__ void sgd_update_kernel(size_t n, float* __restrict__ w, float* __rest
 }
 
 // ------------------------------------------------------------------------------------------------ host side
-struct WgPlan { WgParams p; size_t partial_bytes; int ctas; };
+struct WgPlan { WgParams p; size_t partial_bytes; int ctas; bool simt; };
 
 static int wgrad_plan(const dr_conv_desc* d, int B, int H, int W, WgPlan* out) {
     if (!d || d->k <= 0 || d->stride <= 0 || d->pad < 0 || d->Cin <= 0 || d->Cout <= 0 || B < 0 || H <= 0 || W <= 0) return DR_ERR_INVALID_ARG;
     if (H + 2 * d->pad < d->k || W + 2 * d->pad < d->k) return DR_ERR_INVALID_ARG;
-    if ((d->Cin & 7) || d->Cin < 64 || (d->Cout & 7) || d->k > 255) return DR_ERR_UNSUPPORTED;   // TMA rows of 128 bytes; 16-byte pitches
+    if (d->k > 255) return DR_ERR_UNSUPPORTED;
     WgParams& p = out->p;
+    out->simt = (d->Cin & 7) || d->Cin < 64 || (d->Cout & 7);     // TMA wants rows of 128 bytes and 16-byte pitches
     p.Cin = d->Cin; p.Cout = d->Cout; p.k = d->k; p.stride = d->stride; p.pad = d->pad;
     p.Ho = (H + 2 * d->pad - d->k) / d->stride + 1;
     p.Wo = (W + 2 * d->pad - d->k) / d->stride + 1;
@@ -411,7 +436,7 @@ static int wgrad_plan(const dr_conv_desc* d, int B, int H, int W, WgPlan* out) {
     if (s < 1) s = 1;
     p.splits = s;
     out->ctas = tiles * s * (p.pair ? 2 : 1);
-    out->partial_bytes = p.M ? (size_t)s * d->Cout * p.K * sizeof(float) : 0;      // an empty batch needs no scratch
+    out->partial_bytes = (p.M && !out->simt) ? (size_t)s * d->Cout * p.K * sizeof(float) : 0;   // an empty batch needs no scratch
     return DR_OK;
 }
 
@@ -433,13 +458,21 @@ extern "C" int dr_conv_wgrad(const dr_conv_desc* desc, int B, int H, int W, cons
     WgPlan pl;
     const int st = wgrad_plan(desc, B, H, W, &pl);
     if (st != DR_OK) return st;
-    if (!x || !dz || !dw || !workspace) return DR_ERR_INVALID_ARG;
+    if (!x || !dz || !dw || (!workspace && pl.partial_bytes)) return DR_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(dz) || !aligned16(dw) || ((uintptr_t)workspace & 255)) return DR_ERR_ALIGNMENT;
     if (workspace_bytes < pl.partial_bytes) return DR_ERR_WORKSPACE;
     cudaStream_t s = (cudaStream_t)stream;
     WgParams& p = pl.p;
     const size_t n = (size_t)p.Cout * p.K;
     if (p.M == 0) return cuda_status(cudaMemsetAsync(dw, 0, n * sizeof(float), s));
+    if (pl.simt) {
+        const int threads = p.Cin >= 128 ? 128 : (p.Cin >= 64 ? 64 : 32);
+        conv_wgrad_simt_kernel<<<(unsigned)(p.Cout * p.k * p.k), threads, 0, s>>>(B, H, W, p.Cin, p.Cout, p.k, p.stride, p.pad, p.Ho, p.Wo,
+                                                                                reinterpret_cast<const __nv_bfloat16*>(x),
+                                                                                reinterpret_cast<const __nv_bfloat16*>(dz), dw);
+        count_launch();
+        return launch_status();
+    }
     p.partial = reinterpret_cast<float*>(workspace);
     p.status = dev_status_ptr();
     ConvParams cp = {};

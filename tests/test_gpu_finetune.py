@@ -51,6 +51,8 @@ WGRAD_CASES = [
     (8, 28, 28, 64, 192, 3, 1, 1),      # 6272 pixels: several pixel ranges per output tile
     (1, 7, 7, 64, 8, 3, 1, 1),          # fewer pixels than one block
     (2, 14, 14, 528, 320, 3, 1, 1),     # 9 channel blocks per tap, the last of 16 channels; two column tiles (256 + 64)
+    (2, 9, 9, 24, 20, 3, 1, 1),         # channel counts the tensor-core kernel does not take: the CUDA-core kernel
+    (1, 16, 16, 3, 16, 7, 2, 3),        # three input channels, 7x7 / 2
 ]
 
 
@@ -179,8 +181,9 @@ def test_wgrad_degenerate(dr):
         dr.dr_conv_wgrad(d, 4, 8, 8, x, x, dw, ws, 16)                # workspace too small
     assert e.value.status == dr.DR_ERR_WORKSPACE
     with pytest.raises(dr.DrError) as e:
-        dr.dr_conv_wgrad(desc_of(dr, 3, 1, 1, 24, 64), 4, 8, 8, x, x, dw, ws, ws.numel())
-    assert e.value.status == dr.DR_ERR_UNSUPPORTED
+        dr.dr_conv_wgrad(desc_of(dr, 3, 1, 1, 64, 64), 4, 8, 8, x, x, None, ws, ws.numel())
+    assert e.value.status == dr.DR_ERR_INVALID_ARG
+    assert dr.dr_conv_wgrad_workspace_bytes(desc_of(dr, 3, 1, 1, 24, 64), 4, 8, 8) == 0     # CUDA-core kernel: no scratch
 
 
 @pytest.mark.parametrize("B,H,W,C,relu", [(4, 9, 7, 64, 1), (4, 5, 5, 200, 0), (3, 14, 14, 192, 1), (2, 3, 3, 2048, 1), (1, 1, 1, 8, 1)])
