@@ -307,9 +307,10 @@ int dr_selftest_wait_timeout(long long limit_cycles, void* stream);
 
 /* dZ = dL/dZ for Y = ReLU(Z): (Y - Y_CNN) / B where Y > 0 (everywhere when relu == 0), rounded to bfloat16;
  * db[c] = sum over pixels of that (rounded) dZ; *loss = 1/(2B) * sum (Y - Y_CNN)^2 (loss may be NULL).
- *  y, yt, dz: dense [B,H,W,C] bfloat16 (dz may not alias y or yt), C a multiple of 8 and <= 2048; db: float32 [C].
+ *  y, yt, dz: dense [B,H,W,C] bfloat16 (dz may not alias y or yt); db: float32 [C].  C a multiple of 8 and <= 2048
+ *  takes the vector kernel, other C a plain element-wise one.
  *  workspace: dr_regress_workspace_bytes(C) bytes, 256-byte aligned.  Sums are taken in a fixed order.
- * Errors: INVALID_ARG, UNSUPPORTED (C), ALIGNMENT, WORKSPACE.                                                   */
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE.                                                                   */
 int dr_regress_workspace_bytes(int C, size_t* bytes);
 int dr_regress_grad(int B, int H, int W, int C, const void* y, const void* yt, int relu, void* dz, float* db,
                     float* loss, void* workspace, size_t workspace_bytes, void* stream);

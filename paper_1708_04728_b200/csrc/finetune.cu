@@ -330,6 +330,43 @@ regress_grad_kernel(const uint4* __restrict__ y, const uint4* __restrict__ yt, l
     }
 }
 
+// Channel counts the vector kernel does not take (not a multiple of 8, or more than 2048): element-wise dZ, then one
+// block per channel (and one for the loss) summing its column with a fixed-order tree.  For completeness, not speed.
+__global__ void regress_grad_scalar_kernel(size_t n, float scale, int relu, const __nv_bfloat16* __restrict__ y,
+                                           const __nv_bfloat16* __restrict__ yt, __nv_bfloat16* __restrict__ dz) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const float a = __bfloat162float(y[i]);
+        const float g = (relu && !(a > 0.f)) ? 0.f : (a - __bfloat162float(yt[i])) * scale;
+        dz[i] = __float2bfloat16_rn(g);
+    }
+}
+__global__ void __launch_bounds__(256)
+regress_sums_scalar_kernel(long long M, int C, float loss_scale, const __nv_bfloat16* __restrict__ y, const __nv_bfloat16* __restrict__ yt,
+                           const __nv_bfloat16* __restrict__ dz, float* __restrict__ db, float* __restrict__ loss) {
+    __shared__ float red[256];
+    const int c = blockIdx.x;                       // c == C: the loss
+    float acc = 0.f;
+    if (c < C) {
+        for (long long m = threadIdx.x; m < M; m += 256) acc += __bfloat162float(dz[(size_t)m * C + c]);
+    } else {
+        const size_t n = (size_t)M * C;
+        for (size_t i = threadIdx.x; i < n; i += 256) {
+            const float e = __bfloat162float(y[i]) - __bfloat162float(yt[i]);
+            acc = fmaf(e, e, acc);
+        }
+    }
+    red[threadIdx.x] = acc;
+    __syncthreads();
+    for (int w = 128; w > 0; w >>= 1) {
+        if ((int)threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        if (c < C) db[c] = red[0];
+        else if (loss) *loss = red[0] * loss_scale;
+    }
+}
+
 // db[c] = sum over blocks of the partials, loss = loss_scale * sum of the squared-error partials.  32 columns per
 // block, 16 threads per column: each sums every 16th partial row in order, then the 16 sums are added in order.
 __global__ void __launch_bounds__(512)
@@ -530,13 +567,26 @@ extern "C" int dr_regress_workspace_bytes(int C, size_t* bytes) {
 extern "C" int dr_regress_grad(int B, int H, int W, int C, const void* y, const void* yt, int relu, void* dz, float* db, float* loss,
                                void* workspace, size_t workspace_bytes, void* stream) {
     if (B <= 0 || H <= 0 || W <= 0 || C <= 0 || !y || !yt || !dz || !db || !workspace) return DR_ERR_INVALID_ARG;
-    if ((C & 7) || (C >> 3) > RG_THREADS) return DR_ERR_UNSUPPORTED;
     if (!aligned16(y) || !aligned16(yt) || !aligned16(dz) || ((uintptr_t)workspace & 255)) return DR_ERR_ALIGNMENT;
     size_t need = 0;
     dr_regress_workspace_bytes(C, &need);
     if (workspace_bytes < need) return DR_ERR_WORKSPACE;
     cudaStream_t s = (cudaStream_t)stream;
     const long long M = (long long)B * H * W;
+    if ((C & 7) || (C >> 3) > RG_THREADS) {
+        const size_t n = (size_t)M * C;
+        size_t blocks = (n + 255) / 256;
+        if (blocks > (size_t)num_sms() * 8) blocks = (size_t)num_sms() * 8;
+        regress_grad_scalar_kernel<<<(unsigned)blocks, 256, 0, s>>>(n, 1.f / (float)B, relu ? 1 : 0, reinterpret_cast<const __nv_bfloat16*>(y),
+                                                                   reinterpret_cast<const __nv_bfloat16*>(yt), reinterpret_cast<__nv_bfloat16*>(dz));
+        count_launch();
+        int st0 = launch_status();
+        if (st0 != DR_OK) return st0;
+        regress_sums_scalar_kernel<<<C + 1, 256, 0, s>>>(M, C, 0.5f / (float)B, reinterpret_cast<const __nv_bfloat16*>(y),
+                                                        reinterpret_cast<const __nv_bfloat16*>(yt), reinterpret_cast<const __nv_bfloat16*>(dz), db, loss);
+        count_launch();
+        return launch_status();
+    }
     float* partials = reinterpret_cast<float*>(workspace);
     regress_grad_kernel<<<RG_BLOCKS, RG_THREADS, 0, s>>>(reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(yt), M, C, 1.f / (float)B,
                                                        relu ? 1 : 0, reinterpret_cast<uint4*>(dz), partials);

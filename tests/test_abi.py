@@ -106,8 +106,8 @@ def test_regression_entry_points_validate_before_launch(dr):
         dr.dr_conv_wgrad(d, 4, 8, 8, None, 256, 256, 256, 1 << 30, 0)
     assert e.value.status == dr.DR_ERR_INVALID_ARG
     with pytest.raises(dr.DrError) as e:
-        dr.dr_regress_grad(4, 8, 8, 20, 256, 256, 1, 256, 256, None, 256, 1 << 20, 0)   # channels not a multiple of 8
-    assert e.value.status == dr.DR_ERR_UNSUPPORTED
+        dr.dr_regress_grad(4, 8, 8, 20, 256, 256, 1, 256, 256, None, 260, 1 << 20, 0)   # workspace not 256-byte aligned
+    assert e.value.status == dr.DR_ERR_ALIGNMENT
     with pytest.raises(dr.DrError) as e:
         dr.dr_regress_grad(4, 8, 8, 64, 256, 256, 1, 256, 256, None, 256, 16, 0)
     assert e.value.status == dr.DR_ERR_WORKSPACE

@@ -186,7 +186,8 @@ def test_wgrad_degenerate(dr):
     assert dr.dr_conv_wgrad_workspace_bytes(desc_of(dr, 3, 1, 1, 24, 64), 4, 8, 8) == 0     # CUDA-core kernel: no scratch
 
 
-@pytest.mark.parametrize("B,H,W,C,relu", [(4, 9, 7, 64, 1), (4, 5, 5, 200, 0), (3, 14, 14, 192, 1), (2, 3, 3, 2048, 1), (1, 1, 1, 8, 1)])
+@pytest.mark.parametrize("B,H,W,C,relu", [(4, 9, 7, 64, 1), (4, 5, 5, 200, 0), (3, 14, 14, 192, 1), (2, 3, 3, 2048, 1), (1, 1, 1, 8, 1),
+                                          (4, 6, 5, 20, 1), (2, 2, 2, 2056, 0)])       # the last two: the element-wise kernel
 def test_regress_grad_parity(dr, F, B, H, W, C, relu):
     import torch
     y = S.round_bf16(np.maximum(S.normal(0, f"rg.y{B}.{C}", (B, H, W, C)), 0.0) if relu else S.normal(0, f"rg.y{B}.{C}", (B, H, W, C)))
