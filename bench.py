@@ -296,10 +296,28 @@ def run_finetune(args):
         st, info = dr.dr_device_status()
         assert st == 0, (st, info)
         flops = 2.0 * B * ho * ho * cout * k * k * cin
+        lib = {}
+        if args.cudnn_context:
+            # context only, never on the product path: the vendor library's forward convolution and weight gradient
+            # of the same layer through PyTorch (channels-last bf16, autotuned), timed the same way
+            torch.backends.cudnn.benchmark = True
+            xl = x.permute(0, 3, 1, 2)                     # NHWC storage seen as channels-last NCHW
+            wl = shadow.permute(0, 3, 1, 2)
+            dzl = dz.permute(0, 3, 1, 2)
+            for what, fn in (("cudnn_forward_us", lambda: torch.nn.functional.conv2d(xl, wl, None, s, p)),
+                             ("cudnn_wgrad_us", lambda: torch.nn.grad.conv2d_weight(xl, wl.shape, dzl, s, p))):
+                ts = []
+                for i in range(args.warmup + min(args.steps, 20)):
+                    flush.zero_()
+                    a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(); fn(); e.record(); torch.cuda.synchronize()
+                    if i >= args.warmup:
+                        ts.append(a.elapsed_time(e) * 1e3)
+                lib[what] = statistics.median(ts)
         rows.append({"layer": name, "step_us": t["step"], "step_graph_us": t["step_graph"], "forward_us": t["forward"], "wgrad_us": t["wgrad"],
                      "images_per_s": B / t["step"] * 1e6, "wgrad_tflops": flops / t["wgrad"] * 1e-6,
                      "wgrad_frac": flops / t["wgrad"] * 1e-6 / pk["bf16_tflops"], "forward_tflops": flops / t["forward"] * 1e-6,
-                     "loss": float(loss)})
+                     "loss": float(loss), **lib})
     cpu = None
     if not args.no_cpu_baseline:
         # the checker's own step on a bounded sample: 4 images of the first layer, float64, on the host cores
@@ -339,6 +357,8 @@ def main():
                          "this is the small case the ncu captures under profiles/ run")
     ap.add_argument("--nontensor", action="store_true", help="achieved HBM GB/s of the stand-alone non-tensor kernels")
     ap.add_argument("--finetune", action="store_true", help="time one SGD step of the layer-wise regression of a slim layer (Eq. (w_b))")
+    ap.add_argument("--cudnn-context", action="store_true",
+                    help="with --finetune: also time the vendor library's forward and weight-gradient convolution of the same layers (context)")
     ap.add_argument("--ft-layer", type=int, default=None, help="with --finetune: only layer 0..3 of its list (the small case of the ncu captures)")
     args = ap.parse_args()
     if args.batch is None:
