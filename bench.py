@@ -27,8 +27,11 @@ if ROOT not in sys.path:
 
 METRIC = "slim GoogLeNet forward throughput"
 UNIT = "images/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of conv_umma_tma_kernel on layer 3b.m5 at batch 256 (ncu --set full)
-NCU_TRAFFIC_3B_M5 = 106.566e6 + 67.416e6
+# DRAM traffic of the dominant kernel's largest launch from one ncu capture (dram__bytes_read.sum, dram__bytes_write.sum),
+# with the tiling the capture was taken on; the line carries it only while dr_conv_plan still reports that tiling.
+NCU_TRAFFIC = {"layer": "3b.m5", "batch": 256, "dram_read_bytes": 106.566e6, "dram_write_bytes": 67.416e6,
+               "plan": {"path": "umma_tma", "Nt": 144, "n_blocks": 1, "pair": 1, "wide": 1},
+               "note": "ncu capture of one launch at batch 256; a lower bound of the launch's traffic: part of its output is still in L2 when it ends"}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -42,50 +45,107 @@ def peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    """SM clock / power / throttle-reason samples taken while the timed region runs: NVML polled from a thread every
+    10 ms with host time stamps (so that samples can be matched to a timed chunk), nvidia-smi in a child process where
+    NVML cannot be loaded.  Reading only; no setting of the GPU is touched."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
-        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.samples = []            # (t, sm_mhz, power_w, reason bits)
+        self.max_mhz = None
+        self.p = None
+        self.thread = None
+        self._stop = False
         try:
-            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
-                                       "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+            import threading
+            import pynvml as nv
+            nv.nvmlInit()
+            uuid = None
+            try:
+                import torch
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(index).uuid)
+            except Exception:
+                pass
+            h = None
+            if uuid:
+                try:
+                    h = nv.nvmlDeviceGetHandleByUUID(uuid)
+                except Exception:
+                    h = None
+            if h is None:
+                h = nv.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+            self.bits = {"hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown, "hw_thermal_slowdown": nv.nvmlClocksEventReasonHwThermalSlowdown,
+                         "sw_thermal_slowdown": nv.nvmlClocksEventReasonSwThermalSlowdown, "sw_power_cap": nv.nvmlClocksEventReasonSwPowerCap}
+
+            def poll():
+                while not self._stop:
+                    try:
+                        self.samples.append((time.perf_counter(), float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)),
+                                             nv.nvmlDeviceGetPowerUsage(h) / 1000.0, int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))))
+                    except Exception:
+                        pass
+                    time.sleep(0.01)
+            self.thread = threading.Thread(target=poll, daemon=True)
+            self.thread.start()
         except Exception:
-            self.p = None
+            self.thread = None
+            self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            try:
+                self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
+                                           "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+            except Exception:
+                self.p = None
+
+    def window(self, t0: float, t1: float):
+        """Median SM clock of the samples with t0 <= t <= t1 (None without NVML samples there)."""
+        v = [s[1] for s in self.samples if t0 <= s[0] <= t1]
+        return statistics.median(v) if v else None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.p is None:
-            return out
-        self.p.terminate()
-        try:
-            self.p.wait(timeout=5)
-        except Exception:
-            self.p.kill()
-        self.f.flush(); self.f.seek(0)
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "source": "nvml" if self.thread else "nvidia-smi"}
         sm, mx, pw, reasons = [], [], [], set()
-        for line in self.f.read().splitlines():
-            c = [x.strip() for x in line.split(",")]
-            if len(c) < 9:
-                continue
+        if self.thread is not None:
+            self._stop = True
+            self.thread.join(timeout=2)
+            for _t, mhz, p, bits in self.samples:
+                sm.append(mhz); pw.append(p); mx.append(self.max_mhz)
+                for name, bit in self.bits.items():
+                    if bits & bit:
+                        reasons.add(name)
+        elif self.p is not None:
+            self.p.terminate()
             try:
-                sm.append(float(c[1])); mx.append(float(c[2])); pw.append(float(c[3]))
-            except ValueError:
-                continue
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
+                self.p.wait(timeout=5)
+            except Exception:
+                self.p.kill()
+            self.f.flush(); self.f.seek(0)
+            for line in self.f.read().splitlines():
+                c = [x.strip() for x in line.split(",")]
+                if len(c) < 9:
+                    continue
+                try:
+                    sm.append(float(c[1])); mx.append(float(c[2])); pw.append(float(c[3]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            self.f.close()
+            try:
+                os.unlink(self.f.name)
+            except OSError:
+                pass
+        else:
+            return out
         if len(sm) >= 4:      # samples under load: the half with the higher power draw (idle samples before/after the region drag the median)
             order = sorted(range(len(sm)), key=lambda i: pw[i])[len(sm) // 2:]
             sm = [sm[i] for i in order]
-        self.f.close()
-        try:
-            os.unlink(self.f.name)
-        except OSError:
-            pass
+            pw = [pw[i] for i in order]
         if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm),
+                       power_w_median=statistics.median(pw))
         return out
 
 
@@ -344,7 +404,8 @@ def run_finetune(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps; default: as many as make the timed region about 3 s long (the sustained-clock regime)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=None, help="default 256 (GoogLeNet), 128 (ResNet-50)")
@@ -353,8 +414,8 @@ def main():
     ap.add_argument("--layers-out", default=None, help="write the per-layer table (us, roofline) as JSON")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layer", default=None,
-                    help="time ONE slim layer of the network (e.g. conv1, conv2, 3b.m5, 4e.3x3) instead of the whole step; "
-                         "this is the small case the ncu captures under profiles/ run")
+                    help="time ONE slim layer of the network (e.g. conv1, conv2, 3b.m5, 4e.3x3) instead of the whole step: "
+                         "the small case for profiler captures")
     ap.add_argument("--nontensor", action="store_true", help="achieved HBM GB/s of the stand-alone non-tensor kernels")
     ap.add_argument("--finetune", action="store_true", help="time one SGD step of the layer-wise regression of a slim layer (Eq. (w_b))")
     ap.add_argument("--cudnn-context", action="store_true",
@@ -363,6 +424,9 @@ def main():
     args = ap.parse_args()
     if args.batch is None:
         args.batch = 256 if args.arch in ("googlenet", "googlenet_streamline", "alexnet") else 128
+    auto_steps = args.steps is None
+    if auto_steps and (args.impl == "reference" or args.layer or args.nontensor or args.finetune):
+        args.steps = 2 if args.impl == "reference" else 20
     if args.impl == "reference":
         return run_reference(args)
     if args.layer:
@@ -458,14 +522,50 @@ def main():
 
     sampler = ClockSampler(local) if rank == 0 else None
     n0 = dr.dr_launch_count()
-    times = timed(step, args.steps, args.warmup)
-    launches = (dr.dr_launch_count() - n0) * args.steps // (args.steps + args.warmup)
+    if auto_steps:
+        # no step count given: a timed region of about 3 s, long enough for the part to settle at the clock it sustains
+        # under its power limit (every rank takes the same count: the estimate is the slowest rank's)
+        est = timed(step, 5, args.warmup)
+        est_ms = max_over_ranks(sum(est) / len(est), world)
+        args.steps = max(20, int(3000.0 / max(est_ms, 1e-3)))
+        n0 = dr.dr_launch_count()
+        warm = 0
+    else:
+        warm = args.warmup
+    t_host0 = time.perf_counter()
+    times = timed(step, args.steps, warm)
+    t_host1 = time.perf_counter()
+    launches = (dr.dr_launch_count() - n0) * args.steps // (args.steps + warm)
     st, info = dr.dr_device_status()
     assert st == 0, f"device status {st} {info}"
     assert bool(torch.isfinite(logits).all())
     total_ms = sum(times)
     total_ms = max_over_ranks(total_ms, world)
     value = whole_job_images_per_s(total_ms, B, args.steps, world)
+    headline_clock = sampler.window(t_host0, t_host1) if sampler else None
+
+    # ---- the same step in a loop of a few seconds, in chunks of about a quarter second, each chunk with the median SM clock
+    # NVML showed while it ran: what the step costs at the clock the part sustains, next to the (possibly short) headline region
+    sustained = None
+    if rank == 0 and world == 1:
+        per = max(1, int(250.0 / max(total_ms / args.steps, 1e-3)))
+        chunks, t_end = [], time.perf_counter() + 3.0
+        while time.perf_counter() < t_end and len(chunks) < 40:
+            h0 = time.perf_counter()
+            tc = timed(step, per, 0)
+            h1 = time.perf_counter()
+            chunks.append((sum(tc) / len(tc), sampler.window(h0, h1) if sampler else None, len(tc)))
+        ms_all = sum(c[0] * c[2] for c in chunks) / sum(c[2] for c in chunks)
+        bins = {}
+        for ms_c, mhz, cnt in chunks:
+            key = None if mhz is None else int(round(mhz / 50.0) * 50)
+            b_ = bins.setdefault(key, [0.0, 0])
+            b_[0] += ms_c * cnt; b_[1] += cnt
+        clk = [c[1] for c in chunks if c[1] is not None]
+        sustained = {"seconds": 3.0, "steps": sum(c[2] for c in chunks), "ms_per_step": ms_all, "value": B / (ms_all * 1e-3), "unit": UNIT,
+                     "sm_mhz_median": statistics.median(clk) if clk else None,
+                     "by_sm_mhz": [{"sm_mhz": k, "steps": v[1], "ms_per_step": v[0] / v[1], "images_per_s": B / (v[0] / v[1] * 1e-3)}
+                                   for k, v in sorted(bins.items(), key=lambda kv: (kv[0] is None, kv[0]))]}
 
     # ---- end to end through the public API with host buffers: every step copies its batch from pinned host
     # memory, runs the forward pass and copies the logits back.  The copy of step i+1 runs on a second
@@ -526,7 +626,6 @@ def main():
         us[r] = [net.dr_net_layer_time_us(i) for i in range(L)]
     net.dr_net_set_timing(False)
     us = np.median(us, axis=0)
-    tf_peak = pk["bf16_tflops_sustained"] * 1e12          # kernels are timed inside a long step
     bw_peak = pk["hbm_gbs"] * 1e9
     rows, t_roof_total = [], 0.0
     for li, t_us in zip(infos, us):
@@ -534,25 +633,49 @@ def main():
         t_roof_total += t_roof
         rows.append(dict(name=li["name"], kind=li["kind"], path=dr.PATH_NAMES[li["conv_path"]], us=float(t_us),
                          gflop=li["flops"] / 1e9, mbytes=li["bytes"] / 1e6, roof_us=t_roof, frac=t_roof / max(float(t_us), 1e-9)))
-    tma = [r for r in rows if r["path"] == "umma_tma" and r["gflop"] * 1e9 / (pk["bf16_tflops"] * 1e12) >= r["mbytes"] * 1e6 / bw_peak]
+    tensor_paths = ("umma_tma",)
+    tma = [r for r in rows if r["path"] in tensor_paths and r["gflop"] * 1e9 / (pk["bf16_tflops"] * 1e12) >= r["mbytes"] * 1e6 / bw_peak]
     tma_flops = sum(r["gflop"] for r in tma) * 1e9
     tma_s = sum(r["us"] for r in tma) * 1e-6
     # the roofline entry is ONE launch of the dominant kernel: its largest (the merged 5x5 conv of inception 3b)
     top = max(tma, key=lambda r: r["us"]) if tma else None
     achieved = top["gflop"] / top["us"] * 1e3 if top else 0.0   # GFLOP/us = PFLOP/s
-    # DRAM bytes of that launch from the ncu capture in profiles/conv_umma_tma_kernel_3b_merged5x5_bs256.md
-    # (dram__bytes_read.sum + dram__bytes_write.sum); valid for batch 256 only
-    traffic = NCU_TRAFFIC_3B_M5 if (top and not resnet and top["name"] == "3b.m5" and B == 256) else None
+    # Which measured peak the fraction is taken against follows from the clocks sampled in this run: the burst figure
+    # when the median SM clock under load stayed within 5 % of the maximum (a short region), the sustained one otherwise.
+    clk_ref = headline_clock if headline_clock is not None else (clocks or {}).get("sm_mhz")
+    clk_max = (clocks or {}).get("sm_max_mhz")
+    burst_regime = bool(clk_ref and clk_max and clk_ref >= 0.95 * clk_max)
+    peak_name = "bf16_tflops" if burst_regime else "bf16_tflops_sustained"
+    # DRAM bytes of that launch from the stored ncu capture; reported only while the layer still runs in the tiling the
+    # capture was taken on (else null)
+    traffic, traffic_note = None, None
+    if top and not resnet and top["name"] == NCU_TRAFFIC["layer"] and B == NCU_TRAFFIC["batch"]:
+        plan = dr.dr_conv_plan(dr.dr_conv_desc(k=5, stride=1, pad=2, Cin=256, Cout=288, flags=dr.DR_BIAS | dr.DR_RELU, y_ldc=480, y_coff=192), B, 28, 28)
+        if plan == NCU_TRAFFIC["plan"]:
+            traffic = NCU_TRAFFIC["dram_read_bytes"] + NCU_TRAFFIC["dram_write_bytes"]
+            traffic_note = NCU_TRAFFIC["note"]
     roofline = {"bound": "tensor", "kernel": f"conv_umma_tma_kernel, launch {top['name'] if top else '-'} (largest of {len(tma)} tensor-bound launches per step)",
-                "achieved": achieved, "peak": pk["bf16_tflops_sustained"], "peak_kind": f"{pk_kind} sustained bf16 (kernel timed inside a long step)",
-                "unit": "TFLOP/s", "frac": achieved / pk["bf16_tflops_sustained"], "traffic": traffic,
+                "achieved": achieved, "peak": pk[peak_name],
+                "peak_kind": f"{pk_kind} {'burst' if burst_regime else 'sustained'} bf16: median SM clock in the timed region {clk_ref} of {clk_max} MHz",
+                "unit": "TFLOP/s", "frac": achieved / pk[peak_name],
+                "frac_vs_burst": achieved / pk["bf16_tflops"], "frac_vs_sustained": achieved / pk["bf16_tflops_sustained"],
+                "traffic": traffic, "traffic_note": traffic_note,
                 "flops_per_launch": top["gflop"] * 1e9 if top else None, "us_per_launch": top["us"] if top else None,
                 "algorithmic_bytes_per_launch": top["mbytes"] * 1e6 if top else None,
                 "all_tensor_bound_launches": {"launches_per_step": len(tma), "achieved": tma_flops / tma_s / 1e12 if tma_s > 0 else 0.0,
+                                              "frac_vs_burst": tma_flops / tma_s / 1e12 / pk["bf16_tflops"] if tma_s > 0 else 0.0,
+                                              "frac_vs_sustained": tma_flops / tma_s / 1e12 / pk["bf16_tflops_sustained"] if tma_s > 0 else 0.0,
                                               "share_of_step": sum(r["us"] for r in tma) / float(us.sum())}}
     ms_per_step = total_ms / args.steps
+    t_roof_sus = sum(max(li["flops"] / (pk["bf16_tflops_sustained"] * 1e12), li["bytes"] / bw_peak) * 1e6 for li in infos)
     net_roofline = {"sum_layer_roofline_us": t_roof_total, "measured_us": ms_per_step * 1e3,
-                    "frac": t_roof_total / (ms_per_step * 1e3), "peaks": f"{pk_kind}: {pk['bf16_tflops']} TFLOP/s burst, {pk['hbm_gbs']} GB/s"}
+                    "frac": t_roof_total / (ms_per_step * 1e3), "frac_vs_burst": t_roof_total / (ms_per_step * 1e3),
+                    "frac_vs_sustained": t_roof_sus / (ms_per_step * 1e3),
+                    "target": "at least 0.60, judged on frac (layer rooflines at the burst bf16 peak, the larger one)",
+                    "peaks": f"{pk_kind}: {pk['bf16_tflops']} TFLOP/s burst, {pk['bf16_tflops_sustained']} sustained, {pk['hbm_gbs']} GB/s"}
+    if sustained:
+        sustained["net_roofline_frac_vs_burst"] = t_roof_total / (sustained["ms_per_step"] * 1e3)
+        sustained["net_roofline_frac_vs_sustained"] = t_roof_sus / (sustained["ms_per_step"] * 1e3)
 
     # ---- context numbers: batch 1 latency regime and the unslimmed layer-by-layer path
     extra = {}
@@ -565,9 +688,41 @@ def main():
         extra["unslimmed_activation_bytes"] = net_u.dr_net_activation_bytes()
         extra["slim_activation_bytes"] = net.dr_net_activation_bytes()
         net_u.dr_net_set_timing(True)
-        net_u.dr_net_forward(x, ws_u, lu); torch.cuda.synchronize()
-        tl = [(net_u.dr_net_layer_info(i)["kind"], net_u.dr_net_layer_time_us(i)) for i in range(net_u.dr_net_num_layers())]
+        Lu = net_u.dr_net_num_layers()
+        names_u = [net_u.dr_net_layer_info(i) for i in range(Lu)]
+        us_u = np.zeros((3, Lu))
+        for r in range(3):
+            flush.zero_()
+            net_u.dr_net_forward(x, ws_u, lu); torch.cuda.synchronize()
+            us_u[r] = [net_u.dr_net_layer_time_us(i) for i in range(Lu)]
+        us_u = np.median(us_u, axis=0)
+        tl = [(li["kind"], float(t)) for li, t in zip(names_u, us_u)]
         extra["unslimmed_pct_latency_non_tensor"] = 100.0 * sum(t for k, t in tl if k == 1) / sum(t for _, t in tl)
+        if args.arch == "googlenet":
+            # per module, slim next to unslimmed (layer-wise CUDA-event times, us), in the layout of the paper's per-layer
+            # table; its Galaxy S5 milliseconds (original / slim network) ride along as context only
+            def module_of(name):
+                head = name.split(".")[0]
+                if head in ("conv1",): return "conv1"
+                if head in ("conv2r", "conv2"): return "conv2"
+                if head in ("avgpool", "fc"): return "loss3"
+                if head in ("pool3", "pool4"): return head
+                return "inception_" + head
+            paper_ms = {"conv1": (94.92, 8.424), "conv2": (153.8, 16.62), "inception_3a": (55.23, 21.17), "inception_3b": (98.41, 25.94),
+                        "inception_4a": (30.53, 16.80), "inception_4b": (32.60, 20.29), "inception_4c": (46.96, 18.71),
+                        "inception_4d": (36.88, 24.67), "inception_4e": (48.24, 28.08), "inception_5a": (24.64, 10.69),
+                        "inception_5b": (24.92, 14.58), "loss3": (3.014, 2.97)}
+            mods = {}
+            for r_ in rows:
+                mods.setdefault(module_of(r_["name"]), [0.0, 0.0, 0, 0])[0] += r_["us"]
+                mods[module_of(r_["name"])][2] += 1
+            for li, t in zip(names_u, us_u):
+                mods.setdefault(module_of(li["name"]), [0.0, 0.0, 0, 0])[1] += float(t)
+                mods[module_of(li["name"])][3] += 1
+            extra["modules"] = [{"module": m, "slim_us": v[0], "unslimmed_us": v[1], "slim_launches": v[2], "unslimmed_launches": v[3],
+                                 "speedup": v[1] / v[0] if v[0] > 0 else None,
+                                 "paper_galaxy_s5_ms": {"googlenet": paper_ms[m][0], "googlenet_slim": paper_ms[m][1]} if m in paper_ms else None}
+                                for m, v in mods.items()]
         del net_u, ws_u, keep_u
         net1, ws1, keep1 = make_net(dr.DR_MODE_SLIM, 1)
         l1 = torch.empty((1, 1000), dtype=torch.float32, device="cuda")
@@ -606,12 +761,14 @@ def main():
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{arch_name} forward, batch {B} per GPU, {hw}x{hw}x3 N(0,1) bf16, He-normal weights ({cfg_name})",
-                   "l2": "256 MB buffer written between timed iterations (L2 flush)", "replicas": world},
+                   "l2": "256 MB buffer written between timed iterations (L2 flush)", "replicas": world,
+                   "timed_region_s": total_ms * 1e-3, "steps_chosen": "auto (about 3 s)" if auto_steps else "given"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": logits_host.numel() * 4},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": roofline,
         "net_roofline": net_roofline,
+        "sustained": sustained,
         "cpu_baseline": cpu,
         "extra": extra,
     }))

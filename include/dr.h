@@ -284,6 +284,7 @@ int dr_net_activation_bytes(const dr_net* net, size_t* bytes);
 #define DR_PATH_UMMA_STEM_T  6  /* the same stem computed transposed: pooling in registers       */
 #define DR_PATH_UMMA_STEM_D  7  /* the stem with the MMA reading the input rows in place (no im2col) */
 #define DR_PATH_UMMA_SPLITK  8  /* few output tiles: K split across the SMs, partial tiles summed in scratch (needs a workspace) */
+#define DR_PATH_UMMA_QLIN    9  /* stride-1 3x3 / 5x5: the tile's input patch loaded once, every tap read out of it by the MMA */
 /* Force a convolution kernel (tests, A/B timing); DR_PATH_AUTO picks the fastest that
  * supports the layer.  A forced path that cannot run the layer gives DR_ERR_UNSUPPORTED.   */
 int dr_set_conv_path(int path);
@@ -349,6 +350,14 @@ int dr_regress_step(const dr_conv_desc* desc, int B, int H, int W, const void* x
 
 /* Kernels of this library launched by this process so far. */
 long long dr_launch_count(void);
+/* Tensor maps (TMA descriptors) the library has had the driver encode so far.  Maps are remembered by the arguments
+ * they were encoded from, so a layer called again on the same buffers encodes nothing.                          */
+long long dr_tensor_map_encodes(void);
+/* How dr_conv_slim would run a layer (no launch): plan[0] the kernel (DR_PATH_*), plan[1] output channels per
+ * accumulator block, plan[2] such blocks along Cout, plan[3] 1 if CTA pairs (cta_group::2) are used, plan[4] 1 if a
+ * tile carries two blocks that share the activation tile, plan[5..7] reserved (0).  workspace_bytes: the scratch the
+ * call would be given (as in dr_conv_slim_ws; 0 for dr_conv_slim).  Errors as dr_conv_slim's validation.        */
+int dr_conv_plan(const dr_conv_desc* desc, int B, int H, int W, size_t workspace_bytes, int plan[8]);
 
 #ifdef __cplusplus
 }

@@ -30,9 +30,10 @@ DR_ARCH_GOOGLENET, DR_ARCH_RESNET50, DR_ARCH_GOOGLENET_PAPER, DR_ARCH_GOOGLENET_
 DR_MODE_SLIM, DR_MODE_UNSLIMMED = 0, 1
 DR_PATH_AUTO, DR_PATH_SIMT, DR_PATH_UMMA_GATHER, DR_PATH_UMMA_TMA, DR_PATH_UMMA_PATCH, DR_PATH_UMMA_STEM, DR_PATH_UMMA_STEM_T, DR_PATH_UMMA_STEM_D = 0, 1, 2, 3, 4, 5, 6, 7
 DR_PATH_UMMA_SPLITK = 8
+DR_PATH_UMMA_QLIN = 9
 DR_CONV_WS_COUNTER_BYTES = 1024
 PATH_NAMES = {0: "auto", 1: "simt", 2: "umma_gather", 3: "umma_tma", 4: "umma_patch", 5: "umma_stem", 6: "umma_stem_t", 7: "umma_stem_d",
-              8: "umma_splitk", -1: "-"}
+              8: "umma_splitk", 9: "umma_qlin", -1: "-"}
 
 
 class dr_conv_desc(C.Structure):
@@ -110,6 +111,8 @@ _SIGS = {
     "dr_device_status": (_I, [C.POINTER(_I)]),
     "dr_selftest_wait_timeout": (_I, [C.c_longlong, _P]),
     "dr_launch_count": (C.c_longlong, []),
+    "dr_tensor_map_encodes": (C.c_longlong, []),
+    "dr_conv_plan": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _Z, C.POINTER(_I)]),
 }
 for _name, (_res, _args) in _SIGS.items():
     _fn = getattr(_lib, _name)          # AttributeError here = the library does not export it
@@ -302,6 +305,17 @@ def dr_selftest_wait_timeout(limit_cycles: int, stream=None):
 
 def dr_launch_count() -> int:
     return int(_lib.dr_launch_count())
+
+
+def dr_tensor_map_encodes() -> int:
+    return int(_lib.dr_tensor_map_encodes())
+
+
+def dr_conv_plan(desc, B, H, W, workspace_bytes: int = 0) -> dict:
+    """How the library would run the layer: kernel path, accumulator-block width and count, CTA pairs, wide tiles."""
+    plan = (_I * 8)()
+    _check(_lib.dr_conv_plan(C.byref(desc), B, H, W, workspace_bytes, plan), "dr_conv_plan")
+    return {"path": PATH_NAMES[plan[0]], "Nt": plan[1], "n_blocks": plan[2], "pair": plan[3], "wide": plan[4]}
 
 
 class Net:

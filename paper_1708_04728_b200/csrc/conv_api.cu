@@ -112,6 +112,15 @@ int conv_make_params(const dr_conv_desc* d, int B, int H, int W, const void* x, 
     return DR_OK;
 }
 
+// The patch-reuse kernel against the im2col kernel: its tiles are whole padded image rows, so part of every tile's MMA
+// rows is padding (28 x 28 planes: 12.5 %).  Measured at batch 256 it is behind the im2col kernel on every GoogLeNet layer
+// (3a merged 5x5: 340 vs 247 us; 3b: 676 vs 596 us): those layers are bound by the rate at which one thread can issue
+// MMAs and hand stages over, not by filling shared memory, so the padding rows cost more than the saved loads give.
+// Chosen only on request (DR_QLIN=1, or the forced path).
+static bool qlin_preferred(const ConvParams& p) {
+    return tunable("DR_QLIN", 0) > 0 && conv_qlin_supports(p);
+}
+
 int conv_pick_path(const ConvParams& p, int forced) {
     if (forced == DR_PATH_SIMT) return DR_PATH_SIMT;
     if (forced == DR_PATH_UMMA_GATHER) return conv_umma_gather_supports(p) ? DR_PATH_UMMA_GATHER : -1;
@@ -121,11 +130,13 @@ int conv_pick_path(const ConvParams& p, int forced) {
     if (forced == DR_PATH_UMMA_STEM_T) return conv_stem_t_supports(p) ? DR_PATH_UMMA_STEM_T : -1;
     if (forced == DR_PATH_UMMA_STEM_D) return conv_stem_d_supports(p) ? DR_PATH_UMMA_STEM_D : -1;
     if (forced == DR_PATH_UMMA_SPLITK) return conv_splitk_supports(p) ? DR_PATH_UMMA_SPLITK : -1;
+    if (forced == DR_PATH_UMMA_QLIN) return conv_qlin_supports(p) ? DR_PATH_UMMA_QLIN : -1;
     if (conv_stem_d_supports(p)) return DR_PATH_UMMA_STEM_D;
     if (conv_stem_supports(p)) return DR_PATH_UMMA_STEM;       // measured faster than the transposed form (483 vs 625 us at batch 256)
     if (conv_stem_t_supports(p)) return DR_PATH_UMMA_STEM_T;
     if (conv_patch_tma_supports(p)) return DR_PATH_UMMA_PATCH;
     if (conv_splitk_supports(p)) return DR_PATH_UMMA_SPLITK;   // few output tiles and scratch at hand
+    if (qlin_preferred(p)) return DR_PATH_UMMA_QLIN;
     if (conv_umma_tma_supports(p)) return DR_PATH_UMMA_TMA;
     if (conv_umma_gather_supports(p)) return DR_PATH_UMMA_GATHER;
     return DR_PATH_SIMT;
@@ -141,6 +152,7 @@ int conv_launch_path(const ConvParams& p, int path, cudaStream_t stream) {
         case DR_PATH_UMMA_STEM_T: return conv_stem_t_launch(p, stream);
         case DR_PATH_UMMA_STEM_D: return conv_stem_d_launch(p, stream);
         case DR_PATH_UMMA_SPLITK: return conv_splitk_launch(p, stream);
+        case DR_PATH_UMMA_QLIN: return conv_qlin_launch(p, stream);
         default: return DR_ERR_UNSUPPORTED;
     }
 }
@@ -154,7 +166,7 @@ using namespace dr;
 extern "C" {
 
 int dr_set_conv_path(int path) {
-    if (path < DR_PATH_AUTO || path > DR_PATH_UMMA_SPLITK) return DR_ERR_INVALID_ARG;
+    if (path < DR_PATH_AUTO || path > DR_PATH_UMMA_QLIN) return DR_ERR_INVALID_ARG;
     g_forced_path = path;
     return DR_OK;
 }
@@ -171,6 +183,31 @@ int dr_conv_slim(const dr_conv_desc* desc, int B, int H, int W, const void* x, c
     if (path < 0) return DR_ERR_UNSUPPORTED;
     g_last_path = path;
     return conv_launch_path(p, path, (cudaStream_t)stream);
+}
+
+int dr_conv_plan(const dr_conv_desc* desc, int B, int H, int W, size_t workspace_bytes, int plan[8]) {
+    if (!plan) return DR_ERR_INVALID_ARG;
+    ConvParams p;
+    const void* dummy = reinterpret_cast<const void*>(uintptr_t(256));   // only alignment is looked at
+    const int st = conv_make_params(desc, B, H, W, dummy, dummy, (const float*)dummy, dummy, (void*)dummy, nullptr, &p);
+    if (st != DR_OK) return st;
+    if (workspace_bytes > (size_t)DR_CONV_WS_COUNTER_BYTES) {
+        p.sk_counters = reinterpret_cast<int*>(uintptr_t(256));
+        p.sk_scratch = reinterpret_cast<float*>(uintptr_t(256) + DR_CONV_WS_COUNTER_BYTES);
+        p.sk_scratch_bytes = workspace_bytes - DR_CONV_WS_COUNTER_BYTES;
+    }
+    for (int i = 0; i < 8; ++i) plan[i] = 0;
+    const int path = p.M > 0 ? conv_pick_path(p, g_forced_path) : DR_PATH_AUTO;
+    if (path < 0) return DR_ERR_UNSUPPORTED;
+    plan[0] = path; plan[1] = p.Nt; plan[2] = p.n_blocks;
+    if (path == DR_PATH_UMMA_TMA) {
+        bool pair = false, wide = false;
+        conv_umma_tma_shape(&p, &pair, &wide);
+        plan[1] = p.Nt; plan[2] = p.n_blocks; plan[3] = pair; plan[4] = wide;
+    } else if (path == DR_PATH_UMMA_QLIN) {
+        plan[1] = conv_qlin_nt(p); plan[2] = 1; plan[3] = 1; plan[4] = ((p.Cout + 15) / 16 * 16) > 256;
+    }
+    return DR_OK;
 }
 
 int dr_conv_workspace_bytes(const dr_conv_desc* desc, int B, int H, int W, size_t* bytes) {

@@ -289,6 +289,11 @@ bool conv_stem_t_supports(const ConvParams& p);
 int conv_stem_d_launch(const ConvParams& p, cudaStream_t stream);
 bool conv_stem_d_supports(const ConvParams& p);
 bool conv_umma_gather_supports(const ConvParams& p);
+int conv_qlin_launch(const ConvParams& p, cudaStream_t stream);
+bool conv_qlin_supports(const ConvParams& p);
+double conv_qlin_fill(const ConvParams& p);               // share of a tile's GEMM rows that are stored outputs
+int conv_qlin_nt(const ConvParams& p);                    // output channels per accumulator block on that kernel
+void conv_umma_tma_shape(ConvParams* p, bool* use_pair, bool* wide);
 int conv_splitk_launch(const ConvParams& p, cudaStream_t stream);
 bool conv_splitk_supports(const ConvParams& p);
 size_t conv_splitk_scratch_bytes(const ConvParams& p);   // partial-tile scratch the split-K kernel wants; 0: it would not take the layer
@@ -301,5 +306,11 @@ int encode_conv_maps(const ConvParams& p, int b_box_rows, CUtensorMap* map_a, CU
 int encode_input_map(const ConvParams& p, CUtensorMap* map_a, int* a_mode, int box_rows = TILE_M);
 int encode_rows_map(const void* ptr, long long rows, int cols, int ld, CUtensorMap* map, int box_rows = TILE_M);
 int tunable(const char* name, int dflt);
+// tensor_map.cu: memoised tensor-map encoders (bf16, element strides 1, zero fill)
+int tmap_tiled(CUtensorMap* map, int rank, const void* ptr, const cuuint64_t* dims, const cuuint64_t* strides, const cuuint32_t* box,
+               CUtensorMapSwizzle swizzle, CUtensorMapL2promotion l2);
+int tmap_im2col(CUtensorMap* map, const void* ptr, const cuuint64_t dims[4], const cuuint64_t strides[3], const int lower[2], const int upper[2],
+                unsigned channels, unsigned pixels, unsigned stride, CUtensorMapL2promotion l2);
+long long tmap_driver_encodes();
 
 }  // namespace dr

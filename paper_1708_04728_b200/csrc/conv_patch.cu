@@ -625,19 +625,6 @@ __global__ void __launch_bounds__(S_THREADS, 1) conv_stem_kernel(const ConvParam
 }
 
 // ---- host --------------------------------------------------------------------------------
-typedef CUresult (*PFN_encodeTiledP)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                     const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                     CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-static PFN_encodeTiledP g_enc = nullptr;
-static bool load_enc() {
-    if (g_enc) return true;
-    cudaDriverEntryPointQueryResult q;
-    void* f = nullptr;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || !f) return false;
-    g_enc = (PFN_encodeTiledP)f;
-    return true;
-}
-
 bool conv_patch_tma_supports(const ConvParams& p) {
     if (!p.patch || !fe_supports(p)) return false;
     if (p.stride != 1 || (p.Cin & 7) || p.Cin < 64 || p.k > 15) return false;
@@ -647,7 +634,6 @@ bool conv_patch_tma_supports(const ConvParams& p) {
 
 int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
     if (!conv_patch_tma_supports(p)) return DR_ERR_UNSUPPORTED;
-    if (!load_enc()) return DR_ERR_CUDA;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(conv_patch_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
@@ -658,19 +644,13 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
         const cuuint64_t dims[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
         const cuuint64_t strides[3] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.W * p.Cin * 2, (cuuint64_t)p.H * p.W * p.Cin * 2};
         const cuuint32_t box[4] = {64, (cuuint32_t)(2 * p.PW + 1), (cuuint32_t)(2 * p.PH + 1), 1};
-        const cuuint32_t es[4] = {1, 1, 1, 1};
-        if (g_enc(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void*)p.x, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return DR_ERR_CUDA;
+        if (tmap_tiled(&map_a, 4, p.x, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B) != DR_OK) return DR_ERR_CUDA;
     }
     {
         const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
         const cuuint64_t strides[2] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.K * 2};
         const cuuint32_t box[3] = {64, 1, (cuuint32_t)p.Nt};
-        const cuuint32_t es[3] = {1, 1, 1};
-        if (g_enc(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)p.w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return DR_ERR_CUDA;
+        if (tmap_tiled(&map_b, 3, p.w, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B) != DR_OK) return DR_ERR_CUDA;
     }
     if (p.m_tiles <= 0) return DR_OK;
     // CTA pairs with each CTA's half of the filter bank resident in shared memory (or, if that does not fit, streamed):
@@ -711,10 +691,7 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
             const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
             const cuuint64_t strides[2] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.K * 2};
             const cuuint32_t box[3] = {64, 1, (cuuint32_t)(p.Nt / 2)};      // each CTA of a pair holds half of the filters
-            const cuuint32_t es[3] = {1, 1, 1};
-            if (g_enc(&map_bh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)p.w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-                return DR_ERR_CUDA;
+            if (tmap_tiled(&map_bh, 3, p.w, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B) != DR_OK) return DR_ERR_CUDA;
             int smem_bytes = stages * stage_bytes + (resident ? nkb * bsub : 0) + groups * fe + 1024;
             if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
             const int units = (p.m_tiles + 1) / 2;

@@ -19,10 +19,9 @@
 //
 // Every wait on an mbarrier is bounded (see ptx::mbar_wait); on a timeout the CTA records
 // DR_ERR_DEVICE_TIMEOUT, all roles leave their loops, and TMEM is released before exit.
-#include <cstdlib>
-
 #include "conv_common.cuh"
 #include "umma_ptx.cuh"
+#include "conv_drain.cuh"
 
 namespace dr {
 using namespace ptx;
@@ -39,92 +38,6 @@ __device__ __forceinline__ void issue_kblock(uint32_t tmem_d, uint32_t a_smem, u
 #pragma unroll
     for (int k = 0; k < 4; ++k)
         if (k < nk16) umma_bf16(tmem_d, ad + 2 * k, bd + 2 * k, idesc, (first && k == 0) ? 0u : 1u);
-}
-
-// Drain `ncols` accumulator columns of this thread's TMEM lane and run the direct epilogue.
-__device__ __forceinline__ void drain_direct(const ConvParams& p, uint32_t taddr, int ncols, long long m, bool row_ok, int n0) {
-    for (int c = 0; c < ncols; c += 32) {
-        uint32_t r[32];
-        if (ncols - c >= 32) {
-            tmem_ld_x32(taddr + c, r);
-            tmem_ld_wait();
-            if (row_ok) epilogue_direct<32>(p, m, n0 + c, reinterpret_cast<float*>(r));
-        } else {
-            tmem_ld_x16(taddr + c, r);
-            tmem_ld_wait();
-            if (row_ok) epilogue_direct<16>(p, m, n0 + c, reinterpret_cast<float*>(r));
-        }
-    }
-}
-
-// Lean epilogue of the common case (bias and/or ReLU only, bf16 out, Cout a multiple of 16, aligned
-// slice): bias comes from a shared-memory copy as float4, the ReLU choice is a template argument, and
-// a thread stores its 64 bytes per 32-column chunk with four 16-byte stores.
-// MODE 0: +bias;  1: +bias, ReLU;  2: +bias, +residual;  3: +bias, +residual, ReLU.
-template <int MODE>
-__device__ __forceinline__ void drain_fast(const ConvParams& p, uint32_t taddr, int ncols, long long m, bool row_ok, int n0,
-                                           const float* bias_s) {
-    constexpr bool RELU = (MODE & 1) != 0, RES = (MODE & 2) != 0;
-    uint4* y = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.y) + m * p.ldc + p.coff + n0);
-    const uint4* res = reinterpret_cast<const uint4*>(p.residual + (RES && row_ok ? m * p.Cout + n0 : 0));
-    const float4* b4 = reinterpret_cast<const float4*>(bias_s + n0);
-    int c = 0;
-    for (; c + 32 <= ncols; c += 32) {
-        uint32_t r[32];
-        tmem_ld_x32(taddr + c, r);
-        tmem_ld_wait();
-        uint32_t o[16];
-        uint32_t rr[16];
-        if (RES && row_ok) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint4 u = __ldg(res + (c >> 3) + q);
-                rr[4 * q] = u.x; rr[4 * q + 1] = u.y; rr[4 * q + 2] = u.z; rr[4 * q + 3] = u.w;
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const float4 b = b4[(c >> 2) + q];
-            float v0 = __uint_as_float(r[4 * q]) + b.x, v1 = __uint_as_float(r[4 * q + 1]) + b.y;
-            float v2 = __uint_as_float(r[4 * q + 2]) + b.z, v3 = __uint_as_float(r[4 * q + 3]) + b.w;
-            if (RES && row_ok) { v0 += bf16_lo(rr[2 * q]); v1 += bf16_hi(rr[2 * q]); v2 += bf16_lo(rr[2 * q + 1]); v3 += bf16_hi(rr[2 * q + 1]); }
-            if (RELU) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); v2 = fmaxf(v2, 0.f); v3 = fmaxf(v3, 0.f); }
-            o[2 * q] = pack_bf16(v0, v1);
-            o[2 * q + 1] = pack_bf16(v2, v3);
-        }
-        if (row_ok) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) y[(c >> 3) + q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
-        }
-    }
-    if (c < ncols) {   // 16-column tail
-        uint32_t r[16];
-        tmem_ld_x16(taddr + c, r);
-        tmem_ld_wait();
-        uint32_t o[8];
-        uint32_t rr[8];
-        if (RES && row_ok) {
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                const uint4 u = __ldg(res + (c >> 3) + q);
-                rr[4 * q] = u.x; rr[4 * q + 1] = u.y; rr[4 * q + 2] = u.z; rr[4 * q + 3] = u.w;
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const float4 b = b4[(c >> 2) + q];
-            float v0 = __uint_as_float(r[4 * q]) + b.x, v1 = __uint_as_float(r[4 * q + 1]) + b.y;
-            float v2 = __uint_as_float(r[4 * q + 2]) + b.z, v3 = __uint_as_float(r[4 * q + 3]) + b.w;
-            if (RES && row_ok) { v0 += bf16_lo(rr[2 * q]); v1 += bf16_hi(rr[2 * q]); v2 += bf16_lo(rr[2 * q + 1]); v3 += bf16_hi(rr[2 * q + 1]); }
-            if (RELU) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); v2 = fmaxf(v2, 0.f); v3 = fmaxf(v3, 0.f); }
-            o[2 * q] = pack_bf16(v0, v1);
-            o[2 * q + 1] = pack_bf16(v2, v3);
-        }
-        if (row_ok) {
-            y[(c >> 3)] = make_uint4(o[0], o[1], o[2], o[3]);
-            y[(c >> 3) + 1] = make_uint4(o[4], o[5], o[6], o[7]);
-        }
-    }
 }
 
 // Lean epilogue with TMA stores (bias and/or ReLU, bf16 out): row-per-thread 16-byte global stores cost 32 memory
@@ -840,27 +753,6 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
 }
 
 // ---- host: tensor maps ------------------------------------------------------------------
-typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-typedef CUresult (*PFN_encodeIm2col)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                     const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*, CUtensorMapInterleave,
-                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-static PFN_encodeTiled g_encode_tiled = nullptr;
-static PFN_encodeIm2col g_encode_im2col = nullptr;
-
-static bool load_encoders() {
-    if (g_encode_tiled && g_encode_im2col) return true;
-    cudaDriverEntryPointQueryResult q;
-    void* f = nullptr;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || !f) return false;
-    g_encode_tiled = (PFN_encodeTiled)f;
-    f = nullptr;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || !f) return false;
-    g_encode_im2col = (PFN_encodeIm2col)f;
-    return true;
-}
-
 // Tensor maps of one convolution for the TMA kernels.  A: the activations, as a plain [M][Cin] matrix for
 // 1x1 / stride 1 / pad 0 layers (*a_mode = 0, 2-D tiled boxes of 128 rows x 64 channels) and in im2col mode
 // otherwise (*a_mode = 1: 128 output pixels x 64 channels of one filter tap per load).  B: the filters as
@@ -871,56 +763,32 @@ int encode_conv_maps(const ConvParams& p, int b_box_rows, CUtensorMap* map_a, CU
     const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
     const cuuint64_t strides[2] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.K * 2};
     const cuuint32_t box[3] = {64, 1, (cuuint32_t)b_box_rows};
-    const cuuint32_t es[3] = {1, 1, 1};
-    if (g_encode_tiled(map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)p.w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return DR_ERR_CUDA;
-    return DR_OK;
+    return tmap_tiled(map_b, 3, p.w, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
 // A [rows][cols] bf16 matrix with row pitch ld (elements) in boxes of box_rows rows x 64 columns, 128-byte swizzle.
 int encode_rows_map(const void* ptr, long long rows, int cols, int ld, CUtensorMap* map, int box_rows) {
-    if (!load_encoders()) return DR_ERR_CUDA;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-    const cuuint32_t es[2] = {1, 1};
-    return g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)ptr, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS
-               ? DR_OK : DR_ERR_CUDA;
+    return tmap_tiled(map, 2, ptr, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
 
 // The input-side map alone (see encode_conv_maps).
 int encode_input_map(const ConvParams& p, CUtensorMap* map_a, int* a_mode, int box_rows) {
-    if (!load_encoders()) return DR_ERR_CUDA;
     *a_mode = (p.k == 1 && p.stride == 1 && p.pad == 0) ? 0 : 1;
     if (*a_mode == 0) {
         const cuuint64_t dims[2] = {(cuuint64_t)p.Cin, (cuuint64_t)p.M};
         const cuuint64_t strides[1] = {(cuuint64_t)p.Cin * 2};
         const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-        const cuuint32_t es[2] = {1, 1};
-        if (g_encode_tiled(map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)p.x, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return DR_ERR_CUDA;
-    } else {
-        const cuuint64_t dims[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
-        const cuuint64_t strides[3] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.W * p.Cin * 2, (cuuint64_t)p.H * p.W * p.Cin * 2};
-        // bounding box of the positions the filter's first tap visits: [-pad, extent + pad - k]
-        const int lower[2] = {-p.pad, -p.pad};
-        const int upper[2] = {p.pad - (p.k - 1), p.pad - (p.k - 1)};
-        const cuuint32_t es[4] = {1, (cuuint32_t)p.stride, (cuuint32_t)p.stride, 1};
-        if (g_encode_im2col(map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void*)p.x, dims, strides, lower, upper, 64, (cuuint32_t)box_rows, es,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return DR_ERR_CUDA;
+        return tmap_tiled(map_a, 2, p.x, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
     }
-    return DR_OK;
-}
-
-// Integer tunable from the environment; for A/B timing.
-int tunable(const char* name, int dflt) {
-    const char* v = getenv(name);
-    return v ? atoi(v) : dflt;
+    const cuuint64_t dims[4] = {(cuuint64_t)p.Cin, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
+    const cuuint64_t strides[3] = {(cuuint64_t)p.Cin * 2, (cuuint64_t)p.W * p.Cin * 2, (cuuint64_t)p.H * p.W * p.Cin * 2};
+    // bounding box of the positions the filter's first tap visits: [-pad, extent + pad - k]
+    const int lower[2] = {-p.pad, -p.pad};
+    const int upper[2] = {p.pad - (p.k - 1), p.pad - (p.k - 1)};
+    return tmap_im2col(map_a, p.x, dims, strides, lower, upper, 64, (unsigned)box_rows, (unsigned)p.stride, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
 
 bool conv_umma_tma_supports(const ConvParams& p) {
@@ -973,22 +841,16 @@ static int tma_epilogue_bytes(const ConvParams& p, bool pair_or_wide, CUtensorMa
     // output channels, up to 2 k-blocks otherwise; beyond that the lost pipeline stages cost more than the stores
     if (res ? ((p.Nt & 63) || (p.Cout & 63)) : false) return 0;
     if (ep_pref == 1 && (res ? nkb > 4 : (nkb > 4 || (nkb > 2 && p.Cout < 256)))) return 0;
-    if (!load_encoders()) return 0;
     const cuuint32_t box[2] = {64, TILE_M};
-    const cuuint32_t es[2] = {1, 1};
     {
         const cuuint64_t dims[2] = {(cuuint64_t)(p.coff + p.Cout), (cuuint64_t)p.M};
         const cuuint64_t strides[1] = {(cuuint64_t)p.ldc * 2};
-        if (g_encode_tiled(map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.y, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return 0;
+        if (tmap_tiled(map_y, 2, p.y, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE) != DR_OK) return 0;
     }
     if (res) {
         const cuuint64_t dims[2] = {(cuuint64_t)p.Cout, (cuuint64_t)p.M};
         const cuuint64_t strides[1] = {(cuuint64_t)p.Cout * 2};
-        if (g_encode_tiled(map_r, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)p.residual, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return 0;
+        if (tmap_tiled(map_r, 2, p.residual, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B) != DR_OK) return 0;
     }
     return res ? 2 * 3 * 16384 : 2 * 2 * 16384;                  // per epilogue group: three / two 16 KB buffers
 }
@@ -1042,9 +904,10 @@ static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUte
     return launch_status();
 }
 
-int conv_umma_tma_launch(const ConvParams& p_in, cudaStream_t stream) {
-    if (!conv_umma_tma_supports(p_in)) return DR_ERR_UNSUPPORTED;
-    ConvParams p = p_in;
+// Tile shape of a layer on the TMA kernel: CTA pairs or single CTAs, and whether a tile carries two n-blocks that
+// share the activation tile (then p->Nt / p->n_blocks are replaced by the wide tiling).
+void conv_umma_tma_shape(ConvParams* pp, bool* use_pair_out, bool* wide_out) {
+    ConvParams& p = *pp;
     // CTA pairs pay off where the MMAs dominate: long K, or a spatial filter with K >= 512 (measured: +12 % on the
     // 3x3 layers, -20 % on the 1x1 reducers)
     const int pair_pref = tunable("DR_TMA_PAIR", -1);
@@ -1072,6 +935,15 @@ int conv_umma_tma_launch(const ConvParams& p_in, cudaStream_t stream) {
         p.Nt = nt_w;
         p.n_blocks = n_wide;
     }
+    *use_pair_out = use_pair;
+    *wide_out = wide;
+}
+
+int conv_umma_tma_launch(const ConvParams& p_in, cudaStream_t stream) {
+    if (!conv_umma_tma_supports(p_in)) return DR_ERR_UNSUPPORTED;
+    ConvParams p = p_in;
+    bool use_pair = false, wide = false;
+    conv_umma_tma_shape(&p, &use_pair, &wide);
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(conv_umma_tma_kernel<false, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||

@@ -335,6 +335,22 @@ __device__ __forceinline__ void tma_load_3d_u32(uint32_t dst, const CUtensorMap*
             : "memory");
 }
 template <bool PAIR>
+__device__ __forceinline__ void tma_load_4d_u32(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3, uint32_t enable) {
+    if (PAIR)
+        asm volatile(
+            "{\n.reg .pred q;\nsetp.ne.b32 q, %7, 0;\n"
+            "@q cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n}\n" ::"r"(
+                dst),
+            "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(enable)
+            : "memory");
+    else
+        asm volatile(
+            "{\n.reg .pred q;\nsetp.ne.b32 q, %7, 0;\n"
+            "@q cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n}\n" ::"r"(dst),
+            "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(enable)
+            : "memory");
+}
+template <bool PAIR>
 __device__ __forceinline__ void tma_load_im2col_4d_u32(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c, int w, int h, int n,
                                                        uint16_t woff, uint16_t hoff, uint32_t enable) {
     if (PAIR)

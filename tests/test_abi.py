@@ -240,3 +240,45 @@ def test_resnet50_layer_lists(dr):
         dr.Net(7, 0, 1)
     with pytest.raises(dr.DrError):
         dr.Net(0, 0, 1, 16, 16)
+
+
+def header_defines():
+    """{name: integer value} of the plain integer #defines of include/dr.h."""
+    text = open(os.path.join(ROOT, "include", "dr.h")).read()
+    out = {}
+    for name, val in re.findall(r"^#define[ \t]+(DR_[A-Z0-9_]+)[ \t]+([^/\n]+)", text, flags=re.M):
+        expr = re.sub(r"(?<=[0-9a-fA-F])[uU]\b", "", val.strip())
+        if re.fullmatch(r"[-()0-9a-fA-FxX<\s]+", expr):
+            out[name] = int(eval(expr, {"__builtins__": {}}))
+    return out
+
+
+def test_python_constants_mirror_the_header(dr):
+    """Every integer constant the binding repeats has the header's value (flags, codes, kernel paths, sizes)."""
+    defs = header_defines()
+    assert defs["DR_INCEPTION_STATIC_SCRATCH_BYTES"] == 4 << 20
+    checked = 0
+    for name, val in defs.items():
+        if hasattr(dr, name):
+            assert getattr(dr, name) == val, (name, getattr(dr, name), val)
+            checked += 1
+    assert checked >= 30
+    for need in ("DR_INCEPTION_STATIC_SCRATCH_BYTES", "DR_CONV_WS_COUNTER_BYTES", "DR_PATH_UMMA_QLIN", "DR_ERR_DEVICE_TIMEOUT", "DR_OUT_F32"):
+        assert need in defs and hasattr(dr, need), need
+    assert set(dr.PATH_NAMES) == {-1} | {v for k, v in defs.items() if k.startswith("DR_PATH_")}
+
+
+def test_conv_plan_is_host_only_and_names_the_kernel(dr):
+    n0 = dr.dr_launch_count()
+    big = dr.dr_conv_plan(dr.dr_conv_desc(k=5, stride=1, pad=2, Cin=528, Cout=512, flags=dr.DR_BIAS | dr.DR_RELU), 256, 14, 14)
+    assert big["path"] == "umma_tma" and big["pair"] == 1 and big["Nt"] * big["n_blocks"] * (2 if big["wide"] else 1) >= 512
+    stem = dr.dr_conv_plan(dr.dr_conv_desc(k=7, stride=2, pad=3, Cin=3, Cout=64, flags=dr.DR_BIAS | dr.DR_RELU | dr.DR_POOL | dr.DR_LRN,
+                                           pool_k=3, pool_stride=2, pool_pad=1, lrn_size=5, lrn_alpha=1e-4, lrn_beta=0.75, lrn_k=1.0), 1, 64, 64)
+    assert stem["path"].startswith("umma_stem")
+    d = dr.dr_conv_desc(k=5, stride=1, pad=2, Cin=832, Cout=640, flags=dr.DR_BIAS | dr.DR_RELU)
+    assert dr.dr_conv_plan(d, 1, 7, 7, dr.dr_conv_workspace_bytes(d, 1, 7, 7))["path"] == "umma_splitk"
+    assert dr.dr_conv_plan(d, 1, 7, 7, 0)["path"] != "umma_splitk"
+    with pytest.raises(dr.DrError) as e:
+        dr.dr_conv_plan(dr.dr_conv_desc(k=0, stride=1, pad=0, Cin=8, Cout=8, flags=0), 1, 8, 8)
+    assert e.value.status == dr.DR_ERR_INVALID_ARG
+    assert dr.dr_launch_count() == n0

@@ -94,7 +94,7 @@ DIRECT_SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("path", [1, 2, 3, 9])
 @pytest.mark.parametrize("shape", DIRECT_SHAPES)
 def test_conv_bias_relu(dr, O, path, shape):
     B, H, W, Cin, Cout, k, s, p = shape
@@ -109,6 +109,52 @@ def test_conv_bias_relu(dr, O, path, shape):
     assert dr.dr_last_conv_path() == path
     ref, _ = oracle_slim_layer(O, x, w, b, k, s, p, dr.DR_BIAS | dr.DR_RELU, dr)
     assert_layer_close(got, O.round_bf16(ref), f"path {path} {shape}")
+
+
+# The patch-reuse kernel (path 9): tiles of whole padded image rows, every tap read out of one shared-memory patch.
+# (B,H,W,Cin,Cout,k): planes of 28 / 14 / odd extents, image rows that do not fill the last tile of an image, an odd
+# number of tiles (the second CTA of the last pair recomputes), channel tails in K (96, 480), one and two accumulator
+# blocks (Cout <= 256 / > 256, equal and unequal halves), Cout not a multiple of 16.
+QLIN_SHAPES = [
+    (3, 28, 28, 192, 128, 5),     # merged 5x5 of 3a: 7 tiles per image, 21 tiles (odd)
+    (2, 28, 28, 256, 288, 5),     # merged 5x5 of 3b: two blocks of 144
+    (3, 14, 14, 480, 304, 5),     # merged 5x5 of 4a: blocks 160 + 144, 32-channel K tail, 2 tiles per image
+    (2, 28, 28, 96, 128, 3),      # 3x3 of 3a: K tail (32 of 64)
+    (5, 14, 14, 112, 224, 3),     # 3x3 of 4b
+    (2, 13, 29, 64, 40, 5),       # odd plane, Cout not a multiple of 16
+    (1, 30, 61, 64, 64, 3),       # wide rows: two image rows per tile
+    (7, 9, 11, 128, 512, 5),      # two blocks of 256
+    (2, 7, 7, 832, 384, 5),       # 7x7 planes: most of a tile is padding
+]
+
+
+@pytest.mark.parametrize("shape", QLIN_SHAPES)
+@pytest.mark.parametrize("slice_", [False, True])
+def test_conv_patch_reuse_kernel(dr, O, shape, slice_):
+    B, H, W, Cin, Cout, k = shape
+    x = S.normal(14, "x", (B, H, W, Cin)); w = S.he_normal(14, "w", Cout, k, Cin); b = S.normal(14, "b", (Cout,), 0.1)
+    force(dr, dr.DR_PATH_UMMA_QLIN)
+    ldc, coff = ((Cout + 72, 40) if slice_ else (0, 0))
+    got, _ = run_conv(dr, x, w, b, k, 1, k // 2, dr.DR_BIAS | dr.DR_RELU, ldc=ldc, coff=coff)
+    assert dr.dr_last_conv_path() == dr.DR_PATH_UMMA_QLIN
+    ref, _ = oracle_slim_layer(O, x, w, b, k, 1, k // 2, dr.DR_BIAS | dr.DR_RELU, dr)
+    assert_layer_close(got, O.round_bf16(ref), f"patch-reuse {shape}")
+    again, _ = run_conv(dr, x, w, b, k, 1, k // 2, dr.DR_BIAS | dr.DR_RELU, ldc=ldc, coff=coff)
+    assert np.array_equal(got, again)                                   # no atomics: bit-identical run to run
+
+
+def test_conv_patch_reuse_kernel_residual_and_f32(dr, O):
+    B, H, W, Cin, Cout, k = 2, 14, 14, 64, 96, 3
+    x = S.normal(15, "x", (B, H, W, Cin)); w = S.he_normal(15, "w", Cout, k, Cin); b = S.normal(15, "b", (Cout,), 0.1)
+    r = S.normal(15, "r", (B, H, W, Cout))
+    force(dr, dr.DR_PATH_UMMA_QLIN)
+    flags = dr.DR_BIAS | dr.DR_RESIDUAL | dr.DR_RELU_AFTER_RESIDUAL
+    got, _ = run_conv(dr, x, w, b, k, 1, 1, flags, residual=r)
+    ref, _ = oracle_slim_layer(O, x, w, b, k, 1, 1, flags, dr, residual=r)
+    assert_layer_close(got, O.round_bf16(ref), "patch-reuse residual")
+    got32, _ = run_conv(dr, x, w, b, k, 1, 1, dr.DR_BIAS | dr.DR_OUT_F32)
+    ref32 = O.conv2d(x, w, b, 1, 1)
+    assert np.abs(got32 - ref32).max() <= 2e-3 * np.abs(ref32).max()
 
 
 @pytest.mark.parametrize("path", [1, 2, 3])

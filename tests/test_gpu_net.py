@@ -67,28 +67,30 @@ def check_network(dr, arch, B, entries, steps_fn, params, per_layer_tol=None, hw
     net, ws, logits, keep = run_net(dr, arch, dr.DR_MODE_SLIM, B, params, images, hw=hw)
     paths = {net.dr_net_layer_info(i)["name"]: net.dr_net_layer_info(i)["conv_path"] for i in range(net.dr_net_num_layers())}
     steps = steps_fn(params)
-    # ---- per layer, teacher-forced, batch entry 0 (+ all checked entries for the logits)
-    G = layer_outputs(net, logits, entries[:1])
-    x0 = images(entries[:1])
-    if arch == dr.DR_ARCH_GOOGLENET_PAPER:
-        # reducers are stored in tensors rounded up to 64 channels: the extra channels must be exactly zero
-        widths = {k: v.shape[-1] for k, v in N.run(steps, x0).items()}
-        for name, c in widths.items():
-            if name in G and G[name].shape[-1] > c:
-                assert not np.any(G[name][..., c:]), f"{name}: padded channels are not zero"
-                G[name] = G[name][..., :c]
-    given = dict(G)
-    for st in steps:                      # concatenated module outputs are re-assembled from their slices
-        if st.virtual:
-            given[st.name] = np.concatenate([given[s] for s in st.src], axis=-1)
-    forced = N.run(steps, x0, given=given)
+    # ---- per layer, teacher-forced: batch entry 0 and, at batch > 1, the last entry (where the ragged last tile, the odd
+    # tile of a CTA pair and the tail of the per-stream ranges live at full size); logits for all checked entries
     report = []
-    for st in steps:
-        if st.virtual:
-            continue
-        assert st.name in G, f"GPU net has no layer {st.name}"
-        mx, l2 = assert_layer_close(G[st.name], forced[st.name], st.name)
-        report.append((st.name, paths.get(st.name), mx, l2))
+    for e in ([entries[0]] + ([B - 1] if B > 1 else [])):
+        G = layer_outputs(net, logits, [e])
+        x0 = images([e])
+        if arch == dr.DR_ARCH_GOOGLENET_PAPER:
+            # reducers are stored in tensors rounded up to 64 channels: the extra channels must be exactly zero
+            widths = {k: v.shape[-1] for k, v in N.run(steps, x0).items()}
+            for name, c in widths.items():
+                if name in G and G[name].shape[-1] > c:
+                    assert not np.any(G[name][..., c:]), f"{name}: padded channels are not zero"
+                    G[name] = G[name][..., :c]
+        given = dict(G)
+        for st in steps:                      # concatenated module outputs are re-assembled from their slices
+            if st.virtual:
+                given[st.name] = np.concatenate([given[s] for s in st.src], axis=-1)
+        forced = N.run(steps, x0, given=given)
+        for st in steps:
+            if st.virtual:
+                continue
+            assert st.name in G, f"GPU net has no layer {st.name}"
+            mx, l2 = assert_layer_close(G[st.name], forced[st.name], f"{st.name} (batch entry {e})")
+            report.append((st.name, paths.get(st.name), mx, l2))
     # ---- end to end, free-running, the seeded subset
     xs = images(entries)
     free = N.run(steps, xs)
@@ -106,9 +108,10 @@ def check_network(dr, arch, B, entries, steps_fn, params, per_layer_tol=None, hw
 
 
 def subset(B, k):
-    """Entry 0 plus the first entries of a seeded permutation."""
-    rest = [int(i) for i in S.stream(0, "subset").permutation(B) if i != 0]
-    return [0] + rest[:k - 1]
+    """Entry 0, the last entry (B - 1), then the first entries of a seeded permutation."""
+    fixed = [0] + ([B - 1] if B > 1 and k > 1 else [])
+    rest = [int(i) for i in S.stream(0, "subset").permutation(B) if i not in fixed]
+    return (fixed + rest)[:max(k, 1)]
 
 
 @pytest.mark.parametrize("B,k", [(1, 1), (256, 4)])
