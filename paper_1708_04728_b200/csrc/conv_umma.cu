@@ -458,7 +458,9 @@ int conv_umma_gather_launch(const ConvParams& p, cudaStream_t stream) {
 // few dozen instructions: nested tap / channel-block loops instead of divisions, barrier and
 // stage addresses advanced incrementally, descriptors assembled from 32-bit halves.
 constexpr int T_MAX_STAGES = 8;   // stage = A tile (16 KB) + B tile; as many as fit
-constexpr int T_THREADS = 320;    // warp 0: TMA producer, warp 1: MMA issue + TMEM owner, warps 2-5 / 6-9: two epilogue groups
+constexpr int T_THREADS = 352;    // warp 0: TMA producer, warp 1: MMA issue + TMEM owner, warps 2-5 / 6-9: two epilogue groups,
+                                  // warp 10: second MMA issuer (wide tiles: the accumulator of the second sub-block is its own)
+constexpr int T_MMA2_WARP = 10;
 constexpr int T_BIAS_MAX = 2048;  // channels of the shared-memory bias copy (lean epilogue)
 constexpr int T_SMEM_MAX = 227 * 1024 - 9216;   // dynamic part; the static part holds barriers and the bias copy
 constexpr int T_ACC_COLS = 256;   // columns per accumulator buffer; two buffers = all 512 TMEM columns
@@ -503,8 +505,8 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
     const int nunits = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (tid == 0) {
-        for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], (PAIR ? 8 : 4) * (WIDE ? 2 : 1)); }
+        for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], WIDE ? 2 : 1); }   // WIDE: both issuers commit
+        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], WIDE ? 2 : 1); mbar_init(&sh.tempty[a], (PAIR ? 8 : 4) * (WIDE ? 2 : 1)); }
         for (int a = 0; a < 6; ++a) mbar_init(&sh.rfull[a / 3][a % 3], 1);
         sh.abort = 0;
         fence_barrier_init();
@@ -596,10 +598,15 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        if (rank == 0) {
+    } else if (warp == 1 || warp == T_MMA2_WARP) {
+        if (rank == 0 && (warp == 1 || WIDE)) {
             // -------------------------------------------- MMA issue.  The whole warp walks the loop (so that the
             // addresses and descriptors are warp-uniform values); lane 0 alone issues the MMAs and commits.
+            // One thread hands the tensor core an MMA about every 64 clocks at best and pays the stage hand-over (barrier
+            // probe, fence, commit) on top, which MMAs of fewer than 256 columns do not cover.  The two sub-blocks of a wide
+            // tile have accumulators of their own, so each gets an issuing warp: both wait for the same stage, each
+            // multiplies the shared activation tile by its filter sub-tile, and a stage is free when both have committed.
+            const int sub = warp == 1 ? 0 : 1;
             const uint32_t el = lane == 0 ? 1u : 0u;
             const uint32_t tfull0 = smem_u32(&sh.tfull[0]), tempty0 = smem_u32(&sh.tempty[0]);
             const int last_nk16 = ((p.Cin - ((cpb - 1) << 6)) + 15) >> 4;
@@ -609,11 +616,9 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             bool ready = __all_sync(0xffffffffu, mbar_test_u32(full0, 0) != 0);
             for (int t = unit; t < total && ok; t += nunits, ++it) {
                 const int nb = t / m_units;
-                const int Nj = min(p.Nt, cout16 - nb * tile_n);
-                const uint32_t idesc = make_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, Nj);
-                const int Nj1 = WIDE ? min(p.Nt, cout16 - nb * tile_n - p.Nt) : 0;          // second sub-block; <= 0: none
-                const uint32_t idesc1 = make_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, Nj1 > 0 ? Nj1 : 16);
-                const uint32_t el1 = (WIDE && Nj1 > 0) ? el : 0u;
+                const int Nj = min(p.Nt, cout16 - nb * tile_n - (WIDE ? sub * p.Nt : 0));   // this issuer's (sub-)block; <= 0: none
+                const uint32_t idesc = make_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, Nj > 0 ? Nj : 16);
+                const uint32_t elj = Nj > 0 ? el : 0u;
                 const int acc = WIDE ? 0 : (it & 1), au = WIDE ? it : (it >> 1);
                 if (!__all_sync(0xffffffffu, mbar_wait_u32(tempty0 + 8 * acc, (au & 1) ^ 1, abort_flag))) {
                     if (el && !*abort_flag) report_timeout(p.status, 12, t);
@@ -621,8 +626,9 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d = tmem + (uint32_t)(acc * T_ACC_COLS);
-                uint32_t accum = 0, accum1 = 0;
+                const uint32_t d = tmem + (uint32_t)((WIDE ? sub : acc) * T_ACC_COLS);
+                const uint32_t b_off = (uint32_t)A_TILE_BYTES + (WIDE ? (uint32_t)sub * b_sub_bytes : 0u);
+                uint32_t accum = 0;
                 int cc = 0;
                 for (int remaining = nkb; remaining > 0;) {
                     const int nk = remaining < kpb ? remaining : kpb;
@@ -640,23 +646,14 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                     uint32_t a = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
 #pragma unroll
                     for (int j = 0; j < KPB; ++j, a += (uint32_t)sub_bytes) {
-                        const uint32_t alo = sdesc_lo(a), blo = sdesc_lo(a + A_TILE_BYTES);
+                        const uint32_t alo = sdesc_lo(a), blo = sdesc_lo(a + b_off);
                         const int nk16 = j < nk ? ((cc == cpb - 1) ? last_nk16 : 4) : 0;    // 0: nothing in this sub-stage
                         cc = (cc + 1 == cpb) ? 0 : cc + 1;
-                        umma_bf16_lo<PAIR>(d, alo, blo, idesc, accum, (nk16 > 0) & el);
+                        umma_bf16_lo<PAIR>(d, alo, blo, idesc, accum, (nk16 > 0) & elj);
                         accum = 1;
-                        umma_bf16_lo<PAIR>(d, alo + 2, blo + 2, idesc, 1u, (nk16 > 1) & el);
-                        umma_bf16_lo<PAIR>(d, alo + 4, blo + 4, idesc, 1u, (nk16 > 2) & el);
-                        umma_bf16_lo<PAIR>(d, alo + 6, blo + 6, idesc, 1u, (nk16 > 3) & el);
-                        if (WIDE) {
-                            const uint32_t blo1 = sdesc_lo(a + A_TILE_BYTES + b_sub_bytes);
-                            const uint32_t d1 = d + (uint32_t)T_ACC_COLS;
-                            umma_bf16_lo<PAIR>(d1, alo, blo1, idesc1, accum1, (nk16 > 0) & el1);
-                            accum1 = 1;
-                            umma_bf16_lo<PAIR>(d1, alo + 2, blo1 + 2, idesc1, 1u, (nk16 > 1) & el1);
-                            umma_bf16_lo<PAIR>(d1, alo + 4, blo1 + 4, idesc1, 1u, (nk16 > 2) & el1);
-                            umma_bf16_lo<PAIR>(d1, alo + 6, blo1 + 6, idesc1, 1u, (nk16 > 3) & el1);
-                        }
+                        umma_bf16_lo<PAIR>(d, alo + 2, blo + 2, idesc, 1u, (nk16 > 1) & elj);
+                        umma_bf16_lo<PAIR>(d, alo + 4, blo + 4, idesc, 1u, (nk16 > 2) & elj);
+                        umma_bf16_lo<PAIR>(d, alo + 6, blo + 6, idesc, 1u, (nk16 > 3) & elj);
                     }
                     if (el) umma_commit_u32<PAIR>(empty0 + 8 * s);
                     remaining -= nk;
