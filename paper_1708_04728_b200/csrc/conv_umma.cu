@@ -40,6 +40,13 @@ __device__ __forceinline__ void issue_kblock(uint32_t tmem_d, uint32_t a_smem, u
         if (k < nk16) umma_bf16(tmem_d, ad + 2 * k, bd + 2 * k, idesc, (first && k == 0) ? 0u : 1u);
 }
 
+// Barrier of one epilogue group (128 threads): ids 1 and 2 as immediates, so that the kernel is seen to use three named
+// barriers and not all sixteen (an SM has sixteen for all of its resident CTAs).
+__device__ __forceinline__ void group_bar_sync(int bar) {
+    if (bar == 1) asm volatile("bar.sync 1, 128;" ::: "memory");
+    else asm volatile("bar.sync 2, 128;" ::: "memory");
+}
+
 // Lean epilogue with TMA stores (bias and/or ReLU, bf16 out): row-per-thread 16-byte global stores cost 32 memory
 // wavefronts per warp instruction (32 rows, 32 different lines), which bounds the layers whose output is large
 // against their K (1x1 convolutions at 56x56: 4.2 us per 128 x 256 tile).  Here the four warps of an epilogue group
@@ -80,7 +87,7 @@ __device__ __forceinline__ void drain_tma_store(const ConvParams& p, const CUten
         }
         fence_proxy_async_smem();                                     // these writes are read by the TMA unit
         if (elected) tma_store_wait_read();                           // the store before this one has let go of the other buffer
-        asm volatile("bar.sync %0, 128;" ::"r"(bar) : "memory");
+        group_bar_sync(bar);
         if (elected && tile_ok) {
             tma_store_2d(map_y, stage_u32 + (uint32_t)(it & 1) * 16384u, p.coff + n0 + c, (int)m0);
             tma_store_commit();
@@ -136,7 +143,7 @@ __device__ __forceinline__ bool drain_tma_residual(const ConvParams& p, const CU
             }
         }
         fence_proxy_async_smem();
-        asm volatile("bar.sync %0, 128;" ::"r"(bar) : "memory");
+        group_bar_sync(bar);
         if (elected) {
             tma_store_2d(map_y, stage_u32 + (uint32_t)b * 16384u, p.coff + n0 + c, (int)m0);
             tma_store_commit();
@@ -457,16 +464,17 @@ int conv_umma_gather_launch(const ConvParams& p, cudaStream_t stream) {
 // (a lone thread issues dependent instructions several cycles apart), so both loops are kept to a
 // few dozen instructions: nested tap / channel-block loops instead of divisions, barrier and
 // stage addresses advanced incrementally, descriptors assembled from 32-bit halves.
-constexpr int T_MAX_STAGES = 8;   // stage = A tile (16 KB) + B tile; as many as fit
-constexpr int T_THREADS = 352;    // warp 0: TMA producer, warp 1: MMA issue + TMEM owner, warps 2-5 / 6-9: two epilogue groups,
-                                  // warp 10: second MMA issuer (wide tiles: the accumulator of the second sub-block is its own)
+constexpr int T_MAX_STAGES = 12;  // stage = A tile (16 KB) + B tile; as many as fit (DUAL: two rings of half as many)
+constexpr int T_THREADS = 384;    // warp 0: TMA producer, warp 1: MMA issue + TMEM owner, warps 2-5 / 6-9: two epilogue groups,
+                                  // warp 10: second MMA issuer, warp 11: second producer (DUAL)
 constexpr int T_MMA2_WARP = 10;
+constexpr int T_PROD2_WARP = 11;
 constexpr int T_BIAS_MAX = 2048;  // channels of the shared-memory bias copy (lean epilogue)
 constexpr int T_SMEM_MAX = 227 * 1024 - 9216;   // dynamic part; the static part holds barriers and the bias copy
 constexpr int T_ACC_COLS = 256;   // columns per accumulator buffer; two buffers = all 512 TMEM columns
 
 struct TmaShared {
-    uint64_t full[T_MAX_STAGES], empty[T_MAX_STAGES], tfull[2], tempty[2];
+    uint64_t full[T_MAX_STAGES], empty[T_MAX_STAGES], tfull[4], tempty[4];
     uint64_t rfull[2][3];      // residual boxes of the TMA epilogue: per epilogue group, ring of three
     uint32_t tmem_base;
     int abort;
@@ -478,35 +486,47 @@ struct TmaShared {
 // is loaded once and multiplied against both filter sub-tiles, which halves the activation traffic of layers
 // with more than 256 output channels.  All 512 TMEM columns then belong to one tile: the MMAs of the next tile
 // start when both epilogue groups (group g drains sub-block g) have emptied it.
-template <bool PAIR, int KPB, bool WIDE>
+// DUAL: the CTA runs TWO tile pipelines side by side, each with its own producer warp, MMA-issuing warp, epilogue group,
+// ring of stages (half of the shared memory) and accumulators (half of TMEM: two of up to 128 columns, or one of up to
+// 256).  One thread hands the tensor core an MMA about every 64 clocks at best and pays the stage hand-over (barrier
+// probe, fence, commit) on top, which MMAs of fewer than 256 columns do not cover: with two issuers working on different
+// tiles the tensor core stays fed, and one pipeline's epilogue runs under the other's MMAs.  (Two CTAs per SM would do the
+// same, but a kernel that uses tcgen05 is given an SM to itself.)
+template <bool PAIR, int KPB, bool WIDE, bool DUAL>
 __global__ void __launch_bounds__(T_THREADS, 1)
 conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_r, const int a_mode, const int stages,
                      const int sub_bytes, const int ep_stage_off) {
     constexpr int kpb = KPB;
+    constexpr int NTHREADS = T_THREADS;
+    constexpr int BIAS_MAX = T_BIAS_MAX;
+    constexpr uint32_t TMEM_COLS = 2 * T_ACC_COLS;
+    // accumulator buffers of a tile pipeline and their width in TMEM columns (WIDE: the two sub-blocks of one tile instead)
+    const int nacc = DUAL ? (p.Nt <= 128 ? 2 : 1) : 2;
+    const uint32_t acc_cols = DUAL ? (uint32_t)(T_ACC_COLS / nacc) : (uint32_t)T_ACC_COLS;
     // a pipeline stage holds `kpb` k-blocks (sub-stages of sub_bytes = A tile + B tile): one barrier
     // round trip then covers kpb * 4 MMAs, which keeps the issuing thread ahead of the tensor pipe
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     __shared__ TmaShared sh;
-    __shared__ __align__(16) float bias_s[T_BIAS_MAX];
+    __shared__ __align__(16) float bias_s[BIAS_MAX];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int stage_bytes = kpb * sub_bytes;
     // lean epilogue: bias, ReLU, residual (+ReLU); bf16 out, every 16-column chunk inside Cout, aligned slice.
     // (ReLU before a residual add is the one order it does not take.)
     const bool lean = !(p.flags & DR_OUT_F32) && !((p.flags & DR_RESIDUAL) && (p.flags & DR_RELU)) && (p.Cout & 15) == 0 &&
-                      p.Cout <= T_BIAS_MAX && (p.ldc & 7) == 0 && (p.coff & 7) == 0;
+                      p.Cout <= BIAS_MAX && (p.ldc & 7) == 0 && (p.coff & 7) == 0;
     const bool lrn_ep = (p.flags & DR_LRN) != 0;                // host side guarantees: no pooling, one n-block, lean preconditions
     const int lean_mode = (p.flags & DR_RESIDUAL) ? ((p.flags & DR_RELU_AFTER_RESIDUAL) ? 3 : 2) : ((p.flags & DR_RELU) ? 1 : 0);
     if (lean)
-        for (int i = tid; i < p.Cout; i += T_THREADS) bias_s[i] = (p.flags & DR_BIAS) ? p.bias[i] : 0.f;
+        for (int i = tid; i < p.Cout; i += NTHREADS) bias_s[i] = (p.flags & DR_BIAS) ? p.bias[i] : 0.f;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;        // 0 issues the MMAs
     const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int nunits = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (tid == 0) {
-        for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], WIDE ? 2 : 1); }   // WIDE: both issuers commit
-        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], WIDE ? 2 : 1); mbar_init(&sh.tempty[a], (PAIR ? 8 : 4) * (WIDE ? 2 : 1)); }
+        for (int s = 0; s < (DUAL ? 2 * stages : stages); ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], WIDE ? 2 : 1); }   // WIDE: both issuers commit
+        for (int a = 0; a < 4; ++a) { mbar_init(&sh.tfull[a], WIDE ? 2 : 1); mbar_init(&sh.tempty[a], (PAIR ? 8 : 4) * (WIDE ? 2 : 1)); }
         for (int a = 0; a < 6; ++a) mbar_init(&sh.rfull[a / 3][a % 3], 1);
         sh.abort = 0;
         fence_barrier_init();
@@ -514,8 +534,8 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
         prefetch_tensormap(&map_b);
     }
     if (warp == 1) {
-        if (PAIR) { tmem_alloc_pair(&sh.tmem_base, 2 * T_ACC_COLS); tmem_relinquish_pair(); }
-        else { tmem_alloc(&sh.tmem_base, 2 * T_ACC_COLS); tmem_relinquish(); }
+        if (PAIR) { tmem_alloc_pair(&sh.tmem_base, TMEM_COLS); tmem_relinquish_pair(); }
+        else { tmem_alloc(&sh.tmem_base, TMEM_COLS); tmem_relinquish(); }
     }
     tc_fence_before();
     __syncthreads();
@@ -534,18 +554,20 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
     const int tile_n = WIDE ? 2 * p.Nt : p.Nt;                 // output channels per tile
     const uint32_t b_sub_bytes = WIDE ? (uint32_t)(sub_bytes - A_TILE_BYTES) >> 1 : 0u;   // one filter sub-tile
     const uint32_t smem_base = smem_u32(smem);
-    const uint32_t full0 = smem_u32(&sh.full[0]), empty0 = smem_u32(&sh.empty[0]);
 
-    if (warp == 0) {
-        if (lane == 0) {
-            // -------------------------------------------- TMA producer
+    if (warp == 0 || warp == T_PROD2_WARP) {
+        if (lane == 0 && (warp == 0 || DUAL)) {
+            // -------------------------------------------- TMA producer (DUAL: of pipeline g, ring g)
+            const int g = warp == 0 ? 0 : 1;
+            const uint32_t full0 = smem_u32(&sh.full[g * stages]), empty0 = smem_u32(&sh.empty[g * stages]);
+            const uint32_t ring_base = smem_base + (uint32_t)(g * stages) * (uint32_t)stage_bytes;
             const uint32_t cta_tx = A_TILE_BYTES + (uint32_t)(PAIR ? p.Nt >> 1 : p.Nt) * 128 * (WIDE ? 2 : 1);
             const uint32_t full_mask = PAIR ? PEER_BIT_MASK : 0xFFFFFFFFu;   // pair: bytes are reported to the even CTA
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
             uint32_t ready = mbar_test_u32(empty0, 1);
-            for (int t = unit; t < total && ok; t += nunits) {
+            for (int t = DUAL ? unit + g * nunits : unit; t < total && ok; t += DUAL ? 2 * nunits : nunits) {
                 const int nb = t / m_units, mu = t - nb * m_units;
                 const int n0 = nb * tile_n;
                 int mt = PAIR ? 2 * mu + (int)rank : mu;
@@ -571,7 +593,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                     uint32_t ph2 = ph;
                     if (s2 == stages) { s2 = 0; ph2 ^= 1; }
                     ready = mbar_test_u32(empty0 + 8 * s2, ph2 ^ 1);      // probe the next slot while this one is filled
-                    uint32_t a_dst = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+                    uint32_t a_dst = ring_base + (uint32_t)s * (uint32_t)stage_bytes;
                     const uint32_t fb = (full0 + 8 * s) & full_mask;
                     if (!PAIR) mbar_expect_tx_u32(fb, (uint32_t)nk * cta_tx);
                     else if (rank == 0) mbar_expect_tx_u32(fb, 2u * (uint32_t)nk * cta_tx);
@@ -599,14 +621,17 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
         }
         __syncwarp();
     } else if (warp == 1 || warp == T_MMA2_WARP) {
-        if (rank == 0 && (warp == 1 || WIDE)) {
+        if (rank == 0 && (warp == 1 || WIDE || DUAL)) {
             // -------------------------------------------- MMA issue.  The whole warp walks the loop (so that the
             // addresses and descriptors are warp-uniform values); lane 0 alone issues the MMAs and commits.
             // One thread hands the tensor core an MMA about every 64 clocks at best and pays the stage hand-over (barrier
             // probe, fence, commit) on top, which MMAs of fewer than 256 columns do not cover.  The two sub-blocks of a wide
             // tile have accumulators of their own, so each gets an issuing warp: both wait for the same stage, each
             // multiplies the shared activation tile by its filter sub-tile, and a stage is free when both have committed.
-            const int sub = warp == 1 ? 0 : 1;
+            const int sub = (WIDE && warp != 1) ? 1 : 0;          // WIDE: the sub-block this warp issues
+            const int g = (DUAL && warp != 1) ? 1 : 0;            // DUAL: the pipeline this warp issues
+            const uint32_t full0 = smem_u32(&sh.full[g * stages]), empty0 = smem_u32(&sh.empty[g * stages]);
+            const uint32_t ring_base = smem_base + (uint32_t)(g * stages) * (uint32_t)stage_bytes;
             const uint32_t el = lane == 0 ? 1u : 0u;
             const uint32_t tfull0 = smem_u32(&sh.tfull[0]), tempty0 = smem_u32(&sh.tempty[0]);
             const int last_nk16 = ((p.Cin - ((cpb - 1) << 6)) + 15) >> 4;
@@ -614,19 +639,21 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             uint32_t ph = 0;
             bool ok = true;
             bool ready = __all_sync(0xffffffffu, mbar_test_u32(full0, 0) != 0);
-            for (int t = unit; t < total && ok; t += nunits, ++it) {
+            for (int t = DUAL ? unit + g * nunits : unit; t < total && ok; t += DUAL ? 2 * nunits : nunits, ++it) {
                 const int nb = t / m_units;
                 const int Nj = min(p.Nt, cout16 - nb * tile_n - (WIDE ? sub * p.Nt : 0));   // this issuer's (sub-)block; <= 0: none
                 const uint32_t idesc = make_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, Nj > 0 ? Nj : 16);
                 const uint32_t elj = Nj > 0 ? el : 0u;
-                const int acc = WIDE ? 0 : (it & 1), au = WIDE ? it : (it >> 1);
+                // accumulator buffer of this tile: its hand-over barriers, their parity, its TMEM column
+                const int bsel = WIDE ? 0 : (nacc == 2 ? (it & 1) : 0), au = WIDE ? it : (nacc == 2 ? (it >> 1) : it);
+                const int acc = 2 * g + bsel;
                 if (!__all_sync(0xffffffffu, mbar_wait_u32(tempty0 + 8 * acc, (au & 1) ^ 1, abort_flag))) {
                     if (el && !*abort_flag) report_timeout(p.status, 12, t);
                     *abort_flag = 1;
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d = tmem + (uint32_t)((WIDE ? sub : acc) * T_ACC_COLS);
+                const uint32_t d = tmem + (WIDE ? (uint32_t)sub * (uint32_t)T_ACC_COLS : (uint32_t)(g * T_ACC_COLS) + (uint32_t)bsel * acc_cols);
                 const uint32_t b_off = (uint32_t)A_TILE_BYTES + (WIDE ? (uint32_t)sub * b_sub_bytes : 0u);
                 uint32_t accum = 0;
                 int cc = 0;
@@ -643,7 +670,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                     if (s2 == stages) { s2 = 0; ph2 ^= 1; }
                     ready = __all_sync(0xffffffffu, mbar_test_u32(full0 + 8 * s2, ph2) != 0);   // probe the next slot while this one is issued
                     tc_fence_after();
-                    uint32_t a = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
+                    uint32_t a = ring_base + (uint32_t)s * (uint32_t)stage_bytes;
 #pragma unroll
                     for (int j = 0; j < KPB; ++j, a += (uint32_t)sub_bytes) {
                         const uint32_t alo = sdesc_lo(a), blo = sdesc_lo(a + b_off);
@@ -671,7 +698,12 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
         const int q = warp & 3;
         const int row = q * 32 + lane;
         int ep_it = 0;                                           // chunks this group has handed to the TMA unit so far
+        // tiles of this group: WIDE every tile (sub-block g); else every other tile of the CTA (DUAL: those are pipeline g's)
         for (int t = WIDE ? unit : unit + g * nunits, au = 0; t < total; t += WIDE ? nunits : 2 * nunits, ++au) {
+            // accumulator buffer of this tile, the parity of its hand-over barriers, its TMEM column
+            const int bsel = (DUAL && nacc == 2) ? (au & 1) : 0;
+            const int ab = WIDE ? 0 : (DUAL ? 2 * g + bsel : g);
+            const uint32_t par = (DUAL && nacc == 2) ? (uint32_t)(au >> 1) & 1u : (uint32_t)au & 1u;
             const int nb = t / m_units, mu = t - nb * m_units;
             const int n0 = WIDE ? nb * tile_n + g * p.Nt : nb * p.Nt;      // WIDE: group g drains sub-block g of every tile
             const int Nj = min(p.Nt, cout16 - n0);                         // WIDE: may be <= 0 (no second sub-block)
@@ -683,7 +715,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
                 residual_box_load(&map_r, st, sh.rfull[g], ep_it, n0, (int)((long long)mt * TILE_M));
                 if (Nj > 64) residual_box_load(&map_r, st, sh.rfull[g], ep_it + 1, n0 + 64, (int)((long long)mt * TILE_M));
             }
-            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[WIDE ? 0 : g], au & 1, abort_flag));
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh.tfull[ab], par, abort_flag));
             if (!ok) {
                 if (!*abort_flag) report_timeout(p.status, 14, t);
                 *abort_flag = 1;
@@ -691,7 +723,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             }
             tc_fence_after();
             const long long m = (long long)mt * TILE_M + row;
-            const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * T_ACC_COLS);
+            const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * T_ACC_COLS) + (uint32_t)bsel * acc_cols;
             const bool row_ok = mt < p.m_tiles && m < p.M;
             if (WIDE && Nj <= 0) {
                 // nothing to drain
@@ -728,8 +760,8 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
-                if (PAIR) mbar_arrive_leader(&sh.tempty[WIDE ? 0 : g]);
-                else mbar_arrive(&sh.tempty[WIDE ? 0 : g]);
+                if (PAIR) mbar_arrive_leader(&sh.tempty[ab]);
+                else mbar_arrive(&sh.tempty[ab]);
             }
         }
     }
@@ -744,8 +776,8 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
     if (PAIR) cluster_sync_all();                               // neither CTA leaves while the other may still signal it
     if (p.overlap_prev) grid_dependency_wait();                 // launched ahead of the previous kernel's end: do not finish before it has
     if (warp == 1) {
-        if (PAIR) tmem_dealloc_pair(tmem, 2 * T_ACC_COLS);
-        else tmem_dealloc(tmem, 2 * T_ACC_COLS);
+        if (PAIR) tmem_dealloc_pair(tmem, TMEM_COLS);
+        else tmem_dealloc(tmem, TMEM_COLS);
     }
 }
 
@@ -803,15 +835,14 @@ bool conv_umma_tma_supports(const ConvParams& p) {
     return true;
 }
 
-// Pipeline shape: k-blocks per stage (kpb) and number of stages.  Measured on B200: wide tiles
-// (Nt >= 208) run best with one k-block per barrier round trip, narrower ones with two (their MMAs
-// are short, so the round trip has to cover more of them); never more than the layer has.
-static void pick_pipeline(int sub_bytes, int nkb, int nt, int ep_bytes, int* kpb, int* stages) {
-    const int budget = T_SMEM_MAX - 1024 - ep_bytes;
+// Pipeline shape: k-blocks per stage (kpb) and number of stages within `budget` bytes.  Measured on B200: tiles of at
+// least 208 columns run best with one k-block per barrier round trip, narrower ones with two (their MMAs are short, so
+// the round trip has to cover more of them); never more than the layer has.
+static void pick_pipeline(int budget, int sub_bytes, int nkb, int nt, int* kpb, int* stages) {
     int k = tunable("DR_TMA_KPB", 0);
     if (k <= 0) k = nt >= 208 ? 1 : 2;
     if (k >= 4) k = 4; else if (k == 3) k = 2;          // instantiated: 1, 2, 4
-    while (k > 1 && (k > nkb || budget / (k * sub_bytes) < 2)) k >>= 1;
+    while (k > 1 && (k > nkb || budget / (k * sub_bytes) < 3)) k >>= 1;
     int st = budget / (k * sub_bytes);
     if (st > T_MAX_STAGES) st = T_MAX_STAGES;
     const int forced = tunable("DR_TMA_STAGES", 0);
@@ -852,55 +883,6 @@ static int tma_epilogue_bytes(const ConvParams& p, bool pair_or_wide, CUtensorMa
     return res ? 2 * 3 * 16384 : 2 * 2 * 16384;                  // per epilogue group: three / two 16 KB buffers
 }
 
-static int launch_pair(const ConvParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, int a_mode, bool wide, cudaStream_t stream) {
-    static bool attr_set = false;
-    static int max_clusters = 0;
-    const int sub_bytes = A_TILE_BYTES + (wide ? 2 : 1) * ((p.Nt * 64 + 1023) & ~1023);
-    int kpb, stages;
-    alignas(64) CUtensorMap map_y = map_a, map_r = map_a;        // placeholders when the TMA epilogue is off
-    int ep_bytes = tma_epilogue_bytes(p, true, &map_y, &map_r);
-    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, ep_bytes, &kpb, &stages);
-    if (ep_bytes && stages < 2) {                                // not enough room left for the operand pipeline: do without
-        ep_bytes = 0;
-        pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, 0, &kpb, &stages);
-    }
-    const int ep_off = ep_bytes ? stages * kpb * sub_bytes : 0;
-    int smem_bytes = stages * kpb * sub_bytes + ep_bytes + 1024;
-    if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.blockDim = dim3(T_THREADS); cfg.dynamicSmemBytes = (size_t)smem_bytes; cfg.stream = stream;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(conv_umma_tma_kernel<true, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
-            cudaFuncSetAttribute(conv_umma_tma_kernel<true, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
-            cudaFuncSetAttribute(conv_umma_tma_kernel<true, 4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
-            cudaFuncSetAttribute(conv_umma_tma_kernel<true, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess)
-            return DR_ERR_CUDA;
-        cfg.gridDim = dim3(2 * num_sms());
-        cfg.dynamicSmemBytes = (size_t)T_SMEM_MAX;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, conv_umma_tma_kernel<true, 1, false>, &cfg) != cudaSuccess || max_clusters < 1) return DR_ERR_CUDA;
-        cfg.dynamicSmemBytes = (size_t)smem_bytes;
-        attr_set = true;
-    }
-    const int pair_tiles = ((p.m_tiles + 1) / 2) * p.n_blocks;
-    const int pairs = pair_tiles < max_clusters ? pair_tiles : max_clusters;
-    cfg.gridDim = dim3(2 * pairs);
-    cfg.numAttrs = p.overlap_prev ? 2 : 1;
-    cudaError_t e;
-    if (wide) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 1, true>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
-    else if (kpb == 4) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 4, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
-    else if (kpb == 2) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 2, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
-    else e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<true, 1, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
-    if (e != cudaSuccess) return DR_ERR_CUDA;
-    count_launch();
-    return launch_status();
-}
-
 // Tile shape of a layer on the TMA kernel: CTA pairs or single CTAs, and whether a tile carries two n-blocks that
 // share the activation tile (then p->Nt / p->n_blocks are replaced by the wide tiling).
 void conv_umma_tma_shape(ConvParams* pp, bool* use_pair_out, bool* wide_out) {
@@ -936,56 +918,130 @@ void conv_umma_tma_shape(ConvParams* pp, bool* use_pair_out, bool* wide_out) {
     *wide_out = wide;
 }
 
+namespace {
+struct TmaLaunch {
+    const ConvParams* p;
+    const CUtensorMap *map_a, *map_b, *map_y, *map_r;
+    int a_mode, stages, sub_bytes, ep_off, smem_bytes, units;
+    cudaStream_t stream;
+};
+
+// One instantiation: sets its attributes once per device, asks how many clusters fit, launches.
+template <bool PAIR, int KPB, bool WIDE, bool DUAL>
+int launch_variant(const TmaLaunch& L) {
+    static bool ready[64] = {false};
+    static int capacity[64] = {0};                               // resident CTAs (single) / clusters (pairs)
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DR_ERR_CUDA;
+    auto kern = conv_umma_tma_kernel<PAIR, KPB, WIDE, DUAL>;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (PAIR) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = 2; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    cfg.blockDim = dim3(T_THREADS); cfg.stream = L.stream; cfg.attrs = attr;
+    if (!ready[dev]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+        if (PAIR) {
+            cfg.gridDim = dim3(2 * num_sms());
+            cfg.dynamicSmemBytes = (size_t)T_SMEM_MAX;
+            cfg.numAttrs = na;
+            if (cudaOccupancyMaxActiveClusters(&capacity[dev], kern, &cfg) != cudaSuccess || capacity[dev] < 1) return DR_ERR_CUDA;
+        } else {
+            capacity[dev] = num_sms();
+        }
+        ready[dev] = true;
+    }
+    const int n = L.units < capacity[dev] ? L.units : capacity[dev];
+    cfg.gridDim = dim3((unsigned)(PAIR ? 2 * n : n));
+    cfg.dynamicSmemBytes = (size_t)L.smem_bytes;
+    if (L.p->overlap_prev) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.numAttrs = na;
+    if (cudaLaunchKernelEx(&cfg, kern, *L.p, *L.map_a, *L.map_b, *L.map_y, *L.map_r, L.a_mode, L.stages, L.sub_bytes, L.ep_off) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DR_ERR_CUDA;
+    }
+    count_launch();
+    return launch_status();
+}
+
+template <bool PAIR, bool DUAL>
+int launch_kpb(const TmaLaunch& L, int kpb) {
+    if (kpb == 4) return launch_variant<PAIR, 4, false, DUAL>(L);
+    if (kpb == 2) return launch_variant<PAIR, 2, false, DUAL>(L);
+    return launch_variant<PAIR, 1, false, DUAL>(L);
+}
+}  // namespace
+
+// Whether the layer runs as two tile pipelines per CTA (DUAL), and its pipeline shape then: tiles without the TMA-store
+// epilogue, without LRN and without a second sub-block, enough of them that CTAs have more than one, and room for at
+// least three stages in each of the two rings.
+static bool pick_dual(const ConvParams& p, bool use_pair, bool wide, int ep_bytes, int sub_bytes, int nkb, int total, int* kpb, int* stages) {
+    const int pref = tunable("DR_TMA_DUAL", -1);
+    if (pref == 0 || wide || ep_bytes || (p.flags & DR_LRN)) return false;
+    const int capacity = use_pair ? num_sms() / 2 : num_sms();
+    if (pref < 0 && total <= capacity) return false;
+    // Measured at batch 256 (GoogLeNet): a gain where one issuer cannot keep up with its MMAs and the reduction is long
+    // enough to matter, i.e. tiles of at most 224 columns over at least 48 k-blocks (3a / 5a / 5b merged 5x5: 250 -> 216,
+    // 211 -> 174, 231 -> 204 us) and tiles of at most 128 columns (two accumulators per pipeline); a loss on tiles of
+    // 240 and 256 columns, which one issuer keeps busy (4c / 4d merged 5x5: 224 -> 254, 219 -> 246 us), and on short
+    // reductions with wide tiles, where each ring's three stages cover less of the load latency (3b 3x3: 92 -> 113 us).
+    if (pref < 0 && !((p.Nt <= 224 && nkb >= 48) || (p.Nt <= 128 && nkb >= 16))) return false;
+    int k = tunable("DR_TMA_KPB", 0);
+    if (k <= 0) k = 1;
+    if (k >= 4) k = 4; else if (k == 3) k = 2;
+    const int budget = (T_SMEM_MAX - 1024) / 2;
+    while (k > 1 && (k > nkb || budget / (k * sub_bytes) < 3)) k >>= 1;
+    int st = budget / (k * sub_bytes);
+    if (st > T_MAX_STAGES / 2) st = T_MAX_STAGES / 2;
+    if (st < 3) return false;
+    *kpb = k;
+    *stages = st;
+    return true;
+}
+
 int conv_umma_tma_launch(const ConvParams& p_in, cudaStream_t stream) {
     if (!conv_umma_tma_supports(p_in)) return DR_ERR_UNSUPPORTED;
     ConvParams p = p_in;
     bool use_pair = false, wide = false;
     conv_umma_tma_shape(&p, &use_pair, &wide);
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(conv_umma_tma_kernel<false, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
-            cudaFuncSetAttribute(conv_umma_tma_kernel<false, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
-            cudaFuncSetAttribute(conv_umma_tma_kernel<false, 4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess ||
-            cudaFuncSetAttribute(conv_umma_tma_kernel<false, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_MAX) != cudaSuccess)
-            return DR_ERR_CUDA;
-        attr_set = true;
-    }
     alignas(64) CUtensorMap map_a, map_b;
     int a_mode = 0;
     const int est = encode_conv_maps(p, use_pair ? p.Nt / 2 : p.Nt, &map_a, &map_b, &a_mode);   // a pair's CTAs load half of B each
     if (est != DR_OK) return est;
-    const int total = p.m_tiles * p.n_blocks;
+    const int m_units = use_pair ? (p.m_tiles + 1) / 2 : p.m_tiles;
+    const int total = m_units * p.n_blocks;
     if (total <= 0) return DR_OK;
-    if (use_pair) return launch_pair(p, map_a, map_b, a_mode, wide, stream);
-    const int grid = total < num_sms() ? total : num_sms();
-    // as many pipeline stages as shared memory holds (the B tile shrinks with Nt); always more than
-    // half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
-    const int sub_bytes = A_TILE_BYTES + (wide ? 2 : 1) * ((p.Nt * 128 + 1023) & ~1023);
-    int kpb, stages;
+    const int nkb = p.k * p.k * ((p.Cin + 63) / 64);
+    // one k-block of a stage: the activation tile and this CTA's filter tile (half of it in a pair; two sub-tiles if wide)
+    const int b_rows = use_pair ? p.Nt / 2 : p.Nt;
+    const int sub_bytes = A_TILE_BYTES + (wide ? 2 : 1) * ((b_rows * 128 + 1023) & ~1023);
     alignas(64) CUtensorMap map_y = map_a, map_r = map_a;        // placeholders when the TMA epilogue is off
-    int ep_bytes = tma_epilogue_bytes(p, wide, &map_y, &map_r);
-    pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, ep_bytes, &kpb, &stages);
+    int ep_bytes = tma_epilogue_bytes(p, use_pair || wide, &map_y, &map_r);
+    int kpb, stages;
+    pick_pipeline(T_SMEM_MAX - 1024 - ep_bytes, sub_bytes, nkb, wide ? 256 : p.Nt, &kpb, &stages);
     if (ep_bytes && stages < 2) {                                // not enough room left for the operand pipeline: do without
         ep_bytes = 0;
-        pick_pipeline(sub_bytes, p.k * p.k * ((p.Cin + 63) / 64), wide ? 256 : p.Nt, 0, &kpb, &stages);
+        pick_pipeline(T_SMEM_MAX - 1024, sub_bytes, nkb, wide ? 256 : p.Nt, &kpb, &stages);
     }
-    const int ep_off = ep_bytes ? stages * kpb * sub_bytes : 0;
-    int smem_bytes = stages * kpb * sub_bytes + ep_bytes + 1024;
-    if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(T_THREADS); cfg.dynamicSmemBytes = (size_t)smem_bytes; cfg.stream = stream;
-    cfg.attrs = attr; cfg.numAttrs = p.overlap_prev ? 1 : 0;
-    cudaError_t e;
-    if (wide) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<false, 1, true>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
-    else if (kpb == 4) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<false, 4, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
-    else if (kpb == 2) e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<false, 2, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
-    else e = cudaLaunchKernelEx(&cfg, conv_umma_tma_kernel<false, 1, false>, p, map_a, map_b, map_y, map_r, a_mode, stages, sub_bytes, ep_off);
-    if (e != cudaSuccess) { (void)cudaGetLastError(); return DR_ERR_CUDA; }
-    count_launch();
-    return launch_status();
+    const bool dual = pick_dual(p, use_pair, wide, ep_bytes, sub_bytes, nkb, total, &kpb, &stages);
+    TmaLaunch L;
+    L.p = &p; L.map_a = &map_a; L.map_b = &map_b; L.map_y = &map_y; L.map_r = &map_r;
+    L.a_mode = a_mode; L.stages = stages; L.sub_bytes = sub_bytes; L.stream = stream; L.units = total;
+    L.ep_off = ep_bytes ? stages * kpb * sub_bytes : 0;
+    L.smem_bytes = (dual ? 2 : 1) * stages * kpb * sub_bytes + ep_bytes + 1024;
+    // a CTA owns all of TMEM: it takes more than half of an SM's shared memory, so that no second one joins it
+    if (L.smem_bytes < 120 * 1024) L.smem_bytes = 120 * 1024;
+    if (wide) return use_pair ? launch_variant<true, 1, true, false>(L) : launch_variant<false, 1, true, false>(L);
+    if (dual) return use_pair ? launch_kpb<true, true>(L, kpb) : launch_kpb<false, true>(L, kpb);
+    return use_pair ? launch_kpb<true, false>(L, kpb) : launch_kpb<false, false>(L, kpb);
 }
 
 
