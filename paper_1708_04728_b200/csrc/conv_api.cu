@@ -67,6 +67,7 @@ int conv_make_params(const dr_conv_desc* d, int B, int H, int W, const void* x, 
         p.lrn_s3 = (float)(kp * p.lrn_c3 * au * au * au);
         p.lrn_s4 = (float)(kp * p.lrn_c4 * au * au * au * au);
         p.lrn_ss_max = au > 0 ? (float)(0.03125 / au) : 3.0e38f;
+        p.lrn_ss_max2 = au > 0 ? (float)(0.00390625 / au) : 3.0e38f;
     }
     p.ldc = ldc; p.coff = coff;
     p.M = (long long)B * p.Ho * p.Wo;

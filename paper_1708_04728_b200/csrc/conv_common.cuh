@@ -43,6 +43,7 @@ struct ConvParams {
     // the same series in the window sum ss itself, k^(-beta) folded in: scale = s0 + ss (s1 + ss (s2 + ss (s3 + ss s4))),
     // valid while ss < lrn_ss_max (u = (alpha/n) ss / k below 1/32)
     float lrn_s1, lrn_s2, lrn_s3, lrn_s4, lrn_ss_max;
+    float lrn_ss_max2;     // below this (u < 1/256) the series stops after the ss^2 term: the next one is under 4e-8 relative
     int ldc, coff;
     long long M;           // B*Ho*Wo
     int Nt;                // output channels per n-block (multiple of 16, <= 256)

@@ -30,14 +30,16 @@ __device__ __forceinline__ void fe_bar(int id) { asm volatile("bar.sync %0, %1;"
 __host__ __device__ inline bool fe_lrn_first(const ConvParams& p) { return (p.flags & DR_LRN) && (p.flags & DR_LRN_BEFORE_POOL); }
 // bytes of one staged row: bf16 after LRN-first, float32 raw accumulators otherwise (+16 B: 16-byte
 // row-wise stores of a warp then fall on distinct banks)
-__host__ __device__ inline int fe_stage_pitch(const ConvParams& p) { return fe_lrn_first(p) ? (p.Cout * 2 + 16) : (p.Cout * 4 + 16); }
+// With the positions of the maxima asked for (argmax), every staged value is float32: the decision is taken on the
+// unrounded values, as the layer sequence the slim layer stands for would take it.
+__host__ __device__ inline int fe_stage_pitch(const ConvParams& p) { return (fe_lrn_first(p) && !p.argmax) ? (p.Cout * 2 + 16) : (p.Cout * 4 + 16); }
 __host__ __device__ inline int fe_smem_bytes(const ConvParams& p) {
     int b = TILE_M * fe_stage_pitch(p) + 256 * 4;                       // stage + bias copy
     if ((p.flags & DR_LRN) && !fe_lrn_first(p)) b += p.PH * p.PW * (p.Cout + 8) * 4;   // pooled float32 values, 4 floats of halo each side
     return (b + 1023) & ~1023;
 }
 inline bool fe_supports(const ConvParams& p) {
-    if (!(p.flags & DR_POOL) || p.argmax) return false;          // argmax and LRN-only layers: gather kernel
+    if (!(p.flags & DR_POOL)) return false;                      // LRN-only layers: the TMA / gather kernels
     if (p.Cout % 32 || p.Cout > 256) return false;
     if ((p.flags & DR_LRN) && (p.lrn_half != 2 || p.lrn_k <= 0.f || p.lrn_alpha_n < 0.f)) return false;
     if (p.flags & (DR_RESIDUAL | DR_OUT_F32)) return false;
@@ -56,7 +58,10 @@ __device__ __forceinline__ void fe_lrn_scale(const ConvParams& p, const float* s
     float smax = 0.f;
 #pragma unroll
     for (int j = 0; j < N; ++j) smax = fmaxf(smax, ss[j]);
-    if (__all_sync(0xffffffffu, smax < p.lrn_ss_max)) {      // series in ss, k^(-beta) folded into the coefficients
+    if (__all_sync(0xffffffffu, smax < p.lrn_ss_max2)) {     // series in ss, k^(-beta) folded into the coefficients; two terms suffice
+#pragma unroll
+        for (int j = 0; j < N; ++j) scale[j] = fmaf(ss[j], fmaf(ss[j], p.lrn_s2, p.lrn_s1), p.lrn_kpow);
+    } else if (__all_sync(0xffffffffu, smax < p.lrn_ss_max)) {
 #pragma unroll
         for (int j = 0; j < N; ++j) scale[j] = fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], p.lrn_s4, p.lrn_s3), p.lrn_s2), p.lrn_s1), p.lrn_kpow);
     } else {
@@ -92,6 +97,7 @@ __device__ __forceinline__ void fe_load_chunk(uint32_t taddr, const float* bias_
 // ss[j] = ss[j-1] + x[j+2]^2 - x[j-3]^2, restarted from its five terms every 8 channels (a sum that cancels to a few
 // ulps below zero is harmless: the scale is k + (alpha/n) ss with k > 0).  The scale is the series in ss with k^(-beta)
 // folded in while the sum of all squares of the warp's chunk is below lrn_ss_max; exp2/log2 otherwise.
+template <bool F32OUT>
 __device__ __forceinline__ void fe_lrn_chunk(const ConvParams& p, const float* cur, const float* nxt, float& pm2, float& pm1, uint8_t* dst,
                                              bool valid) {
     float sq[36];                                  // squares of x[c0-2 .. c0+33]
@@ -107,12 +113,27 @@ __device__ __forceinline__ void fe_lrn_chunk(const ConvParams& p, const float* c
     }
     // every window sum is at most the sum of all squares = seven disjoint windows + the last square
     const float total = ((ss[0] + ss[5]) + (ss[10] + ss[15])) + ((ss[20] + ss[25]) + (ss[30] + sq[35]));
-    if (__all_sync(0xffffffffu, total < p.lrn_ss_max)) {
+    if (__all_sync(0xffffffffu, total < p.lrn_ss_max2)) {   // the usual case (alpha = 1e-4): two terms are exact to float32 resolution
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sc[j] = fmaf(ss[j], fmaf(ss[j], p.lrn_s2, p.lrn_s1), p.lrn_kpow);
+    } else if (__all_sync(0xffffffffu, total < p.lrn_ss_max)) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) sc[j] = fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], p.lrn_s4, p.lrn_s3), p.lrn_s2), p.lrn_s1), p.lrn_kpow);
     } else {
 #pragma unroll
         for (int j = 0; j < 32; ++j) sc[j] = __powf(fmaf(p.lrn_alpha_n, ss[j], p.lrn_k), -p.lrn_beta);
+    }
+    if (F32OUT) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            float4 v;
+            if (valid) v = make_float4(cur[4 * q] * sc[4 * q], cur[4 * q + 1] * sc[4 * q + 1], cur[4 * q + 2] * sc[4 * q + 2], cur[4 * q + 3] * sc[4 * q + 3]);
+            else v.x = v.y = v.z = v.w = __uint_as_float(0xff800000u);
+            *reinterpret_cast<float4*>(dst + 16 * q) = v;
+        }
+        pm2 = cur[30];
+        pm1 = cur[31];
+        return;
     }
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
@@ -142,6 +163,7 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
     const bool lrn = p.flags & DR_LRN;
     const bool lrn_first = fe_lrn_first(p);
     const bool relu = p.flags & DR_RELU;
+    const bool am = p.argmax != nullptr;
     const int pitch = fe_stage_pitch(p);
     const float* bias_s = reinterpret_cast<const float*>(stage + TILE_M * pitch);
     const int pwc = 2 * p.PW + 1, phc = 2 * p.PH + 1;
@@ -161,10 +183,12 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
         fe_load_chunk(taddr, bias_s, 0, true, relu, xa);
         for (int c0 = 0; c0 < C; c0 += 64) {
             fe_load_chunk(taddr, bias_s, c0 + 32, c0 + 32 < C, relu, xb);
-            fe_lrn_chunk(p, xa, xb, pm2, pm1, srow + c0 * 2, valid);
+            if (am) fe_lrn_chunk<true>(p, xa, xb, pm2, pm1, srow + c0 * 4, valid);
+            else fe_lrn_chunk<false>(p, xa, xb, pm2, pm1, srow + c0 * 2, valid);
             if (c0 + 32 < C) {
                 fe_load_chunk(taddr, bias_s, c0 + 64, c0 + 64 < C, relu, xa);
-                fe_lrn_chunk(p, xb, xa, pm2, pm1, srow + (c0 + 32) * 2, valid);
+                if (am) fe_lrn_chunk<true>(p, xb, xa, pm2, pm1, srow + (c0 + 32) * 4, valid);
+                else fe_lrn_chunk<false>(p, xb, xa, pm2, pm1, srow + (c0 + 32) * 2, valid);
             }
         }
     } else {
@@ -187,7 +211,72 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
     // ---- 3x3 / 2 max over the staged patch
     __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.y);
     const int npp = p.PH * p.PW;
-    if (lrn_first) {
+    if (am) {
+        // Positions wanted: the maximum is taken on float32 values that have been through everything the layer applies
+        // before pooling (bias and ReLU here if LRN did not come first), window positions in row-major order, a later one
+        // wins only if strictly greater: the first maximum, as the pooling layer defines it.  Rows outside the
+        // convolution plane hold -inf and never win; the first window position inside the plane always does over them.
+        float* pooled = reinterpret_cast<float*>(stage + (size_t)TILE_M * pitch + 256 * 4);
+        const int ldp = C + 8;
+        const bool lrn_after = lrn && !lrn_first;
+        const float NEG = __uint_as_float(0xff800000u);
+        const int C4 = C >> 2;
+        for (int item = row; item < npp * C4; item += FE_THREADS) {
+            const int pp = item / C4, c = (item - pp * C4) << 2;
+            const int ppi = pp / p.PW, ppj = pp - ppi * p.PW;
+            const int ph = th * p.PH + ppi, pw = tw * p.PW + ppj;
+            const uint8_t* base = stage + (size_t)((2 * ppi) * pwc + 2 * ppj) * pitch + c * 4;
+            const float4 b4 = *reinterpret_cast<const float4*>(bias_s + c);
+            float m[4] = {NEG, NEG, NEG, NEG};
+            int w[4] = {-1, -1, -1, -1};
+#pragma unroll
+            for (int d = 0; d < 9; ++d) {
+                const float4 u = *reinterpret_cast<const float4*>(base + (size_t)((d / 3) * pwc + (d % 3)) * pitch);
+                float v[4] = {u.x, u.y, u.z, u.w};
+                const int hh = 2 * ph - 1 + d / 3, ww = 2 * pw - 1 + d % 3;
+                const int pos = hh * p.Wo + ww;
+                if (!lrn_first) {
+                    const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (v[k] != NEG) { v[k] += bb[k]; if (relu) v[k] = fmaxf(v[k], 0.f); }
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (v[k] > m[k]) { m[k] = v[k]; w[k] = pos; }
+            }
+            if (lrn_after) {
+                *reinterpret_cast<float4*>(pooled + pp * ldp + 4 + c) = make_float4(m[0], m[1], m[2], m[3]);
+                if (c == 0) { pooled[pp * ldp + 2] = 0.f; pooled[pp * ldp + 3] = 0.f; pooled[pp * ldp + C + 4] = 0.f; pooled[pp * ldp + C + 5] = 0.f; }
+            }
+            if (ph < p.Hy && pw < p.Wy) {
+                const long long q = ((long long)n * p.Hy + ph) * p.Wy + pw;
+                *reinterpret_cast<int4*>(p.argmax + q * C + c) = make_int4(w[0], w[1], w[2], w[3]);
+                if (!lrn_after) {
+                    uint2 o;
+                    o.x = pack_bf16(m[0], m[1]); o.y = pack_bf16(m[2], m[3]);
+                    *reinterpret_cast<uint2*>(y + q * p.ldc + p.coff + c) = o;
+                }
+            }
+        }
+        if (lrn_after) {
+            fe_bar(bar_id);
+            for (int item = row; item < ((npp * C + FE_THREADS - 1) / FE_THREADS) * FE_THREADS; item += FE_THREADS) {
+                const bool active = item < npp * C;
+                const int it2 = active ? item : npp * C - 1;
+                const int pp = it2 / C, c = it2 - pp * C;
+                const int ppi = pp / p.PW, ppj = pp - ppi * p.PW;
+                const int ph = th * p.PH + ppi, pw = tw * p.PW + ppj;
+                const float* s5 = pooled + pp * ldp + 4 + c;               // two zeros of halo on either side of the row
+                float ss[1] = {(s5[-2] * s5[-2] + s5[-1] * s5[-1]) + (s5[0] * s5[0] + s5[1] * s5[1]) + s5[2] * s5[2]}, sc[1];
+                fe_lrn_scale<1>(p, ss, sc);
+                if (active && ph < p.Hy && pw < p.Wy) {
+                    const long long q = ((long long)n * p.Hy + ph) * p.Wy + pw;
+                    y[q * p.ldc + p.coff + c] = __float2bfloat16_rn(s5[0] * sc[0]);
+                }
+            }
+        }
+    } else if (lrn_first) {
         const int C8 = C >> 3;
         const int dpp = FE_THREADS / C8, dc8 = FE_THREADS - dpp * C8;      // step of the (pp, c8) item index per pass
         int pp = row / C8, c8 = row - pp * C8;

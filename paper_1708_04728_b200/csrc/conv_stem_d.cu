@@ -487,6 +487,7 @@ static int sd_smem_bytes(const ConvParams& p, const SdGeom& g) {
 
 bool conv_stem_d_supports(const ConvParams& p) {
     if (!p.patch || !fe_supports(p) || fe_lrn_first(p)) return false;
+    if (p.argmax) return false;                                      // positions of the maxima: the im2col-building stem kernel returns them
     if (p.k != 7 || p.stride != 2 || p.pad != 3 || p.Cin != 3 || p.Cout != 64 || (p.W & 1)) return false;
     if (p.Wo > 124) return false;                                   // one output row per 128-column MMA
     return sd_smem_bytes(p, sd_geom(p)) + 1024 <= SD_SMEM_MAX;

@@ -200,6 +200,7 @@ __device__ __forceinline__ void lrn_chunk(const ConvParams& p, uint32_t taddr, i
 #pragma unroll
     for (int j = 0; j < W + 4; j += 4) total += (sq[j] + sq[j + 1]) + (sq[j + 2] + sq[j + 3]);
     const bool series = !__any_sync(0xffffffffu, !(total < p.lrn_ss_max));
+    const bool series2 = !__any_sync(0xffffffffu, !(total < p.lrn_ss_max2));   // two terms are exact to float32 resolution
     uint32_t o[W / 2];
 #pragma unroll
     for (int j = 0; j < W; j += 2) {
@@ -208,7 +209,8 @@ __device__ __forceinline__ void lrn_chunk(const ConvParams& p, uint32_t taddr, i
         for (int e = 0; e < 2; ++e) {
             const float s1 = ss[j + e];
             float f;
-            if (series) f = fmaf(s1, fmaf(s1, fmaf(s1, fmaf(s1, p.lrn_s4, p.lrn_s3), p.lrn_s2), p.lrn_s1), p.lrn_kpow);
+            if (series2) f = fmaf(s1, fmaf(s1, p.lrn_s2, p.lrn_s1), p.lrn_kpow);
+            else if (series) f = fmaf(s1, fmaf(s1, fmaf(s1, fmaf(s1, p.lrn_s4, p.lrn_s3), p.lrn_s2), p.lrn_s1), p.lrn_kpow);
             else f = exp2f(-p.lrn_beta * log2f(fmaf(p.lrn_alpha_n, s1, p.lrn_k)));
             y2[e] = x[2 + j + e] * f;
         }

@@ -214,6 +214,9 @@ def check_argmax(got_arg, ref_arg, pre_pool, ref_scale):
     return excused
 
 
+# kernels that return the positions of the pooling maxima
+ARGMAX_PATHS = (1, 2, 4, 5)
+
 # fused pooling / LRN epilogues (Cout <= 256): (B,H,W,Cin,Cout,k,s,p, flags-name)
 STAGED = [
     (1, 64, 64, 3, 64, 7, 2, 3, "pool_lrn"),        # the stem configuration: ReLU -> pool -> LRN
@@ -245,7 +248,7 @@ def test_conv_fused_pool_lrn(dr, O, path, case):
     lrn = (5, 1e-4, 0.75, 1.0) if kind == "pool_lrn" else (5, 0.05, 0.75, 1.0)      # second set makes LRN bite
     force(dr, path)
     try:
-        got, arg = run_conv(dr, x, w, b, k, s, p, flags, lrn=lrn, want_argmax=bool(flags & dr.DR_POOL) and path <= 3)
+        got, arg = run_conv(dr, x, w, b, k, s, p, flags, lrn=lrn, want_argmax=bool(flags & dr.DR_POOL) and path in ARGMAX_PATHS)
     except dr.DrError as e:
         if e.status == dr.DR_ERR_UNSUPPORTED and path != dr.DR_PATH_SIMT:
             pytest.skip("path does not take this shape")
@@ -257,7 +260,34 @@ def test_conv_fused_pool_lrn(dr, O, path, case):
         if flags & dr.DR_LRN_BEFORE_POOL:
             pre = O.lrn(pre, *lrn)
         excused = check_argmax(arg, ref_arg, pre, np.abs(pre).max())
-        assert excused <= 0.02 * arg.size + 8, f"{excused} near-ties of {arg.size}"
+        print(f"\n[argmax {kind} path {path} {case[:5]}] {excused} near-ties excused of {arg.size} positions ({100.0 * excused / arg.size:.3f} %)")
+        assert excused <= 0.005 * arg.size + 8, f"{excused} near-ties of {arg.size}"
+
+
+@pytest.mark.parametrize("path", [0, 1, 2, 4])
+@pytest.mark.parametrize("kind", ["pool", "lrn_pool"])
+def test_fused_pool_argmax_exact_ties_take_the_first_position(dr, O, path, kind):
+    """Windows whose values are all exactly zero after ReLU (a large negative bias on some channels): the stored position
+    must be the first of the window in row-major order, bit for bit, on every kernel that returns positions."""
+    B, H, W, Cin, Cout, k, s, p = 2, 22, 18, 64, 64, 3, 1, 1
+    flags = dr.DR_BIAS | dr.DR_RELU | dr.DR_POOL | (dr.DR_LRN | dr.DR_LRN_BEFORE_POOL if kind == "lrn_pool" else 0)
+    x = S.normal(21, "x", (B, H, W, Cin)); w = S.he_normal(21, "w", Cout, k, Cin); b = S.normal(21, "b", (Cout,), 0.01).copy()
+    dead = np.arange(0, Cout, 3)
+    b[dead] = -64.0                                            # far below any pre-activation: ReLU gives exact zeros
+    force(dr, path)
+    try:
+        got, arg = run_conv(dr, x, w, b, k, s, p, flags, want_argmax=True)
+    except dr.DrError as e:
+        if e.status == dr.DR_ERR_UNSUPPORTED and path != dr.DR_PATH_SIMT:
+            pytest.skip("path does not take this shape")
+        raise
+    ref, ref_arg = oracle_slim_layer(O, x, w, b, k, s, p, flags, dr)
+    assert np.all(ref[..., dead] == 0.0) and np.all(got[..., dead] == 0.0)
+    assert np.array_equal(arg[..., dead], ref_arg[..., dead])
+    # first position of a window: row max(2*ph - 1, 0), column max(2*pw - 1, 0)
+    Hy, Wy = ref.shape[1], ref.shape[2]
+    first = (np.maximum(2 * np.arange(Hy) - 1, 0)[:, None] * W + np.maximum(2 * np.arange(Wy) - 1, 0)[None, :]).astype(np.int32)
+    assert np.array_equal(arg[0, :, :, dead[0]], first)
 
 
 def test_inception_3a_config(dr, O):

@@ -200,3 +200,13 @@ def test_net_timing_and_launch_count(dr):
     first = to_host(logits).copy()
     net.dr_net_forward(x, ws, logits)                  # deterministic: no atomics anywhere
     assert np.array_equal(first, to_host(logits))
+    # tensor maps are remembered by what they were encoded from: further passes over the same buffers encode none
+    net.dr_net_set_timing(False)
+    net.dr_net_forward(x, ws, logits)                  # (layers that share a launch sum in another order than when timed apart)
+    untimed = to_host(logits).copy()
+    e0 = dr.dr_tensor_map_encodes()
+    assert e0 > 0
+    net.dr_net_forward(x, ws, logits)
+    net.dr_net_forward(x, ws, logits)
+    assert dr.dr_tensor_map_encodes() == e0
+    assert np.array_equal(untimed, to_host(logits))

@@ -55,6 +55,18 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
         ref, got = to_host(y_ref), to_host(y_new)
         assert_layer_close(got, ref, f"static scratch, case seed {seed}")
         assert np.array_equal(got, ref)          # same kernels, same order: identical bits
+        # and against the CPU checker's unmerged four-branch module directly, not only through the other entry point
+        import oracle.nets as N
+        params = P.inception_params(seed, "m", {"m": row})
+        want = N.run(N.inception_steps(params, "m", "x", table={"m": row}), S.normal(seed, "x", (B, hw, hw, row[0])))["m"]
+        assert_layer_close(got, want, f"static scratch vs checker, case seed {seed}")
+        # the call itself allocates nothing: free device memory and torch's own pool are the same before and after
+        torch.cuda.synchronize()
+        free0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+        dr.dr_inception_slim_static(d, B, hw, hw, x, w, b, y_new)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
+        assert np.array_equal(to_host(y_new), ref)
 
 
 def test_static_scratch_refuses_oversized_request():
