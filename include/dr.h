@@ -153,8 +153,10 @@ int dr_conv_slim_ws(const dr_conv_desc* desc, int B, int H, int W, const void* x
  *   y[..., 0:c3)      = ReLU(conv3x3(ReLU(conv1x1(x; w[0]) + b[0]); w[1]) + b[1])
  *   y[..., c3:c3+cm)  = ReLU(conv5x5(x; w[2]) + b[2])          (pad 2, the merged branches)
  * written in place into y [B,H,W,c3+cm].  workspace holds the 1x1 output:
- * dr_inception_workspace_bytes() bytes.  pool_after != 0 is not built (UNSUPPORTED): run
- * dr_maxpool on y.                                                                          */
+ * dr_inception_workspace_bytes() bytes.  pool_after != 0: the module is followed by the 3x3 / 2, pad 1 max-pooling layer
+ * that follows inception 3b and 4e (Section 3.1: the pooling layer goes with the layer below it): y is then
+ * [B,Hp,Wp,c3+cm] with Hp = (H - 1) / 2 + 1, the un-pooled output is kept in the workspace (which
+ * dr_inception_workspace_bytes sizes accordingly) and pooled from there by dr_maxpool's kernel.                  */
 typedef struct dr_inception_desc {
     int Cin, c3r, c3, cm;
     int pool_after;

@@ -243,6 +243,8 @@ int dr_conv_slim_ws(const dr_conv_desc* desc, int B, int H, int W, const void* x
 int dr_inception_workspace_bytes(const dr_inception_desc* d, int B, int H, int W, size_t* bytes) {
     if (!d || !bytes || B < 0 || H <= 0 || W <= 0 || d->c3r <= 0) return DR_ERR_INVALID_ARG;
     *bytes = ((size_t)B * H * W * d->c3r * 2 + 255) / 256 * 256;
+    // pool_after: the module output before pooling lives in the workspace as well
+    if (d->pool_after) *bytes += ((size_t)B * H * W * ((size_t)d->c3 + d->cm) * 2 + 255) / 256 * 256;
     return DR_OK;
 }
 
@@ -250,12 +252,16 @@ int dr_inception_slim(const dr_inception_desc* d, int B, int H, int W, const voi
                       const float* const b[3], void* y, void* workspace, void* stream) {
     if (!d || !x || !w || !b || !y) return DR_ERR_INVALID_ARG;
     if (d->Cin <= 0 || d->c3r <= 0 || d->c3 <= 0 || d->cm <= 0) return DR_ERR_INVALID_ARG;
-    if (d->pool_after) return DR_ERR_UNSUPPORTED;
     if (!workspace) return DR_ERR_WORKSPACE;
     for (int i = 0; i < 3; ++i)
         if (!w[i] || !b[i]) return DR_ERR_INVALID_ARG;
     if ((d->c3 & 7) || (d->cm & 7)) return DR_ERR_ALIGNMENT;
     const int ldc = d->c3 + d->cm;
+    // pool_after: both convolutions write the un-pooled module output into the workspace (behind the reducer's tensor) and a
+    // 3x3 / 2, pad 1 max-pooling layer brings it to y.  (Pooling is per channel, so it commutes with the concatenation; it is
+    // not absorbed into these convolutions' epilogues: their tiles are runs of 128 consecutive pixels, not 2-D patches.)
+    void* y_out = y;
+    if (d->pool_after) y = (char*)workspace + ((size_t)B * H * W * d->c3r * 2 + 255) / 256 * 256;
     dr_conv_desc c{};
     c.flags = DR_BIAS | DR_RELU;
     // 1x1 reducer of the 3x3 path -> workspace
@@ -268,7 +274,9 @@ int dr_inception_slim(const dr_inception_desc* d, int B, int H, int W, const voi
     if (st != DR_OK) return st;
     // merged 5x5 on the module input -> channels [c3, c3+cm)
     c.k = 5; c.pad = 2; c.Cin = d->Cin; c.Cout = d->cm; c.y_ldc = ldc; c.y_coff = d->c3;
-    return dr_conv_slim(&c, B, H, W, x, w[2], b[2], nullptr, y, nullptr, stream);
+    st = dr_conv_slim(&c, B, H, W, x, w[2], b[2], nullptr, y, nullptr, stream);
+    if (st != DR_OK || !d->pool_after) return st;
+    return dr_maxpool(B, H, W, ldc, 3, 2, 1, y, y_out, nullptr, stream);
 }
 
 // ---- dr_inception_slim_static: the same module with its scratch tensor in a fixed device array ----

@@ -5,6 +5,8 @@
 // the activations each.  On this hardware they are bound by HBM bandwidth, so every kernel
 // moves 128 bits per thread per access, coalesced along the channel axis of NHWC, with a grid
 // sized to a few waves of the SMs.
+#include <cmath>
+
 #include "common.cuh"
 
 namespace dr {
@@ -35,7 +37,12 @@ int num_sms() {
 static inline int grid_for(size_t work_items, int threads) {
     size_t blocks = (work_items + threads - 1) / threads;
     size_t cap = (size_t)num_sms() * 16;           // grid-stride beyond 16 blocks per SM
-    if (blocks > cap) blocks = cap;
+    if (blocks > cap) {
+        // every thread the same number of items: a grid of `cap` blocks over 1.2 x cap blocks' worth of work would run a
+        // second, mostly idle round
+        const size_t iters = (blocks + cap - 1) / cap;
+        blocks = (blocks + iters - 1) / iters;
+    }
     if (blocks < 1) blocks = 1;
     return (int)blocks;
 }
@@ -85,8 +92,11 @@ __global__ void bn_kernel(size_t nvec, int C8, const uint4* __restrict__ x, cons
                           const float* __restrict__ var, float inv_m, float eps, const float* __restrict__ gamma,
                           const float* __restrict__ beta, uint4* __restrict__ y) {
     const size_t stride = (size_t)gridDim.x * blockDim.x;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
-        const int c0 = (int)(i % C8) * 8;
+    const size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int c8 = (int)(i0 % C8);                              // the channel group advances by a fixed step: one division per thread
+    const int step = (int)(stride % C8);
+    for (size_t i = i0; i < nvec; i += stride, c8 = c8 + step >= C8 ? c8 + step - C8 : c8 + step) {
+        const int c0 = c8 * 8;
         uint4 v = __ldg(x + i);
         uint32_t* u = reinterpret_cast<uint32_t*>(&v);
 #pragma unroll
@@ -103,35 +113,46 @@ __global__ void bn_kernel(size_t nvec, int C8, const uint4* __restrict__ x, cons
         y[i] = v;
     }
 }
-// The same with the per-channel constants (mean/m, gamma/sqrt(var/m + eps), beta) computed once per block into shared
-// memory (C <= 4096): per 8 elements six 16-byte shared loads instead of 32 scalar global loads and 8 rsqrt.
+// The same with the per-channel constants folded to y = a x + b' (a = gamma / sqrt(var/m + eps), b' = beta - a mean/m)
+// and computed once per block into shared memory (C <= 4096).  A thread's channel group advances by a fixed step from
+// one vector to its next; when that step is zero (the grid stride is a multiple of the channel groups, the usual case)
+// the sixteen constants stay in registers for the whole loop, otherwise they are four 16-byte shared loads per vector
+// (read per vector, the three-constant form asked more of shared memory than the loads and stores of the data).
 __global__ void bn_smem_kernel(size_t nvec, int C8, const uint4* __restrict__ x, const float* __restrict__ mean,
                                const float* __restrict__ var, float inv_m, float eps, const float* __restrict__ gamma,
                                const float* __restrict__ beta, uint4* __restrict__ y) {
-    extern __shared__ float bn_s[];                       // [3][C]: mu, a, b
+    extern __shared__ float bn_s[];                       // [2][C]: a, b'
     const int C = C8 * 8;
     for (int c = threadIdx.x; c < C; c += blockDim.x) {
-        bn_s[c] = mean ? __ldg(mean + c) * inv_m : 0.f;
-        bn_s[C + c] = (gamma ? __ldg(gamma + c) : 1.f) * (mean ? rsqrtf(__ldg(var + c) * inv_m + eps) : 1.f);
-        bn_s[2 * C + c] = gamma ? __ldg(beta + c) : 0.f;
+        const float a = (gamma ? __ldg(gamma + c) : 1.f) * (mean ? rsqrtf(__ldg(var + c) * inv_m + eps) : 1.f);
+        bn_s[c] = a;
+        bn_s[C + c] = (gamma ? __ldg(beta + c) : 0.f) - a * (mean ? __ldg(mean + c) * inv_m : 0.f);
     }
     __syncthreads();
     const size_t stride = (size_t)gridDim.x * blockDim.x;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
-        const int c0 = (int)(i % C8) * 8;
-        uint4 v = __ldg(x + i);
-        uint32_t* u = reinterpret_cast<uint32_t*>(&v);
-        float mu[8], a[8], b[8];
+    const size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int c8 = (int)(i0 % C8);
+    const int step = (int)(stride % C8);
+    float a[8], b[8];
+    auto load_consts = [&](int c0) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            *reinterpret_cast<float4*>(mu + 4 * h) = *reinterpret_cast<const float4*>(bn_s + c0 + 4 * h);
-            *reinterpret_cast<float4*>(a + 4 * h) = *reinterpret_cast<const float4*>(bn_s + C + c0 + 4 * h);
-            *reinterpret_cast<float4*>(b + 4 * h) = *reinterpret_cast<const float4*>(bn_s + 2 * C + c0 + 4 * h);
+            *reinterpret_cast<float4*>(a + 4 * h) = *reinterpret_cast<const float4*>(bn_s + c0 + 4 * h);
+            *reinterpret_cast<float4*>(b + 4 * h) = *reinterpret_cast<const float4*>(bn_s + C + c0 + 4 * h);
         }
+    };
+    load_consts(c8 * 8);
+    for (size_t i = i0; i < nvec; i += stride) {
+        uint4 v = __ldg(x + i);
+        uint32_t* u = reinterpret_cast<uint32_t*>(&v);
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-            u[j] = pack_bf16((bf16_lo(u[j]) - mu[2 * j]) * a[2 * j] + b[2 * j], (bf16_hi(u[j]) - mu[2 * j + 1]) * a[2 * j + 1] + b[2 * j + 1]);
+            u[j] = pack_bf16(fmaf(bf16_lo(u[j]), a[2 * j], b[2 * j]), fmaf(bf16_hi(u[j]), a[2 * j + 1], b[2 * j + 1]));
         y[i] = v;
+        if (step) {
+            c8 = c8 + step >= C8 ? c8 + step - C8 : c8 + step;
+            load_consts(c8 * 8);
+        }
     }
 }
 __global__ void bn_scalar_kernel(size_t n, int C, const __nv_bfloat16* __restrict__ x, const float* __restrict__ mean,
@@ -229,11 +250,19 @@ __global__ void maxpool3_noarg_kernel(int B, int H, int W, int C8, int Ho, int W
     const size_t total = (size_t)B * Ho * Wo * C8;
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-        const int c8 = (int)(i % C8);
-        size_t q = i / C8;
-        const int wo = (int)(q % Wo); q /= Wo;
-        const int ho = (int)(q % Ho);
-        const size_t n = q / Ho;
+        // the index is split with 32-bit divisions where it fits (a 64-bit division costs several times the rest of the body)
+        int c8, wo, ho;
+        size_t n;
+        if (total <= 0xffffffffull) {
+            const unsigned iu = (unsigned)i, q1 = iu / (unsigned)C8, q2 = q1 / (unsigned)Wo, q3 = q2 / (unsigned)Ho;
+            c8 = (int)(iu - q1 * (unsigned)C8); wo = (int)(q1 - q2 * (unsigned)Wo); ho = (int)(q2 - q3 * (unsigned)Ho); n = q3;
+        } else {
+            c8 = (int)(i % C8);
+            size_t q = i / C8;
+            wo = (int)(q % Wo); q /= Wo;
+            ho = (int)(q % Ho);
+            n = q / Ho;
+        }
         const int h0 = ho * s - p, w0 = wo * s - p;
         uint4 v[9];
         bool ok[9];
@@ -256,6 +285,62 @@ __global__ void maxpool3_noarg_kernel(int B, int H, int W, int C8, int Ho, int W
             for (int j = 0; j < 4; ++j) mm[j] = __hmax2(mm[j], uu[j]);
         }
         y[i] = m;
+    }
+}
+// 3x3 / stride 2: a thread takes a 2 x 2 block of pooled positions (8 channels), whose windows cover 5 x 5 inputs:
+// 25 loads for four outputs instead of 36, all issued before the first maximum.  Taps outside the plane load a clamped,
+// valid address and are replaced by -inf.
+__global__ void __launch_bounds__(256) maxpool3s2_quad_kernel(int B, int H, int W, int C8, int Ho, int Wo, int p, const uint4* __restrict__ x,
+                                                              uint4* __restrict__ y) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see maxpool_kernel
+    const unsigned Ho2 = (unsigned)(Ho + 1) >> 1, Wo2 = (unsigned)(Wo + 1) >> 1;
+    const unsigned total = (unsigned)B * Ho2 * Wo2 * (unsigned)C8;     // the host keeps this below 2^32
+    const unsigned stride = gridDim.x * blockDim.x;
+    const uint4 NEG = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // -inf: padding never wins
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const unsigned q1 = i / (unsigned)C8, q2 = q1 / Wo2, n = q2 / Ho2;
+        const int c8 = (int)(i - q1 * (unsigned)C8), wo = 2 * (int)(q1 - q2 * Wo2), ho = 2 * (int)(q2 - n * Ho2);
+        const int h0 = 2 * ho - p, w0 = 2 * wo - p;
+        const uint4* img = x + (size_t)n * H * W * C8 + c8;
+        uint4 v[25];
+#pragma unroll
+        for (int r = 0; r < 5; ++r)
+#pragma unroll
+            for (int t = 0; t < 5; ++t) {
+                const int hi = h0 + r, wi = w0 + t;
+                const int hc = min(max(hi, 0), H - 1), wc = min(max(wi, 0), W - 1);
+                const uint4 u = __ldg(img + ((size_t)hc * W + wc) * C8);
+                v[5 * r + t] = (hi == hc && wi == wc) ? u : NEG;
+            }
+        // column-wise maxima of the three rows each pooled row needs, then across columns
+#pragma unroll
+        for (int a = 0; a < 2; ++a) {
+            uint4 colmax[5];
+#pragma unroll
+            for (int t = 0; t < 5; ++t) {
+                uint4 m = v[5 * (2 * a) + t];
+                __nv_bfloat162* mm = reinterpret_cast<__nv_bfloat162*>(&m);
+#pragma unroll
+                for (int r = 1; r < 3; ++r) {
+                    const __nv_bfloat162* uu = reinterpret_cast<const __nv_bfloat162*>(&v[5 * (2 * a + r) + t]);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) mm[k] = __hmax2(mm[k], uu[k]);
+                }
+                colmax[t] = m;
+            }
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                uint4 m = colmax[2 * b];
+                __nv_bfloat162* mm = reinterpret_cast<__nv_bfloat162*>(&m);
+#pragma unroll
+                for (int t = 1; t < 3; ++t) {
+                    const __nv_bfloat162* uu = reinterpret_cast<const __nv_bfloat162*>(&colmax[2 * b + t]);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) mm[k] = __hmax2(mm[k], uu[k]);
+                }
+                if (ho + a < Ho && wo + b < Wo) y[(((size_t)n * Ho + ho + a) * Wo + wo + b) * C8 + c8] = m;
+            }
+        }
     }
 }
 __global__ void maxpool_scalar_kernel(int B, int H, int W, int C, int Ho, int Wo, int k, int s, int p,
@@ -296,12 +381,17 @@ __device__ __forceinline__ void unpack8(const uint4& q, float* v) {
 }
 // MAXH: largest half-window this instantiation handles (2 for the usual window of five: two predicated steps
 // instead of eight)
+// The scale (kappa + alpha_n ss)^(-beta) = kappa^(-beta) (1 + u)^(-beta), u = alpha_n ss / kappa: while u < 1/256 for all
+// eight sums of every lane of the warp, its series to the u^2 term is exact to float32 resolution (the next term is below
+// 4e-8) and needs no special-function unit; ser = {kappa^(-beta), c1 alpha_n / kappa ..., c2 (alpha_n / kappa)^2 ..., the ss limit}.
 template <int MAXH>
-__global__ void lrn_kernel(size_t nvec, int C8, int half, float alpha_n, float beta, float kappa,
+__global__ void lrn_kernel(size_t nvec, int C8, int half, float alpha_n, float beta, float kappa, float4 ser,
                            const uint4* __restrict__ x, uint4* __restrict__ y) {
     const size_t stride = (size_t)gridDim.x * blockDim.x;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
-        const int c8 = (int)(i % C8);
+    const size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int c8 = (int)(i0 % C8);                              // advances by a fixed step: one division per thread
+    const int step = (int)(stride % C8);
+    for (size_t i = i0; i < nvec; i += stride, c8 = c8 + step >= C8 ? c8 + step - C8 : c8 + step) {
         float v[24];
         unpack8(__ldg(x + i), v + 8);
         if (c8 > 0) unpack8(__ldg(x + i - 1), v);
@@ -317,14 +407,22 @@ __global__ void lrn_kernel(size_t nvec, int C8, int half, float alpha_n, float b
         float sq[24];
 #pragma unroll
         for (int j = 0; j < 24; ++j) sq[j] = v[j] * v[j];
-        float r[8];
+        float r[8], ssv[8], smax = 0.f;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             float ss = sq[8 + j];
 #pragma unroll
             for (int d = 1; d <= MAXH; ++d)
                 if (d <= half) ss += sq[8 + j - d] + sq[8 + j + d];
-            r[j] = v[8 + j] * lrn_pow(kappa + alpha_n * ss, beta);
+            ssv[j] = ss;
+            smax = fmaxf(smax, ss);
+        }
+        if (__all_sync(__activemask(), smax < ser.w)) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) r[j] = v[8 + j] * fmaf(ssv[j], fmaf(ssv[j], ser.z, ser.y), ser.x);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) r[j] = v[8 + j] * lrn_pow(kappa + alpha_n * ssv[j], beta);
         }
         uint4 o;
         uint32_t* uo = reinterpret_cast<uint32_t*>(&o);
@@ -365,33 +463,41 @@ __global__ void concat_scalar_kernel(size_t n, int C, int ldc, int coff, const _
 // ---------------------------------------------------------------- global average pool
 // One block per (image, 64-channel slab): threads split the plane, partial sums meet in shared
 // memory in a fixed order (deterministic).  blockDim = (64 channels / 2, PIXSPLIT).
-// For C a multiple of 8: one block per (image, slab of 32 x 8 channels), blockDim = (32, 8): a thread sums every 8th
-// position of its 8 channels with 16-byte loads; the eight partial sums meet in shared memory in a fixed order.
-__global__ void avgpool8_kernel(int HW, int C8, const uint4* __restrict__ x, uint4* __restrict__ y) {
-    __shared__ float part[8][32][9];
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see maxpool_noarg_kernel
-    const int n = blockIdx.y, c8 = blockIdx.x * 32 + threadIdx.x;
+// For C a multiple of 8: one block per (image, slab of 64 channels), blockDim = (8 channel groups, 32 pixel lanes): a
+// thread sums every 32nd position of its 8 channels (16-byte loads, all of them in flight at once for planes up to 64
+// pixels); the 32 partial sums of a channel meet in shared memory and are added in lane order (deterministic).
+__global__ void __launch_bounds__(256) avgpool8_kernel(int HW, int C8, const uint4* __restrict__ x, uint4* __restrict__ y) {
+    __shared__ float part[32][8][9];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see maxpool_kernel
+    const int n = blockIdx.y, c8 = blockIdx.x * 8 + threadIdx.x, py = threadIdx.y;
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     if (c8 < C8) {
-        for (int q = threadIdx.y; q < HW; q += 8) {
-            const uint4 v = __ldg(x + ((size_t)n * HW + q) * C8 + c8);
+        const uint4* src = x + (size_t)n * HW * C8 + c8;
+        for (int q0 = py; q0 < HW; q0 += 64) {
+            const bool two = q0 + 32 < HW;
+            const uint4 v = __ldg(src + (size_t)q0 * C8);
+            const uint4 u = two ? __ldg(src + (size_t)(q0 + 32) * C8) : make_uint4(0, 0, 0, 0);
             acc[0] += bf16_lo(v.x); acc[1] += bf16_hi(v.x); acc[2] += bf16_lo(v.y); acc[3] += bf16_hi(v.y);
             acc[4] += bf16_lo(v.z); acc[5] += bf16_hi(v.z); acc[6] += bf16_lo(v.w); acc[7] += bf16_hi(v.w);
+            acc[0] += bf16_lo(u.x); acc[1] += bf16_hi(u.x); acc[2] += bf16_lo(u.y); acc[3] += bf16_hi(u.y);
+            acc[4] += bf16_lo(u.z); acc[5] += bf16_hi(u.z); acc[6] += bf16_lo(u.w); acc[7] += bf16_hi(u.w);
         }
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) part[threadIdx.y][threadIdx.x][j] = acc[j];
+    for (int j = 0; j < 8; ++j) part[py][threadIdx.x][j] = acc[j];
     __syncthreads();
-    if (threadIdx.y == 0 && c8 < C8) {
-        float t[8];
+    const int t = py * 8 + threadIdx.x;                  // 64 threads finish: (channel group, channel)
+    if (t < 64) {
+        const int g = t >> 3, j = t & 7;
+        float sum = 0.f;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            t[j] = 0.f;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) t[j] += part[k][threadIdx.x][j];
-            t[j] = t[j] / (float)HW;
-        }
-        y[(size_t)n * C8 + c8] = make_uint4(pack_bf16(t[0], t[1]), pack_bf16(t[2], t[3]), pack_bf16(t[4], t[5]), pack_bf16(t[6], t[7]));
+        for (int k = 0; k < 32; ++k) sum += part[k][g][j];
+        part[0][g][j] = sum / (float)HW;
+    }
+    __syncthreads();
+    if (py == 0 && c8 < C8) {
+        const float* r = part[0][threadIdx.x];
+        y[(size_t)n * C8 + c8] = make_uint4(pack_bf16(r[0], r[1]), pack_bf16(r[2], r[3]), pack_bf16(r[4], r[5]), pack_bf16(r[6], r[7]));
     }
 }
 
@@ -621,7 +727,7 @@ int dr_bn(int B, int H, int W, int C, const void* x, const float* mean, const fl
     if (n == 0) return DR_OK;
     DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
     if (C % 8 == 0 && C <= 4096)
-        bn_smem_kernel<<<grid_for(n / 8, 256), 256, 3 * C * sizeof(float), (cudaStream_t)stream>>>(n / 8, C / 8, (const uint4*)x, mean, var, 1.f / m, eps, gamma, beta, (uint4*)y);
+        bn_smem_kernel<<<grid_for(n / 8, 256), 256, 2 * C * sizeof(float), (cudaStream_t)stream>>>(n / 8, C / 8, (const uint4*)x, mean, var, 1.f / m, eps, gamma, beta, (uint4*)y);
     else if (C % 8 == 0)
         bn_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, C / 8, (const uint4*)x, mean, var, 1.f / m, eps, gamma, beta, (uint4*)y);
     else
@@ -637,7 +743,7 @@ int dr_scale(int B, int H, int W, int C, const void* x, const float* gamma, cons
     if (n == 0) return DR_OK;
     DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
     if (C % 8 == 0 && C <= 4096)
-        bn_smem_kernel<<<grid_for(n / 8, 256), 256, 3 * C * sizeof(float), (cudaStream_t)stream>>>(n / 8, C / 8, (const uint4*)x, nullptr, nullptr, 1.f, 0.f, gamma, beta, (uint4*)y);
+        bn_smem_kernel<<<grid_for(n / 8, 256), 256, 2 * C * sizeof(float), (cudaStream_t)stream>>>(n / 8, C / 8, (const uint4*)x, nullptr, nullptr, 1.f, 0.f, gamma, beta, (uint4*)y);
     else if (C % 8 == 0)
         bn_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, C / 8, (const uint4*)x, nullptr, nullptr, 1.f, 0.f, gamma, beta, (uint4*)y);
     else
@@ -654,7 +760,9 @@ int dr_maxpool(int B, int H, int W, int C, int k, int s, int p, const void* x, v
     const size_t n = (size_t)B * Ho * Wo * C;
     if (n == 0) return DR_OK;
     DR_REQUIRE(aligned16(x) && aligned16(y) && (!argmax || aligned16(argmax)), DR_ERR_ALIGNMENT);
-    if (C % 8 == 0 && !argmax && k == 3)
+    if (C % 8 == 0 && !argmax && k == 3 && s == 2 && (size_t)B * ((Ho + 1) / 2) * ((Wo + 1) / 2) * (C / 8) < 0xffffffffull)
+        maxpool3s2_quad_kernel<<<grid_for((size_t)B * ((Ho + 1) / 2) * ((Wo + 1) / 2) * (C / 8), 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C / 8, Ho, Wo, p, (const uint4*)x, (uint4*)y);
+    else if (C % 8 == 0 && !argmax && k == 3)
         maxpool3_noarg_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C / 8, Ho, Wo, s, p, (const uint4*)x, (uint4*)y);
     else if (C % 8 == 0 && !argmax)
         maxpool_noarg_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C / 8, Ho, Wo, k, s, p, (const uint4*)x, (uint4*)y);
@@ -672,11 +780,16 @@ int dr_lrn(int B, int H, int W, int C, int size, float alpha, float beta, float 
     const size_t n = (size_t)B * H * W * C;
     if (n == 0) return DR_OK;
     DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
+    float4 ser = make_float4(0.f, 0.f, 0.f, -1.f);          // no series unless kappa > 0 and alpha >= 0
+    if (k > 0.f && alpha >= 0.f) {
+        const double au = (double)(alpha / size) / k, kp = pow((double)k, -(double)beta), be = beta;
+        ser = make_float4((float)kp, (float)(-be * kp * au), (float)(be * (be + 1) / 2 * kp * au * au), au > 0 ? (float)(0.00390625 / au) : 3.0e38f);
+    }
     if (C % 8 == 0)
         if (size / 2 <= 2)
-            lrn_kernel<2><<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, C / 8, size / 2, alpha / size, beta, k, (const uint4*)x, (uint4*)y);
+            lrn_kernel<2><<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, C / 8, size / 2, alpha / size, beta, k, ser, (const uint4*)x, (uint4*)y);
         else
-            lrn_kernel<8><<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, C / 8, size / 2, alpha / size, beta, k, (const uint4*)x, (uint4*)y);
+            lrn_kernel<8><<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(n / 8, C / 8, size / 2, alpha / size, beta, k, ser, (const uint4*)x, (uint4*)y);
     else
         lrn_scalar_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(n, C, size / 2, alpha / size, beta, k, (const __nv_bfloat16*)x, (__nv_bfloat16*)y);
     count_launch();
@@ -702,7 +815,7 @@ int dr_avgpool_global(int B, int H, int W, int C, const void* x, void* y, void* 
     DR_REQUIRE(aligned16(x) && aligned16(y), DR_ERR_ALIGNMENT);
     DR_REQUIRE(C % 2 == 0, DR_ERR_UNSUPPORTED);
     if (C % 8 == 0) {
-        dim3 grid((C / 8 + 31) / 32, B), block(32, 8);
+        dim3 grid((C / 8 + 7) / 8, B), block(8, 32);
         avgpool8_kernel<<<grid, block, 0, (cudaStream_t)stream>>>(H * W, C / 8, (const uint4*)x, (uint4*)y);
         count_launch();
         return launch_status();

@@ -322,6 +322,37 @@ def test_inception_3a_config(dr, O):
     assert_layer_close(got[..., c3:], forced["3a.m5"], "3a.m5")
 
 
+def test_inception_with_pooling_after(dr, O):
+    """pool_after: the module followed by the 3x3 / 2 max-pooling layer of inception 3b / 4e, odd plane (13 x 15)."""
+    import oracle.nets as N
+    import torch
+    row = (64, 32, 64, 96, 16, 32, 32)                   # (Cin; c1, c3r, c3, c5r, c5, pp): a small module
+    cin, c1, c3r, c3, _, c5, pp = row
+    cm = c1 + c5 + pp
+    params = P.inception_params(3, "m", {"m": row})
+    B, H, W = 3, 13, 15
+    x = S.normal(3, "x", (B, H, W, cin))
+    wm = torch.empty((cm, 5, 5, cin), dtype=torch.bfloat16, device="cuda")
+    dr.dr_embed_filter(c1, cin, 1, 5, to_dev_bf16(params["m.b1.w"]), 0, wm)
+    dr.dr_embed_filter(c5, cin, 5, 5, to_dev_bf16(params["m.b5.w"]), c1, wm)
+    dr.dr_embed_filter(pp, cin, 3, 5, to_dev_bf16(params["m.bp.w"]), c1 + c5, wm)
+    bm = to_dev_f32(np.concatenate([params["m.b1.b"], params["m.b5.b"], params["m.bp.b"]]))
+    d = dr.dr_inception_desc(Cin=cin, c3r=c3r, c3=c3, cm=cm, pool_after=1)
+    d0 = dr.dr_inception_desc(Cin=cin, c3r=c3r, c3=c3, cm=cm, pool_after=0)
+    need = dr.dr_inception_workspace_bytes(d, B, H, W)
+    assert need >= dr.dr_inception_workspace_bytes(d0, B, H, W) + B * H * W * (c3 + cm) * 2
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    Hp, Wp = (H - 1) // 2 + 1, (W - 1) // 2 + 1
+    y = torch.full((B, Hp, Wp, c3 + cm), 768.0, dtype=torch.bfloat16, device="cuda")
+    dr.dr_set_conv_path(dr.DR_PATH_AUTO)
+    dr.dr_inception_slim(d, B, H, W, to_dev_bf16(x), [to_dev_bf16(params["m.3x3r.w"]), to_dev_bf16(params["m.3x3.w"]), wm],
+                         [to_dev_f32(params["m.3x3r.b"]), to_dev_f32(params["m.3x3.b"]), bm], y, ws)
+    assert dr.dr_device_status()[0] == 0
+    full = N.run(N.inception_steps(params, "m", "x", table={"m": row}), x)["m"]
+    want, _ = O.maxpool(O.round_bf16(full), 3, 2, 1)
+    assert_layer_close(to_host(y), want, "module + pool")
+
+
 def test_bounded_wait_reports_timeout_and_context_survives(dr, O):
     """A wait that can never be satisfied runs out after its limit, leaves DR_ERR_DEVICE_TIMEOUT in the status
     record, and the next layer on the same context still computes correctly."""
