@@ -114,10 +114,10 @@ int conv_make_params(const dr_conv_desc* d, int B, int H, int W, const void* x, 
 }
 
 // The patch-reuse kernel against the im2col kernel: its tiles are whole padded image rows, so part of every tile's MMA
-// rows is padding (28 x 28 planes: 12.5 %).  Measured at batch 256 it is behind the im2col kernel on every GoogLeNet layer
-// (3a merged 5x5: 340 vs 247 us; 3b: 676 vs 596 us): those layers are bound by the rate at which one thread can issue
-// MMAs and hand stages over, not by filling shared memory, so the padding rows cost more than the saved loads give.
-// Chosen only on request (DR_QLIN=1, or the forced path).
+// rows is padding (28 x 28 planes: 12.5 %, 14 x 14: 23 %).  Measured at batch 256 (GoogLeNet) it is level with the im2col
+// kernel where that one is bound by filling shared memory and behind it elsewhere (us, patch-reuse / im2col: 3a merged
+// 5x5 221 / 215, 3b 541 / 475, 4a 320 / 246; 3x3 of 3a 76 / 72, 3b 82 / 90, 4d 66 / 68, 4e 72 / 68): the saved loads
+// are paid back in padding rows.  Chosen only on request (DR_QLIN=1, or the forced path).
 static bool qlin_preferred(const ConvParams& p) {
     return tunable("DR_QLIN", 0) > 0 && conv_qlin_supports(p);
 }

@@ -16,7 +16,9 @@
 //
 // CTA pairs (cta_group::2, M = 256: each CTA its own tile and patch, half of every filter tile), accumulators in
 // TMEM, double-buffered across tiles (or, WIDE: two n sub-blocks of one tile at TMEM columns 0 and 256 sharing the patch),
-// roles as in conv_umma_tma_kernel: warp 0 producer, warp 1 MMA issue, warps 2-5 / 6-9 two epilogue groups.
+// roles as in conv_umma_tma_kernel: warp 0 producer, warp 1 MMA issue (WIDE: a second issuing warp for the second
+// sub-block), warps 2-5 / 6-9 two epilogue groups.  A stage of the filter ring holds the tiles of several consecutive taps (a whole
+// filter row where three such stages fit), so one barrier hand-over covers that many times four MMAs.
 // Every wait is bounded; on a timeout the CTA records DR_ERR_DEVICE_TIMEOUT, all roles leave, TMEM is released.
 #include "conv_common.cuh"
 #include "umma_ptx.cuh"
@@ -25,7 +27,8 @@
 namespace dr {
 using namespace ptx;
 
-constexpr int Q_THREADS = 320;
+constexpr int Q_THREADS = 352;      // warp 0 producer, warp 1 MMA issue, warps 2-5 / 6-9 epilogue groups, warp 10 second MMA issuer (WIDE)
+constexpr int Q_MMA2_WARP = 10;
 constexpr int Q_MAX_STAGES = 12;
 constexpr int Q_BIAS_MAX = 512;
 constexpr int Q_SMEM_MAX = 227 * 1024 - 4096;   // dynamic part; the static part holds barriers and the bias copy
@@ -41,6 +44,7 @@ struct QlinPlan {
     int a_bytes, a_tx;                 // patch buffer (1024-byte multiple) and the bytes one patch load delivers
     int b_sub_bytes;                   // one CTA's half of one filter sub-tile (1024-byte multiple)
     int stages, wide, m_tiles;
+    int tps;                           // filter taps per stage of the filter ring: one barrier hand-over covers 4 * tps MMAs
 };
 
 template <bool WIDE>
@@ -61,10 +65,10 @@ conv_qlin_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, 
     const int stages = pl.stages;
 
     if (tid == 0) {
-        for (int s = 0; s < stages; ++s) { mbar_init(&sh.bfull[s], 1); mbar_init(&sh.bempty[s], 1); }
+        for (int s = 0; s < stages; ++s) { mbar_init(&sh.bfull[s], 1); mbar_init(&sh.bempty[s], WIDE ? 2 : 1); }   // WIDE: both issuers commit
         for (int a = 0; a < 2; ++a) {
-            mbar_init(&sh.afull[a], 1); mbar_init(&sh.aempty[a], 1);
-            mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 8 * (WIDE ? 2 : 1));
+            mbar_init(&sh.afull[a], 1); mbar_init(&sh.aempty[a], WIDE ? 2 : 1);
+            mbar_init(&sh.tfull[a], WIDE ? 2 : 1); mbar_init(&sh.tempty[a], 8 * (WIDE ? 2 : 1));
         }
         sh.abort = 0;
         fence_barrier_init();
@@ -88,14 +92,16 @@ conv_qlin_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, 
     const int Nj1 = WIDE ? cout16 - p.Nt : 0;                   // second sub-block (WIDE)
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t b_base = smem_base + 2u * (uint32_t)pl.a_bytes;
-    const uint32_t b_stage_bytes = (uint32_t)pl.b_sub_bytes * (WIDE ? 2u : 1u);
+    const uint32_t b_tap_bytes = (uint32_t)pl.b_sub_bytes * (WIDE ? 2u : 1u);   // one tap's filter tile(s)
+    const uint32_t b_stage_bytes = b_tap_bytes * (uint32_t)pl.tps;                // a stage: the tiles of `tps` consecutive taps
     const uint32_t bfull0 = smem_u32(&sh.bfull[0]), bempty0 = smem_u32(&sh.bempty[0]);
     const uint32_t afull0 = smem_u32(&sh.afull[0]), aempty0 = smem_u32(&sh.aempty[0]);
 
     if (warp == 0) {
         if (lane == 0) {
-            // -------------------------------------------- TMA producer: per channel block one patch, then the taps' filter tiles
-            const uint32_t b_tx = (uint32_t)(p.Nt >> 1) * 128u * (WIDE ? 2u : 1u);   // a box always delivers its full size (rows past the tensor: zeros)
+            // -------------------------------------------- TMA producer: per channel block one patch, then one stage per
+            // filter row: the filter tiles of its k taps
+            const uint32_t b_tx = (uint32_t)(p.Nt >> 1) * 128u * (WIDE ? 2u : 1u);   // per tap; boxes always deliver their full size
             int s = 0, ia = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -117,7 +123,8 @@ conv_qlin_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, 
                     const uint32_t fa = (afull0 + 8 * ab) & PEER_BIT_MASK;
                     if (rank == 0) mbar_expect_tx_u32(fa, 2u * (uint32_t)pl.a_tx);
                     tma_load_4d_u32<true>(smem_base + (uint32_t)ab * (uint32_t)pl.a_bytes, &map_a, fa, cb << 6, -p.pad, i0 - p.pad, img, 1u);
-                    for (int tap = 0; tap < taps; ++tap) {
+                    for (int tap = 0; tap < taps;) {
+                        const int nt = min(pl.tps, taps - tap);
                         if (!ready && !mbar_wait_slow_u32(bempty0 + 8 * s, ph ^ 1, abort_flag)) {
                             if (!*abort_flag) report_timeout(p.status, 72, t);
                             *abort_flag = 1;
@@ -129,10 +136,12 @@ conv_qlin_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, 
                         if (s2 == stages) { s2 = 0; ph2 ^= 1; }
                         ready = mbar_test_u32(bempty0 + 8 * s2, ph2 ^ 1);      // probe the next slot while this one is filled
                         const uint32_t fb = (bfull0 + 8 * s) & PEER_BIT_MASK;
-                        const uint32_t dst = b_base + (uint32_t)s * b_stage_bytes;
-                        if (rank == 0) mbar_expect_tx_u32(fb, 2u * b_tx);
-                        tma_load_3d_u32<true>(dst, &map_b, fb, cb << 6, tap, brow, 1u);
-                        if (WIDE) tma_load_3d_u32<true>(dst + (uint32_t)pl.b_sub_bytes, &map_b, fb, cb << 6, tap, brow1, 1u);
+                        uint32_t dst = b_base + (uint32_t)s * b_stage_bytes;
+                        if (rank == 0) mbar_expect_tx_u32(fb, 2u * b_tx * (uint32_t)nt);
+                        for (int j = 0; j < nt; ++j, ++tap, dst += b_tap_bytes) {
+                            tma_load_3d_u32<true>(dst, &map_b, fb, cb << 6, tap, brow, 1u);
+                            if (WIDE) tma_load_3d_u32<true>(dst + (uint32_t)pl.b_sub_bytes, &map_b, fb, cb << 6, tap, brow1, 1u);
+                        }
                         s = s2;
                         ph = ph2;
                     }
@@ -140,16 +149,20 @@ conv_qlin_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, 
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        if (rank == 0) {
-            // -------------------------------------------- MMA issue: the whole warp walks the loop, lane 0 issues
-            const uint32_t el = lane == 0 ? 1u : 0u;
-            const uint32_t el1 = (WIDE && Nj1 > 0) ? el : 0u;
+    } else if (warp == 1 || warp == Q_MMA2_WARP) {
+        if (rank == 0 && (warp == 1 || WIDE)) {
+            // -------------------------------------------- MMA issue: the whole warp walks the loop, lane 0 issues.  WIDE: warp 1
+            // issues the first sub-block's MMAs, the second issuing warp the other's (accumulators of their own); a stage or a
+            // patch buffer is free when both have committed.
+            const int sub = warp == 1 ? 0 : 1;
+            const int Ns = sub ? Nj1 : Nj;
+            const uint32_t el = (lane == 0 && Ns > 0) ? 1u : 0u;
+            const uint32_t elc = lane == 0 ? 1u : 0u;
             const uint32_t tfull0 = smem_u32(&sh.tfull[0]), tempty0 = smem_u32(&sh.tempty[0]);
             const int last_nk16 = ((p.Cin - ((cpb - 1) << 6)) + 15) >> 4;
-            const uint32_t idesc = make_idesc_bf16(2 * TILE_M, Nj);
-            const uint32_t idesc1 = make_idesc_bf16(2 * TILE_M, Nj1 > 0 ? Nj1 : 16);
+            const uint32_t idesc = make_idesc_bf16(2 * TILE_M, Ns > 0 ? Ns : 16);
             const uint32_t row_step = (uint32_t)pl.P * 8u;      // one patch row in descriptor units of 16 bytes
+            const uint32_t b_off = (uint32_t)sub * (uint32_t)pl.b_sub_bytes;
             int s = 0, it = 0, ia = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -157,61 +170,56 @@ conv_qlin_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, 
             for (int t = unit; t < total && ok; t += nunits, ++it) {
                 const int acc = WIDE ? 0 : (it & 1), au = WIDE ? it : (it >> 1);
                 if (!__all_sync(0xffffffffu, mbar_wait_u32(tempty0 + 8 * acc, (au & 1) ^ 1, abort_flag))) {
-                    if (el && !*abort_flag) report_timeout(p.status, 73, t);
+                    if (elc && !*abort_flag) report_timeout(p.status, 73, t);
                     *abort_flag = 1;
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d = tmem + (uint32_t)(acc * 256);
+                const uint32_t d = tmem + (uint32_t)((WIDE ? sub : acc) * 256);
                 uint32_t accum = 0;
                 for (int cb = 0; cb < cpb && ok; ++cb, ++ia) {
                     const int ab = ia & 1;
                     if (!__all_sync(0xffffffffu, mbar_wait_u32(afull0 + 8 * ab, (uint32_t)(ia >> 1) & 1u, abort_flag))) {
-                        if (el && !*abort_flag) report_timeout(p.status, 74, t);
+                        if (elc && !*abort_flag) report_timeout(p.status, 74, t);
                         *abort_flag = 1;
                         ok = false;
                         break;
                     }
                     const int nk16 = (cb == cpb - 1) ? last_nk16 : 4;
-                    const uint32_t a_lo0 = sdesc_lo(smem_base + (uint32_t)ab * (uint32_t)pl.a_bytes);
-                    uint32_t a_row = a_lo0;
-                    for (int r = 0; r < p.k && ok; ++r, a_row += row_step) {
-                        uint32_t alo = a_row;
-                        for (int sx = 0; sx < p.k; ++sx, alo += 8u) {
-                            if (!ready && !__all_sync(0xffffffffu, mbar_wait_slow_u32(bfull0 + 8 * s, ph, abort_flag))) {
-                                if (el && !*abort_flag) report_timeout(p.status, 75, t);
-                                *abort_flag = 1;
-                                ok = false;
-                                break;
-                            }
-                            int s2 = s + 1;
-                            uint32_t ph2 = ph;
-                            if (s2 == stages) { s2 = 0; ph2 ^= 1; }
-                            ready = __all_sync(0xffffffffu, mbar_test_u32(bfull0 + 8 * s2, ph2) != 0);   // probe the next slot while this one is issued
-                            tc_fence_after();
-                            const uint32_t blo = sdesc_lo(b_base + (uint32_t)s * b_stage_bytes);
+                    uint32_t a_row = sdesc_lo(smem_base + (uint32_t)ab * (uint32_t)pl.a_bytes);
+                    uint32_t alo = a_row;
+                    int sx = 0;
+                    for (int tap = 0; tap < taps;) {
+                        const int nt = min(pl.tps, taps - tap);
+                        if (!ready && !__all_sync(0xffffffffu, mbar_wait_slow_u32(bfull0 + 8 * s, ph, abort_flag))) {
+                            if (elc && !*abort_flag) report_timeout(p.status, 75, t);
+                            *abort_flag = 1;
+                            ok = false;
+                            break;
+                        }
+                        int s2 = s + 1;
+                        uint32_t ph2 = ph;
+                        if (s2 == stages) { s2 = 0; ph2 ^= 1; }
+                        ready = __all_sync(0xffffffffu, mbar_test_u32(bfull0 + 8 * s2, ph2) != 0);   // probe the next slot while this one is issued
+                        tc_fence_after();
+                        uint32_t blo = sdesc_lo(b_base + (uint32_t)s * b_stage_bytes + b_off);
+                        for (int j = 0; j < nt; ++j, ++tap, blo += b_tap_bytes >> 4) {
                             umma_bf16_lo<true>(d, alo, blo, idesc, accum, (nk16 > 0) & el);
                             accum = 1;
                             umma_bf16_lo<true>(d, alo + 2, blo + 2, idesc, 1u, (nk16 > 1) & el);
                             umma_bf16_lo<true>(d, alo + 4, blo + 4, idesc, 1u, (nk16 > 2) & el);
                             umma_bf16_lo<true>(d, alo + 6, blo + 6, idesc, 1u, (nk16 > 3) & el);
-                            if (WIDE) {
-                                const uint32_t blo1 = sdesc_lo(b_base + (uint32_t)s * b_stage_bytes + (uint32_t)pl.b_sub_bytes);
-                                const uint32_t d1 = d + 256u;
-                                const uint32_t first = (cb == 0 && r == 0 && sx == 0) ? 0u : 1u;
-                                umma_bf16_lo<true>(d1, alo, blo1, idesc1, first, (nk16 > 0) & el1);
-                                umma_bf16_lo<true>(d1, alo + 2, blo1 + 2, idesc1, 1u, (nk16 > 1) & el1);
-                                umma_bf16_lo<true>(d1, alo + 4, blo1 + 4, idesc1, 1u, (nk16 > 2) & el1);
-                                umma_bf16_lo<true>(d1, alo + 6, blo1 + 6, idesc1, 1u, (nk16 > 3) & el1);
-                            }
-                            if (el) umma_commit_u32<true>(bempty0 + 8 * s);
-                            s = s2;
-                            ph = ph2;
+                            // next tap: one pixel on, or the start of the next filter row
+                            alo += 8u;
+                            if (++sx == p.k) { sx = 0; a_row += row_step; alo = a_row; }
                         }
+                        if (elc) umma_commit_u32<true>(bempty0 + 8 * s);
+                        s = s2;
+                        ph = ph2;
                     }
-                    if (ok && el) umma_commit_u32<true>(aempty0 + 8 * ab);   // the patch buffer may be refilled once these MMAs are done
+                    if (ok && elc) umma_commit_u32<true>(aempty0 + 8 * ab);   // the patch buffer may be refilled once these MMAs are done
                 }
-                if (ok && el) umma_commit_u32<true>(tfull0 + 8 * acc);
+                if (ok && elc) umma_commit_u32<true>(tfull0 + 8 * acc);
             }
         }
         __syncwarp();
@@ -293,8 +301,11 @@ static bool qlin_plan(const ConvParams& p, QlinPlan* out) {
     if (pl.wide && cout16 - nt < 32) return false;                 // MMAs of 256 rows take N >= 32
     pl.b_sub_bytes = (((nt >> 1) * 128) + 1023) & ~1023;
     const int budget = Q_SMEM_MAX - 1024 - 2 * pl.a_bytes;
-    const int st = budget / (pl.b_sub_bytes * (pl.wide ? 2 : 1));
-    if (st < 3) return false;
+    const int tap_bytes = pl.b_sub_bytes * (pl.wide ? 2 : 1);
+    if (budget / tap_bytes < 3) return false;
+    pl.tps = p.k;                                                  // a whole filter row per stage if three such stages fit
+    while (pl.tps > 1 && budget / (tap_bytes * pl.tps) < 3) --pl.tps;
+    const int st = budget / (tap_bytes * pl.tps);
     pl.stages = st > Q_MAX_STAGES ? Q_MAX_STAGES : st;
     *out = pl;
     return true;
@@ -359,7 +370,7 @@ int conv_qlin_launch(const ConvParams& p_in, cudaStream_t stream) {
     }
     const int units = (pl.m_tiles + 1) / 2;
     const int pairs = units < max_clusters ? units : max_clusters;
-    int smem_bytes = 2 * pl.a_bytes + pl.stages * pl.b_sub_bytes * (pl.wide ? 2 : 1) + 1024;
+    int smem_bytes = 2 * pl.a_bytes + pl.stages * pl.b_sub_bytes * (pl.wide ? 2 : 1) * pl.tps + 1024;
     if (smem_bytes < 120 * 1024) smem_bytes = 120 * 1024;       // one CTA per SM: each owns all of TMEM
     cfg.gridDim = dim3(2 * pairs);
     cfg.dynamicSmemBytes = (size_t)smem_bytes;
