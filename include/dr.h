@@ -318,6 +318,14 @@ int dr_regress_workspace_bytes(int C, size_t* bytes);
 int dr_regress_grad(int B, int H, int W, int C, const void* y, const void* yt, int relu, void* dz, float* db,
                     float* loss, void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same for a SHARD of a mini-batch (a data-parallel step: the mini-batch of `batch` images is split over ranks, this
+ * call sees B <= batch of them).  Eq. (w_b) sums over samples, so with the mini-batch's constant in every shard,
+ *   dZ = (Y - Y_CNN) / batch,   loss = 1/(2 batch) * sum over the shard,
+ * the shards' db, loss (and the filter gradients taken from their dZ) ADD UP to the whole step's: a sum-all-reduce of
+ * dW, db and loss over the ranks, then dr_sgd_update on every rank.  dr_regress_grad is this call with batch = B.     */
+int dr_regress_grad_shard(int B, int batch, int H, int W, int C, const void* y, const void* yt, int relu, void* dz,
+                          float* db, float* loss, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Filter gradient of the convolution of `desc` (k, stride, pad, Cin, Cout; flags and y_ldc are not looked at):
  *   dw[j][r][s][c] = sum over (n, ho, wo) of dz[n][ho][wo][j] * x[n][ho*stride - pad + r][wo*stride - pad + s][c]
  * with x zero outside the image.  x: [B,H,W,Cin] dense bfloat16; dz: [B,Ho,Wo,Cout] dense bfloat16;
@@ -343,12 +351,21 @@ int dr_sgd_update(size_t n, float* w, float* v, const float* g, float lr, float 
  * The bias takes no weight decay.  workspace: dr_regress_step_workspace_bytes bytes, 256-byte aligned, zero-filled
  * before the first call (the forward pass of a layer with few output tiles keeps its tile counters there and
  * leaves them at zero; the gradient scratch in front of them is overwritten every call).
- * Errors: INVALID_ARG, UNSUPPORTED (flags, channel slice, Cin < 64 or channels not multiples of 8), ALIGNMENT,
- * WORKSPACE, and whatever the forward pass returns.                                                           */
+ * Layers with Cin < 64 or channel counts that are not multiples of 8 are taken too (on the plain kernels of
+ * dr_conv_wgrad / dr_regress_grad).  Errors: INVALID_ARG, UNSUPPORTED (flags other than bias / ReLU, a channel slice),
+ * ALIGNMENT, WORKSPACE, and whatever the forward pass returns.                                                */
 int dr_regress_step_workspace_bytes(const dr_conv_desc* desc, int B, int H, int W, size_t* bytes);
 int dr_regress_step(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* yt, float* w, float* b,
                     float* vw, float* vb, void* w_bf16, float lr, float momentum, float decay, void* y, void* dz,
                     float* dw, float* db, float* loss, void* workspace, size_t workspace_bytes, void* stream);
+
+/* One rank's part of a data-parallel step: forward on its shard (B of the mini-batch's `batch` images), dr_regress_grad_shard,
+ * dr_conv_wgrad; no update.  dw, db, *loss are the shard's contributions (see dr_regress_grad_shard): sum them over the
+ * ranks (e.g. one all-reduce of Cout*k*k*Cin + Cout + 1 floats), then call dr_sgd_update for the filters and the bias as
+ * dr_regress_step does.  Arguments, workspace (dr_regress_step_workspace_bytes) and errors as dr_regress_step.        */
+int dr_regress_shard_grads(const dr_conv_desc* desc, int B, int batch, int H, int W, const void* x, const void* yt,
+                           const void* w_bf16, const float* b, void* y, void* dz, float* dw, float* db, float* loss,
+                           void* workspace, size_t workspace_bytes, void* stream);
 
 /* Kernels of this library launched by this process so far. */
 long long dr_launch_count(void);

@@ -28,17 +28,29 @@ def slim_forward(x, w, b, stride=1, pad=0, relu=True):
     return np.maximum(z, 0.0) if relu else z
 
 
-def regression_loss(y, yt):
-    """1/(2B) * sum_i ||Y_CNN^i - Y^i||_F^2 (Eq. (w_b) with the constant of the reading above)."""
+def regression_loss(y, yt, batch=None):
+    """1/(2B) * sum_i ||Y_CNN^i - Y^i||_F^2 (Eq. (w_b) with the constant of the reading above).
+
+    `batch`: the B of the constant when y holds only some of the mini-batch's samples (a shard of a data-parallel
+    step): the objective is a sum over samples, so the shards' values add up to the mini-batch's."""
     d = np.asarray(y, np.float64) - np.asarray(yt, np.float64)
-    return float(np.sum(d * d) / (2.0 * y.shape[0]))
+    return float(np.sum(d * d) / (2.0 * (batch or y.shape[0])))
 
 
-def grad_preactivation(y, yt, relu=True):
-    """dL/dZ for Y = ReLU(Z): (Y - Y_CNN) / B where the unit is active (Y > 0), zero elsewhere."""
+def grad_preactivation(y, yt, relu=True, batch=None):
+    """dL/dZ for Y = ReLU(Z): (Y - Y_CNN) / B where the unit is active (Y > 0), zero elsewhere (`batch` as above)."""
     y = np.asarray(y, np.float64)
-    g = (y - np.asarray(yt, np.float64)) / y.shape[0]
+    g = (y - np.asarray(yt, np.float64)) / (batch or y.shape[0])
     return np.where(y > 0.0, g, 0.0) if relu else g
+
+
+def shard_gradients(x, yt, w, b, batch, stride=1, pad=0, relu=True):
+    """What one rank of a data-parallel step contributes from its shard (x, yt) of a mini-batch of `batch` samples:
+    (dW, db, loss), each a sum over the shard's samples with the mini-batch's constant.  Eq. (w_b) sums over samples, so
+    adding these over a partition of the mini-batch gives the gradient and loss of the whole of it."""
+    y = slim_forward(x, w, b, stride, pad, relu)
+    dz = grad_preactivation(y, yt, relu, batch)
+    return conv2d_wgrad(x, dz, w.shape[1], stride, pad), bias_grad(dz), regression_loss(y, yt, batch)
 
 
 def conv2d_wgrad(x, dz, k, stride=1, pad=0):

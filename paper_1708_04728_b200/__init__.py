@@ -75,6 +75,8 @@ _SIGS = {
     "dr_conv_slim": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _P, _P, _P]),
     "dr_regress_workspace_bytes": (_I, [_I, C.POINTER(_Z)]),
     "dr_regress_grad": (_I, [_I, _I, _I, _I, _P, _P, _I, _P, _P, _P, _P, _Z, _P]),
+    "dr_regress_grad_shard": (_I, [_I, _I, _I, _I, _I, _P, _P, _I, _P, _P, _P, _P, _Z, _P]),
+    "dr_regress_shard_grads": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z, _P]),
     "dr_conv_wgrad_workspace_bytes": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, C.POINTER(_Z)]),
     "dr_conv_wgrad": (_I, [C.POINTER(dr_conv_desc), _I, _I, _I, _P, _P, _P, _P, _Z, _P]),
     "dr_sgd_update": (_I, [_Z, _P, _P, _P, _F, _F, _F, _P, _P]),
@@ -214,6 +216,16 @@ def dr_regress_step(desc, B, H, W, x, yt, w, b, vw, vb, w_bf16, lr, momentum, de
     _check(_lib.dr_regress_step(C.byref(desc), B, H, W, _ptr(x), _ptr(yt), _ptr(w), _ptr(b), _ptr(vw), _ptr(vb), _ptr(w_bf16),
                                 lr, momentum, decay, _ptr(y), _ptr(dz), _ptr(dw), _ptr(db), _ptr(loss), _ptr(workspace),
                                 workspace_bytes, _stream(stream)), "dr_regress_step")
+
+
+def dr_regress_grad_shard(B, batch, H, W, Cc, y, yt, relu, dz, db, loss, workspace, workspace_bytes, stream=None):
+    _check(_lib.dr_regress_grad_shard(B, batch, H, W, Cc, _ptr(y), _ptr(yt), int(relu), _ptr(dz), _ptr(db), _ptr(loss), _ptr(workspace),
+                                      workspace_bytes, _stream(stream)), "dr_regress_grad_shard")
+
+
+def dr_regress_shard_grads(desc, B, batch, H, W, x, yt, w_bf16, b, y, dz, dw, db, loss, workspace, workspace_bytes, stream=None):
+    _check(_lib.dr_regress_shard_grads(C.byref(desc), B, batch, H, W, _ptr(x), _ptr(yt), _ptr(w_bf16), _ptr(b), _ptr(y), _ptr(dz), _ptr(dw),
+                                       _ptr(db), _ptr(loss), _ptr(workspace), workspace_bytes, _stream(stream)), "dr_regress_shard_grads")
 
 
 def dr_conv_workspace_bytes(desc, B, H, W) -> int:

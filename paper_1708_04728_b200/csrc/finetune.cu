@@ -566,7 +566,12 @@ extern "C" int dr_regress_workspace_bytes(int C, size_t* bytes) {
 
 extern "C" int dr_regress_grad(int B, int H, int W, int C, const void* y, const void* yt, int relu, void* dz, float* db, float* loss,
                                void* workspace, size_t workspace_bytes, void* stream) {
-    if (B <= 0 || H <= 0 || W <= 0 || C <= 0 || !y || !yt || !dz || !db || !workspace) return DR_ERR_INVALID_ARG;
+    return dr_regress_grad_shard(B, B, H, W, C, y, yt, relu, dz, db, loss, workspace, workspace_bytes, stream);
+}
+
+extern "C" int dr_regress_grad_shard(int B, int batch, int H, int W, int C, const void* y, const void* yt, int relu, void* dz, float* db,
+                                     float* loss, void* workspace, size_t workspace_bytes, void* stream) {
+    if (B <= 0 || batch < B || H <= 0 || W <= 0 || C <= 0 || !y || !yt || !dz || !db || !workspace) return DR_ERR_INVALID_ARG;
     if (!aligned16(y) || !aligned16(yt) || !aligned16(dz) || ((uintptr_t)workspace & 255)) return DR_ERR_ALIGNMENT;
     size_t need = 0;
     dr_regress_workspace_bytes(C, &need);
@@ -577,23 +582,23 @@ extern "C" int dr_regress_grad(int B, int H, int W, int C, const void* y, const 
         const size_t n = (size_t)M * C;
         size_t blocks = (n + 255) / 256;
         if (blocks > (size_t)num_sms() * 8) blocks = (size_t)num_sms() * 8;
-        regress_grad_scalar_kernel<<<(unsigned)blocks, 256, 0, s>>>(n, 1.f / (float)B, relu ? 1 : 0, reinterpret_cast<const __nv_bfloat16*>(y),
+        regress_grad_scalar_kernel<<<(unsigned)blocks, 256, 0, s>>>(n, 1.f / (float)batch, relu ? 1 : 0, reinterpret_cast<const __nv_bfloat16*>(y),
                                                                    reinterpret_cast<const __nv_bfloat16*>(yt), reinterpret_cast<__nv_bfloat16*>(dz));
         count_launch();
         int st0 = launch_status();
         if (st0 != DR_OK) return st0;
-        regress_sums_scalar_kernel<<<C + 1, 256, 0, s>>>(M, C, 0.5f / (float)B, reinterpret_cast<const __nv_bfloat16*>(y),
+        regress_sums_scalar_kernel<<<C + 1, 256, 0, s>>>(M, C, 0.5f / (float)batch, reinterpret_cast<const __nv_bfloat16*>(y),
                                                         reinterpret_cast<const __nv_bfloat16*>(yt), reinterpret_cast<const __nv_bfloat16*>(dz), db, loss);
         count_launch();
         return launch_status();
     }
     float* partials = reinterpret_cast<float*>(workspace);
-    regress_grad_kernel<<<RG_BLOCKS, RG_THREADS, 0, s>>>(reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(yt), M, C, 1.f / (float)B,
+    regress_grad_kernel<<<RG_BLOCKS, RG_THREADS, 0, s>>>(reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(yt), M, C, 1.f / (float)batch,
                                                        relu ? 1 : 0, reinterpret_cast<uint4*>(dz), partials);
     count_launch();
     int st = launch_status();
     if (st != DR_OK) return st;
-    regress_finalize_kernel<<<(C + 1 + 31) / 32, 512, 0, s>>>(partials, RG_BLOCKS, C, 0.5f / (float)B, db, loss);
+    regress_finalize_kernel<<<(C + 1 + 31) / 32, 512, 0, s>>>(partials, RG_BLOCKS, C, 0.5f / (float)batch, db, loss);
     count_launch();
     return launch_status();
 }
@@ -619,6 +624,29 @@ extern "C" int dr_regress_step_workspace_bytes(const dr_conv_desc* desc, int B, 
     if (st != DR_OK) return st;
     *bytes = round256(a) + round256(b) + round256(c);
     return DR_OK;
+}
+
+extern "C" int dr_regress_shard_grads(const dr_conv_desc* desc, int B, int batch, int H, int W, const void* x, const void* yt, const void* w_bf16,
+                                      const float* b, void* y, void* dz, float* dw, float* db, float* loss, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+    if (!desc || !x || !yt || !b || !w_bf16 || !y || !dz || !dw || !db || !workspace || batch < B) return DR_ERR_INVALID_ARG;
+    if (!(desc->flags & DR_BIAS) || (desc->flags & ~(unsigned)(DR_BIAS | DR_RELU))) return DR_ERR_UNSUPPORTED;
+    if ((desc->y_ldc && desc->y_ldc != desc->Cout) || desc->y_coff) return DR_ERR_UNSUPPORTED;
+    if ((uintptr_t)workspace & 255) return DR_ERR_ALIGNMENT;
+    size_t wa = 0, wb = 0, wc = 0, need = 0;
+    int st = dr_regress_step_workspace_bytes(desc, B, H, W, &need);
+    if (st != DR_OK) return st;
+    if (workspace_bytes < need) return DR_ERR_WORKSPACE;
+    dr_conv_wgrad_workspace_bytes(desc, B, H, W, &wa);
+    dr_regress_workspace_bytes(desc->Cout, &wb);
+    dr_conv_workspace_bytes(desc, B, H, W, &wc);
+    char* ws = reinterpret_cast<char*>(workspace);
+    const int Ho = (H + 2 * desc->pad - desc->k) / desc->stride + 1, Wo = (W + 2 * desc->pad - desc->k) / desc->stride + 1;
+    st = dr_conv_slim_ws(desc, B, H, W, x, w_bf16, b, nullptr, y, nullptr, wc ? ws + round256(wa) + round256(wb) : nullptr, wc, stream);
+    if (st != DR_OK) return st;
+    st = dr_regress_grad_shard(B, batch, Ho, Wo, desc->Cout, y, yt, (desc->flags & DR_RELU) ? 1 : 0, dz, db, loss, ws + round256(wa), wb, stream);
+    if (st != DR_OK) return st;
+    return dr_conv_wgrad(desc, B, H, W, x, dz, dw, ws, wa, stream);
 }
 
 extern "C" int dr_regress_step(const dr_conv_desc* desc, int B, int H, int W, const void* x, const void* yt, float* w, float* b, float* vw,

@@ -287,3 +287,66 @@ def test_regression_steps_on_a_folded_layer(dr, F):
     for i, (a, r) in enumerate(zip(gpu_losses, ref_losses)):
         assert abs(a - r) <= 2e-2 * r, f"step {i}: loss {a} vs {r}"
     assert gpu_losses[-1] < 0.7 * gpu_losses[0], gpu_losses
+
+
+def _step_buffers(dr, B, Ho, Wo, Cin, Cout, k):
+    import torch
+    y = torch.zeros((B, Ho, Wo, Cout), dtype=torch.bfloat16, device="cuda")
+    return (y, torch.zeros_like(y), torch.zeros((Cout, k, k, Cin), dtype=torch.float32, device="cuda"),
+            torch.zeros(Cout, dtype=torch.float32, device="cuda"), torch.zeros(1, dtype=torch.float32, device="cuda"))
+
+
+def test_shard_gradients_add_up_to_the_whole_step(dr, F):
+    """A data-parallel step on one GPU: the mini-batch of 6 in uneven shards (4 + 2), each through dr_regress_shard_grads
+    with the mini-batch's constant; the shards' dW, db and loss, added, are the checker's for the whole mini-batch."""
+    B, H, W, Cin, Cout, k, s, p = 6, 14, 14, 64, 64, 3, 1, 1
+    x = S.round_bf16(S.normal(5, "dp.x", (B, H, W, Cin)))
+    yt = S.round_bf16(np.abs(S.normal(5, "dp.yt", (B, H, W, Cout))))
+    w0 = S.round_bf16(S.he_normal(5, "dp.w", Cout, k, Cin)); b0 = S.normal(5, "dp.b", (Cout,), 0.05).astype(np.float32).astype(np.float64)
+    d = desc_of(dr, k, s, p, Cin, Cout, dr.DR_BIAS | dr.DR_RELU)
+    wbf, bd = to_dev_bf16(w0), to_dev_f32(b0)
+    tot_dw, tot_db, tot_loss, ys = 0.0, 0.0, 0.0, []
+    for a, e in ((0, 4), (4, 6)):
+        n = e - a
+        ws = workspace(dr.dr_regress_step_workspace_bytes(d, n, H, W), poison=False); ws.zero_()
+        y, dz, dw, db, loss = _step_buffers(dr, n, H, W, Cin, Cout, k)
+        dr.dr_regress_shard_grads(d, n, B, H, W, to_dev_bf16(x[a:e]), to_dev_bf16(yt[a:e]), wbf, bd, y, dz, dw, db, loss, ws, ws.numel())
+        status_ok(dr)
+        tot_dw = tot_dw + to_host(dw); tot_db = tot_db + to_host(db); tot_loss += float(loss)
+        ys.append(to_host(y))
+    y_gpu = np.concatenate(ys)
+    dz_ref = F.grad_preactivation(y_gpu, yt)                      # teacher-forced on the stored forward output
+    mx, l2 = err_norms(tot_dw, F.conv2d_wgrad(x, dz_ref, k, s, p))
+    assert mx <= LAYER_MAX and l2 <= LAYER_L2, (mx, l2)
+    mx, l2 = err_norms(tot_db, F.bias_grad(dz_ref))
+    assert mx <= LAYER_MAX and l2 <= LAYER_L2, (mx, l2)
+    assert abs(tot_loss - F.regression_loss(y_gpu, yt)) <= 1e-4 * tot_loss
+    # free-running against the checker's own shard sums
+    parts = [F.shard_gradients(x[a:e], yt[a:e], w0, b0, B, s, p) for a, e in ((0, 4), (4, 6))]
+    assert err_norms(tot_dw, parts[0][0] + parts[1][0])[1] <= 2e-2
+    with pytest.raises(dr.DrError) as e:                           # a shard cannot be larger than its mini-batch
+        dr.dr_regress_shard_grads(d, 4, 2, H, W, wbf, wbf, wbf, bd, y, dz, dw, db, loss, ws, ws.numel())
+    assert e.value.status == dr.DR_ERR_INVALID_ARG
+
+
+def test_regression_step_on_channel_counts_the_tensor_kernels_do_not_take(dr, F):
+    """A whole step on a layer with 24 input and 36 output channels (plain kernels throughout)."""
+    import torch
+    B, H, W, Cin, Cout, k, s, p = 3, 9, 11, 24, 36, 3, 1, 1
+    x = S.round_bf16(S.normal(6, "odd.x", (B, H, W, Cin)))
+    yt = S.round_bf16(np.abs(S.normal(6, "odd.yt", (B, H, W, Cout))))
+    w0 = S.round_bf16(S.he_normal(6, "odd.w", Cout, k, Cin)); b0 = np.zeros(Cout)
+    d = desc_of(dr, k, s, p, Cin, Cout, dr.DR_BIAS | dr.DR_RELU)
+    ws = workspace(dr.dr_regress_step_workspace_bytes(d, B, H, W) + 256, poison=False); ws.zero_()
+    wd, bd = to_dev_f32(w0), to_dev_f32(b0)
+    vw, vb, shadow = torch.zeros_like(wd), torch.zeros_like(bd), to_dev_bf16(w0)
+    y, dz, dw, db, loss = _step_buffers(dr, B, H, W, Cin, Cout, k)
+    dr.dr_regress_step(d, B, H, W, to_dev_bf16(x), to_dev_bf16(yt), wd, bd, vw, vb, shadow, 1e-3, 0.9, 0.0, y, dz, dw, db, loss, ws, ws.numel())
+    status_ok(dr)
+    y_gpu = to_host(y)
+    assert err_norms(y_gpu, F.slim_forward(x, w0, b0, s, p))[1] <= LAYER_L2
+    dz_ref = F.grad_preactivation(y_gpu, yt)
+    mx, l2 = err_norms(to_host(dw), F.conv2d_wgrad(x, dz_ref, k, s, p))
+    assert mx <= LAYER_MAX and l2 <= LAYER_L2, (mx, l2)
+    w1_ref, _ = F.sgd_update(w0, np.zeros_like(w0), to_host(dw), 1e-3, 0.9, 0.0)
+    assert err_norms(to_host(wd), w1_ref)[0] <= 1e-6

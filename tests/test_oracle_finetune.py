@@ -147,3 +147,21 @@ def test_steps_recover_a_realisable_teacher():
         losses.append(loss)
     assert losses[-1] < 1e-10 * losses[0] and all(b_ <= a_ for a_, b_ in zip(losses[5:], losses[6:]) if a_ > 1e-20 * losses[0])
     np.testing.assert_allclose(w, wt, atol=1e-5); np.testing.assert_allclose(b, bt, atol=1e-5)
+
+
+def test_shard_gradients_add_up_to_the_mini_batch_gradient():
+    """Eq. (w_b) is a sum over samples: gradients and loss of any partition of the mini-batch, each taken with the
+    mini-batch's 1/B, add up to the whole step's (uneven shards, stride 2, ReLU)."""
+    rng = np.random.default_rng(11)
+    B, H, Cin, Cout, k, s, p = 5, 7, 3, 4, 3, 2, 1
+    x = rng.normal(size=(B, H, H, Cin)); w = rng.normal(size=(Cout, k, k, Cin)) * 0.3; b = rng.normal(size=Cout) * 0.1
+    Ho = (H + 2 * p - k) // s + 1
+    yt = np.abs(rng.normal(size=(B, Ho, Ho, Cout)))
+    _, _, _, _, loss, dw, db = F.regression_step(x, yt, w, b, np.zeros_like(w), np.zeros_like(b), 0.1, 0.0, 0.0, s, p)
+    parts = [F.shard_gradients(x[a:e], yt[a:e], w, b, B, s, p) for a, e in ((0, 2), (2, 3), (3, 5))]
+    assert np.allclose(sum(q[0] for q in parts), dw, rtol=0, atol=1e-12)
+    assert np.allclose(sum(q[1] for q in parts), db, rtol=0, atol=1e-12)
+    assert abs(sum(q[2] for q in parts) - loss) < 1e-12
+    # a shard taken as a mini-batch of its own differs by the ratio of the batch sizes
+    own = F.regression_step(x[:2], yt[:2], w, b, np.zeros_like(w), np.zeros_like(b), 0.1, 0.0, 0.0, s, p)
+    assert np.allclose(parts[0][0] * (B / 2), own[5], atol=1e-12)
