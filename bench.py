@@ -291,7 +291,19 @@ def run_nontensor(args):
             if i >= args.warmup:
                 ts.append(a.elapsed_time(e) * 1e3)
         us = statistics.median(ts)
-        rows.append({"kernel": name, "us": us, "mbytes": nbytes / 1e6, "gbs": nbytes / us * 1e-3, "frac": nbytes / us * 1e-3 / pk["hbm_gbs"]})
+        # context: a plain device copy that moves the same number of bytes (half read, half written), timed the same way:
+        # what the copy the peak was measured with reaches at THIS size (small tensors do not reach the large-copy rate)
+        src = torch.empty(max(int(nbytes) // 2, 16), dtype=torch.uint8, device="cuda"); dst = torch.empty_like(src)
+        tc = []
+        for i in range(args.warmup + 5):
+            flush.zero_()
+            a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); dst.copy_(src); e.record(); torch.cuda.synchronize()
+            if i >= args.warmup:
+                tc.append(a.elapsed_time(e) * 1e3)
+        copy_us = statistics.median(tc)
+        rows.append({"kernel": name, "us": us, "mbytes": nbytes / 1e6, "gbs": nbytes / us * 1e-3, "frac": nbytes / us * 1e-3 / pk["hbm_gbs"],
+                     "copy_same_bytes_us": copy_us, "frac_of_copy_same_bytes": copy_us / us})
     print(json.dumps({"batch": B, "peak_gbs": pk["hbm_gbs"], "peak_kind": pk_kind, "kernels": rows}))
 
 

@@ -283,7 +283,7 @@ int dr_net_activation_bytes(const dr_net* net, size_t* bytes);
 #define DR_PATH_UMMA_TMA     3  /* tcgen05 MMA, operands loaded by TMA (im2col / tiled)          */
 #define DR_PATH_UMMA_PATCH   4  /* pooling layers: 2-D output patches, TMA box loads, fused pool/LRN */
 #define DR_PATH_UMMA_STEM    5  /* the 7x7/2 3-channel stem with fused pool/LRN                  */
-#define DR_PATH_UMMA_STEM_T  6  /* the same stem computed transposed: pooling in registers       */
+#define DR_PATH_RETIRED_6    6  /* number of a removed kernel; forcing it gives DR_ERR_UNSUPPORTED  */
 #define DR_PATH_UMMA_STEM_D  7  /* the stem with the MMA reading the input rows in place (no im2col) */
 #define DR_PATH_UMMA_SPLITK  8  /* few output tiles: K split across the SMs, partial tiles summed in scratch (needs a workspace) */
 #define DR_PATH_UMMA_QLIN    9  /* stride-1 3x3 / 5x5: the tile's input patch loaded once, every tap read out of it by the MMA */

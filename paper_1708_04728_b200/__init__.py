@@ -28,11 +28,11 @@ DR_BIAS, DR_RELU, DR_POOL, DR_LRN, DR_RESIDUAL = 0x01, 0x02, 0x04, 0x08, 0x10
 DR_LRN_BEFORE_POOL, DR_RELU_AFTER_RESIDUAL, DR_OUT_F32 = 0x20, 0x40, 0x80
 DR_ARCH_GOOGLENET, DR_ARCH_RESNET50, DR_ARCH_GOOGLENET_PAPER, DR_ARCH_GOOGLENET_STREAMLINE, DR_ARCH_ALEXNET = 0, 1, 2, 3, 4
 DR_MODE_SLIM, DR_MODE_UNSLIMMED = 0, 1
-DR_PATH_AUTO, DR_PATH_SIMT, DR_PATH_UMMA_GATHER, DR_PATH_UMMA_TMA, DR_PATH_UMMA_PATCH, DR_PATH_UMMA_STEM, DR_PATH_UMMA_STEM_T, DR_PATH_UMMA_STEM_D = 0, 1, 2, 3, 4, 5, 6, 7
+DR_PATH_AUTO, DR_PATH_SIMT, DR_PATH_UMMA_GATHER, DR_PATH_UMMA_TMA, DR_PATH_UMMA_PATCH, DR_PATH_UMMA_STEM, DR_PATH_RETIRED_6, DR_PATH_UMMA_STEM_D = 0, 1, 2, 3, 4, 5, 6, 7
 DR_PATH_UMMA_SPLITK = 8
 DR_PATH_UMMA_QLIN = 9
 DR_CONV_WS_COUNTER_BYTES = 1024
-PATH_NAMES = {0: "auto", 1: "simt", 2: "umma_gather", 3: "umma_tma", 4: "umma_patch", 5: "umma_stem", 6: "umma_stem_t", 7: "umma_stem_d",
+PATH_NAMES = {0: "auto", 1: "simt", 2: "umma_gather", 3: "umma_tma", 4: "umma_patch", 5: "umma_stem", 6: "retired", 7: "umma_stem_d",
               8: "umma_splitk", 9: "umma_qlin", -1: "-"}
 
 

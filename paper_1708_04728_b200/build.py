@@ -17,7 +17,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdeeprebirth.so")
-SOURCES = ["nontensor.cu", "tensor_map.cu", "conv_api.cu", "conv_simt.cu", "conv_umma.cu", "conv_qlin.cu", "conv_splitk.cu", "conv_patch.cu", "conv_stem_t.cu", "conv_stem_d.cu", "net.cu", "finetune.cu"]
+SOURCES = ["nontensor.cu", "tensor_map.cu", "conv_api.cu", "conv_simt.cu", "conv_umma.cu", "conv_qlin.cu", "conv_splitk.cu", "conv_patch.cu", "conv_stem_d.cu", "net.cu", "finetune.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", INCLUDE]
 

@@ -128,13 +128,12 @@ int conv_pick_path(const ConvParams& p, int forced) {
     if (forced == DR_PATH_UMMA_TMA) return conv_umma_tma_supports(p) ? DR_PATH_UMMA_TMA : -1;
     if (forced == DR_PATH_UMMA_PATCH) return conv_patch_tma_supports(p) ? DR_PATH_UMMA_PATCH : -1;
     if (forced == DR_PATH_UMMA_STEM) return conv_stem_supports(p) ? DR_PATH_UMMA_STEM : -1;
-    if (forced == DR_PATH_UMMA_STEM_T) return conv_stem_t_supports(p) ? DR_PATH_UMMA_STEM_T : -1;
+    if (forced == DR_PATH_RETIRED_6) return -1;                 // a retired kernel's number: nothing runs under it
     if (forced == DR_PATH_UMMA_STEM_D) return conv_stem_d_supports(p) ? DR_PATH_UMMA_STEM_D : -1;
     if (forced == DR_PATH_UMMA_SPLITK) return conv_splitk_supports(p) ? DR_PATH_UMMA_SPLITK : -1;
     if (forced == DR_PATH_UMMA_QLIN) return conv_qlin_supports(p) ? DR_PATH_UMMA_QLIN : -1;
     if (conv_stem_d_supports(p)) return DR_PATH_UMMA_STEM_D;
-    if (conv_stem_supports(p)) return DR_PATH_UMMA_STEM;       // measured faster than the transposed form (483 vs 625 us at batch 256)
-    if (conv_stem_t_supports(p)) return DR_PATH_UMMA_STEM_T;
+    if (conv_stem_supports(p)) return DR_PATH_UMMA_STEM;
     if (conv_patch_tma_supports(p)) return DR_PATH_UMMA_PATCH;
     if (conv_splitk_supports(p)) return DR_PATH_UMMA_SPLITK;   // few output tiles and scratch at hand
     if (qlin_preferred(p)) return DR_PATH_UMMA_QLIN;
@@ -150,7 +149,6 @@ int conv_launch_path(const ConvParams& p, int path, cudaStream_t stream) {
         case DR_PATH_UMMA_TMA: return conv_umma_tma_launch(p, stream);
         case DR_PATH_UMMA_PATCH: return conv_patch_tma_launch(p, stream);
         case DR_PATH_UMMA_STEM: return conv_stem_launch(p, stream);
-        case DR_PATH_UMMA_STEM_T: return conv_stem_t_launch(p, stream);
         case DR_PATH_UMMA_STEM_D: return conv_stem_d_launch(p, stream);
         case DR_PATH_UMMA_SPLITK: return conv_splitk_launch(p, stream);
         case DR_PATH_UMMA_QLIN: return conv_qlin_launch(p, stream);

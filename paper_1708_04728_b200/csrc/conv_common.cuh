@@ -285,8 +285,6 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream);
 bool conv_patch_tma_supports(const ConvParams& p);
 int conv_stem_launch(const ConvParams& p, cudaStream_t stream);
 bool conv_stem_supports(const ConvParams& p);
-int conv_stem_t_launch(const ConvParams& p, cudaStream_t stream);
-bool conv_stem_t_supports(const ConvParams& p);
 int conv_stem_d_launch(const ConvParams& p, cudaStream_t stream);
 bool conv_stem_d_supports(const ConvParams& p);
 bool conv_umma_gather_supports(const ConvParams& p);
