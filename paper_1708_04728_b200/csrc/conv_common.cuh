@@ -55,6 +55,9 @@ struct ConvParams {
     int overlap_prev;      // TMA kernel: 1 = the layer does not read what the kernel before it in the stream writes; it is
                            // launched with programmatic serialization (its CTAs fill SMs that kernel has left) and waits
                            // for that kernel only before it exits, so that whatever follows sees both complete
+    int pdl_wait;          // TMA kernel: 1 = launched with programmatic serialization behind the kernel whose output it reads: its
+                           // CTAs may start (barriers, tensor memory, descriptors) while that kernel's last CTAs still run, and
+                           // wait for its completion before the first load of activations
     int* sk_counters;      // split-K kernel only (nullptr: not available): DR_CONV_WS_COUNTER_BYTES of zeroed tile counters
     float* sk_scratch;     // and scratch for the partial tiles
     size_t sk_scratch_bytes;

@@ -563,6 +563,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
             const int g = warp == 0 ? 0 : 1;
             const uint32_t full0 = smem_u32(&sh.full[g * stages]), empty0 = smem_u32(&sh.empty[g * stages]);
             const uint32_t ring_base = smem_base + (uint32_t)(g * stages) * (uint32_t)stage_bytes;
+            if (p.pdl_wait) grid_dependency_wait();            // the kernel before this one has written the activations
             const uint32_t cta_tx = A_TILE_BYTES + (uint32_t)(PAIR ? p.Nt >> 1 : p.Nt) * 128 * (WIDE ? 2 : 1);
             const uint32_t full_mask = PAIR ? PEER_BIT_MASK : 0xFFFFFFFFu;   // pair: bytes are reported to the even CTA
             int s = 0;
@@ -699,6 +700,7 @@ conv_umma_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map
         const int g = (warp - 2) >> 2;
         const int q = warp & 3;
         const int row = q * 32 + lane;
+        if (p.pdl_wait && (p.flags & DR_RESIDUAL)) grid_dependency_wait();   // the residual may be that kernel's output too
         int ep_it = 0;                                           // chunks this group has handed to the TMA unit so far
         // tiles of this group: WIDE every tile (sub-block g); else every other tile of the CTA (DUAL: those are pipeline g's)
         for (int t = WIDE ? unit : unit + g * nunits, au = 0; t < total; t += WIDE ? nunits : 2 * nunits, ++au) {
@@ -960,7 +962,7 @@ int launch_variant(const TmaLaunch& L) {
     const int n = L.units < capacity[dev] ? L.units : capacity[dev];
     cfg.gridDim = dim3((unsigned)(PAIR ? 2 * n : n));
     cfg.dynamicSmemBytes = (size_t)L.smem_bytes;
-    if (L.p->overlap_prev) {
+    if (L.p->overlap_prev || L.p->pdl_wait) {
         attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[na].val.programmaticStreamSerializationAllowed = 1;
         ++na;

@@ -724,6 +724,10 @@ int dr_net_forward(dr_net* n, const void* x, void* workspace, float* logits, voi
                         const Tensor& tc = n->T(oc.in0);
                         st = conv_make_params(&oc.cd, tc.B, tc.H, tc.W, out, oc.w.resolve(n->raw, ws), (const float*)oc.b.resolve(n->raw, ws),
                                               nullptr, (char*)tensor_ptr(n, oc.out, x, arena, logits), nullptr, &pc);
+                        // the reducer may start while the kernel before it drains (it waits before its first load); the merged 5x5
+                        // behind it stays an ordinary launch, so that the 3x3, which starts early and reads the reducer's output
+                        // without waiting, cannot start before the reducer has completed
+                        p.pdl_wait = (i > 0 && tunable("DR_NET_PDL", 1) != 0) ? 1 : 0;
                         if (st == DR_OK) st = conv_launch_path(p, op.path, s);
                         if (st == DR_OK) st = conv_launch_path(pa, oa.path, s);
                         if (st == DR_OK) {
@@ -744,6 +748,8 @@ int dr_net_forward(dr_net* n, const void* x, void* workspace, float* logits, voi
                 }
                 if (st == DR_OK) {
                     set_splitk_scratch(n, op, (char*)workspace, &p);
+                    // a layer of its own on the TMA kernel: its CTAs may set up while the kernel before it drains
+                    if (op.path == DR_PATH_UMMA_TMA && i > 0 && !n->timing && tunable("DR_NET_PDL", 1) != 0) p.pdl_wait = 1;
                     st = conv_launch_path(p, op.path, s);
                 }
                 break;
