@@ -645,7 +645,7 @@ def main():
         t_roof_total += t_roof
         rows.append(dict(name=li["name"], kind=li["kind"], path=dr.PATH_NAMES[li["conv_path"]], us=float(t_us),
                          gflop=li["flops"] / 1e9, mbytes=li["bytes"] / 1e6, roof_us=t_roof, frac=t_roof / max(float(t_us), 1e-9)))
-    tensor_paths = ("umma_tma",)
+    tensor_paths = ("umma_tma",)          # the dominant kernel; layers on other kernels are in the per-layer table
     tma = [r for r in rows if r["path"] in tensor_paths and r["gflop"] * 1e9 / (pk["bf16_tflops"] * 1e12) >= r["mbytes"] * 1e6 / bw_peak]
     tma_flops = sum(r["gflop"] for r in tma) * 1e9
     tma_s = sum(r["us"] for r in tma) * 1e-6

@@ -113,13 +113,19 @@ int conv_make_params(const dr_conv_desc* d, int B, int H, int W, const void* x, 
     return DR_OK;
 }
 
-// The patch-reuse kernel against the im2col kernel: its tiles are whole padded image rows, so part of every tile's MMA
-// rows is padding (28 x 28 planes: 12.5 %, 14 x 14: 23 %).  Measured at batch 256 (GoogLeNet) it is level with the im2col
-// kernel where that one is bound by filling shared memory and behind it elsewhere (us, patch-reuse / im2col: 3a merged
-// 5x5 221 / 215, 3b 541 / 475, 4a 320 / 246; 3x3 of 3a 76 / 72, 3b 82 / 90, 4d 66 / 68, 4e 72 / 68): the saved loads
-// are paid back in padding rows.  Chosen only on request (DR_QLIN=1, or the forced path).
+// The patch-reuse kernel against the im2col kernel.  Its tiles are whole padded image rows, so part of every tile's MMA
+// rows is padding (28 x 28 planes: 12.5 %, 14 x 14: 23 %); in exchange the activations are loaded once per channel block
+// instead of once per tap, and with at most 128 output channels two tiles per CTA run side by side on double-buffered
+// accumulators.  Measured at batch 256 (us, patch-reuse / im2col): a gain for tiles of at most 128 channels on planes of
+// 28 x 28 and more (3a merged 5x5 181 / 216, 3a 3x3 55 / 73; ResNet-50 stage 2 and 3 3x3 54 / 61 and 38 / 42), a loss
+// where a tile's accumulator takes all its TMEM half or the layer runs on wide tiles (3b 3x3 117 / 90, 4c 3x3 47 / 37,
+// 3b merged 5x5 549 / 481, 4a 324 / 248).  DR_QLIN = 0 / 1 overrides (never / wherever it can).
 static bool qlin_preferred(const ConvParams& p) {
-    return tunable("DR_QLIN", 0) > 0 && conv_qlin_supports(p);
+    const int pref = tunable("DR_QLIN", -1);
+    if (pref == 0 || !conv_qlin_supports(p)) return false;
+    if (pref > 0) return true;
+    const int cout16 = (p.Cout + 15) / 16 * 16;
+    return cout16 <= 128 && conv_qlin_fill(p) >= 0.8 && p.m_tiles >= 2 * num_sms();
 }
 
 int conv_pick_path(const ConvParams& p, int forced) {

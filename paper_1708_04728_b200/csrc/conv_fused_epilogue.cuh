@@ -92,6 +92,27 @@ __device__ __forceinline__ void fe_load_chunk(uint32_t taddr, const float* bias_
     }
 }
 
+// The registers of a TMEM load that has just been waited for, passed through an empty volatile statement: what reads them
+// stays behind the wait in program order.
+__device__ __forceinline__ void fe_pin32(uint32_t* r) {
+#pragma unroll
+    for (int j = 0; j < 32; j += 8)
+        asm volatile("" : "+r"(r[j]), "+r"(r[j + 1]), "+r"(r[j + 2]), "+r"(r[j + 3]), "+r"(r[j + 4]), "+r"(r[j + 5]), "+r"(r[j + 6]), "+r"(r[j + 7]));
+}
+// raw accumulators of 32 columns starting at channel c -> + bias, ReLU
+__device__ __forceinline__ void fe_convert_chunk(const uint32_t* r, const float* bias_s, int c, bool relu, float* x) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const float4 b4 = *reinterpret_cast<const float4*>(bias_s + c + 4 * q);
+        const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float v = __uint_as_float(r[4 * q + k]) + bb[k];
+            x[4 * q + k] = relu ? fmaxf(v, 0.f) : v;
+        }
+    }
+}
+
 // LRN (window of five) of the 32 channels in cur, given the two channels before (pm2, pm1) and the chunk after;
 // the result goes to dst as bfloat16 (-inf for rows outside the convolution plane).  The window sum slides:
 // ss[j] = ss[j-1] + x[j+2]^2 - x[j-3]^2, restarted from its five terms every 8 channels (a sum that cancels to a few
@@ -156,7 +177,9 @@ __device__ __forceinline__ void fe_lrn_chunk(const ConvParams& p, const float* c
 // Called by the 4 warps of one epilogue group together (a kernel may run two groups on alternate tiles,
 // each with its own stage buffer and named barrier); `release` is invoked by each warp once its TMEM
 // reads are done.
-template <class Release>
+// PREFETCH (kernels that give the epilogue warps registers for it): the TMEM load of the next 32-channel chunk is in
+// flight while the LRN of the current one is computed.
+template <bool PREFETCH, class Release>
 __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, uint32_t taddr, uint8_t* stage, int row, int bar_id,
                                                Release release) {
     const int C = p.Cout;
@@ -176,7 +199,34 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
     uint8_t* srow = stage + (size_t)row * pitch;
 
     // ---- drain TMEM (+ bias, ReLU, LRN when LRN comes first), stage
-    if (lrn_first) {
+    if (lrn_first && PREFETCH && !am) {
+        // as below, with the raw accumulators of the chunk after the next one requested before the LRN of the current one
+        float xa[32], xb[32];
+        uint32_t raw[32];
+        float pm2 = 0.f, pm1 = 0.f;
+        fe_load_chunk(taddr, bias_s, 0, true, relu, xa);
+        if (32 < C) ptx::tmem_ld_x32(taddr + 32, raw);
+        for (int c0 = 0; c0 < C; c0 += 64) {
+            const bool has_b = c0 + 32 < C;
+            if (has_b) { ptx::tmem_ld_wait(); fe_pin32(raw); fe_convert_chunk(raw, bias_s, c0 + 32, relu, xb); }
+            else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) xb[j] = 0.f;
+            }
+            if (c0 + 64 < C) ptx::tmem_ld_x32(taddr + c0 + 64, raw);
+            fe_lrn_chunk<false>(p, xa, xb, pm2, pm1, srow + c0 * 2, valid);
+            if (has_b) {
+                const bool has_a = c0 + 64 < C;
+                if (has_a) { ptx::tmem_ld_wait(); fe_pin32(raw); fe_convert_chunk(raw, bias_s, c0 + 64, relu, xa); }
+                else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) xa[j] = 0.f;
+                }
+                if (c0 + 96 < C) ptx::tmem_ld_x32(taddr + c0 + 96, raw);
+                fe_lrn_chunk<false>(p, xb, xa, pm2, pm1, srow + (c0 + 32) * 2, valid);
+            }
+        }
+    } else if (lrn_first) {
         // two register chunks used alternately as "current" and "next" (no copy between them)
         float xa[32], xb[32];
         float pm2 = 0.f, pm1 = 0.f;                      // x[c-2], x[c-1] of the chunk before

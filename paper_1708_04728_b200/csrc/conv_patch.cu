@@ -188,7 +188,7 @@ conv_patch_tma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap ma
                 }
                 tc_fence_after();
                 uint64_t* te = &sh.tempty[acc];
-                fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * 256), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
+                fused_epilogue<false>(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * 256), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
                     __syncwarp();
                     if (lane == 0) mbar_arrive(te);
                 });
@@ -229,7 +229,12 @@ __device__ __forceinline__ void tma_load_4d_tile_pair(uint32_t dst, const CUtens
                  : "memory");
 }
 
-__global__ void __launch_bounds__(P_THREADS, 1)
+// Warps in groups of four (the unit in which registers are re-assigned): warps 0-3 = producer, MMA issuer and two idle
+// warps, which give registers up; warps 4-7 and 8-11 = the two epilogue groups, which take them (the fused LRN epilogue
+// keeps two 32-channel chunks, their squares, window sums and scales, and a TMEM load in flight, in registers).
+constexpr int PP_THREADS = 384;
+constexpr int PP_REGS_AUX = 40, PP_REGS_EPI = 232;      // 128 * 40 + 256 * 232 = 384 * 168, the registers of the launch
+__global__ void __launch_bounds__(PP_THREADS, 1)
 conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const int stages,
                        const int stage_bytes, const int groups, const int resident, const int bsub_bytes) {
     extern __shared__ uint8_t smem_raw[];
@@ -254,8 +259,8 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
     }
     if (warp == 1) { tmem_alloc_pair(&sh.tmem_base, 512); tmem_relinquish_pair(); }
     const int fe_bytes = fe_smem_bytes(p);
-    fe_init(p, fe_stage, tid, P_THREADS);
-    if (groups > 1) fe_init(p, fe_stage + fe_bytes, tid, P_THREADS);
+    fe_init(p, fe_stage, tid, PP_THREADS);
+    if (groups > 1) fe_init(p, fe_stage + fe_bytes, tid, PP_THREADS);
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();                                                      // both CTAs' barriers exist before any remote arrive
@@ -274,6 +279,7 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
     const uint32_t half_rows = (uint32_t)p.Nt >> 1;
 
     if (warp == 0) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX));
         if (lane == 0) {
             const uint32_t a_tx = (uint32_t)(pwc * phc) * 128u;
             const uint32_t b_tx = half_rows * 128u;
@@ -331,23 +337,27 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0 && rank == 0) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX));
+        if (rank == 0) {
+            // the whole warp walks the loop (addresses and descriptors are warp-uniform), lane 0 alone issues and commits:
+            // measured faster than a loop run by one lane inside a divergent branch
+            const uint32_t el = lane == 0 ? 1u : 0u;
             const uint32_t tfull0 = smem_u32(&sh.tfull[0]), tempty0 = smem_u32(&sh.tempty[0]);
             const int last_nk16 = ((p.Cin - ((cpb - 1) << 6)) + 15) >> 4;
             const uint32_t idesc = make_idesc_bf16(2 * TILE_M, p.Nt);
             int s = 0, it = 0;
             uint32_t ph = 0;
             bool ok = true;
-            if (resident && !mbar_wait(&sh.wfull, 0, abort_flag)) {
-                if (!*abort_flag) report_timeout(p.status, 45, 0);
+            if (resident && !__all_sync(0xffffffffu, mbar_wait(&sh.wfull, 0, abort_flag))) {
+                if (el && !*abort_flag) report_timeout(p.status, 45, 0);
                 *abort_flag = 1;
                 ok = false;
             }
-            uint32_t ready = mbar_test_u32(full0, 0);
+            bool ready = __all_sync(0xffffffffu, mbar_test_u32(full0, 0) != 0);
             for (int u = unit; u < units && ok; u += nunits, ++it) {
                 const int acc = it & 1, au = it >> 1;
-                if (!mbar_wait_u32(tempty0 + 8 * acc, (au & 1) ^ 1, abort_flag)) {
-                    if (!*abort_flag) report_timeout(p.status, 42, u);
+                if (!__all_sync(0xffffffffu, mbar_wait_u32(tempty0 + 8 * acc, (au & 1) ^ 1, abort_flag))) {
+                    if (el && !*abort_flag) report_timeout(p.status, 42, u);
                     *abort_flag = 1;
                     break;
                 }
@@ -356,8 +366,8 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
                 uint32_t accum = 0;
                 int cc = 0;
                 for (int kb = 0; kb < nkb; ++kb) {
-                    if (!ready && !mbar_wait_slow_u32(full0 + 8 * s, ph, abort_flag)) {
-                        if (!*abort_flag) report_timeout(p.status, 43, u);
+                    if (!ready && !__all_sync(0xffffffffu, mbar_wait_slow_u32(full0 + 8 * s, ph, abort_flag))) {
+                        if (el && !*abort_flag) report_timeout(p.status, 43, u);
                         *abort_flag = 1;
                         ok = false;
                         break;
@@ -365,29 +375,32 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
                     int s2 = s + 1;
                     uint32_t ph2 = ph;
                     if (s2 == stages) { s2 = 0; ph2 ^= 1; }
-                    ready = mbar_test_u32(full0 + 8 * s2, ph2);
+                    ready = __all_sync(0xffffffffu, mbar_test_u32(full0 + 8 * s2, ph2) != 0);
                     tc_fence_after();
                     const uint32_t a = smem_base + (uint32_t)s * (uint32_t)stage_bytes;
                     const uint32_t alo = sdesc_lo(a);
                     const uint32_t blo = sdesc_lo(resident ? b_res0 + (uint32_t)kb * (uint32_t)bsub_bytes : a + P_A_BYTES);
                     const int nk16 = (cc == cpb - 1) ? last_nk16 : 4;
                     cc = (cc + 1 == cpb) ? 0 : cc + 1;
-                    umma_bf16_lo<true>(d, alo, blo, idesc, accum, 1u);
+                    umma_bf16_lo<true>(d, alo, blo, idesc, accum, el);
                     accum = 1;
-                    umma_bf16_lo<true>(d, alo + 2, blo + 2, idesc, 1u, nk16 > 1);
-                    umma_bf16_lo<true>(d, alo + 4, blo + 4, idesc, 1u, nk16 > 2);
-                    umma_bf16_lo<true>(d, alo + 6, blo + 6, idesc, 1u, nk16 > 3);
-                    umma_commit_u32<true>(empty0 + 8 * s);
+                    umma_bf16_lo<true>(d, alo + 2, blo + 2, idesc, 1u, (nk16 > 1) & el);
+                    umma_bf16_lo<true>(d, alo + 4, blo + 4, idesc, 1u, (nk16 > 2) & el);
+                    umma_bf16_lo<true>(d, alo + 6, blo + 6, idesc, 1u, (nk16 > 3) & el);
+                    if (el) umma_commit_u32<true>(empty0 + 8 * s);
                     s = s2;
                     ph = ph2;
                 }
-                if (ok) umma_commit_u32<true>(tfull0 + 8 * acc);
+                if (ok && el) umma_commit_u32<true>(tfull0 + 8 * acc);
             }
         }
         __syncwarp();
+    } else if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX));   // idle warps of the first group of four
     } else {
         // epilogue groups of four warps, as in conv_patch_tma_kernel; each CTA drains its own patch
-        const int g = (warp - 2) >> 2;
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(PP_REGS_EPI));
+        const int g = (warp - 4) >> 2;
         const int q = warp & 3;
         const int row = q * 32 + lane;
         if (g < groups) {
@@ -405,7 +418,7 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
                 }
                 tc_fence_after();
                 uint64_t* te = &sh.tempty[acc];
-                fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * 256), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
+                fused_epilogue<true>(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * 256), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
                     __syncwarp();
                     if (lane == 0) mbar_arrive_leader(te);
                 });
@@ -608,7 +621,7 @@ __global__ void __launch_bounds__(S_THREADS, 1) conv_stem_kernel(const ConvParam
             }
             tc_fence_after();
             uint64_t* te = &sh.tempty[g];
-            fused_epilogue(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 64), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
+            fused_epilogue<false>(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 64), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(te);
             });
@@ -675,11 +688,13 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
             }
         if (groups) {
             if (stages > P_MAX_STAGES) stages = P_MAX_STAGES;
+            const int forced_stages = tunable("DR_PATCH_STAGES", 0);
+            if (forced_stages >= 2 && forced_stages < stages) stages = forced_stages;
             cudaLaunchConfig_t cfg = {};
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeClusterDimension;
             attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-            cfg.blockDim = dim3(P_THREADS); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
+            cfg.blockDim = dim3(PP_THREADS); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
             if (!pair_attr) {
                 if (cudaFuncSetAttribute(conv_patch_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
                 cfg.gridDim = dim3(2 * num_sms());

@@ -996,8 +996,10 @@ static bool pick_dual(const ConvParams& p, bool use_pair, bool wide, int ep_byte
     // enough to matter, i.e. tiles of at most 224 columns over at least 48 k-blocks (3a / 5a / 5b merged 5x5: 250 -> 216,
     // 211 -> 174, 231 -> 204 us) and tiles of at most 128 columns (two accumulators per pipeline); a loss on tiles of
     // 240 and 256 columns, which one issuer keeps busy (4c / 4d merged 5x5: 224 -> 254, 219 -> 246 us), and on short
-    // reductions with wide tiles, where each ring's three stages cover less of the load latency (3b 3x3: 92 -> 113 us).
-    if (pref < 0 && !((p.Nt <= 224 && nkb >= 48) || (p.Nt <= 128 && nkb >= 16))) return false;
+    // reductions with wide tiles, where each ring's three stages cover less of the load latency (3b 3x3: 92 -> 113 us), and
+    // on 1x1 layers (4a reducer: 22.5 -> 24.6 us).
+    // Spatial filters over 64-channel tiles (ResNet-50 stage 2, 3x3 with 64 output channels, 9 k-blocks): 78 -> 62 us.
+    if (pref < 0 && !((p.Nt <= 224 && nkb >= 48) || (p.Nt <= 128 && nkb >= 16) || (p.Nt <= 128 && p.k > 1 && nkb >= 8))) return false;
     int k = tunable("DR_TMA_KPB", 0);
     if (k <= 0) k = 1;
     if (k >= 4) k = 4; else if (k == 3) k = 2;
