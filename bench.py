@@ -29,7 +29,7 @@ METRIC = "slim GoogLeNet forward throughput"
 UNIT = "images/s"
 # DRAM traffic of the dominant kernel's largest launch from one ncu capture (dram__bytes_read.sum, dram__bytes_write.sum),
 # with the tiling the capture was taken on; the line carries it only while dr_conv_plan still reports that tiling.
-NCU_TRAFFIC = {"layer": "3b.m5", "batch": 256, "dram_read_bytes": 106.566e6, "dram_write_bytes": 67.416e6,
+NCU_TRAFFIC = {"layer": "3b.m5", "batch": 256, "dram_read_bytes": 106.605e6, "dram_write_bytes": 67.799e6,
                "plan": {"path": "umma_tma", "Nt": 144, "n_blocks": 1, "pair": 1, "wide": 1},
                "note": "ncu capture of one launch at batch 256; a lower bound of the launch's traffic: part of its output is still in L2 when it ends"}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -425,6 +425,9 @@ def main():
                     help="googlenet = the headline workload; resnet50 = the BN-folded bottleneck network (context)")
     ap.add_argument("--layers-out", default=None, help="write the per-layer table (us, roofline) as JSON")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="only the timed region, the end-to-end loop and the per-layer table: no sustained loop, no unslimmed / batch-1 "
+                         "context runs (for profiler launch lists)")
     ap.add_argument("--layer", default=None,
                     help="time ONE slim layer of the network (e.g. conv1, conv2, 3b.m5, 4e.3x3) instead of the whole step: "
                          "the small case for profiler captures")
@@ -559,7 +562,7 @@ def main():
     # ---- the same step in a loop of a few seconds, in chunks of about a quarter second, each chunk with the median SM clock
     # NVML showed while it ran: what the step costs at the clock the part sustains, next to the (possibly short) headline region
     sustained = None
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.no_extras:
         per = max(1, int(250.0 / max(total_ms / args.steps, 1e-3)))
         chunks, t_end = [], time.perf_counter() + 3.0
         while time.perf_counter() < t_end and len(chunks) < 40:
@@ -618,7 +621,6 @@ def main():
     e2e_ms = max_over_ranks(e2e_ms, world)
     e2e_value = whole_job_images_per_s(e2e_ms, B, e2e_steps, world)
     assert bool(torch.isfinite(logits_host).all())
-    clocks = sampler.stop() if sampler else None
 
     if rank != 0:
         if world > 1:
@@ -631,12 +633,19 @@ def main():
     L = net.dr_net_num_layers()
     infos = [net.dr_net_layer_info(i) for i in range(L)]
     us = np.zeros((reps, L))
+    t_layers0 = time.perf_counter()
     for r in range(reps):
         flush.zero_()
         step()
         torch.cuda.synchronize()
         us[r] = [net.dr_net_layer_time_us(i) for i in range(L)]
+    t_layers1 = time.perf_counter()
     net.dr_net_set_timing(False)
+    layer_clock = sampler.window(t_layers0, t_layers1) if sampler else None
+    clocks = sampler.stop() if sampler else None
+    if clocks and headline_clock is not None:
+        clocks["sm_mhz"] = headline_clock                  # the median over the timed region's own window
+        clocks["sm_mhz_per_layer_pass"] = layer_clock
     us = np.median(us, axis=0)
     bw_peak = pk["hbm_gbs"] * 1e9
     rows, t_roof_total = [], 0.0
@@ -654,10 +663,14 @@ def main():
     achieved = top["gflop"] / top["us"] * 1e3 if top else 0.0   # GFLOP/us = PFLOP/s
     # Which measured peak the fraction is taken against follows from the clocks sampled in this run: the burst figure
     # when the median SM clock under load stayed within 5 % of the maximum (a short region), the sustained one otherwise.
-    clk_ref = headline_clock if headline_clock is not None else (clocks or {}).get("sm_mhz")
+    # (the launch's duration comes from the per-layer pass: five steps with an event pair around every launch, so that pass's clock)
+    clk_ref = layer_clock if layer_clock is not None else (headline_clock if headline_clock is not None else (clocks or {}).get("sm_mhz"))
     clk_max = (clocks or {}).get("sm_max_mhz")
     burst_regime = bool(clk_ref and clk_max and clk_ref >= 0.95 * clk_max)
-    peak_name = "bf16_tflops" if burst_regime else "bf16_tflops_sustained"
+    # A launch that runs above the sustained figure (taken by the driver at the clock a seconds-long GEMM loop settles at, far
+    # below what this step's mix of layers sustains) is not bounded by it: the burst figure, the larger one, is then the ceiling.
+    above_sustained = achieved > pk["bf16_tflops_sustained"]
+    peak_name = "bf16_tflops" if (burst_regime or above_sustained) else "bf16_tflops_sustained"
     # DRAM bytes of that launch from the stored ncu capture; reported only while the layer still runs in the tiling the
     # capture was taken on (else null)
     traffic, traffic_note = None, None
@@ -668,7 +681,8 @@ def main():
             traffic_note = NCU_TRAFFIC["note"]
     roofline = {"bound": "tensor", "kernel": f"conv_umma_tma_kernel, launch {top['name'] if top else '-'} (largest of {len(tma)} tensor-bound launches per step)",
                 "achieved": achieved, "peak": pk[peak_name],
-                "peak_kind": f"{pk_kind} {'burst' if burst_regime else 'sustained'} bf16: median SM clock in the timed region {clk_ref} of {clk_max} MHz",
+                "peak_kind": f"{pk_kind} {'burst' if peak_name == 'bf16_tflops' else 'sustained'} bf16: median SM clock while the per-layer times were taken {clk_ref} of {clk_max} MHz"
+                             + ("; the launch runs above the sustained figure, so the burst figure is the ceiling used" if above_sustained and not burst_regime else ""),
                 "unit": "TFLOP/s", "frac": achieved / pk[peak_name],
                 "frac_vs_burst": achieved / pk["bf16_tflops"], "frac_vs_sustained": achieved / pk["bf16_tflops_sustained"],
                 "traffic": traffic, "traffic_note": traffic_note,
@@ -692,6 +706,8 @@ def main():
     # ---- context numbers: batch 1 latency regime and the unslimmed layer-by-layer path
     extra = {}
     try:
+        if args.no_extras:
+            raise RuntimeError("skipped (--no-extras)")
         net_u, ws_u, keep_u = make_net(dr.DR_MODE_UNSLIMMED, B)
         lu = torch.empty_like(logits)
         tu = timed(lambda: net_u.dr_net_forward(x, ws_u, lu), 5, 2)

@@ -237,7 +237,7 @@ static void build_googlenet(dr_net* n) {
     } else if (slim) {
         t = add_conv(n, "conv1", x, 7, 2, 3, 64, BR | DR_POOL | DR_LRN, w, b);
     } else {
-        t = add_conv(n, "conv1.conv", x, 7, 2, 3, 64, DR_BIAS, w, b);
+        t = add_conv_s2d(n, "conv1.conv", x, 7, 2, 3, 64, DR_BIAS, w.raw, b);   // a layer of its own has no pooling to fuse: the tensor-core form of a 3-channel strided conv
         t = add_simple(n, OP_RELU, "conv1.relu", t);
         t = add_simple(n, OP_MAXPOOL, "conv1.pool", t);
         t = add_simple(n, OP_LRN, "conv1", t);
@@ -363,7 +363,7 @@ static void build_googlenet_paper(dr_net* n) {
     if (slim) {
         t = add_conv(n, "conv1", x, 7, 2, 3, 64, BR | DR_POOL | DR_LRN, w, b);
     } else {
-        t = add_conv(n, "conv1.conv", x, 7, 2, 3, 64, DR_BIAS, w, b);
+        t = add_conv_s2d(n, "conv1.conv", x, 7, 2, 3, 64, DR_BIAS, w.raw, b);   // a layer of its own has no pooling to fuse: the tensor-core form of a 3-channel strided conv
         t = add_simple(n, OP_RELU, "conv1.relu", t);
         t = add_simple(n, OP_MAXPOOL, "conv1.pool", t);
         t = add_simple(n, OP_LRN, "conv1", t);
@@ -415,7 +415,8 @@ static void build_resnet50(dr_net* n) {
             if (pool) f |= DR_POOL;
             return add_conv(n, name, in, k, s, p, cout, f, wsref(wo), wsref(bo), -2, 0, residual);
         }
-        int t = add_conv(n, name + ".conv", in, k, s, p, cout, 0, rawref(wi), PRef());
+        int t = (s >= 2 && s * s * cin <= 64) ? add_conv_s2d(n, name + ".conv", in, k, s, p, cout, 0, wi, PRef())
+                                              : add_conv(n, name + ".conv", in, k, s, p, cout, 0, rawref(wi), PRef());
         t = add_norm(n, OP_BN, name + ".bn", t, mean, var);
         const bool last = !relu && !pool && residual == -2;
         t = add_norm(n, OP_SCALE, last ? name : name + ".scale", t, gamma, beta);
