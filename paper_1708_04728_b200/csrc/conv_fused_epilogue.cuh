@@ -422,4 +422,143 @@ __device__ __forceinline__ void fused_epilogue(const ConvParams& p, int tile, ui
     fe_bar(bar_id);                                       // the stage may be overwritten by the next tile
 }
 
+// fe_lrn_chunk for threads with few registers (bfloat16 output only): the bound that selects the series is the sum of
+// all 36 squares (every window sum is at most that), so no window sum has to be kept; sums and scales are consumed
+// eight channels at a time.
+__device__ __forceinline__ void fe_lrn_chunk_lean(const ConvParams& p, const float* cur, const float* nxt, float& pm2, float& pm1, uint8_t* dst,
+                                                  bool valid) {
+    float total = fmaf(pm2, pm2, pm1 * pm1);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) total = fmaf(cur[j], cur[j], total);
+    total = fmaf(nxt[0], nxt[0], fmaf(nxt[1], nxt[1], total));
+    const int mode = __all_sync(0xffffffffu, total < p.lrn_ss_max2) ? 0 : (__all_sync(0xffffffffu, total < p.lrn_ss_max) ? 1 : 2);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        float x[12];                               // channels 8q-2 .. 8q+9 of the chunk
+#pragma unroll
+        for (int j = 0; j < 12; ++j) {
+            const int c = 8 * q - 2 + j;
+            x[j] = c == -2 ? pm2 : c == -1 ? pm1 : c < 32 ? cur[c < 0 ? 0 : (c > 31 ? 31 : c)] : nxt[c - 32 > 1 ? 1 : c - 32];
+        }
+        float sq[12], ss[8], sc[8];
+#pragma unroll
+        for (int j = 0; j < 12; ++j) sq[j] = x[j] * x[j];
+        ss[0] = (sq[0] + sq[1]) + (sq[2] + sq[3]) + sq[4];
+#pragma unroll
+        for (int j = 1; j < 8; ++j) ss[j] = (ss[j - 1] - sq[j - 1]) + sq[j + 4];
+        if (mode == 0) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) sc[j] = fmaf(ss[j], fmaf(ss[j], p.lrn_s2, p.lrn_s1), p.lrn_kpow);
+        } else if (mode == 1) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) sc[j] = fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], fmaf(ss[j], p.lrn_s4, p.lrn_s3), p.lrn_s2), p.lrn_s1), p.lrn_kpow);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) sc[j] = __powf(fmaf(p.lrn_alpha_n, ss[j], p.lrn_k), -p.lrn_beta);
+        }
+        uint4 v;
+        if (valid) {
+            v.x = pack_bf16(x[2] * sc[0], x[3] * sc[1]);
+            v.y = pack_bf16(x[4] * sc[2], x[5] * sc[3]);
+            v.z = pack_bf16(x[6] * sc[4], x[7] * sc[5]);
+            v.w = pack_bf16(x[8] * sc[6], x[9] * sc[7]);
+        } else {
+            v.x = v.y = v.z = v.w = 0xFF80FF80u;     // -inf, -inf
+        }
+        *reinterpret_cast<uint4*>(dst + 16 * q) = v;
+    }
+    pm2 = cur[30];
+    pm1 = cur[31];
+}
+
+// The LRN-first epilogue (ReLU -> LRN -> pool, no positions) run by TWO groups of four warps on one tile: part 0 takes
+// channels [0, C/2), part 1 [C/2, C) of every row (C a multiple of 64), each with the two channels beyond its range
+// that the window of five needs; both parts pool and store together (256 threads).  A tile's accumulator is then
+// held half as long, which is what bounds a layer whose drain (the LRN arithmetic) takes longer than its MMAs.
+// `row` = 0..127 within the part; the named barrier `bar_id` is shared by the 256 threads.
+constexpr int FE_SPLIT_THREADS = 2 * FE_THREADS;
+__device__ __forceinline__ void fe_bar_split(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(FE_SPLIT_THREADS) : "memory"); }
+inline bool fe_split_supports(const ConvParams& p) { return fe_supports(p) && fe_lrn_first(p) && !p.argmax && p.Cout % 64 == 0; }
+
+template <class Release>
+__device__ __forceinline__ void fused_epilogue_split(const ConvParams& p, int tile, uint32_t taddr, uint8_t* stage, int row, int part, int bar_id,
+                                                     Release release) {
+    const int C = p.Cout, H = C >> 1;
+    const bool relu = p.flags & DR_RELU;
+    const int pitch = fe_stage_pitch(p);
+    const float* bias_s = reinterpret_cast<const float*>(stage + TILE_M * pitch);
+    const int pwc = 2 * p.PW + 1, phc = 2 * p.PH + 1;
+    const int per = p.tiles_h * p.tiles_w;
+    const int n = tile / per, t = tile - n * per;
+    const int th = t / p.tiles_w, tw = t - th * p.tiles_w;
+    const int pi = row / pwc, pj = row - pi * pwc;
+    const int ho = 2 * th * p.PH - 1 + pi, wo = 2 * tw * p.PW - 1 + pj;
+    const bool valid = pi < phc && ho >= 0 && ho < p.Ho && wo >= 0 && wo < p.Wo;
+    uint8_t* srow = stage + (size_t)row * pitch;
+    const int c_lo = part * H, c_hi = c_lo + H;
+
+    // ---- drain this part's channels: + bias, ReLU, LRN, stage as bf16.  One 32-channel chunk is live at a time; the
+    // two channels after it come from a two-column load of their own (tensor-memory loads are cheap, registers are not).
+    float pm2 = 0.f, pm1 = 0.f;
+    if (part) {                                            // channels c_lo-2, c_lo-1: the last two of the 16 columns before c_lo
+        uint32_t r[16];
+        ptx::tmem_ld_x16(taddr + c_lo - 16, r);
+        ptx::tmem_ld_wait();
+        const float v2 = __uint_as_float(r[14]) + bias_s[c_lo - 2], v1 = __uint_as_float(r[15]) + bias_s[c_lo - 1];
+        pm2 = relu ? fmaxf(v2, 0.f) : v2;
+        pm1 = relu ? fmaxf(v1, 0.f) : v1;
+    }
+    for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
+        uint32_t r[32], r2[2] = {0u, 0u};
+        const bool more = c0 + 32 < C;
+        ptx::tmem_ld_x32(taddr + c0, r);
+        if (more) ptx::tmem_ld_x2(taddr + c0 + 32, r2);
+        ptx::tmem_ld_wait();
+        fe_pin32(r);
+        asm volatile("" : "+r"(r2[0]), "+r"(r2[1]));
+        float x[32], nx[2];
+        fe_convert_chunk(r, bias_s, c0, relu, x);
+        if (more) {
+            const float v0 = __uint_as_float(r2[0]) + bias_s[c0 + 32], v1 = __uint_as_float(r2[1]) + bias_s[c0 + 33];
+            nx[0] = relu ? fmaxf(v0, 0.f) : v0;
+            nx[1] = relu ? fmaxf(v1, 0.f) : v1;
+        } else {
+            nx[0] = 0.f; nx[1] = 0.f;
+        }
+        fe_lrn_chunk_lean(p, x, nx, pm2, pm1, srow + c0 * 2, valid);
+    }
+    ptx::tc_fence_before();
+    release();                                            // this warp no longer needs the accumulator
+    fe_bar_split(bar_id);
+
+    // ---- 3x3 / 2 max over the staged patch, all 256 threads
+    __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.y);
+    const int npp = p.PH * p.PW;
+    const int C8 = C >> 3;
+    const int tix = part * FE_THREADS + row;
+    const int dpp = FE_SPLIT_THREADS / C8, dc8 = FE_SPLIT_THREADS - dpp * C8;
+    int pp = tix / C8, c8 = tix - pp * C8;
+    while (pp < npp) {
+        const int ppi = pp / p.PW, ppj = pp - ppi * p.PW;
+        const int ph = th * p.PH + ppi, pw = tw * p.PW + ppj;
+        if (ph < p.Hy && pw < p.Wy) {
+            const uint8_t* base = stage + (size_t)((2 * ppi) * pwc + 2 * ppj) * pitch + c8 * 16;
+            uint4 m = *reinterpret_cast<const uint4*>(base);
+            __nv_bfloat162* mm = reinterpret_cast<__nv_bfloat162*>(&m);
+#pragma unroll
+            for (int d = 1; d < 9; ++d) {
+                const uint4 u = *reinterpret_cast<const uint4*>(base + (size_t)((d / 3) * pwc + (d % 3)) * pitch);
+                const __nv_bfloat162* uu = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) mm[k] = __hmax2(mm[k], uu[k]);
+            }
+            const long long q = ((long long)n * p.Hy + ph) * p.Wy + pw;
+            *reinterpret_cast<uint4*>(y + q * p.ldc + p.coff + c8 * 8) = m;
+        }
+        pp += dpp; c8 += dc8;
+        if (c8 >= C8) { c8 -= C8; ++pp; }
+    }
+    fe_bar_split(bar_id);                                 // the stage may be overwritten by the next tile
+}
+
 }  // namespace dr

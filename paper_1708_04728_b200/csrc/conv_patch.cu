@@ -232,9 +232,17 @@ __device__ __forceinline__ void tma_load_4d_tile_pair(uint32_t dst, const CUtens
 // Warps in groups of four (the unit in which registers are re-assigned): warps 0-3 = producer, MMA issuer and two idle
 // warps, which give registers up; warps 4-7 and 8-11 = the two epilogue groups, which take them (the fused LRN epilogue
 // keeps two 32-channel chunks, their squares, window sums and scales, and a TMEM load in flight, in registers).
-constexpr int PP_THREADS = 384;
+//
+// SPLIT (LRN before the pool, channel count a multiple of 64): each of the two tile groups is eight warps, four per half
+// of the channels (fused_epilogue_split).  The accumulator of a tile is occupied while its MMAs run and while it is
+// drained, and with two accumulators a tile cannot take less than half of that sum; the drain of an LRN-first layer
+// (the LRN arithmetic of 192 channels per row) is longer than the MMAs, and two warps per row halve it.  640 threads:
+// 128 * 32 + 512 * 112 registers = 640 * 96.
+constexpr int PP_THREADS = 384, PP_THREADS_SPLIT = 640;
 constexpr int PP_REGS_AUX = 40, PP_REGS_EPI = 232;      // 128 * 40 + 256 * 232 = 384 * 168, the registers of the launch
-__global__ void __launch_bounds__(PP_THREADS, 1)
+constexpr int PP_REGS_AUX_SPLIT = 32, PP_REGS_EPI_SPLIT = 112;   // 128 * 32 + 512 * 112 = 640 * 96
+template <bool SPLIT>
+__global__ void __launch_bounds__(SPLIT ? PP_THREADS_SPLIT : PP_THREADS, 1)
 conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const int stages,
                        const int stage_bytes, const int groups, const int resident, const int bsub_bytes) {
     extern __shared__ uint8_t smem_raw[];
@@ -250,7 +258,7 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
 
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 8); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], SPLIT ? 16 : 8); }   // the epilogue warps of both CTAs
         mbar_init(&sh.wfull, 1);
         sh.abort = 0;
         fence_barrier_init();
@@ -259,8 +267,8 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
     }
     if (warp == 1) { tmem_alloc_pair(&sh.tmem_base, 512); tmem_relinquish_pair(); }
     const int fe_bytes = fe_smem_bytes(p);
-    fe_init(p, fe_stage, tid, PP_THREADS);
-    if (groups > 1) fe_init(p, fe_stage + fe_bytes, tid, PP_THREADS);
+    fe_init(p, fe_stage, tid, (int)blockDim.x);
+    if (groups > 1) fe_init(p, fe_stage + fe_bytes, tid, (int)blockDim.x);
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();                                                      // both CTAs' barriers exist before any remote arrive
@@ -279,7 +287,7 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
     const uint32_t half_rows = (uint32_t)p.Nt >> 1;
 
     if (warp == 0) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX));
+        if (SPLIT) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX_SPLIT)); else asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX));
         if (lane == 0) {
             const uint32_t a_tx = (uint32_t)(pwc * phc) * 128u;
             const uint32_t b_tx = half_rows * 128u;
@@ -337,7 +345,7 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
         }
         __syncwarp();
     } else if (warp == 1) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX));
+        if (SPLIT) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX_SPLIT)); else asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX));
         if (rank == 0) {
             // the whole warp walks the loop (addresses and descriptors are warp-uniform), lane 0 alone issues and commits:
             // measured faster than a loop run by one lane inside a divergent branch
@@ -396,11 +404,13 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
         }
         __syncwarp();
     } else if (warp < 4) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX));   // idle warps of the first group of four
+        if (SPLIT) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX_SPLIT)); else asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PP_REGS_AUX));   // idle warps of the first group of four
     } else {
         // epilogue groups of four warps, as in conv_patch_tma_kernel; each CTA drains its own patch
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(PP_REGS_EPI));
-        const int g = (warp - 4) >> 2;
+        if (SPLIT) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(PP_REGS_EPI_SPLIT));
+        else asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(PP_REGS_EPI));
+        const int g = SPLIT ? (warp - 4) >> 3 : (warp - 4) >> 2;            // tile group
+        const int part = SPLIT ? ((warp - 4) >> 2) & 1 : 0;                  // half of the channels (SPLIT)
         const int q = warp & 3;
         const int row = q * 32 + lane;
         if (g < groups) {
@@ -418,10 +428,13 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
                 }
                 tc_fence_after();
                 uint64_t* te = &sh.tempty[acc];
-                fused_epilogue<true>(p, t, tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * 256), fe_stage + g * fe_bytes, row, 1 + 2 * g, [&]() {
+                const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * 256);
+                auto release = [&]() {
                     __syncwarp();
                     if (lane == 0) mbar_arrive_leader(te);
-                });
+                };
+                if (SPLIT) fused_epilogue_split(p, t, taddr, fe_stage + g * fe_bytes, row, part, 1 + g, release);
+                else fused_epilogue<true>(p, t, taddr, fe_stage + g * fe_bytes, row, 1 + 2 * g, release);
             }
         }
     }
@@ -694,12 +707,23 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeClusterDimension;
             attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-            cfg.blockDim = dim3(PP_THREADS); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
+            // two warps per row for the drain where the LRN comes first (see the kernel's comment)
+            const bool split = fe_split_supports(p) && tunable("DR_PATCH_SPLIT", 1) != 0;
+            cfg.blockDim = dim3(split ? PP_THREADS_SPLIT : PP_THREADS); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
             if (!pair_attr) {
-                if (cudaFuncSetAttribute(conv_patch_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
-                cfg.gridDim = dim3(2 * num_sms());
-                cfg.dynamicSmemBytes = (size_t)P_SMEM_MAX;
-                if (cudaOccupancyMaxActiveClusters(&max_clusters, conv_patch_pair_kernel, &cfg) != cudaSuccess || max_clusters < 1) return DR_ERR_CUDA;
+                if (cudaFuncSetAttribute(conv_patch_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+                if (cudaFuncSetAttribute(conv_patch_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
+                int mc[2] = {0, 0};
+                for (int v = 0; v < 2; ++v) {
+                    cudaLaunchConfig_t q = cfg;
+                    q.blockDim = dim3(v ? PP_THREADS_SPLIT : PP_THREADS);
+                    q.gridDim = dim3(2 * num_sms());
+                    q.dynamicSmemBytes = (size_t)P_SMEM_MAX;
+                    const cudaError_t e = v ? cudaOccupancyMaxActiveClusters(&mc[v], conv_patch_pair_kernel<true>, &q)
+                                            : cudaOccupancyMaxActiveClusters(&mc[v], conv_patch_pair_kernel<false>, &q);
+                    if (e != cudaSuccess || mc[v] < 1) return DR_ERR_CUDA;
+                }
+                max_clusters = mc[0] < mc[1] ? mc[0] : mc[1];
                 pair_attr = true;
             }
             alignas(64) CUtensorMap map_bh;
@@ -713,7 +737,9 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
             const int pairs = units < max_clusters ? units : max_clusters;
             cfg.gridDim = dim3(2 * pairs);
             cfg.dynamicSmemBytes = (size_t)smem_bytes;
-            if (cudaLaunchKernelEx(&cfg, conv_patch_pair_kernel, p, map_a, map_bh, stages, stage_bytes, groups, resident, bsub) != cudaSuccess) return DR_ERR_CUDA;
+            const cudaError_t le = split ? cudaLaunchKernelEx(&cfg, conv_patch_pair_kernel<true>, p, map_a, map_bh, stages, stage_bytes, groups, resident, bsub)
+                                         : cudaLaunchKernelEx(&cfg, conv_patch_pair_kernel<false>, p, map_a, map_bh, stages, stage_bytes, groups, resident, bsub);
+            if (le != cudaSuccess) return DR_ERR_CUDA;
             count_launch();
             return launch_status();
         }

@@ -410,7 +410,7 @@ static bool splitk_shape_ok(const ConvParams& p) {
 // Choice of n-block width and slice count for a layer that may use `budget` CTAs.  Measured on B200 (batch 1,
 // GoogLeNet's inception layers): n-blocks of about 80 columns and at most 32 slices are within a microsecond of
 // the best plan of every layer; a slice has at least two k-blocks unless `single` allows plans without splitting.
-static bool splitk_plan_budget(const ConvParams& p, int budget, bool single, SkPlan* out) {
+static bool splitk_plan_budget(const ConvParams& p, int budget, bool single, SkPlan* out, int s_cap = 0) {
     if (!splitk_shape_ok(p)) return false;
     const int cpb = (p.Cin + 63) >> 6;
     const int nkb = p.k * p.k * cpb;
@@ -429,6 +429,7 @@ static bool splitk_plan_budget(const ConvParams& p, int budget, bool single, SkP
     int s_max = tunable("DR_SPLITK_S", 0);
     if (s_max <= 0) s_max = 32;
     if (S > s_max) S = s_max;
+    if (s_cap > 0 && S > s_cap) S = s_cap;
     if (S < 1) S = 1;
     if (S < 2 && !single) return false;
     SkPlan b{};
@@ -485,12 +486,12 @@ static bool splitk_group_plan(const ConvParams& a, const ConvParams& b, const Co
     if (tunable("DR_SPLITK_PAIR", 1) == 0) return false;
     if (a.x != b.x || a.B != b.B || a.H != b.H || a.W != b.W || a.Cin != b.Cin) return false;
     const int small = tunable("DR_SPLITK_SMALL_CTAS", 48);
-    if (!splitk_plan_budget(b, small, true, pb)) return false;
+    if (!splitk_plan_budget(b, small, true, pb, tunable("DR_SPLITK_B_S", 0))) return false;
     int used = b.m_tiles * pb->n_blocks * pb->splits;
     long long tiles = (long long)b.m_tiles * pb->n_blocks;
     if (c) {
         if (c->x != b.y || c->Cin != b.Cout || b.ldc != b.Cout || b.coff != 0 || (b.flags & DR_OUT_F32)) return false;   // c reads b's dense output
-        if (!splitk_plan_budget(*c, small, true, pc)) return false;
+        if (!splitk_plan_budget(*c, small, true, pc, tunable("DR_SPLITK_C_S", 0))) return false;
         const int used_c = c->m_tiles * pc->n_blocks * pc->splits;
         if (used_c > used) used = used_c;
         tiles += (long long)c->m_tiles * pc->n_blocks + 1;

@@ -898,7 +898,8 @@ void conv_umma_tma_shape(ConvParams* pp, bool* use_pair_out, bool* wide_out) {
     // More than 256 output channels and a long K: wide tiles (two n-blocks per tile sharing the activation tile) of
     // near-equal sub-blocks, e.g. 288 -> one tile of 144 + 144, unless the coarser tiles cost more in rounds of the
     // persistent grid than the shared activation tile saves (measured: 5 to 9 % on the merged 5x5 layers of stage 4;
-    // short-K layers lose more to the epilogue, which wide tiles do not overlap with the next tile's MMAs).
+    // short-K layers lose more to the epilogue, which wide tiles do not overlap with the next tile's MMAs; 3x3 layers of
+    // 27 k-blocks still gain: 4d / 4e 3x3 at batch 256, 67.6 -> 57.4 and 68.0 -> 61.4 us).
     const int cout16_ = (p.Cout + 15) / 16 * 16;
     const int wide_pref = tunable("DR_TMA_WIDE", -1);
     bool wide = false;
@@ -911,7 +912,7 @@ void conv_umma_tma_shape(ConvParams* pp, bool* use_pair_out, bool* wide_out) {
         const long long cost_n = (m_units * p.n_blocks + capacity - 1) / capacity * p.Nt;
         const long long cost_w = (m_units * n_wide + capacity - 1) / capacity * 2 * nt_w;
         const int nkb_ = p.k * p.k * ((p.Cin + 63) / 64);
-        wide = wide_pref >= 0 ? wide_pref != 0 : (cout16_ > 256 && nkb_ >= 48 && cost_w * 95 <= cost_n * 100);
+        wide = wide_pref >= 0 ? wide_pref != 0 : (cout16_ > 256 && (nkb_ >= 48 || (p.k > 1 && nkb_ >= 24)) && cost_w * 95 <= cost_n * 100);
         if (p.flags & DR_LRN) wide = false;                      // the LRN window runs along one accumulator row
     }
     if (wide) {
