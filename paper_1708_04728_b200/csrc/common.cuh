@@ -29,6 +29,9 @@ __device__ __forceinline__ void report_timeout(int* status, int site, int tile) 
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? DR_OK : DR_ERR_CUDA; }
 inline int launch_status() { return cuda_status(cudaGetLastError()); }
+// Set by the network executor around its own pooling launches: the kernel is then launched with programmatic stream
+// serialization (it may be scheduled while the layer before it drains and waits for that layer before its first load).
+extern thread_local bool g_pool_pdl;
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

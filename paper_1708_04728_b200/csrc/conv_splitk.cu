@@ -17,6 +17,15 @@
 //
 // Scratch memory: `counters` (one int per output tile, zero on entry, back at zero when the kernel has finished) and `scratch`
 // (tiles x splits x Nt/4 x 128 float4, contents irrelevant on entry).
+//
+// Cluster form of steps 2-4 (the short jobs of an inception module, where the hand-over is most of the time): the
+// slices of a tile are the CTAs of one thread-block cluster; each keeps its partial tile in its own shared memory,
+// a cluster barrier replaces the counter, and every CTA sums its share over the cluster's shared memories
+// (distributed shared memory) in slice order: no trip through L2, the same fixed summation order.
+#include <map>
+#include <mutex>
+#include <utility>
+
 #include "conv_common.cuh"
 #include "umma_ptx.cuh"
 
@@ -37,6 +46,7 @@ struct SkShared {
 
 struct SkPlan {
     int nt, n_blocks, splits, kps, nkb, stages, sub_bytes;
+    int cluster;              // slices of a tile = ranks of a cluster of `splits` CTAs
     uint32_t tmem_cols;
     size_t scratch_bytes;
 };
@@ -55,6 +65,7 @@ struct alignas(64) SkJob {
     CUtensorMap map_a, map_b;
     ConvParams p;
     int a_mode, stages, sub_bytes, splits, kps;
+    int cluster;              // 1: the slices of a tile are the ranks of a cluster (splits = cluster size); partials in shared memory
     int ctas;                 // work items of this job = tiles x slices
     uint32_t tmem_cols;
     float* scratch;
@@ -63,6 +74,7 @@ struct alignas(64) SkJob {
 struct SkJobs {
     SkJob j[3];
     int n;                    // 1, 2 or 3 jobs
+    int cs;                   // cluster size of the launch (1: no clusters)
     int small_begin;          // first CTA of the small group (n >= 2)
     int* dep;                 // n == 3: counter on which job 2 waits for job 1
 };
@@ -85,7 +97,9 @@ __device__ __forceinline__ void sk_run_job(const SkJob* const J, const int bid, 
     int* __restrict__ counters = J->counters;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // work item of this CTA: K slice `split` of output tile (mt, nb)
+    // work item of this CTA: K slice `split` of output tile (mt, nb); in the cluster form the slice is the cluster rank
+    // (the job's first CTA starts a cluster) and trailing slices may be empty (they contribute zeros)
+    const bool clustered = J->cluster != 0;
     const int split = bid % splits, tile = bid / splits;
     const int nb = tile / p.m_tiles, mt = tile - nb * p.m_tiles;
     const int n0 = nb * p.Nt;
@@ -93,7 +107,7 @@ __device__ __forceinline__ void sk_run_job(const SkJob* const J, const int bid, 
     const int Nj = min(p.Nt, cout16 - n0);
     const int cpb = (p.Cin + 63) >> 6;
     const int nkb = p.k * p.k * cpb;
-    const int kb0 = split * kps, kb1 = min(nkb, kb0 + kps);
+    const int kb0 = min(nkb, split * kps), kb1 = min(nkb, kb0 + kps);
 
     volatile int* abort_flag = &sh.abort;
     const uint32_t smem_base = smem_u32(smem);
@@ -208,12 +222,18 @@ __device__ __forceinline__ void sk_run_job(const SkJob* const J, const int bid, 
             const bool row_ok = m < p.M;
             const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16);
             // partial tile layout [column quad][row]: the 32 rows of a warp are 512 contiguous bytes per store
-            float4* dst = reinterpret_cast<float4*>(scratch + ((size_t)tile * splits + split) * TILE_M * p.Nt) + row;
+            // (cluster form: in this CTA's shared memory, where the pipeline stages were)
+            float4* dst = (clustered ? reinterpret_cast<float4*>(smem) : reinterpret_cast<float4*>(scratch + ((size_t)tile * splits + split) * TILE_M * p.Nt)) + row;
+            const bool empty = kb1 <= kb0;                 // no k-block in this slice: the accumulator was never written
             int c = 0;
             for (; c + 32 <= Nj; c += 32) {
                 uint32_t v[32];
                 tmem_ld_x32(taddr + c, v);
                 tmem_ld_wait();
+                if (empty) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
                 if (row_ok) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
@@ -225,6 +245,10 @@ __device__ __forceinline__ void sk_run_job(const SkJob* const J, const int bid, 
                 uint32_t v[16];
                 tmem_ld_x16(taddr + c, v);
                 tmem_ld_wait();
+                if (empty) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = 0u;
+                }
                 if (row_ok) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
@@ -247,7 +271,8 @@ __device__ __forceinline__ void sk_run_job(const SkJob* const J, const int bid, 
     const int f0 = split * per, f1 = min(total, f0 + per);
     tc_fence_before();
     __syncthreads();                     // the whole partial tile has been written (by this CTA's threads, in CTA order)
-    if (tid == 0) {
+    if (clustered) cluster_sync_all();   // ... and so have the partial tiles of the other slices (every thread of the cluster arrives)
+    if (!clustered && tid == 0) {
         __threadfence();                 // ... and is visible device-wide before the arrival is (cumulative over the barrier)
         // the counter runs 0 .. 2*splits-1 and wraps to zero: first arrivals take it to `splits`, second ones back to 0
         const unsigned old = atomicInc(reinterpret_cast<unsigned*>(&counters[tile]), 2u * (unsigned)splits - 1u);
@@ -272,6 +297,7 @@ __device__ __forceinline__ void sk_run_job(const SkJob* const J, const int bid, 
         for (int base = f0 + tid; base < f1; base += 4 * SK_THREADS) {
             int row[4], col[4];
             const float4* src[4];
+            uint32_t soff[4];
             float4 acc[4], bias[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -280,6 +306,7 @@ __device__ __forceinline__ void sk_run_job(const SkJob* const J, const int bid, 
                 row[q] = e - cq * valid_rows;
                 col[q] = n0 + 4 * cq;
                 src[q] = part + (size_t)cq * TILE_M + row[q];
+                soff[q] = (uint32_t)(cq * TILE_M + row[q]) * 16u;
                 acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
                 bias[q] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if ((p.flags & DR_BIAS) && col[q] < p.Cout)
@@ -289,7 +316,7 @@ __device__ __forceinline__ void sk_run_job(const SkJob* const J, const int bid, 
             for (int sp = 0; sp < splits; ++sp) {
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const float4 v = __ldcg(src[q] + (size_t)sp * slice4);
+                    const float4 v = clustered ? ld_shared_cluster_f4(mapa_shared(smem_base, (uint32_t)sp) + soff[q]) : __ldcg(src[q] + (size_t)sp * slice4);
                     acc[q].x += v.x; acc[q].y += v.y; acc[q].z += v.z; acc[q].w += v.w;
                 }
             }
@@ -320,12 +347,13 @@ __device__ __forceinline__ void sk_run_job(const SkJob* const J, const int bid, 
     __syncthreads();                     // every thread of this CTA has finished reading the partials and has stored its outputs
     if (tid == 0) {
         // second arrival, not waited for: the last of them wraps the counter back to zero
-        red_inc_gpu(&counters[tile], 2u * (unsigned)splits - 1u);
+        if (!clustered) red_inc_gpu(&counters[tile], 2u * (unsigned)splits - 1u);
         if (dep_signal) {                // this CTA's share of the job's output is in memory: tell the job that reads it
             __threadfence();
             red_inc_gpu(dep, dep_wrap);
         }
     }
+    if (clustered) cluster_sync_all();   // no CTA of the cluster reads this one's shared memory any more (it may be refilled, or the CTA may exit)
 }
 
 __global__ void __launch_bounds__(SK_THREADS, 1) conv_splitk_kernel(const __grid_constant__ SkJobs jobs) {
@@ -448,6 +476,39 @@ static bool splitk_plan_budget(const ConvParams& p, int budget, bool single, SkP
     return true;
 }
 
+// Cluster form of a short job: exactly `cs` slices per tile (trailing ones may be empty), n-blocks of about 80 columns,
+// fewer if the job would not fit `budget` CTAs.
+static bool splitk_plan_cluster(const ConvParams& p, int budget, int cs, SkPlan* out) {
+    if (!splitk_shape_ok(p)) return false;
+    const int cpb = (p.Cin + 63) >> 6;
+    const int nkb = p.k * p.k * cpb;
+    if (nkb < 2) return false;
+    const int cout16 = (p.Cout + 15) & ~15;
+    const int nb_min = (cout16 + 255) / 256;
+    int nb = (cout16 + 40) / 80;
+    if (nb < nb_min) nb = nb_min;
+    while (nb > nb_min && (long long)p.m_tiles * nb * cs > budget) --nb;
+    int nt = ((cout16 + nb - 1) / nb + 15) / 16 * 16;
+    while ((long long)nt * (nb - 1) >= cout16 && nb > 1) { --nb; nt = ((cout16 + nb - 1) / nb + 15) / 16 * 16; }
+    const long long tiles = (long long)p.m_tiles * nb;
+    if (tiles > SK_MAX_TILES || tiles * cs > budget) return false;
+    SkPlan b{};
+    b.kps = (nkb + cs - 1) / cs;
+    b.splits = cs;
+    b.cluster = 1;
+    b.nt = nt; b.n_blocks = nb; b.nkb = nkb;
+    b.sub_bytes = SK_A_BYTES + ((b.nt * 128 + 1023) & ~1023);
+    int st = (tunable("DR_SPLITK_SMEM_KB", 200) * 1024 - 1024) / b.sub_bytes;
+    if (st > SK_MAX_STAGES) st = SK_MAX_STAGES;
+    if (st > b.kps) st = b.kps;
+    b.stages = st;
+    b.tmem_cols = 32;
+    while ((int)b.tmem_cols < b.nt) b.tmem_cols <<= 1;
+    b.scratch_bytes = 0;                                  // partial tiles stay in shared memory
+    *out = b;
+    return true;
+}
+
 // A layer on its own: worth splitting when the persistent kernel would leave most of the GPU idle AND walk a long K
 // per CTA.  Measured: from about 24 k-blocks on (16 when the layer has only one or two output tiles); below that
 // the hand-over between the slices costs more than the shorter loop saves (the 1x1 reducers stay where they were).
@@ -482,10 +543,46 @@ bool conv_splitk_supports(const ConvParams& p) {
 // the 1x1 reducer, job 1) and optionally `c` (the convolution that reads b's output, job 2).  b and c share a small
 // group of CTAs, a takes the rest.  Scratch: a's, then b's, then c's; counters: a's tiles, b's, c's, then the
 // counter on which c waits for b.
+static int group_smem_bytes(const SkPlan& pa, const SkPlan& pb, const SkPlan* pc) {
+    int smem = pa.stages * pa.sub_bytes;
+    const SkPlan* small[2] = {&pb, pc};
+    for (const SkPlan* q : small) {
+        if (!q) continue;
+        if (q->stages * q->sub_bytes > smem) smem = q->stages * q->sub_bytes;
+        if (q->cluster && q->nt * 512 > smem) smem = q->nt * 512;       // the partial tile of a cluster job lives where the stages were
+    }
+    return smem + 1024;
+}
+
+static int max_active_clusters(int cs, int smem_bytes);
+
 static bool splitk_group_plan(const ConvParams& a, const ConvParams& b, const ConvParams* c, SkPlan* pa, SkPlan* pb, SkPlan* pc) {
     if (tunable("DR_SPLITK_PAIR", 1) == 0) return false;
     if (a.x != b.x || a.B != b.B || a.H != b.H || a.W != b.W || a.Cin != b.Cin) return false;
     const int small = tunable("DR_SPLITK_SMALL_CTAS", 48);
+    // Cluster form for the two short jobs of a three-job launch (the chain reducer -> 3x3 is the critical path of a
+    // module at batch 1); the long job keeps the hand-over through L2.  Every CTA of the launch must be resident at once.
+    const int cs = tunable("DR_SPLITK_CLUSTER", 4);      // measured: 4 beats 8 (the device holds 33 clusters of 4, 15 of 8) and 2
+    if (cs > 1 && cs <= 8 && c && c->x == b.y && c->Cin == b.Cout && b.ldc == b.Cout && b.coff == 0 && !(b.flags & DR_OUT_F32)) {
+        SkPlan qb, qc, qa, alone;
+        if (splitk_plan_cluster(b, small, cs, &qb) && splitk_plan_cluster(*c, small, cs, &qc) && splitk_plan(a, &alone)) {
+            const int used_b = b.m_tiles * qb.n_blocks * cs, used_c = c->m_tiles * qc.n_blocks * cs;
+            const int used = used_b > used_c ? used_b : used_c;
+            // the device holds fewer CTAs in clusters than singly (a cluster sits inside one GPC): plan against that number
+            const int smem_cap = tunable("DR_SPLITK_SMEM_KB", 200) * 1024 + 1024;
+            int cap = max_active_clusters(cs, smem_cap) * cs;
+            if (cap > num_sms()) cap = num_sms();
+            const int budget_a = (cap - used) / cs * cs;
+            if (budget_a >= 2 * cs && splitk_plan_budget(a, budget_a, false, &qa)) {
+                const int ctas_a = (a.m_tiles * qa.n_blocks * qa.splits + cs - 1) / cs * cs;
+                const long long tiles = (long long)a.m_tiles * qa.n_blocks + (long long)b.m_tiles * qb.n_blocks + (long long)c->m_tiles * qc.n_blocks + 1;
+                if (tiles <= SK_MAX_TILES && group_smem_bytes(qa, qb, &qc) <= smem_cap && (ctas_a + used) <= cap) {
+                    *pa = qa; *pb = qb; *pc = qc;
+                    return true;
+                }
+            }
+        }
+    }
     if (!splitk_plan_budget(b, small, true, pb, tunable("DR_SPLITK_B_S", 0))) return false;
     int used = b.m_tiles * pb->n_blocks * pb->splits;
     long long tiles = (long long)b.m_tiles * pb->n_blocks;
@@ -523,6 +620,7 @@ static int fill_job(const ConvParams& p0, const SkPlan& pl, float* scratch, int*
     const int est = encode_conv_maps(j->p, pl.nt, &j->map_a, &j->map_b, &j->a_mode);
     if (est != DR_OK) return est;
     j->stages = pl.stages; j->sub_bytes = pl.sub_bytes; j->splits = pl.splits; j->kps = pl.kps; j->tmem_cols = pl.tmem_cols;
+    j->cluster = pl.cluster;
     j->scratch = scratch; j->counters = counters;
     j->ctas = p0.m_tiles * pl.n_blocks * pl.splits;
     return DR_OK;
@@ -538,9 +636,9 @@ static int launch_jobs(const SkJobs& jobs, int ctas, int smem_bytes, cudaStream_
     // prefetches its filters meanwhile; the grid never exceeds the SM count, and the kernel before it never waits on
     // this one, so every slice becomes resident.  DR_SPLITK_PDL=0: a cooperative launch (residency checked by the
     // runtime), no overlap.
-    const bool pdl = tunable("DR_SPLITK_PDL", 1) != 0;
+    const bool pdl = tunable("DR_SPLITK_PDL", 1) != 0 || jobs.cs > 1;
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     if (pdl) {
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -554,12 +652,43 @@ static int launch_jobs(const SkJobs& jobs, int ctas, int smem_bytes, cudaStream_
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (jobs.cs > 1) {                   // residency of every cluster was checked when the plan was made
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)jobs.cs; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
     if (cudaLaunchKernelEx(&cfg, conv_splitk_kernel, jobs) != cudaSuccess) {
         (void)cudaGetLastError();
         return DR_ERR_CUDA;
     }
     count_launch();
     return launch_status();
+}
+
+// How many clusters of `cs` CTAs with `smem_bytes` of dynamic shared memory the device holds at once (memoised).
+static int max_active_clusters(int cs, int smem_bytes) {
+    static std::mutex mu;
+    static std::map<std::pair<int, int>, int> memo;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    const std::pair<int, int> key(dev * 16 + cs, smem_bytes);
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = memo.find(key);
+    if (it != memo.end()) return it->second;
+    int n = 0;
+    if (cudaFuncSetAttribute(conv_splitk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_SMEM_MAX) == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.gridDim = dim3((unsigned)(num_sms() / cs * cs));
+        cfg.blockDim = dim3(SK_THREADS);
+        cfg.dynamicSmemBytes = (size_t)smem_bytes;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&n, conv_splitk_kernel, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+    }
+    memo[key] = n;
+    return n;
 }
 
 int conv_splitk_launch(const ConvParams& p, cudaStream_t stream) {
@@ -584,22 +713,21 @@ int conv_splitk_group_launch(const ConvParams& a, const ConvParams& b, const Con
     int* counters = a.sk_counters + a.m_tiles * pa.n_blocks;
     st = fill_job(b, pb, reinterpret_cast<float*>(scratch), counters, &jobs.j[1]);
     if (st != DR_OK) return st;
-    int smem = pa.stages * pa.sub_bytes;
-    if (pb.stages * pb.sub_bytes > smem) smem = pb.stages * pb.sub_bytes;
+    const int cs = (c && pb.cluster && pc.cluster) ? pb.splits : 1;
     int small = jobs.j[1].ctas;
     jobs.n = 2;
+    jobs.cs = cs;
     if (c) {
         scratch += pb.scratch_bytes;
         counters += b.m_tiles * pb.n_blocks;
         st = fill_job(*c, pc, reinterpret_cast<float*>(scratch), counters, &jobs.j[2]);
         if (st != DR_OK) return st;
         jobs.dep = counters + c->m_tiles * pc.n_blocks;
-        if (pc.stages * pc.sub_bytes > smem) smem = pc.stages * pc.sub_bytes;
         if (jobs.j[2].ctas > small) small = jobs.j[2].ctas;
         jobs.n = 3;
     }
-    jobs.small_begin = jobs.j[0].ctas;
-    return launch_jobs(jobs, jobs.j[0].ctas + small, smem + 1024, stream);
+    jobs.small_begin = (jobs.j[0].ctas + cs - 1) / cs * cs;              // the small group starts a cluster
+    return launch_jobs(jobs, jobs.small_begin + small, group_smem_bytes(pa, pb, c ? &pc : nullptr), stream);
 }
 
 }  // namespace dr

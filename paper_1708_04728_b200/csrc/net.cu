@@ -756,7 +756,11 @@ int dr_net_forward(dr_net* n, const void* x, void* workspace, float* logits, voi
                 break;
             }
             case OP_RELU: st = dr_relu((size_t)ti.B * ti.H * ti.W * ti.C, in0, out, stream); break;
-            case OP_MAXPOOL: st = dr_maxpool(ti.B, ti.H, ti.W, ti.C, 3, 2, op.pool_pad, in0, out, nullptr, stream); break;
+            case OP_MAXPOOL:
+                g_pool_pdl = i > 0 && !n->timing && tunable("DR_NET_PDL", 1) != 0;
+                st = dr_maxpool(ti.B, ti.H, ti.W, ti.C, 3, 2, op.pool_pad, in0, out, nullptr, stream);
+                g_pool_pdl = false;
+                break;
             case OP_LRN: st = dr_lrn(ti.B, ti.H, ti.W, ti.C, 5, 1e-4f, 0.75f, 1.f, in0, out, stream); break;
             case OP_BN:
                 st = dr_bn(ti.B, ti.H, ti.W, ti.C, in0, (const float*)op.v0.resolve(n->raw, ws), (const float*)op.v1.resolve(n->raw, ws),
@@ -767,7 +771,11 @@ int dr_net_forward(dr_net* n, const void* x, void* workspace, float* logits, voi
                 break;
             case OP_ADD: st = dr_add((size_t)ti.B * ti.H * ti.W * ti.C, in0, in1, out, stream); break;
             case OP_CONCAT: st = dr_concat((size_t)ti.B * ti.H * ti.W, ti.C, in0, to.C, op.coff, out, stream); break;
-            case OP_AVGPOOL: st = dr_avgpool_global(ti.B, ti.H, ti.W, ti.C, in0, out, stream); break;
+            case OP_AVGPOOL:
+                g_pool_pdl = i > 0 && !n->timing && tunable("DR_NET_PDL", 1) != 0;
+                st = dr_avgpool_global(ti.B, ti.H, ti.W, ti.C, in0, out, stream);
+                g_pool_pdl = false;
+                break;
             case OP_S2D: st = dr_space_to_depth(ti.B, ti.H, ti.W, ti.C, op.s2d_k, op.s2d_s, op.s2d_pad, to.C, in0, out, stream); break;
         }
         if (st != DR_OK) return st;

@@ -287,12 +287,27 @@ __global__ void maxpool3_noarg_kernel(int B, int H, int W, int C8, int Ho, int W
         y[i] = m;
     }
 }
+thread_local bool g_pool_pdl = false;
+// An ordinary launch, or one with programmatic stream serialization when the network executor asks for it (the
+// kernels that take this path execute griddepcontrol.wait before their first load).
+template <class... KArgs, class... Args>
+static void launch_maybe_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+    cfg.attrs = attr; cfg.numAttrs = g_pool_pdl ? 1 : 0;
+    (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // 3x3 / stride 2: a thread takes a 2 x 2 block of pooled positions (8 channels), whose windows cover 5 x 5 inputs:
 // 25 loads for four outputs instead of 36, all issued before the first maximum.  Taps outside the plane load a clamped,
 // valid address and are replaced by -inf.
 __global__ void __launch_bounds__(256) maxpool3s2_quad_kernel(int B, int H, int W, int C8, int Ho, int Wo, int p, const uint4* __restrict__ x,
                                                               uint4* __restrict__ y) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see maxpool_kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");                // no-op unless launched with programmatic serialization
     const unsigned Ho2 = (unsigned)(Ho + 1) >> 1, Wo2 = (unsigned)(Wo + 1) >> 1;
     const unsigned total = (unsigned)B * Ho2 * Wo2 * (unsigned)C8;     // the host keeps this below 2^32
     const unsigned stride = gridDim.x * blockDim.x;
@@ -469,6 +484,7 @@ __global__ void concat_scalar_kernel(size_t n, int C, int ldc, int coff, const _
 __global__ void __launch_bounds__(256) avgpool8_kernel(int HW, int C8, const uint4* __restrict__ x, uint4* __restrict__ y) {
     __shared__ float part[32][8][9];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see maxpool_kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");                // no-op unless launched with programmatic serialization
     const int n = blockIdx.y, c8 = blockIdx.x * 8 + threadIdx.x, py = threadIdx.y;
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     if (c8 < C8) {
@@ -761,7 +777,8 @@ int dr_maxpool(int B, int H, int W, int C, int k, int s, int p, const void* x, v
     if (n == 0) return DR_OK;
     DR_REQUIRE(aligned16(x) && aligned16(y) && (!argmax || aligned16(argmax)), DR_ERR_ALIGNMENT);
     if (C % 8 == 0 && !argmax && k == 3 && s == 2 && (size_t)B * ((Ho + 1) / 2) * ((Wo + 1) / 2) * (C / 8) < 0xffffffffull)
-        maxpool3s2_quad_kernel<<<grid_for((size_t)B * ((Ho + 1) / 2) * ((Wo + 1) / 2) * (C / 8), 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C / 8, Ho, Wo, p, (const uint4*)x, (uint4*)y);
+        launch_maybe_pdl(maxpool3s2_quad_kernel, dim3(grid_for((size_t)B * ((Ho + 1) / 2) * ((Wo + 1) / 2) * (C / 8), 256)), dim3(256), (cudaStream_t)stream, B, H, W, C / 8, Ho, Wo,
+                         p, (const uint4*)x, (uint4*)y);
     else if (C % 8 == 0 && !argmax && k == 3)
         maxpool3_noarg_kernel<<<grid_for(n / 8, 256), 256, 0, (cudaStream_t)stream>>>(B, H, W, C / 8, Ho, Wo, s, p, (const uint4*)x, (uint4*)y);
     else if (C % 8 == 0 && !argmax)
@@ -816,7 +833,7 @@ int dr_avgpool_global(int B, int H, int W, int C, const void* x, void* y, void* 
     DR_REQUIRE(C % 2 == 0, DR_ERR_UNSUPPORTED);
     if (C % 8 == 0) {
         dim3 grid((C / 8 + 7) / 8, B), block(8, 32);
-        avgpool8_kernel<<<grid, block, 0, (cudaStream_t)stream>>>(H * W, C / 8, (const uint4*)x, (uint4*)y);
+        launch_maybe_pdl(avgpool8_kernel, grid, block, (cudaStream_t)stream, H * W, C / 8, (const uint4*)x, (uint4*)y);
         count_launch();
         return launch_status();
     }
