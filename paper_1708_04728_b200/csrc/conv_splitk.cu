@@ -47,6 +47,7 @@ struct SkShared {
 struct SkPlan {
     int nt, n_blocks, splits, kps, nkb, stages, sub_bytes;
     int cluster;              // slices of a tile = ranks of a cluster of `splits` CTAs
+    int own_ctas;             // (job 2 of a group) runs on CTAs of its own rather than behind job 1
     uint32_t tmem_cols;
     size_t scratch_bytes;
 };
@@ -76,6 +77,7 @@ struct SkJobs {
     int n;                    // 1, 2 or 3 jobs
     int cs;                   // cluster size of the launch (1: no clusters)
     int small_begin;          // first CTA of the small group (n >= 2)
+    int c_begin;              // n == 3: first CTA of job 2; == small_begin when jobs 1 and 2 share their CTAs, beyond job 1's otherwise
     int* dep;                 // n == 3: counter on which job 2 waits for job 1
 };
 
@@ -362,9 +364,12 @@ __global__ void __launch_bounds__(SK_THREADS, 1) conv_splitk_kernel(const __grid
     __shared__ SkShared sh;
     const int tid = threadIdx.x, warp = tid >> 5;
     const bool small = jobs.n >= 2 && (int)blockIdx.x >= jobs.small_begin;
-    const int bid = small ? (int)blockIdx.x - jobs.small_begin : (int)blockIdx.x;
-    const int j0 = small ? 1 : 0;                               // first job of this CTA
-    const int j1 = small && jobs.n == 3 ? 2 : j0;               // last job of this CTA
+    // job 2 on CTAs of its own (they request their filters at once and wait for job 1 with nothing else to do), or behind
+    // job 1 on the same CTAs
+    const bool own_c = jobs.n == 3 && jobs.c_begin > jobs.small_begin && (int)blockIdx.x >= jobs.c_begin;
+    const int bid = own_c ? (int)blockIdx.x - jobs.c_begin : small ? (int)blockIdx.x - jobs.small_begin : (int)blockIdx.x;
+    const int j0 = own_c ? 2 : small ? 1 : 0;                   // first job of this CTA
+    const int j1 = (small && jobs.n == 3 && jobs.c_begin == jobs.small_begin) ? 2 : j0;   // last job of this CTA
     uint32_t tmem_cols = 32;
     for (int j = j0; j <= j1; ++j) tmem_cols = max(tmem_cols, jobs.j[j].tmem_cols);
 
@@ -411,7 +416,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) conv_splitk_kernel(const __grid
         if (has_work) {
             if (j == 0) sk_run_job(&jobs.j[0], bid, sh, smem, tmem, true, nullptr, -1, false, 0u);
             else if (j == 1) sk_run_job(&jobs.j[1], bid, sh, smem, tmem, true, jobs.dep, -1, jobs.n == 3, dep_wrap);
-            else sk_run_job(&jobs.j[2], bid, sh, smem, tmem, false, jobs.dep, jobs.j[1].ctas, false, dep_wrap);
+            else sk_run_job(&jobs.j[2], bid, sh, smem, tmem, j == j0, jobs.dep, jobs.j[1].ctas, false, dep_wrap);
         } else if (j == j0 && warp == 0) {
             grid_dependency_wait();
         }
@@ -567,7 +572,11 @@ static bool splitk_group_plan(const ConvParams& a, const ConvParams& b, const Co
         SkPlan qb, qc, qa, alone;
         if (splitk_plan_cluster(b, small, cs, &qb) && splitk_plan_cluster(*c, small, cs, &qc) && splitk_plan(a, &alone)) {
             const int used_b = b.m_tiles * qb.n_blocks * cs, used_c = c->m_tiles * qc.n_blocks * cs;
-            const int used = used_b > used_c ? used_b : used_c;
+            // CTAs of its own for the 3x3 where the long job keeps at least half of the device: a CTA that ran the reducer
+            // first starts its 3x3 slice about 3 us after the others (barriers set up again, filters requested late)
+            const bool own = tunable("DR_SPLITK_OWN_CTAS", 1) != 0 && used_b + used_c <= num_sms() / 2;
+            const int used = own ? used_b + used_c : (used_b > used_c ? used_b : used_c);
+            qc.own_ctas = own ? 1 : 0;
             // the device holds fewer CTAs in clusters than singly (a cluster sits inside one GPC): plan against that number
             const int smem_cap = tunable("DR_SPLITK_SMEM_KB", 200) * 1024 + 1024;
             int cap = max_active_clusters(cs, smem_cap) * cs;
@@ -590,7 +599,8 @@ static bool splitk_group_plan(const ConvParams& a, const ConvParams& b, const Co
         if (c->x != b.y || c->Cin != b.Cout || b.ldc != b.Cout || b.coff != 0 || (b.flags & DR_OUT_F32)) return false;   // c reads b's dense output
         if (!splitk_plan_budget(*c, small, true, pc, tunable("DR_SPLITK_C_S", 0))) return false;
         const int used_c = c->m_tiles * pc->n_blocks * pc->splits;
-        if (used_c > used) used = used_c;
+        if (tunable("DR_SPLITK_OWN_CTAS", 1) != 0 && used + used_c <= num_sms() / 2) { used += used_c; pc->own_ctas = 1; }   // as in the cluster form
+        else if (used_c > used) used = used_c;
         tiles += (long long)c->m_tiles * pc->n_blocks + 1;
     }
     SkPlan alone;
@@ -727,6 +737,11 @@ int conv_splitk_group_launch(const ConvParams& a, const ConvParams& b, const Con
         jobs.n = 3;
     }
     jobs.small_begin = (jobs.j[0].ctas + cs - 1) / cs * cs;              // the small group starts a cluster
+    jobs.c_begin = jobs.small_begin;
+    if (c && pc.own_ctas) {
+        jobs.c_begin = jobs.small_begin + jobs.j[1].ctas;                // a multiple of the cluster size
+        small = jobs.j[1].ctas + jobs.j[2].ctas;
+    }
     return launch_jobs(jobs, jobs.small_begin + small, group_smem_bytes(pa, pb, c ? &pc : nullptr), stream);
 }
 
