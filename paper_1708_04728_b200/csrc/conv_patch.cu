@@ -307,6 +307,7 @@ conv_patch_pair_kernel(const ConvParams p, const __grid_constant__ CUtensorMap m
             uint32_t ph = 0;
             bool ok = true;
             uint32_t ready = mbar_test_u32(empty0, 1);
+            if (p.pdl_wait) grid_dependency_wait();                          // the kernel before this one has written the activations
             for (int u = unit; u < units && ok; u += nunits) {
                 int t = 2 * u + (int)rank;
                 if (t >= total) t = total - 1;                               // odd patch count: the peer repeats the last patch (same values stored twice)
@@ -704,9 +705,11 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
             const int forced_stages = tunable("DR_PATCH_STAGES", 0);
             if (forced_stages >= 2 && forced_stages < stages) stages = forced_stages;
             cudaLaunchConfig_t cfg = {};
-            cudaLaunchAttribute attr[1];
+            cudaLaunchAttribute attr[2];
             attr[0].id = cudaLaunchAttributeClusterDimension;
             attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // used when p.pdl_wait: the producer waits before its first activation load
+            attr[1].val.programmaticStreamSerializationAllowed = 1;
             // two warps per row for the drain where the LRN comes first (see the kernel's comment)
             const bool split = fe_split_supports(p) && tunable("DR_PATCH_SPLIT", 1) != 0;
             cfg.blockDim = dim3(split ? PP_THREADS_SPLIT : PP_THREADS); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
@@ -737,6 +740,7 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
             const int pairs = units < max_clusters ? units : max_clusters;
             cfg.gridDim = dim3(2 * pairs);
             cfg.dynamicSmemBytes = (size_t)smem_bytes;
+            cfg.numAttrs = p.pdl_wait ? 2 : 1;
             const cudaError_t le = split ? cudaLaunchKernelEx(&cfg, conv_patch_pair_kernel<true>, p, map_a, map_bh, stages, stage_bytes, groups, resident, bsub)
                                          : cudaLaunchKernelEx(&cfg, conv_patch_pair_kernel<false>, p, map_a, map_bh, stages, stage_bytes, groups, resident, bsub);
             if (le != cudaSuccess) return DR_ERR_CUDA;

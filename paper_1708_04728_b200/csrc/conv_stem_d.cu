@@ -187,6 +187,7 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
     // everything starts at zero: padding slots, the two spare elements of every slot, unused filter slots, LRN halos
     for (int i = tid; i < total_bytes / 16; i += SD_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
+    grid_launch_dependents();            // the layer behind this one may set up on free SMs (it waits for this kernel before it reads)
     // filters.  K = block*32 + j*8 + e: slot j of the window, element e = pixel-in-pair*3 + channel; tap s = 2j + pixel - 1
     for (int i = tid; i < 64 * 147; i += SD_THREADS) {
         const int c = i / 147, e0 = i - c * 147;

@@ -750,7 +750,7 @@ int dr_net_forward(dr_net* n, const void* x, void* workspace, float* logits, voi
                 if (st == DR_OK) {
                     set_splitk_scratch(n, op, (char*)workspace, &p);
                     // a layer of its own on the TMA kernel: its CTAs may set up while the kernel before it drains
-                    if (op.path == DR_PATH_UMMA_TMA && i > 0 && !n->timing && tunable("DR_NET_PDL", 1) != 0) p.pdl_wait = 1;
+                    if ((op.path == DR_PATH_UMMA_TMA || op.path == DR_PATH_UMMA_PATCH) && i > 0 && !n->timing && tunable("DR_NET_PDL", 1) != 0) p.pdl_wait = 1;
                     st = conv_launch_path(p, op.path, s);
                 }
                 break;
