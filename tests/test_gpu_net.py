@@ -210,3 +210,21 @@ def test_net_timing_and_launch_count(dr):
     net.dr_net_forward(x, ws, logits)
     assert dr.dr_tensor_map_encodes() == e0
     assert np.array_equal(untimed, to_host(logits))
+
+
+@pytest.mark.parametrize("env", [{"DR_SPLITK_CLUSTER": "1"}, {"DR_SPLITK_CLUSTER": "1", "DR_SPLITK_OWN_CTAS": "0"}, {"DR_SPLITK_CLUSTER": "8"},
+                                 {"DR_NET_PDL": "0"}])
+def test_single_image_forward_in_the_other_hand_over_forms(env):
+    """The split-K launch of an inception module has several forms chosen per process (hand-over through L2 or through a
+    cluster's shared memory, the 3x3 on CTAs of its own or behind the reducer, programmatic launches or ordinary ones): the
+    single-image network passes its parity test in each of them."""
+    import os
+    import subprocess
+    import sys
+    e = dict(os.environ)
+    e.update(env)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_net.py"), "-q", "-x", "-m", "gpu", "-k", "test_googlenet_slim and 1-1",
+                        "-p", "no:cacheprovider"], cwd=root, env=e, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    assert "1 passed" in r.stdout, r.stdout[-2000:]
