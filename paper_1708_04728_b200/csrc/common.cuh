@@ -19,6 +19,15 @@ inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_
 int* dev_status_ptr();   // device address of the record on the current device (host call)
 int num_sms();
 
+// A "done once" flag kept per device: function attributes (opt-in shared memory sizes) and occupancy figures belong
+// to the device that was current when they were set or queried.
+struct PerDeviceFlag {
+    std::atomic<unsigned long long> bits{0};
+    static int dev() { int d = 0; (void)cudaGetDevice(&d); return d & 63; }
+    bool get() const { return (bits.load(std::memory_order_acquire) >> dev()) & 1ull; }
+    void set() { bits.fetch_or(1ull << dev(), std::memory_order_release); }
+};
+
 __device__ __forceinline__ void report_timeout(int* status, int site, int tile) {
     if (atomicCAS(&status[0], 0, DR_ERR_DEVICE_TIMEOUT) == 0) {
         status[1] = site;

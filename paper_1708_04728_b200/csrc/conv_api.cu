@@ -5,8 +5,8 @@
 
 namespace dr {
 
-static int g_forced_path = DR_PATH_AUTO;
-static int g_last_path = -1;
+static std::atomic<int> g_forced_path{DR_PATH_AUTO};    // test hooks: process-wide, read and written atomically
+static std::atomic<int> g_last_path{-1};
 
 // Fill the derived fields of ConvParams from a descriptor.  Returns a status.
 int conv_make_params(const dr_conv_desc* d, int B, int H, int W, const void* x, const void* w, const float* b,

@@ -661,10 +661,10 @@ bool conv_patch_tma_supports(const ConvParams& p) {
 
 int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
     if (!conv_patch_tma_supports(p)) return DR_ERR_UNSUPPORTED;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceFlag attr_set;
+    if (!attr_set.get()) {
         if (cudaFuncSetAttribute(conv_patch_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
-        attr_set = true;
+        attr_set.set();
     }
     alignas(64) CUtensorMap map_a, map_b;
     {
@@ -683,8 +683,9 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
     // CTA pairs with each CTA's half of the filter bank resident in shared memory (or, if that does not fit, streamed):
     // the filters are what this layer moves most of otherwise.  Measured on GoogLeNet conv2 at batch 256.
     if (tunable("DR_PATCH_PAIR", 1) != 0 && p.m_tiles >= 2 && (p.Nt & 31) == 0) {
-        static bool pair_attr = false;
-        static int max_clusters = 0;
+        static PerDeviceFlag pair_attr;
+        static int max_clusters_dev[64] = {};
+        int& max_clusters = max_clusters_dev[PerDeviceFlag::dev()];
         const int nkb = p.k * p.k * ((p.Cin + 63) / 64);
         const int bsub = ((p.Nt / 2) * 128 + 1023) & ~1023;
         const int budget = P_SMEM_MAX - 2048;
@@ -713,7 +714,7 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
             // two warps per row for the drain where the LRN comes first (see the kernel's comment)
             const bool split = fe_split_supports(p) && tunable("DR_PATCH_SPLIT", 1) != 0;
             cfg.blockDim = dim3(split ? PP_THREADS_SPLIT : PP_THREADS); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
-            if (!pair_attr) {
+            if (!pair_attr.get()) {
                 if (cudaFuncSetAttribute(conv_patch_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
                 if (cudaFuncSetAttribute(conv_patch_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
                 int mc[2] = {0, 0};
@@ -727,7 +728,7 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
                     if (e != cudaSuccess || mc[v] < 1) return DR_ERR_CUDA;
                 }
                 max_clusters = mc[0] < mc[1] ? mc[0] : mc[1];
-                pair_attr = true;
+                pair_attr.set();
             }
             alignas(64) CUtensorMap map_bh;
             const cuuint64_t dims[3] = {(cuuint64_t)p.Cin, (cuuint64_t)(p.k * p.k), (cuuint64_t)p.Cout};
@@ -781,10 +782,10 @@ bool conv_stem_supports(const ConvParams& p) {
 
 int conv_stem_launch(const ConvParams& p, cudaStream_t stream) {
     if (!conv_stem_supports(p)) return DR_ERR_UNSUPPORTED;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceFlag attr_set;
+    if (!attr_set.get()) {
         if (cudaFuncSetAttribute(conv_stem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
-        attr_set = true;
+        attr_set.set();
     }
     if (p.m_tiles <= 0) return DR_OK;
     int rows, words;

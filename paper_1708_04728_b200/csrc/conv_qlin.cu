@@ -576,8 +576,9 @@ int conv_qlin_launch(const ConvParams& p_in, cudaStream_t stream) {
     ConvParams p = p_in;
     p.Nt = conv_qlin_nt(p);
     p.n_blocks = 1;
-    static bool attr_set = false;
-    static int max_clusters = 0;
+    static PerDeviceFlag attr_set;
+    static int max_clusters_dev[64] = {};
+        int& max_clusters = max_clusters_dev[PerDeviceFlag::dev()];
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -585,7 +586,7 @@ int conv_qlin_launch(const ConvParams& p_in, cudaStream_t stream) {
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(Q_THREADS); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
-    if (!attr_set) {
+    if (!attr_set.get()) {
         if (cudaFuncSetAttribute(conv_qlin_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Q_SMEM_MAX) != cudaSuccess ||
             cudaFuncSetAttribute(conv_qlin2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Q_SMEM_MAX) != cudaSuccess ||
             cudaFuncSetAttribute(conv_qlin_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Q_SMEM_MAX) != cudaSuccess)
@@ -593,7 +594,7 @@ int conv_qlin_launch(const ConvParams& p_in, cudaStream_t stream) {
         cfg.gridDim = dim3(2 * num_sms());
         cfg.dynamicSmemBytes = (size_t)Q_SMEM_MAX;
         if (cudaOccupancyMaxActiveClusters(&max_clusters, conv_qlin_kernel<false>, &cfg) != cudaSuccess || max_clusters < 1) return DR_ERR_CUDA;
-        attr_set = true;
+        attr_set.set();
     }
     alignas(64) CUtensorMap map_a, map_b;
     {

@@ -119,11 +119,11 @@ int conv_simt_launch(const ConvParams& p, cudaStream_t stream) {
     size_t smem = sizeof(float) * (SIMT_BK * (TILE_M + 4) + SIMT_BK * (SIMT_BN + 4));
     if (staged) smem += sizeof(float) * ((size_t)TILE_M * (p.Cout + 1) + (pool_then_lrn ? (size_t)p.PH * p.PW * (p.Cout + 1) : 0));
     if (smem > 227 * 1024) return DR_ERR_UNSUPPORTED;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceFlag attr_set;
+    if (!attr_set.get()) {
         if (cudaFuncSetAttribute(conv_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
             return DR_ERR_CUDA;
-        attr_set = true;
+        attr_set.set();
     }
     if (p.m_tiles <= 0) return DR_OK;
     dim3 grid(p.m_tiles, staged ? 1 : p.n_blocks);

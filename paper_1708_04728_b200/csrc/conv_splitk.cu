@@ -637,10 +637,10 @@ static int fill_job(const ConvParams& p0, const SkPlan& pl, float* scratch, int*
 }
 
 static int launch_jobs(const SkJobs& jobs, int ctas, int smem_bytes, cudaStream_t stream) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceFlag attr_set;
+    if (!attr_set.get()) {
         if (cudaFuncSetAttribute(conv_splitk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
-        attr_set = true;
+        attr_set.set();
     }
     // Launch mode.  Programmatic (default): the kernel may start while the previous kernel of the stream drains, and
     // prefetches its filters meanwhile; the grid never exceeds the SM count, and the kernel before it never waits on

@@ -496,11 +496,11 @@ bool conv_stem_d_supports(const ConvParams& p) {
 
 int conv_stem_d_launch(const ConvParams& p, cudaStream_t stream) {
     if (!conv_stem_d_supports(p)) return DR_ERR_UNSUPPORTED;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceFlag attr_set;
+    if (!attr_set.get()) {
         if (cudaFuncSetAttribute(conv_stem_d_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SD_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
         if (cudaFuncSetAttribute(conv_stem_d_kernel<112>, cudaFuncAttributeMaxDynamicSharedMemorySize, SD_SMEM_MAX) != cudaSuccess) return DR_ERR_CUDA;
-        attr_set = true;
+        attr_set.set();
     }
     const SdGeom g = sd_geom(p);
     if (g.total <= 0) return DR_OK;

@@ -438,10 +438,10 @@ bool conv_umma_gather_supports(const ConvParams& p) {
 
 int conv_umma_gather_launch(const ConvParams& p, cudaStream_t stream) {
     if (!conv_umma_gather_supports(p)) return DR_ERR_UNSUPPORTED;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceFlag attr_set;
+    if (!attr_set.get()) {
         if (cudaFuncSetAttribute(conv_umma_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM) != cudaSuccess) return DR_ERR_CUDA;
-        attr_set = true;
+        attr_set.set();
     }
     if (p.m_tiles <= 0) return DR_OK;
     dim3 grid(p.m_tiles, p.n_blocks);

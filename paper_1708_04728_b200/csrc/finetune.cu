@@ -521,8 +521,8 @@ extern "C" int dr_conv_wgrad(const dr_conv_desc* desc, int B, int H, int W, cons
     int est = encode_input_map(cp, &map_x, &a_mode, p.pix);
     if (est == DR_OK) est = encode_rows_map(dz, p.M, p.Cout, p.Cout, &map_dz, p.pix);
     if (est != DR_OK) return est;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceFlag attr_set;
+    if (!attr_set.get()) {
         if (cudaFuncSetAttribute(conv_wgrad_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_MAX + 1024) != cudaSuccess ||
             cudaFuncSetAttribute(conv_wgrad_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_MAX + 1024) != cudaSuccess ||
             cudaFuncSetAttribute(conv_wgrad_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_MAX + 1024) != cudaSuccess ||
@@ -530,7 +530,7 @@ extern "C" int dr_conv_wgrad(const dr_conv_desc* desc, int B, int H, int W, cons
             (void)cudaGetLastError();
             return DR_ERR_CUDA;
         }
-        attr_set = true;
+        attr_set.set();
     }
     {
         cudaLaunchConfig_t cfg = {};

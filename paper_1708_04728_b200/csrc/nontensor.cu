@@ -23,15 +23,17 @@ int* dev_status_ptr() {
     return ptr[dev];
 }
 
-static int g_num_sms = 0;
+static std::atomic<int> g_num_sms[64];
 int num_sms() {
-    if (!g_num_sms) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
-        if (g_num_sms <= 0) g_num_sms = 148;
+    int dev = 0;
+    (void)cudaGetDevice(&dev);
+    std::atomic<int>& slot = g_num_sms[dev & 63];
+    int n = slot.load(std::memory_order_relaxed);
+    if (!n) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) { (void)cudaGetLastError(); n = 148; }
+        slot.store(n, std::memory_order_relaxed);
     }
-    return g_num_sms;
+    return n;
 }
 
 static inline int grid_for(size_t work_items, int threads) {
