@@ -694,9 +694,11 @@ int conv_patch_tma_launch(const ConvParams& p, cudaStream_t stream) {
         const int res_pref = tunable("DR_PATCH_RESIDENT", -1);
         // two epilogue groups first (the fused LRN / pooling epilogue is what bounds these layers: conv2 takes 336 us with
         // two groups and streamed half-filters, 433 us with one group and resident filters), then resident filters
+        const int g_pref = tunable("DR_PATCH_PAIR_GROUPS", 0);
         for (int g = 2; g >= 1 && !groups; --g)
             for (int res = 1; res >= 0 && !groups; --res) {
                 if (res_pref >= 0 && res != res_pref) continue;
+                if (g_pref > 0 && g != g_pref) continue;
                 const int sb = P_A_BYTES + (res ? 0 : bsub);
                 const int left = budget - g * fe - (res ? nkb * bsub : 0);
                 if (left / sb >= 3) { groups = g; resident = res; stage_bytes = sb; stages = left / sb; }
