@@ -256,11 +256,17 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
         // ------------------------------------------------------------- MMA issue of stream g
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(SD_REGS_AUX));
         const int g = warp - 16;
-        if (lane == 0) {
+        {
+            // The whole warp walks the loop (every value below is warp-uniform) and lane 0 alone issues the MMAs and the
+            // commits: a lone lane inside a divergent branch issues one MMA per 120-210 cycles, a converged warp with a
+            // predicated MMA one per 64, which is what the 18 MMAs of a tile need.
+            const uint32_t el = lane == 0 ? 1u : 0u;
             SdSegments seg(gm.total, streams, 2 * blockIdx.x + g, gm.NP);
             const uint32_t ring = smem_u32(ring0 + g * ring_bytes);
             const uint32_t wt = smem_u32(Wt);
             const uint32_t idesc = make_idesc_bf16(128, 128);
+            const uint64_t a0 = sd_desc(wt, 2048u, 128u);                  // filters: K chunk (2r + h) is 4096 bytes = 256 descriptor units further
+            const uint64_t bhi = sd_desc(0u, 16u, 128u);                   // image row: everything but the start address
             long long Qb = 0, qready = 0;
             uint32_t tcount = 0;
             bool dead = false;
@@ -270,13 +276,13 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
                 for (int t = 0; t < T; ++t, ++tcount) {
                     bool ok = true;
                     while (ok && qready <= Qb + t + 2) {
-                        ok = mbar_wait(&sh.qfull[g][(int)(qready % SD_NQ)], (uint32_t)(qready / SD_NQ) & 1, abort_flag);
+                        ok = __all_sync(0xffffffffu, mbar_wait(&sh.qfull[g][(int)(qready % SD_NQ)], (uint32_t)(qready / SD_NQ) & 1, abort_flag));
                         ++qready;
                     }
                     const uint32_t buf = tcount & 1;
-                    ok = ok && mbar_wait(&sh.tempty[g][buf], ((tcount >> 1) & 1) ^ 1, abort_flag);
+                    ok = ok && __all_sync(0xffffffffu, mbar_wait(&sh.tempty[g][buf], ((tcount >> 1) & 1) ^ 1, abort_flag));
                     if (!ok) {
-                        if (!*abort_flag) report_timeout(p.status, 62, (int)tcount);
+                        if (el && !*abort_flag) report_timeout(p.status, 62, (int)tcount);
                         *abort_flag = 1;
                         dead = true;
                         break;
@@ -290,19 +296,22 @@ __global__ void __launch_bounds__(SD_THREADS, 1) conv_stem_d_kernel(const ConvPa
                         int R = row0 + r;
                         if (R >= SD_NR) R -= SD_NR;
                         const uint32_t brow = ring + (uint32_t)R * gm.pitch;
+                        const uint64_t b0 = bhi | (uint64_t)((brow & 0x3FFFFu) >> 4);
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            umma_bf16(d, sd_desc(wt + (uint32_t)(2 * r + h) * 4096u, 2048u, 128u), sd_desc(brow + 32u * h, 16u, 128u), idesc,
-                                      (r | h) != 0);
-                        }
+                        for (int h = 0; h < 2; ++h)
+                            umma_bf16_pred(d, a0 + (uint64_t)((2 * r + h) * 256), b0 + (uint64_t)(2 * h), idesc, (r | h) != 0, el);
                     }
-                    umma_commit(&sh.tfull[g][buf]);
-                    umma_commit(&sh.qempty[g][(int)((Qb + t) % SD_NQ)]);
+                    if (el) {
+                        umma_commit(&sh.tfull[g][buf]);
+                        umma_commit(&sh.qempty[g][(int)((Qb + t) % SD_NQ)]);
+                    }
+                    __syncwarp();
                 }
-                if (!dead) {
+                if (!dead && el) {
                     umma_commit(&sh.qempty[g][(int)((Qb + T) % SD_NQ)]);
                     umma_commit(&sh.qempty[g][(int)((Qb + T + 1) % SD_NQ)]);
                 }
+                __syncwarp();
                 Qb += T + 2;
             }
         }
